@@ -1,0 +1,729 @@
+/*
+ * CPU oracle of the HAPMoE planner hot path -- TEST INFRASTRUCTURE, not a product path.
+ * See hap_oracle.h.  Plain loops, fp64 for the cost formulas (one IEEE operation per
+ * operator, no contraction: build with -ffp-contract=off), exact int64 afterwards.
+ */
+#include "hap_oracle.h"
+#include <math.h>
+#include <string.h>
+#include <stdlib.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef unsigned __int128 u128;
+
+/* ------------------------------------------------------------------------------------ *
+ * Cluster helpers: device counts per type and the slowest uplink of a type.
+ * ------------------------------------------------------------------------------------ */
+static void type_counts(const orc_problem *pr, int64_t *m)
+{
+    for (int h = 0; h < pr->T; ++h) m[h] = 0;
+    for (int n = 0; n < pr->n_nodes; ++n) m[pr->node_type[n]] += pr->node_size[pr->node_type[n]];
+}
+
+static double type_bw_inter(const orc_problem *pr, int h)
+{
+    double best = 0.0;
+    int seen = 0;
+    for (int n = 0; n < pr->n_nodes; ++n)
+        if (pr->node_type[n] == h) {
+            if (!seen || pr->node_bw_inter[n] < best) best = pr->node_bw_inter[n];
+            seen = 1;
+        }
+    return best;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Multiset permutations in lexicographic order (types ascending).
+ * ------------------------------------------------------------------------------------ */
+static uint64_t sat_mul_div(uint64_t r, uint64_t mul, uint64_t div, uint64_t sat)
+{
+    if (r >= sat) return sat;
+    u128 v = (u128)r * mul / div;   /* exact: callers keep r*mul divisible by div */
+    return v >= sat ? sat : (uint64_t)v;
+}
+
+/* number of distinct sequences with cnt[h] copies of type h, saturated at `sat`:
+ * the product over types of C(placed + cnt[h], cnt[h]), each binomial built one factor at a time */
+uint64_t orc_multiset_count(const int32_t *cnt, int T, uint64_t sat)
+{
+    uint64_t r = 1;
+    int placed = 0;
+    for (int h = 0; h < T; ++h) {
+        for (int i = 1; i <= cnt[h]; ++i)
+            r = sat_mul_div(r, (uint64_t)(placed + i), (uint64_t)i, sat);   /* C(placed+i, i) from C(placed+i-1, i-1) */
+        placed += cnt[h];
+    }
+    return r;
+}
+
+int orc_unrank_multiset(const int32_t *cnt_in, int T, int PP, uint64_t idx, uint8_t *seq)
+{
+    int32_t cnt[ORC_MAX_TYPES];
+    for (int h = 0; h < T; ++h) cnt[h] = cnt_in[h];
+    for (int pos = 0; pos < PP; ++pos) {
+        int chosen = -1;
+        for (int h = 0; h < T && chosen < 0; ++h) {
+            if (cnt[h] == 0) continue;
+            cnt[h]--;
+            uint64_t below = orc_multiset_count(cnt, T, UINT64_MAX);
+            if (idx < below) chosen = h;
+            else { idx -= below; cnt[h]++; }
+        }
+        if (chosen < 0) return -1;
+        seq[pos] = (uint8_t)chosen;
+    }
+    return 0;
+}
+
+uint64_t orc_rank_multiset(const int32_t *cnt_in, int T, int PP, const uint8_t *seq)
+{
+    int32_t cnt[ORC_MAX_TYPES];
+    uint64_t rank = 0;
+    for (int h = 0; h < T; ++h) cnt[h] = cnt_in[h];
+    for (int pos = 0; pos < PP; ++pos) {
+        for (int h = 0; h < seq[pos]; ++h) {
+            if (cnt[h] == 0) continue;
+            cnt[h]--;
+            rank += orc_multiset_count(cnt, T, UINT64_MAX);
+            cnt[h]++;
+        }
+        cnt[seq[pos]]--;
+    }
+    return rank;
+}
+
+static uint64_t factorial_u64(int n)
+{
+    uint64_t r = 1;
+    for (int i = 2; i <= n; ++i) r *= (uint64_t)i;
+    return r;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Enumeration of the 6-D parallel space x micro-batch (order defines candidate indices).
+ * ------------------------------------------------------------------------------------ */
+int orc_enumerate(const orc_problem *pr, orc_pconf *out, uint64_t cap, uint64_t *n_pconf, uint64_t *n_cand)
+{
+    int64_t m[ORC_MAX_TYPES];
+    type_counts(pr, m);
+    int64_t W = 0;
+    for (int h = 0; h < pr->T; ++h) W += m[h];
+    uint64_t np = 0, off = 0;
+    for (int ipp = 0; ipp < pr->npp; ++ipp) {
+        int PP = pr->pp_list[ipp];
+        if (PP > pr->N || PP > ORC_MAX_PP || W % PP != 0) continue;
+        int64_t G = W / PP;
+        /* mapping mode and count depend on (PP) only */
+        int homog = 1;
+        int32_t cnt[ORC_MAX_TYPES];
+        for (int h = 0; h < pr->T; ++h) {
+            if (m[h] % G != 0) homog = 0;
+            cnt[h] = (int32_t)(m[h] / G);
+        }
+        uint64_t nms = homog ? orc_multiset_count(cnt, pr->T, UINT64_MAX) : 0;
+        int mode = (homog && nms <= pr->map_cap) ? ORC_MODE_MULTISET : ORC_MODE_BLOCK;
+        uint64_t nmap = mode == ORC_MODE_MULTISET ? nms : factorial_u64(pr->T);
+        for (int itp = 0; itp < pr->ntp; ++itp) {
+            int TP = pr->tp_list[itp];
+            if (G % TP != 0 || TP > pr->tp_max || pr->nq % TP != 0 || pr->nkv % TP != 0) continue;
+            for (int icp = 0; icp < pr->ncp; ++icp) {
+                int CP = pr->cp_list[icp];
+                if (G % ((int64_t)TP * CP) != 0 || pr->S % (2 * CP) != 0) continue;
+                int64_t DP = G / ((int64_t)TP * CP);
+                for (int iep = 0; iep < pr->nep; ++iep) {
+                    int EP = pr->ep_list[iep];
+                    if (pr->E % EP != 0 || G % EP != 0) continue;
+                    for (int itpe = 0; itpe < pr->ntpe; ++itpe) {
+                        int TPE = pr->tpe_list[itpe];
+                        if (G % ((int64_t)EP * TPE) != 0 || TPE > pr->tp_max) continue;
+                        int64_t EDP = G / ((int64_t)EP * TPE);
+                        for (int ib = 0; ib < pr->nmb; ++ib) {
+                            int b = pr->mb_list[ib];
+                            if (pr->GB % (DP * b) != 0) continue;
+                            int64_t M = pr->GB / (DP * b);
+                            if (out) {
+                                if (np >= cap) return -2;
+                                orc_pconf *q = &out[np];
+                                q->PP = PP; q->TP = TP; q->CP = CP; q->DP = (int32_t)DP; q->EP = EP;
+                                q->TPE = TPE; q->b = b; q->M = (int32_t)M; q->EDP = (int32_t)EDP;
+                                q->G = (int32_t)G; q->itp = itp; q->icp = icp; q->ib = ib; q->iep = iep;
+                                q->mode = mode; q->pad = 0; q->nmap = nmap; q->offset = off;
+                            }
+                            off += nmap * (uint64_t)pr->n_rc;
+                            np++;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    *n_pconf = np;
+    *n_cand = off;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Mapping of device groups to stages.
+ * ------------------------------------------------------------------------------------ */
+int orc_decode(const orc_problem *pr, const orc_pconf *pc, uint64_t map_idx, orc_mapping *out)
+{
+    int64_t m[ORC_MAX_TYPES];
+    type_counts(pr, m);
+    const int PP = pc->PP, T = pr->T;
+    const int64_t G = pc->G;
+    if (map_idx >= pc->nmap) return -1;
+    memset(out, 0, sizeof(*out));
+    out->PP = PP;
+    /* per stage: type and position (within that type's device line) of first and last device */
+    int tfirst[ORC_MAX_PP], tlast[ORC_MAX_PP];
+    int64_t ofirst[ORC_MAX_PP], olast[ORC_MAX_PP];
+    if (pc->mode == ORC_MODE_MULTISET) {
+        int32_t cnt[ORC_MAX_TYPES];
+        uint8_t seq[ORC_MAX_PP];
+        int used[ORC_MAX_TYPES] = {0, 0, 0, 0};
+        for (int h = 0; h < T; ++h) cnt[h] = (int32_t)(m[h] / G);
+        if (orc_unrank_multiset(cnt, T, PP, map_idx, seq) != 0) return -1;
+        for (int s = 0; s < PP; ++s) {
+            int h = seq[s];
+            int q = used[h]++;
+            out->mask[s] = (uint8_t)(1u << h);
+            tfirst[s] = tlast[s] = h;
+            ofirst[s] = (int64_t)q * G;
+            olast[s] = (int64_t)(q + 1) * G - 1;
+        }
+    } else {
+        /* map_idx-th permutation of the types in lexicographic order */
+        int sigma[ORC_MAX_TYPES], avail[ORC_MAX_TYPES];
+        uint64_t idx = map_idx;
+        for (int h = 0; h < T; ++h) avail[h] = h;
+        for (int pos = 0; pos < T; ++pos) {
+            uint64_t f = factorial_u64(T - 1 - pos);
+            int pick = (int)(idx / f);
+            idx %= f;
+            sigma[pos] = avail[pick];
+            for (int t = pick; t + 1 < T - pos; ++t) avail[t] = avail[t + 1];
+        }
+        int64_t start[ORC_MAX_TYPES + 1];
+        start[0] = 0;
+        for (int bq = 0; bq < T; ++bq) start[bq + 1] = start[bq] + m[sigma[bq]];
+        for (int s = 0; s < PP; ++s) {
+            int64_t lo = (int64_t)s * G, hi = (int64_t)(s + 1) * G - 1;
+            for (int bq = 0; bq < T; ++bq) {
+                if (start[bq + 1] <= lo || start[bq] > hi) continue;   /* block does not overlap */
+                out->mask[s] |= (uint8_t)(1u << sigma[bq]);
+                if (start[bq] <= lo && lo < start[bq + 1]) { tfirst[s] = sigma[bq]; ofirst[s] = lo - start[bq]; }
+                if (start[bq] <= hi && hi < start[bq + 1]) { tlast[s] = sigma[bq]; olast[s] = hi - start[bq]; }
+            }
+        }
+    }
+    for (int s = 1; s < PP; ++s) {
+        int ta = tlast[s - 1], tb = tfirst[s];
+        out->ha[s] = (uint8_t)ta;
+        out->hb[s] = (uint8_t)tb;
+        if (ta != tb) out->cls[s] = ORC_CROSS;
+        else out->cls[s] = (olast[s - 1] / pr->node_size[ta] == ofirst[s] / pr->node_size[tb]) ? ORC_INTRA : ORC_INTER;
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Layer cost (Eq. 2, Eq. 3, imbalance scaling) and stage-level coefficients.
+ * c2 / c2f: [T][N][2] (forward, backward); coef / coeff: [T][ORC_NCOEF].
+ * ------------------------------------------------------------------------------------ */
+typedef struct { const orc_problem *pr; int h; double bw_inter; } linkctx;
+
+static int link_cls(const linkctx *lc, int64_t ext) { return ext <= lc->pr->node_size[lc->h] ? ORC_INTRA : ORC_INTER; }
+static double link_bw(const linkctx *lc, int cls) { return cls == ORC_INTRA ? lc->pr->bw_intra[lc->h] : lc->bw_inter; }
+
+/* ring-style collective over w ranks spanning `ext` devices moving D bytes */
+static double coll(const linkctx *lc, int64_t w, int64_t ext, double D)
+{
+    if (w == 1) return 0.0;
+    int c = link_cls(lc, ext);
+    double lat = lc->pr->alpha[c] * (double)(w - 1);
+    double vol = (D * (double)(w - 1)) / (double)w;
+    return lat + vol / link_bw(lc, c);
+}
+
+int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, double *c2f,
+                    int64_t *coef, double *coeff)
+{
+    const int N = pr->N, T = pr->T;
+    const int TP = pc->TP, CP = pc->CP, DP = pc->DP, EP = pc->EP, TPE = pc->TPE, EDP = pc->EDP, b = pc->b;
+    const int64_t G = pc->G;
+    const int64_t tok = (int64_t)b * pr->S / CP;
+    const int64_t Hkv = (int64_t)pr->H * pr->nkv / pr->nq;
+    const int64_t H = pr->H;
+    double bwi[ORC_MAX_TYPES];
+    for (int h = 0; h < T; ++h) bwi[h] = type_bw_inter(pr, h);
+
+    for (int h = 0; h < T; ++h) {
+        linkctx lc = { pr, h, bwi[h] };
+        const double thb = (double)tok * (double)H;        /* token*hidden elements per rank */
+        const double Dtp = thb * pr->beta;
+        const double imb = 1.0 + pr->gamma * (pr->rho[pc->iep] - 1.0);
+        /* expert dispatch / combine: Eq. 3 bytes, best of all-to-all and all-gather */
+        double tdisp;
+        if (EP == 1) tdisp = 0.0;
+        else {
+            double Dmoe = ((thb * pr->beta) * (double)pr->k) * (1.0 - 1.0 / (double)EP);
+            double Dag = (thb * pr->beta) * (double)(EP - 1);
+            int c = link_cls(&lc, (int64_t)EP * TPE);
+            double fa = pr->alpha[c] * (double)(EP - 1) + Dmoe / link_bw(&lc, c);
+            double fg = pr->alpha[c] * (double)(EP - 1) + Dag / link_bw(&lc, c);
+            tdisp = (fa <= fg) ? fa : fg;
+        }
+        const double ttpA = 2.0 * coll(&lc, TP, TP, Dtp);
+        const double ttpD = 2.0 * coll(&lc, TP, TP, Dtp);
+        const double ttpM = 2.0 * coll(&lc, TPE, TPE, Dtp);
+        const double Dkv = ((((2.0 * (double)b) * (double)pr->S) * (double)Hkv) * pr->beta) / (double)TP;
+        const double tcp = coll(&lc, CP, (int64_t)TP * CP, Dkv);
+        const double tr = pr->croute[h] * thb;
+        double commF[2], commB[2];
+        commF[ORC_DENSE] = pr->ovl_tp * (ttpA + ttpD) + pr->ovl_cp * tcp;
+        commB[ORC_DENSE] = pr->ovl_tp * (ttpA + ttpD) + pr->ovl_cp * (2.0 * tcp);
+        commF[ORC_MOE] = pr->ovl_tp * (ttpA + ttpM) + pr->ovl_cp * tcp;
+        commB[ORC_MOE] = pr->ovl_tp * (ttpA + ttpM) + pr->ovl_cp * (2.0 * tcp);
+
+        const int64_t i4 = (((int64_t)h * pr->ntp + pc->itp) * pr->ncp + pc->icp) * pr->nmb + pc->ib;
+        for (int l = 0; l < N; ++l) {
+            const double a = pr->tdf[i4 * N + l], f = pr->tff[i4 * N + l];
+            const double ab = pr->tdb[i4 * N + l], fb = pr->tfb[i4 * N + l];
+            double cf, cb;
+            if (pr->kind[l] == ORC_DENSE) {
+                cf = a + commF[ORC_DENSE];
+                cb = ab + commB[ORC_DENSE];
+            } else {
+                const double den = (pr->eta[h] * (double)EP) * (double)TPE;
+                const double xf = (pr->kappa * f) / den;
+                const double mf = (xf + 2.0 * tdisp) * imb;
+                cf = (((a - f) + mf) + tr) + commF[ORC_MOE];
+                const double xb = (pr->kappa * fb) / den;
+                const double mb = (xb + 2.0 * tdisp) * imb;
+                cb = (((ab - fb) + mb) + 2.0 * tr) + commB[ORC_MOE];
+            }
+            if (c2f) { c2f[((int64_t)h * N + l) * 2] = cf; c2f[((int64_t)h * N + l) * 2 + 1] = cb; }
+            if (c2) { c2[((int64_t)h * N + l) * 2] = llrint(cf); c2[((int64_t)h * N + l) * 2 + 1] = llrint(cb); }
+        }
+
+        /* stage-level coefficients */
+        double v[ORC_NCOEF];
+        v[ORC_KPRE] = pr->tpre[i4];
+        v[ORC_KPOST] = pr->tpost[i4];
+        v[ORC_KP2P_INTRA] = 2.0 * (pr->alpha[ORC_INTRA] + (Dtp / (double)TP) / pr->bw_intra[h]);
+        v[ORC_KP2P_INTER] = 2.0 * (pr->alpha[ORC_INTER] + (Dtp / (double)TP) / bwi[h]);
+        for (int h2 = 0; h2 < ORC_MAX_TYPES; ++h2) {
+            double bo = h2 < T ? bwi[h2] : bwi[h];
+            double bmin = bwi[h] < bo ? bwi[h] : bo;
+            v[ORC_KP2P_CROSS + h2] = 2.0 * (pr->alpha[ORC_CROSS] + (Dtp / (double)TP) / (bmin * pr->chi));
+        }
+        const double shd = 6.0 + 12.0 / (double)((int64_t)DP * CP);
+        const double she = 6.0 + 12.0 / (double)EDP;
+        const int64_t Pattn = H * (H + 2 * Hkv) + H * H + 2 * H;
+        const int64_t Pffn_d = 3 * H * (int64_t)pr->F_dense, Pffn_e = 3 * H * (int64_t)pr->F_exp;
+        const int64_t Pe = (int64_t)(pr->E / EP) * Pffn_e;
+        int64_t Pd[2];
+        Pd[ORC_DENSE] = Pattn + Pffn_d;
+        Pd[ORC_MOE] = Pattn + (int64_t)pr->n_shared * Pffn_e;
+        const int64_t Prt = H * (int64_t)pr->E;
+        v[ORC_MW + ORC_DENSE] = ((double)Pd[ORC_DENSE] / (double)TP) * shd;
+        v[ORC_MW + ORC_MOE] = ((double)Pd[ORC_MOE] / (double)TP + (double)Prt) * shd + ((double)Pe / (double)TPE) * she;
+        for (int kd = 0; kd < 2; ++kd) v[ORC_MA + kd] = (thb * pr->act_coef[kd]) / (double)TP;
+        v[ORC_MX] = ((2.0 * ((thb * pr->beta) * (double)pr->k)) * (1.0 - 1.0 / (double)EP)) * pr->capf
+                    + ((double)tok * (double)pr->E) * 4.0;
+        v[ORC_MPRE] = (((double)pr->V * (double)H) / (double)TP) * shd;
+        v[ORC_MPOST] = v[ORC_MPRE];
+        const int cG = link_cls(&lc, G);
+        const double bwG = link_bw(&lc, cG);
+        const int64_t wd = (int64_t)DP * CP;
+        const double vfd = (double)(wd - 1) / (double)wd, vfe = (double)(EDP - 1) / (double)EDP;
+        for (int kd = 0; kd < 2; ++kd) {
+            const int64_t Pdd = Pd[kd] + (kd == ORC_MOE ? Prt : 0);
+            const double Pel = kd == ORC_MOE ? (double)Pe / (double)TPE : 0.0;
+            v[ORC_SBW + kd] = pr->ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG)
+                                            + (((6.0 * Pel) * vfe) / bwG));
+            v[ORC_OPT + kd] = pr->copt[h] * ((double)Pdd / (double)((int64_t)TP * DP * CP) + Pel / (double)EDP);
+        }
+        v[ORC_SLAT] = pr->ovl_dp * (pr->alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
+        for (int q = 0; q < ORC_NCOEF; ++q) {
+            if (coeff) coeff[h * ORC_NCOEF + q] = v[q];
+            if (coef) coef[h * ORC_NCOEF + q] = llrint(v[q]);
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Stage cost with minimal feasible recomputation (integer arithmetic).
+ * Stage index i is 1-based; the span is layers a..b-1, i.e. (a, b] in prefix terms.
+ * ------------------------------------------------------------------------------------ */
+static int64_t mask_max(const orc_problem *pr, unsigned mask, const int64_t *coef, int q)
+{
+    int64_t best = 0;
+    int seen = 0;
+    for (int h = 0; h < pr->T; ++h)
+        if (mask & (1u << h)) {
+            int64_t x = coef[h * ORC_NCOEF + q];
+            if (!seen || x > best) best = x;
+            seen = 1;
+        }
+    return best;
+}
+
+int orc_window(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, int32_t *nmin, int32_t *nmax)
+{
+    const int PP = pc->PP, N = pr->N;
+    if (pr->delta_q < 0) {
+        for (int s = 0; s < PP; ++s) { nmin[s] = 1; nmax[s] = N - PP + 1; }
+        return 0;
+    }
+    int64_t Pst[ORC_MAX_PP], Ps = 0;
+    for (int s = 0; s < PP; ++s) {
+        int64_t p = 0;
+        int seen = 0;
+        for (int h = 0; h < pr->T; ++h)
+            if (mp->mask[s] & (1u << h)) {
+                if (!seen || pr->P[h] < p) p = pr->P[h];
+                seen = 1;
+            }
+        Pst[s] = p;
+        Ps += p;
+    }
+    for (int s = 0; s < PP; ++s) {
+        int64_t lo = ((int64_t)(1024 - pr->delta_q) * Pst[s] * N) / (1024 * Ps);
+        int64_t num = (int64_t)(1024 + pr->delta_q) * Pst[s] * N, den = 1024 * Ps;
+        int64_t hi = (num + den - 1) / den;
+        if (lo < 1) lo = 1;
+        if (hi > N - PP + 1) hi = N - PP + 1;
+        nmin[s] = (int32_t)lo;
+        nmax[s] = (int32_t)hi;
+    }
+    return 1;
+}
+
+/* Per-candidate stage data: the rows of Sec. "stage cost" built once, then every span is O(R). */
+typedef struct {
+    int N, PP, R;
+    int64_t M;
+    uint32_t rc_mask;
+    const int32_t *xi_q, *tau_q;
+    int64_t PF[ORC_MAX_PP][ORC_MAX_N + 1];   /* prefix sums of the forward row of stage s */
+    int64_t PB[ORC_MAX_PP][ORC_MAX_N + 1];   /* prefix sums of the backward row of stage s */
+    int64_t PW[ORC_MAX_N + 1], PA[ORC_MAX_N + 1];   /* weight / activation bytes (type independent) */
+    int32_t PK[ORC_MAX_N + 1];               /* number of MoE layers among the first l */
+    int64_t cap[ORC_MAX_PP], K[ORC_MAX_PP], mpre, mpost, mx;
+    int32_t nmin[ORC_MAX_PP], nmax[ORC_MAX_PP];
+} stage_ctx;
+
+static void ctx_build(stage_ctx *cx, const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                      uint32_t rc_mask, const int64_t *c2, const int64_t *coef)
+{
+    const int N = pr->N, PP = pc->PP;
+    cx->N = N; cx->PP = PP; cx->R = pr->R; cx->M = pc->M; cx->rc_mask = rc_mask;
+    cx->xi_q = pr->xi_q; cx->tau_q = pr->tau_q;
+    orc_window(pr, pc, mp, cx->nmin, cx->nmax);
+    cx->PW[0] = cx->PA[0] = 0; cx->PK[0] = 0;
+    for (int l = 0; l < N; ++l) {
+        /* weight / activation bytes do not depend on the device type: row of type 0 */
+        cx->PW[l + 1] = cx->PW[l] + coef[ORC_MW + pr->kind[l]];
+        cx->PA[l + 1] = cx->PA[l] + coef[ORC_MA + pr->kind[l]];
+        cx->PK[l + 1] = cx->PK[l] + (pr->kind[l] == ORC_MOE ? 1 : 0);
+    }
+    cx->mpre = coef[ORC_MPRE]; cx->mpost = coef[ORC_MPOST]; cx->mx = coef[ORC_MX];
+    for (int s = 0; s < PP; ++s) {
+        const unsigned mask = mp->mask[s];
+        const int i = s + 1;
+        /* a (possibly mixed) stage runs each layer at the pace of its slowest member type */
+        cx->PF[s][0] = cx->PB[s][0] = 0;
+        for (int l = 0; l < N; ++l) {
+            int64_t F = 0, Bk = 0;
+            int seen = 0;
+            for (int h = 0; h < pr->T; ++h)
+                if (mask & (1u << h)) {
+                    int64_t qf = c2[((int64_t)h * N + l) * 2], qb = c2[((int64_t)h * N + l) * 2 + 1];
+                    if (!seen || qf > F) F = qf;
+                    if (!seen || qb > Bk) Bk = qb;
+                    seen = 1;
+                }
+            cx->PF[s][l + 1] = cx->PF[s][l] + F;
+            cx->PB[s][l + 1] = cx->PB[s][l] + Bk;
+        }
+        /* it must fit its smallest member */
+        int64_t cap = 0;
+        int seen = 0;
+        for (int h = 0; h < pr->T; ++h)
+            if (mask & (1u << h)) {
+                if (!seen || pr->cap_eff[h] < cap) cap = pr->cap_eff[h];
+                seen = 1;
+            }
+        cx->cap[s] = cap;
+        /* stage constant: embedding / head work and the p2p transfer into this stage */
+        int64_t K = 0;
+        if (i == 1) K += mask_max(pr, mask, coef, ORC_KPRE);
+        if (i == PP) K += mask_max(pr, mask, coef, ORC_KPOST);
+        if (i > 1) {
+            int hb = mp->hb[s], ha = mp->ha[s];
+            if (mp->cls[s] == ORC_INTRA) K += coef[hb * ORC_NCOEF + ORC_KP2P_INTRA];
+            else if (mp->cls[s] == ORC_INTER) K += coef[hb * ORC_NCOEF + ORC_KP2P_INTER];
+            else K += coef[hb * ORC_NCOEF + ORC_KP2P_CROSS + ha];
+        }
+        cx->K[s] = K;
+    }
+}
+
+/* cost of stage i (1-based) holding layers a..b-1 */
+static int64_t ctx_stage_cost(const stage_ctx *cx, int i, int a, int b, int *r_out)
+{
+    const int s = i - 1, PP = cx->PP;
+    if (r_out) *r_out = -1;
+    const int n = b - a;
+    if (n < cx->nmin[s] || n > cx->nmax[s]) return ORC_INF;          /* Pruning 1: load-balance window */
+    /* memory: M_w + M_act + M_moe-extra */
+    const int has_moe = cx->PK[b] - cx->PK[a] > 0;
+    const int64_t Wb = (cx->PW[b] - cx->PW[a]) + (i == 1 ? cx->mpre : 0) + (i == PP ? cx->mpost : 0)
+                       + (has_moe ? cx->mx : 0);
+    const int64_t Mstore = cx->M < PP - i + 1 ? cx->M : PP - i + 1;    /* 1F1B in-flight micro-batches */
+    const int64_t A = Mstore * (cx->PA[b] - cx->PA[a]);
+    int rstar = -1;
+    for (int r = 0; r < cx->R && rstar < 0; ++r)
+        if ((cx->rc_mask >> r) & 1u)
+            if (Wb + ((int64_t)cx->xi_q[r] * A) / 1024 <= cx->cap[s]) rstar = r;    /* minimal feasible level */
+    if (rstar < 0) return ORC_INF;                                   /* Pruning 2: memory */
+    if (r_out) *r_out = rstar;
+    const int64_t SF = cx->PF[s][b] - cx->PF[s][a], SB = cx->PB[s][b] - cx->PB[s][a];
+    return SF + SB + ((int64_t)cx->tau_q[rstar] * SF) / 1024 + cx->K[s];
+}
+
+int64_t orc_stage_cost(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                       uint32_t rc_mask, const int64_t *c2, const int64_t *coef,
+                       int i, int a, int b, int *r_out)
+{
+    stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+    if (!cx) return -1;
+    ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+    int64_t c = ctx_stage_cost(cx, i, a, b, r_out);
+    free(cx);
+    return c;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Min-max pipeline partitioning recurrence, backtrace and Eq. 4 closed form.
+ * dp_table: [(PP+1)][(N+1)] or NULL; ch_table: same shape, 255 where undefined.
+ * ------------------------------------------------------------------------------------ */
+int orc_candidate(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                  const int64_t *c2, const int64_t *coef, orc_result *res,
+                  int64_t *dp_table, uint8_t *ch_table)
+{
+    const int N = pr->N, PP = pc->PP;
+    stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+    int64_t *DPt = (int64_t *)malloc(sizeof(int64_t) * (size_t)(PP + 1) * (N + 1));
+    uint8_t *CH = (uint8_t *)malloc((size_t)(PP + 1) * (N + 1));
+    if (!DPt || !CH || !cx) { free(DPt); free(CH); free(cx); return -1; }
+    ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+#define DPAT(i, j) DPt[(size_t)(i) * (N + 1) + (j)]
+#define CHAT(i, j) CH[(size_t)(i) * (N + 1) + (j)]
+    for (int i = 0; i <= PP; ++i)
+        for (int j = 0; j <= N; ++j) { DPAT(i, j) = ORC_INF; CHAT(i, j) = 255; }
+    DPAT(0, 0) = 0;
+    for (int i = 1; i <= PP; ++i)
+        for (int j = i; j <= N - PP + i; ++j)
+            for (int k = i - 1; k <= j - 1; ++k) {
+                if (DPAT(i - 1, k) >= ORC_INF) continue;
+                int64_t c = ctx_stage_cost(cx, i, k, j, NULL);
+                int64_t v = DPAT(i - 1, k) > c ? DPAT(i - 1, k) : c;
+                if (v < DPAT(i, j)) { DPAT(i, j) = v; CHAT(i, j) = (uint8_t)k; }   /* strict: smallest k wins */
+            }
+    memset(res, 0, sizeof(*res));
+    res->bottleneck = DPAT(PP, N);
+    if (dp_table) memcpy(dp_table, DPt, sizeof(int64_t) * (size_t)(PP + 1) * (N + 1));
+    if (ch_table) memcpy(ch_table, CH, (size_t)(PP + 1) * (N + 1));
+    if (res->bottleneck >= ORC_INF) {
+        res->T_iter = res->T_pipe = ORC_INF;
+        free(DPt); free(CH); free(cx);
+        return 1;
+    }
+    /* backtrace */
+    int64_t sum = 0, mx = 0, tsync = 0, topt = 0;
+    int j = N;
+    for (int i = PP; i >= 1; --i) {
+        int k = CHAT(i, j), r;
+        int64_t c = ctx_stage_cost(cx, i, k, j, &r);
+        res->n[i - 1] = (uint8_t)(j - k);
+        res->r[i - 1] = (uint8_t)r;
+        res->c[i - 1] = c;
+        sum += c;
+        if (c > mx) mx = c;
+        /* gradient synchronisation and optimizer step of this stage (after the partition is fixed) */
+        unsigned mask = mp->mask[i - 1];
+        int64_t sy = mask_max(pr, mask, coef, ORC_SLAT), op = 0;
+        for (int l = k; l < j; ++l) {
+            sy += mask_max(pr, mask, coef, ORC_SBW + pr->kind[l]);
+            op += mask_max(pr, mask, coef, ORC_OPT + pr->kind[l]);
+        }
+        if (sy > tsync) tsync = sy;
+        if (op > topt) topt = op;
+        j = k;
+    }
+    res->T_pipe = sum + (int64_t)(pc->M - 1) * mx;     /* sum(stage) + (M-1) * max(stage) */
+    res->T_sync = tsync;
+    res->T_opt = topt;
+    res->T_iter = res->T_pipe + tsync + topt;
+    free(DPt); free(CH); free(cx);
+#undef DPAT
+#undef CHAT
+    return 0;
+}
+
+/* Exhaustive minimum over every contiguous partition of layers 1..j into stages 1..i of the
+ * largest stage cost (no recurrence, no memo): the plain definition of the bottleneck. */
+static void bf_rec(const stage_ctx *cx, int stage, int nstages, int start, int end,
+                   int64_t cur_max, int64_t *best, uint64_t *count)
+{
+    if (stage == nstages) {
+        int64_t c = ctx_stage_cost(cx, stage, start, end, NULL);
+        int64_t v = c > cur_max ? c : cur_max;
+        if (v < *best) *best = v;
+        (*count)++;
+        return;
+    }
+    /* leave at least one layer for each later stage */
+    for (int cut = start + 1; cut <= end - (nstages - stage); ++cut) {
+        int64_t c = ctx_stage_cost(cx, stage, start, cut, NULL);
+        int64_t v = c > cur_max ? c : cur_max;
+        bf_rec(cx, stage + 1, nstages, cut, end, v, best, count);
+    }
+}
+
+int64_t orc_bruteforce(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                       const int64_t *c2, const int64_t *coef, int i, int j, uint64_t *n_partitions)
+{
+    int64_t best = ORC_INF;
+    uint64_t count = 0;
+    if (i == 0) { if (n_partitions) *n_partitions = 0; return j == 0 ? 0 : ORC_INF; }
+    if (j >= i) {
+        stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+        if (!cx) return -1;
+        ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+        bf_rec(cx, 1, i, 0, j, 0, &best, &count);
+        free(cx);
+    }
+    if (n_partitions) *n_partitions = count;
+    return best > ORC_INF ? ORC_INF : best;
+}
+
+/* ------------------------------------------------------------------------------------ *
+ * Candidate index -> evaluation; exhaustive search with (cost, index) argmin.
+ * ------------------------------------------------------------------------------------ */
+static int64_t find_pconf(const orc_pconf *pcs, uint64_t n_pconf, uint64_t n_rc, uint64_t index)
+{
+    for (uint64_t p = 0; p < n_pconf; ++p)
+        if (index >= pcs[p].offset && index < pcs[p].offset + pcs[p].nmap * n_rc) return (int64_t)p;
+    return -1;
+}
+
+int orc_eval_index(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t index,
+                   orc_plan *out, int64_t *dp_table, uint8_t *ch_table)
+{
+    int64_t p = find_pconf(pcs, n_pconf, (uint64_t)pr->n_rc, index);
+    if (p < 0) return -1;
+    const orc_pconf *pc = &pcs[p];
+    uint64_t local = index - pc->offset;
+    uint64_t map_idx = local / (uint64_t)pr->n_rc, rc_idx = local % (uint64_t)pr->n_rc;
+    int64_t *c2 = (int64_t *)malloc(sizeof(int64_t) * (size_t)pr->T * pr->N * 2);
+    int64_t coef[ORC_MAX_TYPES * ORC_NCOEF];
+    if (!c2) return -1;
+    orc_layer_costs(pr, pc, c2, NULL, coef, NULL);
+    memset(out, 0, sizeof(*out));
+    out->index = index;
+    out->pc = *pc;
+    out->rc_mask = pr->rc_masks[rc_idx];
+    int rcode = orc_decode(pr, pc, map_idx, &out->map);
+    if (rcode == 0) rcode = orc_candidate(pr, pc, &out->map, out->rc_mask, c2, coef, &out->res, dp_table, ch_table);
+    free(c2);
+    return rcode < 0 ? rcode : 0;
+}
+
+int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t first, uint64_t count,
+               int64_t *costs, int64_t *bottlenecks, orc_plan *best, uint64_t *n_feasible)
+{
+    int64_t *c2 = (int64_t *)malloc(sizeof(int64_t) * (size_t)pr->T * pr->N * 2);
+    int64_t coef[ORC_MAX_TYPES * ORC_NCOEF];
+    int64_t best_cost = ORC_INF;
+    uint64_t feas = 0;
+    if (!c2) return -1;
+    if (best) { memset(best, 0, sizeof(*best)); best->res.T_iter = ORC_INF; best->index = UINT64_MAX; }
+    for (uint64_t p = 0; p < n_pconf; ++p) {
+        const orc_pconf *pc = &pcs[p];
+        uint64_t lo = pc->offset, hi = pc->offset + pc->nmap * (uint64_t)pr->n_rc;
+        if (hi <= first || lo >= first + count) continue;
+        orc_layer_costs(pr, pc, c2, NULL, coef, NULL);
+        for (uint64_t map_idx = 0; map_idx < pc->nmap; ++map_idx) {
+            orc_mapping mp;
+            int decoded = 0;
+            for (int rc = 0; rc < pr->n_rc; ++rc) {
+                uint64_t idx = lo + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
+                if (idx < first || idx >= first + count) continue;
+                if (!decoded) { orc_decode(pr, pc, map_idx, &mp); decoded = 1; }
+                orc_result res;
+                orc_candidate(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL, NULL);
+                if (costs) costs[idx - first] = res.T_iter;
+                if (bottlenecks) bottlenecks[idx - first] = res.bottleneck;
+                if (res.T_iter < ORC_INF) feas++;
+                if (res.T_iter < best_cost) {           /* ascending index + strict: lowest index wins */
+                    best_cost = res.T_iter;
+                    if (best) {
+                        best->index = idx; best->pc = *pc; best->map = mp;
+                        best->rc_mask = pr->rc_masks[rc]; best->res = res;
+                    }
+                }
+            }
+        }
+    }
+    if (n_feasible) *n_feasible = feas;
+    free(c2);
+    return 0;
+}
+
+/* Timing harness: evaluates every candidate of configurations p_first, p_first+stride, ...
+ * (threads > 1 spreads configurations over OpenMP threads; the per-candidate work is the
+ * plain code above).  Returns the (cost, index) minimum over what it evaluated. */
+int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
+                      uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index)
+{
+    int64_t gbest = ORC_INF;
+    uint64_t gidx = UINT64_MAX, done = 0;
+    if (p_stride == 0) p_stride = 1;
+    int64_t nsel = p_first < n_pconf ? (int64_t)((n_pconf - p_first + p_stride - 1) / p_stride) : 0;
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : done)
+    for (int64_t q = 0; q < nsel; ++q) {
+        uint64_t p = p_first + (uint64_t)q * p_stride;
+        const orc_pconf *pc = &pcs[p];
+        int64_t *c2 = (int64_t *)malloc(sizeof(int64_t) * (size_t)pr->T * pr->N * 2);
+        int64_t coef[ORC_MAX_TYPES * ORC_NCOEF];
+        int64_t lbest = ORC_INF;
+        uint64_t lidx = UINT64_MAX;
+        orc_layer_costs(pr, pc, c2, NULL, coef, NULL);
+        for (uint64_t map_idx = 0; map_idx < pc->nmap; ++map_idx) {
+            orc_mapping mp;
+            orc_decode(pr, pc, map_idx, &mp);
+            for (int rc = 0; rc < pr->n_rc; ++rc) {
+                orc_result res;
+                orc_candidate(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL, NULL);
+                uint64_t idx = pc->offset + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
+                if (res.T_iter < lbest) { lbest = res.T_iter; lidx = idx; }
+                done++;
+            }
+        }
+        free(c2);
+#pragma omp critical
+        {
+            if (lbest < gbest || (lbest == gbest && lidx < gidx)) { gbest = lbest; gidx = lidx; }
+        }
+    }
+    *n_done = done;
+    *best_cost = gbest;
+    *best_index = gidx;
+    return 0;
+}

@@ -1,0 +1,126 @@
+/*
+ * CPU oracle of the HAPMoE planner hot path -- TEST INFRASTRUCTURE, not a product path.
+ *
+ * A plain, slow, single-threaded restatement of what the planner computes: the 6-D
+ * enumeration, the MoE-aware layer cost (Eq. 2, Eq. 3, load-imbalance scaling), the stage
+ * memory model with minimal feasible recomputation, the per-candidate min-max pipeline
+ * partitioning recurrence, the 1F1B closed-form iteration latency (Eq. 4) and the global
+ * argmin (Eq. 1).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+ * call it.  It shares no code with the CUDA library.
+ *
+ * Parity status: every function below is pinned by tests that do not go through this file's
+ * own formulas (hand-computed cost terms, brute force over all contiguous partitions,
+ * closed forms and invariants).  Nothing here is "parity unpinned".
+ */
+#ifndef HAP_ORACLE_H
+#define HAP_ORACLE_H
+#include <stdint.h>
+
+#define ORC_MAX_TYPES 4
+#define ORC_MAX_PP 32
+#define ORC_MAX_N 255
+#define ORC_MAX_RC 4
+#define ORC_INF ((int64_t)1 << 62)
+
+enum { ORC_DENSE = 0, ORC_MOE = 1 };
+enum { ORC_INTRA = 0, ORC_INTER = 1, ORC_CROSS = 2 };
+enum { ORC_MODE_MULTISET = 0, ORC_MODE_BLOCK = 1 };
+
+/* stage-level coefficients per (configuration, device type), all rounded to int64 */
+enum {
+    ORC_KPRE = 0, ORC_KPOST = 1, ORC_KP2P_INTRA = 2, ORC_KP2P_INTER = 3,
+    ORC_KP2P_CROSS = 4, /* +h' for the sending type, 4 entries */
+    ORC_SLAT = 8, ORC_SBW = 9, /* +kind */ ORC_OPT = 11, /* +kind */
+    ORC_MW = 13, /* +kind */ ORC_MA = 15, /* +kind */ ORC_MX = 17, ORC_MPRE = 18, ORC_MPOST = 19,
+    ORC_NCOEF = 20
+};
+
+typedef struct {
+    /* model */
+    int32_t N, S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
+    double beta;
+    const uint8_t *kind;
+    /* cluster */
+    int32_t T;
+    const int64_t *P, *C;
+    const int32_t *node_size;
+    const double *bw_intra;
+    int32_t n_nodes;
+    const int32_t *node_type;
+    const double *node_bw_inter;
+    /* profile */
+    int32_t ntp, ncp, nmb, nep;
+    const int32_t *tp_list, *cp_list, *mb_list, *ep_list;
+    const double *tdf, *tdb, *tff, *tfb, *tpre, *tpost, *eta, *croute;
+    double kappa;
+    const double *alpha;
+    double chi;
+    const double *rho;
+    double gamma, ovl_tp, ovl_cp, ovl_dp;
+    const double *act_coef;
+    double capf;
+    const double *copt;
+    const int64_t *cap_eff;
+    int32_t R;
+    const int32_t *xi_q, *tau_q;
+    /* search options */
+    int32_t npp, ntpe;
+    const int32_t *pp_list, *tpe_list;
+    int32_t tp_max, delta_q;
+    uint64_t map_cap;
+    int32_t n_rc;
+    const uint32_t *rc_masks;
+} orc_problem;
+
+typedef struct {
+    int32_t PP, TP, CP, DP, EP, TPE, b, M, EDP, G;
+    int32_t itp, icp, ib, iep, mode, pad;
+    uint64_t nmap, offset;
+} orc_pconf;
+
+typedef struct {
+    int32_t PP;
+    uint8_t mask[ORC_MAX_PP];   /* bit h set: stage overlaps device type h */
+    uint8_t cls[ORC_MAX_PP];    /* link class of the boundary entering stage s (s >= 1) */
+    uint8_t ha[ORC_MAX_PP];     /* type of the last device of stage s-1 */
+    uint8_t hb[ORC_MAX_PP];     /* type of the first device of stage s */
+} orc_mapping;
+
+typedef struct {
+    int64_t T_iter, bottleneck, T_pipe, T_sync, T_opt;
+    uint8_t n[ORC_MAX_PP];   /* layers per stage */
+    uint8_t r[ORC_MAX_PP];   /* recompute level per stage */
+    int64_t c[ORC_MAX_PP];   /* stage cost of the chosen partition */
+} orc_result;
+
+typedef struct {
+    uint64_t index;
+    orc_pconf pc;
+    orc_mapping map;
+    uint32_t rc_mask;
+    orc_result res;
+} orc_plan;
+
+int orc_enumerate(const orc_problem *pr, orc_pconf *out, uint64_t cap, uint64_t *n_pconf, uint64_t *n_cand);
+uint64_t orc_multiset_count(const int32_t *cnt, int T, uint64_t sat);
+int orc_unrank_multiset(const int32_t *cnt, int T, int PP, uint64_t idx, uint8_t *seq);
+uint64_t orc_rank_multiset(const int32_t *cnt, int T, int PP, const uint8_t *seq);
+int orc_decode(const orc_problem *pr, const orc_pconf *pc, uint64_t map_idx, orc_mapping *out);
+int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, double *c2f,
+                    int64_t *coef, double *coeff);
+int64_t orc_stage_cost(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                       uint32_t rc_mask, const int64_t *c2, const int64_t *coef,
+                       int i, int a, int b, int *r_out);
+int orc_window(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, int32_t *nmin, int32_t *nmax);
+int orc_candidate(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                  const int64_t *c2, const int64_t *coef, orc_result *res,
+                  int64_t *dp_table, uint8_t *ch_table);
+int64_t orc_bruteforce(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                       const int64_t *c2, const int64_t *coef, int i, int j, uint64_t *n_partitions);
+int orc_eval_index(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t index,
+                   orc_plan *out, int64_t *dp_table, uint8_t *ch_table);
+int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t first, uint64_t count,
+               int64_t *costs, int64_t *bottlenecks, orc_plan *best, uint64_t *n_feasible);
+int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
+                      uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index);
+#endif
