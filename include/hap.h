@@ -1,0 +1,230 @@
+/*
+ * libhap -- C ABI of the HAPMoE planner hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates the paper's MoE-aware cost model over the 6-D parallel space
+ * (DP, PP, TP, CP, EP, TPE) x device-group-to-stage mappings x recomputation policies,
+ * runs the per-candidate non-uniform pipeline-partitioning dynamic program under per-stage
+ * memory feasibility and returns the argmin plan (problem statement: Sec. 3.2, Eq. 1).
+ *
+ * Conventions
+ *  - Every function returns a hap_status; nothing throws, exits or prints.
+ *  - Descriptor structs and the arrays they point to are HOST memory owned by the caller;
+ *    hap_problem_create copies them, so they may be freed right after it returns.
+ *  - Arguments named dev_* are DEVICE pointers owned by the caller (for example the
+ *    data_ptr() of a torch tensor) on the device that was current at hap_problem_create.
+ *    The library never frees or reallocates them.  Nullable ones are marked.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Kernels are
+ *    enqueued on it and the call returns without waiting, except where a function returns
+ *    host values: that function synchronises `stream` (only that stream) before returning.
+ *  - A hap_problem is not thread safe; use one per thread or serialise calls.
+ *  - Times are nanoseconds, memory is bytes, both as int64 after round-to-nearest-even of
+ *    the fp64 formula value ("integer mode").  HAP_INF marks an infeasible candidate.
+ */
+#ifndef HAP_H
+#define HAP_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HAP_MAX_TYPES 4      /* device types |H| */
+#define HAP_MAX_PP 32        /* pipeline stages */
+#define HAP_MAX_LAYERS 255   /* N */
+#define HAP_MAX_RC 4         /* recomputation levels R */
+#define HAP_MAX_RC_MASKS 8   /* recomputation policies n_rc */
+#define HAP_MAX_LIST 16      /* entries of any degree list */
+#define HAP_INF ((int64_t)1 << 62)
+
+typedef enum {
+    HAP_OK = 0,
+    HAP_E_INVALID = 1,     /* bad descriptor or argument */
+    HAP_E_NOMEM = 2,       /* host or device allocation failed */
+    HAP_E_CUDA = 3,        /* a CUDA call failed; see hap_last_error */
+    HAP_E_RANGE = 4,       /* index range outside the candidate space, or a cost overflowed */
+    HAP_E_STATE = 5,       /* call order violated (e.g. hap_pipeline_dp before hap_enumerate) */
+    HAP_E_INFEASIBLE = 6   /* every candidate violates the memory constraint of Eq. 1 */
+} hap_status;
+
+enum { HAP_DENSE = 0, HAP_MOE = 1 };                  /* layer kind */
+enum { HAP_INTRA = 0, HAP_INTER = 1, HAP_CROSS = 2 }; /* link class (Sec. 3.3: intra-node, inter-node, cross-type) */
+enum { HAP_MAP_MULTISET = 0, HAP_MAP_BLOCK = 1 };     /* mapping mode of a configuration */
+
+/* Column layout of the per-(configuration, device type) stage coefficient row. */
+enum {
+    HAP_KPRE = 0,        /* embedding work charged to the first stage, ns */
+    HAP_KPOST = 1,       /* LM head + loss work charged to the last stage, ns */
+    HAP_KP2P_INTRA = 2,  /* activation + gradient transfer into a stage over an intra-node link, ns */
+    HAP_KP2P_INTER = 3,  /* same, inter-node link between devices of one type */
+    HAP_KP2P_CROSS = 4,  /* same, cross-type link; +h' where h' is the sending type (4 entries) */
+    HAP_SLAT = 8,        /* latency part of T_dp-sync, ns */
+    HAP_SBW = 9,         /* bandwidth part of T_dp-sync per layer; +kind */
+    HAP_OPT = 11,        /* T_opt per layer; +kind */
+    HAP_MW = 13,         /* weights + gradients + optimizer state per layer, bytes; +kind */
+    HAP_MA = 15,         /* activation bytes per layer per stored micro-batch; +kind */
+    HAP_MX = 17,         /* M_moe-extra of a stage that holds at least one MoE layer, bytes */
+    HAP_MPRE = 18,       /* embedding weights on the first stage, bytes */
+    HAP_MPOST = 19,      /* LM head weights on the last stage, bytes */
+    HAP_NCOEF = 20
+};
+
+/* Model and training hyper-parameters (Sec. 3.2 "Input": N, S, H, E, k, batch sizes). */
+typedef struct {
+    int32_t N;          /* layers, 1..HAP_MAX_LAYERS */
+    int32_t S;          /* sequence length */
+    int32_t H;          /* hidden size */
+    int32_t E;          /* routed experts per MoE layer */
+    int32_t k;          /* top-k */
+    int32_t n_shared;   /* shared experts per MoE layer */
+    int32_t F_dense;    /* FFN width of dense layers */
+    int32_t F_exp;      /* FFN width of one expert */
+    int32_t nq, nkv;    /* attention heads / KV heads */
+    int32_t V;          /* vocabulary */
+    int32_t GB;         /* global batch (sequences) */
+    double beta;        /* bytes per activation element */
+    const uint8_t *kind; /* [N] HAP_DENSE / HAP_MOE */
+} hap_model;
+
+/* Cluster: device-type triples (P_h, C_h, B_h) and inventory {m_h} as a node list. */
+typedef struct {
+    int32_t n_types;               /* 1..HAP_MAX_TYPES; every type must own at least one node */
+    const int64_t *P;              /* [n_types] peak GFLOP/s (used by the load-balance window) */
+    const int64_t *C;              /* [n_types] raw memory capacity, bytes (informational) */
+    const int32_t *node_size;      /* [n_types] devices per node of the type */
+    const double *bw_intra;        /* [n_types] bytes/ns inside a node */
+    int32_t n_nodes;
+    const int32_t *node_type;      /* [n_nodes] type id of each node; a type's device line lists its nodes in this order */
+    const double *node_bw_inter;   /* [n_nodes] bytes/ns of the node's uplink; a type uses the minimum over its nodes */
+} hap_cluster;
+
+/* Profiled lookup tables and calibrated coefficients (Sec. 3.3 and 3.4: compute table,
+ * communication primitive table, memory calibration).  Table layout: row-major
+ * [type][itp][icp][ib][layer] for the per-layer tables, [type][itp][icp][ib] for tpre/tpost,
+ * where itp/icp/ib index tp_list/cp_list/mb_list. */
+typedef struct {
+    int32_t ntp, ncp, nmb, nep;
+    const int32_t *tp_list, *cp_list, *mb_list, *ep_list;
+    const double *tdf, *tdb;     /* t_dense forward / backward of one micro-batch, ns */
+    const double *tff, *tfb;     /* t_ffn forward / backward (the part the experts replace), ns */
+    const double *tpre, *tpost;  /* embedding / LM-head+loss forward+backward, ns */
+    const double *eta;           /* [n_types] device-efficiency factor of Eq. 2, in (0,1] */
+    const double *croute;        /* [n_types] router cost, ns per token*hidden element */
+    double kappa;                /* the numerator constant of Eq. 2's expert term ("2" as printed) */
+    const double *alpha;         /* [3] latency per collective step for HAP_INTRA/INTER/CROSS, ns */
+    double chi;                  /* bandwidth factor of a cross-type link */
+    const double *rho;           /* [nep] load imbalance (max expert load / mean load), >= 1 */
+    double gamma;                /* imbalance weight in [0,1] */
+    double ovl_tp, ovl_cp, ovl_dp; /* exposed fraction of TP / CP / DP collectives */
+    const double *act_coef;      /* [2] activation bytes per token*hidden element, by layer kind */
+    double capf;                 /* capacity factor of the dispatch buffers */
+    const double *copt;          /* [n_types] optimizer time, ns per parameter */
+    const int64_t *cap_eff;      /* [n_types] usable memory after calibration, bytes */
+    int32_t R;                   /* recomputation levels, 1..HAP_MAX_RC; level 0 = none */
+    const int32_t *xi_q;         /* [R] activation-memory factor xi(r) in 1/1024 */
+    const int32_t *tau_q;        /* [R] fraction of the forward pass re-executed, in 1/1024 */
+} hap_profile;
+
+typedef struct {
+    int32_t npp, ntpe;
+    const int32_t *pp_list, *tpe_list;  /* pipeline and expert-TP degrees to try (ascending) */
+    int32_t tp_max;                      /* TP and TPE are limited to this */
+    int32_t delta_q;                     /* load-balance window delta in 1/1024 (Pruning 1); < 0 disables */
+    uint64_t map_cap;                    /* enumerate all distinct stage-type sequences only up to this count (<= 2^56) */
+    int32_t n_rc;                        /* recomputation policies, 1..HAP_MAX_RC_MASKS */
+    const uint32_t *rc_masks;            /* [n_rc] bit r set: level r allowed; per stage the lowest feasible allowed level is used */
+    int32_t prune;                       /* hap_search_best may skip candidates whose lower bound exceeds the incumbent */
+} hap_search_opts;
+
+/* One accepted parallel configuration x micro-batch size.  Candidate index of
+ * (map_idx, rc_idx) in configuration p: offset + map_idx * n_rc + rc_idx. */
+typedef struct {
+    int32_t PP, TP, CP, DP, EP, TPE, b, M, EDP, G;
+    int32_t itp, icp, ib, iep, mode, reserved;
+    uint64_t nmap, offset;
+} hap_pconf;
+
+/* Decoded candidate (device mapping {h_i} of Sec. 3.2 plus the recomputation policy). */
+typedef struct {
+    uint64_t index;
+    uint32_t pconf, rc_mask;
+    uint64_t map_idx;
+    uint8_t PP, pad[7];
+    uint8_t mask[HAP_MAX_PP];   /* bit h: stage overlaps device type h */
+    uint8_t link[HAP_MAX_PP];   /* boundary into stage s>=1: class | sending type << 2 | receiving type << 4 */
+} hap_candidate;
+
+/* The plan of Sec. 3.2 "Output": configuration, partition, device mapping, recomputation. */
+typedef struct {
+    uint64_t index;
+    int32_t PP, TP, CP, DP, EP, TPE, b, M;
+    uint32_t rc_mask, pad;
+    uint8_t n[HAP_MAX_PP];      /* layers per stage, sum = N */
+    uint8_t mask[HAP_MAX_PP];   /* device types of each stage */
+    uint8_t r[HAP_MAX_PP];      /* recomputation level per stage */
+    int64_t T_iter, bottleneck, T_pipe, T_sync, T_opt;
+} hap_plan;
+
+typedef struct {
+    uint64_t n_pconf, n_candidates;
+    uint64_t n_evaluated;   /* candidates whose dynamic program ran */
+    uint64_t n_pruned;      /* candidates skipped by the lower bound */
+    uint64_t n_feasible;    /* evaluated candidates with a finite cost */
+    float ms_layer_cost, ms_dp, ms_total;   /* CUDA-event times of the phases on `stream` */
+} hap_search_stats;
+
+typedef struct hap_problem hap_problem;
+
+/* Sec. 3.2: takes the planner's inputs.  Validates, copies the descriptors and uploads the
+ * tables to the current device.  *out is NULL on failure. */
+hap_status hap_problem_create(const hap_model *, const hap_cluster *, const hap_profile *,
+                              const hap_search_opts *, hap_problem **out);
+void hap_problem_destroy(hap_problem *);
+
+/* Sec. 3.5 / 5.1 "searches the 6D parallel space": enumerates every (PP,TP,CP,DP,EP,TPE) with
+ * PP*TP*CP*DP = #devices, EP*TPE | TP*CP*DP, EP | E, x micro-batch size, in a fixed
+ * lexicographic order, counts the stage mappings of each and builds the device-side tables. */
+hap_status hap_enumerate(hap_problem *, uint64_t *n_pconf, uint64_t *n_candidates);
+hap_status hap_get_pconfs(const hap_problem *, hap_pconf *host_out, uint64_t cap);
+
+/* Device assignment {h_i}: decodes candidates [first, first+count) into dev_out[count]. */
+hap_status hap_decode(hap_problem *, uint64_t first, uint64_t count, hap_candidate *dev_out, void *stream);
+
+/* Eq. 2, Eq. 3, load-imbalance scaling, exposed collective time, memory model coefficients
+ * (Sec. 3.3), T_dp-sync / T_opt coefficients (Eq. 4).
+ * dev_c2:   [n_pconf][n_types][N][2] forward/backward ns per layer (nullable)
+ * dev_coef: [n_pconf][n_types][HAP_NCOEF] (nullable)
+ * hap_eval_layer_costs_f64 writes the unrounded fp64 values in the same layouts. */
+hap_status hap_eval_layer_costs(hap_problem *, int64_t *dev_c2, int64_t *dev_coef, void *stream);
+hap_status hap_eval_layer_costs_f64(hap_problem *, double *dev_c2, double *dev_coef, void *stream);
+
+/* Sec. 3.5 (non-uniform layer assignment, Pruning 1 and 2) with the min-max recurrence
+ * DP[i][j] = min_k max(DP[i-1][k], cost_i(k,j)), backtrace, and Eq. 4 in the closed form
+ * sum_i c_i + (M-1) max_i c_i + T_dp-sync + T_opt, for candidates [first, first+count).
+ * Recomputes the layer costs into library-owned memory first.  No candidate is skipped.
+ * dev_cost, dev_bottleneck: [count] (HAP_INF when infeasible)
+ * dev_partition, dev_recompute: [count][HAP_MAX_PP] (nullable; zero when infeasible)
+ * dev_dp_table: [count][HAP_MAX_PP+1][N+1] int64, rows 0..PP written (nullable)
+ * dev_choice:   [count][HAP_MAX_PP+1][N+1] uint8, smallest optimal split k, 255 = none (nullable) */
+hap_status hap_pipeline_dp(hap_problem *, uint64_t first, uint64_t count, int64_t *dev_cost,
+                           int64_t *dev_bottleneck, uint8_t *dev_partition, uint8_t *dev_recompute,
+                           int64_t *dev_dp_table, uint8_t *dev_choice, void *stream);
+
+/* Eq. 1: layer costs, dynamic program and argmin over candidates [first, first+count) with
+ * ties going to the lowest index; writes the plan to host memory.  Synchronises `stream`.
+ * host_stats is nullable.  Returns HAP_E_INFEASIBLE when no candidate is feasible. */
+hap_status hap_search_range(hap_problem *, uint64_t first, uint64_t count, hap_plan *host_out,
+                            hap_search_stats *host_stats, void *stream);
+/* The whole candidate space. */
+hap_status hap_search_best(hap_problem *, hap_plan *host_out, hap_search_stats *host_stats, void *stream);
+
+/* Lexicographic (cost, index) minimum of a device cost array: writes dev_out[0] = cost,
+ * dev_out[1] = index (as int64) of the minimum of dev_cost[0..count). */
+hap_status hap_argmin(hap_problem *, const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream);
+
+const char *hap_status_str(hap_status);
+const char *hap_last_error(const hap_problem *);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HAP_H */

@@ -690,7 +690,8 @@ int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, ui
  * (threads > 1 spreads configurations over OpenMP threads; the per-candidate work is the
  * plain code above).  Returns the (cost, index) minimum over what it evaluated. */
 int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
-                      uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index)
+                      uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
+                      int64_t *costs, int64_t *bottlenecks)
 {
     int64_t gbest = ORC_INF;
     uint64_t gidx = UINT64_MAX, done = 0;
@@ -712,6 +713,8 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
                 orc_result res;
                 orc_candidate(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL, NULL);
                 uint64_t idx = pc->offset + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
+                if (costs) costs[idx] = res.T_iter;              /* indexed by candidate, whole space */
+                if (bottlenecks) bottlenecks[idx] = res.bottleneck;
                 if (res.T_iter < lbest) { lbest = res.T_iter; lidx = idx; }
                 done++;
             }

@@ -122,5 +122,6 @@ int orc_eval_index(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf
 int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t first, uint64_t count,
                int64_t *costs, int64_t *bottlenecks, orc_plan *best, uint64_t *n_feasible);
 int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
-                      uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index);
+                      uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
+                      int64_t *costs, int64_t *bottlenecks);
 #endif

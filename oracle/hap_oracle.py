@@ -243,14 +243,20 @@ class Oracle:
         assert rc == 0
         return costs, bn, (plan_to_dict(best) if best.res.T_iter < INF else None), int(feas.value)
 
-    def search_pconfs(self, p_first: int = 0, p_stride: int = 1, threads: int = 1):
-        """Timing harness: all candidates of every `p_stride`-th configuration."""
+    def search_pconfs(self, p_first: int = 0, p_stride: int = 1, threads: int = 1, want_costs: bool = False):
+        """All candidates of every `p_stride`-th configuration, configurations spread over `threads`
+        OpenMP threads.  Returns (n evaluated, best cost, best index[, costs, bottlenecks])."""
         done = C.c_uint64(); bc = C.c_int64(); bi = C.c_uint64()
+        costs = np.full(self.n_cand, -1, np.int64) if want_costs else None
+        bn = np.full(self.n_cand, -1, np.int64) if want_costs else None
         try:
             omp = C.CDLL("libgomp.so.1")
             omp.omp_set_num_threads(C.c_int(threads))
         except OSError:
             pass
         self.L.orc_search_pconfs(C.byref(self.s), _ptr(self.pconfs), C.c_uint64(self.n_pconf), C.c_uint64(p_first),
-                                 C.c_uint64(p_stride), C.byref(done), C.byref(bc), C.byref(bi))
+                                 C.c_uint64(p_stride), C.byref(done), C.byref(bc), C.byref(bi),
+                                 _ptr(costs) if want_costs else None, _ptr(bn) if want_costs else None)
+        if want_costs:
+            return int(done.value), int(bc.value), int(bi.value), costs, bn
         return int(done.value), int(bc.value), int(bi.value)

@@ -1,0 +1,276 @@
+"""ctypes binding of libhap.so: same names as the C ABI, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+from .build import LIB
+
+MAX_TYPES, MAX_PP, MAX_LAYERS, NCOEF = 4, 32, 255, 20
+INF = 1 << 62
+COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, SBW=9, OPT=11,
+            MW=13, MA=15, MX=17, MPRE=18, MPOST=19)
+STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE", "HAP_E_STATE", "HAP_E_INFEASIBLE"]
+EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
+           "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_search_range",
+           "hap_search_best", "hap_argmin", "hap_status_str", "hap_last_error"]
+
+
+class HapError(RuntimeError):
+    def __init__(self, status: int, msg: str = ""):
+        self.status = status
+        self.name = STATUS[status] if 0 <= status < len(STATUS) else f"status {status}"
+        super().__init__(f"{self.name}: {msg}" if msg else self.name)
+
+
+class _Model(C.Structure):
+    _fields_ = [*[(n, C.c_int32) for n in ("N", "S", "H", "E", "k", "n_shared", "F_dense", "F_exp", "nq", "nkv", "V", "GB")],
+                ("beta", C.c_double), ("kind", C.c_void_p)]
+
+
+class _Cluster(C.Structure):
+    _fields_ = [("n_types", C.c_int32), ("P", C.c_void_p), ("C", C.c_void_p), ("node_size", C.c_void_p),
+                ("bw_intra", C.c_void_p), ("n_nodes", C.c_int32), ("node_type", C.c_void_p), ("node_bw_inter", C.c_void_p)]
+
+
+class _Profile(C.Structure):
+    _fields_ = [("ntp", C.c_int32), ("ncp", C.c_int32), ("nmb", C.c_int32), ("nep", C.c_int32),
+                ("tp_list", C.c_void_p), ("cp_list", C.c_void_p), ("mb_list", C.c_void_p), ("ep_list", C.c_void_p),
+                ("tdf", C.c_void_p), ("tdb", C.c_void_p), ("tff", C.c_void_p), ("tfb", C.c_void_p),
+                ("tpre", C.c_void_p), ("tpost", C.c_void_p), ("eta", C.c_void_p), ("croute", C.c_void_p),
+                ("kappa", C.c_double), ("alpha", C.c_void_p), ("chi", C.c_double), ("rho", C.c_void_p),
+                ("gamma", C.c_double), ("ovl_tp", C.c_double), ("ovl_cp", C.c_double), ("ovl_dp", C.c_double),
+                ("act_coef", C.c_void_p), ("capf", C.c_double), ("copt", C.c_void_p), ("cap_eff", C.c_void_p),
+                ("R", C.c_int32), ("xi_q", C.c_void_p), ("tau_q", C.c_void_p)]
+
+
+class _Opts(C.Structure):
+    _fields_ = [("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
+                ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64), ("n_rc", C.c_int32),
+                ("rc_masks", C.c_void_p), ("prune", C.c_int32)]
+
+
+class _Plan(C.Structure):
+    _fields_ = [("index", C.c_uint64), *[(n, C.c_int32) for n in ("PP", "TP", "CP", "DP", "EP", "TPE", "b", "M")],
+                ("rc_mask", C.c_uint32), ("pad", C.c_uint32), ("n", C.c_uint8 * MAX_PP), ("mask", C.c_uint8 * MAX_PP),
+                ("r", C.c_uint8 * MAX_PP), ("T_iter", C.c_int64), ("bottleneck", C.c_int64), ("T_pipe", C.c_int64),
+                ("T_sync", C.c_int64), ("T_opt", C.c_int64)]
+
+
+class _Stats(C.Structure):
+    _fields_ = [("n_pconf", C.c_uint64), ("n_candidates", C.c_uint64), ("n_evaluated", C.c_uint64),
+                ("n_pruned", C.c_uint64), ("n_feasible", C.c_uint64), ("ms_layer_cost", C.c_float),
+                ("ms_dp", C.c_float), ("ms_total", C.c_float)]
+
+
+PCONF_DTYPE = np.dtype([(n, np.int32) for n in ("PP", "TP", "CP", "DP", "EP", "TPE", "b", "M", "EDP", "G",
+                                                "itp", "icp", "ib", "iep", "mode", "reserved")]
+                       + [("nmap", np.uint64), ("offset", np.uint64)])
+CANDIDATE_DTYPE = np.dtype([("index", np.uint64), ("pconf", np.uint32), ("rc_mask", np.uint32), ("map_idx", np.uint64),
+                            ("PP", np.uint8), ("pad", np.uint8, (7,)), ("mask", np.uint8, (MAX_PP,)),
+                            ("link", np.uint8, (MAX_PP,))])
+
+_lib = None
+
+
+def load_library():
+    """Loads libhap.so; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB):
+            raise HapError(5, f"{LIB} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
+        L = C.CDLL(LIB)
+        L.hap_status_str.restype = C.c_char_p
+        L.hap_last_error.restype = C.c_char_p
+        L.hap_last_error.argtypes = [C.c_void_p]
+        L.hap_problem_destroy.restype = None
+        L.hap_problem_destroy.argtypes = [C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _dev(t) -> C.c_void_p:
+    """Device pointer of a CUDA torch tensor (or None)."""
+    if t is None:
+        return C.c_void_p(0)
+    assert t.is_cuda and t.is_contiguous()
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+class HapProblem:
+    """Owner of a hap_problem* handle."""
+
+    def __init__(self, handle: int, pb):
+        self.h = C.c_void_p(handle)
+        self.N, self.T = int(pb.N), int(pb.P.shape[0])
+        self.n_pconf = self.n_cand = None
+
+    def check(self, status: int):
+        if status != 0:
+            msg = load_library().hap_last_error(self.h)
+            raise HapError(status, msg.decode() if msg else "")
+
+    def close(self):
+        if self.h:
+            load_library().hap_problem_destroy(self.h)
+            self.h = C.c_void_p(0)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def hap_problem_create(pb, prune: int = 0) -> HapProblem:
+    """Marshals a plain-data problem (see gen.problems.Problem) into the C descriptors."""
+    L = load_library()
+    keep = []
+
+    def arr(name, dtype):
+        a = np.ascontiguousarray(np.asarray(getattr(pb, name), dtype=dtype))
+        keep.append(a)
+        return _ptr(a)
+
+    mo = _Model()
+    for n in ("N", "S", "H", "E", "k", "n_shared", "F_dense", "F_exp", "nq", "nkv", "V", "GB"):
+        setattr(mo, n, int(getattr(pb, n)))
+    mo.beta = float(pb.beta)
+    mo.kind = arr("kind", np.uint8)
+    cl = _Cluster()
+    cl.n_types = int(pb.P.shape[0])
+    cl.P, cl.C, cl.node_size = arr("P", np.int64), arr("C", np.int64), arr("node_size", np.int32)
+    cl.bw_intra = arr("bw_intra", np.float64)
+    cl.n_nodes = int(pb.node_type.shape[0])
+    cl.node_type, cl.node_bw_inter = arr("node_type", np.int32), arr("node_bw_inter", np.float64)
+    pf = _Profile()
+    pf.ntp, pf.ncp, pf.nmb, pf.nep = len(pb.tp_list), len(pb.cp_list), len(pb.mb_list), len(pb.ep_list)
+    for n in ("tp_list", "cp_list", "mb_list", "ep_list", "xi_q", "tau_q"):
+        setattr(pf, n, arr(n, np.int32))
+    for n in ("tdf", "tdb", "tff", "tfb", "tpre", "tpost", "eta", "croute", "alpha", "rho", "act_coef", "copt"):
+        setattr(pf, n, arr(n, np.float64))
+    for n in ("kappa", "chi", "gamma", "ovl_tp", "ovl_cp", "ovl_dp", "capf"):
+        setattr(pf, n, float(getattr(pb, n)))
+    pf.cap_eff = arr("cap_eff", np.int64)
+    pf.R = len(pb.xi_q)
+    so = _Opts()
+    so.npp, so.ntpe = len(pb.pp_list), len(pb.tpe_list)
+    so.pp_list, so.tpe_list = arr("pp_list", np.int32), arr("tpe_list", np.int32)
+    so.tp_max, so.delta_q, so.map_cap = int(pb.tp_max), int(pb.delta_q), int(pb.map_cap)
+    so.n_rc = len(pb.rc_masks)
+    so.rc_masks = arr("rc_masks", np.uint32)
+    so.prune = int(prune)
+    out = C.c_void_p(0)
+    st = L.hap_problem_create(C.byref(mo), C.byref(cl), C.byref(pf), C.byref(so), C.byref(out))
+    if st != 0:
+        raise HapError(st, "hap_problem_create")
+    return HapProblem(out.value, pb)
+
+
+def hap_problem_destroy(hp: HapProblem):
+    hp.close()
+
+
+def hap_enumerate(hp: HapProblem):
+    a, b = C.c_uint64(), C.c_uint64()
+    hp.check(load_library().hap_enumerate(hp.h, C.byref(a), C.byref(b)))
+    hp.n_pconf, hp.n_cand = int(a.value), int(b.value)
+    return hp.n_pconf, hp.n_cand
+
+
+def hap_get_pconfs(hp: HapProblem) -> np.ndarray:
+    out = np.zeros(hp.n_pconf, PCONF_DTYPE)
+    hp.check(load_library().hap_get_pconfs(hp.h, _ptr(out), C.c_uint64(hp.n_pconf)))
+    return out
+
+
+def hap_decode(hp: HapProblem, first: int, count: int, stream=None) -> np.ndarray:
+    import torch
+    buf = torch.empty(max(count, 1) * CANDIDATE_DTYPE.itemsize, dtype=torch.uint8, device="cuda")
+    hp.check(load_library().hap_decode(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(buf), _stream(stream)))
+    torch.cuda.current_stream().synchronize()
+    return np.frombuffer(buf.cpu().numpy().tobytes(), dtype=CANDIDATE_DTYPE)[:count]
+
+
+def hap_eval_layer_costs(hp: HapProblem, c2=None, coef=None, stream=None, want_c2=True, want_coef=True):
+    """Returns (c2 [n_pconf][T][N][2], coef [n_pconf][T][NCOEF]) int64 CUDA tensors."""
+    import torch
+    if c2 is None and want_c2:
+        c2 = torch.empty((hp.n_pconf, hp.T, hp.N, 2), dtype=torch.int64, device="cuda")
+    if coef is None and want_coef:
+        coef = torch.empty((hp.n_pconf, hp.T, NCOEF), dtype=torch.int64, device="cuda")
+    hp.check(load_library().hap_eval_layer_costs(hp.h, _dev(c2), _dev(coef), _stream(stream)))
+    return c2, coef
+
+
+def hap_eval_layer_costs_f64(hp: HapProblem, stream=None):
+    import torch
+    c2 = torch.empty((hp.n_pconf, hp.T, hp.N, 2), dtype=torch.float64, device="cuda")
+    coef = torch.empty((hp.n_pconf, hp.T, NCOEF), dtype=torch.float64, device="cuda")
+    hp.check(load_library().hap_eval_layer_costs_f64(hp.h, _dev(c2), _dev(coef), _stream(stream)))
+    return c2, coef
+
+
+def hap_pipeline_dp(hp: HapProblem, first: int, count: int, *, partition=False, tables=False, stream=None, out=None):
+    """Evaluates candidates [first, first+count).  Returns a dict of CUDA tensors."""
+    import torch
+    o = out or {}
+    if "cost" not in o:
+        o["cost"] = torch.empty(count, dtype=torch.int64, device="cuda")
+        o["bottleneck"] = torch.empty(count, dtype=torch.int64, device="cuda")
+        if partition:
+            o["partition"] = torch.empty((count, MAX_PP), dtype=torch.uint8, device="cuda")
+            o["recompute"] = torch.empty((count, MAX_PP), dtype=torch.uint8, device="cuda")
+        if tables:
+            o["dp_table"] = torch.full((count, MAX_PP + 1, hp.N + 1), -1, dtype=torch.int64, device="cuda")
+            o["choice"] = torch.full((count, MAX_PP + 1, hp.N + 1), 254, dtype=torch.uint8, device="cuda")
+    hp.check(load_library().hap_pipeline_dp(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(o["cost"]),
+                                            _dev(o["bottleneck"]), _dev(o.get("partition")), _dev(o.get("recompute")),
+                                            _dev(o.get("dp_table")), _dev(o.get("choice")), _stream(stream)))
+    return o
+
+
+def _plan_dict(pl: _Plan) -> dict:
+    PP = pl.PP
+    return dict(index=int(pl.index), **{n: int(getattr(pl, n)) for n in ("PP", "TP", "CP", "DP", "EP", "TPE", "b", "M")},
+                rc_mask=int(pl.rc_mask), n=[int(x) for x in pl.n[:PP]], mask=[int(x) for x in pl.mask[:PP]],
+                r=[int(x) for x in pl.r[:PP]], T_iter=int(pl.T_iter), bottleneck=int(pl.bottleneck),
+                T_pipe=int(pl.T_pipe), T_sync=int(pl.T_sync), T_opt=int(pl.T_opt))
+
+
+def _stats_dict(st: _Stats) -> dict:
+    return {n: (float(getattr(st, n)) if n.startswith("ms_") else int(getattr(st, n))) for n, _ in _Stats._fields_}
+
+
+def hap_search_range(hp: HapProblem, first: int, count: int, stream=None):
+    pl, st = _Plan(), _Stats()
+    hp.check(load_library().hap_search_range(hp.h, C.c_uint64(first), C.c_uint64(count), C.byref(pl), C.byref(st),
+                                             _stream(stream)))
+    return _plan_dict(pl), _stats_dict(st)
+
+
+def hap_search_best(hp: HapProblem, stream=None):
+    pl, st = _Plan(), _Stats()
+    hp.check(load_library().hap_search_best(hp.h, C.byref(pl), C.byref(st), _stream(stream)))
+    return _plan_dict(pl), _stats_dict(st)
+
+
+def hap_argmin(hp: HapProblem, cost, stream=None):
+    """(cost, index) minimum of an int64 CUDA tensor, lowest index on ties; returns a 2-element CUDA tensor."""
+    import torch
+    out = torch.empty(2, dtype=torch.int64, device="cuda")
+    hp.check(load_library().hap_argmin(hp.h, _dev(cost), C.c_uint64(cost.numel()), _dev(out), _stream(stream)))
+    return out

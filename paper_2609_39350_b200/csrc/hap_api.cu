@@ -1,0 +1,556 @@
+// Host side of libhap: descriptor validation and copies, enumeration of the 6-D space,
+// work partitioning, kernel launches.  Every step of the hot path runs in the kernels of
+// hap_device.cuh; nothing here evaluates a cost.
+#include "hap_device.cuh"
+
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace hap;
+
+struct hap_problem {
+    int device = 0;
+    // host copies
+    hap_model model{};
+    std::vector<uint8_t> kind;
+    int T = 0;
+    std::vector<int64_t> P, C, cap_eff;
+    std::vector<int32_t> node_size, node_type, tp_list, cp_list, mb_list, ep_list, pp_list, tpe_list, xi_q, tau_q;
+    std::vector<double> bw_intra, node_bw_inter, eta, croute, alpha, rho, act_coef, copt;
+    std::vector<uint32_t> rc_masks;
+    hap_profile prof{};
+    hap_search_opts opts{};
+    int64_t m[HAP_MAX_TYPES] = {0, 0, 0, 0};
+    int64_t W = 0;
+    // enumeration
+    bool enumerated = false;
+    std::vector<hap_pconf> pconfs;
+    uint64_t n_cand = 0;
+    int pp_max = 1;
+    std::vector<WorkItem> items;           // sorted by descending work per candidate
+    // device
+    DevConst dc{};
+    double *d_tables = nullptr;            // all six tables in one allocation
+    hap_pconf *d_pconf = nullptr;
+    WorkItem *d_items = nullptr;
+    i64 *d_c2 = nullptr, *d_coef = nullptr;
+    i64 *d_pcost = nullptr;                // per-block partial minima
+    u64 *d_pindex = nullptr;
+    u64 *d_counters = nullptr;             // [0] evaluated [1] feasible [2] pruned [3] incumbent
+    i64 *d_best = nullptr;                 // (cost, index) of the search
+    void *d_single = nullptr;              // outputs of the one-candidate re-evaluation
+    size_t n_partial = 0;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    std::string err;
+};
+
+// device-side landing area of the one-candidate re-evaluation that fills the plan
+struct SingleOut {
+    i64 cost, bott, detail[3];
+    uint8_t part[HAP_MAX_PP], rec[HAP_MAX_PP];
+    hap_candidate cand;
+};
+
+static hap_status fail(hap_problem *p, hap_status s, const char *fmt, ...)
+{
+    if (p) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof(buf), fmt, ap);
+        va_end(ap);
+        p->err = buf;
+    }
+    return s;
+}
+
+#define CUDA_TRY(p, call)                                                                          \
+    do {                                                                                           \
+        cudaError_t e_ = (call);                                                                   \
+        if (e_ != cudaSuccess)                                                                     \
+            return fail(p, e_ == cudaErrorMemoryAllocation ? HAP_E_NOMEM : HAP_E_CUDA, "%s: %s", #call, \
+                        cudaGetErrorString(e_));                                                   \
+    } while (0)
+
+extern "C" const char *hap_status_str(hap_status s)
+{
+    switch (s) {
+    case HAP_OK: return "HAP_OK";
+    case HAP_E_INVALID: return "HAP_E_INVALID";
+    case HAP_E_NOMEM: return "HAP_E_NOMEM";
+    case HAP_E_CUDA: return "HAP_E_CUDA";
+    case HAP_E_RANGE: return "HAP_E_RANGE";
+    case HAP_E_STATE: return "HAP_E_STATE";
+    case HAP_E_INFEASIBLE: return "HAP_E_INFEASIBLE";
+    }
+    return "HAP_E_?";
+}
+
+extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.c_str() : "null problem"; }
+
+static void release_device(hap_problem *p)
+{
+    cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
+    cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
+    for (auto &e : p->ev) if (e) cudaEventDestroy(e);
+}
+
+extern "C" void hap_problem_destroy(hap_problem *p)
+{
+    if (!p) return;
+    cudaSetDevice(p->device);
+    release_device(p);
+    delete p;
+}
+
+template <class T>
+static bool copy_list(std::vector<T> &dst, const T *src, int n)
+{
+    if (n < 0 || (n > 0 && !src)) return false;
+    dst.assign(src, src + n);
+    return true;
+}
+
+static bool finite_nonneg(const std::vector<double> &v)
+{
+    for (double x : v) if (!(x >= 0.0) || x > 1e300) return false;
+    return true;
+}
+
+extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster *cl, const hap_profile *pf,
+                                         const hap_search_opts *so, hap_problem **out)
+{
+    if (!out) return HAP_E_INVALID;
+    *out = nullptr;
+    if (!mo || !cl || !pf || !so) return HAP_E_INVALID;
+    hap_problem *p = new (std::nothrow) hap_problem();
+    if (!p) return HAP_E_NOMEM;
+    // the problem is handed back even on failure paths below only through *out on success
+    struct Guard { hap_problem *p; bool keep = false; ~Guard() { if (!keep) { release_device(p); delete p; } } } guard{p};
+
+    // ---- validate and copy ------------------------------------------------------------------
+    const int N = mo->N, T = cl->n_types;
+    if (N < 1 || N > HAP_MAX_LAYERS || !mo->kind) return HAP_E_INVALID;
+    if (T < 1 || T > HAP_MAX_TYPES || cl->n_nodes < 1) return HAP_E_INVALID;
+    if (mo->S < 1 || mo->H < 1 || mo->E < 1 || mo->k < 1 || mo->nq < 1 || mo->nkv < 1 || mo->GB < 1 || mo->V < 0 ||
+        mo->n_shared < 0 || mo->F_dense < 0 || mo->F_exp < 0 || !(mo->beta > 0.0) || mo->nq % mo->nkv != 0)
+        return HAP_E_INVALID;
+    if (pf->ntp < 1 || pf->ncp < 1 || pf->nmb < 1 || pf->nep < 1 || pf->ntp > HAP_MAX_LIST || pf->ncp > HAP_MAX_LIST ||
+        pf->nmb > HAP_MAX_LIST || pf->nep > HAP_MAX_LIST || pf->R < 1 || pf->R > HAP_MAX_RC)
+        return HAP_E_INVALID;
+    if (so->npp < 1 || so->npp > HAP_MAX_LIST || so->ntpe < 1 || so->ntpe > HAP_MAX_LIST || so->n_rc < 1 ||
+        so->n_rc > HAP_MAX_RC_MASKS || so->map_cap < 1 || so->map_cap > (1ull << 56) || so->delta_q >= 1024)
+        return HAP_E_INVALID;
+    p->model = *mo;
+    p->kind.assign(mo->kind, mo->kind + N);
+    p->model.kind = nullptr;
+    for (uint8_t kd : p->kind) if (kd > 1) return HAP_E_INVALID;
+    p->T = T;
+    bool ok = copy_list(p->P, cl->P, T) && copy_list(p->C, cl->C, T) && copy_list(p->node_size, cl->node_size, T) &&
+              copy_list(p->bw_intra, cl->bw_intra, T) && copy_list(p->node_type, cl->node_type, cl->n_nodes) &&
+              copy_list(p->node_bw_inter, cl->node_bw_inter, cl->n_nodes) &&
+              copy_list(p->tp_list, pf->tp_list, pf->ntp) && copy_list(p->cp_list, pf->cp_list, pf->ncp) &&
+              copy_list(p->mb_list, pf->mb_list, pf->nmb) && copy_list(p->ep_list, pf->ep_list, pf->nep) &&
+              copy_list(p->eta, pf->eta, T) && copy_list(p->croute, pf->croute, T) && copy_list(p->alpha, pf->alpha, 3) &&
+              copy_list(p->rho, pf->rho, pf->nep) && copy_list(p->act_coef, pf->act_coef, 2) &&
+              copy_list(p->copt, pf->copt, T) && copy_list(p->cap_eff, pf->cap_eff, T) &&
+              copy_list(p->xi_q, pf->xi_q, pf->R) && copy_list(p->tau_q, pf->tau_q, pf->R) &&
+              copy_list(p->pp_list, so->pp_list, so->npp) && copy_list(p->tpe_list, so->tpe_list, so->ntpe) &&
+              copy_list(p->rc_masks, so->rc_masks, so->n_rc);
+    if (!ok || !pf->tdf || !pf->tdb || !pf->tff || !pf->tfb || !pf->tpre || !pf->tpost) return HAP_E_INVALID;
+    p->prof = *pf;
+    p->opts = *so;
+    for (int h = 0; h < T; ++h) {
+        if (p->P[h] < 1 || p->P[h] > (1ll << 40) || p->node_size[h] < 1 || !(p->bw_intra[h] > 0.0) || p->cap_eff[h] < 0 ||
+            !(p->eta[h] > 0.0))
+            return HAP_E_INVALID;
+    }
+    double bw_inter[HAP_MAX_TYPES];
+    bool has[HAP_MAX_TYPES] = {false, false, false, false};
+    for (int n = 0; n < cl->n_nodes; ++n) {
+        const int t = p->node_type[n];
+        if (t < 0 || t >= T || !(p->node_bw_inter[n] > 0.0)) return HAP_E_INVALID;
+        p->m[t] += p->node_size[t];
+        bw_inter[t] = has[t] ? std::min(bw_inter[t], p->node_bw_inter[n]) : p->node_bw_inter[n];
+        has[t] = true;
+    }
+    for (int h = 0; h < T; ++h) { if (!has[h]) return HAP_E_INVALID; p->W += p->m[h]; }
+    auto positive = [](const std::vector<int32_t> &v) { for (int x : v) if (x < 1) return false; return true; };
+    if (!positive(p->tp_list) || !positive(p->cp_list) || !positive(p->mb_list) || !positive(p->ep_list) ||
+        !positive(p->pp_list) || !positive(p->tpe_list))
+        return HAP_E_INVALID;
+    for (int r = 0; r < pf->R; ++r) if (p->xi_q[r] < 0 || p->tau_q[r] < 0 || p->xi_q[r] > (1 << 20) || p->tau_q[r] > (1 << 20)) return HAP_E_INVALID;
+    for (uint32_t mk : p->rc_masks) if (mk == 0 || mk >= (1u << pf->R)) return HAP_E_INVALID;
+    if (!finite_nonneg(p->croute) || !finite_nonneg(p->alpha) || !finite_nonneg(p->act_coef) || !finite_nonneg(p->copt) ||
+        !(pf->kappa >= 0.0) || !(pf->chi > 0.0) || !(pf->gamma >= 0.0) || !(pf->ovl_tp >= 0.0) || !(pf->ovl_cp >= 0.0) ||
+        !(pf->ovl_dp >= 0.0) || !(pf->capf >= 0.0))
+        return HAP_E_INVALID;
+    for (double r : p->rho) if (!(r >= 1.0)) return HAP_E_INVALID;
+
+    const size_t n4 = (size_t)T * pf->ntp * pf->ncp * pf->nmb, n5 = n4 * N;
+    std::vector<double> tables(4 * n5 + 2 * n4);
+    const double *srcs[6] = {pf->tdf, pf->tdb, pf->tff, pf->tfb, pf->tpre, pf->tpost};
+    size_t at = 0;
+    for (int t = 0; t < 6; ++t) {
+        const size_t n = t < 4 ? n5 : n4;
+        std::memcpy(tables.data() + at, srcs[t], n * sizeof(double));
+        at += n;
+    }
+    for (double x : tables) if (!(x >= 0.0) || x > 1e15) return HAP_E_INVALID;   // finite, non-negative, < 2^50 ns
+    for (size_t i = 0; i < n5; ++i)                                              // t_dense includes its FFN
+        if (tables[i] < tables[2 * n5 + i] || tables[n5 + i] < tables[3 * n5 + i]) return HAP_E_INVALID;
+
+    // ---- device ------------------------------------------------------------------------------
+    if (cudaGetDevice(&p->device) != cudaSuccess) return HAP_E_CUDA;
+    if (cudaMalloc(&p->d_tables, tables.size() * sizeof(double)) != cudaSuccess) return HAP_E_NOMEM;
+    if (cudaMemcpy(p->d_tables, tables.data(), tables.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess)
+        return HAP_E_CUDA;
+    for (auto &e : p->ev) if (cudaEventCreate(&e) != cudaSuccess) return HAP_E_CUDA;
+
+    DevConst &dc = p->dc;
+    std::memset(&dc, 0, sizeof(dc));
+    dc.N = N; dc.T = T; dc.R = pf->R; dc.n_rc = so->n_rc; dc.ntp = pf->ntp; dc.ncp = pf->ncp; dc.nmb = pf->nmb; dc.nep = pf->nep;
+    dc.S = mo->S; dc.H = mo->H; dc.E = mo->E; dc.k = mo->k; dc.n_shared = mo->n_shared; dc.F_dense = mo->F_dense;
+    dc.F_exp = mo->F_exp; dc.nq = mo->nq; dc.nkv = mo->nkv; dc.V = mo->V; dc.GB = mo->GB; dc.delta_q = so->delta_q;
+    dc.beta = mo->beta; dc.kappa = pf->kappa; dc.chi = pf->chi; dc.gamma = pf->gamma; dc.ovl_tp = pf->ovl_tp;
+    dc.ovl_cp = pf->ovl_cp; dc.ovl_dp = pf->ovl_dp; dc.capf = pf->capf;
+    for (int i = 0; i < 3; ++i) dc.alpha[i] = p->alpha[i];
+    for (int h = 0; h < T; ++h) {
+        dc.eta[h] = p->eta[h]; dc.croute[h] = p->croute[h]; dc.copt[h] = p->copt[h]; dc.bw_intra[h] = p->bw_intra[h];
+        dc.bw_inter[h] = bw_inter[h]; dc.P[h] = p->P[h]; dc.cap_eff[h] = p->cap_eff[h]; dc.m[h] = p->m[h];
+        dc.node_size[h] = p->node_size[h];
+    }
+    dc.act_coef[0] = p->act_coef[0]; dc.act_coef[1] = p->act_coef[1];
+    for (int i = 0; i < pf->nep; ++i) dc.rho[i] = p->rho[i];
+    for (int i = 0; i < so->n_rc; ++i) dc.rc_masks[i] = p->rc_masks[i];
+    dc.tau_linear = 1;
+    for (int r = 0; r < pf->R; ++r) { dc.xi_q[r] = p->xi_q[r]; dc.tau_q[r] = p->tau_q[r]; if (p->tau_q[r] % 1024) dc.tau_linear = 0; }
+    for (int l = 0; l < N; ++l) if (p->kind[l] == HAP_MOE) dc.kindbits[l >> 6] |= 1ull << (l & 63);
+    dc.tdf = p->d_tables; dc.tdb = dc.tdf + n5; dc.tff = dc.tdb + n5; dc.tfb = dc.tff + n5;
+    dc.tpre = dc.tfb + n5; dc.tpost = dc.tpre + n4;
+
+    guard.keep = true;
+    *out = p;
+    return HAP_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// enumeration (host; at most a few thousand rows)
+// ------------------------------------------------------------------------------------------
+static uint64_t binom_sat(int n, int k, uint64_t sat)
+{
+    if (k < 0 || k > n) return 0;
+    if (k > n - k) k = n - k;
+    unsigned __int128 r = 1;
+    for (int i = 1; i <= k; ++i) {
+        r = r * (unsigned)(n - k + i) / (unsigned)i;
+        if (r > sat) return sat;
+    }
+    return (uint64_t)r;
+}
+
+// distinct sequences with cnt[h] stages of type h: product of binomials, saturating
+static uint64_t sequences_sat(const int *cnt, int T, uint64_t sat)
+{
+    int rem = 0;
+    for (int h = 0; h < T; ++h) rem += cnt[h];
+    unsigned __int128 r = 1;
+    for (int h = 0; h < T; ++h) {
+        r *= binom_sat(rem, cnt[h], sat);
+        if (r > sat) return sat;
+        rem -= cnt[h];
+    }
+    return (uint64_t)r;
+}
+
+static double cells_per_candidate(int N, int PP)
+{
+    if (PP == 1) return 1.0;
+    const double w = N - PP + 1;
+    return 2.0 * w + (PP - 2) * w * (w + 1) / 2.0;
+}
+
+extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t *n_candidates)
+{
+    if (!p) return HAP_E_INVALID;
+    if (cudaSetDevice(p->device) != cudaSuccess) return fail(p, HAP_E_CUDA, "cudaSetDevice");
+    if (!p->enumerated) {
+        const hap_model &mo = p->model;
+        const int N = mo.N, T = p->T;
+        std::vector<hap_pconf> rows;
+        uint64_t off = 0;
+        int pp_max = 1;
+        const uint64_t SAT = 1ull << 62;
+        for (int PP : p->pp_list) {
+            if (PP > N || PP > HAP_MAX_PP || p->W % PP) continue;
+            const int64_t G = p->W / PP;
+            if (G > 0x7fffffffll) continue;
+            bool homog = true;
+            int cnt[HAP_MAX_TYPES] = {0, 0, 0, 0};
+            for (int h = 0; h < T; ++h) { if (p->m[h] % G) homog = false; cnt[h] = (int)(p->m[h] / G); }
+            const uint64_t nms = homog ? sequences_sat(cnt, T, SAT) : 0;
+            const int mode = (homog && nms <= p->opts.map_cap) ? HAP_MAP_MULTISET : HAP_MAP_BLOCK;
+            uint64_t nmap = nms;
+            if (mode == HAP_MAP_BLOCK) { nmap = 1; for (int i = 2; i <= T; ++i) nmap *= (uint64_t)i; }
+            for (int itp = 0; itp < (int)p->tp_list.size(); ++itp) {
+                const int TP = p->tp_list[itp];
+                if (G % TP || TP > p->opts.tp_max || mo.nq % TP || mo.nkv % TP) continue;
+                for (int icp = 0; icp < (int)p->cp_list.size(); ++icp) {
+                    const int CP = p->cp_list[icp];
+                    if (G % ((int64_t)TP * CP) || mo.S % (2 * CP)) continue;
+                    const int64_t DP = G / ((int64_t)TP * CP);
+                    for (int iep = 0; iep < (int)p->ep_list.size(); ++iep) {
+                        const int EP = p->ep_list[iep];
+                        if (mo.E % EP || G % EP) continue;
+                        for (int TPE : p->tpe_list) {
+                            if (G % ((int64_t)EP * TPE) || TPE > p->opts.tp_max) continue;
+                            const int64_t EDP = G / ((int64_t)EP * TPE);
+                            for (int ib = 0; ib < (int)p->mb_list.size(); ++ib) {
+                                const int b = p->mb_list[ib];
+                                if (mo.GB % (DP * b)) continue;
+                                hap_pconf q{};
+                                q.PP = PP; q.TP = TP; q.CP = CP; q.DP = (int)DP; q.EP = EP; q.TPE = TPE; q.b = b;
+                                q.M = (int)(mo.GB / (DP * b)); q.EDP = (int)EDP; q.G = (int)G;
+                                q.itp = itp; q.icp = icp; q.ib = ib; q.iep = iep; q.mode = mode; q.reserved = 0;
+                                q.nmap = nmap; q.offset = off;
+                                if (nmap > (SAT - off) / (uint64_t)p->opts.n_rc) return fail(p, HAP_E_RANGE, "candidate space overflows 2^62");
+                                off += nmap * (uint64_t)p->opts.n_rc;
+                                rows.push_back(q);
+                                pp_max = std::max(pp_max, PP);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        if (rows.empty()) return fail(p, HAP_E_INFEASIBLE, "no parallel configuration divides the cluster");
+        if (rows.size() > 0xffffffffull) return fail(p, HAP_E_RANGE, "too many configurations");
+
+        // work items: chunks of one configuration's candidates with about equal recurrence work,
+        // heaviest candidates first so that the tail of the grid is made of light blocks
+        std::vector<WorkItem> items;
+        const double target = 8.0 * 4.0 * cells_per_candidate(N, std::min(pp_max, 8)) + 4096.0;
+        for (size_t pi = 0; pi < rows.size(); ++pi) {
+            const uint64_t total = rows[pi].nmap * (uint64_t)p->opts.n_rc;
+            const double per = cells_per_candidate(N, rows[pi].PP) + 64.0;
+            uint64_t chunk = (uint64_t)std::max(1.0, target / per);
+            chunk = std::max<uint64_t>(chunk, kDpWarps);
+            chunk = std::min<uint64_t>(chunk, 1u << 20);
+            for (uint64_t lo = 0; lo < total; lo += chunk) {
+                WorkItem it; it.p = (uint32_t)pi; it.lo = lo; it.count = (uint32_t)std::min<uint64_t>(chunk, total - lo);
+                items.push_back(it);
+            }
+        }
+        std::stable_sort(items.begin(), items.end(), [&](const WorkItem &a, const WorkItem &b) {
+            return rows[a.p].PP > rows[b.p].PP;
+        });
+
+        p->pconfs.swap(rows);
+        p->items.swap(items);
+        p->n_cand = off;
+        p->pp_max = pp_max;
+        const size_t np = p->pconfs.size();
+        CUDA_TRY(p, cudaMalloc(&p->d_pconf, np * sizeof(hap_pconf)));
+        CUDA_TRY(p, cudaMemcpy(p->d_pconf, p->pconfs.data(), np * sizeof(hap_pconf), cudaMemcpyHostToDevice));
+        CUDA_TRY(p, cudaMalloc(&p->d_items, p->items.size() * sizeof(WorkItem)));
+        CUDA_TRY(p, cudaMemcpy(p->d_items, p->items.data(), p->items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
+        CUDA_TRY(p, cudaMalloc(&p->d_c2, np * T * N * 2 * sizeof(i64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_coef, np * T * HAP_NCOEF * sizeof(i64)));
+        p->n_partial = std::max<size_t>(p->items.size(), 1024);
+        CUDA_TRY(p, cudaMalloc(&p->d_pcost, p->n_partial * sizeof(i64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_pindex, p->n_partial * sizeof(u64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_counters, 8 * sizeof(u64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_best, 2 * sizeof(i64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_single, sizeof(SingleOut)));
+        p->dc.pconf = p->d_pconf;
+        p->dc.n_pconf = np;
+        const size_t smem = dp_smem_bytes(N, pp_max);
+        if (smem > 227 * 1024) return fail(p, HAP_E_RANGE, "shared memory need %zu exceeds the SM", smem);
+        CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        p->enumerated = true;
+    }
+    if (n_pconf) *n_pconf = p->pconfs.size();
+    if (n_candidates) *n_candidates = p->n_cand;
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_get_pconfs(const hap_problem *p, hap_pconf *host_out, uint64_t cap)
+{
+    if (!p || !host_out) return HAP_E_INVALID;
+    if (!p->enumerated) return HAP_E_STATE;
+    if (cap < p->pconfs.size()) return HAP_E_RANGE;
+    std::memcpy(host_out, p->pconfs.data(), p->pconfs.size() * sizeof(hap_pconf));
+    return HAP_OK;
+}
+
+static hap_status enter(hap_problem *p)
+{
+    if (!p) return HAP_E_INVALID;
+    if (!p->enumerated) return fail(p, HAP_E_STATE, "hap_enumerate has not run");
+    if (cudaSetDevice(p->device) != cudaSuccess) return fail(p, HAP_E_CUDA, "cudaSetDevice");
+    return HAP_OK;
+}
+
+static hap_status check_range(hap_problem *p, uint64_t first, uint64_t count)
+{
+    if (first > p->n_cand || count > p->n_cand - first) return fail(p, HAP_E_RANGE, "candidate range outside [0, %llu)", (unsigned long long)p->n_cand);
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_decode(hap_problem *p, uint64_t first, uint64_t count, hap_candidate *dev_out, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    if (count == 0) return HAP_OK;
+    if (!dev_out) return HAP_E_INVALID;
+    const uint64_t blocks = (count + 3) / 4;
+    if (blocks > 0x7fffffffull) return fail(p, HAP_E_RANGE, "count too large for one launch");
+    decode_kernel<<<(unsigned)blocks, 128, 0, (cudaStream_t)stream>>>(p->dc, first, count, dev_out);
+    CUDA_TRY(p, cudaGetLastError());
+    return HAP_OK;
+}
+
+static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st)
+{
+    const unsigned blocks = (unsigned)((p->pconfs.size() + 3) / 4);
+    if (quant) layer_cost_kernel<true><<<blocks, 128, 0, st>>>(p->dc, c2, coef, nullptr, nullptr);
+    else layer_cost_kernel<false><<<blocks, 128, 0, st>>>(p->dc, nullptr, nullptr, c2f, coeff);
+    CUDA_TRY(p, cudaGetLastError());
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_eval_layer_costs(hap_problem *p, int64_t *dev_c2, int64_t *dev_coef, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!dev_c2 && !dev_coef) return HAP_OK;
+    return launch_layer_costs(p, (i64 *)dev_c2, (i64 *)dev_coef, nullptr, nullptr, true, (cudaStream_t)stream);
+}
+
+extern "C" hap_status hap_eval_layer_costs_f64(hap_problem *p, double *dev_c2, double *dev_coef, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!dev_c2 && !dev_coef) return HAP_OK;
+    return launch_layer_costs(p, nullptr, nullptr, dev_c2, dev_coef, false, (cudaStream_t)stream);
+}
+
+// work items that can intersect the candidate range: all of them (each block clips); the
+// full-range case is the hot one
+static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaStream_t st)
+{
+    const size_t smem = dp_smem_bytes(p->model.N, p->pp_max);
+    const unsigned blocks = (unsigned)p->items.size();
+    if (search) pipeline_dp_kernel<true><<<blocks, kDpWarps * 32, smem, st>>>(p->dc, p->d_items, p->d_c2, p->d_coef, out, p->pp_max);
+    else pipeline_dp_kernel<false><<<blocks, kDpWarps * 32, smem, st>>>(p->dc, p->d_items, p->d_c2, p->d_coef, out, p->pp_max);
+    CUDA_TRY(p, cudaGetLastError());
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t count, int64_t *dev_cost,
+                                      int64_t *dev_bottleneck, uint8_t *dev_partition, uint8_t *dev_recompute,
+                                      int64_t *dev_dp_table, uint8_t *dev_choice, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    if (count == 0) return HAP_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    DpOut out{};
+    out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
+    out.recompute = dev_recompute; out.dp_table = (i64 *)dev_dp_table; out.choice = dev_choice;
+    out.first = first; out.count = count;
+    return launch_dp(p, out, false, st);
+}
+
+extern "C" hap_status hap_argmin(hap_problem *p, const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!dev_cost || !dev_out || count == 0) return HAP_E_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    const unsigned blocks = (unsigned)std::min<uint64_t>((count + 255) / 256, 1024);
+    argmin_partial_kernel<<<blocks, 256, 0, st>>>((const i64 *)dev_cost, count, p->d_pcost, p->d_pindex);
+    CUDA_TRY(p, cudaGetLastError());
+    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, blocks, (i64 *)dev_out);
+    CUDA_TRY(p, cudaGetLastError());
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t count, hap_plan *host_out,
+                                       hap_search_stats *host_stats, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!host_out) return HAP_E_INVALID;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    if (count == 0) return fail(p, HAP_E_RANGE, "empty candidate range");
+    cudaStream_t st = (cudaStream_t)stream;
+    std::memset(host_out, 0, sizeof(*host_out));
+    CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
+    CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
+    DpOut out{};
+    out.first = first; out.count = count; out.search = 1; out.prune = p->opts.prune;
+    out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
+    out.incumbent = p->d_counters + 3;
+    if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
+    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best);
+    CUDA_TRY(p, cudaGetLastError());
+    CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
+    i64 best[2];
+    u64 counters[4];
+    CUDA_TRY(p, cudaMemcpyAsync(best, p->d_best, sizeof(best), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaMemcpyAsync(counters, p->d_counters, sizeof(counters), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaStreamSynchronize(st));
+    if (host_stats) {
+        std::memset(host_stats, 0, sizeof(*host_stats));
+        host_stats->n_pconf = p->pconfs.size(); host_stats->n_candidates = p->n_cand;
+        host_stats->n_evaluated = counters[0]; host_stats->n_feasible = counters[1]; host_stats->n_pruned = counters[2];
+        cudaEventElapsedTime(&host_stats->ms_layer_cost, p->ev[0], p->ev[1]);
+        cudaEventElapsedTime(&host_stats->ms_dp, p->ev[1], p->ev[2]);
+        host_stats->ms_total = host_stats->ms_layer_cost + host_stats->ms_dp;
+    }
+    if (best[0] >= kInf) return fail(p, HAP_E_INFEASIBLE, "no candidate satisfies the memory constraint");
+
+    // re-evaluate the winner alone to obtain its partition and recomputation levels
+    const u64 win = (u64)best[1];
+    SingleOut *d1 = (SingleOut *)p->d_single;
+    DpOut one{};
+    one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
+    one.recompute = d1->rec; one.first = win; one.count = 1;
+    if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
+    decode_kernel<<<1, 32, 0, st>>>(p->dc, win, 1, &d1->cand);
+    CUDA_TRY(p, cudaGetLastError());
+    SingleOut h1;
+    CUDA_TRY(p, cudaMemcpyAsync(&h1, d1, sizeof(h1), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaStreamSynchronize(st));
+    const hap_candidate &hc = h1.cand;
+    if (h1.cost != best[0]) return fail(p, HAP_E_CUDA, "winner re-evaluation disagrees with the search");
+    const hap_pconf &pc = p->pconfs[hc.pconf];
+    host_out->index = win;
+    host_out->PP = pc.PP; host_out->TP = pc.TP; host_out->CP = pc.CP; host_out->DP = pc.DP; host_out->EP = pc.EP;
+    host_out->TPE = pc.TPE; host_out->b = pc.b; host_out->M = pc.M; host_out->rc_mask = hc.rc_mask;
+    std::memcpy(host_out->n, h1.part, HAP_MAX_PP);
+    std::memcpy(host_out->r, h1.rec, HAP_MAX_PP);
+    std::memcpy(host_out->mask, hc.mask, HAP_MAX_PP);
+    host_out->T_iter = h1.cost; host_out->bottleneck = h1.bott;
+    host_out->T_pipe = h1.detail[0]; host_out->T_sync = h1.detail[1]; host_out->T_opt = h1.detail[2];
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_search_best(hap_problem *p, hap_plan *host_out, hap_search_stats *host_stats, void *stream)
+{
+    if (!p) return HAP_E_INVALID;
+    if (!p->enumerated) return fail(p, HAP_E_STATE, "hap_enumerate has not run");
+    return hap_search_range(p, 0, p->n_cand, host_out, host_stats, stream);
+}

@@ -1,0 +1,771 @@
+// Device-side data layout and kernels of libhap (sm_100a).
+//
+// Kernels
+//   layer_cost_kernel   Eq. 2 / Eq. 3 / imbalance scaling and the stage coefficients, one warp
+//                       per configuration, fp64 with one IEEE operation per operator
+//                       (the translation unit is compiled with --fmad=false).
+//   decode_kernel       candidate index -> stage type masks and boundary link classes.
+//   pipeline_dp_kernel  one warp per candidate: stage rows in shared memory (built once per
+//                       block for the block's configuration), min-max recurrence with lanes
+//                       over the end layer j, backtrace, Eq. 4 closed form; optionally the
+//                       block-level (cost, index) minimum for the search.
+//   argmin kernels      lexicographic (cost, index) minimum, block partials then one block.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "../../include/hap.h"
+
+namespace hap {
+
+typedef long long i64;
+typedef unsigned long long u64;
+
+constexpr int kMaxMasks = (1 << HAP_MAX_TYPES) - 1;
+constexpr int kDpWarps = 8;           // warps per block of the DP kernel
+constexpr i64 kInf = (i64)1 << 62;
+
+// Everything a kernel needs besides the big tables; passed by value.
+struct DevConst {
+    int N, T, R, n_rc, ntp, ncp, nmb, nep;
+    int S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
+    int delta_q, tau_linear, pad0;
+    double beta, kappa, chi, gamma, ovl_tp, ovl_cp, ovl_dp, capf;
+    double alpha[3];
+    double eta[HAP_MAX_TYPES], croute[HAP_MAX_TYPES], copt[HAP_MAX_TYPES];
+    double bw_intra[HAP_MAX_TYPES], bw_inter[HAP_MAX_TYPES];
+    double act_coef[2];
+    double rho[HAP_MAX_LIST];
+    i64 P[HAP_MAX_TYPES], cap_eff[HAP_MAX_TYPES], m[HAP_MAX_TYPES];
+    int node_size[HAP_MAX_TYPES];
+    unsigned rc_masks[HAP_MAX_RC_MASKS];
+    int xi_q[HAP_MAX_RC], tau_q[HAP_MAX_RC];
+    u64 kindbits[4];                  // bit l set: layer l is an MoE layer
+    const double *tdf, *tdb, *tff, *tfb, *tpre, *tpost;
+    const hap_pconf *pconf;           // device copy of the configuration table
+    u64 n_pconf;
+};
+
+// One block of DP work: candidates [lo, lo+count) (local to configuration p).
+struct WorkItem {
+    uint32_t p;
+    uint32_t count;
+    u64 lo;
+};
+
+struct DpOut {
+    i64 *cost, *bottleneck;
+    uint8_t *partition, *recompute;
+    i64 *dp_table;
+    uint8_t *choice;
+    i64 *detail;                      // [count][3] T_pipe, T_sync, T_opt (nullable)
+    u64 first, count;                 // global candidate range that is written
+    // search mode
+    i64 *partial_cost;                // [gridDim.x]
+    u64 *partial_index;               // [gridDim.x]
+    u64 *counters;                    // [0] evaluated, [1] feasible, [2] pruned
+    u64 *incumbent;                   // running minimum of T_iter, for pruning
+    int search, prune;
+};
+
+// ------------------------------------------------------------------------------------------
+// small helpers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int moe_before(const DevConst &dc, int l)
+{   // number of MoE layers among layers 0..l-1
+    int n = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        int lo = w * 64;
+        if (l >= lo + 64) n += __popcll(dc.kindbits[w]);
+        else if (l > lo) n += __popcll(dc.kindbits[w] & ((1ull << (l - lo)) - 1ull));
+    }
+    return n;
+}
+
+__device__ __forceinline__ int layer_kind(const DevConst &dc, int l)
+{
+    return (int)((dc.kindbits[l >> 6] >> (l & 63)) & 1ull);
+}
+
+__device__ __forceinline__ i64 shfl_i64(i64 v, int src)
+{
+    return __shfl_sync(0xffffffffu, v, src);
+}
+
+__device__ __forceinline__ i64 warp_max_i64(i64 v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { i64 t = __shfl_xor_sync(0xffffffffu, v, o); v = t > v ? t : v; }
+    return v;
+}
+
+__device__ __forceinline__ i64 warp_sum_i64(i64 v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// lexicographic minimum of (cost, index) over the warp
+__device__ __forceinline__ void warp_argmin(i64 &c, u64 &ix)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        i64 c2 = __shfl_xor_sync(0xffffffffu, c, o);
+        u64 i2 = __shfl_xor_sync(0xffffffffu, ix, o);
+        if (c2 < c || (c2 == c && i2 < ix)) { c = c2; ix = i2; }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// layer cost (Eq. 2, Eq. 3) and stage coefficients
+// ------------------------------------------------------------------------------------------
+struct LinkCtx { double bw_intra, bw_inter; int node_size; };
+
+__device__ __forceinline__ int link_class(const LinkCtx &lc, i64 ext) { return ext <= lc.node_size ? HAP_INTRA : HAP_INTER; }
+__device__ __forceinline__ double link_bw(const LinkCtx &lc, int cls) { return cls == HAP_INTRA ? lc.bw_intra : lc.bw_inter; }
+
+// collective over w ranks that span `ext` consecutive devices, D bytes per rank
+__device__ __forceinline__ double collective_ns(const DevConst &dc, const LinkCtx &lc, i64 w, i64 ext, double D)
+{
+    if (w == 1) return 0.0;
+    const int cls = link_class(lc, ext);
+    const double lat = dc.alpha[cls] * (double)(w - 1);
+    const double vol = (D * (double)(w - 1)) / (double)w;
+    return lat + vol / link_bw(lc, cls);
+}
+
+struct TypeConst {      // per (configuration, type) values used by every layer
+    double disp2, imb, den, tr, tr2, commF[2], commB[2];
+};
+
+template <bool QUANT>
+__device__ __forceinline__ void store_pair(i64 *qi, double *qd, size_t at, double a, double b)
+{
+    if (QUANT) {
+        longlong2 v; v.x = __double2ll_rn(a); v.y = __double2ll_rn(b);
+        *reinterpret_cast<longlong2 *>(qi + at) = v;
+    } else {
+        double2 v; v.x = a; v.y = b;
+        *reinterpret_cast<double2 *>(qd + at) = v;
+    }
+}
+
+template <bool QUANT>
+__global__ void __launch_bounds__(128)
+layer_cost_kernel(const DevConst dc, i64 *c2, i64 *coef, double *c2f, double *coeff)
+{
+    __shared__ TypeConst tcs[4][HAP_MAX_TYPES];
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const u64 p = (u64)blockIdx.x * 4 + wib;
+    if (p >= dc.n_pconf) return;
+    const hap_pconf pc = dc.pconf[p];
+    const int N = dc.N, T = dc.T;
+    const int TP = pc.TP, CP = pc.CP, DP = pc.DP, EP = pc.EP, TPE = pc.TPE, EDP = pc.EDP, b = pc.b;
+    const i64 G = pc.G;
+    const i64 tok = (i64)b * dc.S / CP;
+    const i64 H = dc.H;
+    const i64 Hkv = H * dc.nkv / dc.nq;
+    const double thb = (double)tok * (double)H;
+    const double Dtp = thb * dc.beta;
+
+    if (lane < T) {
+        const int h = lane;
+        LinkCtx lc; lc.bw_intra = dc.bw_intra[h]; lc.bw_inter = dc.bw_inter[h]; lc.node_size = dc.node_size[h];
+        TypeConst tc;
+        tc.imb = 1.0 + dc.gamma * (dc.rho[pc.iep] - 1.0);
+        double tdisp = 0.0;
+        if (EP != 1) {
+            const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
+            const double Dag = (thb * dc.beta) * (double)(EP - 1);
+            const int cls = link_class(lc, (i64)EP * TPE);
+            const double fa = dc.alpha[cls] * (double)(EP - 1) + Dmoe / link_bw(lc, cls);
+            const double fg = dc.alpha[cls] * (double)(EP - 1) + Dag / link_bw(lc, cls);
+            tdisp = (fa <= fg) ? fa : fg;
+        }
+        tc.disp2 = 2.0 * tdisp;
+        const double ttpA = 2.0 * collective_ns(dc, lc, TP, TP, Dtp);
+        const double ttpD = ttpA;
+        const double ttpM = 2.0 * collective_ns(dc, lc, TPE, TPE, Dtp);
+        const double Dkv = ((((2.0 * (double)b) * (double)dc.S) * (double)Hkv) * dc.beta) / (double)TP;
+        const double tcp = collective_ns(dc, lc, CP, (i64)TP * CP, Dkv);
+        tc.tr = dc.croute[h] * thb;
+        tc.tr2 = 2.0 * tc.tr;
+        tc.commF[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
+        tc.commB[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
+        tc.commF[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
+        tc.commB[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
+        tc.den = (dc.eta[h] * (double)EP) * (double)TPE;
+        tcs[wib][h] = tc;
+
+        if ((QUANT && coef) || (!QUANT && coeff)) {
+            double v[HAP_NCOEF];
+            const size_t i4 = (((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib;
+            v[HAP_KPRE] = dc.tpre[i4];
+            v[HAP_KPOST] = dc.tpost[i4];
+            const double Dp = Dtp / (double)TP;
+            v[HAP_KP2P_INTRA] = 2.0 * (dc.alpha[HAP_INTRA] + Dp / dc.bw_intra[h]);
+            v[HAP_KP2P_INTER] = 2.0 * (dc.alpha[HAP_INTER] + Dp / dc.bw_inter[h]);
+#pragma unroll
+            for (int h2 = 0; h2 < HAP_MAX_TYPES; ++h2) {
+                const double bo = h2 < T ? dc.bw_inter[h2] : dc.bw_inter[h];
+                const double bmin = dc.bw_inter[h] < bo ? dc.bw_inter[h] : bo;
+                v[HAP_KP2P_CROSS + h2] = 2.0 * (dc.alpha[HAP_CROSS] + Dp / (bmin * dc.chi));
+            }
+            const i64 wd = (i64)DP * CP;
+            const double shd = 6.0 + 12.0 / (double)wd;
+            const double she = 6.0 + 12.0 / (double)EDP;
+            const i64 Pattn = H * (H + 2 * Hkv) + H * H + 2 * H;
+            const i64 Pffn_d = 3 * H * (i64)dc.F_dense, Pffn_e = 3 * H * (i64)dc.F_exp;
+            const i64 Pe = (i64)(dc.E / EP) * Pffn_e;
+            const i64 Prt = H * (i64)dc.E;
+            i64 Pd[2];
+            Pd[HAP_DENSE] = Pattn + Pffn_d;
+            Pd[HAP_MOE] = Pattn + (i64)dc.n_shared * Pffn_e;
+            const double PeT = (double)Pe / (double)TPE;
+            v[HAP_MW + HAP_DENSE] = ((double)Pd[HAP_DENSE] / (double)TP) * shd;
+            v[HAP_MW + HAP_MOE] = ((double)Pd[HAP_MOE] / (double)TP + (double)Prt) * shd + PeT * she;
+            v[HAP_MA + HAP_DENSE] = (thb * dc.act_coef[HAP_DENSE]) / (double)TP;
+            v[HAP_MA + HAP_MOE] = (thb * dc.act_coef[HAP_MOE]) / (double)TP;
+            v[HAP_MX] = ((2.0 * ((thb * dc.beta) * (double)dc.k)) * (1.0 - 1.0 / (double)EP)) * dc.capf
+                        + ((double)tok * (double)dc.E) * 4.0;
+            v[HAP_MPRE] = (((double)dc.V * (double)H) / (double)TP) * shd;
+            v[HAP_MPOST] = v[HAP_MPRE];
+            const int cG = link_class(lc, G);
+            const double bwG = link_bw(lc, cG);
+            const double vfd = (double)(wd - 1) / (double)wd, vfe = (double)(EDP - 1) / (double)EDP;
+#pragma unroll
+            for (int kd = 0; kd < 2; ++kd) {
+                const i64 Pdd = Pd[kd] + (kd == HAP_MOE ? Prt : 0);
+                const double Pel = kd == HAP_MOE ? PeT : 0.0;
+                v[HAP_SBW + kd] = dc.ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG)
+                                               + (((6.0 * Pel) * vfe) / bwG));
+                v[HAP_OPT + kd] = dc.copt[h] * ((double)Pdd / (double)((i64)TP * DP * CP) + Pel / (double)EDP);
+            }
+            v[HAP_SLAT] = dc.ovl_dp * (dc.alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
+            const size_t at = ((size_t)p * T + h) * HAP_NCOEF;
+#pragma unroll
+            for (int q = 0; q < HAP_NCOEF; ++q) {
+                if (QUANT) coef[at + q] = __double2ll_rn(v[q]);
+                else coeff[at + q] = v[q];
+            }
+        }
+    }
+    __syncwarp();
+    if ((QUANT && !c2) || (!QUANT && !c2f)) return;
+
+    const size_t out0 = (size_t)p * T * N * 2;
+    for (int u = lane; u < T * N; u += 32) {
+        const int h = u / N, l = u - h * N;
+        const TypeConst &tc = tcs[wib][h];
+        const size_t i5 = ((((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib) * N + l;
+        const double a = dc.tdf[i5], ab = dc.tdb[i5];
+        double cf, cb;
+        if (layer_kind(dc, l) == HAP_DENSE) {
+            cf = a + tc.commF[HAP_DENSE];
+            cb = ab + tc.commB[HAP_DENSE];
+        } else {
+            const double f = dc.tff[i5], fb = dc.tfb[i5];
+            const double xf = (dc.kappa * f) / tc.den;
+            const double mf = (xf + tc.disp2) * tc.imb;
+            cf = (((a - f) + mf) + tc.tr) + tc.commF[HAP_MOE];
+            const double xb = (dc.kappa * fb) / tc.den;
+            const double mb = (xb + tc.disp2) * tc.imb;
+            cb = (((ab - fb) + mb) + tc.tr2) + tc.commB[HAP_MOE];
+        }
+        store_pair<QUANT>(c2, c2f, out0 + (size_t)u * 2, cf, cb);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// candidate decode: every lane of the warp calls this; lane s < PP receives stage s
+// ------------------------------------------------------------------------------------------
+struct StageMap {
+    int mask;       // types the stage overlaps
+    int cls;        // link class of the boundary into the stage (stage >= 1)
+    int ha, hb;     // sending / receiving device type of that boundary
+};
+
+__device__ __forceinline__ StageMap decode_stage(const DevConst &dc, const hap_pconf &pc, u64 map_idx, int lane)
+{
+    StageMap sm; sm.mask = 0; sm.cls = 0; sm.ha = 0; sm.hb = 0;
+    const int PP = pc.PP, T = dc.T;
+    const i64 G = pc.G;
+    if (pc.mode == HAP_MAP_MULTISET) {
+        // unrank the map_idx-th sequence (lexicographic, types ascending) of a multiset;
+        // the number of completions after placing type h is tot * cnt[h] / rem (exact)
+        int cnt[HAP_MAX_TYPES], used[HAP_MAX_TYPES];
+#pragma unroll
+        for (int h = 0; h < HAP_MAX_TYPES; ++h) { cnt[h] = h < T ? (int)(dc.m[h] / G) : 0; used[h] = 0; }
+        u64 tot = pc.nmap, idx = map_idx;
+        int my_h = 0, my_q = 0, prev_h = 0, last_h = 0;
+        for (int pos = 0; pos < PP; ++pos) {
+            const unsigned rem = (unsigned)(PP - pos);
+            int pick = 0;
+            bool found = false;
+#pragma unroll
+            for (int h = 0; h < HAP_MAX_TYPES; ++h) {
+                if (!found && cnt[h] > 0) {
+                    const u64 below = tot * (u64)cnt[h] / rem;
+                    if (idx < below) { pick = h; tot = below; found = true; }
+                    else idx -= below;
+                }
+            }
+            int q = 0;
+#pragma unroll
+            for (int h = 0; h < HAP_MAX_TYPES; ++h)
+                if (h == pick) { q = used[h]; used[h]++; cnt[h]--; }
+            if (pos == lane) { my_h = pick; my_q = q; prev_h = last_h; }
+            last_h = pick;
+        }
+        if (lane < PP) {
+            sm.mask = 1 << my_h;
+            sm.hb = my_h;
+            sm.ha = prev_h;
+            if (lane > 0) {
+                if (prev_h != my_h) sm.cls = HAP_CROSS;
+                else {
+                    // consecutive stages of one type are consecutive in that type's device line
+                    const i64 first = (i64)my_q * G;
+                    const int ns = dc.node_size[my_h];
+                    sm.cls = ((first - 1) / ns == first / ns) ? HAP_INTRA : HAP_INTER;
+                }
+            }
+        }
+    } else {
+        // map_idx-th permutation of the types (lexicographic); device line = type blocks in that order
+        int sigma[HAP_MAX_TYPES];
+        {
+            unsigned avail = (1u << T) - 1u;
+            u64 idx = map_idx;
+            u64 f = 1;
+            for (int i = 2; i < T; ++i) f *= (u64)i;          // (T-1)!
+#pragma unroll
+            for (int pos = 0; pos < HAP_MAX_TYPES; ++pos) {
+                sigma[pos] = 0;
+                if (pos < T) {
+                    int pick = (int)(idx / f);
+                    idx -= (u64)pick * f;
+                    if (T - 1 - pos > 0) f /= (u64)(T - 1 - pos);
+                    // pick-th set bit of avail
+                    unsigned a = avail;
+                    for (int t = 0; t < pick; ++t) a &= a - 1;
+                    const int h = __ffs(a) - 1;
+                    sigma[pos] = h;
+                    avail &= ~(1u << h);
+                }
+            }
+        }
+        if (lane < PP) {
+            const i64 lo = (i64)lane * G, hi = lo + G - 1;
+            i64 start = 0;
+            int ta = 0, tb = 0;
+            i64 oa = 0, ob = 0;
+#pragma unroll
+            for (int bq = 0; bq < HAP_MAX_TYPES; ++bq) {
+                if (bq < T) {
+                    const int h = sigma[bq];
+                    const i64 end = start + dc.m[h];
+                    if (start <= hi && end > lo) sm.mask |= 1 << h;
+                    if (start <= lo && lo < end) { tb = h; ob = lo - start; }
+                    if (lane > 0 && start <= lo - 1 && lo - 1 < end) { ta = h; oa = lo - 1 - start; }
+                    start = end;
+                }
+            }
+            sm.ha = ta; sm.hb = tb;
+            if (lane > 0) {
+                if (ta != tb) sm.cls = HAP_CROSS;
+                else sm.cls = (oa / dc.node_size[ta] == ob / dc.node_size[tb]) ? HAP_INTRA : HAP_INTER;
+            }
+        }
+    }
+    return sm;
+}
+
+// configuration that owns candidate index c (binary search over the offsets)
+__device__ __forceinline__ u64 find_pconf(const DevConst &dc, u64 c)
+{
+    u64 lo = 0, hi = dc.n_pconf;            // invariant: offset[lo] <= c < offset[hi] (virtual)
+    while (hi - lo > 1) {
+        const u64 mid = (lo + hi) >> 1;
+        if (dc.pconf[mid].offset <= c) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__global__ void decode_kernel(const DevConst dc, u64 first, u64 count, hap_candidate *out)
+{
+    const u64 w = ((u64)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= count) return;
+    const u64 c = first + w;
+    const u64 p = find_pconf(dc, c);
+    const hap_pconf pc = dc.pconf[p];
+    const u64 local = c - pc.offset;
+    const u64 map_idx = local / (u64)dc.n_rc;
+    const int rc = (int)(local - map_idx * (u64)dc.n_rc);
+    const StageMap sm = decode_stage(dc, pc, map_idx, lane);
+    hap_candidate *o = out + w;
+    if (lane == 0) {
+        o->index = c; o->pconf = (uint32_t)p; o->rc_mask = dc.rc_masks[rc]; o->map_idx = map_idx;
+        o->PP = (uint8_t)pc.PP;
+        for (int i = 0; i < 7; ++i) o->pad[i] = 0;
+    }
+    o->mask[lane] = lane < pc.PP ? (uint8_t)sm.mask : 0;
+    o->link[lane] = (lane < pc.PP && lane > 0) ? (uint8_t)(sm.cls | (sm.ha << 2) | (sm.hb << 4)) : 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// pipeline DP
+// ------------------------------------------------------------------------------------------
+struct DpSmem {
+    i64 *sC;      // [kMaxMasks][N+1] prefix of forward+backward per type mask
+    i64 *sF;      // [kMaxMasks][N+1] prefix of forward per type mask
+    i64 *sW;      // [N+1] prefix of weight bytes
+    i64 *sA;      // [N+1] prefix of activation bytes per stored micro-batch
+    i64 *rows;    // per warp: prev[N+1], cur[N+1]
+    uint8_t *ch;  // per warp: [PPmax][N+1]
+};
+
+__host__ __device__ inline size_t dp_smem_bytes(int N, int PPmax)
+{
+    const size_t n1 = (size_t)N + 1;
+    size_t b = (size_t)kMaxMasks * n1 * 8 * 2 + n1 * 8 * 2 + (size_t)kDpWarps * n1 * 8 * 2;
+    size_t chb = ((size_t)PPmax * n1 + 15) / 16 * 16;
+    return b + (size_t)kDpWarps * chb + 64;
+}
+
+// cost of one stage span (a, b] for the lane's own stage; used in the backtrace
+struct StagePar {
+    int mask, first, last;      // first / last: stage 1 / stage PP flags
+    i64 cap, K, mstore;
+    int nmin, nmax;
+};
+
+__device__ __forceinline__ bool span_fits(const DevConst &dc, const i64 *sW, const i64 *sA, const StagePar &sp,
+                                          i64 extra, i64 mx, int a, int b, int r)
+{
+    const bool has_moe = moe_before(dc, b) - moe_before(dc, a) > 0;
+    const i64 Wb = (sW[b] - sW[a]) + extra + (has_moe ? mx : 0);
+    const i64 A = sp.mstore * (sA[b] - sA[a]);
+    return Wb + ((i64)dc.xi_q[r] * A) / 1024 <= sp.cap;
+}
+
+template <bool SEARCH>
+__global__ void __launch_bounds__(kDpWarps * 32)
+pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef, DpOut out, int PPmax)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int N = dc.N, T = dc.T, n1 = N + 1;
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const WorkItem it = items[blockIdx.x];
+    const hap_pconf pc = dc.pconf[it.p];
+    const int PP = pc.PP;
+    {   // blocks whose candidates all lie outside the requested range have nothing to do
+        const u64 c0 = pc.offset + it.lo, c1 = c0 + it.count;
+        if (c1 <= out.first || c0 >= out.first + out.count) {
+            if (SEARCH && threadIdx.x == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
+            return;
+        }
+    }
+
+    i64 *sC = reinterpret_cast<i64 *>(smem_raw);
+    i64 *sF = sC + (size_t)kMaxMasks * n1;
+    i64 *sW = sF + (size_t)kMaxMasks * n1;
+    i64 *sA = sW + n1;
+    i64 *rows = sA + n1 + (size_t)wib * 2 * n1;
+    const size_t chb = ((size_t)PPmax * n1 + 15) / 16 * 16;
+    uint8_t *chw = reinterpret_cast<uint8_t *>(sA + n1 + (size_t)kDpWarps * 2 * n1) + (size_t)wib * chb;
+
+    // ---- block prologue: rows of this configuration ------------------------------------
+    const i64 *c2p = c2 + (size_t)it.p * T * N * 2;
+    const i64 *cfp = coef + (size_t)it.p * T * HAP_NCOEF;
+    const int nmask = (1 << T) - 1;
+    for (int mk = 1 + wib; mk <= nmask + 1; mk += kDpWarps) {
+        // masks 1..nmask: time rows; the extra round (mk == nmask+1) builds the byte rows
+        i64 runC = 0, runF = 0;
+        for (int base = 0; base < N; base += 32) {
+            const int l = base + lane;
+            i64 vC = 0, vF = 0;
+            if (l < N) {
+                if (mk <= nmask) {
+                    i64 F = 0, B = 0;
+                    for (int h = 0; h < T; ++h)
+                        if (mk >> h & 1) {
+                            const longlong2 q = *reinterpret_cast<const longlong2 *>(c2p + ((size_t)h * N + l) * 2);
+                            F = q.x > F ? q.x : F;
+                            B = q.y > B ? q.y : B;
+                        }
+                    vC = F + B; vF = F;
+                } else {
+                    const int kd = layer_kind(dc, l);
+                    vC = cfp[HAP_MW + kd]; vF = cfp[HAP_MA + kd];
+                }
+            }
+            // inclusive warp scan
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const i64 tC = __shfl_up_sync(0xffffffffu, vC, o), tF = __shfl_up_sync(0xffffffffu, vF, o);
+                if (lane >= o) { vC += tC; vF += tF; }
+            }
+            vC += runC; vF += runF;
+            if (l < N) {
+                if (mk <= nmask) { sC[(size_t)(mk - 1) * n1 + l + 1] = vC; sF[(size_t)(mk - 1) * n1 + l + 1] = vF; }
+                else { sW[l + 1] = vC; sA[l + 1] = vF; }
+            }
+            runC = shfl_i64(vC, 31); runF = shfl_i64(vF, 31);
+        }
+        if (lane == 0) {
+            if (mk <= nmask) { sC[(size_t)(mk - 1) * n1] = 0; sF[(size_t)(mk - 1) * n1] = 0; }
+            else { sW[0] = 0; sA[0] = 0; }
+        }
+    }
+    __syncthreads();
+
+    const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
+    i64 best_cost = kInf;
+    u64 best_index = ~0ull;
+    u64 n_eval = 0, n_feas = 0;
+
+    for (u64 w = wib; w < it.count; w += kDpWarps) {
+        const u64 local = it.lo + w;
+        const u64 c = pc.offset + local;
+        if (c < out.first || c >= out.first + out.count) continue;
+        const u64 map_idx = local / (u64)dc.n_rc;
+        const unsigned rc_mask = dc.rc_masks[(int)(local - map_idx * (u64)dc.n_rc)];
+        const StageMap smap = decode_stage(dc, pc, map_idx, lane);
+
+        // ---- per-stage parameters, lane s holds stage s+1 ---------------------------------
+        StagePar sp;
+        sp.mask = smap.mask; sp.first = lane == 0; sp.last = lane == PP - 1;
+        sp.cap = 0; sp.K = 0; sp.mstore = 0; sp.nmin = 1; sp.nmax = N - PP + 1;
+        i64 Pmin = 0;
+        if (lane < PP) {
+            i64 kpre = 0, kpost = 0;
+            bool seen = false;
+            for (int h = 0; h < T; ++h)
+                if (smap.mask >> h & 1) {
+                    const i64 *row = cfp + h * HAP_NCOEF;
+                    if (!seen || dc.cap_eff[h] < sp.cap) sp.cap = dc.cap_eff[h];
+                    if (!seen || dc.P[h] < Pmin) Pmin = dc.P[h];
+                    if (!seen || row[HAP_KPRE] > kpre) kpre = row[HAP_KPRE];
+                    if (!seen || row[HAP_KPOST] > kpost) kpost = row[HAP_KPOST];
+                    seen = true;
+                }
+            if (sp.first) sp.K += kpre;
+            if (sp.last) sp.K += kpost;
+            if (lane > 0) {
+                const i64 *row = cfp + smap.hb * HAP_NCOEF;
+                sp.K += smap.cls == HAP_INTRA ? row[HAP_KP2P_INTRA]
+                        : (smap.cls == HAP_INTER ? row[HAP_KP2P_INTER] : row[HAP_KP2P_CROSS + smap.ha]);
+            }
+            const int inflight = PP - lane;                 // PP - i + 1 with i = lane + 1
+            sp.mstore = pc.M < inflight ? pc.M : inflight;
+        }
+        if (dc.delta_q >= 0) {
+            const i64 Ps = warp_sum_i64(lane < PP ? Pmin : 0);
+            if (lane < PP) {
+                const i64 den = 1024 * Ps;
+                i64 lo = ((i64)(1024 - dc.delta_q) * Pmin * N) / den;
+                i64 hi = ((i64)(1024 + dc.delta_q) * Pmin * N + den - 1) / den;
+                if (lo < 1) lo = 1;
+                if (hi > N - PP + 1) hi = N - PP + 1;
+                sp.nmin = (int)lo; sp.nmax = (int)hi;
+            }
+        }
+
+        // ---- recurrence ------------------------------------------------------------------
+        i64 *prev = rows, *cur = rows + n1;
+        for (int j = lane; j <= N; j += 32) prev[j] = j == 0 ? 0 : kInf;
+        if (out.dp_table && !SEARCH) {
+            i64 *t = out.dp_table + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
+            for (int j = lane; j <= N; j += 32) t[j] = j == 0 ? 0 : kInf;
+        }
+        if (out.choice && !SEARCH) {
+            uint8_t *t = out.choice + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
+            for (int j = lane; j <= N; j += 32) t[j] = 255;
+        }
+        __syncwarp();
+        for (int i = 1; i <= PP; ++i) {
+            const int src = i - 1;
+            const int mask = __shfl_sync(0xffffffffu, sp.mask, src);
+            const i64 cap = shfl_i64(sp.cap, src), K = shfl_i64(sp.K, src), mstore = shfl_i64(sp.mstore, src);
+            const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
+            const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
+            const i64 *rC = sC + (size_t)(mask - 1) * n1, *rF = sF + (size_t)(mask - 1) * n1;
+            uint8_t *chrow = chw + (size_t)(i - 1) * n1;
+            const int jlo = i, jhi = N - PP + i;
+            for (int j = lane; j <= N; j += 32) {
+                i64 best = kInf;
+                int arg = 255;
+                if (j >= jlo && j <= jhi) {
+                    int klo = j - nmax; if (klo < i - 1) klo = i - 1;
+                    const int khi = j - nmin;                 // nmin >= 1 keeps k <= j-1
+                    if (klo <= khi) {
+                        const i64 Cj = rC[j] + K, Fj = rF[j], Wj = sW[j] + extra, Aj = sA[j];
+                        const int moe_j = moe_before(dc, j);
+                        // feasibility is monotone in k (shorter spans need less memory): for each allowed
+                        // level find the first feasible k; levels are ordered so that these thresholds do
+                        // not increase with the level
+                        int seg_hi = khi;                      // k range still to be assigned a level
+                        for (int r = 0; r < dc.R && seg_hi >= klo; ++r) {
+                            if (!((rc_mask >> r) & 1u)) continue;
+                            int lo = klo, hi = seg_hi + 1;     // first feasible k in [klo, seg_hi+1]
+                            while (lo < hi) {
+                                const int mid = (lo + hi) >> 1;
+                                const bool has_moe = moe_j - moe_before(dc, mid) > 0;
+                                const i64 Wb = (Wj - sW[mid]) + (has_moe ? mx : 0);
+                                const i64 A = mstore * (Aj - sA[mid]);
+                                if (Wb + ((i64)dc.xi_q[r] * A) / 1024 <= cap) hi = mid; else lo = mid + 1;
+                            }
+                            // k in [lo, seg_hi] runs at level r
+                            const i64 tau = dc.tau_q[r];
+                            for (int k = seg_hi; k >= lo; --k) {
+                                const i64 pv = prev[k];
+                                const i64 cst = (Cj - rC[k]) + (tau * (Fj - rF[k])) / 1024;
+                                const i64 v = pv > cst ? pv : cst;
+                                if (v <= best && v < kInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
+                            }
+                            seg_hi = lo - 1;
+                        }
+                    }
+                }
+                cur[j] = best;
+                chrow[j] = (uint8_t)arg;
+            }
+            __syncwarp();
+            if (!SEARCH) {
+                if (out.dp_table) {
+                    i64 *t = out.dp_table + ((size_t)(c - out.first) * (HAP_MAX_PP + 1) + i) * n1;
+                    for (int j = lane; j <= N; j += 32) t[j] = cur[j];
+                }
+                if (out.choice) {
+                    uint8_t *t = out.choice + ((size_t)(c - out.first) * (HAP_MAX_PP + 1) + i) * n1;
+                    for (int j = lane; j <= N; j += 32) t[j] = chrow[j];
+                }
+            }
+            i64 *tmp = prev; prev = cur; cur = tmp;
+        }
+        const i64 bott = prev[N];
+        __syncwarp();
+
+        // ---- backtrace, Eq. 4 -----------------------------------------------------------
+        i64 T_iter = kInf, T_pipe = kInf, T_sync = 0, T_opt = 0;
+        int my_n = 0, my_r = 0;
+        if (bott < kInf) {
+            int a_me = 0, b_me = 0;
+            int j = N;
+            for (int i = PP; i >= 1; --i) {
+                const int k = chw[(size_t)(i - 1) * n1 + j];
+                if (lane == i - 1) { a_me = k; b_me = j; }
+                j = k;
+            }
+            i64 c_me = 0, sync_me = 0, opt_me = 0;
+            if (lane < PP) {
+                const i64 extra = (sp.first ? mpre : 0) + (sp.last ? mpost : 0);
+                int r = 0;
+                for (; r < dc.R; ++r)
+                    if (((rc_mask >> r) & 1u) && span_fits(dc, sW, sA, sp, extra, mx, a_me, b_me, r)) break;
+                const i64 *rC = sC + (size_t)(sp.mask - 1) * n1, *rF = sF + (size_t)(sp.mask - 1) * n1;
+                c_me = (rC[b_me] - rC[a_me]) + ((i64)dc.tau_q[r] * (rF[b_me] - rF[a_me])) / 1024 + sp.K;
+                my_n = b_me - a_me; my_r = r;
+                const i64 n_moe = moe_before(dc, b_me) - moe_before(dc, a_me), n_dense = (b_me - a_me) - n_moe;
+                i64 slat = 0, sbd = 0, sbm = 0, opd = 0, opm = 0;
+                bool seen = false;
+                for (int h = 0; h < T; ++h)
+                    if (sp.mask >> h & 1) {
+                        const i64 *row = cfp + h * HAP_NCOEF;
+                        if (!seen || row[HAP_SLAT] > slat) slat = row[HAP_SLAT];
+                        if (!seen || row[HAP_SBW] > sbd) sbd = row[HAP_SBW];
+                        if (!seen || row[HAP_SBW + 1] > sbm) sbm = row[HAP_SBW + 1];
+                        if (!seen || row[HAP_OPT] > opd) opd = row[HAP_OPT];
+                        if (!seen || row[HAP_OPT + 1] > opm) opm = row[HAP_OPT + 1];
+                        seen = true;
+                    }
+                sync_me = slat + n_dense * sbd + n_moe * sbm;
+                opt_me = n_dense * opd + n_moe * opm;
+            }
+            const i64 sum = warp_sum_i64(c_me), mxc = warp_max_i64(c_me);
+            const i64 tsync = warp_max_i64(sync_me), topt = warp_max_i64(opt_me);
+            T_pipe = sum + (i64)(pc.M - 1) * mxc;
+            T_sync = tsync; T_opt = topt;
+            T_iter = T_pipe + tsync + topt;
+        }
+        if (SEARCH) {
+            n_eval++;
+            if (T_iter < kInf) n_feas++;
+            if (T_iter < best_cost || (T_iter == best_cost && c < best_index)) { best_cost = T_iter; best_index = c; }
+        } else {
+            const u64 o = c - out.first;
+            if (lane == 0) {
+                if (out.cost) out.cost[o] = T_iter;
+                if (out.bottleneck) out.bottleneck[o] = bott < kInf ? bott : kInf;
+                if (out.detail) { out.detail[o * 3] = T_pipe; out.detail[o * 3 + 1] = T_sync; out.detail[o * 3 + 2] = T_opt; }
+            }
+            if (out.partition) out.partition[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < kInf ? my_n : 0);
+            if (out.recompute) out.recompute[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < kInf ? my_r : 0);
+        }
+        __syncwarp();
+    }
+
+    if (SEARCH) {
+        __shared__ i64 wcost[kDpWarps];
+        __shared__ u64 widx[kDpWarps];
+        if (lane == 0) {
+            wcost[wib] = best_cost; widx[wib] = best_index;
+            if (n_eval) atomicAdd(out.counters + 0, n_eval);
+            if (n_feas) atomicAdd(out.counters + 1, n_feas);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            i64 bc = wcost[0]; u64 bi = widx[0];
+            for (int q = 1; q < kDpWarps; ++q)
+                if (wcost[q] < bc || (wcost[q] == bc && widx[q] < bi)) { bc = wcost[q]; bi = widx[q]; }
+            out.partial_cost[blockIdx.x] = bc;
+            out.partial_index[blockIdx.x] = bi;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// argmin: stage 1 reduces a slice per block, stage 2 (one block) reduces the partials
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex)
+{
+    i64 bc = kInf; u64 bi = ~0ull;
+    for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (u64)gridDim.x * blockDim.x) {
+        const i64 v = cost[i];
+        if (v < bc) { bc = v; bi = i; }      // ascending i per thread: strict keeps the lowest index
+    }
+    warp_argmin(bc, bi);
+    __shared__ i64 sc[8]; __shared__ u64 si[8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) { sc[w] = bc; si[w] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int q = 1; q < 8; ++q) if (sc[q] < bc || (sc[q] == bc && si[q] < bi)) { bc = sc[q]; bi = si[q]; }
+        pcost[blockIdx.x] = bc; pindex[blockIdx.x] = bi;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2)
+{
+    i64 bc = kInf; u64 bi = ~0ull;
+    for (u64 i = threadIdx.x; i < n; i += blockDim.x) {
+        const i64 v = pcost[i]; const u64 ix = pindex[i];
+        if (v < bc || (v == bc && ix < bi)) { bc = v; bi = ix; }
+    }
+    warp_argmin(bc, bi);
+    __shared__ i64 sc[8]; __shared__ u64 si[8];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    if (lane == 0) { sc[w] = bc; si[w] = bi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int q = 1; q < 8; ++q) if (sc[q] < bc || (sc[q] == bc && si[q] < bi)) { bc = sc[q]; bi = si[q]; }
+        out2[0] = bc; out2[1] = (i64)bi;
+    }
+}
+
+}  // namespace hap

@@ -1,0 +1,223 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Integer mode: layer costs, coefficients, decoded mappings, DP tables, split choices, partitions,
+recomputation levels, bottlenecks, iteration times and the winning index must be bit-identical.
+The unrounded fp64 layer costs must agree within 1e-9 relative (they are the same IEEE operations
+in the same order, so in practice they agree exactly)."""
+import os
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from gen import problems  # noqa: E402
+from oracle import Oracle, INF  # noqa: E402
+
+CONFIGS = ["tiny", "small", "mixtral", "dsv2", "stress"]
+NTHREADS = max(1, len(os.sched_getaffinity(0)))
+
+
+@pytest.fixture(scope="module")
+def hap():
+    import paper_2609_39350_b200 as hap
+    from paper_2609_39350_b200.build import build_library
+    build_library()
+    assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
+    return hap
+
+
+_cache = {}
+
+
+def setup(hap, name, **kw):
+    key = (name, tuple(sorted(kw.items())))
+    if key not in _cache:
+        pb = problems.make_problem(name, **kw)
+        hp = hap.hap_problem_create(pb)
+        hap.hap_enumerate(hp)
+        _cache[key] = (pb, hp, Oracle(pb))
+    return _cache[key]
+
+
+@pytest.mark.parametrize("name", CONFIGS)
+def test_enumeration_is_identical(hap, name):
+    pb, hp, o = setup(hap, name)
+    assert (hp.n_pconf, hp.n_cand) == (o.n_pconf, o.n_cand)
+    got = hap.hap_get_pconfs(hp)
+    for f in ("PP", "TP", "CP", "DP", "EP", "TPE", "b", "M", "EDP", "G", "itp", "icp", "ib", "iep", "mode", "nmap", "offset"):
+        assert np.array_equal(got[f], o.pconfs[f]), f
+
+
+@pytest.mark.parametrize("name", CONFIGS)
+def test_layer_costs_and_coefficients_bit_exact(hap, name):
+    pb, hp, o = setup(hap, name)
+    c2, coef = hap.hap_eval_layer_costs(hp)
+    c2f, coeff = hap.hap_eval_layer_costs_f64(hp)
+    torch.cuda.synchronize()
+    c2, coef, c2f, coeff = c2.cpu().numpy(), coef.cpu().numpy(), c2f.cpu().numpy(), coeff.cpu().numpy()
+    step = 1 if o.n_pconf <= 4000 else 3
+    for p in list(range(0, o.n_pconf, step)) + [o.n_pconf - 1]:
+        e2, e2f, ecoef, ecoeff = o.layer_costs(p)
+        assert np.array_equal(c2[p], e2), p
+        assert np.array_equal(coef[p], ecoef), p
+        assert np.allclose(c2f[p], e2f, rtol=1e-9, atol=0.0), p
+        assert np.allclose(coeff[p], ecoeff, rtol=1e-9, atol=0.0), p
+
+
+@pytest.mark.parametrize("name", CONFIGS)
+def test_decode_matches_oracle(hap, name):
+    pb, hp, o = setup(hap, name)
+    n_rc = len(pb.rc_masks)
+    rng = np.random.default_rng(11)
+    if o.n_cand <= 80000:
+        ranges = [(0, o.n_cand)]
+    else:
+        starts = sorted(set([0, o.n_cand - 700] + rng.integers(0, o.n_cand - 700, 30).tolist()))
+        ranges = [(s, 700) for s in starts]
+    for first, count in ranges:
+        got = hap.hap_decode(hp, first, count)
+        for q in range(0, count, 1 if count <= 2000 else 7):
+            idx = first + q
+            p = o.find_pconf(idx)
+            local = idx - int(o.pconfs["offset"][p])
+            mp = o.decode(p, local // n_rc)
+            PP = int(o.pconfs["PP"][p])
+            g = got[q]
+            assert int(g["index"]) == idx and int(g["pconf"]) == p and int(g["PP"]) == PP
+            assert int(g["map_idx"]) == local // n_rc and int(g["rc_mask"]) == int(pb.rc_masks[local % n_rc])
+            assert g["mask"][:PP].tolist() == list(mp.mask[:PP]) and not g["mask"][PP:].any()
+            link = [(mp.cls[s] | (mp.ha[s] << 2) | (mp.hb[s] << 4)) if s else 0 for s in range(PP)]
+            assert g["link"][:PP].tolist() == link, (idx, g["link"][:PP].tolist(), link)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}),
+                                     ("dsv2", {}), ("stress", {})])
+def test_every_candidate_cost_and_bottleneck_bit_exact(hap, name, kw):
+    """Whole candidate space, in the launch configuration the benchmark times."""
+    pb, hp, o = setup(hap, name, **kw)
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=NTHREADS, want_costs=True)
+    assert done == o.n_cand
+    got_c, got_b = out["cost"].cpu().numpy(), out["bottleneck"].cpu().numpy()
+    bad = np.nonzero(got_c != costs)[0]
+    assert bad.size == 0, (bad[:10], got_c[bad[:10]], costs[bad[:10]])
+    assert np.array_equal(got_b, bn)
+    # argmin of the device cost array: lowest cost, lowest index on ties
+    am = hap.hap_argmin(hp, out["cost"]).cpu().numpy()
+    assert (int(am[0]), int(am[1])) == (bc, bi)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}),
+                                     ("dsv2", {}), ("stress", {})])
+def test_tables_partitions_and_recompute_bit_exact(hap, name, kw):
+    pb, hp, o = setup(hap, name, **kw)
+    rng = np.random.default_rng(3)
+    if o.n_cand <= 2000:
+        ranges = [(0, o.n_cand)]
+    else:
+        starts = sorted(set([0, o.n_cand - 64] + rng.integers(0, o.n_cand - 64, 24).tolist()))
+        ranges = [(s, 64) for s in starts]
+    N = pb.N
+    for first, count in ranges:
+        out = hap.hap_pipeline_dp(hp, first, count, partition=True, tables=True)
+        torch.cuda.synchronize()
+        dp, ch = out["dp_table"].cpu().numpy(), out["choice"].cpu().numpy()
+        part, rec = out["partition"].cpu().numpy(), out["recompute"].cpu().numpy()
+        cost, bott = out["cost"].cpu().numpy(), out["bottleneck"].cpu().numpy()
+        for q in range(0, count, 1 if o.n_cand <= 2000 else 5):
+            plan, edp, ech = o.eval_index(first + q, tables=True)
+            PP = plan["PP"]
+            assert np.array_equal(dp[q, :PP + 1], edp), (first + q)
+            assert np.array_equal(ch[q, :PP + 1], ech), (first + q)
+            assert (dp[q, PP + 1:] == -1).all() and (ch[q, PP + 1:] == 254).all()     # rows beyond PP untouched
+            assert cost[q] == plan["T_iter"] and bott[q] == plan["bottleneck"]
+            if plan["T_iter"] < INF:
+                assert part[q, :PP].tolist() == plan["n"] and rec[q, :PP].tolist() == plan["r"]
+                assert int(part[q].sum()) == N
+            else:
+                assert not part[q].any() and not rec[q].any()
+            assert not part[q, PP:].any()
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}),
+                                     ("dsv2", {}), ("stress", {})])
+def test_search_best_returns_the_oracle_plan(hap, name, kw):
+    pb, hp, o = setup(hap, name, **kw)
+    plan, stats = hap.hap_search_best(hp)
+    done, bc, bi = o.search_pconfs(0, 1, threads=NTHREADS)
+    assert (plan["T_iter"], plan["index"]) == (bc, bi)
+    eplan, _, _ = o.eval_index(bi)
+    for key in ("PP", "TP", "CP", "DP", "EP", "TPE", "b", "M", "n", "r", "mask", "rc_mask", "bottleneck", "T_pipe", "T_sync", "T_opt"):
+        assert plan[key] == eplan[key], key
+    assert stats["n_candidates"] == o.n_cand and stats["n_evaluated"] + stats["n_pruned"] == o.n_cand
+    assert sum(plan["n"]) == pb.N
+
+
+def test_sub_ranges_ragged_edges_and_errors(hap):
+    pb, hp, o = setup(hap, "small")
+    costs, bn, best, feas = o.search(1000, 3001)
+    out = hap.hap_pipeline_dp(hp, 1000, 3001)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["cost"].cpu().numpy(), costs)
+    plan, stats = hap.hap_search_range(hp, 1000, 3001)
+    assert plan["index"] == best["index"] and plan["T_iter"] == best["T_iter"] and stats["n_evaluated"] == 3001
+    # single candidate, last candidate, empty range
+    one = hap.hap_pipeline_dp(hp, o.n_cand - 1, 1)
+    torch.cuda.synchronize()
+    assert int(one["cost"].cpu()[0]) == o.eval_index(o.n_cand - 1)[0]["T_iter"]
+    hap.hap_pipeline_dp(hp, 5, 0)
+    with pytest.raises(hap.HapError) as e:
+        hap.hap_pipeline_dp(hp, o.n_cand - 1, 2)
+    assert e.value.name == "HAP_E_RANGE"
+    with pytest.raises(hap.HapError):
+        hap.hap_search_range(hp, 0, 0)
+
+
+def test_all_infeasible_and_bad_descriptors(hap):
+    pb = problems.small()
+    pb.cap_eff[:] = 1 << 20
+    hp = hap.hap_problem_create(pb)
+    hap.hap_enumerate(hp)
+    with pytest.raises(hap.HapError) as e:
+        hap.hap_search_range(hp, 0, 5000)
+    assert e.value.name == "HAP_E_INFEASIBLE"
+    out = hap.hap_pipeline_dp(hp, 0, 5000, partition=True)
+    torch.cuda.synchronize()
+    assert (out["cost"].cpu().numpy() == INF).all() and not out["partition"].cpu().numpy().any()
+    hap.hap_problem_destroy(hp)
+    bad = problems.tiny()
+    bad.tff[0, 0, 0, 0, 0] = bad.tdf[0, 0, 0, 0, 0] * 2       # FFN slower than the layer that contains it
+    with pytest.raises(hap.HapError) as e:
+        hap.hap_problem_create(bad)
+    assert e.value.name == "HAP_E_INVALID"
+    hp2 = hap.hap_problem_create(problems.tiny())
+    with pytest.raises(hap.HapError) as e:
+        hap.hap_pipeline_dp(hp2, 0, 1)                          # before hap_enumerate
+    assert e.value.name == "HAP_E_STATE"
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_small_problems_with_tight_memory(hap, seed):
+    """Mixed layer kinds, recomputation policies, windows and tight capacities on small random problems."""
+    pb = problems.random_small(seed, N=9 + seed, T=2 + seed % 2, nodes_per_type=(2, 2, 1)[:2 + seed % 2],
+                               node_size=2, window=(seed % 2 == 0), first_dense=True)
+    hp = hap.hap_problem_create(pb)
+    hap.hap_enumerate(hp)
+    o = Oracle(pb)
+    assert hp.n_cand == o.n_cand
+    costs, bn, best, feas = o.search()
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand, partition=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["cost"].cpu().numpy(), costs) and np.array_equal(out["bottleneck"].cpu().numpy(), bn)
+    part, rec = out["partition"].cpu().numpy(), out["recompute"].cpu().numpy()
+    for idx in range(0, o.n_cand, 5):
+        plan, _, _ = o.eval_index(idx)
+        if plan["T_iter"] < INF:
+            assert part[idx, :plan["PP"]].tolist() == plan["n"] and rec[idx, :plan["PP"]].tolist() == plan["r"]
+    if best is not None:
+        plan, _ = hap.hap_search_best(hp)
+        assert plan["index"] == best["index"] and plan["n"] == best["n"] and plan["r"] == best["r"]
+    hap.hap_problem_destroy(hp)

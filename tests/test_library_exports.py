@@ -1,0 +1,43 @@
+"""The C-ABI library loads without a GPU and exports every function include/hap.h declares."""
+import ctypes
+import os
+import re
+
+import paper_2609_39350_b200 as hap
+from paper_2609_39350_b200.build import build_library, LIB
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "hap.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hap_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_functions_are_exported_and_bound():
+    build_library()
+    lib = ctypes.CDLL(LIB)
+    names = _declared_functions()
+    assert "hap_problem_create" in names and "hap_search_best" in names and "hap_pipeline_dp" in names
+    for n in names:
+        assert getattr(lib, n) is not None, n
+    assert sorted(hap.EXPORTS) == names
+    for n in names:
+        if n not in ("hap_status_str", "hap_last_error"):
+            assert hasattr(hap, n), f"python binding lacks {n}"
+
+
+def test_status_strings_and_null_arguments():
+    lib = hap.load_library()
+    assert lib.hap_status_str(0) == b"HAP_OK" and lib.hap_status_str(6) == b"HAP_E_INFEASIBLE"
+    out = ctypes.c_void_p(0)
+    assert lib.hap_problem_create(None, None, None, None, ctypes.byref(out)) == 1 and not out.value
+    assert lib.hap_enumerate(None, None, None) == 1
+    lib.hap_problem_destroy(None)
+
+
+def test_layouts_match_the_header_sizes():
+    from paper_2609_39350_b200 import binding as b
+    assert b.PCONF_DTYPE.itemsize == 80 and b.CANDIDATE_DTYPE.itemsize == 96
+    assert ctypes.sizeof(b._Plan) == 8 + 8 * 4 + 8 + 3 * 32 + 5 * 8
