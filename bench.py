@@ -1,0 +1,298 @@
+#!/usr/bin/env python
+"""Benchmark of the planner hot path: candidate plans evaluated per second.
+
+One step = one pass of the whole hot path over the workload's candidate space: layer costs
+(Eq. 2 / Eq. 3) for every configuration, the pipeline dynamic program for every candidate
+(no pruning), and the (cost, index) argmin.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload stress] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) the candidate space is sharded over the ranks
+in contiguous, work-balanced ranges and the ranks exchange one (cost, index) pair per step.
+`--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "candidate_plans_per_second"
+UNIT = "candidates/s"
+SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower() == "active":
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def cpu_cores() -> int:
+    return max(1, len(os.sched_getaffinity(0)))
+
+
+def oracle_sample(pb, budget_s: float, threads: int):
+    """Times the CPU oracle on every `stride`-th configuration so that the run takes about budget_s."""
+    from oracle import Oracle
+    o = Oracle(pb)
+    probe = max(1, o.n_pconf // 64)
+    t0 = time.perf_counter()
+    done, _, _ = o.search_pconfs(0, probe, threads=threads)
+    dt = max(time.perf_counter() - t0, 1e-6)
+    est_full = dt * o.n_cand / max(done, 1)
+    stride = max(1, int(round(est_full / budget_s)))
+    t0 = time.perf_counter()
+    done, bc, bi = o.search_pconfs(0, stride, threads=threads)
+    dt = time.perf_counter() - t0
+    return dict(value=done / dt, seconds=dt, candidates=done, stride=stride, n_pconf=o.n_pconf, n_cand=o.n_cand)
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from gen import problems
+    pb = problems.make_problem(args.workload)
+    threads = cpu_cores()
+    budget = max(2.0, min(30.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(pb, budget / 4, threads)
+    vals, secs, sample = [], [], None
+    for _ in range(args.steps):
+        sample = oracle_sample(pb, budget, threads)
+        vals.append(sample["value"]); secs.append(sample["seconds"])
+    value = statistics.median(vals)
+    desc = (f"every {sample['stride']}-th of {sample['n_pconf']} configurations of {args.workload} "
+            f"({sample['candidates']} of {sample['n_cand']} candidates) per step")
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * statistics.median(secs), higher_is_better=True,
+                scaling="strong", vs_baseline=None, dtype="int64", data="synthetic",
+                config=dict(workload=args.workload, n_candidates=sample["n_cand"], sample=desc),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=threads, kind="oracle", sample=desc),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="stress")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    import paper_2609_39350_b200 as hap
+    from paper_2609_39350_b200.sharding import shard_ranges, exchange_minimum
+    from gen import problems
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    warmup = max(args.warmup, 3)
+
+    pb = problems.make_problem(args.workload)
+    hp = hap.hap_problem_create(pb)
+    n_pconf, n_cand = hap.hap_enumerate(hp)
+    pconfs = hap.hap_get_pconfs(hp)
+    first, count = shard_ranges(pconfs, len(pb.rc_masks), pb.N, world)[rank]
+    stream = torch.cuda.current_stream()
+
+    out = {"cost": torch.empty(max(count, 1), dtype=torch.int64, device="cuda"),
+           "bottleneck": torch.empty(max(count, 1), dtype=torch.int64, device="cuda")}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # larger than the 126 MB L2
+
+    def step():
+        hap.hap_pipeline_dp(hp, first, count, out=out)
+        return hap.hap_argmin(hp, out["cost"][:count]) if count else None
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        flush.fill_(1)
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    dp_ms, lc_ms, cells = [], [], 0
+    best = None
+    barrier()
+    t_wall = time.perf_counter()
+    for a, b in ev:
+        flush.fill_(1)                       # untimed: evicts the previous step's data from L2
+        a.record(stream)
+        am = step()
+        if world > 1:
+            c, i = (int(x) for x in am.tolist())
+            best = exchange_minimum(c, i + first, device="cuda")
+        b.record(stream)
+        b.synchronize()
+        lc, dpk, cells = hap.hap_get_timings(hp)
+        lc_ms.append(lc); dp_ms.append(dpk)
+    barrier()
+    t_wall = time.perf_counter() - t_wall
+    clocks = sampler.stop()
+    if world == 1:
+        c, i = (int(x) for x in am.tolist())
+        best = (c, i + first)
+
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(total_ms.item())
+    ms_per_step = total_ms / args.steps
+    value = n_cand * args.steps / (total_ms * 1e-3)
+
+    # full search through the search entry point (pruning allowed), wall clock call to return
+    search_ms = []
+    for _ in range(3):
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        plan, stats = hap.hap_search_range(hp, first, count)
+        search_ms.append(1e3 * (time.perf_counter() - t0))
+
+    # end to end through the C ABI from host buffers: create (H2D of the tables), enumerate (H2D of the
+    # configuration table), search, read the plan back
+    e2e_ms = []
+    h2d = sum(int(getattr(pb, n).nbytes) for n in ("tdf", "tdb", "tff", "tfb", "tpre", "tpost")) + int(pconfs.nbytes)
+    d2h = 8 * 2 + 8 * 4 + 200
+    for _ in range(3):
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        hp2 = hap.hap_problem_create(pb)
+        hap.hap_enumerate(hp2)
+        plan2, _ = hap.hap_search_range(hp2, first, count)
+        e2e_ms.append(1e3 * (time.perf_counter() - t0))
+        hap.hap_problem_destroy(hp2)
+    e2e_t = torch.tensor([statistics.median(e2e_ms)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
+    e2e_value = n_cand / (float(e2e_t.item()) * 1e-3)
+
+    if rank == 0:
+        peaks, peak_kind = read_peaks()
+        dp_med, lc_med = statistics.median(dp_ms), statistics.median(lc_ms)
+        sm_mhz = clocks["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)
+        alu_peak = SM_COUNT * SCHEDULERS_PER_SM * LANES * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+        achieved = 4.0 * cells / (dp_med * 1e-3) / 1e12
+        units = n_pconf * hp.T * pb.N
+        lc_gbs = 16.0 * units / (lc_med * 1e-3) / 1e9
+        line = dict(
+            metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=warmup,
+            ms_per_step=ms_per_step, higher_is_better=True, scaling="strong", vs_baseline=None, dtype="int64",
+            data="synthetic",
+            config=dict(workload=args.workload, n_pconf=n_pconf, n_candidates=n_cand, layers=pb.N, devices=pb.W,
+                        window_delta_q=int(pb.delta_q), l2="flushed between steps (256 MiB fill, untimed)",
+                        timing="sum of per-step CUDA-event times, max over ranks",
+                        parallelism=f"candidate ranges over {world} gpu(s)"),
+            clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"]),
+            e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                     ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
+            gpu_launches=4 * args.steps,
+            full_search_ms=statistics.median(search_ms),
+            best=dict(cost=best[0], index=best[1], search_index=plan["index"]),
+            kernels_ms=dict(layer_cost=lc_med, pipeline_dp=dp_med),
+            roofline=dict(bound="alu", kernel="pipeline_dp_kernel", achieved=achieved, peak=alu_peak, unit="Tops/s",
+                          frac=achieved / alu_peak, traffic=None, cells_per_launch=cells,
+                          ops_per_cell=4, peak_source=f"{SM_COUNT} SMs x {SCHEDULERS_PER_SM} schedulers x {LANES} lanes x "
+                          f"{peaks.get('sm_max_mhz', 1965.0)} MHz ({peak_kind} clock)", sm_mhz_seen=sm_mhz),
+            roofline_layer_cost=dict(bound="hbm", kernel="layer_cost_kernel", achieved=lc_gbs, peak=peaks["hbm_gbs"],
+                                     unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=None,
+                                     bytes_per_launch=16 * units, peak_source=f"hbm_gbs ({peak_kind})"),
+            wall_s=t_wall,
+        )
+        if world == 1 and not args.no_cpu_baseline:
+            s = oracle_sample(pb, 15.0, cpu_cores())
+            line["cpu_baseline"] = dict(value=s["value"], unit=UNIT, cores=cpu_cores(), kind="oracle",
+                                        sample=f"every {s['stride']}-th of {s['n_pconf']} configurations of "
+                                               f"{args.workload}: {s['candidates']} candidates in {s['seconds']:.1f} s")
+        print(json.dumps(line))
+    hap.hap_problem_destroy(hp)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

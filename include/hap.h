@@ -221,6 +221,12 @@ hap_status hap_search_best(hap_problem *, hap_plan *host_out, hap_search_stats *
  * dev_out[1] = index (as int64) of the minimum of dev_cost[0..count). */
 hap_status hap_argmin(hap_problem *, const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream);
 
+/* Measurement aid: CUDA-event durations (ms) of the layer-cost kernel and of the dynamic-program
+ * kernel of the most recent hap_pipeline_dp / hap_search_* call, and the number of recurrence cell
+ * updates (k, j pairs inside the window and the memory limit) that launch evaluated.  Waits for that
+ * call's kernels.  Any output may be NULL. */
+hap_status hap_get_timings(hap_problem *, float *ms_layer_cost, float *ms_dp, uint64_t *cells);
+
 const char *hap_status_str(hap_status);
 const char *hap_last_error(const hap_problem *);
 

@@ -16,7 +16,7 @@ COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, S
 STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE", "HAP_E_STATE", "HAP_E_INFEASIBLE"]
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_search_range",
-           "hap_search_best", "hap_argmin", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_get_timings", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -266,6 +266,13 @@ def hap_search_best(hp: HapProblem, stream=None):
     pl, st = _Plan(), _Stats()
     hp.check(load_library().hap_search_best(hp.h, C.byref(pl), C.byref(st), _stream(stream)))
     return _plan_dict(pl), _stats_dict(st)
+
+
+def hap_get_timings(hp: HapProblem):
+    """(ms of the layer-cost kernel, ms of the DP kernel, recurrence cells) of the last DP/search call."""
+    a, b, c = C.c_float(), C.c_float(), C.c_uint64()
+    hp.check(load_library().hap_get_timings(hp.h, C.byref(a), C.byref(b), C.byref(c)))
+    return float(a.value), float(b.value), int(c.value)
 
 
 def hap_argmin(hp: HapProblem, cost, stream=None):

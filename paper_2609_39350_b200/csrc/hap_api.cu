@@ -45,6 +45,7 @@ struct hap_problem {
     i64 *d_best = nullptr;                 // (cost, index) of the search
     void *d_single = nullptr;              // outputs of the one-candidate re-evaluation
     size_t n_partial = 0;
+    bool timed = false;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     std::string err;
 };
@@ -371,8 +372,6 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         p->dc.n_pconf = np;
         const size_t smem = dp_smem_bytes(N, pp_max);
         if (smem > 227 * 1024) return fail(p, HAP_E_RANGE, "shared memory need %zu exceeds the SM", smem);
-        CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         p->enumerated = true;
     }
     if (n_pconf) *n_pconf = p->pconfs.size();
@@ -448,6 +447,15 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
 {
     const size_t smem = dp_smem_bytes(p->model.N, p->pp_max);
     const unsigned blocks = (unsigned)p->items.size();
+    // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
+    // process: raise it (never lower it) before a launch that needs more
+    static size_t smem_limit[64][2];
+    const int dev = p->device & 63;
+    if (smem > smem_limit[dev][search]) {
+        if (search) CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        else CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        smem_limit[dev][search] = smem;
+    }
     if (search) pipeline_dp_kernel<true><<<blocks, kDpWarps * 32, smem, st>>>(p->dc, p->d_items, p->d_c2, p->d_coef, out, p->pp_max);
     else pipeline_dp_kernel<false><<<blocks, kDpWarps * 32, smem, st>>>(p->dc, p->d_items, p->d_c2, p->d_coef, out, p->pp_max);
     CUDA_TRY(p, cudaGetLastError());
@@ -463,12 +471,31 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     if ((s = check_range(p, first, count)) != HAP_OK) return s;
     if (count == 0) return HAP_OK;
     cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
+    CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
     if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     DpOut out{};
+    out.counters = p->d_counters;
     out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
     out.recompute = dev_recompute; out.dp_table = (i64 *)dev_dp_table; out.choice = dev_choice;
     out.first = first; out.count = count;
-    return launch_dp(p, out, false, st);
+    if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
+    p->timed = true;
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_get_timings(hap_problem *p, float *ms_layer_cost, float *ms_dp, uint64_t *cells)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!p->timed) return fail(p, HAP_E_STATE, "no hap_pipeline_dp or hap_search_* call to report on");
+    CUDA_TRY(p, cudaEventSynchronize(p->ev[2]));
+    if (ms_layer_cost) CUDA_TRY(p, cudaEventElapsedTime(ms_layer_cost, p->ev[0], p->ev[1]));
+    if (ms_dp) CUDA_TRY(p, cudaEventElapsedTime(ms_dp, p->ev[1], p->ev[2]));
+    if (cells) CUDA_TRY(p, cudaMemcpy(cells, p->d_counters + 4, sizeof(u64), cudaMemcpyDeviceToHost));
+    return HAP_OK;
 }
 
 extern "C" hap_status hap_argmin(hap_problem *p, const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream)
@@ -507,6 +534,7 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best);
     CUDA_TRY(p, cudaGetLastError());
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
+    p->timed = true;
     i64 best[2];
     u64 counters[4];
     CUDA_TRY(p, cudaMemcpyAsync(best, p->d_best, sizeof(best), cudaMemcpyDeviceToHost, st));

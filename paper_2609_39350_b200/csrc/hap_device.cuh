@@ -62,7 +62,7 @@ struct DpOut {
     // search mode
     i64 *partial_cost;                // [gridDim.x]
     u64 *partial_index;               // [gridDim.x]
-    u64 *counters;                    // [0] evaluated, [1] feasible, [2] pruned
+    u64 *counters;                    // [0] evaluated, [1] feasible, [2] pruned, [4] recurrence cells (nullable)
     u64 *incumbent;                   // running minimum of T_iter, for pruning
     int search, prune;
 };
@@ -525,7 +525,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
     i64 best_cost = kInf;
     u64 best_index = ~0ull;
-    u64 n_eval = 0, n_feas = 0;
+    u64 n_eval = 0, n_feas = 0, n_cells = 0;
 
     for (u64 w = wib; w < it.count; w += kDpWarps) {
         const u64 local = it.lo + w;
@@ -620,6 +620,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                             }
                             // k in [lo, seg_hi] runs at level r
                             const i64 tau = dc.tau_q[r];
+                            n_cells += (u64)(seg_hi - lo + 1);
                             for (int k = seg_hi; k >= lo; --k) {
                                 const i64 pv = prev[k];
                                 const i64 cst = (Cj - rC[k]) + (tau * (Fj - rF[k])) / 1024;
@@ -708,6 +709,10 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         __syncwarp();
     }
 
+    if (out.counters) {
+        n_cells = (u64)warp_sum_i64((i64)n_cells);
+        if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
+    }
     if (SEARCH) {
         __shared__ i64 wcost[kDpWarps];
         __shared__ u64 widx[kDpWarps];

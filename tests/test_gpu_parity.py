@@ -202,7 +202,7 @@ def test_all_infeasible_and_bad_descriptors(hap):
 @pytest.mark.parametrize("seed", range(4))
 def test_random_small_problems_with_tight_memory(hap, seed):
     """Mixed layer kinds, recomputation policies, windows and tight capacities on small random problems."""
-    pb = problems.random_small(seed, N=9 + seed, T=2 + seed % 2, nodes_per_type=(2, 2, 1)[:2 + seed % 2],
+    pb = problems.random_small(seed, N=9 + seed, T=2 + seed % 2, nodes_per_type=((2, 2), (2, 1, 1))[seed % 2],
                                node_size=2, window=(seed % 2 == 0), first_dense=True)
     hp = hap.hap_problem_create(pb)
     hap.hap_enumerate(hp)
