@@ -32,7 +32,10 @@ struct hap_problem {
     std::vector<hap_pconf> pconfs;
     uint64_t n_cand = 0;
     int pp_max = 1;
-    std::vector<WorkItem> items;           // sorted by descending work per candidate
+    std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; };
+    std::vector<PpClass> classes;
+    uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     // device
     DevConst dc{};
     double *d_tables = nullptr;            // all six tables in one allocation
@@ -97,7 +100,7 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 static void release_device(hap_problem *p)
 {
     cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
-    cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
+    cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
 }
 
@@ -269,7 +272,7 @@ static uint64_t sequences_sat(const int *cnt, int T, uint64_t sat)
     return (uint64_t)r;
 }
 
-static double cells_per_candidate(int N, int PP)
+[[maybe_unused]] static double cells_per_candidate(int N, int PP)
 {
     if (PP == 1) return 1.0;
     const double w = N - PP + 1;
@@ -332,27 +335,46 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         if (rows.empty()) return fail(p, HAP_E_INFEASIBLE, "no parallel configuration divides the cluster");
         if (rows.size() > 0xffffffffull) return fail(p, HAP_E_RANGE, "too many configurations");
 
-        // work items: chunks of one configuration's candidates with about equal recurrence work,
-        // heaviest candidates first so that the tail of the grid is made of light blocks
+        // PP classes (heaviest first).  Each class is one launch with its own block shape; a class keeps a
+        // table of its decoded mappings when that table is small.
+        std::vector<int> pps;
+        for (const auto &r : rows) if (std::find(pps.begin(), pps.end(), r.PP) == pps.end()) pps.push_back(r.PP);
+        std::sort(pps.begin(), pps.end(), [](int a, int b) { return a > b; });
         std::vector<WorkItem> items;
-        const double target = 8.0 * 4.0 * cells_per_candidate(N, std::min(pp_max, 8)) + 4096.0;
-        for (size_t pi = 0; pi < rows.size(); ++pi) {
-            const uint64_t total = rows[pi].nmap * (uint64_t)p->opts.n_rc;
-            const double per = cells_per_candidate(N, rows[pi].PP) + 64.0;
-            uint64_t chunk = (uint64_t)std::max(1.0, target / per);
-            chunk = std::max<uint64_t>(chunk, kDpWarps);
-            chunk = std::min<uint64_t>(chunk, 1u << 20);
-            for (uint64_t lo = 0; lo < total; lo += chunk) {
-                WorkItem it; it.p = (uint32_t)pi; it.lo = lo; it.count = (uint32_t)std::min<uint64_t>(chunk, total - lo);
-                items.push_back(it);
+        std::vector<hap_problem::PpClass> classes;
+        u64 tab_bytes = 0;
+        for (int PP : pps) {
+            hap_problem::PpClass cl{};
+            cl.PP = PP;
+            cl.warps = 0;
+            for (int w = kDpWarps; w >= 1; w >>= 1) {
+                cl.smem = dp_smem_bytes(N, PP, T, p->prof.R, w);
+                if (cl.smem <= 227 * 1024) { cl.warps = w; break; }
             }
+            if (!cl.warps) return fail(p, HAP_E_RANGE, "shared memory need %zu of a PP=%d block exceeds the SM", cl.smem, PP);
+            const int slices = std::max(1, cl.warps / p->opts.n_rc);
+            const uint64_t chunk = 64ull * slices;
+            cl.item_lo = items.size();
+            uint64_t nmap = 0;
+            for (size_t pi = 0; pi < rows.size(); ++pi) {
+                if (rows[pi].PP != PP) continue;
+                nmap = rows[pi].nmap;
+                for (uint64_t lo = 0; lo < nmap; lo += chunk) {
+                    WorkItem it; it.p = (uint32_t)pi; it.lo = lo; it.count = (uint32_t)std::min<uint64_t>(chunk, nmap - lo);
+                    items.push_back(it);
+                }
+            }
+            cl.item_hi = items.size();
+            cl.has_tab = nmap * (uint64_t)PP * 2 <= (64ull << 20) && tab_bytes + nmap * PP * 2 <= (256ull << 20);
+            cl.map_base = tab_bytes;
+            if (cl.has_tab) tab_bytes += (nmap * (uint64_t)PP * 2 + 255) / 256 * 256;
+            classes.push_back(cl);
         }
-        std::stable_sort(items.begin(), items.end(), [&](const WorkItem &a, const WorkItem &b) {
-            return rows[a.p].PP > rows[b.p].PP;
-        });
+        if (items.size() > 0x7fffffffull) return fail(p, HAP_E_RANGE, "too many work items");
 
         p->pconfs.swap(rows);
         p->items.swap(items);
+        p->classes.swap(classes);
         p->n_cand = off;
         p->pp_max = pp_max;
         const size_t np = p->pconfs.size();
@@ -370,8 +392,17 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         CUDA_TRY(p, cudaMalloc(&p->d_single, sizeof(SingleOut)));
         p->dc.pconf = p->d_pconf;
         p->dc.n_pconf = np;
-        const size_t smem = dp_smem_bytes(N, pp_max);
-        if (smem > 227 * 1024) return fail(p, HAP_E_RANGE, "shared memory need %zu exceeds the SM", smem);
+        if (tab_bytes) {
+            CUDA_TRY(p, cudaMalloc(&p->d_maptab, tab_bytes));
+            for (const auto &cl : p->classes) {
+                if (!cl.has_tab) continue;
+                const WorkItem &rep = p->items[cl.item_lo];
+                const u64 nmap = p->pconfs[rep.p].nmap;
+                maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128>>>(p->dc, rep.p, nmap, p->d_maptab + cl.map_base);
+                CUDA_TRY(p, cudaGetLastError());
+            }
+            CUDA_TRY(p, cudaDeviceSynchronize());
+        }
         p->enumerated = true;
     }
     if (n_pconf) *n_pconf = p->pconfs.size();
@@ -441,24 +472,32 @@ extern "C" hap_status hap_eval_layer_costs_f64(hap_problem *p, double *dev_c2, d
     return launch_layer_costs(p, nullptr, nullptr, dev_c2, dev_coef, false, (cudaStream_t)stream);
 }
 
-// work items that can intersect the candidate range: all of them (each block clips); the
-// full-range case is the hot one
+// One launch per PP class (each has its own block shape); every block clips to the candidate range.
 static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaStream_t st)
 {
-    const size_t smem = dp_smem_bytes(p->model.N, p->pp_max);
-    const unsigned blocks = (unsigned)p->items.size();
     // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
     // process: raise it (never lower it) before a launch that needs more
     static size_t smem_limit[64][2];
     const int dev = p->device & 63;
-    if (smem > smem_limit[dev][search]) {
-        if (search) CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        else CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        smem_limit[dev][search] = smem;
+    for (const auto &cl : p->classes) {
+        // skip classes whose candidates all lie outside the range
+        const WorkItem &a = p->items[cl.item_lo], &b = p->items[cl.item_hi - 1];
+        const u64 c0 = p->pconfs[a.p].offset, c1 = p->pconfs[b.p].offset + p->pconfs[b.p].nmap * (u64)p->opts.n_rc;
+        const bool outside = c1 <= out.first || c0 >= out.first + out.count;
+        if (outside && !search) continue;
+        if (cl.smem > smem_limit[dev][search]) {
+            if (search) CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl.smem));
+            else CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl.smem));
+            smem_limit[dev][search] = cl.smem;
+        }
+        const unsigned blocks = (unsigned)(cl.item_hi - cl.item_lo);
+        const uint8_t *tab = cl.has_tab ? p->d_maptab + cl.map_base : nullptr;
+        DpOut o = out;
+        if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
+        if (search) pipeline_dp_kernel<true><<<blocks, cl.warps * 32, cl.smem, st>>>(p->dc, p->d_items + cl.item_lo, p->d_c2, p->d_coef, tab, o, cl.warps);
+        else pipeline_dp_kernel<false><<<blocks, cl.warps * 32, cl.smem, st>>>(p->dc, p->d_items + cl.item_lo, p->d_c2, p->d_coef, tab, o, cl.warps);
+        CUDA_TRY(p, cudaGetLastError());
     }
-    if (search) pipeline_dp_kernel<true><<<blocks, kDpWarps * 32, smem, st>>>(p->dc, p->d_items, p->d_c2, p->d_coef, out, p->pp_max);
-    else pipeline_dp_kernel<false><<<blocks, kDpWarps * 32, smem, st>>>(p->dc, p->d_items, p->d_c2, p->d_coef, out, p->pp_max);
-    CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
 }
 

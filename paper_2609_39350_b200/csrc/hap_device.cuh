@@ -19,6 +19,7 @@ namespace hap {
 
 typedef long long i64;
 typedef unsigned long long u64;
+typedef unsigned int u32;
 
 constexpr int kMaxMasks = (1 << HAP_MAX_TYPES) - 1;
 constexpr int kDpWarps = 8;           // warps per block of the DP kernel
@@ -45,7 +46,7 @@ struct DevConst {
     u64 n_pconf;
 };
 
-// One block of DP work: candidates [lo, lo+count) (local to configuration p).
+// One block of DP work: mappings [lo, lo+count) of configuration p, every recompute policy.
 struct WorkItem {
     uint32_t p;
     uint32_t count;
@@ -416,53 +417,71 @@ __global__ void decode_kernel(const DevConst dc, u64 first, u64 count, hap_candi
 }
 
 // ------------------------------------------------------------------------------------------
-// pipeline DP
+// mapping table: decoded (mask, link) byte pairs per stage for every mapping of one PP class,
+// built once per problem so that the DP kernel does not unrank per candidate
 // ------------------------------------------------------------------------------------------
-struct DpSmem {
-    i64 *sC;      // [kMaxMasks][N+1] prefix of forward+backward per type mask
-    i64 *sF;      // [kMaxMasks][N+1] prefix of forward per type mask
-    i64 *sW;      // [N+1] prefix of weight bytes
-    i64 *sA;      // [N+1] prefix of activation bytes per stored micro-batch
-    i64 *rows;    // per warp: prev[N+1], cur[N+1]
-    uint8_t *ch;  // per warp: [PPmax][N+1]
-};
-
-__host__ __device__ inline size_t dp_smem_bytes(int N, int PPmax)
+__global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *tab)
 {
-    const size_t n1 = (size_t)N + 1;
-    size_t b = (size_t)kMaxMasks * n1 * 8 * 2 + n1 * 8 * 2 + (size_t)kDpWarps * n1 * 8 * 2;
-    size_t chb = ((size_t)PPmax * n1 + 15) / 16 * 16;
-    return b + (size_t)kDpWarps * chb + 64;
+    const u64 w = ((u64)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= nmap) return;
+    const hap_pconf pc = dc.pconf[p_rep];
+    const StageMap sm = decode_stage(dc, pc, w, lane);
+    if (lane < pc.PP) {
+        uint8_t *o = tab + (w * (u64)pc.PP + lane) * 2;
+        o[0] = (uint8_t)sm.mask;
+        o[1] = (uint8_t)(lane > 0 ? (sm.cls | (sm.ha << 2) | (sm.hb << 4)) : 0);
+    }
 }
 
-// cost of one stage span (a, b] for the lane's own stage; used in the backtrace
+// ------------------------------------------------------------------------------------------
+// pipeline DP
+// ------------------------------------------------------------------------------------------
+// Shared memory of one block (all candidates of a block belong to one configuration):
+//   sC, sF   [kMaxMasks][N+1]  prefix sums of forward+backward / forward time per type mask
+//   sW, sA   [N+1]             prefix sums of weight bytes / activation bytes per micro-batch
+//   thr      [PP][T][R][N+1]   u8: first split k for which stage i on a device of capacity type t
+//                              fits layers (k, j] at recomputation level r (j = none)
+//   per warp: rows [(PP+1)][N+1] i64 (one DP row per stage, kept so that the next mapping can reuse
+//             the rows of the stage prefix it shares), ch [PP][N+1] u8 split choices
+__host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int warps)
+{
+    const size_t n1 = (size_t)N + 1;
+    size_t b = (size_t)kMaxMasks * n1 * 16 + n1 * 16;
+    b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    b += (size_t)warps * (((size_t)(PP + 1) * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
+    return b + 32;
+}
+
 struct StagePar {
-    int mask, first, last;      // first / last: stage 1 / stage PP flags
-    i64 cap, K, mstore;
-    int nmin, nmax;
+    int mask, capt;             // type mask; index of the type whose capacity binds
+    i64 K;                      // stage constant: pre/post work + p2p transfer into the stage
+    int nmin, nmax;             // load-balance window on the layer count
+    int bl, bh;                 // band of end layers j that can be reached at this stage
 };
 
-__device__ __forceinline__ bool span_fits(const DevConst &dc, const i64 *sW, const i64 *sA, const StagePar &sp,
-                                          i64 extra, i64 mx, int a, int b, int r)
+__device__ __forceinline__ bool span_fits(const DevConst &dc, const i64 *sW, const i64 *sA, i64 extra, i64 mx,
+                                          i64 mstore, i64 cap, int a, int b, int r)
 {
     const bool has_moe = moe_before(dc, b) - moe_before(dc, a) > 0;
     const i64 Wb = (sW[b] - sW[a]) + extra + (has_moe ? mx : 0);
-    const i64 A = sp.mstore * (sA[b] - sA[a]);
-    return Wb + ((i64)dc.xi_q[r] * A) / 1024 <= sp.cap;
+    const i64 A = mstore * (sA[b] - sA[a]);
+    return Wb + ((i64)dc.xi_q[r] * A) / 1024 <= cap;
 }
 
 template <bool SEARCH>
 __global__ void __launch_bounds__(kDpWarps * 32)
-pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef, DpOut out, int PPmax)
+pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef,
+                   const uint8_t *maptab, DpOut out, int nwarps)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int N = dc.N, T = dc.T, n1 = N + 1;
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const WorkItem it = items[blockIdx.x];
     const hap_pconf pc = dc.pconf[it.p];
-    const int PP = pc.PP;
+    const int PP = pc.PP, n_rc = dc.n_rc;
     {   // blocks whose candidates all lie outside the requested range have nothing to do
-        const u64 c0 = pc.offset + it.lo, c1 = c0 + it.count;
+        const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
         if (c1 <= out.first || c0 >= out.first + out.count) {
             if (SEARCH && threadIdx.x == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
             return;
@@ -473,16 +492,22 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     i64 *sF = sC + (size_t)kMaxMasks * n1;
     i64 *sW = sF + (size_t)kMaxMasks * n1;
     i64 *sA = sW + n1;
-    i64 *rows = sA + n1 + (size_t)wib * 2 * n1;
-    const size_t chb = ((size_t)PPmax * n1 + 15) / 16 * 16;
-    uint8_t *chw = reinterpret_cast<uint8_t *>(sA + n1 + (size_t)kDpWarps * 2 * n1) + (size_t)wib * chb;
+    uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
+    const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    const size_t row_bytes = (size_t)(PP + 1) * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
+    unsigned char *wbase = thr + thr_bytes + (size_t)wib * (row_bytes + ch_bytes);
+    i64 *rows = reinterpret_cast<i64 *>(wbase);
+    uint8_t *chw = wbase + row_bytes;
 
-    // ---- block prologue: rows of this configuration ------------------------------------
+    // ---- block prologue 1: rows of this configuration -----------------------------------
     const i64 *c2p = c2 + (size_t)it.p * T * N * 2;
     const i64 *cfp = coef + (size_t)it.p * T * HAP_NCOEF;
     const int nmask = (1 << T) - 1;
-    for (int mk = 1 + wib; mk <= nmask + 1; mk += kDpWarps) {
-        // masks 1..nmask: time rows; the extra round (mk == nmask+1) builds the byte rows
+    const bool multiset = pc.mode == HAP_MAP_MULTISET;
+    for (int mk = 1 + wib; mk <= nmask + 1; mk += nwarps) {
+        // masks 1..nmask: time rows (homogeneous stages need the single-type masks only);
+        // the extra round (mk == nmask+1) builds the byte rows
+        if (mk <= nmask && multiset && (mk & (mk - 1))) continue;
         i64 runC = 0, runF = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
@@ -502,9 +527,8 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                     vC = cfp[HAP_MW + kd]; vF = cfp[HAP_MA + kd];
                 }
             }
-            // inclusive warp scan
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
+            for (int o = 1; o < 32; o <<= 1) {      // inclusive warp scan
                 const i64 tC = __shfl_up_sync(0xffffffffu, vC, o), tF = __shfl_up_sync(0xffffffffu, vF, o);
                 if (lane >= o) { vC += tC; vF += tF; }
             }
@@ -522,103 +546,182 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     }
     __syncthreads();
 
+    // ---- block prologue 2: memory thresholds ----------------------------------------------
+    // Feasibility of a span (k, j] is monotone: a shorter span needs no more memory, and the first
+    // feasible k does not decrease with j.  One thread sweeps j for one (stage, capacity type, level).
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
+    for (int q = threadIdx.x; q < PP * T * R; q += nwarps * 32) {
+        const int r = q % R, t = (q / R) % T, i = q / (R * T) + 1;
+        const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
+        const int inflight = PP - i + 1;
+        const i64 mstore = pc.M < inflight ? pc.M : inflight;
+        const i64 cap = dc.cap_eff[t];
+        uint8_t *row = thr + (size_t)q * n1;
+        int k = 0;
+        row[0] = 0;
+        for (int j = 1; j <= N; ++j) {
+            while (k < j && !span_fits(dc, sW, sA, extra, mx, mstore, cap, k, j, r)) ++k;
+            row[j] = (uint8_t)k;
+        }
+    }
+    // load-balance window per device type when every mapping uses the same multiset of stage types
+    __shared__ int winT[HAP_MAX_TYPES][2];
+    if (threadIdx.x < T) {
+        int lo = 1, hi = N - PP + 1;
+        if (dc.delta_q >= 0 && multiset) {
+            i64 Ps = 0;
+            for (int h = 0; h < T; ++h) Ps += (dc.m[h] / pc.G) * dc.P[h];
+            const i64 den = 1024 * Ps, Ph = dc.P[threadIdx.x];
+            i64 a = ((i64)(1024 - dc.delta_q) * Ph * N) / den;
+            i64 b = ((i64)(1024 + dc.delta_q) * Ph * N + den - 1) / den;
+            lo = a < 1 ? 1 : (int)a;
+            hi = b > N - PP + 1 ? N - PP + 1 : (int)b;
+        }
+        winT[threadIdx.x][0] = lo; winT[threadIdx.x][1] = hi;
+    }
+    __syncthreads();
+
     i64 best_cost = kInf;
     u64 best_index = ~0ull;
     u64 n_eval = 0, n_feas = 0, n_cells = 0;
+    const bool want_tables = !SEARCH && (out.dp_table != nullptr || out.choice != nullptr);
 
-    for (u64 w = wib; w < it.count; w += kDpWarps) {
-        const u64 local = it.lo + w;
-        const u64 c = pc.offset + local;
-        if (c < out.first || c >= out.first + out.count) continue;
-        const u64 map_idx = local / (u64)dc.n_rc;
-        const unsigned rc_mask = dc.rc_masks[(int)(local - map_idx * (u64)dc.n_rc)];
-        const StageMap smap = decode_stage(dc, pc, map_idx, lane);
+    // warp -> (recompute policy, slice of consecutive mappings); consecutive mappings share a prefix of
+    // stage types, and the DP rows of a shared prefix are reused
+    const int slices = nwarps / n_rc > 0 ? nwarps / n_rc : 1;
+    const int my_rc = wib % n_rc, my_slice = wib / n_rc;
+    const bool active_warp = wib < slices * n_rc || n_rc > nwarps;
+    const u32 per_slice = (it.count + slices - 1) / slices;
+    for (int rc_idx = my_rc; rc_idx < n_rc && active_warp; rc_idx += nwarps) {
+      const unsigned rc_mask = dc.rc_masks[rc_idx];
+      const u32 m_lo = (u32)my_slice * per_slice;
+      const u32 m_hi = m_lo + per_slice < it.count ? m_lo + per_slice : it.count;
+      int valid_rows = 0;                  // rows[0..valid_rows] hold the DP of the previous mapping's prefix
+      int prev_mask = -1, prev_link = -1;
+      for (u32 mi = m_lo; mi < m_hi; ++mi) {
+        const u64 map_idx = it.lo + mi;
+        const u64 c = pc.offset + map_idx * (u64)n_rc + (u64)rc_idx;
+        if (c < out.first || c >= out.first + out.count) { valid_rows = 0; prev_mask = -1; continue; }
 
-        // ---- per-stage parameters, lane s holds stage s+1 ---------------------------------
+        // ---- stage types of this mapping, lane s holds stage s+1 -----------------------------
+        int mask = 0, link = 0;
+        if (maptab) {
+            if (lane < PP) {
+                const uchar2 ml = *reinterpret_cast<const uchar2 *>(maptab + (map_idx * (u64)PP + lane) * 2);
+                mask = ml.x; link = ml.y;
+            }
+        } else {
+            const StageMap smap = decode_stage(dc, pc, map_idx, lane);
+            mask = smap.mask; link = lane > 0 && lane < PP ? (smap.cls | (smap.ha << 2) | (smap.hb << 4)) : 0;
+        }
+        const unsigned differ = __ballot_sync(0xffffffffu, lane < PP && (mask != prev_mask || link != prev_link));
+        int s0 = differ ? __ffs(differ) - 1 : PP;      // stages 1..s0 are shared with the previous mapping
+        prev_mask = mask; prev_link = link;
+
         StagePar sp;
-        sp.mask = smap.mask; sp.first = lane == 0; sp.last = lane == PP - 1;
-        sp.cap = 0; sp.K = 0; sp.mstore = 0; sp.nmin = 1; sp.nmax = N - PP + 1;
+        sp.mask = mask; sp.capt = 0; sp.K = 0; sp.nmin = 1; sp.nmax = N - PP + 1; sp.bl = 0; sp.bh = 0;
         i64 Pmin = 0;
         if (lane < PP) {
-            i64 kpre = 0, kpost = 0;
+            i64 kpre = 0, kpost = 0, cap = 0;
             bool seen = false;
             for (int h = 0; h < T; ++h)
-                if (smap.mask >> h & 1) {
+                if (mask >> h & 1) {
                     const i64 *row = cfp + h * HAP_NCOEF;
-                    if (!seen || dc.cap_eff[h] < sp.cap) sp.cap = dc.cap_eff[h];
+                    if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; sp.capt = h; }
                     if (!seen || dc.P[h] < Pmin) Pmin = dc.P[h];
                     if (!seen || row[HAP_KPRE] > kpre) kpre = row[HAP_KPRE];
                     if (!seen || row[HAP_KPOST] > kpost) kpost = row[HAP_KPOST];
                     seen = true;
                 }
-            if (sp.first) sp.K += kpre;
-            if (sp.last) sp.K += kpost;
+            if (lane == 0) sp.K += kpre;
+            if (lane == PP - 1) sp.K += kpost;
             if (lane > 0) {
-                const i64 *row = cfp + smap.hb * HAP_NCOEF;
-                sp.K += smap.cls == HAP_INTRA ? row[HAP_KP2P_INTRA]
-                        : (smap.cls == HAP_INTER ? row[HAP_KP2P_INTER] : row[HAP_KP2P_CROSS + smap.ha]);
+                const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3;
+                const i64 *row = cfp + hb * HAP_NCOEF;
+                sp.K += cls == HAP_INTRA ? row[HAP_KP2P_INTRA] : (cls == HAP_INTER ? row[HAP_KP2P_INTER] : row[HAP_KP2P_CROSS + ha]);
             }
-            const int inflight = PP - lane;                 // PP - i + 1 with i = lane + 1
-            sp.mstore = pc.M < inflight ? pc.M : inflight;
         }
         if (dc.delta_q >= 0) {
-            const i64 Ps = warp_sum_i64(lane < PP ? Pmin : 0);
-            if (lane < PP) {
-                const i64 den = 1024 * Ps;
-                i64 lo = ((i64)(1024 - dc.delta_q) * Pmin * N) / den;
-                i64 hi = ((i64)(1024 + dc.delta_q) * Pmin * N + den - 1) / den;
-                if (lo < 1) lo = 1;
-                if (hi > N - PP + 1) hi = N - PP + 1;
-                sp.nmin = (int)lo; sp.nmax = (int)hi;
+            if (multiset) {
+                if (lane < PP) { sp.nmin = winT[__ffs(mask) - 1][0]; sp.nmax = winT[__ffs(mask) - 1][1]; }   // homogeneous stage: its one type
+            } else {
+                s0 = 0;                              // the window depends on the whole mapping: nothing is shared
+                const i64 Ps = warp_sum_i64(lane < PP ? Pmin : 0);
+                if (lane < PP) {
+                    const i64 den = 1024 * Ps;
+                    i64 lo = ((i64)(1024 - dc.delta_q) * Pmin * N) / den;
+                    i64 hi = ((i64)(1024 + dc.delta_q) * Pmin * N + den - 1) / den;
+                    if (lo < 1) lo = 1;
+                    if (hi > N - PP + 1) hi = N - PP + 1;
+                    sp.nmin = (int)lo; sp.nmax = (int)hi;
+                }
             }
         }
+        if (!multiset) s0 = 0;
+        if (s0 > valid_rows) s0 = valid_rows;
+        if (want_tables) s0 = 0;
 
-        // ---- recurrence ------------------------------------------------------------------
-        i64 *prev = rows, *cur = rows + n1;
-        for (int j = lane; j <= N; j += 32) prev[j] = j == 0 ? 0 : kInf;
-        if (out.dp_table && !SEARCH) {
-            i64 *t = out.dp_table + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
-            for (int j = lane; j <= N; j += 32) t[j] = j == 0 ? 0 : kInf;
+        // ---- bands: end layers j that stage i can reach (prefix sums of the window bounds), and from
+        //      which the remaining stages can still reach N (suffix sums; not applied when the caller
+        //      wants the full tables, where such cells hold finite values)
+        {
+            int smin = lane < PP ? sp.nmin : 0, smax = lane < PP ? sp.nmax : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int a = __shfl_up_sync(0xffffffffu, smin, o), b = __shfl_up_sync(0xffffffffu, smax, o);
+                if (lane >= o) { smin += a; smax += b; }
+            }
+            const int tmin = __shfl_sync(0xffffffffu, smin, PP - 1), tmax = __shfl_sync(0xffffffffu, smax, PP - 1);
+            const int i = lane + 1;
+            int bl = smin > i ? smin : i, bh = smax < N - PP + i ? smax : N - PP + i;
+            if (!want_tables) {
+                const int rl = N - (tmax - smax), rh = N - (tmin - smin);   // remaining stages take [tmin-smin, tmax-smax]
+                bl = bl > rl ? bl : rl; bh = bh < rh ? bh : rh;
+            }
+            sp.bl = bl; sp.bh = bh;
         }
-        if (out.choice && !SEARCH) {
-            uint8_t *t = out.choice + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
-            for (int j = lane; j <= N; j += 32) t[j] = 255;
-        }
-        __syncwarp();
-        for (int i = 1; i <= PP; ++i) {
-            const int src = i - 1;
-            const int mask = __shfl_sync(0xffffffffu, sp.mask, src);
-            const i64 cap = shfl_i64(sp.cap, src), K = shfl_i64(sp.K, src), mstore = shfl_i64(sp.mstore, src);
-            const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
-            const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
-            const i64 *rC = sC + (size_t)(mask - 1) * n1, *rF = sF + (size_t)(mask - 1) * n1;
-            uint8_t *chrow = chw + (size_t)(i - 1) * n1;
-            const int jlo = i, jhi = N - PP + i;
+        const bool dead = __any_sync(0xffffffffu, lane < PP && sp.bl > sp.bh);
+
+        // ---- recurrence -------------------------------------------------------------------
+        i64 *tab_out = nullptr; uint8_t *ch_out = nullptr;
+        if (want_tables) {
+            if (out.dp_table) tab_out = out.dp_table + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
+            if (out.choice) ch_out = out.choice + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
             for (int j = lane; j <= N; j += 32) {
-                i64 best = kInf;
-                int arg = 255;
-                if (j >= jlo && j <= jhi) {
-                    int klo = j - nmax; if (klo < i - 1) klo = i - 1;
-                    const int khi = j - nmin;                 // nmin >= 1 keeps k <= j-1
+                if (tab_out) tab_out[j] = j == 0 ? 0 : kInf;
+                if (ch_out) ch_out[j] = 255;
+            }
+        }
+        if (s0 == 0 && lane == 0) rows[0] = 0;           // DP[0][0] = 0; the band of stage 0 is {0}
+        __syncwarp();
+        i64 bott = kInf;
+        if (!dead || want_tables) {
+            int pbl = 0, pbh = 0;                          // band of the previous stage
+            if (s0 > 0) { pbl = __shfl_sync(0xffffffffu, sp.bl, s0 - 1); pbh = __shfl_sync(0xffffffffu, sp.bh, s0 - 1); }
+            for (int i = s0 + 1; i <= PP; ++i) {
+                const int src = i - 1;
+                const int smask = __shfl_sync(0xffffffffu, sp.mask, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
+                const i64 K = shfl_i64(sp.K, src);
+                const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
+                const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
+                const i64 *rC = sC + (size_t)(smask - 1) * n1, *rF = sF + (size_t)(smask - 1) * n1;
+                const i64 *prev = rows + (size_t)(i - 1) * n1;
+                i64 *cur = rows + (size_t)i * n1;
+                uint8_t *chrow = chw + (size_t)(i - 1) * n1;
+                const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
+                for (int j = bl + lane; j <= bh; j += 32) {
+                    i64 best = kInf;
+                    int arg = 255;
+                    int klo = j - nmax; if (klo < pbl) klo = pbl;
+                    int khi = j - nmin; if (khi > pbh) khi = pbh;
                     if (klo <= khi) {
-                        const i64 Cj = rC[j] + K, Fj = rF[j], Wj = sW[j] + extra, Aj = sA[j];
-                        const int moe_j = moe_before(dc, j);
-                        // feasibility is monotone in k (shorter spans need less memory): for each allowed
-                        // level find the first feasible k; levels are ordered so that these thresholds do
-                        // not increase with the level
-                        int seg_hi = khi;                      // k range still to be assigned a level
-                        for (int r = 0; r < dc.R && seg_hi >= klo; ++r) {
+                        const i64 Cj = rC[j] + K, Fj = rF[j];
+                        int seg_hi = khi;                     // k range still to be assigned a level
+                        for (int r = 0; r < R && seg_hi >= klo; ++r) {
                             if (!((rc_mask >> r) & 1u)) continue;
-                            int lo = klo, hi = seg_hi + 1;     // first feasible k in [klo, seg_hi+1]
-                            while (lo < hi) {
-                                const int mid = (lo + hi) >> 1;
-                                const bool has_moe = moe_j - moe_before(dc, mid) > 0;
-                                const i64 Wb = (Wj - sW[mid]) + (has_moe ? mx : 0);
-                                const i64 A = mstore * (Aj - sA[mid]);
-                                if (Wb + ((i64)dc.xi_q[r] * A) / 1024 <= cap) hi = mid; else lo = mid + 1;
-                            }
-                            // k in [lo, seg_hi] runs at level r
+                            int lo = th[(size_t)r * n1 + j];   // first k that fits at level r
+                            if (lo < klo) lo = klo;
+                            if (lo > seg_hi) continue;
                             const i64 tau = dc.tau_q[r];
                             n_cells += (u64)(seg_hi - lo + 1);
                             for (int k = seg_hi; k >= lo; --k) {
@@ -630,24 +733,26 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                             seg_hi = lo - 1;
                         }
                     }
+                    cur[j] = best;
+                    chrow[j] = (uint8_t)arg;
                 }
-                cur[j] = best;
-                chrow[j] = (uint8_t)arg;
+                __syncwarp();
+                if (want_tables) {
+                    for (int j = lane; j <= N; j += 32) {
+                        const bool in = j >= bl && j <= bh;
+                        if (tab_out) tab_out[(size_t)i * n1 + j] = in ? cur[j] : kInf;
+                        if (ch_out) ch_out[(size_t)i * n1 + j] = in ? chrow[j] : (uint8_t)255;
+                    }
+                }
+                pbl = bl; pbh = bh;
             }
-            __syncwarp();
-            if (!SEARCH) {
-                if (out.dp_table) {
-                    i64 *t = out.dp_table + ((size_t)(c - out.first) * (HAP_MAX_PP + 1) + i) * n1;
-                    for (int j = lane; j <= N; j += 32) t[j] = cur[j];
-                }
-                if (out.choice) {
-                    uint8_t *t = out.choice + ((size_t)(c - out.first) * (HAP_MAX_PP + 1) + i) * n1;
-                    for (int j = lane; j <= N; j += 32) t[j] = chrow[j];
-                }
-            }
-            i64 *tmp = prev; prev = cur; cur = tmp;
+            valid_rows = dead ? 0 : PP;
+            // N lies in the last band unless the windows cannot add up to N (possible only without the
+            // suffix restriction, i.e. when tables are written)
+            if (!dead && pbl <= N && N <= pbh) bott = rows[(size_t)PP * n1 + N];
+        } else {
+            valid_rows = 0;
         }
-        const i64 bott = prev[N];
         __syncwarp();
 
         // ---- backtrace, Eq. 4 -----------------------------------------------------------
@@ -663,10 +768,10 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             }
             i64 c_me = 0, sync_me = 0, opt_me = 0;
             if (lane < PP) {
-                const i64 extra = (sp.first ? mpre : 0) + (sp.last ? mpost : 0);
+                const uint8_t *th = thr + ((size_t)lane * T + sp.capt) * R * n1;
                 int r = 0;
-                for (; r < dc.R; ++r)
-                    if (((rc_mask >> r) & 1u) && span_fits(dc, sW, sA, sp, extra, mx, a_me, b_me, r)) break;
+                for (; r < R; ++r)
+                    if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b_me] <= a_me) break;
                 const i64 *rC = sC + (size_t)(sp.mask - 1) * n1, *rF = sF + (size_t)(sp.mask - 1) * n1;
                 c_me = (rC[b_me] - rC[a_me]) + ((i64)dc.tau_q[r] * (rF[b_me] - rF[a_me])) / 1024 + sp.K;
                 my_n = b_me - a_me; my_r = r;
@@ -707,6 +812,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             if (out.recompute) out.recompute[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < kInf ? my_r : 0);
         }
         __syncwarp();
+      }
     }
 
     if (out.counters) {
@@ -724,7 +830,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         __syncthreads();
         if (threadIdx.x == 0) {
             i64 bc = wcost[0]; u64 bi = widx[0];
-            for (int q = 1; q < kDpWarps; ++q)
+            for (int q = 1; q < nwarps; ++q)
                 if (wcost[q] < bc || (wcost[q] == bc && widx[q] < bi)) { bc = wcost[q]; bi = widx[q]; }
             out.partial_cost[blockIdx.x] = bc;
             out.partial_index[blockIdx.x] = bi;
