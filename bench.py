@@ -144,6 +144,7 @@ def main():
     ap.add_argument("--workload", default="stress")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--delta-q", type=int, default=None, help="override the load-balance window (1/1024; <0 = off)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -166,6 +167,8 @@ def main():
     warmup = max(args.warmup, 3)
 
     pb = problems.make_problem(args.workload)
+    if args.delta_q is not None:
+        pb.delta_q = args.delta_q
     hp = hap.hap_problem_create(pb)
     n_pconf, n_cand = hap.hap_enumerate(hp)
     pconfs = hap.hap_get_pconfs(hp)

@@ -442,6 +442,7 @@ __global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *t
 //   sW, sA   [N+1]             prefix sums of weight bytes / activation bytes per micro-batch
 //   thr      [PP][T][R][N+1]   u8: first split k for which stage i on a device of capacity type t
 //                              fits layers (k, j] at recomputation level r (j = none)
+//   sK       [N+1]             u8: number of MoE layers among the first l layers
 //   per warp: rows [(PP+1)][N+1] i64 (one DP row per stage, kept so that the next mapping can reuse
 //             the rows of the stage prefix it shares), ch [PP][N+1] u8 split choices
 __host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int warps)
@@ -449,6 +450,7 @@ __host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int
     const size_t n1 = (size_t)N + 1;
     size_t b = (size_t)kMaxMasks * n1 * 16 + n1 * 16;
     b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    b += (n1 + 15) / 16 * 16;                                   // MoE-layer prefix counts
     b += (size_t)warps * (((size_t)(PP + 1) * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
     return b + 32;
 }
@@ -460,14 +462,21 @@ struct StagePar {
     int bl, bh;                 // band of end layers j that can be reached at this stage
 };
 
-__device__ __forceinline__ bool span_fits(const DevConst &dc, const i64 *sW, const i64 *sA, i64 extra, i64 mx,
-                                          i64 mstore, i64 cap, int a, int b, int r)
+__device__ __forceinline__ bool span_fits(const i64 *sW, const i64 *sA, const uint8_t *sK, i64 extra, i64 mx,
+                                          i64 mstore, i64 cap, i64 xi, int a, int b)
 {
-    const bool has_moe = moe_before(dc, b) - moe_before(dc, a) > 0;
+    const bool has_moe = sK[b] != sK[a];
     const i64 Wb = (sW[b] - sW[a]) + extra + (has_moe ? mx : 0);
     const i64 A = mstore * (sA[b] - sA[a]);
-    return Wb + ((i64)dc.xi_q[r] * A) / 1024 <= cap;
+    return Wb + ((xi * A) >> 10) <= cap;               // A >= 0: the shift is the floor division by 1024
 }
+
+// per type mask: what a stage made of these device types costs beyond its layers (slowest member),
+// which member's memory binds, and the slowest member's compute rate for the load-balance window
+struct MaskInfo {
+    i64 kpre, kpost, slat, sbw[2], opt[2], Pmin;
+    int capt, pad;
+};
 
 template <bool SEARCH>
 __global__ void __launch_bounds__(kDpWarps * 32)
@@ -494,8 +503,10 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     i64 *sA = sW + n1;
     uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
     const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    uint8_t *sK = thr + thr_bytes;
     const size_t row_bytes = (size_t)(PP + 1) * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
-    unsigned char *wbase = thr + thr_bytes + (size_t)wib * (row_bytes + ch_bytes);
+    unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
+    __shared__ MaskInfo minfo[kMaxMasks];
     i64 *rows = reinterpret_cast<i64 *>(wbase);
     uint8_t *chw = wbase + row_bytes;
 
@@ -544,6 +555,29 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             else { sW[0] = 0; sA[0] = 0; }
         }
     }
+    for (int l = threadIdx.x; l <= N; l += nwarps * 32) sK[l] = (uint8_t)moe_before(dc, l);
+    if (threadIdx.x < nmask) {
+        const int mk = threadIdx.x + 1;
+        MaskInfo mi;
+        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
+        i64 cap = 0;
+        bool seen = false;
+        for (int h = 0; h < T; ++h)
+            if (mk >> h & 1) {
+                const i64 *row = cfp + h * HAP_NCOEF;
+                if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; mi.capt = h; }
+                if (!seen || dc.P[h] < mi.Pmin) mi.Pmin = dc.P[h];
+                if (!seen || row[HAP_KPRE] > mi.kpre) mi.kpre = row[HAP_KPRE];
+                if (!seen || row[HAP_KPOST] > mi.kpost) mi.kpost = row[HAP_KPOST];
+                if (!seen || row[HAP_SLAT] > mi.slat) mi.slat = row[HAP_SLAT];
+                if (!seen || row[HAP_SBW] > mi.sbw[0]) mi.sbw[0] = row[HAP_SBW];
+                if (!seen || row[HAP_SBW + 1] > mi.sbw[1]) mi.sbw[1] = row[HAP_SBW + 1];
+                if (!seen || row[HAP_OPT] > mi.opt[0]) mi.opt[0] = row[HAP_OPT];
+                if (!seen || row[HAP_OPT + 1] > mi.opt[1]) mi.opt[1] = row[HAP_OPT + 1];
+                seen = true;
+            }
+        minfo[threadIdx.x] = mi;
+    }
     __syncthreads();
 
     // ---- block prologue 2: memory thresholds ----------------------------------------------
@@ -555,12 +589,12 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
         const int inflight = PP - i + 1;
         const i64 mstore = pc.M < inflight ? pc.M : inflight;
-        const i64 cap = dc.cap_eff[t];
+        const i64 cap = dc.cap_eff[t], xi = dc.xi_q[r];
         uint8_t *row = thr + (size_t)q * n1;
         int k = 0;
         row[0] = 0;
         for (int j = 1; j <= N; ++j) {
-            while (k < j && !span_fits(dc, sW, sA, extra, mx, mstore, cap, k, j, r)) ++k;
+            while (k < j && !span_fits(sW, sA, sK, extra, mx, mstore, cap, xi, k, j)) ++k;
             row[j] = (uint8_t)k;
         }
     }
@@ -622,19 +656,10 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         sp.mask = mask; sp.capt = 0; sp.K = 0; sp.nmin = 1; sp.nmax = N - PP + 1; sp.bl = 0; sp.bh = 0;
         i64 Pmin = 0;
         if (lane < PP) {
-            i64 kpre = 0, kpost = 0, cap = 0;
-            bool seen = false;
-            for (int h = 0; h < T; ++h)
-                if (mask >> h & 1) {
-                    const i64 *row = cfp + h * HAP_NCOEF;
-                    if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; sp.capt = h; }
-                    if (!seen || dc.P[h] < Pmin) Pmin = dc.P[h];
-                    if (!seen || row[HAP_KPRE] > kpre) kpre = row[HAP_KPRE];
-                    if (!seen || row[HAP_KPOST] > kpost) kpost = row[HAP_KPOST];
-                    seen = true;
-                }
-            if (lane == 0) sp.K += kpre;
-            if (lane == PP - 1) sp.K += kpost;
+            const MaskInfo &mi = minfo[mask - 1];
+            sp.capt = mi.capt; Pmin = mi.Pmin;
+            if (lane == 0) sp.K += mi.kpre;
+            if (lane == PP - 1) sp.K += mi.kpost;
             if (lane > 0) {
                 const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3;
                 const i64 *row = cfp + hb * HAP_NCOEF;
@@ -726,7 +751,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                             n_cells += (u64)(seg_hi - lo + 1);
                             for (int k = seg_hi; k >= lo; --k) {
                                 const i64 pv = prev[k];
-                                const i64 cst = (Cj - rC[k]) + (tau * (Fj - rF[k])) / 1024;
+                                const i64 cst = (Cj - rC[k]) + ((tau * (Fj - rF[k])) >> 10);   // forward sums are non-negative
                                 const i64 v = pv > cst ? pv : cst;
                                 if (v <= best && v < kInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
                             }
@@ -773,23 +798,12 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 for (; r < R; ++r)
                     if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b_me] <= a_me) break;
                 const i64 *rC = sC + (size_t)(sp.mask - 1) * n1, *rF = sF + (size_t)(sp.mask - 1) * n1;
-                c_me = (rC[b_me] - rC[a_me]) + ((i64)dc.tau_q[r] * (rF[b_me] - rF[a_me])) / 1024 + sp.K;
+                c_me = (rC[b_me] - rC[a_me]) + (((i64)dc.tau_q[r] * (rF[b_me] - rF[a_me])) >> 10) + sp.K;
                 my_n = b_me - a_me; my_r = r;
-                const i64 n_moe = moe_before(dc, b_me) - moe_before(dc, a_me), n_dense = (b_me - a_me) - n_moe;
-                i64 slat = 0, sbd = 0, sbm = 0, opd = 0, opm = 0;
-                bool seen = false;
-                for (int h = 0; h < T; ++h)
-                    if (sp.mask >> h & 1) {
-                        const i64 *row = cfp + h * HAP_NCOEF;
-                        if (!seen || row[HAP_SLAT] > slat) slat = row[HAP_SLAT];
-                        if (!seen || row[HAP_SBW] > sbd) sbd = row[HAP_SBW];
-                        if (!seen || row[HAP_SBW + 1] > sbm) sbm = row[HAP_SBW + 1];
-                        if (!seen || row[HAP_OPT] > opd) opd = row[HAP_OPT];
-                        if (!seen || row[HAP_OPT + 1] > opm) opm = row[HAP_OPT + 1];
-                        seen = true;
-                    }
-                sync_me = slat + n_dense * sbd + n_moe * sbm;
-                opt_me = n_dense * opd + n_moe * opm;
+                const i64 n_moe = (int)sK[b_me] - (int)sK[a_me], n_dense = (b_me - a_me) - n_moe;
+                const MaskInfo &mi = minfo[sp.mask - 1];
+                sync_me = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
+                opt_me = n_dense * mi.opt[0] + n_moe * mi.opt[1];
             }
             const i64 sum = warp_sum_i64(c_me), mxc = warp_max_i64(c_me);
             const i64 tsync = warp_max_i64(sync_me), topt = warp_max_i64(opt_me);
