@@ -33,7 +33,7 @@ struct hap_problem {
     uint64_t n_cand = 0;
     int pp_max = 1;
     std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
-    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; };
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     // device
@@ -42,6 +42,7 @@ struct hap_problem {
     hap_pconf *d_pconf = nullptr;
     WorkItem *d_items = nullptr;
     i64 *d_c2 = nullptr, *d_coef = nullptr;
+    TypeConst *d_tc = nullptr;              // scratch: per (configuration, type) constants of the layer-cost kernels
     i64 *d_pcost = nullptr;                // per-block partial minima
     u64 *d_pindex = nullptr;
     u64 *d_counters = nullptr;             // [0] evaluated [1] feasible [2] pruned [3] incumbent
@@ -100,7 +101,7 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 static void release_device(hap_problem *p)
 {
     cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
-    cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
+    cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
 }
 
@@ -347,11 +348,17 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             hap_problem::PpClass cl{};
             cl.PP = PP;
             cl.warps = 0;
-            for (int w = kDpWarps; w >= 1; w >>= 1) {
-                cl.smem = dp_smem_bytes(N, PP, T, p->prof.R, w);
-                if (cl.smem <= 227 * 1024) { cl.warps = w; break; }
+            for (const auto &r : rows) if (r.PP == PP) { cl.multiset = r.mode == HAP_MAP_MULTISET; break; }
+            // most warps per SM: try block shapes from large to small, keep the one with the most resident warps
+            int best_resident = 0;
+            for (int w : {12, 8, 6, 4, 2, 1}) {
+                const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0);
+                if (sm > 227 * 1024) continue;
+                const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), 64 / w);
+                const int resident = std::min(per_sm * w, 24);           // registers allow about 24 warps per SM
+                if (resident > best_resident) { best_resident = resident; cl.warps = w; cl.smem = sm; }
             }
-            if (!cl.warps) return fail(p, HAP_E_RANGE, "shared memory need %zu of a PP=%d block exceeds the SM", cl.smem, PP);
+            if (!cl.warps) return fail(p, HAP_E_RANGE, "shared memory need of a PP=%d block exceeds the SM", PP);
             const int slices = std::max(1, cl.warps / p->opts.n_rc);
             const uint64_t chunk = 64ull * slices;
             cl.item_lo = items.size();
@@ -384,6 +391,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         CUDA_TRY(p, cudaMemcpy(p->d_items, p->items.data(), p->items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
         CUDA_TRY(p, cudaMalloc(&p->d_c2, np * T * N * 2 * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_coef, np * T * HAP_NCOEF * sizeof(i64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_tc, np * T * sizeof(TypeConst)));
         p->n_partial = std::max<size_t>(p->items.size(), 1024);
         CUDA_TRY(p, cudaMalloc(&p->d_pcost, p->n_partial * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_pindex, p->n_partial * sizeof(u64)));
@@ -449,9 +457,17 @@ extern "C" hap_status hap_decode(hap_problem *p, uint64_t first, uint64_t count,
 
 static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st)
 {
-    const unsigned blocks = (unsigned)((p->pconfs.size() + 3) / 4);
-    if (quant) layer_cost_kernel<true><<<blocks, 128, 0, st>>>(p->dc, c2, coef, nullptr, nullptr);
-    else layer_cost_kernel<false><<<blocks, 128, 0, st>>>(p->dc, nullptr, nullptr, c2f, coeff);
+    const u64 nph = (u64)p->pconfs.size() * HAP_MAX_TYPES;
+    const unsigned b1 = (unsigned)((nph + kLcThreads - 1) / kLcThreads);
+    if (quant) type_const_kernel<true><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr);
+    else type_const_kernel<false><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff);
+    CUDA_TRY(p, cudaGetLastError());
+    if ((quant && c2) || (!quant && c2f)) {
+        const unsigned b2 = (unsigned)(p->pconfs.size() * p->T);
+        const unsigned thr = (unsigned)((p->model.N + 31) / 32 * 32);
+        if (quant) layer_cost_kernel<true><<<b2, thr, 0, st>>>(p->dc, p->d_tc, c2, nullptr);
+        else layer_cost_kernel<false><<<b2, thr, 0, st>>>(p->dc, p->d_tc, nullptr, c2f);
+    }
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
 }
@@ -477,7 +493,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
 {
     // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
     // process: raise it (never lower it) before a launch that needs more
-    static size_t smem_limit[64][2];
+    static size_t smem_limit[64][4];
     const int dev = p->device & 63;
     for (const auto &cl : p->classes) {
         // skip classes whose candidates all lie outside the range
@@ -485,18 +501,24 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const u64 c0 = p->pconfs[a.p].offset, c1 = p->pconfs[b.p].offset + p->pconfs[b.p].nmap * (u64)p->opts.n_rc;
         const bool outside = c1 <= out.first || c0 >= out.first + out.count;
         if (outside && !search) continue;
-        if (cl.smem > smem_limit[dev][search]) {
-            if (search) CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl.smem));
-            else CUDA_TRY(p, cudaFuncSetAttribute(pipeline_dp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl.smem));
-            smem_limit[dev][search] = cl.smem;
+        const bool lin = p->dc.tau_linear != 0;
+        const int variant = (search ? 2 : 0) + (lin ? 1 : 0);
+        const void *fn = variant == 0 ? (const void *)pipeline_dp_kernel<false, false>
+                         : variant == 1 ? (const void *)pipeline_dp_kernel<false, true>
+                         : variant == 2 ? (const void *)pipeline_dp_kernel<true, false>
+                                        : (const void *)pipeline_dp_kernel<true, true>;
+        if (cl.smem > smem_limit[dev][variant]) {
+            CUDA_TRY(p, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl.smem));
+            smem_limit[dev][variant] = cl.smem;
         }
         const unsigned blocks = (unsigned)(cl.item_hi - cl.item_lo);
         const uint8_t *tab = cl.has_tab ? p->d_maptab + cl.map_base : nullptr;
         DpOut o = out;
         if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
-        if (search) pipeline_dp_kernel<true><<<blocks, cl.warps * 32, cl.smem, st>>>(p->dc, p->d_items + cl.item_lo, p->d_c2, p->d_coef, tab, o, cl.warps);
-        else pipeline_dp_kernel<false><<<blocks, cl.warps * 32, cl.smem, st>>>(p->dc, p->d_items + cl.item_lo, p->d_c2, p->d_coef, tab, o, cl.warps);
-        CUDA_TRY(p, cudaGetLastError());
+        const WorkItem *its = p->d_items + cl.item_lo;
+        int nw = cl.warps;
+        void *args[] = {(void *)&p->dc, (void *)&its, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tab, (void *)&o, (void *)&nw};
+        CUDA_TRY(p, cudaLaunchKernel(fn, dim3(blocks), dim3(cl.warps * 32), args, cl.smem, st));
     }
     return HAP_OK;
 }

@@ -22,7 +22,7 @@ typedef unsigned long long u64;
 typedef unsigned int u32;
 
 constexpr int kMaxMasks = (1 << HAP_MAX_TYPES) - 1;
-constexpr int kDpWarps = 8;           // warps per block of the DP kernel
+constexpr int kDpWarps = 12;          // most warps per block of the DP kernel
 constexpr i64 kInf = (i64)1 << 62;
 
 // Everything a kernel needs besides the big tables; passed by value.
@@ -137,7 +137,8 @@ __device__ __forceinline__ double collective_ns(const DevConst &dc, const LinkCt
 }
 
 struct TypeConst {      // per (configuration, type) values used by every layer
-    double disp2, imb, den, tr, tr2, commF[2], commB[2];
+    double disp2, imb, den, rden, tr, tr2, commF[2], commB[2];
+    long long row;          // table row (itp, icp, ib) of the configuration
 };
 
 template <bool QUANT>
@@ -152,130 +153,152 @@ __device__ __forceinline__ void store_pair(i64 *qi, double *qd, size_t at, doubl
     }
 }
 
-template <bool QUANT>
-__global__ void __launch_bounds__(128)
-layer_cost_kernel(const DevConst dc, i64 *c2, i64 *coef, double *c2f, double *coeff)
+constexpr int kLcThreads = 128;
+
+// a / b for a divisor whose correctly rounded reciprocal y = RN(1/b) is known: q0 = RN(a*y), the exact
+// residual r = a - b*q0 (one fused operation) and q = RN(q0 + r*y) give the correctly rounded quotient
+// (Markstein's division theorem), i.e. the same bits as the IEEE division a / b, at three operations.
+__device__ __forceinline__ double div_by(double a, double b, double y)
 {
-    __shared__ TypeConst tcs[4][HAP_MAX_TYPES];
-    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const u64 p = (u64)blockIdx.x * 4 + wib;
-    if (p >= dc.n_pconf) return;
-    const hap_pconf pc = dc.pconf[p];
-    const int N = dc.N, T = dc.T;
-    const int TP = pc.TP, CP = pc.CP, DP = pc.DP, EP = pc.EP, TPE = pc.TPE, EDP = pc.EDP, b = pc.b;
-    const i64 G = pc.G;
-    const i64 tok = (i64)b * dc.S / CP;
+    const double q0 = a * y;
+    const double r = __fma_rn(-b, q0, a);
+    return __fma_rn(r, y, q0);
+}
+
+// Phase 1 (type_const_kernel): one thread per (configuration, type) computes the per-type constants of
+// Eq. 2 / Eq. 3 into a scratch array and the stage coefficients.  Phase 2 (layer_cost_kernel): one thread
+// per (configuration, type, layer) unit, consecutive threads writing consecutive 16-byte results.
+template <bool QUANT>
+__global__ void __launch_bounds__(kLcThreads)
+type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff)
+{
+    const int T = dc.T;
     const i64 H = dc.H;
     const i64 Hkv = H * dc.nkv / dc.nq;
-    const double thb = (double)tok * (double)H;
-    const double Dtp = thb * dc.beta;
-
-    if (lane < T) {
-        const int h = lane;
-        LinkCtx lc; lc.bw_intra = dc.bw_intra[h]; lc.bw_inter = dc.bw_inter[h]; lc.node_size = dc.node_size[h];
-        TypeConst tc;
-        tc.imb = 1.0 + dc.gamma * (dc.rho[pc.iep] - 1.0);
-        double tdisp = 0.0;
-        if (EP != 1) {
-            const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
-            const double Dag = (thb * dc.beta) * (double)(EP - 1);
-            const int cls = link_class(lc, (i64)EP * TPE);
-            const double fa = dc.alpha[cls] * (double)(EP - 1) + Dmoe / link_bw(lc, cls);
-            const double fg = dc.alpha[cls] * (double)(EP - 1) + Dag / link_bw(lc, cls);
-            tdisp = (fa <= fg) ? fa : fg;
-        }
-        tc.disp2 = 2.0 * tdisp;
-        const double ttpA = 2.0 * collective_ns(dc, lc, TP, TP, Dtp);
-        const double ttpD = ttpA;
-        const double ttpM = 2.0 * collective_ns(dc, lc, TPE, TPE, Dtp);
-        const double Dkv = ((((2.0 * (double)b) * (double)dc.S) * (double)Hkv) * dc.beta) / (double)TP;
-        const double tcp = collective_ns(dc, lc, CP, (i64)TP * CP, Dkv);
-        tc.tr = dc.croute[h] * thb;
-        tc.tr2 = 2.0 * tc.tr;
-        tc.commF[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
-        tc.commB[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
-        tc.commF[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
-        tc.commB[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
-        tc.den = (dc.eta[h] * (double)EP) * (double)TPE;
-        tcs[wib][h] = tc;
-
-        if ((QUANT && coef) || (!QUANT && coeff)) {
-            double v[HAP_NCOEF];
-            const size_t i4 = (((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib;
-            v[HAP_KPRE] = dc.tpre[i4];
-            v[HAP_KPOST] = dc.tpost[i4];
-            const double Dp = Dtp / (double)TP;
-            v[HAP_KP2P_INTRA] = 2.0 * (dc.alpha[HAP_INTRA] + Dp / dc.bw_intra[h]);
-            v[HAP_KP2P_INTER] = 2.0 * (dc.alpha[HAP_INTER] + Dp / dc.bw_inter[h]);
-#pragma unroll
-            for (int h2 = 0; h2 < HAP_MAX_TYPES; ++h2) {
-                const double bo = h2 < T ? dc.bw_inter[h2] : dc.bw_inter[h];
-                const double bmin = dc.bw_inter[h] < bo ? dc.bw_inter[h] : bo;
-                v[HAP_KP2P_CROSS + h2] = 2.0 * (dc.alpha[HAP_CROSS] + Dp / (bmin * dc.chi));
+    {
+        const u64 gid = (u64)blockIdx.x * kLcThreads + threadIdx.x;
+        const u64 p = gid / HAP_MAX_TYPES;
+        const int h = (int)(gid % HAP_MAX_TYPES);
+        if (p < dc.n_pconf && h < T) {
+            const hap_pconf pc = dc.pconf[p];
+            const int TP = pc.TP, CP = pc.CP, DP = pc.DP, EP = pc.EP, TPE = pc.TPE, EDP = pc.EDP, b = pc.b;
+            const i64 G = pc.G;
+            const i64 tok = (i64)b * dc.S / CP;
+            const double thb = (double)tok * (double)H;
+            const double Dtp = thb * dc.beta;
+            LinkCtx lc; lc.bw_intra = dc.bw_intra[h]; lc.bw_inter = dc.bw_inter[h]; lc.node_size = dc.node_size[h];
+            TypeConst tc;
+            tc.imb = 1.0 + dc.gamma * (dc.rho[pc.iep] - 1.0);
+            double tdisp = 0.0;
+            if (EP != 1) {
+                const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
+                const double Dag = (thb * dc.beta) * (double)(EP - 1);
+                const int cls = link_class(lc, (i64)EP * TPE);
+                const double fa = dc.alpha[cls] * (double)(EP - 1) + Dmoe / link_bw(lc, cls);
+                const double fg = dc.alpha[cls] * (double)(EP - 1) + Dag / link_bw(lc, cls);
+                tdisp = (fa <= fg) ? fa : fg;
             }
-            const i64 wd = (i64)DP * CP;
-            const double shd = 6.0 + 12.0 / (double)wd;
-            const double she = 6.0 + 12.0 / (double)EDP;
-            const i64 Pattn = H * (H + 2 * Hkv) + H * H + 2 * H;
-            const i64 Pffn_d = 3 * H * (i64)dc.F_dense, Pffn_e = 3 * H * (i64)dc.F_exp;
-            const i64 Pe = (i64)(dc.E / EP) * Pffn_e;
-            const i64 Prt = H * (i64)dc.E;
-            i64 Pd[2];
-            Pd[HAP_DENSE] = Pattn + Pffn_d;
-            Pd[HAP_MOE] = Pattn + (i64)dc.n_shared * Pffn_e;
-            const double PeT = (double)Pe / (double)TPE;
-            v[HAP_MW + HAP_DENSE] = ((double)Pd[HAP_DENSE] / (double)TP) * shd;
-            v[HAP_MW + HAP_MOE] = ((double)Pd[HAP_MOE] / (double)TP + (double)Prt) * shd + PeT * she;
-            v[HAP_MA + HAP_DENSE] = (thb * dc.act_coef[HAP_DENSE]) / (double)TP;
-            v[HAP_MA + HAP_MOE] = (thb * dc.act_coef[HAP_MOE]) / (double)TP;
-            v[HAP_MX] = ((2.0 * ((thb * dc.beta) * (double)dc.k)) * (1.0 - 1.0 / (double)EP)) * dc.capf
-                        + ((double)tok * (double)dc.E) * 4.0;
-            v[HAP_MPRE] = (((double)dc.V * (double)H) / (double)TP) * shd;
-            v[HAP_MPOST] = v[HAP_MPRE];
-            const int cG = link_class(lc, G);
-            const double bwG = link_bw(lc, cG);
-            const double vfd = (double)(wd - 1) / (double)wd, vfe = (double)(EDP - 1) / (double)EDP;
+            tc.disp2 = 2.0 * tdisp;
+            const double ttpA = 2.0 * collective_ns(dc, lc, TP, TP, Dtp);
+            const double ttpD = ttpA;
+            const double ttpM = 2.0 * collective_ns(dc, lc, TPE, TPE, Dtp);
+            const double Dkv = ((((2.0 * (double)b) * (double)dc.S) * (double)Hkv) * dc.beta) / (double)TP;
+            const double tcp = collective_ns(dc, lc, CP, (i64)TP * CP, Dkv);
+            tc.tr = dc.croute[h] * thb;
+            tc.tr2 = 2.0 * tc.tr;
+            tc.commF[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
+            tc.commB[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
+            tc.commF[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
+            tc.commB[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
+            tc.den = (dc.eta[h] * (double)EP) * (double)TPE;
+            tc.rden = 1.0 / tc.den;
+            tc.row = (pc.itp * dc.ncp + pc.icp) * dc.nmb + pc.ib;
+            tcg[p * T + h] = tc;
+
+            if ((QUANT && coef) || (!QUANT && coeff)) {
+                double v[HAP_NCOEF];
+                const size_t i4 = (((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib;
+                v[HAP_KPRE] = dc.tpre[i4];
+                v[HAP_KPOST] = dc.tpost[i4];
+                const double Dp = Dtp / (double)TP;
+                v[HAP_KP2P_INTRA] = 2.0 * (dc.alpha[HAP_INTRA] + Dp / dc.bw_intra[h]);
+                v[HAP_KP2P_INTER] = 2.0 * (dc.alpha[HAP_INTER] + Dp / dc.bw_inter[h]);
 #pragma unroll
-            for (int kd = 0; kd < 2; ++kd) {
-                const i64 Pdd = Pd[kd] + (kd == HAP_MOE ? Prt : 0);
-                const double Pel = kd == HAP_MOE ? PeT : 0.0;
-                v[HAP_SBW + kd] = dc.ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG)
-                                               + (((6.0 * Pel) * vfe) / bwG));
-                v[HAP_OPT + kd] = dc.copt[h] * ((double)Pdd / (double)((i64)TP * DP * CP) + Pel / (double)EDP);
-            }
-            v[HAP_SLAT] = dc.ovl_dp * (dc.alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
-            const size_t at = ((size_t)p * T + h) * HAP_NCOEF;
+                for (int h2 = 0; h2 < HAP_MAX_TYPES; ++h2) {
+                    const double bo = h2 < T ? dc.bw_inter[h2] : dc.bw_inter[h];
+                    const double bmin = dc.bw_inter[h] < bo ? dc.bw_inter[h] : bo;
+                    v[HAP_KP2P_CROSS + h2] = 2.0 * (dc.alpha[HAP_CROSS] + Dp / (bmin * dc.chi));
+                }
+                const i64 wd = (i64)DP * CP;
+                const double shd = 6.0 + 12.0 / (double)wd;
+                const double she = 6.0 + 12.0 / (double)EDP;
+                const i64 Pattn = H * (H + 2 * Hkv) + H * H + 2 * H;
+                const i64 Pffn_d = 3 * H * (i64)dc.F_dense, Pffn_e = 3 * H * (i64)dc.F_exp;
+                const i64 Pe = (i64)(dc.E / EP) * Pffn_e;
+                const i64 Prt = H * (i64)dc.E;
+                i64 Pd[2];
+                Pd[HAP_DENSE] = Pattn + Pffn_d;
+                Pd[HAP_MOE] = Pattn + (i64)dc.n_shared * Pffn_e;
+                const double PeT = (double)Pe / (double)TPE;
+                v[HAP_MW + HAP_DENSE] = ((double)Pd[HAP_DENSE] / (double)TP) * shd;
+                v[HAP_MW + HAP_MOE] = ((double)Pd[HAP_MOE] / (double)TP + (double)Prt) * shd + PeT * she;
+                v[HAP_MA + HAP_DENSE] = (thb * dc.act_coef[HAP_DENSE]) / (double)TP;
+                v[HAP_MA + HAP_MOE] = (thb * dc.act_coef[HAP_MOE]) / (double)TP;
+                v[HAP_MX] = ((2.0 * ((thb * dc.beta) * (double)dc.k)) * (1.0 - 1.0 / (double)EP)) * dc.capf
+                            + ((double)tok * (double)dc.E) * 4.0;
+                v[HAP_MPRE] = (((double)dc.V * (double)H) / (double)TP) * shd;
+                v[HAP_MPOST] = v[HAP_MPRE];
+                const int cG = link_class(lc, G);
+                const double bwG = link_bw(lc, cG);
+                const double vfd = (double)(wd - 1) / (double)wd, vfe = (double)(EDP - 1) / (double)EDP;
 #pragma unroll
-            for (int q = 0; q < HAP_NCOEF; ++q) {
-                if (QUANT) coef[at + q] = __double2ll_rn(v[q]);
-                else coeff[at + q] = v[q];
+                for (int kd = 0; kd < 2; ++kd) {
+                    const i64 Pdd = Pd[kd] + (kd == HAP_MOE ? Prt : 0);
+                    const double Pel = kd == HAP_MOE ? PeT : 0.0;
+                    v[HAP_SBW + kd] = dc.ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG)
+                                                   + (((6.0 * Pel) * vfe) / bwG));
+                    v[HAP_OPT + kd] = dc.copt[h] * ((double)Pdd / (double)((i64)TP * DP * CP) + Pel / (double)EDP);
+                }
+                v[HAP_SLAT] = dc.ovl_dp * (dc.alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
+                const size_t at = ((size_t)p * T + h) * HAP_NCOEF;
+#pragma unroll
+                for (int q = 0; q < HAP_NCOEF; ++q) {
+                    if (QUANT) coef[at + q] = __double2ll_rn(v[q]);
+                    else coeff[at + q] = v[q];
+                }
             }
         }
     }
-    __syncwarp();
-    if ((QUANT && !c2) || (!QUANT && !c2f)) return;
+}
 
-    const size_t out0 = (size_t)p * T * N * 2;
-    for (int u = lane; u < T * N; u += 32) {
-        const int h = u / N, l = u - h * N;
-        const TypeConst &tc = tcs[wib][h];
-        const size_t i5 = ((((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib) * N + l;
-        const double a = dc.tdf[i5], ab = dc.tdb[i5];
-        double cf, cb;
-        if (layer_kind(dc, l) == HAP_DENSE) {
-            cf = a + tc.commF[HAP_DENSE];
-            cb = ab + tc.commB[HAP_DENSE];
-        } else {
-            const double f = dc.tff[i5], fb = dc.tfb[i5];
-            const double xf = (dc.kappa * f) / tc.den;
-            const double mf = (xf + tc.disp2) * tc.imb;
-            cf = (((a - f) + mf) + tc.tr) + tc.commF[HAP_MOE];
-            const double xb = (dc.kappa * fb) / tc.den;
-            const double mb = (xb + tc.disp2) * tc.imb;
-            cb = (((ab - fb) + mb) + tc.tr2) + tc.commB[HAP_MOE];
-        }
-        store_pair<QUANT>(c2, c2f, out0 + (size_t)u * 2, cf, cb);
+// one block per (configuration, type), threads over the layers
+template <bool QUANT>
+__global__ void __launch_bounds__(256)
+layer_cost_kernel(const DevConst dc, const TypeConst *tcg, i64 *c2, double *c2f)
+{
+    const int N = dc.N;
+    const unsigned ph = blockIdx.x;                                     // p*T + h
+    const int l = threadIdx.x;
+    if (l >= N) return;
+    const int h = (int)(ph % (unsigned)dc.T);
+    const TypeConst tc = tcg[ph];
+    const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
+    const size_t i5 = (size_t)h * stride_h + (size_t)tc.row * N + l;
+    const double a = dc.tdf[i5], ab = dc.tdb[i5];
+    double cf, cb;
+    if (layer_kind(dc, l) == HAP_DENSE) {
+        cf = a + tc.commF[HAP_DENSE];
+        cb = ab + tc.commB[HAP_DENSE];
+    } else {
+        const double f = dc.tff[i5], fb = dc.tfb[i5];
+        const double xf = div_by(dc.kappa * f, tc.den, tc.rden);
+        const double mf = (xf + tc.disp2) * tc.imb;
+        cf = (((a - f) + mf) + tc.tr) + tc.commF[HAP_MOE];
+        const double xb = div_by(dc.kappa * fb, tc.den, tc.rden);
+        const double mb = (xb + tc.disp2) * tc.imb;
+        cb = (((ab - fb) + mb) + tc.tr2) + tc.commB[HAP_MOE];
     }
+    store_pair<QUANT>(c2, c2f, ((size_t)ph * N + l) * 2, cf, cb);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -438,25 +461,30 @@ __global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *t
 // pipeline DP
 // ------------------------------------------------------------------------------------------
 // Shared memory of one block (all candidates of a block belong to one configuration):
-//   sC, sF   [kMaxMasks][N+1]  prefix sums of forward+backward / forward time per type mask
-//   sW, sA   [N+1]             prefix sums of weight bytes / activation bytes per micro-batch
-//   thr      [PP][T][R][N+1]   u8: first split k for which stage i on a device of capacity type t
+//   sR   [mask rows][RW][N+1]  i64 prefix sums of stage time per type mask.  LINEAR (every tau_q a
+//                              multiple of 1024): one row per recomputation level r holding
+//                              fwd+bwd + (tau_r/1024)*fwd, so a span costs one subtraction; otherwise
+//                              two rows (fwd+bwd, fwd) and the general formula.  Homogeneous (multiset)
+//                              configurations keep one mask row per device type, block mode one per mask.
+//   sW, sA [N+1]               i64 prefix sums of weight bytes / activation bytes per micro-batch
+//   thr  [PP][T][R][N+1]       u8: first split k for which stage i on a device of capacity type t
 //                              fits layers (k, j] at recomputation level r (j = none)
-//   sK       [N+1]             u8: number of MoE layers among the first l layers
-//   per warp: rows [(PP+1)][N+1] i64 (one DP row per stage, kept so that the next mapping can reuse
-//             the rows of the stage prefix it shares), ch [PP][N+1] u8 split choices
-__host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int warps)
+//   sK   [N+1]                 u8: number of MoE layers among the first l layers
+//   per warp: rows [PP][N+1] i64 (one DP row per stage, kept so that the next mapping can reuse the rows
+//             of the stage prefix it shares), ch [PP][N+1] u8 split choices
+__host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int warps, bool multiset, bool linear)
 {
     const size_t n1 = (size_t)N + 1;
-    size_t b = (size_t)kMaxMasks * n1 * 16 + n1 * 16;
+    const size_t mrows = multiset ? (size_t)T : (size_t)((1 << T) - 1);
+    size_t b = mrows * (linear ? (size_t)R : 2) * n1 * 8 + n1 * 16;
     b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
-    b += (n1 + 15) / 16 * 16;                                   // MoE-layer prefix counts
-    b += (size_t)warps * (((size_t)(PP + 1) * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
+    b += (n1 + 15) / 16 * 16;
+    b += (size_t)warps * (((size_t)PP * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
     return b + 32;
 }
 
 struct StagePar {
-    int mask, capt;             // type mask; index of the type whose capacity binds
+    int mrow, capt;             // row of the stage's type mask in sR; index of the type whose capacity binds
     i64 K;                      // stage constant: pre/post work + p2p transfer into the stage
     int nmin, nmax;             // load-balance window on the layer count
     int bl, bh;                 // band of end layers j that can be reached at this stage
@@ -478,7 +506,7 @@ struct MaskInfo {
     int capt, pad;
 };
 
-template <bool SEARCH>
+template <bool SEARCH, bool LINEAR>
 __global__ void __launch_bounds__(kDpWarps * 32)
 pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef,
                    const uint8_t *maptab, DpOut out, int nwarps)
@@ -496,35 +524,38 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             return;
         }
     }
+    const bool multiset = pc.mode == HAP_MAP_MULTISET;
+    const int nmask = (1 << T) - 1;
+    const int mrows = multiset ? T : nmask;
+    const int RW = LINEAR ? R : 2;
 
-    i64 *sC = reinterpret_cast<i64 *>(smem_raw);
-    i64 *sF = sC + (size_t)kMaxMasks * n1;
-    i64 *sW = sF + (size_t)kMaxMasks * n1;
+    i64 *sR = reinterpret_cast<i64 *>(smem_raw);
+    i64 *sW = sR + (size_t)mrows * RW * n1;
     i64 *sA = sW + n1;
     uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
     const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
     uint8_t *sK = thr + thr_bytes;
-    const size_t row_bytes = (size_t)(PP + 1) * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
+    const size_t row_bytes = (size_t)PP * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
     unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
-    __shared__ MaskInfo minfo[kMaxMasks];
-    i64 *rows = reinterpret_cast<i64 *>(wbase);
+    i64 *rows = reinterpret_cast<i64 *>(wbase);            // row of stage i at rows + (i-1)*n1
     uint8_t *chw = wbase + row_bytes;
+    __shared__ MaskInfo minfo[kMaxMasks];
+    __shared__ i64 sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
+    __shared__ i64 szero[1];                               // the row of "stage 0": DP[0][0] = 0
+    __shared__ int winT[HAP_MAX_TYPES][2];
 
     // ---- block prologue 1: rows of this configuration -----------------------------------
     const i64 *c2p = c2 + (size_t)it.p * T * N * 2;
     const i64 *cfp = coef + (size_t)it.p * T * HAP_NCOEF;
-    const int nmask = (1 << T) - 1;
-    const bool multiset = pc.mode == HAP_MAP_MULTISET;
-    for (int mk = 1 + wib; mk <= nmask + 1; mk += nwarps) {
-        // masks 1..nmask: time rows (homogeneous stages need the single-type masks only);
-        // the extra round (mk == nmask+1) builds the byte rows
-        if (mk <= nmask && multiset && (mk & (mk - 1))) continue;
+    for (int mr = wib; mr <= mrows; mr += nwarps) {
+        // mr < mrows: time rows of one type mask; mr == mrows: the byte rows
+        const int mk = multiset ? (1 << mr) : mr + 1;
         i64 runC = 0, runF = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
             i64 vC = 0, vF = 0;
             if (l < N) {
-                if (mk <= nmask) {
+                if (mr < mrows) {
                     i64 F = 0, B = 0;
                     for (int h = 0; h < T; ++h)
                         if (mk >> h & 1) {
@@ -545,13 +576,18 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             }
             vC += runC; vF += runF;
             if (l < N) {
-                if (mk <= nmask) { sC[(size_t)(mk - 1) * n1 + l + 1] = vC; sF[(size_t)(mk - 1) * n1 + l + 1] = vF; }
-                else { sW[l + 1] = vC; sA[l + 1] = vF; }
+                if (mr < mrows) {
+                    if (LINEAR) {
+                        for (int r = 0; r < R; ++r) sR[((size_t)mr * RW + r) * n1 + l + 1] = vC + (i64)(dc.tau_q[r] >> 10) * vF;
+                    } else {
+                        sR[((size_t)mr * RW) * n1 + l + 1] = vC; sR[((size_t)mr * RW + 1) * n1 + l + 1] = vF;
+                    }
+                } else { sW[l + 1] = vC; sA[l + 1] = vF; }
             }
             runC = shfl_i64(vC, 31); runF = shfl_i64(vF, 31);
         }
         if (lane == 0) {
-            if (mk <= nmask) { sC[(size_t)(mk - 1) * n1] = 0; sF[(size_t)(mk - 1) * n1] = 0; }
+            if (mr < mrows) { for (int r = 0; r < RW; ++r) sR[((size_t)mr * RW + r) * n1] = 0; }
             else { sW[0] = 0; sA[0] = 0; }
         }
     }
@@ -578,6 +614,11 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             }
         minfo[threadIdx.x] = mi;
     }
+    if (threadIdx.x >= 32 && threadIdx.x < 32 + T * 6) {
+        const int q = threadIdx.x - 32, h = q / 6, e = q % 6;
+        sP2P[h][e] = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
+    }
+    if (threadIdx.x == 0) szero[0] = 0;
     __syncthreads();
 
     // ---- block prologue 2: memory thresholds ----------------------------------------------
@@ -599,7 +640,6 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         }
     }
     // load-balance window per device type when every mapping uses the same multiset of stage types
-    __shared__ int winT[HAP_MAX_TYPES][2];
     if (threadIdx.x < T) {
         int lo = 1, hi = N - PP + 1;
         if (dc.delta_q >= 0 && multiset) {
@@ -619,6 +659,9 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     u64 best_index = ~0ull;
     u64 n_eval = 0, n_feas = 0, n_cells = 0;
     const bool want_tables = !SEARCH && (out.dp_table != nullptr || out.choice != nullptr);
+    int red0 = 1;                                    // reductions over the stages span the next power of two >= PP lanes
+    while (red0 < PP) red0 <<= 1;
+    red0 >>= 1;
 
     // warp -> (recompute policy, slice of consecutive mappings); consecutive mappings share a prefix of
     // stage types, and the DP rows of a shared prefix are reused
@@ -630,47 +673,48 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
       const unsigned rc_mask = dc.rc_masks[rc_idx];
       const u32 m_lo = (u32)my_slice * per_slice;
       const u32 m_hi = m_lo + per_slice < it.count ? m_lo + per_slice : it.count;
-      int valid_rows = 0;                  // rows[0..valid_rows] hold the DP of the previous mapping's prefix
+      int valid_rows = 0;                  // DP rows of stages 1..valid_rows of the previous mapping are intact
       int prev_mask = -1, prev_link = -1;
+      uchar2 next_ml = make_uchar2(0, 0);
+      if (maptab && m_lo < m_hi && lane < PP)
+          next_ml = *reinterpret_cast<const uchar2 *>(maptab + ((it.lo + m_lo) * (u64)PP + lane) * 2);
       for (u32 mi = m_lo; mi < m_hi; ++mi) {
         const u64 map_idx = it.lo + mi;
         const u64 c = pc.offset + map_idx * (u64)n_rc + (u64)rc_idx;
-        if (c < out.first || c >= out.first + out.count) { valid_rows = 0; prev_mask = -1; continue; }
 
         // ---- stage types of this mapping, lane s holds stage s+1 -----------------------------
         int mask = 0, link = 0;
         if (maptab) {
-            if (lane < PP) {
-                const uchar2 ml = *reinterpret_cast<const uchar2 *>(maptab + (map_idx * (u64)PP + lane) * 2);
-                mask = ml.x; link = ml.y;
-            }
+            mask = next_ml.x; link = next_ml.y;
+            if (mi + 1 < m_hi && lane < PP)        // fetch the next mapping while this one is evaluated
+                next_ml = *reinterpret_cast<const uchar2 *>(maptab + ((map_idx + 1) * (u64)PP + lane) * 2);
         } else {
             const StageMap smap = decode_stage(dc, pc, map_idx, lane);
             mask = smap.mask; link = lane > 0 && lane < PP ? (smap.cls | (smap.ha << 2) | (smap.hb << 4)) : 0;
         }
+        if (c < out.first || c >= out.first + out.count) { valid_rows = 0; prev_mask = -1; continue; }
         const unsigned differ = __ballot_sync(0xffffffffu, lane < PP && (mask != prev_mask || link != prev_link));
         int s0 = differ ? __ffs(differ) - 1 : PP;      // stages 1..s0 are shared with the previous mapping
         prev_mask = mask; prev_link = link;
 
         StagePar sp;
-        sp.mask = mask; sp.capt = 0; sp.K = 0; sp.nmin = 1; sp.nmax = N - PP + 1; sp.bl = 0; sp.bh = 0;
+        sp.mrow = 0; sp.capt = 0; sp.K = 0; sp.nmin = 1; sp.nmax = N - PP + 1; sp.bl = 0; sp.bh = 0;
         i64 Pmin = 0;
         if (lane < PP) {
-            const MaskInfo &mi = minfo[mask - 1];
-            sp.capt = mi.capt; Pmin = mi.Pmin;
-            if (lane == 0) sp.K += mi.kpre;
-            if (lane == PP - 1) sp.K += mi.kpost;
+            const MaskInfo &mi_ = minfo[mask - 1];
+            sp.mrow = multiset ? __ffs(mask) - 1 : mask - 1;
+            sp.capt = mi_.capt; Pmin = mi_.Pmin;
+            if (lane == 0) sp.K += mi_.kpre;
+            if (lane == PP - 1) sp.K += mi_.kpost;
             if (lane > 0) {
                 const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3;
-                const i64 *row = cfp + hb * HAP_NCOEF;
-                sp.K += cls == HAP_INTRA ? row[HAP_KP2P_INTRA] : (cls == HAP_INTER ? row[HAP_KP2P_INTER] : row[HAP_KP2P_CROSS + ha]);
+                sp.K += sP2P[hb][cls == HAP_CROSS ? 2 + ha : cls];
             }
         }
         if (dc.delta_q >= 0) {
             if (multiset) {
-                if (lane < PP) { sp.nmin = winT[__ffs(mask) - 1][0]; sp.nmax = winT[__ffs(mask) - 1][1]; }   // homogeneous stage: its one type
+                if (lane < PP) { sp.nmin = winT[sp.mrow][0]; sp.nmax = winT[sp.mrow][1]; }   // homogeneous stage: its one type
             } else {
-                s0 = 0;                              // the window depends on the whole mapping: nothing is shared
                 const i64 Ps = warp_sum_i64(lane < PP ? Pmin : 0);
                 if (lane < PP) {
                     const i64 den = 1024 * Ps;
@@ -682,7 +726,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 }
             }
         }
-        if (!multiset) s0 = 0;
+        if (!multiset) s0 = 0;               // block mode: window and bands depend on the whole mapping
         if (s0 > valid_rows) s0 = valid_rows;
         if (want_tables) s0 = 0;
 
@@ -717,21 +761,19 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 if (ch_out) ch_out[j] = 255;
             }
         }
-        if (s0 == 0 && lane == 0) rows[0] = 0;           // DP[0][0] = 0; the band of stage 0 is {0}
-        __syncwarp();
         i64 bott = kInf;
         if (!dead || want_tables) {
-            int pbl = 0, pbh = 0;                          // band of the previous stage
+            int pbl = 0, pbh = 0;                          // band of the previous stage (stage 0: {0})
             if (s0 > 0) { pbl = __shfl_sync(0xffffffffu, sp.bl, s0 - 1); pbh = __shfl_sync(0xffffffffu, sp.bh, s0 - 1); }
             for (int i = s0 + 1; i <= PP; ++i) {
                 const int src = i - 1;
-                const int smask = __shfl_sync(0xffffffffu, sp.mask, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
+                const int mrow = __shfl_sync(0xffffffffu, sp.mrow, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
                 const i64 K = shfl_i64(sp.K, src);
                 const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
                 const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
-                const i64 *rC = sC + (size_t)(smask - 1) * n1, *rF = sF + (size_t)(smask - 1) * n1;
-                const i64 *prev = rows + (size_t)(i - 1) * n1;
-                i64 *cur = rows + (size_t)i * n1;
+                const i64 *rM = sR + (size_t)mrow * RW * n1;
+                const i64 *prev = i == 1 ? szero : rows + (size_t)(i - 2) * n1;
+                i64 *cur = rows + (size_t)(i - 1) * n1;
                 uint8_t *chrow = chw + (size_t)(i - 1) * n1;
                 const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
                 for (int j = bl + lane; j <= bh; j += 32) {
@@ -740,20 +782,31 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                     int klo = j - nmax; if (klo < pbl) klo = pbl;
                     int khi = j - nmin; if (khi > pbh) khi = pbh;
                     if (klo <= khi) {
-                        const i64 Cj = rC[j] + K, Fj = rF[j];
                         int seg_hi = khi;                     // k range still to be assigned a level
                         for (int r = 0; r < R && seg_hi >= klo; ++r) {
                             if (!((rc_mask >> r) & 1u)) continue;
                             int lo = th[(size_t)r * n1 + j];   // first k that fits at level r
                             if (lo < klo) lo = klo;
                             if (lo > seg_hi) continue;
-                            const i64 tau = dc.tau_q[r];
                             n_cells += (u64)(seg_hi - lo + 1);
-                            for (int k = seg_hi; k >= lo; --k) {
-                                const i64 pv = prev[k];
-                                const i64 cst = (Cj - rC[k]) + ((tau * (Fj - rF[k])) >> 10);   // forward sums are non-negative
-                                const i64 v = pv > cst ? pv : cst;
-                                if (v <= best && v < kInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
+                            if (LINEAR) {
+                                const i64 *rr = rM + (size_t)r * n1;
+                                const i64 Cj = rr[j] + K;
+                                for (int k = seg_hi; k >= lo; --k) {
+                                    const i64 pv = prev[k];
+                                    const i64 cst = Cj - rr[k];
+                                    const i64 v = pv > cst ? pv : cst;
+                                    if (v <= best && v < kInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
+                                }
+                            } else {
+                                const i64 *rC = rM, *rF = rM + n1;
+                                const i64 Cj = rC[j] + K, Fj = rF[j], tau = dc.tau_q[r];
+                                for (int k = seg_hi; k >= lo; --k) {
+                                    const i64 pv = prev[k];
+                                    const i64 cst = (Cj - rC[k]) + ((tau * (Fj - rF[k])) >> 10);   // forward sums are non-negative
+                                    const i64 v = pv > cst ? pv : cst;
+                                    if (v <= best && v < kInf) { best = v; arg = k; }
+                                }
                             }
                             seg_hi = lo - 1;
                         }
@@ -774,7 +827,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             valid_rows = dead ? 0 : PP;
             // N lies in the last band unless the windows cannot add up to N (possible only without the
             // suffix restriction, i.e. when tables are written)
-            if (!dead && pbl <= N && N <= pbh) bott = rows[(size_t)PP * n1 + N];
+            if (!dead && pbl <= N && N <= pbh) bott = rows[(size_t)(PP - 1) * n1 + N];
         } else {
             valid_rows = 0;
         }
@@ -797,19 +850,24 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 int r = 0;
                 for (; r < R; ++r)
                     if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b_me] <= a_me) break;
-                const i64 *rC = sC + (size_t)(sp.mask - 1) * n1, *rF = sF + (size_t)(sp.mask - 1) * n1;
-                c_me = (rC[b_me] - rC[a_me]) + (((i64)dc.tau_q[r] * (rF[b_me] - rF[a_me])) >> 10) + sp.K;
+                const i64 *rM = sR + (size_t)sp.mrow * RW * n1;
+                if (LINEAR) c_me = (rM[(size_t)r * n1 + b_me] - rM[(size_t)r * n1 + a_me]) + sp.K;
+                else c_me = (rM[b_me] - rM[a_me]) + (((i64)dc.tau_q[r] * (rM[n1 + b_me] - rM[n1 + a_me])) >> 10) + sp.K;
                 my_n = b_me - a_me; my_r = r;
                 const i64 n_moe = (int)sK[b_me] - (int)sK[a_me], n_dense = (b_me - a_me) - n_moe;
-                const MaskInfo &mi = minfo[sp.mask - 1];
-                sync_me = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
-                opt_me = n_dense * mi.opt[0] + n_moe * mi.opt[1];
+                const MaskInfo &mi_ = minfo[mask - 1];
+                sync_me = mi_.slat + n_dense * mi_.sbw[0] + n_moe * mi_.sbw[1];
+                opt_me = n_dense * mi_.opt[0] + n_moe * mi_.opt[1];
             }
-            const i64 sum = warp_sum_i64(c_me), mxc = warp_max_i64(c_me);
-            const i64 tsync = warp_max_i64(sync_me), topt = warp_max_i64(opt_me);
-            T_pipe = sum + (i64)(pc.M - 1) * mxc;
-            T_sync = tsync; T_opt = topt;
-            T_iter = T_pipe + tsync + topt;
+            i64 sum = c_me, mxc = c_me;
+            for (int o = red0; o > 0; o >>= 1) {          // lanes >= PP hold zeros
+                const i64 t1 = __shfl_xor_sync(0xffffffffu, sum, o), t2 = __shfl_xor_sync(0xffffffffu, mxc, o);
+                const i64 t3 = __shfl_xor_sync(0xffffffffu, sync_me, o), t4 = __shfl_xor_sync(0xffffffffu, opt_me, o);
+                sum += t1; mxc = t2 > mxc ? t2 : mxc; sync_me = t3 > sync_me ? t3 : sync_me; opt_me = t4 > opt_me ? t4 : opt_me;
+            }
+            T_pipe = shfl_i64(sum + (i64)(pc.M - 1) * mxc, 0);
+            T_sync = shfl_i64(sync_me, 0); T_opt = shfl_i64(opt_me, 0);
+            T_iter = T_pipe + T_sync + T_opt;
         }
         if (SEARCH) {
             n_eval++;

@@ -199,11 +199,17 @@ def test_all_infeasible_and_bad_descriptors(hap):
     assert e.value.name == "HAP_E_STATE"
 
 
-@pytest.mark.parametrize("seed", range(4))
+@pytest.mark.parametrize("seed", range(8))
 def test_random_small_problems_with_tight_memory(hap, seed):
-    """Mixed layer kinds, recomputation policies, windows and tight capacities on small random problems."""
-    pb = problems.random_small(seed, N=9 + seed, T=2 + seed % 2, nodes_per_type=((2, 2), (2, 1, 1))[seed % 2],
+    """Mixed layer kinds, recomputation policies, windows and tight capacities on small random problems;
+    seeds >= 4 use three recomputation levels whose time factors are not multiples of 1024 (the general
+    stage-cost formula) and policies that skip a level."""
+    pb = problems.random_small(seed, N=9 + seed % 4, T=2 + seed % 2, nodes_per_type=((2, 2), (2, 1, 1))[seed % 2],
                                node_size=2, window=(seed % 2 == 0), first_dense=True)
+    if seed >= 4:
+        pb.xi_q = np.ascontiguousarray(np.array([1024, 512, 64], np.int32))
+        pb.tau_q = np.ascontiguousarray(np.array([0, 300, 1000], np.int32))
+        pb.rc_masks = np.ascontiguousarray(np.array([0b001, 0b011, 0b111, 0b101], np.uint32))
     hp = hap.hap_problem_create(pb)
     hap.hap_enumerate(hp)
     o = Oracle(pb)
