@@ -33,7 +33,7 @@ struct hap_problem {
     uint64_t n_cand = 0;
     int pp_max = 1;
     std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
-    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; };
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     // device
@@ -51,6 +51,7 @@ struct hap_problem {
     size_t n_partial = 0;
     bool timed = false;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev_fork = nullptr;          // classes run on their own streams between this event and their `done` events
     std::string err;
 };
 
@@ -103,6 +104,8 @@ static void release_device(hap_problem *p)
     cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
     cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
+    if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); }
 }
 
 extern "C" void hap_problem_destroy(hap_problem *p)
@@ -347,14 +350,20 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         for (int PP : pps) {
             hap_problem::PpClass cl{};
             cl.PP = PP;
+            cl.masks_used = 0xffffffffu;
+            cl.stream = nullptr; cl.done = nullptr;
             cl.warps = 0;
             for (const auto &r : rows) if (r.PP == PP) { cl.multiset = r.mode == HAP_MAP_MULTISET; break; }
             // most warps per SM: try block shapes from large to small, keep the one with the most resident warps
             int best_resident = 0;
+            uint64_t class_nmap = 0;
+            for (const auto &r : rows) if (r.PP == PP) { class_nmap = r.nmap; break; }
+            const uint64_t per_pconf = class_nmap * (uint64_t)p->opts.n_rc;     // candidates a block can have at most
             for (int w : {12, 8, 6, 4, 2, 1}) {
+                if ((uint64_t)w * 8 > per_pconf && w > 2) continue;             // keep about 8 candidates per warp
                 const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0);
                 if (sm > 227 * 1024) continue;
-                const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), 64 / w);
+                const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), std::min(32, 64 / w));
                 const int resident = std::min(per_sm * w, 24);           // registers allow about 24 warps per SM
                 if (resident > best_resident) { best_resident = resident; cl.warps = w; cl.smem = sm; }
             }
@@ -400,6 +409,11 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         CUDA_TRY(p, cudaMalloc(&p->d_single, sizeof(SingleOut)));
         p->dc.pconf = p->d_pconf;
         p->dc.n_pconf = np;
+        CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+        for (auto &cl : p->classes) {
+            CUDA_TRY(p, cudaStreamCreateWithFlags(&cl.stream, cudaStreamNonBlocking));
+            CUDA_TRY(p, cudaEventCreateWithFlags(&cl.done, cudaEventDisableTiming));
+        }
         if (tab_bytes) {
             CUDA_TRY(p, cudaMalloc(&p->d_maptab, tab_bytes));
             for (const auto &cl : p->classes) {
@@ -410,6 +424,16 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 CUDA_TRY(p, cudaGetLastError());
             }
             CUDA_TRY(p, cudaDeviceSynchronize());
+            // which type masks occur in a class: the DP kernel builds stage rows for those only
+            std::vector<uint8_t> tab(tab_bytes);
+            CUDA_TRY(p, cudaMemcpy(tab.data(), p->d_maptab, tab_bytes, cudaMemcpyDeviceToHost));
+            for (auto &cl : p->classes) {
+                if (!cl.has_tab) continue;
+                const u64 nmap = p->pconfs[p->items[cl.item_lo].p].nmap;
+                unsigned used = 0;
+                for (u64 e = 0; e < nmap * (u64)cl.PP; ++e) used |= 1u << tab[cl.map_base + e * 2];
+                cl.masks_used = used;
+            }
         }
         p->enumerated = true;
     }
@@ -495,7 +519,16 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     // process: raise it (never lower it) before a launch that needs more
     static size_t smem_limit[64][4];
     const int dev = p->device & 63;
-    for (const auto &cl : p->classes) {
+    // fork: every PP class runs on its own stream so that the tail of one class overlaps the next
+    CUDA_TRY(p, cudaEventRecord(p->ev_fork, st));
+    // the class with the most work goes first; the others fill the SMs it leaves free and its tail
+    std::vector<const hap_problem::PpClass *> order;
+    for (const auto &cl : p->classes) order.push_back(&cl);
+    std::stable_sort(order.begin(), order.end(), [](const hap_problem::PpClass *a, const hap_problem::PpClass *b) {
+        return (a->item_hi - a->item_lo) * (size_t)a->PP > (b->item_hi - b->item_lo) * (size_t)b->PP;
+    });
+    for (const hap_problem::PpClass *clp : order) {
+        const hap_problem::PpClass &cl = *clp;
         // skip classes whose candidates all lie outside the range
         const WorkItem &a = p->items[cl.item_lo], &b = p->items[cl.item_hi - 1];
         const u64 c0 = p->pconfs[a.p].offset, c1 = p->pconfs[b.p].offset + p->pconfs[b.p].nmap * (u64)p->opts.n_rc;
@@ -517,8 +550,12 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
         const WorkItem *its = p->d_items + cl.item_lo;
         int nw = cl.warps;
-        void *args[] = {(void *)&p->dc, (void *)&its, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tab, (void *)&o, (void *)&nw};
-        CUDA_TRY(p, cudaLaunchKernel(fn, dim3(blocks), dim3(cl.warps * 32), args, cl.smem, st));
+        unsigned used = cl.masks_used;
+        void *args[] = {(void *)&p->dc, (void *)&its, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tab, (void *)&o, (void *)&nw, (void *)&used};
+        CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
+        CUDA_TRY(p, cudaLaunchKernel(fn, dim3(blocks), dim3(cl.warps * 32), args, cl.smem, cl.stream));
+        CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
+        CUDA_TRY(p, cudaStreamWaitEvent(st, cl.done, 0));      // join
     }
     return HAP_OK;
 }

@@ -479,7 +479,8 @@ __host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int
     size_t b = mrows * (linear ? (size_t)R : 2) * n1 * 8 + n1 * 16;
     b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
     b += (n1 + 15) / 16 * 16;
-    b += (size_t)warps * (((size_t)PP * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
+    const size_t nrows = multiset ? (size_t)PP : (size_t)(PP < 2 ? PP : 2);   // rows are reused only across multiset mappings
+    b += (size_t)warps * ((nrows * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
     return b + 32;
 }
 
@@ -509,7 +510,7 @@ struct MaskInfo {
 template <bool SEARCH, bool LINEAR>
 __global__ void __launch_bounds__(kDpWarps * 32)
 pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef,
-                   const uint8_t *maptab, DpOut out, int nwarps)
+                   const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
@@ -535,9 +536,10 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
     const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
     uint8_t *sK = thr + thr_bytes;
-    const size_t row_bytes = (size_t)PP * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
+    const int nrows = multiset ? PP : (PP < 2 ? PP : 2);   // block mode shares nothing between mappings: two rotating rows
+    const size_t row_bytes = (size_t)nrows * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
     unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
-    i64 *rows = reinterpret_cast<i64 *>(wbase);            // row of stage i at rows + (i-1)*n1
+    i64 *rows = reinterpret_cast<i64 *>(wbase);            // row of stage i at rows + ((i-1) % nrows)*n1
     uint8_t *chw = wbase + row_bytes;
     __shared__ MaskInfo minfo[kMaxMasks];
     __shared__ i64 sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
@@ -550,6 +552,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     for (int mr = wib; mr <= mrows; mr += nwarps) {
         // mr < mrows: time rows of one type mask; mr == mrows: the byte rows
         const int mk = multiset ? (1 << mr) : mr + 1;
+        if (mr < mrows && !((masks_used >> mk) & 1u)) continue;     // no mapping of this class has such a stage
         i64 runC = 0, runF = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
@@ -772,8 +775,9 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
                 const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
                 const i64 *rM = sR + (size_t)mrow * RW * n1;
-                const i64 *prev = i == 1 ? szero : rows + (size_t)(i - 2) * n1;
-                i64 *cur = rows + (size_t)(i - 1) * n1;
+                const int ri = multiset ? i - 1 : (i - 1) & 1;          // two rotating rows in block mode
+                const i64 *prev = i == 1 ? szero : rows + (multiset ? ri - 1 : ri ^ 1) * n1;
+                i64 *cur = rows + ri * n1;
                 uint8_t *chrow = chw + (size_t)(i - 1) * n1;
                 const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
                 for (int j = bl + lane; j <= bh; j += 32) {
@@ -827,7 +831,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             valid_rows = dead ? 0 : PP;
             // N lies in the last band unless the windows cannot add up to N (possible only without the
             // suffix restriction, i.e. when tables are written)
-            if (!dead && pbl <= N && N <= pbh) bott = rows[(size_t)(PP - 1) * n1 + N];
+            if (!dead && pbl <= N && N <= pbh) bott = rows[(size_t)(multiset ? PP - 1 : (PP - 1) & 1) * n1 + N];
         } else {
             valid_rows = 0;
         }
