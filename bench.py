@@ -30,6 +30,9 @@ METRIC = "candidate_plans_per_second"
 UNIT = "candidates/s"
 SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of the DP launches of one pass, from the ncu capture summarised
+# in profiles/pipeline_dp_kernel_stress.md
+NCU_DP_TRAFFIC_BYTES = {"stress": 64.0e6}
 
 
 def read_peaks():
@@ -153,7 +156,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2609_39350_b200 as hap
-    from paper_2609_39350_b200.sharding import shard_ranges, exchange_minimum
+    from paper_2609_39350_b200.sharding import shard_ranges, exchange_minimum, recurrence_cells
     from gen import problems
 
     rank = int(os.environ.get("RANK", "0"))
@@ -259,7 +262,11 @@ def main():
         dp_med, lc_med = statistics.median(dp_ms), statistics.median(lc_ms)
         sm_mhz = clocks["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)
         alu_peak = SM_COUNT * SCHEDULERS_PER_SM * LANES * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
-        achieved = 4.0 * cells / (dp_med * 1e-3) / 1e12
+        # algorithmic work of the DP kernel: 4 semiring operations (prefix difference, max, min, arg-select) per
+        # cell update of the plain recurrence, 2w + (PP-2)w(w+1)/2 cells per candidate with w = N-PP+1
+        cells_plain = float(sum(recurrence_cells(pb.N, int(r["PP"])) * int(r["nmap"]) * len(pb.rc_masks) for r in pconfs))
+        achieved = 4.0 * cells_plain / (dp_med * 1e-3) / 1e12
+        achieved_visited = 4.0 * cells / (dp_med * 1e-3) / 1e12
         units = n_pconf * hp.T * pb.N
         lc_gbs = 16.0 * units / (lc_med * 1e-3) / 1e9
         line = dict(
@@ -277,9 +284,15 @@ def main():
             full_search_ms=statistics.median(search_ms),
             best=dict(cost=best[0], index=best[1], search_index=plan["index"]),
             kernels_ms=dict(layer_cost=lc_med, pipeline_dp=dp_med),
-            roofline=dict(bound="alu", kernel="pipeline_dp_kernel", achieved=achieved, peak=alu_peak, unit="Tops/s",
-                          frac=achieved / alu_peak, traffic=None, cells_per_launch=cells,
-                          ops_per_cell=4, peak_source=f"{SM_COUNT} SMs x {SCHEDULERS_PER_SM} schedulers x {LANES} lanes x "
+            roofline=dict(bound="alu", kernel="pipeline_dp_kernel (one launch per PP class, concurrent streams)",
+                          achieved=achieved, peak=alu_peak, unit="Tops/s", frac=achieved / alu_peak,
+                          traffic=NCU_DP_TRAFFIC_BYTES.get(args.workload) if args.delta_q is None else None,
+                          ops_per_cell=4, cells_plain_recurrence=cells_plain, cells_visited=cells,
+                          frac_visited_cells_only=achieved_visited / alu_peak,
+                          note="achieved counts every cell of the plain recurrence; the kernel skips cells that the "
+                               "load-balance window, the reachable-layer bands, the memory thresholds and shared stage "
+                               "prefixes make +INF or identical, so it visits only cells_visited of them",
+                          peak_source=f"{SM_COUNT} SMs x {SCHEDULERS_PER_SM} schedulers x {LANES} lanes x "
                           f"{peaks.get('sm_max_mhz', 1965.0)} MHz ({peak_kind} clock)", sm_mhz_seen=sm_mhz),
             roofline_layer_cost=dict(bound="hbm", kernel="layer_cost_kernel", achieved=lc_gbs, peak=peaks["hbm_gbs"],
                                      unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=None,
