@@ -221,6 +221,28 @@ hap_status hap_search_best(hap_problem *, hap_plan *host_out, hap_search_stats *
  * dev_out[1] = index (as int64) of the minimum of dev_cost[0..count). */
 hap_status hap_argmin(hap_problem *, const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream);
 
+/* No counterpart in the paper: a variant of hap_argmin for callers that must not allocate.
+ *
+ * Some users of this library run it inside a process whose device memory has already been handed
+ * over in full to another owner (a framework's caching allocator, a fixed arena sized at start-up),
+ * or inside a steady-state loop where cudaMalloc / cudaFree are unwelcome because they can fail once
+ * memory is committed and because they stall the whole device.  Such a caller cannot create a
+ * hap_problem (that allocates) just to reduce a cost array it already holds.  This entry point needs
+ * no problem handle and calls no cudaMalloc, cudaFree or other allocating routine: the per-block
+ * partial minima go to a 64 KiB array that is part of the library image, so every GPU that loads the
+ * library keeps those 64 KiB until the process exits.
+ *
+ * dev_cost: [count] int64 on the current device; dev_out: 2 x int64 on the same device, receives
+ * (minimum cost, its lowest index).  Kernels are enqueued on `stream`; the call does not wait.
+ * Limit: 1 <= count <= HAP_ARGMIN_STATIC_MAX_COUNT, otherwise HAP_E_RANGE and nothing is launched.
+ * The first call on a device looks up the array's device address (one runtime query, cached per
+ * device); make that first call outside any stream capture.  All calls on a device share the one
+ * array and it keeps whatever the last call left there; a call writes every partial it later reads,
+ * so nothing needs clearing, but two calls whose kernels overlap on the GPU (different streams)
+ * race on it: keep calls on one device ordered. */
+#define HAP_ARGMIN_STATIC_MAX_COUNT ((uint64_t)1 << 26)
+hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream);
+
 /* Measurement aid: CUDA-event durations (ms) of the layer-cost kernel and of the dynamic-program
  * kernel of the most recent hap_pipeline_dp / hap_search_* call, and the number of recurrence cell
  * updates (k, j pairs inside the window and the memory limit) that launch evaluated.  Waits for that

@@ -16,7 +16,7 @@ COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, S
 STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE", "HAP_E_STATE", "HAP_E_INFEASIBLE"]
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_search_range",
-           "hap_search_best", "hap_argmin", "hap_get_timings", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_get_timings", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -266,6 +266,24 @@ def hap_search_best(hp: HapProblem, stream=None):
     pl, st = _Plan(), _Stats()
     hp.check(load_library().hap_search_best(hp.h, C.byref(pl), C.byref(st), _stream(stream)))
     return _plan_dict(pl), _stats_dict(st)
+
+
+ARGMIN_STATIC_MAX_COUNT = 1 << 26
+
+
+def hap_argmin_static(cost, out=None, stream=None, count=None):
+    """(cost, index) minimum of an int64 CUDA tensor through the entry point that allocates nothing
+    inside the library: no problem handle, scratch in the library image.  `out` is a 2-element int64
+    CUDA tensor (made here with torch if not given; pass your own when the caller must not allocate).
+    `count` defaults to cost.numel()."""
+    import torch
+    if out is None:
+        out = torch.empty(2, dtype=torch.int64, device=cost.device)
+    n = cost.numel() if count is None else count
+    st = load_library().hap_argmin_static(_dev(cost), C.c_uint64(n), _dev(out), _stream(stream))
+    if st != 0:
+        raise HapError(st, "hap_argmin_static: count must be in [1, 2^26] and the pointers non-null" if st in (1, 4) else "hap_argmin_static")
+    return out
 
 
 def hap_get_timings(hp: HapProblem):

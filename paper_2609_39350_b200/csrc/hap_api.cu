@@ -680,3 +680,43 @@ extern "C" hap_status hap_search_best(hap_problem *p, hap_plan *host_out, hap_se
     if (!p->enumerated) return fail(p, HAP_E_STATE, "hap_enumerate has not run");
     return hap_search_range(p, 0, p->n_cand, host_out, host_stats, stream);
 }
+
+// ------------------------------------------------------------------------------------------
+// hap_argmin_static: the (cost, index) minimum without any allocation
+// ------------------------------------------------------------------------------------------
+// Scratch for the per-block partial minima lives in the library image itself.  Every device that
+// loads the library carries these 64 KiB until the process exits.
+constexpr unsigned kStaticArgminTile = 16384;                                   // costs per block
+constexpr unsigned kStaticArgminBlocks = (unsigned)(HAP_ARGMIN_STATIC_MAX_COUNT / kStaticArgminTile);
+static __device__ __align__(256) unsigned char g_argmin_static_scratch[kStaticArgminBlocks * 16];
+
+// In host code the name above is only a handle for the runtime, not an address a kernel can use.
+// The device address is looked up once per device (with that device current) and cached here.
+static void *g_argmin_static_ptr[64];
+static bool g_argmin_static_ready[64];
+
+extern "C" hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream)
+{
+    if (!dev_cost || !dev_out) return HAP_E_INVALID;
+    if (count == 0 || count > HAP_ARGMIN_STATIC_MAX_COUNT) return HAP_E_RANGE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return HAP_E_CUDA;
+    if (dev < 0 || dev >= 64) return HAP_E_RANGE;
+    if (!g_argmin_static_ready[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_argmin_static_scratch) != cudaSuccess || !ptr) return HAP_E_CUDA;
+        g_argmin_static_ptr[dev] = ptr;
+        g_argmin_static_ready[dev] = true;
+    }
+    i64 *pcost = reinterpret_cast<i64 *>(g_argmin_static_ptr[dev]);
+    u64 *pindex = reinterpret_cast<u64 *>(pcost + kStaticArgminBlocks);
+    cudaStream_t st = (cudaStream_t)stream;
+    const unsigned blocks = (unsigned)((count + kStaticArgminTile - 1) / kStaticArgminTile);
+    // every partial that the second kernel reads is written by the first one in this same call, so
+    // nothing left in the scratch by an earlier call is ever read and nothing has to be cleared
+    argmin_partial_kernel<<<blocks, 256, 0, st>>>((const i64 *)dev_cost, count, pcost, pindex);
+    if (cudaGetLastError() != cudaSuccess) return HAP_E_CUDA;
+    argmin_final_kernel<<<1, 256, 0, st>>>(pcost, pindex, blocks, (i64 *)dev_out);
+    if (cudaGetLastError() != cudaSuccess) return HAP_E_CUDA;
+    return HAP_OK;
+}
