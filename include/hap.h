@@ -243,6 +243,12 @@ hap_status hap_argmin(hap_problem *, const int64_t *dev_cost, uint64_t count, in
 #define HAP_ARGMIN_STATIC_MAX_COUNT ((uint64_t)1 << 26)
 hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream);
 
+/* Measurement aid: the number of recurrence cells (i, j, k) of candidates [first, first+count) whose stage
+ * cost is finite, i.e. k inside the load-balance window of stage i (Pruning 1) and the span within the memory
+ * limit at some allowed recomputation level (Pruning 2).  This is the recurrence work the method defines for
+ * the range, independent of what the dynamic-program kernel skips or shares.  Synchronises `stream`. */
+hap_status hap_count_cells(hap_problem *, uint64_t first, uint64_t count, uint64_t *host_cells, void *stream);
+
 /* Measurement aid: CUDA-event durations (ms) of the layer-cost kernel and of the dynamic-program
  * kernel of the most recent hap_pipeline_dp / hap_search_* call, and the number of recurrence cell
  * updates (k, j pairs inside the window and the memory limit) that launch evaluated.  Waits for that

@@ -16,7 +16,7 @@ COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, S
 STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE", "HAP_E_STATE", "HAP_E_INFEASIBLE"]
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_search_range",
-           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_get_timings", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_count_cells", "hap_get_timings", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -266,6 +266,13 @@ def hap_search_best(hp: HapProblem, stream=None):
     pl, st = _Plan(), _Stats()
     hp.check(load_library().hap_search_best(hp.h, C.byref(pl), C.byref(st), _stream(stream)))
     return _plan_dict(pl), _stats_dict(st)
+
+
+def hap_count_cells(hp: HapProblem, first: int, count: int, stream=None) -> int:
+    """Finite-cost recurrence cells of candidates [first, first+count) (measurement aid)."""
+    c = C.c_uint64()
+    hp.check(load_library().hap_count_cells(hp.h, C.c_uint64(first), C.c_uint64(count), C.byref(c), _stream(stream)))
+    return int(c.value)
 
 
 ARGMIN_STATIC_MAX_COUNT = 1 << 26

@@ -517,7 +517,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
 {
     // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
     // process: raise it (never lower it) before a launch that needs more
-    static size_t smem_limit[64][4];
+    static size_t smem_limit[64][6];
     const int dev = p->device & 63;
     // fork: every PP class runs on its own stream so that the tail of one class overlaps the next
     CUDA_TRY(p, cudaEventRecord(p->ev_fork, st));
@@ -535,8 +535,9 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const bool outside = c1 <= out.first || c0 >= out.first + out.count;
         if (outside && !search) continue;
         const bool lin = p->dc.tau_linear != 0;
-        const int variant = (search ? 2 : 0) + (lin ? 1 : 0);
-        const void *fn = variant == 0 ? (const void *)pipeline_dp_kernel<false, false>
+        const int variant = out.count_only ? 4 + (lin ? 1 : 0) : (search ? 2 : 0) + (lin ? 1 : 0);
+        const void *fn = out.count_only ? (lin ? (const void *)pipeline_dp_kernel<false, true, true> : (const void *)pipeline_dp_kernel<false, false, true>)
+                         : variant == 0 ? (const void *)pipeline_dp_kernel<false, false>
                          : variant == 1 ? (const void *)pipeline_dp_kernel<false, true>
                          : variant == 2 ? (const void *)pipeline_dp_kernel<true, false>
                                         : (const void *)pipeline_dp_kernel<true, true>;
@@ -581,6 +582,25 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_count_cells(hap_problem *p, uint64_t first, uint64_t count, uint64_t *host_cells, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!host_cells) return HAP_E_INVALID;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    *host_cells = 0;
+    if (count == 0) return HAP_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    DpOut out{};
+    out.counters = p->d_counters; out.first = first; out.count = count; out.count_only = 1;
+    if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaMemcpyAsync(host_cells, p->d_counters + 4, sizeof(u64), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaStreamSynchronize(st));
     return HAP_OK;
 }
 

@@ -66,6 +66,7 @@ struct DpOut {
     u64 *counters;                    // [0] evaluated, [1] feasible, [2] pruned, [4] recurrence cells (nullable)
     u64 *incumbent;                   // running minimum of T_iter, for pruning
     int search, prune;
+    int count_only;                   // instrumentation: count the finite-cost cells of each candidate, run no recurrence
 };
 
 // ------------------------------------------------------------------------------------------
@@ -507,7 +508,7 @@ struct MaskInfo {
     int capt, pad;
 };
 
-template <bool SEARCH, bool LINEAR>
+template <bool SEARCH, bool LINEAR, bool COUNT = false>
 __global__ void __launch_bounds__(kDpWarps * 32)
 pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef,
                    const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
@@ -753,6 +754,27 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             sp.bl = bl; sp.bh = bh;
         }
         const bool dead = __any_sync(0xffffffffu, lane < PP && sp.bl > sp.bh);
+        if (COUNT) {
+            // cells (i, j, k) of this candidate's recurrence whose stage cost is finite: k inside the load-balance
+            // window of stage i and the span (k, j] within the memory limit at some allowed level
+            for (int i = 1; i <= PP; ++i) {
+                const int src = i - 1;
+                const int capt = __shfl_sync(0xffffffffu, sp.capt, src);
+                const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
+                const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
+                for (int j = i + lane; j <= N - PP + i; j += 32) {
+                    int klo = j - nmax; if (klo < i - 1) klo = i - 1;
+                    const int khi = j - nmin;
+                    int kf = 255;
+                    for (int r = 0; r < R; ++r)
+                        if ((rc_mask >> r) & 1u) { const int t = th[(size_t)r * n1 + j]; kf = t < kf ? t : kf; }
+                    if (kf > klo) klo = kf;
+                    if (klo <= khi) n_cells += (u64)(khi - klo + 1);
+                }
+            }
+            valid_rows = 0;
+            continue;
+        }
 
         // ---- recurrence -------------------------------------------------------------------
         i64 *tab_out = nullptr; uint8_t *ch_out = nullptr;

@@ -227,3 +227,26 @@ def test_random_small_problems_with_tight_memory(hap, seed):
         plan, _ = hap.hap_search_best(hp)
         assert plan["index"] == best["index"] and plan["n"] == best["n"] and plan["r"] == best["r"]
     hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("kw", [{}, {"window": True}])
+def test_finite_cell_count_matches_stage_cost_enumeration(hap, kw):
+    """hap_count_cells (the roofline's unit count) against a direct enumeration of (i, j, k) with the oracle's
+    stage cost, candidate by candidate."""
+    pb, hp, o = setup(hap, "tiny", **kw)
+    n_rc = len(pb.rc_masks)
+    for idx in list(range(0, o.n_cand, 37)) + [o.n_cand - 1]:
+        p = o.find_pconf(idx)
+        PP = int(o.pconfs["PP"][p])
+        local = idx - int(o.pconfs["offset"][p])
+        mp = o.decode(p, local // n_rc)
+        rc = int(pb.rc_masks[local % n_rc])
+        c2, _, coef, _ = o.layer_costs(p)
+        want = 0
+        for i in range(1, PP + 1):
+            for j in range(i, pb.N - PP + i + 1):
+                for k in range(i - 1, j):
+                    want += o.stage_cost(p, mp, rc, c2, coef, i, k, j)[0] < INF
+        assert hap.hap_count_cells(hp, idx, 1) == want, idx
+    total = hap.hap_count_cells(hp, 0, hp.n_cand)
+    assert total == sum(hap.hap_count_cells(hp, f, c) for f, c in ((0, 700), (700, hp.n_cand - 700)))
