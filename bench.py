@@ -232,13 +232,22 @@ def main():
     cells_finite = hap.hap_count_cells(hp, first, count)        # untimed instrumentation launch
 
     # full search through the search entry point (pruning allowed), wall clock call to return
-    search_ms = []
+    search_ms, pruned_ms = [], []
+    hp_pr = hap.hap_problem_create(pb, prune=1)
+    hap.hap_enumerate(hp_pr)
     for _ in range(3):
         flush.fill_(1)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         plan, stats = hap.hap_search_range(hp, first, count)
         search_ms.append(1e3 * (time.perf_counter() - t0))
+        flush.fill_(1)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        plan_pr, stats_pr = hap.hap_search_range(hp_pr, first, count)
+        pruned_ms.append(1e3 * (time.perf_counter() - t0))
+    assert plan_pr == plan
+    hap.hap_problem_destroy(hp_pr)
 
     # end to end through the C ABI from host buffers: create (H2D of the tables), enumerate (H2D of the
     # configuration table), search, read the plan back
@@ -283,6 +292,8 @@ def main():
                      ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
             gpu_launches=(4 + len(set(int(x) for x in pconfs["PP"]))) * args.steps,
             full_search_ms=statistics.median(search_ms),
+            full_search_pruned=dict(ms=statistics.median(pruned_ms), n_pruned=stats_pr["n_pruned"],
+                                    n_evaluated=stats_pr["n_evaluated"]),
             best=dict(cost=best[0], index=best[1], search_index=plan["index"]),
             kernels_ms=dict(layer_cost=lc_med, pipeline_dp=dp_med),
             roofline=dict(bound="alu", kernel="pipeline_dp_kernel (one launch per PP class, concurrent streams)",

@@ -209,6 +209,20 @@ hap_status hap_pipeline_dp(hap_problem *, uint64_t first, uint64_t count, int64_
                            int64_t *dev_bottleneck, uint8_t *dev_partition, uint8_t *dev_recompute,
                            int64_t *dev_dp_table, uint8_t *dev_choice, void *stream);
 
+/* fp64 mode of hap_pipeline_dp: layer times and time coefficients stay unrounded doubles (the recomputation
+ * factor is tau_q / 1024.0, an infeasible cost is +infinity); the memory test uses the same integer byte
+ * coefficients as the integer mode.  Results agree with a plain fp64 evaluation to about 1e-12 relative
+ * (prefix sums are formed in a different order), not bit for bit.
+ * dev_cost, dev_bottleneck: [count] double; dev_partition, dev_recompute: [count][HAP_MAX_PP] (nullable). */
+hap_status hap_pipeline_dp_f64(hap_problem *, uint64_t first, uint64_t count, double *dev_cost,
+                               double *dev_bottleneck, uint8_t *dev_partition, uint8_t *dev_recompute,
+                               void *stream);
+/* fp64 mode of hap_search_range (no pruning).  The plan's time fields are the fp64 values rounded to
+ * integer ns; the unrounded iteration time and bottleneck go to host_T_iter / host_bottleneck (nullable).
+ * Synchronises `stream`. */
+hap_status hap_search_range_f64(hap_problem *, uint64_t first, uint64_t count, hap_plan *host_out,
+                                double *host_T_iter, double *host_bottleneck, void *stream);
+
 /* Eq. 1: layer costs, dynamic program and argmin over candidates [first, first+count) with
  * ties going to the lowest index; writes the plan to host memory.  Synchronises `stream`.
  * host_stats is nullable.  Returns HAP_E_INFEASIBLE when no candidate is feasible. */

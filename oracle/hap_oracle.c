@@ -730,3 +730,202 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
     *best_index = gidx;
     return 0;
 }
+
+
+/* ==================================================================================== *
+ * fp64 mode: the same definitions with the layer costs and time coefficients kept as doubles
+ * (no rounding to integer ns); the memory test stays on the integer byte coefficients, the
+ * recomputation time factor is tau_q / 1024.0 and an infeasible cost is +infinity.
+ * ==================================================================================== */
+typedef struct {
+    int N, PP, R;
+    int64_t M;
+    uint32_t rc_mask;
+    const int32_t *xi_q, *tau_q;
+    double PF[ORC_MAX_PP][ORC_MAX_N + 1], PB[ORC_MAX_PP][ORC_MAX_N + 1];
+    int64_t PW[ORC_MAX_N + 1], PA[ORC_MAX_N + 1];
+    int32_t PK[ORC_MAX_N + 1];
+    int64_t cap[ORC_MAX_PP], mpre, mpost, mx;
+    double K[ORC_MAX_PP];
+    int32_t nmin[ORC_MAX_PP], nmax[ORC_MAX_PP];
+} stage_ctx_f;
+
+static double mask_max_f(const orc_problem *pr, unsigned mask, const double *coeff, int q)
+{
+    double best = 0.0;
+    int seen = 0;
+    for (int h = 0; h < pr->T; ++h)
+        if (mask & (1u << h)) {
+            double x = coeff[h * ORC_NCOEF + q];
+            if (!seen || x > best) best = x;
+            seen = 1;
+        }
+    return best;
+}
+
+static void ctx_build_f(stage_ctx_f *cx, const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                        uint32_t rc_mask, const double *c2f, const int64_t *coef, const double *coeff)
+{
+    const int N = pr->N, PP = pc->PP;
+    cx->N = N; cx->PP = PP; cx->R = pr->R; cx->M = pc->M; cx->rc_mask = rc_mask;
+    cx->xi_q = pr->xi_q; cx->tau_q = pr->tau_q;
+    orc_window(pr, pc, mp, cx->nmin, cx->nmax);
+    cx->PW[0] = cx->PA[0] = 0; cx->PK[0] = 0;
+    for (int l = 0; l < N; ++l) {
+        cx->PW[l + 1] = cx->PW[l] + coef[ORC_MW + pr->kind[l]];
+        cx->PA[l + 1] = cx->PA[l] + coef[ORC_MA + pr->kind[l]];
+        cx->PK[l + 1] = cx->PK[l] + (pr->kind[l] == ORC_MOE ? 1 : 0);
+    }
+    cx->mpre = coef[ORC_MPRE]; cx->mpost = coef[ORC_MPOST]; cx->mx = coef[ORC_MX];
+    for (int s = 0; s < PP; ++s) {
+        const unsigned mask = mp->mask[s];
+        const int i = s + 1;
+        cx->PF[s][0] = cx->PB[s][0] = 0.0;
+        for (int l = 0; l < N; ++l) {
+            double F = 0.0, Bk = 0.0;
+            int seen = 0;
+            for (int h = 0; h < pr->T; ++h)
+                if (mask & (1u << h)) {
+                    double qf = c2f[((int64_t)h * N + l) * 2], qb = c2f[((int64_t)h * N + l) * 2 + 1];
+                    if (!seen || qf > F) F = qf;
+                    if (!seen || qb > Bk) Bk = qb;
+                    seen = 1;
+                }
+            cx->PF[s][l + 1] = cx->PF[s][l] + F;
+            cx->PB[s][l + 1] = cx->PB[s][l] + Bk;
+        }
+        int64_t cap = 0;
+        int seen = 0;
+        for (int h = 0; h < pr->T; ++h)
+            if (mask & (1u << h)) {
+                if (!seen || pr->cap_eff[h] < cap) cap = pr->cap_eff[h];
+                seen = 1;
+            }
+        cx->cap[s] = cap;
+        double K = 0.0;
+        if (i == 1) K += mask_max_f(pr, mask, coeff, ORC_KPRE);
+        if (i == PP) K += mask_max_f(pr, mask, coeff, ORC_KPOST);
+        if (i > 1) {
+            int hb = mp->hb[s], ha = mp->ha[s];
+            if (mp->cls[s] == ORC_INTRA) K += coeff[hb * ORC_NCOEF + ORC_KP2P_INTRA];
+            else if (mp->cls[s] == ORC_INTER) K += coeff[hb * ORC_NCOEF + ORC_KP2P_INTER];
+            else K += coeff[hb * ORC_NCOEF + ORC_KP2P_CROSS + ha];
+        }
+        cx->K[s] = K;
+    }
+}
+
+static double ctx_stage_cost_f(const stage_ctx_f *cx, int i, int a, int b, int *r_out)
+{
+    const int s = i - 1, PP = cx->PP;
+    if (r_out) *r_out = -1;
+    const int n = b - a;
+    if (n < cx->nmin[s] || n > cx->nmax[s]) return INFINITY;
+    const int has_moe = cx->PK[b] - cx->PK[a] > 0;
+    const int64_t Wb = (cx->PW[b] - cx->PW[a]) + (i == 1 ? cx->mpre : 0) + (i == PP ? cx->mpost : 0)
+                       + (has_moe ? cx->mx : 0);
+    const int64_t Mstore = cx->M < PP - i + 1 ? cx->M : PP - i + 1;
+    const int64_t A = Mstore * (cx->PA[b] - cx->PA[a]);
+    int rstar = -1;
+    for (int r = 0; r < cx->R && rstar < 0; ++r)
+        if ((cx->rc_mask >> r) & 1u)
+            if (Wb + ((int64_t)cx->xi_q[r] * A) / 1024 <= cx->cap[s]) rstar = r;
+    if (rstar < 0) return INFINITY;
+    if (r_out) *r_out = rstar;
+    const double SF = cx->PF[s][b] - cx->PF[s][a], SB = cx->PB[s][b] - cx->PB[s][a];
+    return SF + SB + ((double)cx->tau_q[rstar] / 1024.0) * SF + cx->K[s];
+}
+
+int orc_candidate_f64(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                      const double *c2f, const int64_t *coef, const double *coeff, orc_result_f *res)
+{
+    const int N = pr->N, PP = pc->PP;
+    stage_ctx_f *cx = (stage_ctx_f *)malloc(sizeof(stage_ctx_f));
+    double *DPt = (double *)malloc(sizeof(double) * (size_t)(PP + 1) * (N + 1));
+    uint8_t *CH = (uint8_t *)malloc((size_t)(PP + 1) * (N + 1));
+    if (!DPt || !CH || !cx) { free(DPt); free(CH); free(cx); return -1; }
+    ctx_build_f(cx, pr, pc, mp, rc_mask, c2f, coef, coeff);
+#define DPAT(i, j) DPt[(size_t)(i) * (N + 1) + (j)]
+#define CHAT(i, j) CH[(size_t)(i) * (N + 1) + (j)]
+    for (int i = 0; i <= PP; ++i)
+        for (int j = 0; j <= N; ++j) { DPAT(i, j) = INFINITY; CHAT(i, j) = 255; }
+    DPAT(0, 0) = 0.0;
+    for (int i = 1; i <= PP; ++i)
+        for (int j = i; j <= N - PP + i; ++j)
+            for (int k = i - 1; k <= j - 1; ++k) {
+                if (!(DPAT(i - 1, k) < INFINITY)) continue;
+                double c = ctx_stage_cost_f(cx, i, k, j, NULL);
+                double v = DPAT(i - 1, k) > c ? DPAT(i - 1, k) : c;
+                if (v < DPAT(i, j)) { DPAT(i, j) = v; CHAT(i, j) = (uint8_t)k; }
+            }
+    memset(res, 0, sizeof(*res));
+    res->bottleneck = DPAT(PP, N);
+    if (!(res->bottleneck < INFINITY)) {
+        res->T_iter = res->T_pipe = INFINITY;
+        free(DPt); free(CH); free(cx);
+        return 1;
+    }
+    double sum = 0.0, mx = 0.0, tsync = 0.0, topt = 0.0;
+    int j = N;
+    for (int i = PP; i >= 1; --i) {
+        int k = CHAT(i, j), r;
+        double c = ctx_stage_cost_f(cx, i, k, j, &r);
+        res->n[i - 1] = (uint8_t)(j - k);
+        res->r[i - 1] = (uint8_t)r;
+        res->c[i - 1] = c;
+        if (c > mx) mx = c;
+        unsigned mask = mp->mask[i - 1];
+        double sy = mask_max_f(pr, mask, coeff, ORC_SLAT), op = 0.0;
+        for (int l = k; l < j; ++l) {
+            sy += mask_max_f(pr, mask, coeff, ORC_SBW + pr->kind[l]);
+            op += mask_max_f(pr, mask, coeff, ORC_OPT + pr->kind[l]);
+        }
+        if (sy > tsync) tsync = sy;
+        if (op > topt) topt = op;
+        j = k;
+    }
+    for (int i = 0; i < PP; ++i) sum += res->c[i];          /* stage 1 .. PP */
+    res->T_pipe = sum + (double)(pc->M - 1) * mx;
+    res->T_sync = tsync;
+    res->T_opt = topt;
+    res->T_iter = res->T_pipe + tsync + topt;
+    free(DPt); free(CH); free(cx);
+#undef DPAT
+#undef CHAT
+    return 0;
+}
+
+/* every candidate of every p_stride-th configuration in fp64 mode (OpenMP over configurations);
+ * costs / bottlenecks are indexed by candidate over the whole space, partitions as [n_cand][ORC_MAX_PP] */
+int orc_search_pconfs_f64(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
+                          uint64_t p_stride, uint64_t *n_done, double *costs, double *bottlenecks, uint8_t *parts)
+{
+    uint64_t done = 0;
+    if (p_stride == 0) p_stride = 1;
+    int64_t nsel = p_first < n_pconf ? (int64_t)((n_pconf - p_first + p_stride - 1) / p_stride) : 0;
+#pragma omp parallel for schedule(dynamic, 1) reduction(+ : done)
+    for (int64_t q = 0; q < nsel; ++q) {
+        uint64_t p = p_first + (uint64_t)q * p_stride;
+        const orc_pconf *pc = &pcs[p];
+        double *c2f = (double *)malloc(sizeof(double) * (size_t)pr->T * pr->N * 2);
+        int64_t coef[ORC_MAX_TYPES * ORC_NCOEF];
+        double coeff[ORC_MAX_TYPES * ORC_NCOEF];
+        orc_layer_costs(pr, pc, NULL, c2f, coef, coeff);
+        for (uint64_t map_idx = 0; map_idx < pc->nmap; ++map_idx) {
+            orc_mapping mp;
+            orc_decode(pr, pc, map_idx, &mp);
+            for (int rc = 0; rc < pr->n_rc; ++rc) {
+                orc_result_f res;
+                orc_candidate_f64(pr, pc, &mp, pr->rc_masks[rc], c2f, coef, coeff, &res);
+                uint64_t idx = pc->offset + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
+                if (costs) costs[idx] = res.T_iter;
+                if (bottlenecks) bottlenecks[idx] = res.bottleneck;
+                if (parts) memcpy(parts + idx * ORC_MAX_PP, res.n, ORC_MAX_PP);
+                done++;
+            }
+        }
+        free(c2f);
+    }
+    *n_done = done;
+    return 0;
+}

@@ -124,4 +124,15 @@ int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, ui
 int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
                       uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
                       int64_t *costs, int64_t *bottlenecks);
+
+/* fp64 mode (no rounding of times to integer ns); see hap_oracle.c */
+typedef struct {
+    double T_iter, bottleneck, T_pipe, T_sync, T_opt;
+    uint8_t n[ORC_MAX_PP], r[ORC_MAX_PP];
+    double c[ORC_MAX_PP];
+} orc_result_f;
+int orc_candidate_f64(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                      const double *c2f, const int64_t *coef, const double *coeff, orc_result_f *res);
+int orc_search_pconfs_f64(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
+                          uint64_t p_stride, uint64_t *n_done, double *costs, double *bottlenecks, uint8_t *parts);
 #endif

@@ -71,6 +71,12 @@ class Result(C.Structure):
                 ("r", C.c_uint8 * MAX_PP), ("c", C.c_int64 * MAX_PP)]
 
 
+class ResultF(C.Structure):
+    _fields_ = [("T_iter", C.c_double), ("bottleneck", C.c_double), ("T_pipe", C.c_double),
+                ("T_sync", C.c_double), ("T_opt", C.c_double), ("n", C.c_uint8 * MAX_PP),
+                ("r", C.c_uint8 * MAX_PP), ("c", C.c_double * MAX_PP)]
+
+
 class Plan(C.Structure):
     _fields_ = [("index", C.c_uint64), ("pc", PConf), ("map", Mapping), ("rc_mask", C.c_uint32), ("res", Result)]
 
@@ -260,3 +266,34 @@ class Oracle:
         if want_costs:
             return int(done.value), int(bc.value), int(bi.value), costs, bn
         return int(done.value), int(bc.value), int(bi.value)
+
+    # ---- fp64 mode ---------------------------------------------------------------------
+    def candidate_f64(self, p, mp, rc_mask, c2f, coef, coeff) -> ResultF:
+        res = ResultF()
+        self.L.orc_candidate_f64(C.byref(self.s), self._pc(p), C.byref(mp), C.c_uint32(rc_mask), _ptr(c2f), _ptr(coef),
+                                 _ptr(coeff), C.byref(res))
+        return res
+
+    def eval_index_f64(self, index: int) -> dict:
+        p = self.find_pconf(index)
+        n_rc = len(self.pb.rc_masks)
+        local = index - int(self.pconfs["offset"][p])
+        mp = self.decode(p, local // n_rc)
+        _, c2f, coef, coeff = self.layer_costs(p)
+        res = self.candidate_f64(p, mp, int(self.pb.rc_masks[local % n_rc]), c2f, coef, coeff)
+        PP = int(self.pconfs["PP"][p])
+        return dict(T_iter=res.T_iter, bottleneck=res.bottleneck, T_pipe=res.T_pipe, T_sync=res.T_sync, T_opt=res.T_opt,
+                    n=[int(x) for x in res.n[:PP]], r=[int(x) for x in res.r[:PP]], c=[float(x) for x in res.c[:PP]])
+
+    def search_pconfs_f64(self, p_first: int = 0, p_stride: int = 1, threads: int = 1):
+        """fp64-mode costs, bottlenecks and partitions of every candidate of every p_stride-th configuration."""
+        done = C.c_uint64()
+        costs = np.full(self.n_cand, -1.0, np.float64); bn = np.full(self.n_cand, -1.0, np.float64)
+        parts = np.zeros((self.n_cand, MAX_PP), np.uint8)
+        try:
+            C.CDLL("libgomp.so.1").omp_set_num_threads(C.c_int(threads))
+        except OSError:
+            pass
+        self.L.orc_search_pconfs_f64(C.byref(self.s), _ptr(self.pconfs), C.c_uint64(self.n_pconf), C.c_uint64(p_first),
+                                     C.c_uint64(p_stride), C.byref(done), _ptr(costs), _ptr(bn), _ptr(parts))
+        return int(done.value), costs, bn, parts

@@ -15,7 +15,8 @@ COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, S
             MW=13, MA=15, MX=17, MPRE=18, MPOST=19)
 STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE", "HAP_E_STATE", "HAP_E_INFEASIBLE"]
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
-           "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_search_range",
+           "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
+           "hap_search_range", "hap_search_range_f64",
            "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_count_cells", "hap_get_timings", "hap_status_str", "hap_last_error"]
 
 
@@ -241,6 +242,29 @@ def hap_pipeline_dp(hp: HapProblem, first: int, count: int, *, partition=False, 
                                             _dev(o["bottleneck"]), _dev(o.get("partition")), _dev(o.get("recompute")),
                                             _dev(o.get("dp_table")), _dev(o.get("choice")), _stream(stream)))
     return o
+
+
+def hap_pipeline_dp_f64(hp: HapProblem, first: int, count: int, *, partition=False, stream=None):
+    """fp64 mode: unrounded costs and bottlenecks (float64 CUDA tensors), optionally partitions and levels."""
+    import torch
+    o = {"cost": torch.empty(count, dtype=torch.float64, device="cuda"),
+         "bottleneck": torch.empty(count, dtype=torch.float64, device="cuda")}
+    if partition:
+        o["partition"] = torch.empty((count, MAX_PP), dtype=torch.uint8, device="cuda")
+        o["recompute"] = torch.empty((count, MAX_PP), dtype=torch.uint8, device="cuda")
+    hp.check(load_library().hap_pipeline_dp_f64(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(o["cost"]),
+                                                _dev(o["bottleneck"]), _dev(o.get("partition")), _dev(o.get("recompute")),
+                                                _stream(stream)))
+    return o
+
+
+def hap_search_range_f64(hp: HapProblem, first: int, count: int, stream=None):
+    pl, t, b = _Plan(), C.c_double(), C.c_double()
+    hp.check(load_library().hap_search_range_f64(hp.h, C.c_uint64(first), C.c_uint64(count), C.byref(pl), C.byref(t),
+                                                 C.byref(b), _stream(stream)))
+    d = _plan_dict(pl)
+    d["T_iter_f64"], d["bottleneck_f64"] = float(t.value), float(b.value)
+    return d
 
 
 def _plan_dict(pl: _Plan) -> dict:

@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdarg>
 #include <cstdio>
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <string>
@@ -42,6 +43,9 @@ struct hap_problem {
     hap_pconf *d_pconf = nullptr;
     WorkItem *d_items = nullptr;
     i64 *d_c2 = nullptr, *d_coef = nullptr;
+    double *d_c2f = nullptr, *d_coeff = nullptr;   // fp64-mode layer costs and coefficients (allocated on first use)
+    i64 *d_fcost = nullptr;                 // fp64-mode search: per-candidate costs (bit patterns), allocated on first use
+    i64 *d_lb = nullptr;                    // scratch: per-configuration lower bound on the summed stage time
     TypeConst *d_tc = nullptr;              // scratch: per (configuration, type) constants of the layer-cost kernels
     i64 *d_pcost = nullptr;                // per-block partial minima
     u64 *d_pindex = nullptr;
@@ -75,6 +79,8 @@ static hap_status fail(hap_problem *p, hap_status s, const char *fmt, ...)
     return s;
 }
 
+static hap_status argmin_launch(hap_problem *p, const hap::i64 *dev_cost, uint64_t count, hap::i64 *dev_out, cudaStream_t st, hap::i64 init);
+
 #define CUDA_TRY(p, call)                                                                          \
     do {                                                                                           \
         cudaError_t e_ = (call);                                                                   \
@@ -102,7 +108,7 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 static void release_device(hap_problem *p)
 {
     cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
-    cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
+    cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); }
@@ -401,6 +407,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         CUDA_TRY(p, cudaMalloc(&p->d_c2, np * T * N * 2 * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_coef, np * T * HAP_NCOEF * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_tc, np * T * sizeof(TypeConst)));
+        CUDA_TRY(p, cudaMalloc(&p->d_lb, np * sizeof(i64)));
         p->n_partial = std::max<size_t>(p->items.size(), 1024);
         CUDA_TRY(p, cudaMalloc(&p->d_pcost, p->n_partial * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_pindex, p->n_partial * sizeof(u64)));
@@ -479,7 +486,8 @@ extern "C" hap_status hap_decode(hap_problem *p, uint64_t first, uint64_t count,
     return HAP_OK;
 }
 
-static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st)
+static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st,
+                                     i64 *lb_sum = nullptr)
 {
     const u64 nph = (u64)p->pconfs.size() * HAP_MAX_TYPES;
     const unsigned b1 = (unsigned)((nph + kLcThreads - 1) / kLcThreads);
@@ -487,10 +495,10 @@ static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double 
     else type_const_kernel<false><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff);
     CUDA_TRY(p, cudaGetLastError());
     if ((quant && c2) || (!quant && c2f)) {
-        const unsigned b2 = (unsigned)(p->pconfs.size() * p->T);
+        const unsigned b2 = (unsigned)p->pconfs.size();
         const unsigned thr = (unsigned)((p->model.N + 31) / 32 * 32);
-        if (quant) layer_cost_kernel<true><<<b2, thr, 0, st>>>(p->dc, p->d_tc, c2, nullptr);
-        else layer_cost_kernel<false><<<b2, thr, 0, st>>>(p->dc, p->d_tc, nullptr, c2f);
+        if (quant) layer_cost_kernel<true><<<b2, thr, 0, st>>>(p->dc, p->d_tc, c2, nullptr, lb_sum);
+        else layer_cost_kernel<false><<<b2, thr, 0, st>>>(p->dc, p->d_tc, nullptr, c2f, nullptr);
     }
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
@@ -513,11 +521,11 @@ extern "C" hap_status hap_eval_layer_costs_f64(hap_problem *p, double *dev_c2, d
 }
 
 // One launch per PP class (each has its own block shape); every block clips to the candidate range.
-static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaStream_t st)
+static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaStream_t st, bool f64 = false)
 {
     // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
     // process: raise it (never lower it) before a launch that needs more
-    static size_t smem_limit[64][6];
+    static size_t smem_limit[64][8];
     const int dev = p->device & 63;
     // fork: every PP class runs on its own stream so that the tail of one class overlaps the next
     CUDA_TRY(p, cudaEventRecord(p->ev_fork, st));
@@ -535,8 +543,9 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const bool outside = c1 <= out.first || c0 >= out.first + out.count;
         if (outside && !search) continue;
         const bool lin = p->dc.tau_linear != 0;
-        const int variant = out.count_only ? 4 + (lin ? 1 : 0) : (search ? 2 : 0) + (lin ? 1 : 0);
-        const void *fn = out.count_only ? (lin ? (const void *)pipeline_dp_kernel<false, true, true> : (const void *)pipeline_dp_kernel<false, false, true>)
+        const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (search ? 2 : 0) + (lin ? 1 : 0);
+        const void *fn = f64 ? (lin ? (const void *)pipeline_dp_kernel<false, true, false, double> : (const void *)pipeline_dp_kernel<false, false, false, double>)
+                         : out.count_only ? (lin ? (const void *)pipeline_dp_kernel<false, true, true> : (const void *)pipeline_dp_kernel<false, false, true>)
                          : variant == 0 ? (const void *)pipeline_dp_kernel<false, false>
                          : variant == 1 ? (const void *)pipeline_dp_kernel<false, true>
                          : variant == 2 ? (const void *)pipeline_dp_kernel<true, false>
@@ -552,7 +561,9 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const WorkItem *its = p->d_items + cl.item_lo;
         int nw = cl.warps;
         unsigned used = cl.masks_used;
-        void *args[] = {(void *)&p->dc, (void *)&its, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tab, (void *)&o, (void *)&nw, (void *)&used};
+        void *c2arg = f64 ? (void *)p->d_c2f : (void *)p->d_c2;
+        void *cvarg = f64 ? (void *)p->d_coeff : (void *)p->d_coef;
+        void *args[] = {(void *)&p->dc, (void *)&its, (void *)&c2arg, (void *)&p->d_coef, (void *)&cvarg, (void *)&tab, (void *)&o, (void *)&nw, (void *)&used};
         CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
         CUDA_TRY(p, cudaLaunchKernel(fn, dim3(blocks), dim3(cl.warps * 32), args, cl.smem, cl.stream));
         CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
@@ -582,6 +593,89 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
+    return HAP_OK;
+}
+
+static hap_status ensure_f64_buffers(hap_problem *p)
+{
+    const size_t np = p->pconfs.size();
+    if (!p->d_c2f) CUDA_TRY(p, cudaMalloc(&p->d_c2f, np * p->T * p->model.N * 2 * sizeof(double)));
+    if (!p->d_coeff) CUDA_TRY(p, cudaMalloc(&p->d_coeff, np * p->T * HAP_NCOEF * sizeof(double)));
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_pipeline_dp_f64(hap_problem *p, uint64_t first, uint64_t count, double *dev_cost,
+                                          double *dev_bottleneck, uint8_t *dev_partition, uint8_t *dev_recompute,
+                                          void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    if (count == 0) return HAP_OK;
+    if ((s = ensure_f64_buffers(p)) != HAP_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
+    CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
+    // the memory model stays on the integer byte coefficients; times stay unrounded
+    if ((s = launch_layer_costs(p, nullptr, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, nullptr, nullptr, p->d_c2f, p->d_coeff, false, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
+    DpOut out{};
+    out.counters = p->d_counters;
+    out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
+    out.recompute = dev_recompute; out.first = first; out.count = count;
+    if ((s = launch_dp(p, out, false, st, true)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
+    p->timed = true;
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_search_range_f64(hap_problem *p, uint64_t first, uint64_t count, hap_plan *host_out,
+                                           double *host_T_iter, double *host_bottleneck, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!host_out) return HAP_E_INVALID;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    if (count == 0) return fail(p, HAP_E_RANGE, "empty candidate range");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!p->d_fcost) CUDA_TRY(p, cudaMalloc(&p->d_fcost, (size_t)p->n_cand * sizeof(i64)));
+    if ((s = hap_pipeline_dp_f64(p, first, count, (double *)p->d_fcost, nullptr, nullptr, nullptr, stream)) != HAP_OK) return s;
+    // non-negative doubles order like their bit patterns read as int64 (+inf is the largest), so the integer
+    // (cost, index) argmin serves the fp64 costs unchanged
+    if ((s = argmin_launch(p, p->d_fcost, count, p->d_best, st, 0x7fffffffffffffffll)) != HAP_OK) return s;
+    i64 best[2];
+    CUDA_TRY(p, cudaMemcpyAsync(best, p->d_best, sizeof(best), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaStreamSynchronize(st));
+    double bc;
+    std::memcpy(&bc, &best[0], sizeof(bc));
+    std::memset(host_out, 0, sizeof(*host_out));
+    if (!(bc < 1.0e300)) return fail(p, HAP_E_INFEASIBLE, "no candidate satisfies the memory constraint");
+    const u64 win = first + (u64)best[1];
+    SingleOut *d1 = (SingleOut *)p->d_single;
+    DpOut one{};
+    one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
+    one.recompute = d1->rec; one.first = win; one.count = 1;
+    if ((s = launch_dp(p, one, false, st, true)) != HAP_OK) return s;
+    decode_kernel<<<1, 32, 0, st>>>(p->dc, win, 1, &d1->cand);
+    CUDA_TRY(p, cudaGetLastError());
+    SingleOut h1;
+    CUDA_TRY(p, cudaMemcpyAsync(&h1, d1, sizeof(h1), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaStreamSynchronize(st));
+    const hap_candidate &hc = h1.cand;
+    const hap_pconf &pc = p->pconfs[hc.pconf];
+    host_out->index = win;
+    host_out->PP = pc.PP; host_out->TP = pc.TP; host_out->CP = pc.CP; host_out->DP = pc.DP; host_out->EP = pc.EP;
+    host_out->TPE = pc.TPE; host_out->b = pc.b; host_out->M = pc.M; host_out->rc_mask = hc.rc_mask;
+    std::memcpy(host_out->n, h1.part, HAP_MAX_PP);
+    std::memcpy(host_out->r, h1.rec, HAP_MAX_PP);
+    std::memcpy(host_out->mask, hc.mask, HAP_MAX_PP);
+    double v[5];
+    std::memcpy(&v[0], &h1.cost, 8); std::memcpy(&v[1], &h1.bott, 8); std::memcpy(&v[2], h1.detail, 24);
+    host_out->T_iter = (int64_t)llrint(v[0]); host_out->bottleneck = (int64_t)llrint(v[1]);
+    host_out->T_pipe = (int64_t)llrint(v[2]); host_out->T_sync = (int64_t)llrint(v[3]); host_out->T_opt = (int64_t)llrint(v[4]);
+    if (host_T_iter) *host_T_iter = v[0];
+    if (host_bottleneck) *host_bottleneck = v[1];
     return HAP_OK;
 }
 
@@ -616,18 +710,22 @@ extern "C" hap_status hap_get_timings(hap_problem *p, float *ms_layer_cost, floa
     return HAP_OK;
 }
 
+static hap_status argmin_launch(hap_problem *p, const i64 *dev_cost, uint64_t count, i64 *dev_out, cudaStream_t st, i64 init)
+{
+    const unsigned blocks = (unsigned)std::min<uint64_t>((count + 255) / 256, 1024);
+    argmin_partial_kernel<<<blocks, 256, 0, st>>>(dev_cost, count, p->d_pcost, p->d_pindex, init);
+    CUDA_TRY(p, cudaGetLastError());
+    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, blocks, dev_out, init);
+    CUDA_TRY(p, cudaGetLastError());
+    return HAP_OK;
+}
+
 extern "C" hap_status hap_argmin(hap_problem *p, const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream)
 {
     hap_status s = enter(p);
     if (s != HAP_OK) return s;
     if (!dev_cost || !dev_out || count == 0) return HAP_E_INVALID;
-    cudaStream_t st = (cudaStream_t)stream;
-    const unsigned blocks = (unsigned)std::min<uint64_t>((count + 255) / 256, 1024);
-    argmin_partial_kernel<<<blocks, 256, 0, st>>>((const i64 *)dev_cost, count, p->d_pcost, p->d_pindex);
-    CUDA_TRY(p, cudaGetLastError());
-    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, blocks, (i64 *)dev_out);
-    CUDA_TRY(p, cudaGetLastError());
-    return HAP_OK;
+    return argmin_launch(p, (const i64 *)dev_cost, count, (i64 *)dev_out, (cudaStream_t)stream, kInf);
 }
 
 extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t count, hap_plan *host_out,
@@ -640,16 +738,18 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     if (count == 0) return fail(p, HAP_E_RANGE, "empty candidate range");
     cudaStream_t st = (cudaStream_t)stream;
     std::memset(host_out, 0, sizeof(*host_out));
-    CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
+    const u64 init_counters[8] = {0, 0, 0, (u64)kInf, 0, 0, 0, 0};           // [3] = incumbent starts at +INF
+    CUDA_TRY(p, cudaMemcpyAsync(p->d_counters, init_counters, sizeof(init_counters), cudaMemcpyHostToDevice, st));
     CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
-    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st, p->d_lb)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     DpOut out{};
+    out.lb_sum = p->d_lb;
     out.first = first; out.count = count; out.search = 1; out.prune = p->opts.prune;
     out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
     out.incumbent = p->d_counters + 3;
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
-    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best);
+    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best, kInf);
     CUDA_TRY(p, cudaGetLastError());
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
@@ -734,9 +834,9 @@ extern "C" hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count,
     const unsigned blocks = (unsigned)((count + kStaticArgminTile - 1) / kStaticArgminTile);
     // every partial that the second kernel reads is written by the first one in this same call, so
     // nothing left in the scratch by an earlier call is ever read and nothing has to be cleared
-    argmin_partial_kernel<<<blocks, 256, 0, st>>>((const i64 *)dev_cost, count, pcost, pindex);
+    argmin_partial_kernel<<<blocks, 256, 0, st>>>((const i64 *)dev_cost, count, pcost, pindex, kInf);
     if (cudaGetLastError() != cudaSuccess) return HAP_E_CUDA;
-    argmin_final_kernel<<<1, 256, 0, st>>>(pcost, pindex, blocks, (i64 *)dev_out);
+    argmin_final_kernel<<<1, 256, 0, st>>>(pcost, pindex, blocks, (i64 *)dev_out, kInf);
     if (cudaGetLastError() != cudaSuccess) return HAP_E_CUDA;
     return HAP_OK;
 }

@@ -65,6 +65,7 @@ struct DpOut {
     u64 *partial_index;               // [gridDim.x]
     u64 *counters;                    // [0] evaluated, [1] feasible, [2] pruned, [4] recurrence cells (nullable)
     u64 *incumbent;                   // running minimum of T_iter, for pruning
+    const i64 *lb_sum;                // per configuration: sum over layers of the cheapest type's time
     int search, prune;
     int count_only;                   // instrumentation: count the finite-cost cells of each candidate, run no recurrence
 };
@@ -272,34 +273,74 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff)
     }
 }
 
-// one block per (configuration, type), threads over the layers
+// one block per configuration, one thread per layer; a thread handles its layer for every device type, so
+// that up to 16 table reads are in flight per thread before the first result is needed
 template <bool QUANT>
 __global__ void __launch_bounds__(256)
-layer_cost_kernel(const DevConst dc, const TypeConst *tcg, i64 *c2, double *c2f)
+layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__restrict__ c2, double *__restrict__ c2f,
+                  i64 *__restrict__ lb_sum)
 {
-    const int N = dc.N;
-    const unsigned ph = blockIdx.x;                                     // p*T + h
-    const int l = threadIdx.x;
-    if (l >= N) return;
-    const int h = (int)(ph % (unsigned)dc.T);
-    const TypeConst tc = tcg[ph];
-    const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
-    const size_t i5 = (size_t)h * stride_h + (size_t)tc.row * N + l;
-    const double a = dc.tdf[i5], ab = dc.tdb[i5];
-    double cf, cb;
-    if (layer_kind(dc, l) == HAP_DENSE) {
-        cf = a + tc.commF[HAP_DENSE];
-        cb = ab + tc.commB[HAP_DENSE];
-    } else {
-        const double f = dc.tff[i5], fb = dc.tfb[i5];
-        const double xf = div_by(dc.kappa * f, tc.den, tc.rden);
-        const double mf = (xf + tc.disp2) * tc.imb;
-        cf = (((a - f) + mf) + tc.tr) + tc.commF[HAP_MOE];
-        const double xb = div_by(dc.kappa * fb, tc.den, tc.rden);
-        const double mb = (xb + tc.disp2) * tc.imb;
-        cb = (((ab - fb) + mb) + tc.tr2) + tc.commB[HAP_MOE];
+    __shared__ TypeConst tcs[HAP_MAX_TYPES];
+    __shared__ i64 s_lb[8];
+    const int N = dc.N, T = dc.T;
+    const unsigned p = blockIdx.x;
+    {   // stage the configuration's per-type constants (11 doubles each) in shared memory
+        constexpr int W = sizeof(TypeConst) / 8;
+        const double *src = reinterpret_cast<const double *>(tcg + (size_t)p * T);
+        double *dst = reinterpret_cast<double *>(tcs);
+        for (int q = threadIdx.x; q < T * W; q += blockDim.x) dst[q] = src[q];
     }
-    store_pair<QUANT>(c2, c2f, ((size_t)ph * N + l) * 2, cf, cb);
+    __syncthreads();
+    const int l = threadIdx.x;
+    i64 lmin = 0;                       // min over device types of this layer's forward+backward time
+    if (l < N) {
+    const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
+    const bool dense = layer_kind(dc, l) == HAP_DENSE;
+    double a[HAP_MAX_TYPES], ab[HAP_MAX_TYPES], f[HAP_MAX_TYPES], fb[HAP_MAX_TYPES];
+#pragma unroll
+    for (int h = 0; h < HAP_MAX_TYPES; ++h) {
+        if (h < T) {
+            const size_t i5 = (size_t)h * stride_h + (size_t)tcs[h].row * N + l;
+            a[h] = __ldg(dc.tdf + i5); ab[h] = __ldg(dc.tdb + i5);
+            f[h] = dense ? 0.0 : __ldg(dc.tff + i5); fb[h] = dense ? 0.0 : __ldg(dc.tfb + i5);
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < HAP_MAX_TYPES; ++h) {
+        if (h < T) {
+            const TypeConst &tc = tcs[h];
+            double cf, cb;
+            if (dense) {
+                cf = a[h] + tc.commF[HAP_DENSE];
+                cb = ab[h] + tc.commB[HAP_DENSE];
+            } else {
+                const double xf = div_by(dc.kappa * f[h], tc.den, tc.rden);
+                const double mf = (xf + tc.disp2) * tc.imb;
+                cf = (((a[h] - f[h]) + mf) + tc.tr) + tc.commF[HAP_MOE];
+                const double xb = div_by(dc.kappa * fb[h], tc.den, tc.rden);
+                const double mb = (xb + tc.disp2) * tc.imb;
+                cb = (((ab[h] - fb[h]) + mb) + tc.tr2) + tc.commB[HAP_MOE];
+            }
+            store_pair<QUANT>(c2, c2f, (((size_t)p * T + h) * N + l) * 2, cf, cb);
+            if (QUANT) {
+                const i64 q = __double2ll_rn(cf) + __double2ll_rn(cb);
+                lmin = (h == 0 || q < lmin) ? q : lmin;
+            }
+        }
+    }
+    }
+    // every layer runs on some device type, so the sum over layers of the cheapest type's time bounds the
+    // summed stage time of every candidate of this configuration from below (used by the search's pruning)
+    if (QUANT && lb_sum) {
+        lmin = warp_sum_i64(lmin);
+        if ((threadIdx.x & 31) == 0) s_lb[threadIdx.x >> 5] = lmin;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            i64 t = 0;
+            for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += s_lb[w];
+            lb_sum[p] = t;
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -485,9 +526,10 @@ __host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int
     return b + 32;
 }
 
+template <typename VT>
 struct StagePar {
     int mrow, capt;             // row of the stage's type mask in sR; index of the type whose capacity binds
-    i64 K;                      // stage constant: pre/post work + p2p transfer into the stage
+    VT K;                       // stage constant: pre/post work + p2p transfer into the stage
     int nmin, nmax;             // load-balance window on the layer count
     int bl, bh;                 // band of end layers j that can be reached at this stage
 };
@@ -501,18 +543,34 @@ __device__ __forceinline__ bool span_fits(const i64 *sW, const i64 *sA, const ui
     return Wb + ((xi * A) >> 10) <= cap;               // A >= 0: the shift is the floor division by 1024
 }
 
+// value type of the times: int64 (rounded ns, exact arithmetic) or double (fp64 mode)
+template <typename VT> struct ValInf;
+template <> struct ValInf<i64> { static __device__ __forceinline__ i64 get() { return kInf; } };
+template <> struct ValInf<double> { static __device__ __forceinline__ double get() { return __longlong_as_double(0x7ff0000000000000ll); } };
+
+template <typename VT> __device__ __forceinline__ VT shfl_v(VT v, int src) { return __shfl_sync(0xffffffffu, v, src); }
+
+// forward-recomputation time: floor(tau * F / 1024) on integers (F >= 0), (tau / 1024.0) * F in fp64 mode
+__device__ __forceinline__ i64 tau_term(i64 tau, i64 F) { return (tau * F) >> 10; }
+__device__ __forceinline__ double tau_term(i64 tau, double F) { return ((double)tau / 1024.0) * F; }
+
 // per type mask: what a stage made of these device types costs beyond its layers (slowest member),
 // which member's memory binds, and the slowest member's compute rate for the load-balance window
+template <typename VT>
 struct MaskInfo {
-    i64 kpre, kpost, slat, sbw[2], opt[2], Pmin;
+    VT kpre, kpost, slat, sbw[2], opt[2];
+    i64 Pmin;
     int capt, pad;
 };
 
-template <bool SEARCH, bool LINEAR, bool COUNT = false>
+template <bool SEARCH, bool LINEAR, bool COUNT = false, typename VT = i64>
 __global__ void __launch_bounds__(kDpWarps * 32)
-pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, const i64 *coef,
+pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const i64 *coef, const VT *coefv,
                    const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
 {
+    // c2: layer times; coef: integer coefficients (memory bytes); coefv: time coefficients in the value type
+    // (the same array as coef in integer mode)
+    const VT vInf = ValInf<VT>::get();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -526,13 +584,30 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
             return;
         }
     }
+    if (SEARCH && out.prune) {
+        // T_iter >= sum_i c_i + (M-1) max_i c_i >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on
+        // the summed stage time.  Skipping needs bound > incumbent (strict): the result cannot change.
+        const i64 S = out.lb_sum[it.p];
+        const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
+        const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+        if ((u64)lb > inc) {
+            if (threadIdx.x == 0) {
+                out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
+                // candidates of this block inside the requested range
+                const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
+                const u64 a = c0 > out.first ? c0 : out.first, b = c1 < out.first + out.count ? c1 : out.first + out.count;
+                atomicAdd(out.counters + 2, b - a);
+            }
+            return;
+        }
+    }
     const bool multiset = pc.mode == HAP_MAP_MULTISET;
     const int nmask = (1 << T) - 1;
     const int mrows = multiset ? T : nmask;
     const int RW = LINEAR ? R : 2;
 
-    i64 *sR = reinterpret_cast<i64 *>(smem_raw);
-    i64 *sW = sR + (size_t)mrows * RW * n1;
+    VT *sR = reinterpret_cast<VT *>(smem_raw);
+    i64 *sW = reinterpret_cast<i64 *>(sR + (size_t)mrows * RW * n1);
     i64 *sA = sW + n1;
     uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
     const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
@@ -540,71 +615,80 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     const int nrows = multiset ? PP : (PP < 2 ? PP : 2);   // block mode shares nothing between mappings: two rotating rows
     const size_t row_bytes = (size_t)nrows * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
     unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
-    i64 *rows = reinterpret_cast<i64 *>(wbase);            // row of stage i at rows + ((i-1) % nrows)*n1
+    VT *rows = reinterpret_cast<VT *>(wbase);            // row of stage i at rows + ((i-1) % nrows)*n1
     uint8_t *chw = wbase + row_bytes;
-    __shared__ MaskInfo minfo[kMaxMasks];
-    __shared__ i64 sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
-    __shared__ i64 szero[1];                               // the row of "stage 0": DP[0][0] = 0
+    __shared__ MaskInfo<VT> minfo[kMaxMasks];
+    __shared__ VT sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
+    __shared__ VT szero[1];                               // the row of "stage 0": DP[0][0] = 0
     __shared__ int winT[HAP_MAX_TYPES][2];
 
     // ---- block prologue 1: rows of this configuration -----------------------------------
-    const i64 *c2p = c2 + (size_t)it.p * T * N * 2;
+    const VT *c2p = c2 + (size_t)it.p * T * N * 2;
     const i64 *cfp = coef + (size_t)it.p * T * HAP_NCOEF;
-    for (int mr = wib; mr <= mrows; mr += nwarps) {
-        // mr < mrows: time rows of one type mask; mr == mrows: the byte rows
+    const VT *cvp = coefv + (size_t)it.p * T * HAP_NCOEF;
+    for (int mr = wib; mr < mrows; mr += nwarps) {
+        // time rows of one type mask: per layer the slowest member type, then prefix sums
         const int mk = multiset ? (1 << mr) : mr + 1;
-        if (mr < mrows && !((masks_used >> mk) & 1u)) continue;     // no mapping of this class has such a stage
-        i64 runC = 0, runF = 0;
+        if (!((masks_used >> mk) & 1u)) continue;                   // no mapping of this class has such a stage
+        VT runC = 0, runF = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
-            i64 vC = 0, vF = 0;
+            VT vC = 0, vF = 0;
             if (l < N) {
-                if (mr < mrows) {
-                    i64 F = 0, B = 0;
-                    for (int h = 0; h < T; ++h)
-                        if (mk >> h & 1) {
-                            const longlong2 q = *reinterpret_cast<const longlong2 *>(c2p + ((size_t)h * N + l) * 2);
-                            F = q.x > F ? q.x : F;
-                            B = q.y > B ? q.y : B;
-                        }
-                    vC = F + B; vF = F;
-                } else {
-                    const int kd = layer_kind(dc, l);
-                    vC = cfp[HAP_MW + kd]; vF = cfp[HAP_MA + kd];
-                }
+                VT F = 0, B = 0;
+                for (int h = 0; h < T; ++h)
+                    if (mk >> h & 1) {
+                        const VT qx = c2p[((size_t)h * N + l) * 2], qy = c2p[((size_t)h * N + l) * 2 + 1];
+                        F = qx > F ? qx : F;
+                        B = qy > B ? qy : B;
+                    }
+                vC = F + B; vF = F;
             }
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {      // inclusive warp scan
-                const i64 tC = __shfl_up_sync(0xffffffffu, vC, o), tF = __shfl_up_sync(0xffffffffu, vF, o);
+                const VT tC = __shfl_up_sync(0xffffffffu, vC, o), tF = __shfl_up_sync(0xffffffffu, vF, o);
                 if (lane >= o) { vC += tC; vF += tF; }
             }
             vC += runC; vF += runF;
             if (l < N) {
-                if (mr < mrows) {
-                    if (LINEAR) {
-                        for (int r = 0; r < R; ++r) sR[((size_t)mr * RW + r) * n1 + l + 1] = vC + (i64)(dc.tau_q[r] >> 10) * vF;
-                    } else {
-                        sR[((size_t)mr * RW) * n1 + l + 1] = vC; sR[((size_t)mr * RW + 1) * n1 + l + 1] = vF;
-                    }
-                } else { sW[l + 1] = vC; sA[l + 1] = vF; }
+                if (LINEAR) {
+                    for (int r = 0; r < R; ++r) sR[((size_t)mr * RW + r) * n1 + l + 1] = vC + (VT)(dc.tau_q[r] >> 10) * vF;
+                } else {
+                    sR[((size_t)mr * RW) * n1 + l + 1] = vC; sR[((size_t)mr * RW + 1) * n1 + l + 1] = vF;
+                }
             }
-            runC = shfl_i64(vC, 31); runF = shfl_i64(vF, 31);
+            runC = shfl_v(vC, 31); runF = shfl_v(vF, 31);
         }
-        if (lane == 0) {
-            if (mr < mrows) { for (int r = 0; r < RW; ++r) sR[((size_t)mr * RW + r) * n1] = 0; }
-            else { sW[0] = 0; sA[0] = 0; }
+        if (lane == 0) for (int r = 0; r < RW; ++r) sR[((size_t)mr * RW + r) * n1] = 0;
+    }
+    if (wib == mrows % nwarps) {
+        // byte rows (integers in both modes): weights and activations per layer kind, prefix sums
+        i64 runW = 0, runA = 0;
+        for (int base = 0; base < N; base += 32) {
+            const int l = base + lane;
+            i64 vW = 0, vA = 0;
+            if (l < N) { const int kd = layer_kind(dc, l); vW = cfp[HAP_MW + kd]; vA = cfp[HAP_MA + kd]; }
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const i64 tW = __shfl_up_sync(0xffffffffu, vW, o), tA = __shfl_up_sync(0xffffffffu, vA, o);
+                if (lane >= o) { vW += tW; vA += tA; }
+            }
+            vW += runW; vA += runA;
+            if (l < N) { sW[l + 1] = vW; sA[l + 1] = vA; }
+            runW = shfl_i64(vW, 31); runA = shfl_i64(vA, 31);
         }
+        if (lane == 0) { sW[0] = 0; sA[0] = 0; }
     }
     for (int l = threadIdx.x; l <= N; l += nwarps * 32) sK[l] = (uint8_t)moe_before(dc, l);
     if (threadIdx.x < nmask) {
         const int mk = threadIdx.x + 1;
-        MaskInfo mi;
-        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
+        MaskInfo<VT> mi;
+        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
         i64 cap = 0;
         bool seen = false;
         for (int h = 0; h < T; ++h)
             if (mk >> h & 1) {
-                const i64 *row = cfp + h * HAP_NCOEF;
+                const VT *row = cvp + h * HAP_NCOEF;
                 if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; mi.capt = h; }
                 if (!seen || dc.P[h] < mi.Pmin) mi.Pmin = dc.P[h];
                 if (!seen || row[HAP_KPRE] > mi.kpre) mi.kpre = row[HAP_KPRE];
@@ -620,7 +704,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     }
     if (threadIdx.x >= 32 && threadIdx.x < 32 + T * 6) {
         const int q = threadIdx.x - 32, h = q / 6, e = q % 6;
-        sP2P[h][e] = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
+        sP2P[h][e] = cvp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
     }
     if (threadIdx.x == 0) szero[0] = 0;
     __syncthreads();
@@ -659,7 +743,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
     }
     __syncthreads();
 
-    i64 best_cost = kInf;
+    VT best_cost = vInf;
     u64 best_index = ~0ull;
     u64 n_eval = 0, n_feas = 0, n_cells = 0;
     const bool want_tables = !SEARCH && (out.dp_table != nullptr || out.choice != nullptr);
@@ -701,11 +785,11 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         int s0 = differ ? __ffs(differ) - 1 : PP;      // stages 1..s0 are shared with the previous mapping
         prev_mask = mask; prev_link = link;
 
-        StagePar sp;
+        StagePar<VT> sp;
         sp.mrow = 0; sp.capt = 0; sp.K = 0; sp.nmin = 1; sp.nmax = N - PP + 1; sp.bl = 0; sp.bh = 0;
         i64 Pmin = 0;
         if (lane < PP) {
-            const MaskInfo &mi_ = minfo[mask - 1];
+            const MaskInfo<VT> &mi_ = minfo[mask - 1];
             sp.mrow = multiset ? __ffs(mask) - 1 : mask - 1;
             sp.capt = mi_.capt; Pmin = mi_.Pmin;
             if (lane == 0) sp.K += mi_.kpre;
@@ -777,33 +861,33 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         }
 
         // ---- recurrence -------------------------------------------------------------------
-        i64 *tab_out = nullptr; uint8_t *ch_out = nullptr;
+        VT *tab_out = nullptr; uint8_t *ch_out = nullptr;
         if (want_tables) {
-            if (out.dp_table) tab_out = out.dp_table + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
+            if (out.dp_table) tab_out = reinterpret_cast<VT *>(out.dp_table) + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
             if (out.choice) ch_out = out.choice + (size_t)(c - out.first) * (HAP_MAX_PP + 1) * n1;
             for (int j = lane; j <= N; j += 32) {
-                if (tab_out) tab_out[j] = j == 0 ? 0 : kInf;
+                if (tab_out) tab_out[j] = j == 0 ? (VT)0 : vInf;
                 if (ch_out) ch_out[j] = 255;
             }
         }
-        i64 bott = kInf;
+        VT bott = vInf;
         if (!dead || want_tables) {
             int pbl = 0, pbh = 0;                          // band of the previous stage (stage 0: {0})
             if (s0 > 0) { pbl = __shfl_sync(0xffffffffu, sp.bl, s0 - 1); pbh = __shfl_sync(0xffffffffu, sp.bh, s0 - 1); }
             for (int i = s0 + 1; i <= PP; ++i) {
                 const int src = i - 1;
                 const int mrow = __shfl_sync(0xffffffffu, sp.mrow, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
-                const i64 K = shfl_i64(sp.K, src);
+                const VT K = shfl_v(sp.K, src);
                 const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
                 const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
-                const i64 *rM = sR + (size_t)mrow * RW * n1;
+                const VT *rM = sR + (size_t)mrow * RW * n1;
                 const int ri = multiset ? i - 1 : (i - 1) & 1;          // two rotating rows in block mode
-                const i64 *prev = i == 1 ? szero : rows + (multiset ? ri - 1 : ri ^ 1) * n1;
-                i64 *cur = rows + ri * n1;
+                const VT *prev = i == 1 ? szero : rows + (multiset ? ri - 1 : ri ^ 1) * n1;
+                VT *cur = rows + ri * n1;
                 uint8_t *chrow = chw + (size_t)(i - 1) * n1;
                 const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
                 for (int j = bl + lane; j <= bh; j += 32) {
-                    i64 best = kInf;
+                    VT best = vInf;
                     int arg = 255;
                     int klo = j - nmax; if (klo < pbl) klo = pbl;
                     int khi = j - nmin; if (khi > pbh) khi = pbh;
@@ -816,22 +900,23 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                             if (lo > seg_hi) continue;
                             n_cells += (u64)(seg_hi - lo + 1);
                             if (LINEAR) {
-                                const i64 *rr = rM + (size_t)r * n1;
-                                const i64 Cj = rr[j] + K;
+                                const VT *rr = rM + (size_t)r * n1;
+                                const VT Cj = rr[j] + K;
                                 for (int k = seg_hi; k >= lo; --k) {
-                                    const i64 pv = prev[k];
-                                    const i64 cst = Cj - rr[k];
-                                    const i64 v = pv > cst ? pv : cst;
-                                    if (v <= best && v < kInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
+                                    const VT pv = prev[k];
+                                    const VT cst = Cj - rr[k];
+                                    const VT v = pv > cst ? pv : cst;
+                                    if (v <= best && v < vInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
                                 }
                             } else {
-                                const i64 *rC = rM, *rF = rM + n1;
-                                const i64 Cj = rC[j] + K, Fj = rF[j], tau = dc.tau_q[r];
+                                const VT *rC = rM, *rF = rM + n1;
+                                const VT Cj = rC[j] + K, Fj = rF[j];
+                                const i64 tau = dc.tau_q[r];
                                 for (int k = seg_hi; k >= lo; --k) {
-                                    const i64 pv = prev[k];
-                                    const i64 cst = (Cj - rC[k]) + ((tau * (Fj - rF[k])) >> 10);   // forward sums are non-negative
-                                    const i64 v = pv > cst ? pv : cst;
-                                    if (v <= best && v < kInf) { best = v; arg = k; }
+                                    const VT pv = prev[k];
+                                    const VT cst = (Cj - rC[k]) + tau_term(tau, Fj - rF[k]);   // forward sums are non-negative
+                                    const VT v = pv > cst ? pv : cst;
+                                    if (v <= best && v < vInf) { best = v; arg = k; }
                                 }
                             }
                             seg_hi = lo - 1;
@@ -844,7 +929,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 if (want_tables) {
                     for (int j = lane; j <= N; j += 32) {
                         const bool in = j >= bl && j <= bh;
-                        if (tab_out) tab_out[(size_t)i * n1 + j] = in ? cur[j] : kInf;
+                        if (tab_out) tab_out[(size_t)i * n1 + j] = in ? cur[j] : vInf;
                         if (ch_out) ch_out[(size_t)i * n1 + j] = in ? chrow[j] : (uint8_t)255;
                     }
                 }
@@ -860,9 +945,9 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         __syncwarp();
 
         // ---- backtrace, Eq. 4 -----------------------------------------------------------
-        i64 T_iter = kInf, T_pipe = kInf, T_sync = 0, T_opt = 0;
+        VT T_iter = vInf, T_pipe = vInf, T_sync = 0, T_opt = 0;
         int my_n = 0, my_r = 0;
-        if (bott < kInf) {
+        if (bott < vInf) {
             int a_me = 0, b_me = 0;
             int j = N;
             for (int i = PP; i >= 1; --i) {
@@ -870,44 +955,50 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
                 if (lane == i - 1) { a_me = k; b_me = j; }
                 j = k;
             }
-            i64 c_me = 0, sync_me = 0, opt_me = 0;
+            VT c_me = 0, sync_me = 0, opt_me = 0;
             if (lane < PP) {
                 const uint8_t *th = thr + ((size_t)lane * T + sp.capt) * R * n1;
                 int r = 0;
                 for (; r < R; ++r)
                     if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b_me] <= a_me) break;
-                const i64 *rM = sR + (size_t)sp.mrow * RW * n1;
+                const VT *rM = sR + (size_t)sp.mrow * RW * n1;
                 if (LINEAR) c_me = (rM[(size_t)r * n1 + b_me] - rM[(size_t)r * n1 + a_me]) + sp.K;
-                else c_me = (rM[b_me] - rM[a_me]) + (((i64)dc.tau_q[r] * (rM[n1 + b_me] - rM[n1 + a_me])) >> 10) + sp.K;
+                else c_me = ((rM[b_me] - rM[a_me]) + tau_term((i64)dc.tau_q[r], rM[n1 + b_me] - rM[n1 + a_me])) + sp.K;
                 my_n = b_me - a_me; my_r = r;
-                const i64 n_moe = (int)sK[b_me] - (int)sK[a_me], n_dense = (b_me - a_me) - n_moe;
-                const MaskInfo &mi_ = minfo[mask - 1];
+                const VT n_moe = (VT)((int)sK[b_me] - (int)sK[a_me]), n_dense = (VT)(b_me - a_me) - n_moe;
+                const MaskInfo<VT> &mi_ = minfo[mask - 1];
                 sync_me = mi_.slat + n_dense * mi_.sbw[0] + n_moe * mi_.sbw[1];
                 opt_me = n_dense * mi_.opt[0] + n_moe * mi_.opt[1];
             }
-            i64 sum = c_me, mxc = c_me;
+            VT sum = c_me, mxc = c_me;
             for (int o = red0; o > 0; o >>= 1) {          // lanes >= PP hold zeros
-                const i64 t1 = __shfl_xor_sync(0xffffffffu, sum, o), t2 = __shfl_xor_sync(0xffffffffu, mxc, o);
-                const i64 t3 = __shfl_xor_sync(0xffffffffu, sync_me, o), t4 = __shfl_xor_sync(0xffffffffu, opt_me, o);
+                const VT t1 = __shfl_xor_sync(0xffffffffu, sum, o), t2 = __shfl_xor_sync(0xffffffffu, mxc, o);
+                const VT t3 = __shfl_xor_sync(0xffffffffu, sync_me, o), t4 = __shfl_xor_sync(0xffffffffu, opt_me, o);
                 sum += t1; mxc = t2 > mxc ? t2 : mxc; sync_me = t3 > sync_me ? t3 : sync_me; opt_me = t4 > opt_me ? t4 : opt_me;
             }
-            T_pipe = shfl_i64(sum + (i64)(pc.M - 1) * mxc, 0);
-            T_sync = shfl_i64(sync_me, 0); T_opt = shfl_i64(opt_me, 0);
+            T_pipe = shfl_v(sum + (VT)(pc.M - 1) * mxc, 0);
+            T_sync = shfl_v(sync_me, 0); T_opt = shfl_v(opt_me, 0);
             T_iter = T_pipe + T_sync + T_opt;
         }
         if (SEARCH) {
             n_eval++;
-            if (T_iter < kInf) n_feas++;
-            if (T_iter < best_cost || (T_iter == best_cost && c < best_index)) { best_cost = T_iter; best_index = c; }
+            if (T_iter < vInf) n_feas++;
+            if (T_iter < best_cost || (T_iter == best_cost && c < best_index)) {
+                best_cost = T_iter; best_index = c;
+                if (out.prune && lane == 0) atomicMin(out.incumbent, (u64)(i64)T_iter);
+            }
         } else {
             const u64 o = c - out.first;
             if (lane == 0) {
-                if (out.cost) out.cost[o] = T_iter;
-                if (out.bottleneck) out.bottleneck[o] = bott < kInf ? bott : kInf;
-                if (out.detail) { out.detail[o * 3] = T_pipe; out.detail[o * 3 + 1] = T_sync; out.detail[o * 3 + 2] = T_opt; }
+                if (out.cost) reinterpret_cast<VT *>(out.cost)[o] = T_iter;
+                if (out.bottleneck) reinterpret_cast<VT *>(out.bottleneck)[o] = bott;
+                if (out.detail) {
+                    VT *d = reinterpret_cast<VT *>(out.detail);
+                    d[o * 3] = T_pipe; d[o * 3 + 1] = T_sync; d[o * 3 + 2] = T_opt;
+                }
             }
-            if (out.partition) out.partition[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < kInf ? my_n : 0);
-            if (out.recompute) out.recompute[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < kInf ? my_r : 0);
+            if (out.partition) out.partition[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < vInf ? my_n : 0);
+            if (out.recompute) out.recompute[o * HAP_MAX_PP + lane] = (uint8_t)(T_iter < vInf ? my_r : 0);
         }
         __syncwarp();
       }
@@ -921,7 +1012,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
         __shared__ i64 wcost[kDpWarps];
         __shared__ u64 widx[kDpWarps];
         if (lane == 0) {
-            wcost[wib] = best_cost; widx[wib] = best_index;
+            wcost[wib] = (i64)best_cost; widx[wib] = best_index;
             if (n_eval) atomicAdd(out.counters + 0, n_eval);
             if (n_feas) atomicAdd(out.counters + 1, n_feas);
         }
@@ -940,9 +1031,11 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const i64 *c2, cons
 // argmin: stage 1 reduces a slice per block, stage 2 (one block) reduces the partials
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex)
+argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex, i64 init)
 {
-    i64 bc = kInf; u64 bi = ~0ull;
+    // `init` is the value reported when nothing is smaller: HAP_INF for integer costs, INT64_MAX when the
+    // array holds the bit patterns of non-negative doubles (which order like the doubles themselves)
+    i64 bc = init; u64 bi = ~0ull;
     for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (u64)gridDim.x * blockDim.x) {
         const i64 v = cost[i];
         if (v < bc) { bc = v; bi = i; }      // ascending i per thread: strict keeps the lowest index
@@ -959,9 +1052,9 @@ argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex)
 }
 
 __global__ void __launch_bounds__(256)
-argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2)
+argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2, i64 init)
 {
-    i64 bc = kInf; u64 bi = ~0ull;
+    i64 bc = init; u64 bi = ~0ull;
     for (u64 i = threadIdx.x; i < n; i += blockDim.x) {
         const i64 v = pcost[i]; const u64 ix = pindex[i];
         if (v < bc || (v == bc && ix < bi)) { bc = v; bi = ix; }

@@ -250,3 +250,58 @@ def test_finite_cell_count_matches_stage_cost_enumeration(hap, kw):
         assert hap.hap_count_cells(hp, idx, 1) == want, idx
     total = hap.hap_count_cells(hp, 0, hp.n_cand)
     assert total == sum(hap.hap_count_cells(hp, f, c) for f, c in ((0, 700), (700, hp.n_cand - 700)))
+
+
+@pytest.mark.parametrize("name", CONFIGS)
+def test_pruned_search_returns_the_same_plan(hap, name):
+    """Lower-bound pruning against the running incumbent must not change the answer (strict bound, ties to the
+    lowest index), whatever order the blocks ran in."""
+    pb, hp, o = setup(hap, name)
+    ref, stats0 = hap.hap_search_best(hp)
+    hp2 = hap.hap_problem_create(pb, prune=1)
+    hap.hap_enumerate(hp2)
+    for _ in range(3):
+        plan, stats = hap.hap_search_best(hp2)
+        assert plan == ref
+        assert stats["n_evaluated"] + stats["n_pruned"] == o.n_cand and stats0["n_pruned"] == 0
+    if name in ("dsv2", "stress"):
+        assert stats["n_pruned"] > 0
+    # a sub-range that does not contain the global optimum
+    first, count = o.n_cand // 3, o.n_cand // 5
+    a, _ = hap.hap_search_range(hp, first, count)
+    b, sb = hap.hap_search_range(hp2, first, count)
+    assert a == b and sb["n_evaluated"] + sb["n_pruned"] == count
+    hap.hap_problem_destroy(hp2)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}),
+                                     ("dsv2", {}), ("stress", {})])
+def test_fp64_mode_costs_within_1e9_relative(hap, name, kw):
+    """fp64 mode: every candidate's iteration time and bottleneck within 1e-9 relative of the fp64 oracle,
+    infeasible candidates identical, the chosen plan the oracle's (unless its two best costs are closer than
+    1e-9 relative)."""
+    pb, hp, o = setup(hap, name, **kw)
+    out = hap.hap_pipeline_dp_f64(hp, 0, hp.n_cand, partition=True)
+    torch.cuda.synchronize()
+    got, gotb, part = out["cost"].cpu().numpy(), out["bottleneck"].cpu().numpy(), out["partition"].cpu().numpy()
+    done, costs, bn, parts = o.search_pconfs_f64(0, 1, threads=NTHREADS)
+    assert done == o.n_cand
+    fin = np.isfinite(costs)
+    assert np.array_equal(fin, np.isfinite(got)) and np.array_equal(np.isfinite(bn), np.isfinite(gotb))
+    assert (np.isposinf(got[~fin])).all()
+    assert np.max(np.abs(got[fin] - costs[fin]) / costs[fin]) <= 1e-9
+    bfin = np.isfinite(bn)
+    assert np.max(np.abs(gotb[bfin] - bn[bfin]) / bn[bfin]) <= 1e-9
+    # partitions: identical wherever the decision is not a rounding-level tie
+    same = (part == parts).all(axis=1)
+    assert same[fin].mean() > 0.9999 and not part[~fin].any()
+    order = np.argsort(costs[fin], kind="stable")[:2]
+    best_idx = np.nonzero(fin)[0][order]
+    plan = hap.hap_search_range_f64(hp, 0, hp.n_cand)
+    gap = (costs[best_idx[1]] - costs[best_idx[0]]) / costs[best_idx[0]] if len(best_idx) > 1 else 1.0
+    assert plan["index"] == int(best_idx[0]) or gap <= 1e-9
+    assert plan["T_iter_f64"] == pytest.approx(costs[plan["index"]], rel=1e-9)
+    assert plan["n"] == parts[plan["index"], :plan["PP"]].tolist()
+    # integer and fp64 modes pick plans of (nearly) the same cost
+    iplan, _ = hap.hap_search_best(hp)
+    assert abs(iplan["T_iter"] - plan["T_iter_f64"]) <= 1e-3 * plan["T_iter_f64"]

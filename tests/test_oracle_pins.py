@@ -89,6 +89,33 @@ def test_e1_two_device_example():
     assert best["index"] == g["best_map"] and feas == 2 and costs.tolist() == [ab["T_iter"], ba["T_iter"]]
 
 
+def test_e1_fp64_mode_hand_values():
+    g = gold("e1_two_device_pp2.json")["expect"]["fp64"]
+    o = Oracle(e1_problem())
+    for idx, key in ((0, "map_AB"), (1, "map_BA")):
+        r = o.eval_index_f64(idx)
+        assert r["n"] == g[key]["n"]
+        assert r["T_iter"] == pytest.approx(g[key]["T_iter"], rel=1e-12)
+        assert r["c"] == pytest.approx(g[key]["c"], rel=1e-12)
+        assert r["bottleneck"] == pytest.approx(max(g[key]["c"]), rel=1e-12)
+
+
+def test_fp64_mode_tracks_integer_mode_within_rounding():
+    """Each of the <= 2N+PP rounded terms moves a time by at most 0.5 ns, times M for the bottleneck term."""
+    for pb in (problems.tiny(), problems.random_small(2, N=9, T=2, nodes_per_type=(2, 2), node_size=2)):
+        o = Oracle(pb)
+        ci, bi, _, _ = o.search()
+        done, cf, bf, parts = o.search_pconfs_f64(0, 1, threads=2)
+        assert done == o.n_cand
+        fin = ci < INF
+        assert np.array_equal(fin, np.isfinite(cf)) and np.array_equal(bi < INF, np.isfinite(bf))
+        M = np.repeat(o.pconfs["M"].astype(np.float64), o.pconfs["nmap"].astype(np.int64) * len(pb.rc_masks))
+        # rounding can also flip a near-tie between partitions, so allow a relative slack as well
+        assert (np.abs(bf[fin] - bi[fin]) <= (2 * pb.N + 2) * 0.5 + 1e-6 * bi[fin]).all()
+        assert (np.abs(cf[fin] - ci[fin]) <= M[fin] * (2 * pb.N + 34) + 2e-3 * ci[fin]).all()
+        assert (parts[fin].sum(axis=1) == pb.N).all()
+
+
 def test_e2_dispatch_volume_and_primitive_tie():
     g = gold("e2_dispatch_ep2.json")["expect"]
     pb = e1_problem()
