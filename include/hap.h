@@ -19,6 +19,10 @@
  *  - A hap_problem is not thread safe; use one per thread or serialise calls.
  *  - Times are nanoseconds, memory is bytes, both as int64 after round-to-nearest-even of
  *    the fp64 formula value ("integer mode").  HAP_INF marks an infeasible candidate.
+ *  - Value limits (so that every sum stays below 2^62): global batch x layers <= 2^22, a layer's
+ *    forward or backward time < 2^36 ns, a stage constant < 2^40 ns.  A violation found on the device is
+ *    reported as HAP_E_RANGE by the next call that synchronises (hap_search_*, hap_count_cells,
+ *    hap_get_timings); asynchronous calls cannot report it themselves.
  */
 #ifndef HAP_H
 #define HAP_H
@@ -124,6 +128,9 @@ typedef struct {
     const int32_t *tau_q;        /* [R] fraction of the forward pass re-executed, in 1/1024 */
 } hap_profile;
 
+/* hap_search_opts.flags */
+#define HAP_OPT_NO_MAPTAB 1   /* keep no table of decoded mappings on the device: the DP kernel unranks each mapping itself */
+
 typedef struct {
     int32_t npp, ntpe;
     const int32_t *pp_list, *tpe_list;  /* pipeline and expert-TP degrees to try (ascending) */
@@ -132,7 +139,8 @@ typedef struct {
     uint64_t map_cap;                    /* enumerate all distinct stage-type sequences only up to this count (<= 2^56) */
     int32_t n_rc;                        /* recomputation policies, 1..HAP_MAX_RC_MASKS */
     const uint32_t *rc_masks;            /* [n_rc] bit r set: level r allowed; per stage the lowest feasible allowed level is used */
-    int32_t prune;                       /* hap_search_best may skip candidates whose lower bound exceeds the incumbent */
+    int32_t prune;                       /* hap_search_* may skip candidates whose lower bound exceeds the incumbent */
+    int32_t flags;                       /* HAP_OPT_* bits */
 } hap_search_opts;
 
 /* One accepted parallel configuration x micro-batch size.  Candidate index of

@@ -51,7 +51,7 @@ class _Profile(C.Structure):
 class _Opts(C.Structure):
     _fields_ = [("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
                 ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64), ("n_rc", C.c_int32),
-                ("rc_masks", C.c_void_p), ("prune", C.c_int32)]
+                ("rc_masks", C.c_void_p), ("prune", C.c_int32), ("flags", C.c_int32)]
 
 
 class _Plan(C.Structure):
@@ -136,7 +136,10 @@ class HapProblem:
             pass
 
 
-def hap_problem_create(pb, prune: int = 0) -> HapProblem:
+OPT_NO_MAPTAB = 1
+
+
+def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     """Marshals a plain-data problem (see gen.problems.Problem) into the C descriptors."""
     L = load_library()
     keep = []
@@ -174,6 +177,7 @@ def hap_problem_create(pb, prune: int = 0) -> HapProblem:
     so.n_rc = len(pb.rc_masks)
     so.rc_masks = arr("rc_masks", np.uint32)
     so.prune = int(prune)
+    so.flags = int(flags)
     out = C.c_void_p(0)
     st = L.hap_problem_create(C.byref(mo), C.byref(cl), C.byref(pf), C.byref(so), C.byref(out))
     if st != 0:

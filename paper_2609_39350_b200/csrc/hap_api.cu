@@ -45,6 +45,7 @@ struct hap_problem {
     i64 *d_c2 = nullptr, *d_coef = nullptr;
     double *d_c2f = nullptr, *d_coeff = nullptr;   // fp64-mode layer costs and coefficients (allocated on first use)
     i64 *d_fcost = nullptr;                 // fp64-mode search: per-candidate costs (bit patterns), allocated on first use
+    u64 *d_range = nullptr;                 // sticky flag: a cost left the supported value range
     i64 *d_lb = nullptr;                    // scratch: per-configuration lower bound on the summed stage time
     TypeConst *d_tc = nullptr;              // scratch: per (configuration, type) constants of the layer-cost kernels
     i64 *d_pcost = nullptr;                // per-block partial minima
@@ -108,7 +109,7 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 static void release_device(hap_problem *p)
 {
     cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
-    cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
+    cudaFree(p->d_range); cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); }
@@ -151,6 +152,7 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     const int N = mo->N, T = cl->n_types;
     if (N < 1 || N > HAP_MAX_LAYERS || !mo->kind) return HAP_E_INVALID;
     if (T < 1 || T > HAP_MAX_TYPES || cl->n_nodes < 1) return HAP_E_INVALID;
+    if ((int64_t)mo->GB * mo->N > (1ll << 22)) return HAP_E_RANGE;     // keeps M * sum of layer times below 2^62
     if (mo->S < 1 || mo->H < 1 || mo->E < 1 || mo->k < 1 || mo->nq < 1 || mo->nkv < 1 || mo->GB < 1 || mo->V < 0 ||
         mo->n_shared < 0 || mo->F_dense < 0 || mo->F_exp < 0 || !(mo->beta > 0.0) || mo->nq % mo->nkv != 0)
         return HAP_E_INVALID;
@@ -387,7 +389,8 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 }
             }
             cl.item_hi = items.size();
-            cl.has_tab = nmap * (uint64_t)PP * 2 <= (64ull << 20) && tab_bytes + nmap * PP * 2 <= (256ull << 20);
+            cl.has_tab = !(p->opts.flags & HAP_OPT_NO_MAPTAB) && nmap * (uint64_t)PP * 2 <= (64ull << 20) &&
+                         tab_bytes + nmap * PP * 2 <= (256ull << 20);
             cl.map_base = tab_bytes;
             if (cl.has_tab) tab_bytes += (nmap * (uint64_t)PP * 2 + 255) / 256 * 256;
             classes.push_back(cl);
@@ -408,6 +411,8 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         CUDA_TRY(p, cudaMalloc(&p->d_coef, np * T * HAP_NCOEF * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_tc, np * T * sizeof(TypeConst)));
         CUDA_TRY(p, cudaMalloc(&p->d_lb, np * sizeof(i64)));
+        CUDA_TRY(p, cudaMalloc(&p->d_range, sizeof(u64)));
+        CUDA_TRY(p, cudaMemset(p->d_range, 0, sizeof(u64)));
         p->n_partial = std::max<size_t>(p->items.size(), 1024);
         CUDA_TRY(p, cudaMalloc(&p->d_pcost, p->n_partial * sizeof(i64)));
         CUDA_TRY(p, cudaMalloc(&p->d_pindex, p->n_partial * sizeof(u64)));
@@ -466,6 +471,14 @@ static hap_status enter(hap_problem *p)
     return HAP_OK;
 }
 
+static hap_status check_values(hap_problem *p)
+{
+    u64 flag = 0;
+    CUDA_TRY(p, cudaMemcpy(&flag, p->d_range, sizeof(flag), cudaMemcpyDeviceToHost));
+    if (flag) return fail(p, HAP_E_RANGE, "a layer time or stage coefficient exceeds the supported range (see hap.h)");
+    return HAP_OK;
+}
+
 static hap_status check_range(hap_problem *p, uint64_t first, uint64_t count)
 {
     if (first > p->n_cand || count > p->n_cand - first) return fail(p, HAP_E_RANGE, "candidate range outside [0, %llu)", (unsigned long long)p->n_cand);
@@ -491,14 +504,14 @@ static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double 
 {
     const u64 nph = (u64)p->pconfs.size() * HAP_MAX_TYPES;
     const unsigned b1 = (unsigned)((nph + kLcThreads - 1) / kLcThreads);
-    if (quant) type_const_kernel<true><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr);
-    else type_const_kernel<false><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff);
+    if (quant) type_const_kernel<true><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr, p->d_range);
+    else type_const_kernel<false><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff, p->d_range);
     CUDA_TRY(p, cudaGetLastError());
     if ((quant && c2) || (!quant && c2f)) {
         const unsigned b2 = (unsigned)p->pconfs.size();
         const unsigned thr = (unsigned)((p->model.N + 31) / 32 * 32);
-        if (quant) layer_cost_kernel<true><<<b2, thr, 0, st>>>(p->dc, p->d_tc, c2, nullptr, lb_sum);
-        else layer_cost_kernel<false><<<b2, thr, 0, st>>>(p->dc, p->d_tc, nullptr, c2f, nullptr);
+        if (quant) layer_cost_kernel<true><<<b2, thr, 0, st>>>(p->dc, p->d_tc, c2, nullptr, lb_sum, p->d_range);
+        else layer_cost_kernel<false><<<b2, thr, 0, st>>>(p->dc, p->d_tc, nullptr, c2f, nullptr, p->d_range);
     }
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
@@ -695,7 +708,7 @@ extern "C" hap_status hap_count_cells(hap_problem *p, uint64_t first, uint64_t c
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaMemcpyAsync(host_cells, p->d_counters + 4, sizeof(u64), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(p, cudaStreamSynchronize(st));
-    return HAP_OK;
+    return check_values(p);
 }
 
 extern "C" hap_status hap_get_timings(hap_problem *p, float *ms_layer_cost, float *ms_dp, uint64_t *cells)
@@ -707,7 +720,7 @@ extern "C" hap_status hap_get_timings(hap_problem *p, float *ms_layer_cost, floa
     if (ms_layer_cost) CUDA_TRY(p, cudaEventElapsedTime(ms_layer_cost, p->ev[0], p->ev[1]));
     if (ms_dp) CUDA_TRY(p, cudaEventElapsedTime(ms_dp, p->ev[1], p->ev[2]));
     if (cells) CUDA_TRY(p, cudaMemcpy(cells, p->d_counters + 4, sizeof(u64), cudaMemcpyDeviceToHost));
-    return HAP_OK;
+    return check_values(p);
 }
 
 static hap_status argmin_launch(hap_problem *p, const i64 *dev_cost, uint64_t count, i64 *dev_out, cudaStream_t st, i64 init)
@@ -766,6 +779,7 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
         cudaEventElapsedTime(&host_stats->ms_dp, p->ev[1], p->ev[2]);
         host_stats->ms_total = host_stats->ms_layer_cost + host_stats->ms_dp;
     }
+    if ((s = check_values(p)) != HAP_OK) return s;
     if (best[0] >= kInf) return fail(p, HAP_E_INFEASIBLE, "no candidate satisfies the memory constraint");
 
     // re-evaluate the winner alone to obtain its partition and recomputation levels

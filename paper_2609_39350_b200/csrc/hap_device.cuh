@@ -172,7 +172,7 @@ __device__ __forceinline__ double div_by(double a, double b, double y)
 // per (configuration, type, layer) unit, consecutive threads writing consecutive 16-byte results.
 template <bool QUANT>
 __global__ void __launch_bounds__(kLcThreads)
-type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff)
+type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u64 *range_flag)
 {
     const int T = dc.T;
     const i64 H = dc.H;
@@ -263,11 +263,16 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff)
                 }
                 v[HAP_SLAT] = dc.ovl_dp * (dc.alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
                 const size_t at = ((size_t)p * T + h) * HAP_NCOEF;
+                bool bad = false;
 #pragma unroll
                 for (int q = 0; q < HAP_NCOEF; ++q) {
                     if (QUANT) coef[at + q] = __double2ll_rn(v[q]);
                     else coeff[at + q] = v[q];
+                    // time coefficients must stay below 2^40 ns (per-layer ones below 2^36), bytes below 2^50
+                    const double lim = q <= HAP_SLAT ? 1.0995e12 : (q < HAP_MW ? 6.8719e10 : 1.1259e15);
+                    bad |= !(v[q] < lim);
                 }
+                if (bad && range_flag) atomicOr(range_flag, 1ull);
             }
         }
     }
@@ -278,7 +283,7 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff)
 template <bool QUANT>
 __global__ void __launch_bounds__(256)
 layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__restrict__ c2, double *__restrict__ c2f,
-                  i64 *__restrict__ lb_sum)
+                  i64 *__restrict__ lb_sum, u64 *range_flag)
 {
     __shared__ TypeConst tcs[HAP_MAX_TYPES];
     __shared__ i64 s_lb[8];
@@ -322,6 +327,7 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
                 cb = (((ab[h] - fb[h]) + mb) + tc.tr2) + tc.commB[HAP_MOE];
             }
             store_pair<QUANT>(c2, c2f, (((size_t)p * T + h) * N + l) * 2, cf, cb);
+            if (!(cf < 6.8719e10 && cb < 6.8719e10) && range_flag) atomicOr(range_flag, 1ull);   // 2^36 ns per layer
             if (QUANT) {
                 const i64 q = __double2ll_rn(cf) + __double2ll_rn(cb);
                 lmin = (h == 0 || q < lmin) ? q : lmin;
@@ -587,19 +593,24 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
     if (SEARCH && out.prune) {
         // T_iter >= sum_i c_i + (M-1) max_i c_i >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on
         // the summed stage time.  Skipping needs bound > incumbent (strict): the result cannot change.
-        const i64 S = out.lb_sum[it.p];
-        const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
-        const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
-        if ((u64)lb > inc) {
-            if (threadIdx.x == 0) {
+        // The incumbent moves while the block runs, so ONE thread reads it and the whole block follows that
+        // reading: a block must leave as a whole.
+        __shared__ int s_skip;
+        if (threadIdx.x == 0) {
+            const i64 S = out.lb_sum[it.p];
+            const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
+            const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+            s_skip = (u64)lb > inc;
+            if (s_skip) {
                 out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
                 // candidates of this block inside the requested range
                 const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
                 const u64 a = c0 > out.first ? c0 : out.first, b = c1 < out.first + out.count ? c1 : out.first + out.count;
                 atomicAdd(out.counters + 2, b - a);
             }
-            return;
         }
+        __syncthreads();
+        if (s_skip) return;
     }
     const bool multiset = pc.mode == HAP_MAP_MULTISET;
     const int nmask = (1 << T) - 1;

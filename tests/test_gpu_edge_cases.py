@@ -1,0 +1,134 @@
+"""Edge cases of the CUDA path against the oracle: maximum sizes, degenerate sizes, one device type,
+many recomputation levels and policies, in-kernel unranking instead of the mapping table, value limits."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from gen import problems  # noqa: E402
+from gen.problems import DENSE, MOE  # noqa: E402
+from oracle import Oracle, INF  # noqa: E402
+
+
+@pytest.fixture(scope="module")
+def hap():
+    import paper_2609_39350_b200 as hap
+    from paper_2609_39350_b200.build import build_library
+    build_library()
+    assert torch.cuda.is_available()
+    return hap
+
+
+def full_compare(hap, pb, tables_every=0, flags=0):
+    hp = hap.hap_problem_create(pb, flags=flags)
+    hap.hap_enumerate(hp)
+    o = Oracle(pb)
+    assert (hp.n_pconf, hp.n_cand) == (o.n_pconf, o.n_cand)
+    done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=8, want_costs=True)
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand, partition=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["cost"].cpu().numpy(), costs)
+    assert np.array_equal(out["bottleneck"].cpu().numpy(), bn)
+    part, rec = out["partition"].cpu().numpy(), out["recompute"].cpu().numpy()
+    step = max(1, o.n_cand // 300)
+    for idx in range(0, o.n_cand, step):
+        plan, _, _ = o.eval_index(idx)
+        if plan["T_iter"] < INF:
+            assert part[idx, :plan["PP"]].tolist() == plan["n"] and rec[idx, :plan["PP"]].tolist() == plan["r"], idx
+    if tables_every:
+        for idx in range(0, o.n_cand, tables_every):
+            t = hap.hap_pipeline_dp(hp, idx, 1, tables=True)
+            torch.cuda.synchronize()
+            plan, edp, ech = o.eval_index(idx, tables=True)
+            assert np.array_equal(t["dp_table"].cpu().numpy()[0, :plan["PP"] + 1], edp), idx
+            assert np.array_equal(t["choice"].cpu().numpy()[0, :plan["PP"] + 1], ech), idx
+    if (costs < INF).any():
+        plan, stats = hap.hap_search_best(hp)
+        assert (plan["T_iter"], plan["index"]) == (bc, bi)
+    hap.hap_problem_destroy(hp)
+    return o, costs
+
+
+def _model_problem(N, pp_list, nodes_per_type, node_size, P_tf, **kw):
+    T = len(P_tf)
+    kind = kw.pop("kind", [MOE] * N)
+    pb = problems._build("edge", kw.pop("seed", 11), N=N, S=2048, H=1024, E=8, k=2, n_shared=0, F_dense=4096,
+                         F_exp=2048, nq=8, nkv=8, V=32000, GB=kw.pop("GB", 64), kind=kind, P_tf=P_tf,
+                         C_gb=kw.pop("C_gb", [80, 64, 48, 40][:T]), node_size=[node_size] * T,
+                         bw_intra=[900.0, 600.0, 400.0, 300.0][:T], node_type=problems._nodes(list(nodes_per_type)),
+                         bw_inter_fixed=50.0, bw_inter_random=False, zipf_alpha=1.2, mb_list=kw.pop("mb_list", [1]),
+                         rc_masks=kw.pop("rc_masks", [0b11]), delta_q=kw.pop("delta_q", 205),
+                         map_cap=kw.pop("map_cap", 2048))
+    pb.pp_list = np.ascontiguousarray(np.array(pp_list, np.int32))
+    for k, v in kw.items():
+        setattr(pb, k, v)
+    return pb
+
+
+def test_maximum_layers_and_stages(hap):
+    """N = 255 layers, PP up to 32, four device types; multiset and block-mode classes."""
+    pb = _model_problem(255, [1, 2, 4, 8, 16, 32], (1, 1, 1, 1), 8, [400, 300, 250, 150], map_cap=4096,
+                        kind=[DENSE] * 3 + [MOE] * 252)
+    pb.tp_list = pb.tp_list[:1]; pb.tpe_list = pb.tpe_list[:1]; pb.cp_list = pb.cp_list[:1]; pb.ep_list = pb.ep_list[:2]
+    for f in ("tdf", "tdb", "tff", "tfb"):
+        setattr(pb, f, np.ascontiguousarray(getattr(pb, f)[:, :1, :1]))
+    pb.tpre = np.ascontiguousarray(pb.tpre[:, :1, :1]); pb.tpost = np.ascontiguousarray(pb.tpost[:, :1, :1])
+    pb.rho = pb.rho[:2].copy()
+    pb.cap_eff[:] = pb.cap_eff // 4            # make recomputation and infeasibility occur
+    o, costs = full_compare(hap, pb, tables_every=997)
+    assert set(o.pconfs["PP"].tolist()) == {1, 2, 4, 8, 16, 32} and 0 < (costs < INF).sum() < o.n_cand
+    pb.delta_q = -1                             # the same without the window: full-width bands, longer spans
+    pb.pp_list = np.ascontiguousarray(np.array([1, 4, 32], np.int32))
+    full_compare(hap, pb, tables_every=71)
+
+
+@pytest.mark.parametrize("N,pp", [(1, [1]), (2, [1, 2]), (8, [8]), (5, [1, 4])])
+def test_degenerate_layer_counts(hap, N, pp):
+    """One layer; as many stages as layers (every stage holds exactly one layer)."""
+    W = max(pp)
+    pb = _model_problem(N, pp, (W // 2 or 1, W - (W // 2 or 1)) if W > 1 else (1,), 1,
+                        [400, 200] if W > 1 else [400], delta_q=-1, GB=8)
+    full_compare(hap, pb, tables_every=1)
+
+
+def test_single_device_type_and_window(hap):
+    pb = _model_problem(24, [1, 2, 4, 8], (2,), 4, [300], rc_masks=[0b01, 0b11], mb_list=[1, 2])
+    o, costs = full_compare(hap, pb, tables_every=13)
+    assert set(o.pconfs["nmap"].tolist()) == {1}       # one type: exactly one mapping per configuration
+
+
+def test_four_recompute_levels_eight_policies(hap):
+    pb = _model_problem(20, [2, 4], (2, 1, 1), 4, [400, 300, 200], C_gb=[12, 9, 6], delta_q=-1, mb_list=[1, 4])
+    pb.xi_q = np.ascontiguousarray(np.array([1024, 700, 300, 40], np.int32))
+    pb.tau_q = np.ascontiguousarray(np.array([0, 256, 640, 1024], np.int32))
+    pb.rc_masks = np.ascontiguousarray(np.array([1, 2, 4, 8, 3, 5, 10, 15], np.uint32))
+    pb.cap_eff[:] = pb.cap_eff // 3
+    o, costs = full_compare(hap, pb, tables_every=101)
+    levels = set()
+    for idx in range(0, o.n_cand, 11):
+        if costs[idx] < INF:
+            levels |= set(o.eval_index(idx)[0]["r"])
+    assert levels == {0, 1, 2, 3}
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_in_kernel_unranking_without_the_mapping_table(hap, name):
+    full_compare(hap, problems.make_problem(name), flags=hap.OPT_NO_MAPTAB)
+
+
+def test_value_limits_are_reported(hap):
+    pb = problems.tiny()
+    big = pb.copy()
+    for f in ("tdf", "tdb"):
+        getattr(big, f)[:] = getattr(big, f) * 1.0e5 + 1.0e11       # layers of > 2^36 ns
+    hp = hap.hap_problem_create(big)
+    hap.hap_enumerate(hp)
+    with pytest.raises(hap.HapError) as e:
+        hap.hap_search_best(hp)
+    assert e.value.name == "HAP_E_RANGE"
+    hap.hap_problem_destroy(hp)
+    huge_batch = pb.copy(GB=1 << 19)                                # 2^19 sequences x 16 layers > 2^22
+    with pytest.raises(hap.HapError) as e:
+        hap.hap_problem_create(huge_batch)
+    assert e.value.name == "HAP_E_RANGE"
