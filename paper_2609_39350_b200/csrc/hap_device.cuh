@@ -773,6 +773,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
       const u32 m_lo = (u32)my_slice * per_slice;
       const u32 m_hi = m_lo + per_slice < it.count ? m_lo + per_slice : it.count;
       int valid_rows = 0;                  // DP rows of stages 1..valid_rows of the previous mapping are intact
+      int dead_stage = 1 << 30;            // first of those stages whose row holds no finite value (none: large)
       int prev_mask = -1, prev_link = -1;
       uchar2 next_ml = make_uchar2(0, 0);
       if (maptab && m_lo < m_hi && lane < PP)
@@ -791,7 +792,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             const StageMap smap = decode_stage(dc, pc, map_idx, lane);
             mask = smap.mask; link = lane > 0 && lane < PP ? (smap.cls | (smap.ha << 2) | (smap.hb << 4)) : 0;
         }
-        if (c < out.first || c >= out.first + out.count) { valid_rows = 0; prev_mask = -1; continue; }
+        if (c < out.first || c >= out.first + out.count) { valid_rows = 0; dead_stage = 1 << 30; prev_mask = -1; continue; }
         const unsigned differ = __ballot_sync(0xffffffffu, lane < PP && (mask != prev_mask || link != prev_link));
         int s0 = differ ? __ffs(differ) - 1 : PP;      // stages 1..s0 are shared with the previous mapping
         prev_mask = mask; prev_link = link;
@@ -828,6 +829,9 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         if (!multiset) s0 = 0;               // block mode: window and bands depend on the whole mapping
         if (s0 > valid_rows) s0 = valid_rows;
         if (want_tables) s0 = 0;
+        if (dead_stage > s0) dead_stage = 1 << 30;       // the dead row, if any, is not part of the shared prefix
+        // a shared stage prefix that already admits no feasible partition settles this mapping too
+        const bool dead_prefix = dead_stage <= s0;
 
         // ---- bands: end layers j that stage i can reach (prefix sums of the window bounds), and from
         //      which the remaining stages can still reach N (suffix sums; not applied when the caller
@@ -850,6 +854,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         }
         const bool dead = __any_sync(0xffffffffu, lane < PP && sp.bl > sp.bh);
         if (COUNT) {
+            dead_stage = 1 << 30;
             // cells (i, j, k) of this candidate's recurrence whose stage cost is finite: k inside the load-balance
             // window of stage i and the span (k, j] within the memory limit at some allowed level
             for (int i = 1; i <= PP; ++i) {
@@ -882,8 +887,11 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             }
         }
         VT bott = vInf;
-        if (!dead || want_tables) {
+        if (dead_prefix) {
+            valid_rows = s0;                                // rows up to the dead one stay as they are
+        } else if (!dead || want_tables) {
             int pbl = 0, pbh = 0;                          // band of the previous stage (stage 0: {0})
+            int last_stage = PP;
             if (s0 > 0) { pbl = __shfl_sync(0xffffffffu, sp.bl, s0 - 1); pbh = __shfl_sync(0xffffffffu, sp.bh, s0 - 1); }
             for (int i = s0 + 1; i <= PP; ++i) {
                 const int src = i - 1;
@@ -897,6 +905,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                 VT *cur = rows + ri * n1;
                 uint8_t *chrow = chw + (size_t)(i - 1) * n1;
                 const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
+                bool row_alive = false;
                 for (int j = bl + lane; j <= bh; j += 32) {
                     VT best = vInf;
                     int arg = 255;
@@ -935,8 +944,16 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                     }
                     cur[j] = best;
                     chrow[j] = (uint8_t)arg;
+                    row_alive |= best < vInf;
                 }
                 __syncwarp();
+                if (!want_tables && !__any_sync(0xffffffffu, row_alive)) {
+                    // no end layer of this stage is reachable within the memory limit: the candidate and every
+                    // mapping that shares stages 1..i with it are infeasible
+                    dead_stage = i;
+                    last_stage = i;
+                    break;
+                }
                 if (want_tables) {
                     for (int j = lane; j <= N; j += 32) {
                         const bool in = j >= bl && j <= bh;
@@ -946,10 +963,10 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                 }
                 pbl = bl; pbh = bh;
             }
-            valid_rows = dead ? 0 : PP;
+            valid_rows = dead ? 0 : last_stage;
             // N lies in the last band unless the windows cannot add up to N (possible only without the
             // suffix restriction, i.e. when tables are written)
-            if (!dead && pbl <= N && N <= pbh) bott = rows[(size_t)(multiset ? PP - 1 : (PP - 1) & 1) * n1 + N];
+            if (!dead && dead_stage > PP && pbl <= N && N <= pbh) bott = rows[(size_t)(multiset ? PP - 1 : (PP - 1) & 1) * n1 + N];
         } else {
             valid_rows = 0;
         }
