@@ -724,18 +724,37 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
     // Feasibility of a span (k, j] is monotone: a shorter span needs no more memory, and the first
     // feasible k does not decrease with j.  One thread sweeps j for one (stage, capacity type, level).
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
-    for (int q = threadIdx.x; q < PP * T * R; q += nwarps * 32) {
-        const int r = q % R, t = (q / R) % T, i = q / (R * T) + 1;
-        const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
-        const int inflight = PP - i + 1;
-        const i64 mstore = pc.M < inflight ? pc.M : inflight;
-        const i64 cap = dc.cap_eff[t], xi = dc.xi_q[r];
-        uint8_t *row = thr + (size_t)q * n1;
-        int k = 0;
-        row[0] = 0;
-        for (int j = 1; j <= N; ++j) {
-            while (k < j && !span_fits(sW, sA, sK, extra, mx, mstore, cap, xi, k, j)) ++k;
-            row[j] = (uint8_t)k;
+    const int combos = PP * T * R, nthreads = nwarps * 32;
+    if (combos * 7 < nthreads * 2) {
+        // few (stage, type, level) rows for this many threads: one thread per table entry, binary search over k
+        for (int e = threadIdx.x; e < combos * n1; e += nthreads) {
+            const int q = e / n1, j = e - q * n1;
+            const int r = q % R, t = (q / R) % T, i = q / (R * T) + 1;
+            const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
+            const int inflight = PP - i + 1;
+            const i64 mstore = pc.M < inflight ? pc.M : inflight;
+            const i64 cap = dc.cap_eff[t], xi = dc.xi_q[r];
+            int lo = 0, hi = j;                       // first k in [0, j] whose span (k, j] fits; j if none
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (span_fits(sW, sA, sK, extra, mx, mstore, cap, xi, mid, j)) hi = mid; else lo = mid + 1;
+            }
+            thr[(size_t)q * n1 + j] = (uint8_t)lo;
+        }
+    } else {
+        for (int q = threadIdx.x; q < combos; q += nthreads) {
+            const int r = q % R, t = (q / R) % T, i = q / (R * T) + 1;
+            const i64 extra = (i == 1 ? mpre : 0) + (i == PP ? mpost : 0);
+            const int inflight = PP - i + 1;
+            const i64 mstore = pc.M < inflight ? pc.M : inflight;
+            const i64 cap = dc.cap_eff[t], xi = dc.xi_q[r];
+            uint8_t *row = thr + (size_t)q * n1;
+            int k = 0;
+            row[0] = 0;
+            for (int j = 1; j <= N; ++j) {
+                while (k < j && !span_fits(sW, sA, sK, extra, mx, mstore, cap, xi, k, j)) ++k;
+                row[j] = (uint8_t)k;
+            }
         }
     }
     // load-balance window per device type when every mapping uses the same multiset of stage types
