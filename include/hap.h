@@ -130,6 +130,10 @@ typedef struct {
 
 /* hap_search_opts.flags */
 #define HAP_OPT_NO_MAPTAB 1   /* keep no table of decoded mappings on the device: the DP kernel unranks each mapping itself */
+#define HAP_OPT_REFINE 2      /* after the min-max recurrence, choose among the bottleneck-optimal partitions the one with
+                                 the smallest sum of stage costs (Eq. 4's T_edge), smallest split on ties; integer mode only.
+                                 Costs, partitions, levels and the plan then refer to that partition; the DP tables
+                                 returned by hap_pipeline_dp remain those of the min-max recurrence. */
 
 typedef struct {
     int32_t npp, ntpe;

@@ -576,6 +576,103 @@ int orc_candidate(const orc_problem *pr, const orc_pconf *pc, const orc_mapping 
     return 0;
 }
 
+/* ------------------------------------------------------------------------------------ *
+ * Refinement (lexicographic optimum): among the partitions whose largest stage cost equals the
+ * bottleneck B* of the min-max recurrence, take the one with the smallest SUM of stage costs
+ * (Eq. 4's T_edge term), smallest split on ties.  This removes the dependence of the iteration
+ * time on which of the bottleneck-optimal partitions the min-max tie-break happened to pick.
+ * ------------------------------------------------------------------------------------ */
+int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                          const int64_t *c2, const int64_t *coef, orc_result *res)
+{
+    const int N = pr->N, PP = pc->PP;
+    orc_result first;
+    int rc0 = orc_candidate(pr, pc, mp, rc_mask, c2, coef, &first, NULL, NULL);
+    if (rc0 != 0) { *res = first; return rc0; }          /* infeasible (or error): nothing to refine */
+    const int64_t Bstar = first.bottleneck;
+    stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+    int64_t *D = (int64_t *)malloc(sizeof(int64_t) * (size_t)(PP + 1) * (N + 1));
+    uint8_t *CH = (uint8_t *)malloc((size_t)(PP + 1) * (N + 1));
+    if (!D || !CH || !cx) { free(D); free(CH); free(cx); return -1; }
+    ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+#define DAT(i, j) D[(size_t)(i) * (N + 1) + (j)]
+#define CHAT(i, j) CH[(size_t)(i) * (N + 1) + (j)]
+    for (int i = 0; i <= PP; ++i)
+        for (int j = 0; j <= N; ++j) { DAT(i, j) = ORC_INF; CHAT(i, j) = 255; }
+    DAT(0, 0) = 0;
+    for (int i = 1; i <= PP; ++i)
+        for (int j = i; j <= N - PP + i; ++j)
+            for (int k = i - 1; k <= j - 1; ++k) {
+                if (DAT(i - 1, k) >= ORC_INF) continue;
+                int64_t c = ctx_stage_cost(cx, i, k, j, NULL);
+                if (c > Bstar) continue;                         /* keep the bottleneck optimal */
+                int64_t v = DAT(i - 1, k) + c;
+                if (v < DAT(i, j)) { DAT(i, j) = v; CHAT(i, j) = (uint8_t)k; }   /* strict: smallest k wins */
+            }
+    memset(res, 0, sizeof(*res));
+    res->bottleneck = Bstar;
+    int64_t sum = 0, mx = 0, tsync = 0, topt = 0;
+    int j = N;
+    for (int i = PP; i >= 1; --i) {
+        int k = CHAT(i, j), r;
+        int64_t c = ctx_stage_cost(cx, i, k, j, &r);
+        res->n[i - 1] = (uint8_t)(j - k);
+        res->r[i - 1] = (uint8_t)r;
+        res->c[i - 1] = c;
+        sum += c;
+        if (c > mx) mx = c;
+        unsigned mask = mp->mask[i - 1];
+        int64_t sy = mask_max(pr, mask, coef, ORC_SLAT), op = 0;
+        for (int l = k; l < j; ++l) {
+            sy += mask_max(pr, mask, coef, ORC_SBW + pr->kind[l]);
+            op += mask_max(pr, mask, coef, ORC_OPT + pr->kind[l]);
+        }
+        if (sy > tsync) tsync = sy;
+        if (op > topt) topt = op;
+        j = k;
+    }
+    res->T_pipe = sum + (int64_t)(pc->M - 1) * mx;
+    res->T_sync = tsync;
+    res->T_opt = topt;
+    res->T_iter = res->T_pipe + tsync + topt;
+    free(D); free(CH); free(cx);
+#undef DAT
+#undef CHAT
+    return 0;
+}
+
+/* Exhaustive check of the refinement: smallest sum of stage costs over every contiguous partition of
+ * layers 1..j into stages 1..i whose stages all cost at most `limit` (no recurrence, no memo). */
+static void bf_sum_rec(const stage_ctx *cx, int stage, int nstages, int start, int end, int64_t limit,
+                       int64_t cur_sum, int64_t *best)
+{
+    if (stage == nstages) {
+        int64_t c = ctx_stage_cost(cx, stage, start, end, NULL);
+        if (c <= limit && c < ORC_INF && cur_sum + c < *best) *best = cur_sum + c;
+        return;
+    }
+    for (int cut = start + 1; cut <= end - (nstages - stage); ++cut) {
+        int64_t c = ctx_stage_cost(cx, stage, start, cut, NULL);
+        if (c > limit || c >= ORC_INF) continue;
+        bf_sum_rec(cx, stage + 1, nstages, cut, end, limit, cur_sum + c, best);
+    }
+}
+
+int64_t orc_bruteforce_sum(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                           const int64_t *c2, const int64_t *coef, int i, int j, int64_t limit)
+{
+    int64_t best = ORC_INF;
+    if (i == 0) return j == 0 ? 0 : ORC_INF;
+    if (j >= i) {
+        stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+        if (!cx) return -1;
+        ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+        bf_sum_rec(cx, 1, i, 0, j, limit, 0, &best);
+        free(cx);
+    }
+    return best;
+}
+
 /* Exhaustive minimum over every contiguous partition of layers 1..j into stages 1..i of the
  * largest stage cost (no recurrence, no memo): the plain definition of the bottleneck. */
 static void bf_rec(const stage_ctx *cx, int stage, int nstages, int start, int end,
@@ -689,6 +786,9 @@ int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, ui
 /* Timing harness: evaluates every candidate of configurations p_first, p_first+stride, ...
  * (threads > 1 spreads configurations over OpenMP threads; the per-candidate work is the
  * plain code above).  Returns the (cost, index) minimum over what it evaluated. */
+static int g_refine = 0;    /* evaluation mode of the whole-space harnesses below: 0 plain, 1 refined */
+void orc_set_refine(int on) { g_refine = on; }
+
 int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
                       uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
                       int64_t *costs, int64_t *bottlenecks)
@@ -711,7 +811,8 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
             orc_decode(pr, pc, map_idx, &mp);
             for (int rc = 0; rc < pr->n_rc; ++rc) {
                 orc_result res;
-                orc_candidate(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL, NULL);
+                if (g_refine) orc_candidate_refined(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res);
+                else orc_candidate(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL, NULL);
                 uint64_t idx = pc->offset + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
                 if (costs) costs[idx] = res.T_iter;              /* indexed by candidate, whole space */
                 if (bottlenecks) bottlenecks[idx] = res.bottleneck;

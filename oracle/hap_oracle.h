@@ -125,6 +125,13 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
                       uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
                       int64_t *costs, int64_t *bottlenecks);
 
+/* refinement: smallest sum of stage costs among the bottleneck-optimal partitions */
+int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                          const int64_t *c2, const int64_t *coef, orc_result *res);
+int64_t orc_bruteforce_sum(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                           const int64_t *c2, const int64_t *coef, int i, int j, int64_t limit);
+void orc_set_refine(int on);
+
 /* fp64 mode (no rounding of times to integer ns); see hap_oracle.c */
 typedef struct {
     double T_iter, bottleneck, T_pipe, T_sync, T_opt;

@@ -97,6 +97,7 @@ def lib():
         L.orc_rank_multiset.restype = C.c_uint64
         L.orc_stage_cost.restype = C.c_int64
         L.orc_bruteforce.restype = C.c_int64
+        L.orc_bruteforce_sum.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -266,6 +267,36 @@ class Oracle:
         if want_costs:
             return int(done.value), int(bc.value), int(bi.value), costs, bn
         return int(done.value), int(bc.value), int(bi.value)
+
+    # ---- refinement --------------------------------------------------------------------
+    def candidate_refined(self, p, mp, rc_mask, c2, coef) -> Result:
+        res = Result()
+        self.L.orc_candidate_refined(C.byref(self.s), self._pc(p), C.byref(mp), C.c_uint32(rc_mask), _ptr(c2), _ptr(coef),
+                                     C.byref(res))
+        return res
+
+    def eval_index_refined(self, index: int) -> dict:
+        p = self.find_pconf(index)
+        n_rc = len(self.pb.rc_masks)
+        local = index - int(self.pconfs["offset"][p])
+        mp = self.decode(p, local // n_rc)
+        c2, _, coef, _ = self.layer_costs(p)
+        res = self.candidate_refined(p, mp, int(self.pb.rc_masks[local % n_rc]), c2, coef)
+        PP = int(self.pconfs["PP"][p])
+        return dict(T_iter=int(res.T_iter), bottleneck=int(res.bottleneck), T_pipe=int(res.T_pipe), T_sync=int(res.T_sync),
+                    T_opt=int(res.T_opt), n=[int(x) for x in res.n[:PP]], r=[int(x) for x in res.r[:PP]],
+                    c=[int(x) for x in res.c[:PP]], PP=PP, M=int(self.pconfs["M"][p]))
+
+    def bruteforce_sum(self, p, mp, rc_mask, c2, coef, i, j, limit) -> int:
+        return int(self.L.orc_bruteforce_sum(C.byref(self.s), self._pc(p), C.byref(mp), C.c_uint32(rc_mask), _ptr(c2),
+                                             _ptr(coef), C.c_int(i), C.c_int(j), C.c_int64(limit)))
+
+    def search_pconfs_refined(self, p_first: int = 0, p_stride: int = 1, threads: int = 1, want_costs: bool = True):
+        self.L.orc_set_refine(C.c_int(1))
+        try:
+            return self.search_pconfs(p_first, p_stride, threads, want_costs)
+        finally:
+            self.L.orc_set_refine(C.c_int(0))
 
     # ---- fp64 mode ---------------------------------------------------------------------
     def candidate_f64(self, p, mp, rc_mask, c2f, coef, coeff) -> ResultF:

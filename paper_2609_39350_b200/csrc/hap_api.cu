@@ -369,7 +369,8 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             const uint64_t per_pconf = class_nmap * (uint64_t)p->opts.n_rc;     // candidates a block can have at most
             for (int w : {12, 8, 6, 4, 2, 1}) {
                 if ((uint64_t)w * 8 > per_pconf && w > 2) continue;             // keep about 8 candidates per warp
-                const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0);
+                const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0,
+                                                (p->opts.flags & HAP_OPT_REFINE) != 0);
                 if (sm > 227 * 1024) continue;
                 const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), std::min(32, 64 / w));
                 const int resident = std::min(per_sm * w, 24);           // registers allow about 24 warps per SM
@@ -538,7 +539,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
 {
     // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
     // process: raise it (never lower it) before a launch that needs more
-    static size_t smem_limit[64][8];
+    static size_t smem_limit[64][12];
     const int dev = p->device & 63;
     // fork: every PP class runs on its own stream so that the tail of one class overlaps the next
     CUDA_TRY(p, cudaEventRecord(p->ev_fork, st));
@@ -556,13 +557,15 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const bool outside = c1 <= out.first || c0 >= out.first + out.count;
         if (outside && !search) continue;
         const bool lin = p->dc.tau_linear != 0;
-        const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (search ? 2 : 0) + (lin ? 1 : 0);
-        const void *fn = f64 ? (lin ? (const void *)pipeline_dp_kernel<false, true, false, double> : (const void *)pipeline_dp_kernel<false, false, false, double>)
-                         : out.count_only ? (lin ? (const void *)pipeline_dp_kernel<false, true, true> : (const void *)pipeline_dp_kernel<false, false, true>)
-                         : variant == 0 ? (const void *)pipeline_dp_kernel<false, false>
-                         : variant == 1 ? (const void *)pipeline_dp_kernel<false, true>
-                         : variant == 2 ? (const void *)pipeline_dp_kernel<true, false>
-                                        : (const void *)pipeline_dp_kernel<true, true>;
+        const bool refine = (p->opts.flags & HAP_OPT_REFINE) != 0 && !out.count_only;
+        const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (refine ? 8 : 0) + (search ? 2 : 0) + (lin ? 1 : 0);
+        const void *fn;
+        if (f64) fn = lin ? (const void *)pipeline_dp_kernel<false, true, false, double> : (const void *)pipeline_dp_kernel<false, false, false, double>;
+        else if (out.count_only) fn = lin ? (const void *)pipeline_dp_kernel<false, true, true> : (const void *)pipeline_dp_kernel<false, false, true>;
+        else if (refine) fn = search ? (lin ? (const void *)pipeline_dp_kernel<true, true, false, i64, true> : (const void *)pipeline_dp_kernel<true, false, false, i64, true>)
+                                     : (lin ? (const void *)pipeline_dp_kernel<false, true, false, i64, true> : (const void *)pipeline_dp_kernel<false, false, false, i64, true>);
+        else fn = search ? (lin ? (const void *)pipeline_dp_kernel<true, true> : (const void *)pipeline_dp_kernel<true, false>)
+                         : (lin ? (const void *)pipeline_dp_kernel<false, true> : (const void *)pipeline_dp_kernel<false, false>);
         if (cl.smem > smem_limit[dev][variant]) {
             CUDA_TRY(p, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cl.smem));
             smem_limit[dev][variant] = cl.smem;
@@ -625,6 +628,7 @@ extern "C" hap_status hap_pipeline_dp_f64(hap_problem *p, uint64_t first, uint64
     if (s != HAP_OK) return s;
     if ((s = check_range(p, first, count)) != HAP_OK) return s;
     if (count == 0) return HAP_OK;
+    if (p->opts.flags & HAP_OPT_REFINE) return fail(p, HAP_E_INVALID, "the refinement pass exists in integer mode only");
     if ((s = ensure_f64_buffers(p)) != HAP_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));

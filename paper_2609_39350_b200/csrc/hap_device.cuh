@@ -520,7 +520,8 @@ __global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *t
 //   sK   [N+1]                 u8: number of MoE layers among the first l layers
 //   per warp: rows [PP][N+1] i64 (one DP row per stage, kept so that the next mapping can reuse the rows
 //             of the stage prefix it shares), ch [PP][N+1] u8 split choices
-__host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int warps, bool multiset, bool linear)
+__host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int warps, bool multiset, bool linear,
+                                                bool refine = false)
 {
     const size_t n1 = (size_t)N + 1;
     const size_t mrows = multiset ? (size_t)T : (size_t)((1 << T) - 1);
@@ -529,6 +530,7 @@ __host__ __device__ inline size_t dp_smem_bytes(int N, int PP, int T, int R, int
     b += (n1 + 15) / 16 * 16;
     const size_t nrows = multiset ? (size_t)PP : (size_t)(PP < 2 ? PP : 2);   // rows are reused only across multiset mappings
     b += (size_t)warps * ((nrows * n1 * 8) + (((size_t)PP * n1 + 15) / 16 * 16));
+    if (refine) b += (size_t)warps * 2 * n1 * 8;             // two rotating rows of the second (additive) pass
     return b + 32;
 }
 
@@ -569,7 +571,7 @@ struct MaskInfo {
     int capt, pad;
 };
 
-template <bool SEARCH, bool LINEAR, bool COUNT = false, typename VT = i64>
+template <bool SEARCH, bool LINEAR, bool COUNT = false, typename VT = i64, bool REFINE = false>
 __global__ void __launch_bounds__(kDpWarps * 32)
 pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const i64 *coef, const VT *coefv,
                    const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
@@ -628,6 +630,8 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
     unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
     VT *rows = reinterpret_cast<VT *>(wbase);            // row of stage i at rows + ((i-1) % nrows)*n1
     uint8_t *chw = wbase + row_bytes;
+    // second-pass rows (refinement) sit behind all warps' first-pass storage
+    VT *rows2 = reinterpret_cast<VT *>(sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)nwarps * (row_bytes + ch_bytes)) + (size_t)wib * 2 * n1;
     __shared__ MaskInfo<VT> minfo[kMaxMasks];
     __shared__ VT sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
     __shared__ VT szero[1];                               // the row of "stage 0": DP[0][0] = 0
@@ -990,6 +994,50 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             valid_rows = 0;
         }
         __syncwarp();
+
+        if (REFINE && bott < vInf) {
+            // ---- refinement: among the partitions whose stages all cost at most the bottleneck just found, the one
+            //      with the smallest sum of stage costs (additive recurrence, same bands, same tie-break).  Its split
+            //      choices replace those of the first pass; the first pass's rows stay intact for the next mapping.
+            int pbl = 0, pbh = 0;
+            for (int i = 1; i <= PP; ++i) {
+                const int src = i - 1;
+                const int mrow = __shfl_sync(0xffffffffu, sp.mrow, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
+                const VT K = shfl_v(sp.K, src);
+                const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
+                const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
+                const VT *rM = sR + (size_t)mrow * RW * n1;
+                const VT *prev = i == 1 ? szero : rows2 + (size_t)(i & 1) * n1;
+                VT *cur = rows2 + (size_t)((i - 1) & 1) * n1;
+                uint8_t *chrow = chw + (size_t)(i - 1) * n1;
+                const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
+                for (int j = bl + lane; j <= bh; j += 32) {
+                    VT best = vInf;
+                    int arg = 255;
+                    int klo = j - nmax; if (klo < pbl) klo = pbl;
+                    int khi = j - nmin; if (khi > pbh) khi = pbh;
+                    int seg_hi = khi;
+                    for (int r = 0; r < R && seg_hi >= klo; ++r) {
+                        if (!((rc_mask >> r) & 1u)) continue;
+                        int lo = th[(size_t)r * n1 + j];
+                        if (lo < klo) lo = klo;
+                        if (lo > seg_hi) continue;
+                        for (int k = seg_hi; k >= lo; --k) {
+                            VT cst;
+                            if (LINEAR) cst = (rM[(size_t)r * n1 + j] - rM[(size_t)r * n1 + k]) + K;
+                            else cst = ((rM[j] - rM[k]) + tau_term((i64)dc.tau_q[r], rM[n1 + j] - rM[n1 + k])) + K;
+                            const VT v = prev[k] + cst;
+                            if (cst <= bott && v <= best && v < vInf) { best = v; arg = k; }
+                        }
+                        seg_hi = lo - 1;
+                    }
+                    cur[j] = best;
+                    chrow[j] = (uint8_t)arg;
+                }
+                __syncwarp();
+                pbl = bl; pbh = bh;
+            }
+        }
 
         // ---- backtrace, Eq. 4 -----------------------------------------------------------
         VT T_iter = vInf, T_pipe = vInf, T_sync = 0, T_opt = 0;

@@ -305,3 +305,51 @@ def test_fp64_mode_costs_within_1e9_relative(hap, name, kw):
     # integer and fp64 modes pick plans of (nearly) the same cost
     iplan, _ = hap.hap_search_best(hp)
     assert abs(iplan["T_iter"] - plan["T_iter_f64"]) <= 1e-3 * plan["T_iter_f64"]
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}), ("dsv2", {})])
+def test_refinement_pass_bit_exact(hap, name, kw):
+    """HAP_OPT_REFINE: smallest stage-cost sum among the bottleneck-optimal partitions, against the oracle's
+    refined evaluation of every candidate; plan and pruned plan included."""
+    pb = problems.make_problem(name, **kw)
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs_refined(0, 1, threads=NTHREADS)
+    for prune in (0, 1):
+        hp = hap.hap_problem_create(pb, prune=prune, flags=hap.OPT_REFINE)
+        hap.hap_enumerate(hp)
+        if prune == 0:
+            out = hap.hap_pipeline_dp(hp, 0, hp.n_cand, partition=True)
+            torch.cuda.synchronize()
+            assert np.array_equal(out["cost"].cpu().numpy(), costs)
+            assert np.array_equal(out["bottleneck"].cpu().numpy(), bn)
+            part, rec = out["partition"].cpu().numpy(), out["recompute"].cpu().numpy()
+            for idx in range(0, o.n_cand, max(1, o.n_cand // 400)):
+                ref = o.eval_index_refined(idx)
+                if ref["T_iter"] < INF:
+                    assert part[idx, :ref["PP"]].tolist() == ref["n"] and rec[idx, :ref["PP"]].tolist() == ref["r"], idx
+            with pytest.raises(hap.HapError):
+                hap.hap_pipeline_dp_f64(hp, 0, 1)
+        plan, stats = hap.hap_search_best(hp)
+        assert (plan["T_iter"], plan["index"]) == (bc, bi)
+        ref = o.eval_index_refined(bi)
+        assert plan["n"] == ref["n"] and plan["r"] == ref["r"] and plan["T_pipe"] == ref["T_pipe"]
+        hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("seed", [4, 5])
+def test_refinement_on_random_problems_with_general_levels(hap, seed):
+    pb = problems.random_small(seed, N=9 + seed % 4, T=2 + seed % 2, nodes_per_type=((2, 2), (2, 1, 1))[seed % 2],
+                               node_size=2, window=(seed % 2 == 0), first_dense=True)
+    pb.xi_q = np.ascontiguousarray(np.array([1024, 512, 64], np.int32))
+    pb.tau_q = np.ascontiguousarray(np.array([0, 300, 1000], np.int32))
+    pb.rc_masks = np.ascontiguousarray(np.array([0b001, 0b011, 0b111, 0b101], np.uint32))
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs_refined(0, 1, threads=NTHREADS)
+    hp = hap.hap_problem_create(pb, flags=hap.OPT_REFINE)
+    hap.hap_enumerate(hp)
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["cost"].cpu().numpy(), costs)
+    plan, _ = hap.hap_search_best(hp)
+    assert (plan["T_iter"], plan["index"]) == (bc, bi)
+    hap.hap_problem_destroy(hp)

@@ -604,3 +604,67 @@ def test_infeasible_memory_plans_are_never_chosen():
     pb2.cap_eff[:] = 1 << 20
     c2, _, best2, feas2 = Oracle(pb2).search(0, 2000)
     assert feas2 == 0 and best2 is None and (c2 == INF).all()
+
+
+# --------------------------------------------------------------------------------------
+# refinement: smallest stage-cost sum among the bottleneck-optimal partitions
+# --------------------------------------------------------------------------------------
+def _refined_partition_by_bruteforce(o, p, mp, rc, c2, coef, PP, N, limit):
+    n, j = [], N
+    for i in range(PP, 0, -1):
+        target = o.bruteforce_sum(p, mp, rc, c2, coef, i, j, limit)
+        pick = None
+        for k in range(i - 1, j):
+            left = o.bruteforce_sum(p, mp, rc, c2, coef, i - 1, k, limit)
+            c, _ = o.stage_cost(p, mp, rc, c2, coef, i, k, j)
+            if left < INF and c <= limit and left + c == target:
+                pick = k
+                break
+        assert pick is not None
+        n.append(j - pick)
+        j = pick
+    return n[::-1]
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_refinement_is_the_exhaustive_minimum_sum_under_the_bottleneck(seed):
+    pb = problems.random_small(seed, N=8 + seed % 3, T=2, nodes_per_type=(2, 2), node_size=2, window=(seed % 2 == 1),
+                               first_dense=(seed % 2 == 0))
+    o = Oracle(pb)
+    costs, bn, _, _ = o.search()
+    n_rc = len(pb.rc_masks)
+    changed = 0
+    for idx in range(0, o.n_cand, 5):
+        p = o.find_pconf(idx)
+        PP, M = int(o.pconfs["PP"][p]), int(o.pconfs["M"][p])
+        local = idx - int(o.pconfs["offset"][p])
+        mp = o.decode(p, local // n_rc)
+        rc = int(pb.rc_masks[local % n_rc])
+        c2, _, coef, _ = o.layer_costs(p)
+        ref = o.eval_index_refined(idx)
+        if bn[idx] >= INF:
+            assert ref["T_iter"] == INF
+            continue
+        plain, _, _ = o.eval_index(idx)
+        assert ref["bottleneck"] == bn[idx] == max(ref["c"])                 # the bottleneck stays optimal
+        best_sum = o.bruteforce_sum(p, mp, rc, c2, coef, PP, pb.N, int(bn[idx]))
+        assert sum(ref["c"]) == best_sum <= sum(plain["c"])
+        assert ref["n"] == _refined_partition_by_bruteforce(o, p, mp, rc, c2, coef, PP, pb.N, int(bn[idx]))
+        assert ref["T_pipe"] == best_sum + (M - 1) * int(bn[idx]) <= plain["T_pipe"]
+        assert ref["T_iter"] == ref["T_pipe"] + ref["T_sync"] + ref["T_opt"]
+        # no cheaper sum exists even one unit below the bottleneck limit that still reaches B*
+        assert o.bruteforce_sum(p, mp, rc, c2, coef, PP, pb.N, int(bn[idx]) - 1) == INF
+        changed += ref["n"] != plain["n"]
+
+
+def test_refinement_changes_some_partitions_and_never_raises_the_pipeline_time():
+    o = Oracle(problems.tiny())
+    c0, b0, _, _ = o.search()
+    done, bc, bi, c1, b1 = o.search_pconfs_refined(0, 1, threads=2)
+    assert np.array_equal(b0, b1)
+    moved = [i for i in np.nonzero(c0 != c1)[0]]
+    assert len(moved) > 0
+    for i in moved[:20]:
+        plain, _, _ = o.eval_index(int(i))
+        ref = o.eval_index_refined(int(i))
+        assert ref["T_pipe"] <= plain["T_pipe"] and ref["n"] != plain["n"]
