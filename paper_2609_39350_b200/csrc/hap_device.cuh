@@ -571,8 +571,9 @@ struct MaskInfo {
     int capt, pad;
 };
 
+// two blocks of up to 12 warps per SM: the register cap (85) keeps the occupancy independent of ptxas' heuristics
 template <bool SEARCH, bool LINEAR, bool COUNT = false, typename VT = i64, bool REFINE = false>
-__global__ void __launch_bounds__(kDpWarps * 32)
+__global__ void __launch_bounds__(kDpWarps * 32, 2)
 pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const i64 *coef, const VT *coefv,
                    const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
 {
@@ -819,6 +820,26 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         const unsigned differ = __ballot_sync(0xffffffffu, lane < PP && (mask != prev_mask || link != prev_link));
         int s0 = differ ? __ffs(differ) - 1 : PP;      // stages 1..s0 are shared with the previous mapping
         prev_mask = mask; prev_link = link;
+        if (!multiset) s0 = 0;               // block mode: window and bands depend on the whole mapping
+        if (s0 > valid_rows) s0 = valid_rows;
+        if (want_tables) s0 = 0;
+        if (dead_stage > s0) dead_stage = 1 << 30;       // the dead row, if any, is not part of the shared prefix
+        if (!COUNT && dead_stage <= s0) {
+            // a shared stage prefix that already admits no feasible partition settles this mapping too
+            valid_rows = s0;
+            if (SEARCH) n_eval++;
+            else {
+                const u64 o = c - out.first;
+                if (lane == 0) {
+                    if (out.cost) reinterpret_cast<VT *>(out.cost)[o] = vInf;
+                    if (out.bottleneck) reinterpret_cast<VT *>(out.bottleneck)[o] = vInf;
+                    if (out.detail) { VT *d = reinterpret_cast<VT *>(out.detail); d[o * 3] = vInf; d[o * 3 + 1] = 0; d[o * 3 + 2] = 0; }
+                }
+                if (out.partition) out.partition[o * HAP_MAX_PP + lane] = 0;
+                if (out.recompute) out.recompute[o * HAP_MAX_PP + lane] = 0;
+            }
+            continue;
+        }
 
         StagePar<VT> sp;
         sp.mrow = 0; sp.capt = 0; sp.K = 0; sp.nmin = 1; sp.nmax = N - PP + 1; sp.bl = 0; sp.bh = 0;
@@ -849,12 +870,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                 }
             }
         }
-        if (!multiset) s0 = 0;               // block mode: window and bands depend on the whole mapping
-        if (s0 > valid_rows) s0 = valid_rows;
-        if (want_tables) s0 = 0;
-        if (dead_stage > s0) dead_stage = 1 << 30;       // the dead row, if any, is not part of the shared prefix
-        // a shared stage prefix that already admits no feasible partition settles this mapping too
-        const bool dead_prefix = dead_stage <= s0;
+        const bool dead_prefix = false;                  // (handled above, before the stage parameters)
 
         // ---- bands: end layers j that stage i can reach (prefix sums of the window bounds), and from
         //      which the remaining stages can still reach N (suffix sums; not applied when the caller
