@@ -505,8 +505,8 @@ static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double 
 {
     const u64 nph = (u64)p->pconfs.size() * HAP_MAX_TYPES;
     const unsigned b1 = (unsigned)((nph + kLcThreads - 1) / kLcThreads);
-    if (quant) type_const_kernel<true><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr, p->d_range);
-    else type_const_kernel<false><<<b1, kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff, p->d_range);
+    if (quant) type_const_kernel<true><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr, p->d_range);
+    else type_const_kernel<false><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff, p->d_range);
     CUDA_TRY(p, cudaGetLastError());
     if ((quant && c2) || (!quant && c2f)) {
         const unsigned b2 = (unsigned)p->pconfs.size();

@@ -167,115 +167,127 @@ __device__ __forceinline__ double div_by(double a, double b, double y)
     return __fma_rn(r, y, q0);
 }
 
-// Phase 1 (type_const_kernel): one thread per (configuration, type) computes the per-type constants of
-// Eq. 2 / Eq. 3 into a scratch array and the stage coefficients.  Phase 2 (layer_cost_kernel): one thread
-// per (configuration, type, layer) unit, consecutive threads writing consecutive 16-byte results.
+// Phase 1 (type_const_kernel): per (configuration, type) the constants of Eq. 2 / Eq. 3 (into a scratch array)
+// and the 20 stage coefficients.  The work of one (configuration, type) is a chain of about 40 fp64 divisions,
+// so it is cut into three independent roles (blockIdx.y: layer constants; p2p / activation / extra-memory
+// coefficients; weight / sync / optimizer coefficients), one thread per (configuration, type) and role.
+// Phase 2 (layer_cost_kernel): one block per configuration, one thread per layer.
+template <bool QUANT>
+__device__ __forceinline__ bool put_coef(i64 *coef, double *coeff, size_t at, int q, double v)
+{
+    if (QUANT) coef[at + q] = __double2ll_rn(v);
+    else coeff[at + q] = v;
+    // time coefficients must stay below 2^40 ns (per-layer ones below 2^36), bytes below 2^50
+    const double lim = q <= HAP_SLAT ? 1.0995e12 : (q < HAP_MW ? 6.8719e10 : 1.1259e15);
+    return !(v < lim);
+}
+
 template <bool QUANT>
 __global__ void __launch_bounds__(kLcThreads)
 type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u64 *range_flag)
 {
     const int T = dc.T;
+    const int role = blockIdx.y;
     const i64 H = dc.H;
-    const i64 Hkv = H * dc.nkv / dc.nq;
-    {
-        const u64 gid = (u64)blockIdx.x * kLcThreads + threadIdx.x;
-        const u64 p = gid / HAP_MAX_TYPES;
-        const int h = (int)(gid % HAP_MAX_TYPES);
-        if (p < dc.n_pconf && h < T) {
-            const hap_pconf pc = dc.pconf[p];
-            const int TP = pc.TP, CP = pc.CP, DP = pc.DP, EP = pc.EP, TPE = pc.TPE, EDP = pc.EDP, b = pc.b;
-            const i64 G = pc.G;
-            const i64 tok = (i64)b * dc.S / CP;
-            const double thb = (double)tok * (double)H;
-            const double Dtp = thb * dc.beta;
-            LinkCtx lc; lc.bw_intra = dc.bw_intra[h]; lc.bw_inter = dc.bw_inter[h]; lc.node_size = dc.node_size[h];
-            TypeConst tc;
-            tc.imb = 1.0 + dc.gamma * (dc.rho[pc.iep] - 1.0);
-            double tdisp = 0.0;
-            if (EP != 1) {
-                const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
-                const double Dag = (thb * dc.beta) * (double)(EP - 1);
-                const int cls = link_class(lc, (i64)EP * TPE);
-                const double fa = dc.alpha[cls] * (double)(EP - 1) + Dmoe / link_bw(lc, cls);
-                const double fg = dc.alpha[cls] * (double)(EP - 1) + Dag / link_bw(lc, cls);
-                tdisp = (fa <= fg) ? fa : fg;
-            }
-            tc.disp2 = 2.0 * tdisp;
-            const double ttpA = 2.0 * collective_ns(dc, lc, TP, TP, Dtp);
-            const double ttpD = ttpA;
-            const double ttpM = 2.0 * collective_ns(dc, lc, TPE, TPE, Dtp);
-            const double Dkv = ((((2.0 * (double)b) * (double)dc.S) * (double)Hkv) * dc.beta) / (double)TP;
-            const double tcp = collective_ns(dc, lc, CP, (i64)TP * CP, Dkv);
-            tc.tr = dc.croute[h] * thb;
-            tc.tr2 = 2.0 * tc.tr;
-            tc.commF[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
-            tc.commB[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
-            tc.commF[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
-            tc.commB[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
-            tc.den = (dc.eta[h] * (double)EP) * (double)TPE;
-            tc.rden = 1.0 / tc.den;
-            tc.row = (pc.itp * dc.ncp + pc.icp) * dc.nmb + pc.ib;
-            tcg[p * T + h] = tc;
+    const u64 gid = (u64)blockIdx.x * kLcThreads + threadIdx.x;
+    const u64 p = gid / HAP_MAX_TYPES;
+    const int h = (int)(gid % HAP_MAX_TYPES);
+    if (p >= dc.n_pconf || h >= T) return;
+    const bool want_coef = (QUANT && coef) || (!QUANT && coeff);
+    if (role != 0 && !want_coef) return;
+    const hap_pconf pc = dc.pconf[p];
+    const int TP = pc.TP, CP = pc.CP, DP = pc.DP, EP = pc.EP, TPE = pc.TPE, EDP = pc.EDP, b = pc.b;
+    const i64 G = pc.G;
+    const i64 tok = (i64)((unsigned)b * (unsigned)dc.S / (unsigned)CP);
+    const i64 Hkv = (i64)((unsigned)dc.H * (unsigned)dc.nkv / (unsigned)dc.nq);
+    const double thb = (double)tok * (double)H;
+    const double Dtp = thb * dc.beta;
+    LinkCtx lc; lc.bw_intra = dc.bw_intra[h]; lc.bw_inter = dc.bw_inter[h]; lc.node_size = dc.node_size[h];
+    const size_t at = ((size_t)p * T + h) * HAP_NCOEF;
+    bool bad = false;
 
-            if ((QUANT && coef) || (!QUANT && coeff)) {
-                double v[HAP_NCOEF];
-                const size_t i4 = (((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib;
-                v[HAP_KPRE] = dc.tpre[i4];
-                v[HAP_KPOST] = dc.tpost[i4];
-                const double Dp = Dtp / (double)TP;
-                v[HAP_KP2P_INTRA] = 2.0 * (dc.alpha[HAP_INTRA] + Dp / dc.bw_intra[h]);
-                v[HAP_KP2P_INTER] = 2.0 * (dc.alpha[HAP_INTER] + Dp / dc.bw_inter[h]);
-#pragma unroll
-                for (int h2 = 0; h2 < HAP_MAX_TYPES; ++h2) {
-                    const double bo = h2 < T ? dc.bw_inter[h2] : dc.bw_inter[h];
-                    const double bmin = dc.bw_inter[h] < bo ? dc.bw_inter[h] : bo;
-                    v[HAP_KP2P_CROSS + h2] = 2.0 * (dc.alpha[HAP_CROSS] + Dp / (bmin * dc.chi));
-                }
-                const i64 wd = (i64)DP * CP;
-                const double shd = 6.0 + 12.0 / (double)wd;
-                const double she = 6.0 + 12.0 / (double)EDP;
-                const i64 Pattn = H * (H + 2 * Hkv) + H * H + 2 * H;
-                const i64 Pffn_d = 3 * H * (i64)dc.F_dense, Pffn_e = 3 * H * (i64)dc.F_exp;
-                const i64 Pe = (i64)(dc.E / EP) * Pffn_e;
-                const i64 Prt = H * (i64)dc.E;
-                i64 Pd[2];
-                Pd[HAP_DENSE] = Pattn + Pffn_d;
-                Pd[HAP_MOE] = Pattn + (i64)dc.n_shared * Pffn_e;
-                const double PeT = (double)Pe / (double)TPE;
-                v[HAP_MW + HAP_DENSE] = ((double)Pd[HAP_DENSE] / (double)TP) * shd;
-                v[HAP_MW + HAP_MOE] = ((double)Pd[HAP_MOE] / (double)TP + (double)Prt) * shd + PeT * she;
-                v[HAP_MA + HAP_DENSE] = (thb * dc.act_coef[HAP_DENSE]) / (double)TP;
-                v[HAP_MA + HAP_MOE] = (thb * dc.act_coef[HAP_MOE]) / (double)TP;
-                v[HAP_MX] = ((2.0 * ((thb * dc.beta) * (double)dc.k)) * (1.0 - 1.0 / (double)EP)) * dc.capf
-                            + ((double)tok * (double)dc.E) * 4.0;
-                v[HAP_MPRE] = (((double)dc.V * (double)H) / (double)TP) * shd;
-                v[HAP_MPOST] = v[HAP_MPRE];
-                const int cG = link_class(lc, G);
-                const double bwG = link_bw(lc, cG);
-                const double vfd = (double)(wd - 1) / (double)wd, vfe = (double)(EDP - 1) / (double)EDP;
-#pragma unroll
-                for (int kd = 0; kd < 2; ++kd) {
-                    const i64 Pdd = Pd[kd] + (kd == HAP_MOE ? Prt : 0);
-                    const double Pel = kd == HAP_MOE ? PeT : 0.0;
-                    v[HAP_SBW + kd] = dc.ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG)
-                                                   + (((6.0 * Pel) * vfe) / bwG));
-                    v[HAP_OPT + kd] = dc.copt[h] * ((double)Pdd / (double)((i64)TP * DP * CP) + Pel / (double)EDP);
-                }
-                v[HAP_SLAT] = dc.ovl_dp * (dc.alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
-                const size_t at = ((size_t)p * T + h) * HAP_NCOEF;
-                bool bad = false;
-#pragma unroll
-                for (int q = 0; q < HAP_NCOEF; ++q) {
-                    if (QUANT) coef[at + q] = __double2ll_rn(v[q]);
-                    else coeff[at + q] = v[q];
-                    // time coefficients must stay below 2^40 ns (per-layer ones below 2^36), bytes below 2^50
-                    const double lim = q <= HAP_SLAT ? 1.0995e12 : (q < HAP_MW ? 6.8719e10 : 1.1259e15);
-                    bad |= !(v[q] < lim);
-                }
-                if (bad && range_flag) atomicOr(range_flag, 1ull);
-            }
+    if (role == 0) {
+        TypeConst tc;
+        tc.imb = 1.0 + dc.gamma * (dc.rho[pc.iep] - 1.0);
+        double tdisp = 0.0;
+        if (EP != 1) {
+            const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
+            const double Dag = (thb * dc.beta) * (double)(EP - 1);
+            const int cls = link_class(lc, (i64)EP * TPE);
+            const double fa = dc.alpha[cls] * (double)(EP - 1) + Dmoe / link_bw(lc, cls);
+            const double fg = dc.alpha[cls] * (double)(EP - 1) + Dag / link_bw(lc, cls);
+            tdisp = (fa <= fg) ? fa : fg;
         }
+        tc.disp2 = 2.0 * tdisp;
+        const double ttpA = 2.0 * collective_ns(dc, lc, TP, TP, Dtp);
+        const double ttpD = ttpA;
+        const double ttpM = 2.0 * collective_ns(dc, lc, TPE, TPE, Dtp);
+        const double Dkv = ((((2.0 * (double)b) * (double)dc.S) * (double)Hkv) * dc.beta) / (double)TP;
+        const double tcp = collective_ns(dc, lc, CP, (i64)TP * CP, Dkv);
+        tc.tr = dc.croute[h] * thb;
+        tc.tr2 = 2.0 * tc.tr;
+        tc.commF[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
+        tc.commB[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
+        tc.commF[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
+        tc.commB[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
+        tc.den = (dc.eta[h] * (double)EP) * (double)TPE;
+        tc.rden = 1.0 / tc.den;
+        tc.row = (pc.itp * dc.ncp + pc.icp) * dc.nmb + pc.ib;
+        tcg[p * T + h] = tc;
+    } else if (role == 1) {
+        const size_t i4 = (((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib;
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KPRE, dc.tpre[i4]);
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KPOST, dc.tpost[i4]);
+        const double Dp = Dtp / (double)TP;
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_INTRA, 2.0 * (dc.alpha[HAP_INTRA] + Dp / dc.bw_intra[h]));
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_INTER, 2.0 * (dc.alpha[HAP_INTER] + Dp / dc.bw_inter[h]));
+#pragma unroll
+        for (int h2 = 0; h2 < HAP_MAX_TYPES; ++h2) {
+            const double bo = h2 < T ? dc.bw_inter[h2] : dc.bw_inter[h];
+            const double bmin = dc.bw_inter[h] < bo ? dc.bw_inter[h] : bo;
+            bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_CROSS + h2, 2.0 * (dc.alpha[HAP_CROSS] + Dp / (bmin * dc.chi)));
+        }
+        const i64 wd = (i64)DP * CP;
+        const double shd = 6.0 + 12.0 / (double)wd;
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MA + HAP_DENSE, (thb * dc.act_coef[HAP_DENSE]) / (double)TP);
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MA + HAP_MOE, (thb * dc.act_coef[HAP_MOE]) / (double)TP);
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MX,
+                               ((2.0 * ((thb * dc.beta) * (double)dc.k)) * (1.0 - 1.0 / (double)EP)) * dc.capf
+                               + ((double)tok * (double)dc.E) * 4.0);
+        const double mpre = (((double)dc.V * (double)H) / (double)TP) * shd;
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MPRE, mpre);
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MPOST, mpre);
+    } else {
+        const i64 wd = (i64)DP * CP;
+        const double shd = 6.0 + 12.0 / (double)wd;
+        const double she = 6.0 + 12.0 / (double)EDP;
+        const i64 Pattn = H * (H + 2 * Hkv) + H * H + 2 * H;
+        const i64 Pffn_d = 3 * H * (i64)dc.F_dense, Pffn_e = 3 * H * (i64)dc.F_exp;
+        const i64 Pe = (i64)(dc.E / EP) * Pffn_e;
+        const i64 Prt = H * (i64)dc.E;
+        i64 Pd[2];
+        Pd[HAP_DENSE] = Pattn + Pffn_d;
+        Pd[HAP_MOE] = Pattn + (i64)dc.n_shared * Pffn_e;
+        const double PeT = (double)Pe / (double)TPE;
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MW + HAP_DENSE, ((double)Pd[HAP_DENSE] / (double)TP) * shd);
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_MW + HAP_MOE,
+                               ((double)Pd[HAP_MOE] / (double)TP + (double)Prt) * shd + PeT * she);
+        const int cG = link_class(lc, G);
+        const double bwG = link_bw(lc, cG);
+        const double vfd = (double)(wd - 1) / (double)wd, vfe = (double)(EDP - 1) / (double)EDP;
+#pragma unroll
+        for (int kd = 0; kd < 2; ++kd) {
+            const i64 Pdd = Pd[kd] + (kd == HAP_MOE ? Prt : 0);
+            const double Pel = kd == HAP_MOE ? PeT : 0.0;
+            bad |= put_coef<QUANT>(coef, coeff, at, HAP_SBW + kd,
+                                   dc.ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG) + (((6.0 * Pel) * vfe) / bwG)));
+            bad |= put_coef<QUANT>(coef, coeff, at, HAP_OPT + kd,
+                                   dc.copt[h] * ((double)Pdd / (double)((i64)TP * DP * CP) + Pel / (double)EDP));
+        }
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_SLAT,
+                               dc.ovl_dp * (dc.alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1))));
     }
+    if (bad && range_flag) atomicOr(range_flag, 1ull);
 }
 
 // one block per configuration, one thread per layer; a thread handles its layer for every device type, so
