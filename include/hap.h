@@ -145,6 +145,8 @@ typedef struct {
     const uint32_t *rc_masks;            /* [n_rc] bit r set: level r allowed; per stage the lowest feasible allowed level is used */
     int32_t prune;                       /* hap_search_* may skip candidates whose lower bound exceeds the incumbent */
     int32_t flags;                       /* HAP_OPT_* bits */
+    int32_t eta_q;                       /* Pruning 3: drop a candidate whose cross-type transfer time per micro-batch exceeds
+                                            eta x its mean stage time; eta in 1/1024 (2048 = the paper's default 2); <= 0: off */
 } hap_search_opts;
 
 /* One accepted parallel configuration x micro-batch size.  Candidate index of

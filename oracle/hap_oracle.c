@@ -508,6 +508,26 @@ int64_t orc_stage_cost(const orc_problem *pr, const orc_pconf *pc, const orc_map
     return c;
 }
 
+
+/* Pruning 3 (heterogeneous communication): the candidate is dropped when its cross-type communication time
+ * per micro-batch -- here the stage-to-stage transfers over cross-type links, the only cross-type traffic
+ * the model carries -- exceeds eta times the mean stage time, T_hetero > eta * (1/PP) * sum_i c_i.
+ * eta is given in 1/1024 (eta_q = 2048 is the paper's default eta = 2); eta_q <= 0 switches the rule off. */
+static int64_t hetero_comm(const orc_pconf *pc, const orc_mapping *mp, const int64_t *coef)
+{
+    int64_t t = 0;
+    for (int s = 1; s < pc->PP; ++s)
+        if (mp->cls[s] == ORC_CROSS) t += coef[mp->hb[s] * ORC_NCOEF + ORC_KP2P_CROSS + mp->ha[s]];
+    return t;
+}
+
+static int pruned_by_hetero_comm(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                                 const int64_t *coef, int64_t sum_stage)
+{
+    if (pr->eta_q <= 0) return 0;
+    return hetero_comm(pc, mp, coef) * (int64_t)pc->PP * 1024 > (int64_t)pr->eta_q * sum_stage;
+}
+
 /* ------------------------------------------------------------------------------------ *
  * Min-max pipeline partitioning recurrence, backtrace and Eq. 4 closed form.
  * dp_table: [(PP+1)][(N+1)] or NULL; ch_table: same shape, 255 where undefined.
@@ -570,6 +590,7 @@ int orc_candidate(const orc_problem *pr, const orc_pconf *pc, const orc_mapping 
     res->T_sync = tsync;
     res->T_opt = topt;
     res->T_iter = res->T_pipe + tsync + topt;
+    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum)) res->T_iter = res->T_pipe = ORC_INF;   /* Pruning 3 */
     free(DPt); free(CH); free(cx);
 #undef DPAT
 #undef CHAT
@@ -635,6 +656,7 @@ int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_
     res->T_sync = tsync;
     res->T_opt = topt;
     res->T_iter = res->T_pipe + tsync + topt;
+    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum)) res->T_iter = res->T_pipe = ORC_INF;   /* Pruning 3 */
     free(D); free(CH); free(cx);
 #undef DAT
 #undef CHAT
@@ -990,6 +1012,12 @@ int orc_candidate_f64(const orc_problem *pr, const orc_pconf *pc, const orc_mapp
     res->T_sync = tsync;
     res->T_opt = topt;
     res->T_iter = res->T_pipe + tsync + topt;
+    if (pr->eta_q > 0) {                                   /* Pruning 3 on the unrounded values */
+        double th = 0.0;
+        for (int st = 1; st < PP; ++st)
+            if (mp->cls[st] == ORC_CROSS) th += coeff[mp->hb[st] * ORC_NCOEF + ORC_KP2P_CROSS + mp->ha[st]];
+        if (th * (double)PP * 1024.0 > (double)pr->eta_q * sum) res->T_iter = res->T_pipe = INFINITY;
+    }
     free(DPt); free(CH); free(cx);
 #undef DPAT
 #undef CHAT

@@ -70,6 +70,7 @@ typedef struct {
     uint64_t map_cap;
     int32_t n_rc;
     const uint32_t *rc_masks;
+    int32_t eta_q;      /* Pruning 3 threshold eta in 1/1024; <= 0: off */
 } orc_problem;
 
 typedef struct {

@@ -50,7 +50,7 @@ class _Problem(C.Structure):
         ("R", C.c_int32), ("xi_q", C.c_void_p), ("tau_q", C.c_void_p),
         ("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
         ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64),
-        ("n_rc", C.c_int32), ("rc_masks", C.c_void_p),
+        ("n_rc", C.c_int32), ("rc_masks", C.c_void_p), ("eta_q", C.c_int32),
     ]
 
 
@@ -150,6 +150,7 @@ class Oracle:
         s.tp_max, s.delta_q, s.map_cap = int(pb.tp_max), int(pb.delta_q), int(pb.map_cap)
         s.n_rc = len(pb.rc_masks)
         s.rc_masks = arr("rc_masks", np.uint32)
+        s.eta_q = int(getattr(pb, "eta_q", 0))
         self._keep = keep
         self.s = s
         self.N, self.T = int(pb.N), s.T

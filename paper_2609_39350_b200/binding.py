@@ -51,7 +51,7 @@ class _Profile(C.Structure):
 class _Opts(C.Structure):
     _fields_ = [("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
                 ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64), ("n_rc", C.c_int32),
-                ("rc_masks", C.c_void_p), ("prune", C.c_int32), ("flags", C.c_int32)]
+                ("rc_masks", C.c_void_p), ("prune", C.c_int32), ("flags", C.c_int32), ("eta_q", C.c_int32)]
 
 
 class _Plan(C.Structure):
@@ -179,6 +179,7 @@ def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     so.rc_masks = arr("rc_masks", np.uint32)
     so.prune = int(prune)
     so.flags = int(flags)
+    so.eta_q = int(getattr(pb, "eta_q", 0))
     out = C.c_void_p(0)
     st = L.hap_problem_create(C.byref(mo), C.byref(cl), C.byref(pf), C.byref(so), C.byref(out))
     if st != 0:

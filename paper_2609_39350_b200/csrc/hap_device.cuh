@@ -29,7 +29,7 @@ constexpr i64 kInf = (i64)1 << 62;
 struct DevConst {
     int N, T, R, n_rc, ntp, ncp, nmb, nep;
     int S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
-    int delta_q, tau_linear, pad0;
+    int delta_q, tau_linear, eta_q;
     double beta, kappa, chi, gamma, ovl_tp, ovl_cp, ovl_dp, capf;
     double alpha[3];
     double eta[HAP_MAX_TYPES], croute[HAP_MAX_TYPES], copt[HAP_MAX_TYPES];
@@ -1093,6 +1093,8 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                 sync_me = mi_.slat + n_dense * mi_.sbw[0] + n_moe * mi_.sbw[1];
                 opt_me = n_dense * mi_.opt[0] + n_moe * mi_.opt[1];
             }
+            VT het_me = 0;                                  // cross-type transfer into this lane's stage (Pruning 3)
+            if (dc.eta_q > 0 && lane > 0 && lane < PP && (link & 3) == HAP_CROSS) het_me = sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
             VT sum = c_me, mxc = c_me;
             for (int o = red0; o > 0; o >>= 1) {          // lanes >= PP hold zeros
                 const VT t1 = __shfl_xor_sync(0xffffffffu, sum, o), t2 = __shfl_xor_sync(0xffffffffu, mxc, o);
@@ -1102,6 +1104,13 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             T_pipe = shfl_v(sum + (VT)(pc.M - 1) * mxc, 0);
             T_sync = shfl_v(sync_me, 0); T_opt = shfl_v(opt_me, 0);
             T_iter = T_pipe + T_sync + T_opt;
+            if (dc.eta_q > 0) {
+                // Pruning 3: cross-type communication per micro-batch above eta x the mean stage time drops the
+                // candidate (its bottleneck is still reported)
+                for (int o = red0; o > 0; o >>= 1) het_me += __shfl_xor_sync(0xffffffffu, het_me, o);
+                const VT het = shfl_v(het_me, 0), ssum = shfl_v(sum, 0);
+                if (het * (VT)PP * (VT)1024 > (VT)dc.eta_q * ssum) { T_iter = vInf; T_pipe = vInf; }
+            }
         }
         if (SEARCH) {
             n_eval++;

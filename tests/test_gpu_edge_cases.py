@@ -132,3 +132,27 @@ def test_value_limits_are_reported(hap):
     with pytest.raises(hap.HapError) as e:
         hap.hap_problem_create(huge_batch)
     assert e.value.name == "HAP_E_RANGE"
+
+
+@pytest.mark.parametrize("name,eta_q", [("tiny", 64), ("tiny", 16), ("small", 2048), ("small", 24), ("mixtral", 12)])
+def test_heterogeneous_communication_pruning(hap, name, eta_q):
+    """Pruning 3: candidates whose cross-type transfer time exceeds eta x the mean stage time cost +INF."""
+    pb = problems.make_problem(name)
+    base = Oracle(pb).search_pconfs(0, 1, threads=8, want_costs=True)[3]
+    pb.eta_q = eta_q
+    o, costs = full_compare(hap, pb)
+    dropped = int(((costs >= INF) & (base < INF)).sum())
+    assert (dropped > 0) == (eta_q < 2048)
+    assert np.array_equal(costs[costs < INF], base[costs < INF])
+    # fp64 mode applies the same rule to the unrounded values
+    hp = hap.hap_problem_create(pb)
+    hap.hap_enumerate(hp)
+    out = hap.hap_pipeline_dp_f64(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    done, cf, bf, parts = o.search_pconfs_f64(0, 1, threads=8)
+    got = out["cost"].cpu().numpy()
+    agree = np.isfinite(got) == np.isfinite(cf)
+    assert agree.mean() > 0.9999                      # a candidate exactly at the threshold may fall either way
+    fin = np.isfinite(got) & np.isfinite(cf)
+    assert np.max(np.abs(got[fin] - cf[fin]) / cf[fin]) <= 1e-9
+    hap.hap_problem_destroy(hp)

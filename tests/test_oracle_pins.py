@@ -89,6 +89,17 @@ def test_e1_two_device_example():
     assert best["index"] == g["best_map"] and feas == 2 and costs.tolist() == [ab["T_iter"], ba["T_iter"]]
 
 
+def test_e1_heterogeneous_communication_pruning():
+    g = gold("e1_two_device_pp2.json")["expect"]["pruning3"]
+    for eta_q, want in g.items():
+        pb = e1_problem()
+        pb.eta_q = int(eta_q)
+        costs, bn, best, feas = Oracle(pb).search()
+        assert costs.tolist() == [INF if w == "INF" else w for w in want]
+        assert bn.tolist() == [17288745, 18542094]           # the bottleneck itself is not touched by the rule
+        assert (best is None) == (want == ["INF", "INF"])
+
+
 def test_e1_fp64_mode_hand_values():
     g = gold("e1_two_device_pp2.json")["expect"]["fp64"]
     o = Oracle(e1_problem())
