@@ -583,77 +583,21 @@ struct MaskInfo {
     int capt, pad;
 };
 
-// two blocks of up to 12 warps per SM: the register cap (85) keeps the occupancy independent of ptxas' heuristics
-template <bool SEARCH, bool LINEAR, bool COUNT = false, typename VT = i64, bool REFINE = false>
-__global__ void __launch_bounds__(kDpWarps * 32, 2)
-pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const i64 *coef, const VT *coefv,
-                   const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
+// Block prologue shared by the DP kernels: everything that depends on the configuration only.
+// All threads of the block call it; it ends with a barrier.
+template <typename VT, bool LINEAR>
+__device__ __forceinline__ void dp_block_prologue(
+    const DevConst &dc, const hap_pconf &pc, unsigned p_index, const VT *c2, const i64 *coef, const VT *coefv,
+    bool multiset, int mrows, int RW, unsigned masks_used, int nwarps,
+    VT *sR, i64 *sW, i64 *sA, uint8_t *thr, uint8_t *sK, MaskInfo<VT> *minfo, VT (*sP2P)[6], VT *szero, int (*winT)[2])
 {
-    // c2: layer times; coef: integer coefficients (memory bytes); coefv: time coefficients in the value type
-    // (the same array as coef in integer mode)
-    const VT vInf = ValInf<VT>::get();
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP;
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const WorkItem it = items[blockIdx.x];
-    const hap_pconf pc = dc.pconf[it.p];
-    const int PP = pc.PP, n_rc = dc.n_rc;
-    {   // blocks whose candidates all lie outside the requested range have nothing to do
-        const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
-        if (c1 <= out.first || c0 >= out.first + out.count) {
-            if (SEARCH && threadIdx.x == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
-            return;
-        }
-    }
-    if (SEARCH && out.prune) {
-        // T_iter >= sum_i c_i + (M-1) max_i c_i >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on
-        // the summed stage time.  Skipping needs bound > incumbent (strict): the result cannot change.
-        // The incumbent moves while the block runs, so ONE thread reads it and the whole block follows that
-        // reading: a block must leave as a whole.
-        __shared__ int s_skip;
-        if (threadIdx.x == 0) {
-            const i64 S = out.lb_sum[it.p];
-            const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
-            const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
-            s_skip = (u64)lb > inc;
-            if (s_skip) {
-                out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
-                // candidates of this block inside the requested range
-                const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
-                const u64 a = c0 > out.first ? c0 : out.first, b = c1 < out.first + out.count ? c1 : out.first + out.count;
-                atomicAdd(out.counters + 2, b - a);
-            }
-        }
-        __syncthreads();
-        if (s_skip) return;
-    }
-    const bool multiset = pc.mode == HAP_MAP_MULTISET;
     const int nmask = (1 << T) - 1;
-    const int mrows = multiset ? T : nmask;
-    const int RW = LINEAR ? R : 2;
-
-    VT *sR = reinterpret_cast<VT *>(smem_raw);
-    i64 *sW = reinterpret_cast<i64 *>(sR + (size_t)mrows * RW * n1);
-    i64 *sA = sW + n1;
-    uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
-    const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
-    uint8_t *sK = thr + thr_bytes;
-    const int nrows = multiset ? PP : (PP < 2 ? PP : 2);   // block mode shares nothing between mappings: two rotating rows
-    const size_t row_bytes = (size_t)nrows * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
-    unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
-    VT *rows = reinterpret_cast<VT *>(wbase);            // row of stage i at rows + ((i-1) % nrows)*n1
-    uint8_t *chw = wbase + row_bytes;
-    // second-pass rows (refinement) sit behind all warps' first-pass storage
-    VT *rows2 = reinterpret_cast<VT *>(sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)nwarps * (row_bytes + ch_bytes)) + (size_t)wib * 2 * n1;
-    __shared__ MaskInfo<VT> minfo[kMaxMasks];
-    __shared__ VT sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
-    __shared__ VT szero[1];                               // the row of "stage 0": DP[0][0] = 0
-    __shared__ int winT[HAP_MAX_TYPES][2];
-
     // ---- block prologue 1: rows of this configuration -----------------------------------
-    const VT *c2p = c2 + (size_t)it.p * T * N * 2;
-    const i64 *cfp = coef + (size_t)it.p * T * HAP_NCOEF;
-    const VT *cvp = coefv + (size_t)it.p * T * HAP_NCOEF;
+    const VT *c2p = c2 + (size_t)p_index * T * N * 2;
+    const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
+    const VT *cvp = coefv + (size_t)p_index * T * HAP_NCOEF;
     for (int mr = wib; mr < mrows; mr += nwarps) {
         // time rows of one type mask: per layer the slowest member type, then prefix sums
         const int mk = multiset ? (1 << mr) : mr + 1;
@@ -789,6 +733,78 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         winT[threadIdx.x][0] = lo; winT[threadIdx.x][1] = hi;
     }
     __syncthreads();
+
+}
+
+// two blocks of up to 12 warps per SM: the register cap (85) keeps the occupancy independent of ptxas' heuristics
+template <bool SEARCH, bool LINEAR, bool COUNT = false, typename VT = i64, bool REFINE = false>
+__global__ void __launch_bounds__(kDpWarps * 32, 2)
+pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const i64 *coef, const VT *coefv,
+                   const uint8_t *maptab, DpOut out, int nwarps, unsigned masks_used)
+{
+    // c2: layer times; coef: integer coefficients (memory bytes); coefv: time coefficients in the value type
+    // (the same array as coef in integer mode)
+    const VT vInf = ValInf<VT>::get();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const WorkItem it = items[blockIdx.x];
+    const hap_pconf pc = dc.pconf[it.p];
+    const int PP = pc.PP, n_rc = dc.n_rc;
+    {   // blocks whose candidates all lie outside the requested range have nothing to do
+        const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
+        if (c1 <= out.first || c0 >= out.first + out.count) {
+            if (SEARCH && threadIdx.x == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
+            return;
+        }
+    }
+    if (SEARCH && out.prune) {
+        // T_iter >= sum_i c_i + (M-1) max_i c_i >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on
+        // the summed stage time.  Skipping needs bound > incumbent (strict): the result cannot change.
+        // The incumbent moves while the block runs, so ONE thread reads it and the whole block follows that
+        // reading: a block must leave as a whole.
+        __shared__ int s_skip;
+        if (threadIdx.x == 0) {
+            const i64 S = out.lb_sum[it.p];
+            const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
+            const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+            s_skip = (u64)lb > inc;
+            if (s_skip) {
+                out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
+                // candidates of this block inside the requested range
+                const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
+                const u64 a = c0 > out.first ? c0 : out.first, b = c1 < out.first + out.count ? c1 : out.first + out.count;
+                atomicAdd(out.counters + 2, b - a);
+            }
+        }
+        __syncthreads();
+        if (s_skip) return;
+    }
+    const bool multiset = pc.mode == HAP_MAP_MULTISET;
+    const int nmask = (1 << T) - 1;
+    const int mrows = multiset ? T : nmask;
+    const int RW = LINEAR ? R : 2;
+
+    VT *sR = reinterpret_cast<VT *>(smem_raw);
+    i64 *sW = reinterpret_cast<i64 *>(sR + (size_t)mrows * RW * n1);
+    i64 *sA = sW + n1;
+    uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
+    const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    uint8_t *sK = thr + thr_bytes;
+    const int nrows = multiset ? PP : (PP < 2 ? PP : 2);   // block mode shares nothing between mappings: two rotating rows
+    const size_t row_bytes = (size_t)nrows * n1 * 8, ch_bytes = ((size_t)PP * n1 + 15) / 16 * 16;
+    unsigned char *wbase = sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)wib * (row_bytes + ch_bytes);
+    VT *rows = reinterpret_cast<VT *>(wbase);            // row of stage i at rows + ((i-1) % nrows)*n1
+    uint8_t *chw = wbase + row_bytes;
+    // second-pass rows (refinement) sit behind all warps' first-pass storage
+    VT *rows2 = reinterpret_cast<VT *>(sK + ((size_t)n1 + 15) / 16 * 16 + (size_t)nwarps * (row_bytes + ch_bytes)) + (size_t)wib * 2 * n1;
+    __shared__ MaskInfo<VT> minfo[kMaxMasks];
+    __shared__ VT sP2P[HAP_MAX_TYPES][6];                 // per receiving type: intra, inter, cross from type 0..3
+    __shared__ VT szero[1];                               // the row of "stage 0": DP[0][0] = 0
+    __shared__ int winT[HAP_MAX_TYPES][2];
+
+    dp_block_prologue<VT, LINEAR>(dc, pc, it.p, c2, coef, coefv, multiset, mrows, RW, masks_used, nwarps,
+                                  sR, sW, sA, thr, sK, minfo, sP2P, szero, winT);
 
     VT best_cost = vInf;
     u64 best_index = ~0ull;
