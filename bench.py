@@ -231,6 +231,18 @@ def main():
 
     cells_finite = hap.hap_count_cells(hp, first, count)        # untimed instrumentation launch
 
+    # joint recurrence over the device state (all stage-type sequences at once), second call timed
+    joint_ms = None
+    if world == 1:
+        hap.hap_joint_bottleneck(hp)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        flush.fill_(1)
+        a.record(stream)
+        jb = hap.hap_joint_bottleneck(hp)
+        b.record(stream)
+        b.synchronize()
+        joint_ms = a.elapsed_time(b)
+
     # the same pass with the refinement (smallest stage-cost sum among the bottleneck-optimal partitions)
     hp_ref = hap.hap_problem_create(pb, flags=hap.OPT_REFINE)
     hap.hap_enumerate(hp_ref)
@@ -309,6 +321,7 @@ def main():
                      ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
             gpu_launches=(4 + len(set(int(x) for x in pconfs["PP"]))) * args.steps,
             refined_pass=dict(ms=statistics.median(ref_ms), best_cost=ref_best[0], best_index=ref_best[1] + first),
+            joint_recurrence_ms=joint_ms,
             full_search_ms=statistics.median(search_ms),
             full_search_pruned=dict(ms=statistics.median(pruned_ms), n_pruned=stats_pr["n_pruned"],
                                     n_evaluated=stats_pr["n_evaluated"]),

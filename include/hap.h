@@ -271,6 +271,15 @@ hap_status hap_argmin(hap_problem *, const int64_t *dev_cost, uint64_t count, in
 #define HAP_ARGMIN_STATIC_MAX_COUNT ((uint64_t)1 << 26)
 hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream);
 
+/* Sec. 3.5 / Algorithm 1 (HS-DP over the device-group state), with the min-max objective of this library: for every
+ * configuration whose stages are homogeneous (the per-stage device count divides every type's device count) and
+ * every recomputation policy, the minimum over ALL stage-type sequences -- not only the enumerated mappings -- of
+ * the pipeline bottleneck, from one recurrence over (layers placed, stages of each type used, type of the last
+ * stage).  dev_out: [n_pconf][n_rc] int64; HAP_INF when no sequence is feasible, -1 for configurations whose
+ * stages are not homogeneous.  Recomputes the layer costs into library-owned memory first; the first call
+ * allocates its state tables and scratch.  Asynchronous on `stream`. */
+hap_status hap_joint_bottleneck(hap_problem *, int64_t *dev_out, void *stream);
+
 /* Measurement aid: the number of recurrence cells (i, j, k) of candidates [first, first+count) whose stage
  * cost is finite, i.e. k inside the load-balance window of stage i (Pruning 1) and the span within the memory
  * limit at some allowed recomputation level (Pruning 2).  This is the recurrence work the method defines for

@@ -1058,3 +1058,124 @@ int orc_search_pconfs_f64(const orc_problem *pr, const orc_pconf *pcs, uint64_t 
     *n_done = done;
     return 0;
 }
+
+
+/* ==================================================================================== *
+ * Joint recurrence over the device state (the form printed in Sec. 3.5 / Algorithm 1, with the
+ * min-max objective used throughout this library): DP[j][u][t] = smallest achievable largest
+ * stage cost when the first |u| stages hold the first j layers, u[h] of them run on device type h
+ * and the last one on type t.  It replaces the enumeration of stage-type sequences: the value at
+ * u = (all stages placed), j = N is the minimum over ALL sequences of the per-sequence bottleneck.
+ * Defined for configurations whose stages are homogeneous (G divides every m_h).
+ * ==================================================================================== */
+static int64_t joint_stage_cost(const orc_problem *pr, const orc_pconf *pc, uint32_t rc_mask, const int64_t *c2,
+                                const int64_t *coef, const int32_t *nminT, const int32_t *nmaxT,
+                                int i, int t, int tprev, int q, int a, int b)
+{
+    const int N = pr->N, PP = pc->PP;
+    const int n = b - a;
+    if (n < nminT[t] || n > nmaxT[t]) return ORC_INF;
+    int64_t SF = 0, SB = 0, SW = 0, SA = 0;
+    int has_moe = 0;
+    for (int l = a; l < b; ++l) {
+        SF += c2[((int64_t)t * N + l) * 2];
+        SB += c2[((int64_t)t * N + l) * 2 + 1];
+        SW += coef[ORC_MW + pr->kind[l]];
+        SA += coef[ORC_MA + pr->kind[l]];
+        if (pr->kind[l] == ORC_MOE) has_moe = 1;
+    }
+    const int64_t Mstore = pc->M < PP - i + 1 ? pc->M : PP - i + 1;
+    const int64_t Wb = SW + (i == 1 ? coef[ORC_MPRE] : 0) + (i == PP ? coef[ORC_MPOST] : 0) + (has_moe ? coef[ORC_MX] : 0);
+    const int64_t A = Mstore * SA;
+    int rstar = -1;
+    for (int r = 0; r < pr->R && rstar < 0; ++r)
+        if ((rc_mask >> r) & 1u)
+            if (Wb + ((int64_t)pr->xi_q[r] * A) / 1024 <= pr->cap_eff[t]) rstar = r;
+    if (rstar < 0) return ORC_INF;
+    int64_t K = 0;
+    if (i == 1) K += coef[t * ORC_NCOEF + ORC_KPRE];
+    if (i == PP) K += coef[t * ORC_NCOEF + ORC_KPOST];
+    if (i > 1) {
+        if (tprev != t) K += coef[t * ORC_NCOEF + ORC_KP2P_CROSS + tprev];
+        else {
+            /* q-th stage of its type (0-based): it starts at device q*G of the type's device line */
+            const int64_t first = (int64_t)q * pc->G;
+            const int same_node = (first - 1) / pr->node_size[t] == first / pr->node_size[t];
+            K += coef[t * ORC_NCOEF + (same_node ? ORC_KP2P_INTRA : ORC_KP2P_INTER)];
+        }
+    }
+    return SF + SB + ((int64_t)pr->tau_q[rstar] * SF) / 1024 + K;
+}
+
+/* returns the minimum bottleneck over all stage-type sequences, ORC_INF if none is feasible,
+ * -1 if the configuration's stages are not homogeneous */
+int64_t orc_joint_bottleneck(const orc_problem *pr, const orc_pconf *pc, uint32_t rc_mask,
+                             const int64_t *c2, const int64_t *coef)
+{
+    const int N = pr->N, PP = pc->PP, T = pr->T;
+    int64_t m[ORC_MAX_TYPES];
+    type_counts(pr, m);
+    int cnt[ORC_MAX_TYPES] = {0, 0, 0, 0}, stride[ORC_MAX_TYPES];
+    int S = 1;
+    for (int h = 0; h < T; ++h) {
+        if (m[h] % pc->G != 0) return -1;
+        cnt[h] = (int)(m[h] / pc->G);
+    }
+    for (int h = 0; h < ORC_MAX_TYPES; ++h) { stride[h] = S; S *= (h < T ? cnt[h] : 0) + 1; }
+    /* window per type: every sequence has the same multiset of stages, hence the same total rate */
+    int32_t nminT[ORC_MAX_TYPES], nmaxT[ORC_MAX_TYPES];
+    int64_t Ps = 0;
+    for (int h = 0; h < T; ++h) Ps += (int64_t)cnt[h] * pr->P[h];
+    for (int h = 0; h < T; ++h) {
+        int64_t lo = 1, hi = N - PP + 1;
+        if (pr->delta_q >= 0) {
+            lo = ((int64_t)(1024 - pr->delta_q) * pr->P[h] * N) / (1024 * Ps);
+            int64_t num = (int64_t)(1024 + pr->delta_q) * pr->P[h] * N, den = 1024 * Ps;
+            hi = (num + den - 1) / den;
+            if (lo < 1) lo = 1;
+            if (hi > N - PP + 1) hi = N - PP + 1;
+        }
+        nminT[h] = (int32_t)lo; nmaxT[h] = (int32_t)hi;
+    }
+    const size_t cells = (size_t)S * T * (N + 1);
+    int64_t *D = (int64_t *)malloc(sizeof(int64_t) * cells);
+    if (!D) return -2;
+    for (size_t x = 0; x < cells; ++x) D[x] = ORC_INF;
+#define JAT(ui, t, j) D[((size_t)(ui) * T + (t)) * (N + 1) + (j)]
+    for (int i = 1; i <= PP; ++i)                       /* level = number of stages placed */
+        for (int ui = 0; ui < S; ++ui) {
+            int u[ORC_MAX_TYPES], tot = 0;
+            for (int h = 0; h < ORC_MAX_TYPES; ++h) { u[h] = (ui / stride[h]) % ((h < T ? cnt[h] : 0) + 1); tot += u[h]; }
+            if (tot != i) continue;
+            for (int t = 0; t < T; ++t) {
+                if (u[t] == 0) continue;                  /* the last stage is of type t */
+                const int up = ui - stride[t];
+                for (int j = i; j <= N - PP + i; ++j) {
+                    int64_t best = ORC_INF;
+                    if (i == 1) {
+                        best = joint_stage_cost(pr, pc, rc_mask, c2, coef, nminT, nmaxT, 1, t, -1, 0, 0, j);
+                    } else {
+                        for (int tp = 0; tp < T; ++tp) {
+                            const int utp = (up / stride[tp]) % (cnt[tp] + 1);
+                            if (utp == 0) continue;       /* the prefix cannot end with a type it does not contain */
+                            for (int k = i - 1; k <= j - 1; ++k) {
+                                const int64_t pv = JAT(up, tp, k);
+                                if (pv >= ORC_INF) continue;
+                                const int64_t c = joint_stage_cost(pr, pc, rc_mask, c2, coef, nminT, nmaxT, i, t, tp,
+                                                                   u[t] - 1, k, j);
+                                const int64_t v = pv > c ? pv : c;
+                                if (v < best) best = v;
+                            }
+                        }
+                    }
+                    JAT(ui, t, j) = best;
+                }
+            }
+        }
+    int64_t ans = ORC_INF;
+    for (int t = 0; t < T; ++t)
+        if (cnt[t] > 0 && JAT(S - 1, t, N) < ans) ans = JAT(S - 1, t, N);
+#undef JAT
+    free(D);
+    return ans;
+}

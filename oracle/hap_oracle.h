@@ -133,6 +133,10 @@ int64_t orc_bruteforce_sum(const orc_problem *pr, const orc_pconf *pc, const orc
                            const int64_t *c2, const int64_t *coef, int i, int j, int64_t limit);
 void orc_set_refine(int on);
 
+/* joint recurrence over the device state: minimum bottleneck over all stage-type sequences */
+int64_t orc_joint_bottleneck(const orc_problem *pr, const orc_pconf *pc, uint32_t rc_mask,
+                             const int64_t *c2, const int64_t *coef);
+
 /* fp64 mode (no rounding of times to integer ns); see hap_oracle.c */
 typedef struct {
     double T_iter, bottleneck, T_pipe, T_sync, T_opt;

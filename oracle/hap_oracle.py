@@ -98,6 +98,7 @@ def lib():
         L.orc_stage_cost.restype = C.c_int64
         L.orc_bruteforce.restype = C.c_int64
         L.orc_bruteforce_sum.restype = C.c_int64
+        L.orc_joint_bottleneck.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -298,6 +299,12 @@ class Oracle:
             return self.search_pconfs(p_first, p_stride, threads, want_costs)
         finally:
             self.L.orc_set_refine(C.c_int(0))
+
+    # ---- joint recurrence over the device state ----------------------------------------------
+    def joint_bottleneck(self, p: int, rc_mask: int, c2=None, coef=None) -> int:
+        if c2 is None:
+            c2, _, coef, _ = self.layer_costs(p)
+        return int(self.L.orc_joint_bottleneck(C.byref(self.s), self._pc(p), C.c_uint32(rc_mask), _ptr(c2), _ptr(coef)))
 
     # ---- fp64 mode ---------------------------------------------------------------------
     def candidate_f64(self, p, mp, rc_mask, c2f, coef, coeff) -> ResultF:

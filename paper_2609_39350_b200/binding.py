@@ -17,7 +17,7 @@ STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE",
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
            "hap_search_range", "hap_search_range_f64",
-           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_count_cells", "hap_get_timings", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -117,6 +117,7 @@ class HapProblem:
     def __init__(self, handle: int, pb):
         self.h = C.c_void_p(handle)
         self.N, self.T = int(pb.N), int(pb.P.shape[0])
+        self.n_rc = len(pb.rc_masks)
         self.n_pconf = self.n_cand = None
 
     def check(self, status: int):
@@ -296,6 +297,14 @@ def hap_search_best(hp: HapProblem, stream=None):
     pl, st = _Plan(), _Stats()
     hp.check(load_library().hap_search_best(hp.h, C.byref(pl), C.byref(st), _stream(stream)))
     return _plan_dict(pl), _stats_dict(st)
+
+
+def hap_joint_bottleneck(hp: HapProblem, stream=None):
+    """[n_pconf][n_rc] int64 CUDA tensor: minimum bottleneck over all stage-type sequences (-1: not homogeneous)."""
+    import torch
+    out = torch.empty((hp.n_pconf, hp.n_rc), dtype=torch.int64, device="cuda")
+    hp.check(load_library().hap_joint_bottleneck(hp.h, _dev(out), _stream(stream)))
+    return out
 
 
 def hap_count_cells(hp: HapProblem, first: int, count: int, stream=None) -> int:

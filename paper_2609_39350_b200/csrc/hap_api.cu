@@ -46,6 +46,12 @@ struct hap_problem {
     double *d_c2f = nullptr, *d_coeff = nullptr;   // fp64-mode layer costs and coefficients (allocated on first use)
     i64 *d_fcost = nullptr;                 // fp64-mode search: per-candidate costs (bit patterns), allocated on first use
     u64 *d_range = nullptr;                 // sticky flag: a cost left the supported value range
+    // joint device-state recurrence (built on first use)
+    struct JointHost { JointClass jc; std::vector<unsigned> ids; unsigned *d_ids = nullptr; int *d_arrays = nullptr; size_t smem = 0; };
+    std::vector<JointHost> joint;
+    i64 *d_joint_scratch = nullptr;
+    int joint_grid = 0;
+    bool joint_ready = false;
     i64 *d_lb = nullptr;                    // scratch: per-configuration lower bound on the summed stage time
     TypeConst *d_tc = nullptr;              // scratch: per (configuration, type) constants of the layer-cost kernels
     i64 *d_pcost = nullptr;                // per-block partial minima
@@ -109,6 +115,8 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 static void release_device(hap_problem *p)
 {
     cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
+    cudaFree(p->d_joint_scratch);
+    for (auto &j : p->joint) { cudaFree(j.d_ids); cudaFree(j.d_arrays); }
     cudaFree(p->d_range); cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
@@ -693,6 +701,94 @@ extern "C" hap_status hap_search_range_f64(hap_problem *p, uint64_t first, uint6
     host_out->T_pipe = (int64_t)llrint(v[2]); host_out->T_sync = (int64_t)llrint(v[3]); host_out->T_opt = (int64_t)llrint(v[4]);
     if (host_T_iter) *host_T_iter = v[0];
     if (host_bottleneck) *host_bottleneck = v[1];
+    return HAP_OK;
+}
+
+static hap_status joint_setup(hap_problem *p)
+{
+    if (p->joint_ready) return HAP_OK;
+    const int T = p->T, N = p->model.N;
+    size_t lmax_all = 0;
+    std::vector<int> pps;
+    for (const auto &r : p->pconfs) if (std::find(pps.begin(), pps.end(), r.PP) == pps.end()) pps.push_back(r.PP);
+    for (int PP : pps) {
+        const int64_t G = p->W / PP;
+        bool homog = true;
+        for (int h = 0; h < T; ++h) if (p->m[h] % G) homog = false;
+        if (!homog) continue;
+        hap_problem::JointHost jh;
+        JointClass &jc = jh.jc;
+        jc.PP = PP;
+        int S = 1;
+        for (int h = 0; h < HAP_MAX_TYPES; ++h) {
+            jc.cnt[h] = h < T ? (int)(p->m[h] / G) : 0;
+            jc.stride[h] = S;
+            S *= jc.cnt[h] + 1;
+            if (S > (1 << 22)) return fail(p, HAP_E_RANGE, "too many device states for the joint recurrence");
+        }
+        jc.S = S;
+        std::vector<int> lvl_off(PP + 2, 0), st_idx(S), slot(S), level(S);
+        for (int ui = 0; ui < S; ++ui) {
+            int tot = 0;
+            for (int h = 0; h < HAP_MAX_TYPES; ++h) tot += (ui / jc.stride[h]) % (jc.cnt[h] + 1);
+            level[ui] = tot;
+            lvl_off[tot + 1]++;
+        }
+        int lmax = 1;
+        for (int l = 0; l <= PP; ++l) { lmax = std::max(lmax, lvl_off[l + 1]); lvl_off[l + 1] += lvl_off[l]; }
+        std::vector<int> fill(lvl_off.begin(), lvl_off.end() - 1);
+        for (int ui = 0; ui < S; ++ui) { slot[ui] = fill[level[ui]] - lvl_off[level[ui]]; st_idx[fill[level[ui]]++] = ui; }
+        jc.lmax = lmax;
+        lmax_all = std::max(lmax_all, (size_t)lmax);
+        std::vector<int> arrays;
+        arrays.insert(arrays.end(), lvl_off.begin(), lvl_off.end());
+        arrays.insert(arrays.end(), st_idx.begin(), st_idx.end());
+        arrays.insert(arrays.end(), slot.begin(), slot.end());
+        CUDA_TRY(p, cudaMalloc(&jh.d_arrays, arrays.size() * sizeof(int)));
+        CUDA_TRY(p, cudaMemcpy(jh.d_arrays, arrays.data(), arrays.size() * sizeof(int), cudaMemcpyHostToDevice));
+        jc.lvl_off = jh.d_arrays; jc.st_idx = jh.d_arrays + (PP + 2); jc.slot = jc.st_idx + S;
+        for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == PP) jh.ids.push_back((unsigned)pi);
+        CUDA_TRY(p, cudaMalloc(&jh.d_ids, jh.ids.size() * sizeof(unsigned)));
+        CUDA_TRY(p, cudaMemcpy(jh.d_ids, jh.ids.data(), jh.ids.size() * sizeof(unsigned), cudaMemcpyHostToDevice));
+        jh.smem = joint_smem_bytes(N, PP, T, p->prof.R, p->dc.tau_linear != 0);
+        if (jh.smem > 227 * 1024) return fail(p, HAP_E_RANGE, "shared memory need of the joint recurrence exceeds the SM");
+        p->joint.push_back(jh);
+    }
+    p->joint_grid = 2 * 148;
+    if (lmax_all) {
+        const size_t bytes = (size_t)p->joint_grid * 2 * lmax_all * T * (N + 1) * sizeof(i64);
+        CUDA_TRY(p, cudaMalloc(&p->d_joint_scratch, bytes));
+    }
+    p->joint_ready = true;
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_joint_bottleneck(hap_problem *p, int64_t *dev_out, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if (!dev_out) return HAP_E_INVALID;
+    if ((s = joint_setup(p)) != HAP_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t np = p->pconfs.size();
+    CUDA_TRY(p, cudaMemsetAsync(dev_out, 0xff, np * p->opts.n_rc * sizeof(int64_t), st));     // -1: stages not homogeneous
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    static size_t smem_limit[64][2];
+    const int dev = p->device & 63;
+    const bool lin = p->dc.tau_linear != 0;
+    for (const auto &jh : p->joint) {
+        const void *fn = lin ? (const void *)joint_dp_kernel<true> : (const void *)joint_dp_kernel<false>;
+        if (jh.smem > smem_limit[dev][lin]) {
+            CUDA_TRY(p, cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)jh.smem));
+            smem_limit[dev][lin] = jh.smem;
+        }
+        const unsigned n_ids = (unsigned)jh.ids.size();
+        const unsigned grid = std::min<unsigned>(n_ids, (unsigned)p->joint_grid);
+        // scratch slices are sized for the widest class
+        if (lin) joint_dp_kernel<true><<<grid, 256, jh.smem, st>>>(p->dc, jh.d_ids, n_ids, p->d_c2, p->d_coef, jh.jc, p->d_joint_scratch, (i64 *)dev_out);
+        else joint_dp_kernel<false><<<grid, 256, jh.smem, st>>>(p->dc, jh.d_ids, n_ids, p->d_c2, p->d_coef, jh.jc, p->d_joint_scratch, (i64 *)dev_out);
+        CUDA_TRY(p, cudaGetLastError());
+    }
     return HAP_OK;
 }
 

@@ -1176,6 +1176,137 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
 }
 
 // ------------------------------------------------------------------------------------------
+// joint recurrence over the device state (the DP form printed in Sec. 3.5 / Algorithm 1, min-max objective):
+// value[u][t][j] = smallest achievable largest stage cost when the first |u| stages hold the first j layers,
+// u[h] of them on device type h, the last one on type t.  One block per configuration; the states of one
+// level (= number of stages placed) are spread over the block's warps, lanes run over j; two levels of rows
+// live in a per-block slice of a global scratch buffer.  The result for u = "all stages placed", j = N is the
+// minimum, over every stage-type sequence, of the bottleneck the per-candidate kernel computes.
+// ------------------------------------------------------------------------------------------
+struct JointClass {
+    int PP, S, lmax;              // stages; number of states; most states of one level
+    int cnt[HAP_MAX_TYPES];       // stages of each type
+    int stride[HAP_MAX_TYPES];    // mixed-radix strides of the state index
+    const int *lvl_off;           // [PP+2] offsets of each level in st_idx
+    const int *st_idx;            // [S] state indices ordered by level
+    const int *slot;              // [S] rank of a state within its level
+};
+
+__host__ __device__ inline size_t joint_smem_bytes(int N, int PP, int T, int R, bool linear)
+{
+    const size_t n1 = (size_t)N + 1;
+    size_t b = (size_t)T * (linear ? (size_t)R : 2) * n1 * 8 + n1 * 16;
+    b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    b += (n1 + 15) / 16 * 16;
+    return b + 32;
+}
+
+template <bool LINEAR>
+__global__ void __launch_bounds__(256)
+joint_dp_kernel(const DevConst dc, const unsigned *pconf_ids, unsigned n_ids, const i64 *c2, const i64 *coef,
+                JointClass jc, i64 *scratch, i64 *out)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    typedef i64 VT;
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, n_rc = dc.n_rc;
+    const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int PP = jc.PP;
+    const int RW = LINEAR ? R : 2;
+    VT *sR = reinterpret_cast<VT *>(smem_raw);
+    i64 *sW = reinterpret_cast<i64 *>(sR + (size_t)T * RW * n1);
+    i64 *sA = sW + n1;
+    uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
+    uint8_t *sK = thr + ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    __shared__ MaskInfo<VT> minfo[kMaxMasks];
+    __shared__ VT sP2P[HAP_MAX_TYPES][6];
+    __shared__ VT szero[1];
+    __shared__ int winT[HAP_MAX_TYPES][2];
+    const size_t lvl_cells = (size_t)jc.lmax * T * n1;
+    i64 *buf0 = scratch + (size_t)blockIdx.x * 2 * lvl_cells, *buf1 = buf0 + lvl_cells;
+
+    for (unsigned w = blockIdx.x; w < n_ids; w += gridDim.x) {
+        const unsigned p = pconf_ids[w];
+        const hap_pconf pc = dc.pconf[p];
+        __syncthreads();                                  // the previous configuration's tables are no longer read
+        dp_block_prologue<VT, LINEAR>(dc, pc, p, c2, coef, coef, true, T, RW, 0xffffffffu, nwarps,
+                                      sR, sW, sA, thr, sK, minfo, sP2P, szero, winT);
+        for (int rc_idx = 0; rc_idx < n_rc; ++rc_idx) {
+            const unsigned rc_mask = dc.rc_masks[rc_idx];
+            for (int i = 1; i <= PP; ++i) {
+                i64 *cur = (i & 1) ? buf1 : buf0;
+                const i64 *prv = (i & 1) ? buf0 : buf1;
+                const int l0 = jc.lvl_off[i], l1 = jc.lvl_off[i + 1];
+                const int jlo = i, jhi = N - PP + i;
+                for (int pr = wib; pr < (l1 - l0) * T; pr += nwarps) {
+                    const int sl = pr / T, t = pr - sl * T;
+                    const int ui = jc.st_idx[l0 + sl];
+                    const int ut = (ui / jc.stride[t]) % (jc.cnt[t] + 1);
+                    i64 *row = cur + ((size_t)sl * T + t) * n1;
+                    if (ut == 0) continue;                  // no stage of type t placed: rows of such pairs are never read
+                    const int up = ui - jc.stride[t];
+                    const int slot_up = i > 1 ? jc.slot[up] : 0;
+                    const int nmin = winT[t][0], nmax = winT[t][1];
+                    const uint8_t *th = thr + ((size_t)(i - 1) * T + t) * R * n1;
+                    const VT *rM = sR + (size_t)t * RW * n1;
+                    const MaskInfo<VT> &mi = minfo[(1 << t) - 1];
+                    const VT Kbase = (i == 1 ? mi.kpre : 0) + (i == PP ? mi.kpost : 0);
+                    // the q-th stage of its type starts at device q*G of the type's device line
+                    const i64 first = (i64)(ut - 1) * pc.G;
+                    const int same_cls = ((first - 1) / dc.node_size[t] == first / dc.node_size[t]) ? HAP_INTRA : HAP_INTER;
+                    for (int j = lane; j <= N; j += 32) {
+                        VT best = kInf;
+                        if (j >= jlo && j <= jhi) {
+                            int klo = j - nmax; if (klo < i - 1) klo = i - 1;
+                            int khi = j - nmin; if (khi > jhi - 1) khi = jhi - 1;
+                            const int ntp = i == 1 ? 1 : T;
+                            for (int tp = 0; tp < ntp; ++tp) {
+                                const VT *prow = szero;
+                                VT K = Kbase;
+                                int kl = klo, kh = khi;
+                                if (i > 1) {
+                                    const int utp = (up / jc.stride[tp]) % (jc.cnt[tp] + 1);
+                                    if (utp == 0) continue;     // the prefix does not contain type tp
+                                    prow = prv + ((size_t)slot_up * T + tp) * n1;
+                                    K += tp != t ? sP2P[t][2 + tp] : sP2P[t][same_cls];
+                                } else {
+                                    kh = kh < 0 ? kh : 0;       // the first stage starts at layer 0
+                                }
+                                int seg_hi = kh;
+                                for (int r = 0; r < R && seg_hi >= kl; ++r) {
+                                    if (!((rc_mask >> r) & 1u)) continue;
+                                    int lo = th[(size_t)r * n1 + j];
+                                    if (lo < kl) lo = kl;
+                                    if (lo > seg_hi) continue;
+                                    for (int k = seg_hi; k >= lo; --k) {
+                                        VT cst;
+                                        if (LINEAR) cst = (rM[(size_t)r * n1 + j] - rM[(size_t)r * n1 + k]) + K;
+                                        else cst = ((rM[j] - rM[k]) + tau_term((i64)dc.tau_q[r], rM[n1 + j] - rM[n1 + k])) + K;
+                                        const VT pv = prow[k];
+                                        const VT v = pv > cst ? pv : cst;
+                                        best = v < best ? v : best;
+                                    }
+                                    seg_hi = lo - 1;
+                                }
+                            }
+                        }
+                        row[j] = best;
+                    }
+                }
+                __syncthreads();
+            }
+            if (threadIdx.x == 0) {
+                const i64 *fin = (PP & 1) ? buf1 : buf0;      // level PP has the single state "everything placed"
+                VT b = kInf;
+                for (int t = 0; t < T; ++t)
+                    if (jc.cnt[t] > 0) { const VT v = fin[(size_t)t * n1 + N]; b = v < b ? v : b; }
+                out[(size_t)p * n_rc + rc_idx] = b;
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // argmin: stage 1 reduces a slice per block, stage 2 (one block) reduces the partials
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)

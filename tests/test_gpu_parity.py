@@ -353,3 +353,40 @@ def test_refinement_on_random_problems_with_general_levels(hap, seed):
     plan, _ = hap.hap_search_best(hp)
     assert (plan["T_iter"], plan["index"]) == (bc, bi)
     hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}), ("stress", {})])
+def test_joint_device_state_recurrence(hap, name, kw):
+    """hap_joint_bottleneck: equal to the oracle's joint recurrence on sampled configurations; equal to the minimum
+    of the per-candidate bottlenecks wherever all sequences are enumerated; never above it for block orderings."""
+    pb, hp, o = setup(hap, name, **kw)
+    n_rc = len(pb.rc_masks)
+    jb = hap.hap_joint_bottleneck(hp).cpu().numpy()
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    bn = out["bottleneck"].cpu().numpy()
+    m = [0] * pb.T
+    for t in pb.node_type:
+        m[t] += int(pb.node_size[t])
+    n_multiset = n_block_homog = 0
+    for p in range(o.n_pconf):
+        off, nmap, mode, G = (int(o.pconfs[f][p]) for f in ("offset", "nmap", "mode", "G"))
+        homog = all(x % G == 0 for x in m)
+        for rc in range(n_rc):
+            enumerated = bn[off + rc: off + nmap * n_rc: n_rc].min()
+            if not homog:
+                assert jb[p, rc] == -1
+            elif mode == 0:
+                assert jb[p, rc] == enumerated, (p, rc)
+                n_multiset += 1
+            else:
+                assert jb[p, rc] <= enumerated, (p, rc)       # block orderings are a subset of all sequences
+                n_block_homog += 1
+    assert n_multiset > 0
+    if name == "stress":
+        assert n_block_homog > 0
+    rng = np.random.default_rng(1)
+    small_pp = [p for p in range(o.n_pconf) if int(o.pconfs["PP"][p]) <= (8 if pb.N <= 32 else 4)]
+    for p in rng.choice(small_pp, size=min(12, len(small_pp)), replace=False):
+        for rc in range(n_rc):
+            assert jb[p, rc] == o.joint_bottleneck(int(p), int(pb.rc_masks[rc])), (p, rc)

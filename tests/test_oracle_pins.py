@@ -679,3 +679,36 @@ def test_refinement_changes_some_partitions_and_never_raises_the_pipeline_time()
         plain, _, _ = o.eval_index(int(i))
         ref = o.eval_index_refined(int(i))
         assert ref["T_pipe"] <= plain["T_pipe"] and ref["n"] != plain["n"]
+
+
+# --------------------------------------------------------------------------------------
+# joint recurrence over the device state (Sec. 3.5 / Algorithm 1 form)
+# --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("make", [lambda: problems.tiny(), lambda: problems.tiny(window=True),
+                                  lambda: problems.small().copy(map_cap=1 << 40, mb_list=np.array([4], np.int32)),
+                                  lambda: problems.random_small(3, N=9, T=3, nodes_per_type=(2, 1, 1), node_size=2, window=True)])
+def test_joint_device_state_recurrence_equals_minimum_over_enumerated_sequences(make):
+    """One DP over (layers placed, stages of each type used, last type) must return the minimum, over every
+    stage-type sequence, of the per-sequence bottleneck that the enumeration + per-candidate DP gives."""
+    pb = make()
+    if pb.name == "small":
+        for f in ("tdf", "tdb", "tff", "tfb", "tpre", "tpost"):
+            setattr(pb, f, np.ascontiguousarray(np.take(getattr(pb, f), [2], axis=3)))
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=4, want_costs=True)
+    n_rc = len(pb.rc_masks)
+    checked = 0
+    for p in range(o.n_pconf):
+        off, nmap, mode = int(o.pconfs["offset"][p]), int(o.pconfs["nmap"][p]), int(o.pconfs["mode"][p])
+        c2, _, coef, _ = o.layer_costs(p)
+        for rc in range(n_rc):
+            jb = o.joint_bottleneck(p, int(pb.rc_masks[rc]), c2, coef)
+            if mode == 0:
+                assert jb == bn[off + rc: off + nmap * n_rc: n_rc].min(), (p, rc)
+                checked += 1
+            else:
+                G, m = int(o.pconfs["G"][p]), [0] * pb.T
+                for t in pb.node_type:
+                    m[t] += int(pb.node_size[t])
+                assert (jb == -1) == any(x % G for x in m)
+    assert checked > 20
