@@ -32,7 +32,6 @@ struct hap_problem {
     bool enumerated = false;
     std::vector<hap_pconf> pconfs;
     uint64_t n_cand = 0;
-    int pp_max = 1;
     std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
     struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; };
     std::vector<PpClass> classes;
@@ -292,13 +291,6 @@ static uint64_t sequences_sat(const int *cnt, int T, uint64_t sat)
     return (uint64_t)r;
 }
 
-[[maybe_unused]] static double cells_per_candidate(int N, int PP)
-{
-    if (PP == 1) return 1.0;
-    const double w = N - PP + 1;
-    return 2.0 * w + (PP - 2) * w * (w + 1) / 2.0;
-}
-
 extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t *n_candidates)
 {
     if (!p) return HAP_E_INVALID;
@@ -308,7 +300,6 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         const int N = mo.N, T = p->T;
         std::vector<hap_pconf> rows;
         uint64_t off = 0;
-        int pp_max = 1;
         const uint64_t SAT = 1ull << 62;
         for (int PP : p->pp_list) {
             if (PP > N || PP > HAP_MAX_PP || p->W % PP) continue;
@@ -345,7 +336,6 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                                 if (nmap > (SAT - off) / (uint64_t)p->opts.n_rc) return fail(p, HAP_E_RANGE, "candidate space overflows 2^62");
                                 off += nmap * (uint64_t)p->opts.n_rc;
                                 rows.push_back(q);
-                                pp_max = std::max(pp_max, PP);
                             }
                         }
                     }
@@ -410,7 +400,6 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         p->items.swap(items);
         p->classes.swap(classes);
         p->n_cand = off;
-        p->pp_max = pp_max;
         const size_t np = p->pconfs.size();
         CUDA_TRY(p, cudaMalloc(&p->d_pconf, np * sizeof(hap_pconf)));
         CUDA_TRY(p, cudaMemcpy(p->d_pconf, p->pconfs.data(), np * sizeof(hap_pconf), cudaMemcpyHostToDevice));
@@ -858,7 +847,7 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     DpOut out{};
     out.lb_sum = p->d_lb;
-    out.first = first; out.count = count; out.search = 1; out.prune = p->opts.prune;
+    out.first = first; out.count = count; out.prune = p->opts.prune;
     out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
     out.incumbent = p->d_counters + 3;
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;

@@ -1,14 +1,21 @@
 // Device-side data layout and kernels of libhap (sm_100a).
 //
 // Kernels
-//   layer_cost_kernel   Eq. 2 / Eq. 3 / imbalance scaling and the stage coefficients, one warp
-//                       per configuration, fp64 with one IEEE operation per operator
-//                       (the translation unit is compiled with --fmad=false).
-//   decode_kernel       candidate index -> stage type masks and boundary link classes.
-//   pipeline_dp_kernel  one warp per candidate: stage rows in shared memory (built once per
-//                       block for the block's configuration), min-max recurrence with lanes
-//                       over the end layer j, backtrace, Eq. 4 closed form; optionally the
-//                       block-level (cost, index) minimum for the search.
+//   type_const_kernel   per (configuration, type): constants of Eq. 2 / Eq. 3 and the 20 stage
+//                       coefficients, fp64 with one IEEE operation per operator (the translation
+//                       unit is compiled with --fmad=false), three independent roles per pair.
+//   layer_cost_kernel   per (configuration, type, layer): Eq. 2 with imbalance scaling, rounding,
+//                       one block per configuration, one thread per layer.
+//   decode_kernel       candidate index -> stage type masks and boundary link classes;
+//   maptab_kernel       the same for every mapping of one PP class, once per problem.
+//   pipeline_dp_kernel  one warp per candidate: stage rows and memory-threshold tables in shared
+//                       memory (built once per block for the block's configuration), min-max
+//                       recurrence with lanes over the end layer j, optional refinement pass,
+//                       backtrace, Eq. 4 closed form, Pruning 3; in search mode the block-level
+//                       (cost, index) minimum and lower-bound pruning against an atomic incumbent.
+//                       Instantiated on int64 (exact) and double (fp64 mode).
+//   joint_dp_kernel     recurrence over the device-group state: minimum bottleneck over all
+//                       stage-type sequences of a configuration.
 //   argmin kernels      lexicographic (cost, index) minimum, block partials then one block.
 #pragma once
 #include <cuda_runtime.h>
@@ -66,7 +73,7 @@ struct DpOut {
     u64 *counters;                    // [0] evaluated, [1] feasible, [2] pruned, [4] recurrence cells (nullable)
     u64 *incumbent;                   // running minimum of T_iter, for pruning
     const i64 *lb_sum;                // per configuration: sum over layers of the cheapest type's time
-    int search, prune;
+    int prune;                        // search mode: skip blocks whose lower bound exceeds the incumbent
     int count_only;                   // instrumentation: count the finite-cost cells of each candidate, run no recurrence
 };
 
@@ -898,8 +905,6 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                 }
             }
         }
-        const bool dead_prefix = false;                  // (handled above, before the stage parameters)
-
         // ---- bands: end layers j that stage i can reach (prefix sums of the window bounds), and from
         //      which the remaining stages can still reach N (suffix sums; not applied when the caller
         //      wants the full tables, where such cells hold finite values)
@@ -954,9 +959,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             }
         }
         VT bott = vInf;
-        if (dead_prefix) {
-            valid_rows = s0;                                // rows up to the dead one stay as they are
-        } else if (!dead || want_tables) {
+        if (!dead || want_tables) {
             int pbl = 0, pbh = 0;                          // band of the previous stage (stage 0: {0})
             int last_stage = PP;
             if (s0 > 0) { pbl = __shfl_sync(0xffffffffu, sp.bl, s0 - 1); pbh = __shfl_sync(0xffffffffu, sp.bh, s0 - 1); }
