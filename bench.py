@@ -148,6 +148,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--delta-q", type=int, default=None, help="override the load-balance window (1/1024; <0 = off)")
+    ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
+                    help="torch.distributed backend of the (cost, index) exchange when launched with several ranks")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -164,9 +166,14 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    local_rank %= torch.cuda.device_count()
     torch.cuda.set_device(local_rank)
     if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if args.backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        else:
+            dist.init_process_group("gloo")
+    xdev = "cuda" if args.backend == "nccl" else "cpu"
     warmup = max(args.warmup, 3)
 
     pb = problems.make_problem(args.workload)
@@ -209,7 +216,7 @@ def main():
         am = step()
         if world > 1:
             c, i = (int(x) for x in am.tolist())
-            best = exchange_minimum(c, i + first, device="cuda")
+            best = exchange_minimum(c, i + first, device=xdev)
         b.record(stream)
         b.synchronize()
         lc, dpk, cells = hap.hap_get_timings(hp)
@@ -222,7 +229,7 @@ def main():
         best = (c, i + first)
 
     step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device="cuda")
+    total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device=xdev)
     if world > 1:
         dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)
     total_ms = float(total_ms.item())
@@ -292,7 +299,7 @@ def main():
         plan2, _ = hap.hap_search_range(hp2, first, count)
         e2e_ms.append(1e3 * (time.perf_counter() - t0))
         hap.hap_problem_destroy(hp2)
-    e2e_t = torch.tensor([statistics.median(e2e_ms)], dtype=torch.float64, device="cuda")
+    e2e_t = torch.tensor([statistics.median(e2e_ms)], dtype=torch.float64, device=xdev)
     if world > 1:
         dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
     e2e_value = n_cand / (float(e2e_t.item()) * 1e-3)
