@@ -250,22 +250,26 @@ def main():
         b.synchronize()
         joint_ms = a.elapsed_time(b)
 
-    # the same pass with the refinement (smallest stage-cost sum among the bottleneck-optimal partitions)
-    hp_ref = hap.hap_problem_create(pb, flags=hap.OPT_REFINE)
-    hap.hap_enumerate(hp_ref)
-    ref_ms = []
-    for it in range(5):
-        flush.fill_(1)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        hap.hap_pipeline_dp(hp_ref, first, count, out=out)
-        am_ref = hap.hap_argmin(hp_ref, out["cost"][:count])
-        b.record(stream)
-        b.synchronize()
-        if it >= 2:
-            ref_ms.append(a.elapsed_time(b))
-    ref_best = [int(x) for x in am_ref.tolist()]
-    hap.hap_problem_destroy(hp_ref)
+    # the same pass with the refinement (smallest stage-cost sum among the bottleneck-optimal partitions) and with
+    # the exact optimisation of sum + (M-1) max (limit sweep); untimed extras
+    extra_modes = {}
+    for mode_name, flag in (("refined_pass", hap.OPT_REFINE), ("exact_pass", hap.OPT_EXACT)):
+        hp_ref = hap.hap_problem_create(pb, flags=flag)
+        hap.hap_enumerate(hp_ref)
+        ref_ms = []
+        for it in range(5):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            hap.hap_pipeline_dp(hp_ref, first, count, out=out)
+            am_ref = hap.hap_argmin(hp_ref, out["cost"][:count])
+            b.record(stream)
+            b.synchronize()
+            if it >= 2:
+                ref_ms.append(a.elapsed_time(b))
+        ref_best = [int(x) for x in am_ref.tolist()]
+        extra_modes[mode_name] = dict(ms=statistics.median(ref_ms), best_cost=ref_best[0], best_index=ref_best[1] + first)
+        hap.hap_problem_destroy(hp_ref)
 
     # full search through the search entry point (pruning allowed), wall clock call to return
     search_ms, pruned_ms = [], []
@@ -327,7 +331,7 @@ def main():
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                      ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
             gpu_launches=(4 + len(set(int(x) for x in pconfs["PP"]))) * args.steps,
-            refined_pass=dict(ms=statistics.median(ref_ms), best_cost=ref_best[0], best_index=ref_best[1] + first),
+            **extra_modes,
             joint_recurrence_ms=joint_ms,
             full_search_ms=statistics.median(search_ms),
             full_search_pruned=dict(ms=statistics.median(pruned_ms), n_pruned=stats_pr["n_pruned"],

@@ -130,6 +130,10 @@ typedef struct {
 
 /* hap_search_opts.flags */
 #define HAP_OPT_NO_MAPTAB 1   /* keep no table of decoded mappings on the device: the DP kernel unranks each mapping itself */
+#define HAP_OPT_EXACT 4       /* like HAP_OPT_REFINE, but the limit on the stage cost is then swept upward from the bottleneck over
+                                 the stage costs, which yields the partition that minimises sum_i c_i + (M-1) max_i c_i (Eq. 4's
+                                 pipeline term in closed form) over ALL partitions of the candidate; integer mode only.  The
+                                 reported bottleneck stays that of the min-max recurrence. */
 #define HAP_OPT_REFINE 2      /* after the min-max recurrence, choose among the bottleneck-optimal partitions the one with
                                  the smallest sum of stage costs (Eq. 4's T_edge), smallest split on ties; integer mode only.
                                  Costs, partitions, levels and the plan then refer to that partition; the DP tables

@@ -663,6 +663,143 @@ int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_
     return 0;
 }
 
+/* ------------------------------------------------------------------------------------ *
+ * Exact optimum of the pipeline term sum_i c_i + (M-1) max_i c_i (Eq. 4 in its closed form) over the
+ * partitions of one candidate.  For a limit t on the stage cost let f(t) be the smallest stage-cost sum
+ * among partitions whose stages all cost at most t (additive recurrence, smallest split on ties).  The
+ * optimum is reached at a limit that equals some stage cost, so the limits are swept upward from the
+ * bottleneck B*: every pass reports the smallest stage cost it had to skip, which is the next limit.
+ * With f_min = f(infinity), a partition whose largest stage costs t cannot beat the incumbent V once
+ * f_min + (M-1) t >= V, which ends the sweep.  The first limit reaching the smallest value wins.
+ * ------------------------------------------------------------------------------------ */
+typedef struct { int64_t sum, mx, next; int ok; uint8_t k[ORC_MAX_PP + 1]; } add_pass;
+
+static void additive_pass(const stage_ctx *cx, int64_t limit, int64_t *D, uint8_t *CH, add_pass *out)
+{
+    const int N = cx->N, PP = cx->PP;
+#define DAT(i, j) D[(size_t)(i) * (N + 1) + (j)]
+#define CHAT(i, j) CH[(size_t)(i) * (N + 1) + (j)]
+    for (int i = 0; i <= PP; ++i)
+        for (int j = 0; j <= N; ++j) { DAT(i, j) = ORC_INF; CHAT(i, j) = 255; }
+    DAT(0, 0) = 0;
+    out->next = ORC_INF;
+    for (int i = 1; i <= PP; ++i)
+        for (int j = i; j <= N - PP + i; ++j)
+            for (int k = i - 1; k <= j - 1; ++k) {
+                int64_t c = ctx_stage_cost(cx, i, k, j, NULL);
+                if (c >= ORC_INF) continue;
+                if (c > limit) { if (c < out->next) out->next = c; continue; }   /* smallest skipped cost */
+                if (DAT(i - 1, k) >= ORC_INF) continue;
+                int64_t v = DAT(i - 1, k) + c;
+                if (v < DAT(i, j)) { DAT(i, j) = v; CHAT(i, j) = (uint8_t)k; }
+            }
+    out->ok = DAT(PP, N) < ORC_INF;
+    out->sum = DAT(PP, N);
+    out->mx = 0;
+    if (out->ok) {
+        int j = N;
+        out->k[PP] = (uint8_t)N;
+        for (int i = PP; i >= 1; --i) {
+            int k = CHAT(i, j);
+            int64_t c = ctx_stage_cost(cx, i, k, j, NULL);
+            if (c > out->mx) out->mx = c;
+            out->k[i - 1] = (uint8_t)k;
+            j = k;
+        }
+    }
+#undef DAT
+#undef CHAT
+}
+
+int orc_candidate_exact(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                        const int64_t *c2, const int64_t *coef, orc_result *res, int64_t *n_passes)
+{
+    const int N = pr->N, PP = pc->PP;
+    orc_result first;
+    int rc0 = orc_candidate(pr, pc, mp, rc_mask, c2, coef, &first, NULL, NULL);
+    if (n_passes) *n_passes = 0;
+    if (rc0 != 0) { *res = first; return rc0; }
+    const int64_t Bstar = first.bottleneck, M1 = pc->M - 1;
+    stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+    int64_t *D = (int64_t *)malloc(sizeof(int64_t) * (size_t)(PP + 1) * (N + 1));
+    uint8_t *CH = (uint8_t *)malloc((size_t)(PP + 1) * (N + 1));
+    if (!D || !CH || !cx) { free(D); free(CH); free(cx); return -1; }
+    ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+    add_pass best, cur, unl;
+    int64_t passes = 2;
+    additive_pass(cx, Bstar, D, CH, &best);                 /* limit B*: the refinement */
+    additive_pass(cx, ORC_INF - 1, D, CH, &unl);            /* no limit: f_min */
+    int64_t Vbest = best.sum + M1 * best.mx;
+    const int64_t fmin = unl.sum;
+    int64_t t = best.next;
+    while (t < ORC_INF && fmin + M1 * t < Vbest) {
+        additive_pass(cx, t, D, CH, &cur);
+        passes++;
+        if (cur.ok && cur.sum + M1 * cur.mx < Vbest) { best = cur; Vbest = cur.sum + M1 * cur.mx; }
+        t = cur.next;
+    }
+    if (unl.sum + M1 * unl.mx < Vbest) { best = unl; Vbest = unl.sum + M1 * unl.mx; }
+    if (n_passes) *n_passes = passes;
+    /* objective on the chosen partition */
+    memset(res, 0, sizeof(*res));
+    res->bottleneck = Bstar;
+    int64_t sum = 0, mx = 0, tsync = 0, topt = 0;
+    for (int i = 1; i <= PP; ++i) {
+        int k = best.k[i - 1], j = best.k[i], r;
+        int64_t c = ctx_stage_cost(cx, i, k, j, &r);
+        res->n[i - 1] = (uint8_t)(j - k);
+        res->r[i - 1] = (uint8_t)r;
+        res->c[i - 1] = c;
+        sum += c;
+        if (c > mx) mx = c;
+        unsigned mask = mp->mask[i - 1];
+        int64_t sy = mask_max(pr, mask, coef, ORC_SLAT), op = 0;
+        for (int l = k; l < j; ++l) {
+            sy += mask_max(pr, mask, coef, ORC_SBW + pr->kind[l]);
+            op += mask_max(pr, mask, coef, ORC_OPT + pr->kind[l]);
+        }
+        if (sy > tsync) tsync = sy;
+        if (op > topt) topt = op;
+    }
+    res->T_pipe = sum + M1 * mx;
+    res->T_sync = tsync;
+    res->T_opt = topt;
+    res->T_iter = res->T_pipe + tsync + topt;
+    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum)) res->T_iter = res->T_pipe = ORC_INF;
+    free(D); free(CH); free(cx);
+    return 0;
+}
+
+/* Exhaustive minimum of sum + (M-1) max over every contiguous partition (no recurrence, no memo). */
+static void bf_pipe_rec(const stage_ctx *cx, int stage, int nstages, int start, int end, int64_t M1,
+                        int64_t cur_sum, int64_t cur_max, int64_t *best)
+{
+    if (stage == nstages) {
+        int64_t c = ctx_stage_cost(cx, stage, start, end, NULL);
+        if (c >= ORC_INF) return;
+        int64_t mx = c > cur_max ? c : cur_max, v = cur_sum + c + M1 * mx;
+        if (v < *best) *best = v;
+        return;
+    }
+    for (int cut = start + 1; cut <= end - (nstages - stage); ++cut) {
+        int64_t c = ctx_stage_cost(cx, stage, start, cut, NULL);
+        if (c >= ORC_INF) continue;
+        bf_pipe_rec(cx, stage + 1, nstages, cut, end, M1, cur_sum + c, c > cur_max ? c : cur_max, best);
+    }
+}
+
+int64_t orc_bruteforce_pipe(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                            const int64_t *c2, const int64_t *coef)
+{
+    int64_t best = ORC_INF;
+    stage_ctx *cx = (stage_ctx *)malloc(sizeof(stage_ctx));
+    if (!cx) return -1;
+    ctx_build(cx, pr, pc, mp, rc_mask, c2, coef);
+    bf_pipe_rec(cx, 1, pc->PP, 0, pr->N, pc->M - 1, 0, 0, &best);
+    free(cx);
+    return best;
+}
+
 /* Exhaustive check of the refinement: smallest sum of stage costs over every contiguous partition of
  * layers 1..j into stages 1..i whose stages all cost at most `limit` (no recurrence, no memo). */
 static void bf_sum_rec(const stage_ctx *cx, int stage, int nstages, int start, int end, int64_t limit,
@@ -808,7 +945,7 @@ int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, ui
 /* Timing harness: evaluates every candidate of configurations p_first, p_first+stride, ...
  * (threads > 1 spreads configurations over OpenMP threads; the per-candidate work is the
  * plain code above).  Returns the (cost, index) minimum over what it evaluated. */
-static int g_refine = 0;    /* evaluation mode of the whole-space harnesses below: 0 plain, 1 refined */
+static int g_refine = 0;    /* evaluation mode of the whole-space harnesses below: 0 plain, 1 refined, 2 exact pipeline term */
 void orc_set_refine(int on) { g_refine = on; }
 
 int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
@@ -833,7 +970,8 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
             orc_decode(pr, pc, map_idx, &mp);
             for (int rc = 0; rc < pr->n_rc; ++rc) {
                 orc_result res;
-                if (g_refine) orc_candidate_refined(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res);
+                if (g_refine == 2) orc_candidate_exact(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL);
+                else if (g_refine) orc_candidate_refined(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res);
                 else orc_candidate(pr, pc, &mp, pr->rc_masks[rc], c2, coef, &res, NULL, NULL);
                 uint64_t idx = pc->offset + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
                 if (costs) costs[idx] = res.T_iter;              /* indexed by candidate, whole space */

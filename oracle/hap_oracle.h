@@ -132,6 +132,11 @@ int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_
 int64_t orc_bruteforce_sum(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
                            const int64_t *c2, const int64_t *coef, int i, int j, int64_t limit);
 void orc_set_refine(int on);
+/* exact optimum of sum + (M-1) max over the partitions of a candidate */
+int orc_candidate_exact(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                        const int64_t *c2, const int64_t *coef, orc_result *res, int64_t *n_passes);
+int64_t orc_bruteforce_pipe(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,
+                            const int64_t *c2, const int64_t *coef);
 
 /* joint recurrence over the device state: minimum bottleneck over all stage-type sequences */
 int64_t orc_joint_bottleneck(const orc_problem *pr, const orc_pconf *pc, uint32_t rc_mask,

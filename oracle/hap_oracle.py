@@ -99,6 +99,7 @@ def lib():
         L.orc_bruteforce.restype = C.c_int64
         L.orc_bruteforce_sum.restype = C.c_int64
         L.orc_joint_bottleneck.restype = C.c_int64
+        L.orc_bruteforce_pipe.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -295,6 +296,31 @@ class Oracle:
 
     def search_pconfs_refined(self, p_first: int = 0, p_stride: int = 1, threads: int = 1, want_costs: bool = True):
         self.L.orc_set_refine(C.c_int(1))
+        try:
+            return self.search_pconfs(p_first, p_stride, threads, want_costs)
+        finally:
+            self.L.orc_set_refine(C.c_int(0))
+
+    # ---- exact optimum of the pipeline term -----------------------------------------------------
+    def eval_index_exact(self, index: int) -> dict:
+        p = self.find_pconf(index)
+        n_rc = len(self.pb.rc_masks)
+        local = index - int(self.pconfs["offset"][p])
+        mp = self.decode(p, local // n_rc)
+        rc = int(self.pb.rc_masks[local % n_rc])
+        c2, _, coef, _ = self.layer_costs(p)
+        res, passes = Result(), C.c_int64()
+        self.L.orc_candidate_exact(C.byref(self.s), self._pc(p), C.byref(mp), C.c_uint32(rc), _ptr(c2), _ptr(coef),
+                                   C.byref(res), C.byref(passes))
+        PP = int(self.pconfs["PP"][p])
+        brute = int(self.L.orc_bruteforce_pipe(C.byref(self.s), self._pc(p), C.byref(mp), C.c_uint32(rc), _ptr(c2), _ptr(coef)))
+        return dict(T_iter=int(res.T_iter), bottleneck=int(res.bottleneck), T_pipe=int(res.T_pipe), T_sync=int(res.T_sync),
+                    T_opt=int(res.T_opt), n=[int(x) for x in res.n[:PP]], r=[int(x) for x in res.r[:PP]],
+                    c=[int(x) for x in res.c[:PP]], PP=PP, M=int(self.pconfs["M"][p]), passes=int(passes.value),
+                    brute_pipe=brute)
+
+    def search_pconfs_exact(self, p_first: int = 0, p_stride: int = 1, threads: int = 1, want_costs: bool = True):
+        self.L.orc_set_refine(C.c_int(2))
         try:
             return self.search_pconfs(p_first, p_stride, threads, want_costs)
         finally:

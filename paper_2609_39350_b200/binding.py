@@ -139,6 +139,7 @@ class HapProblem:
 
 OPT_NO_MAPTAB = 1
 OPT_REFINE = 2
+OPT_EXACT = 4
 
 
 def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:

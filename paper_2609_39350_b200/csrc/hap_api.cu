@@ -368,7 +368,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             for (int w : {12, 8, 6, 4, 2, 1}) {
                 if ((uint64_t)w * 8 > per_pconf && w > 2) continue;             // keep about 8 candidates per warp
                 const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0,
-                                                (p->opts.flags & HAP_OPT_REFINE) != 0);
+                                                (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0);
                 if (sm > 227 * 1024) continue;
                 const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), std::min(32, 64 / w));
                 const int resident = std::min(per_sm * w, 24);           // registers allow about 24 warps per SM
@@ -554,7 +554,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const bool outside = c1 <= out.first || c0 >= out.first + out.count;
         if (outside && !search) continue;
         const bool lin = p->dc.tau_linear != 0;
-        const bool refine = (p->opts.flags & HAP_OPT_REFINE) != 0 && !out.count_only;
+        const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
         const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (refine ? 8 : 0) + (search ? 2 : 0) + (lin ? 1 : 0);
         const void *fn;
         if (f64) fn = lin ? (const void *)pipeline_dp_kernel<false, true, false, double> : (const void *)pipeline_dp_kernel<false, false, false, double>;
@@ -570,6 +570,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const unsigned blocks = (unsigned)(cl.item_hi - cl.item_lo);
         const uint8_t *tab = cl.has_tab ? p->d_maptab + cl.map_base : nullptr;
         DpOut o = out;
+        o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0;
         if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
         const WorkItem *its = p->d_items + cl.item_lo;
         int nw = cl.warps;
@@ -625,7 +626,7 @@ extern "C" hap_status hap_pipeline_dp_f64(hap_problem *p, uint64_t first, uint64
     if (s != HAP_OK) return s;
     if ((s = check_range(p, first, count)) != HAP_OK) return s;
     if (count == 0) return HAP_OK;
-    if (p->opts.flags & HAP_OPT_REFINE) return fail(p, HAP_E_INVALID, "the refinement pass exists in integer mode only");
+    if (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) return fail(p, HAP_E_INVALID, "the refinement passes exist in integer mode only");
     if ((s = ensure_f64_buffers(p)) != HAP_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));

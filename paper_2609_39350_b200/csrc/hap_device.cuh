@@ -74,6 +74,7 @@ struct DpOut {
     u64 *incumbent;                   // running minimum of T_iter, for pruning
     const i64 *lb_sum;                // per configuration: sum over layers of the cheapest type's time
     int prune;                        // search mode: skip blocks whose lower bound exceeds the incumbent
+    int exact;                        // refinement kernels: sweep the stage-cost limit for the optimum of sum + (M-1) max
     int count_only;                   // instrumentation: count the finite-cost cells of each candidate, run no recurrence
 };
 
@@ -1042,47 +1043,100 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         }
         __syncwarp();
 
+        int ref_a = 0, ref_b = 0;                          // refinement: this lane's stage span of the chosen partition
         if (REFINE && bott < vInf) {
-            // ---- refinement: among the partitions whose stages all cost at most the bottleneck just found, the one
-            //      with the smallest sum of stage costs (additive recurrence, same bands, same tie-break).  Its split
-            //      choices replace those of the first pass; the first pass's rows stay intact for the next mapping.
-            int pbl = 0, pbh = 0;
-            for (int i = 1; i <= PP; ++i) {
-                const int src = i - 1;
-                const int mrow = __shfl_sync(0xffffffffu, sp.mrow, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
-                const VT K = shfl_v(sp.K, src);
-                const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
-                const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
-                const VT *rM = sR + (size_t)mrow * RW * n1;
-                const VT *prev = i == 1 ? szero : rows2 + (size_t)(i & 1) * n1;
-                VT *cur = rows2 + (size_t)((i - 1) & 1) * n1;
-                uint8_t *chrow = chw + (size_t)(i - 1) * n1;
-                const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
-                for (int j = bl + lane; j <= bh; j += 32) {
-                    VT best = vInf;
-                    int arg = 255;
-                    int klo = j - nmax; if (klo < pbl) klo = pbl;
-                    int khi = j - nmin; if (khi > pbh) khi = pbh;
-                    int seg_hi = khi;
-                    for (int r = 0; r < R && seg_hi >= klo; ++r) {
-                        if (!((rc_mask >> r) & 1u)) continue;
-                        int lo = th[(size_t)r * n1 + j];
-                        if (lo < klo) lo = klo;
-                        if (lo > seg_hi) continue;
-                        for (int k = seg_hi; k >= lo; --k) {
-                            VT cst;
-                            if (LINEAR) cst = (rM[(size_t)r * n1 + j] - rM[(size_t)r * n1 + k]) + K;
-                            else cst = ((rM[j] - rM[k]) + tau_term((i64)dc.tau_q[r], rM[n1 + j] - rM[n1 + k])) + K;
-                            const VT v = prev[k] + cst;
-                            if (cst <= bott && v <= best && v < vInf) { best = v; arg = k; }
+            // ---- refinement: an additive recurrence over the same bands with a limit on the stage cost.
+            //      limit = bottleneck: the smallest stage-cost sum among the bottleneck-optimal partitions.
+            //      exact mode: the limit is then swept upward over the stage costs that were skipped, which
+            //      reaches the optimum of sum + (M-1) max over all partitions (see below).
+            //      The first pass's rows stay intact for the next mapping; the split choices are overwritten.
+            const VT M1 = (VT)(pc.M - 1);
+            auto stage_of_lane = [&](int a_, int b_) -> VT {         // cost of this lane's stage over (a_, b_]
+                const uint8_t *th = thr + ((size_t)lane * T + sp.capt) * R * n1;
+                int r = 0;
+                for (; r < R - 1; ++r)          // lowest allowed level that fits (the span is feasible, so one does)
+                    if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b_] <= a_) break;
+                const VT *rM = sR + (size_t)sp.mrow * RW * n1;
+                if (LINEAR) return (rM[(size_t)r * n1 + b_] - rM[(size_t)r * n1 + a_]) + sp.K;
+                return ((rM[b_] - rM[a_]) + tau_term((i64)dc.tau_q[r], rM[n1 + b_] - rM[n1 + a_])) + sp.K;
+            };
+            // one pass: returns false if no partition respects the limit; else the sum, the largest stage cost of
+            // the chosen partition, this lane's span, and in `nxt` the smallest stage cost above the limit
+            auto pass = [&](VT limit, VT &psum, VT &pmax, VT &nxt, int &pa, int &pb) -> bool {
+                int pbl = 0, pbh = 0;
+                VT skipped = vInf;
+                for (int i = 1; i <= PP; ++i) {
+                    const int src = i - 1;
+                    const int mrow = __shfl_sync(0xffffffffu, sp.mrow, src), capt = __shfl_sync(0xffffffffu, sp.capt, src);
+                    const VT K = shfl_v(sp.K, src);
+                    const int nmin = __shfl_sync(0xffffffffu, sp.nmin, src), nmax = __shfl_sync(0xffffffffu, sp.nmax, src);
+                    const int bl = __shfl_sync(0xffffffffu, sp.bl, src), bh = __shfl_sync(0xffffffffu, sp.bh, src);
+                    const VT *rM = sR + (size_t)mrow * RW * n1;
+                    const VT *prev = i == 1 ? szero : rows2 + (size_t)(i & 1) * n1;
+                    VT *cur = rows2 + (size_t)((i - 1) & 1) * n1;
+                    uint8_t *chrow = chw + (size_t)(i - 1) * n1;
+                    const uint8_t *th = thr + ((size_t)(i - 1) * T + capt) * R * n1;
+                    for (int j = bl + lane; j <= bh; j += 32) {
+                        VT best = vInf;
+                        int arg = 255;
+                        int klo = j - nmax; if (klo < pbl) klo = pbl;
+                        int khi = j - nmin; if (khi > pbh) khi = pbh;
+                        int seg_hi = khi;
+                        for (int r = 0; r < R && seg_hi >= klo; ++r) {
+                            if (!((rc_mask >> r) & 1u)) continue;
+                            int lo = th[(size_t)r * n1 + j];
+                            if (lo < klo) lo = klo;
+                            if (lo > seg_hi) continue;
+                            for (int k = seg_hi; k >= lo; --k) {
+                                VT cst;
+                                if (LINEAR) cst = (rM[(size_t)r * n1 + j] - rM[(size_t)r * n1 + k]) + K;
+                                else cst = ((rM[j] - rM[k]) + tau_term((i64)dc.tau_q[r], rM[n1 + j] - rM[n1 + k])) + K;
+                                if (cst > limit) { skipped = cst < skipped ? cst : skipped; continue; }
+                                const VT v = prev[k] + cst;
+                                if (v <= best && v < vInf) { best = v; arg = k; }
+                            }
+                            seg_hi = lo - 1;
                         }
-                        seg_hi = lo - 1;
+                        cur[j] = best;
+                        chrow[j] = (uint8_t)arg;
                     }
-                    cur[j] = best;
-                    chrow[j] = (uint8_t)arg;
+                    __syncwarp();
+                    pbl = bl; pbh = bh;
                 }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) { const VT t = __shfl_xor_sync(0xffffffffu, skipped, o); skipped = t < skipped ? t : skipped; }
+                nxt = skipped;
+                psum = rows2[(size_t)((PP - 1) & 1) * n1 + N];
+                if (!(psum < vInf)) return false;
+                int j = N;
+                pa = 0; pb = 0;
+                for (int i = PP; i >= 1; --i) {
+                    const int k = chw[(size_t)(i - 1) * n1 + j];
+                    if (lane == i - 1) { pa = k; pb = j; }
+                    j = k;
+                }
+                VT c = lane < PP ? stage_of_lane(pa, pb) : (VT)0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) { const VT t = __shfl_xor_sync(0xffffffffu, c, o); c = t > c ? t : c; }
+                pmax = c;
                 __syncwarp();
-                pbl = bl; pbh = bh;
+                return true;
+            };
+            VT bs, bm, nx;
+            pass(bott, bs, bm, nx, ref_a, ref_b);            // always feasible: the min-max partition respects the limit
+            if (out.exact) {
+                // Sweep.  f_min = the smallest sum without a limit; a partition whose largest stage costs t cannot
+                // beat the incumbent V once f_min + (M-1) t >= V.  The first limit that reaches the smallest value wins.
+                VT Vbest = bs + M1 * bm;
+                VT us, um, unx; int ua, ub;
+                pass(vInf - 1, us, um, unx, ua, ub);
+                VT t = nx;
+                while (t < vInf && us + M1 * t < Vbest) {
+                    VT cs, cm, cn; int ca, cb;
+                    if (pass(t, cs, cm, cn, ca, cb) && cs + M1 * cm < Vbest) { Vbest = cs + M1 * cm; ref_a = ca; ref_b = cb; }
+                    t = cn;
+                }
+                if (us + M1 * um < Vbest) { ref_a = ua; ref_b = ub; }
             }
         }
 
@@ -1090,12 +1144,14 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         VT T_iter = vInf, T_pipe = vInf, T_sync = 0, T_opt = 0;
         int my_n = 0, my_r = 0;
         if (bott < vInf) {
-            int a_me = 0, b_me = 0;
-            int j = N;
-            for (int i = PP; i >= 1; --i) {
-                const int k = chw[(size_t)(i - 1) * n1 + j];
-                if (lane == i - 1) { a_me = k; b_me = j; }
-                j = k;
+            int a_me = ref_a, b_me = ref_b;
+            if (!REFINE) {
+                int j = N;
+                for (int i = PP; i >= 1; --i) {
+                    const int k = chw[(size_t)(i - 1) * n1 + j];
+                    if (lane == i - 1) { a_me = k; b_me = j; }
+                    j = k;
+                }
             }
             VT c_me = 0, sync_me = 0, opt_me = 0;
             if (lane < PP) {

@@ -390,3 +390,52 @@ def test_joint_device_state_recurrence(hap, name, kw):
     for p in rng.choice(small_pp, size=min(12, len(small_pp)), replace=False):
         for rc in range(n_rc):
             assert jb[p, rc] == o.joint_bottleneck(int(p), int(pb.rc_masks[rc])), (p, rc)
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {})])
+def test_exact_pipeline_term_mode_bit_exact(hap, name, kw):
+    """HAP_OPT_EXACT: the partition minimising sum + (M-1) max over all partitions of a candidate (limit sweep),
+    against the oracle's sweep for every candidate; plan with and without pruning."""
+    pb = problems.make_problem(name, **kw)
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs_exact(0, 1, threads=NTHREADS)
+    for prune in (0, 1):
+        hp = hap.hap_problem_create(pb, prune=prune, flags=hap.OPT_EXACT)
+        hap.hap_enumerate(hp)
+        if prune == 0:
+            out = hap.hap_pipeline_dp(hp, 0, hp.n_cand, partition=True)
+            torch.cuda.synchronize()
+            got = out["cost"].cpu().numpy()
+            bad = np.nonzero(got != costs)[0]
+            assert bad.size == 0, (bad[:5], got[bad[:5]], costs[bad[:5]])
+            assert np.array_equal(out["bottleneck"].cpu().numpy(), bn)
+            part, rec = out["partition"].cpu().numpy(), out["recompute"].cpu().numpy()
+            for idx in range(0, o.n_cand, max(1, o.n_cand // 300)):
+                ex = o.eval_index_exact(idx)
+                if ex["T_iter"] < INF:
+                    assert part[idx, :ex["PP"]].tolist() == ex["n"] and rec[idx, :ex["PP"]].tolist() == ex["r"], idx
+        plan, stats = hap.hap_search_best(hp)
+        assert (plan["T_iter"], plan["index"]) == (bc, bi)
+        hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("seed", [1, 4, 6])
+def test_exact_mode_on_random_problems(hap, seed):
+    pb = problems.random_small(seed, N=9 + seed % 4, T=2 + seed % 2, nodes_per_type=((2, 2), (2, 1, 1))[seed % 2],
+                               node_size=2, window=(seed % 2 == 0), first_dense=True)
+    if seed >= 4:
+        pb.xi_q = np.ascontiguousarray(np.array([1024, 512, 64], np.int32))
+        pb.tau_q = np.ascontiguousarray(np.array([0, 300, 1000], np.int32))
+        pb.rc_masks = np.ascontiguousarray(np.array([0b001, 0b011, 0b111, 0b101], np.uint32))
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs_exact(0, 1, threads=NTHREADS)
+    hp = hap.hap_problem_create(pb, flags=hap.OPT_EXACT)
+    hap.hap_enumerate(hp)
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["cost"].cpu().numpy(), costs)
+    for idx in range(0, o.n_cand, 41):
+        ex = o.eval_index_exact(idx)
+        if ex["T_iter"] < INF:
+            assert ex["T_pipe"] == ex["brute_pipe"]
+    hap.hap_problem_destroy(hp)

@@ -712,3 +712,30 @@ def test_joint_device_state_recurrence_equals_minimum_over_enumerated_sequences(
                     m[t] += int(pb.node_size[t])
                 assert (jb == -1) == any(x % G for x in m)
     assert checked > 20
+
+
+# --------------------------------------------------------------------------------------
+# exact optimum of the pipeline term sum + (M-1) max by the upward sweep of the stage-cost limit
+# --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("make,step", [(lambda: problems.tiny(), 2), (lambda: problems.tiny(window=True), 3),
+                                       (lambda: problems.random_small(1, N=9, T=2, nodes_per_type=(2, 2), node_size=2), 4),
+                                       (lambda: problems.random_small(6, N=8, T=3, nodes_per_type=(2, 1, 1), node_size=2,
+                                                                      window=True, first_dense=True), 7)])
+def test_limit_sweep_reaches_the_exhaustive_optimum_of_the_pipeline_term(make, step):
+    pb = make()
+    o = Oracle(pb)
+    costs, bn, _, _ = o.search()
+    improved = swept = 0
+    for idx in range(0, o.n_cand, step):
+        ex = o.eval_index_exact(idx)
+        if bn[idx] >= INF:
+            assert ex["T_iter"] == INF
+            continue
+        ref = o.eval_index_refined(idx)
+        assert ex["T_pipe"] == ex["brute_pipe"]                      # the optimum over ALL partitions
+        assert ex["T_pipe"] == sum(ex["c"]) + (ex["M"] - 1) * max(ex["c"]) <= ref["T_pipe"]
+        assert sum(ex["n"]) == pb.N and ex["bottleneck"] == bn[idx] <= max(ex["c"])
+        improved += ex["T_pipe"] < ref["T_pipe"]
+        swept += ex["passes"] > 2
+    if pb.name == "tiny":
+        assert improved > 0 and swept > 0
