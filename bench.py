@@ -253,7 +253,8 @@ def main():
     # the same pass with the refinement (smallest stage-cost sum among the bottleneck-optimal partitions) and with
     # the exact optimisation of sum + (M-1) max (limit sweep); untimed extras
     extra_modes = {}
-    for mode_name, flag in (("refined_pass", hap.OPT_REFINE), ("exact_pass", hap.OPT_EXACT)):
+    for mode_name, flag in (("refined_pass", hap.OPT_REFINE), ("exact_pass", hap.OPT_EXACT),
+                            ("uniform_partition_ablation", hap.OPT_UNIFORM)):
         hp_ref = hap.hap_problem_create(pb, flags=flag)
         hap.hap_enumerate(hp_ref)
         ref_ms = []
@@ -269,6 +270,10 @@ def main():
                 ref_ms.append(a.elapsed_time(b))
         ref_best = [int(x) for x in am_ref.tolist()]
         extra_modes[mode_name] = dict(ms=statistics.median(ref_ms), best_cost=ref_best[0], best_index=ref_best[1] + first)
+        if flag == hap.OPT_UNIFORM and world == 1:
+            # predicted latency of the best uniform-split plan over the best non-uniform plan (planner-level mirror of
+            # the paper's "non-uniform partitioning disabled" ablation; synthetic inputs, context only)
+            extra_modes[mode_name]["latency_ratio_vs_non_uniform"] = ref_best[0] / best[0]
         hap.hap_problem_destroy(hp_ref)
 
     # full search through the search entry point (pruning allowed), wall clock call to return

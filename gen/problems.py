@@ -102,6 +102,7 @@ class Problem:
     rc_masks: np.ndarray  # [n_rc] uint32, allowed recompute levels per policy
     # ---- extras that are not inputs of the method (kept for inspection)
     extra: Dict[str, np.ndarray] = field(default_factory=dict)
+    uniform: int = 0     # ablation: 1 = uniform layer split only (non-uniform partitioning disabled)
     eta_q: int = 0       # Pruning 3 threshold eta in 1/1024 (2048 = the paper's default 2); <= 0 disables it
 
     @property

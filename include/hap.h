@@ -130,6 +130,8 @@ typedef struct {
 
 /* hap_search_opts.flags */
 #define HAP_OPT_NO_MAPTAB 1   /* keep no table of decoded mappings on the device: the DP kernel unranks each mapping itself */
+#define HAP_OPT_UNIFORM 8     /* ablation "non-uniform partitioning disabled" (Sec. 5.5): every stage takes floor(N/PP) or
+                                 ceil(N/PP) layers; the load-balance window is ignored */
 #define HAP_OPT_EXACT 4       /* like HAP_OPT_REFINE, but the limit on the stage cost is then swept upward from the bottleneck over
                                  the stage costs, which yields the partition that minimises sum_i c_i + (M-1) max_i c_i (Eq. 4's
                                  pipeline term in closed form) over ALL partitions of the candidate; integer mode only.  The

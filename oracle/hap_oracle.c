@@ -375,6 +375,11 @@ static int64_t mask_max(const orc_problem *pr, unsigned mask, const int64_t *coe
 int orc_window(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, int32_t *nmin, int32_t *nmax)
 {
     const int PP = pc->PP, N = pr->N;
+    if (pr->uniform) {
+        /* ablation "non-uniform partitioning disabled": every stage takes floor(N/PP) or ceil(N/PP) layers */
+        for (int s = 0; s < PP; ++s) { nmin[s] = N / PP; nmax[s] = (N + PP - 1) / PP; }
+        return 2;
+    }
     if (pr->delta_q < 0) {
         for (int s = 0; s < PP; ++s) { nmin[s] = 1; nmax[s] = N - PP + 1; }
         return 0;
@@ -1266,7 +1271,8 @@ int64_t orc_joint_bottleneck(const orc_problem *pr, const orc_pconf *pc, uint32_
     for (int h = 0; h < T; ++h) Ps += (int64_t)cnt[h] * pr->P[h];
     for (int h = 0; h < T; ++h) {
         int64_t lo = 1, hi = N - PP + 1;
-        if (pr->delta_q >= 0) {
+        if (pr->uniform) { lo = N / PP; hi = (N + PP - 1) / PP; }
+        else if (pr->delta_q >= 0) {
             lo = ((int64_t)(1024 - pr->delta_q) * pr->P[h] * N) / (1024 * Ps);
             int64_t num = (int64_t)(1024 + pr->delta_q) * pr->P[h] * N, den = 1024 * Ps;
             hi = (num + den - 1) / den;

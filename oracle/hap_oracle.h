@@ -71,6 +71,7 @@ typedef struct {
     int32_t n_rc;
     const uint32_t *rc_masks;
     int32_t eta_q;      /* Pruning 3 threshold eta in 1/1024; <= 0: off */
+    int32_t uniform;    /* ablation: uniform layer split only (floor/ceil of N/PP layers per stage) */
 } orc_problem;
 
 typedef struct {

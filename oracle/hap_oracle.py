@@ -50,7 +50,7 @@ class _Problem(C.Structure):
         ("R", C.c_int32), ("xi_q", C.c_void_p), ("tau_q", C.c_void_p),
         ("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
         ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64),
-        ("n_rc", C.c_int32), ("rc_masks", C.c_void_p), ("eta_q", C.c_int32),
+        ("n_rc", C.c_int32), ("rc_masks", C.c_void_p), ("eta_q", C.c_int32), ("uniform", C.c_int32),
     ]
 
 
@@ -153,6 +153,7 @@ class Oracle:
         s.n_rc = len(pb.rc_masks)
         s.rc_masks = arr("rc_masks", np.uint32)
         s.eta_q = int(getattr(pb, "eta_q", 0))
+        s.uniform = int(getattr(pb, "uniform", 0))
         self._keep = keep
         self.s = s
         self.N, self.T = int(pb.N), s.T

@@ -140,6 +140,7 @@ class HapProblem:
 OPT_NO_MAPTAB = 1
 OPT_REFINE = 2
 OPT_EXACT = 4
+OPT_UNIFORM = 8
 
 
 def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
@@ -180,7 +181,7 @@ def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     so.n_rc = len(pb.rc_masks)
     so.rc_masks = arr("rc_masks", np.uint32)
     so.prune = int(prune)
-    so.flags = int(flags)
+    so.flags = int(flags) | (OPT_UNIFORM if int(getattr(pb, "uniform", 0)) else 0)
     so.eta_q = int(getattr(pb, "eta_q", 0))
     out = C.c_void_p(0)
     st = L.hap_problem_create(C.byref(mo), C.byref(cl), C.byref(pf), C.byref(so), C.byref(out))

@@ -36,7 +36,7 @@ constexpr i64 kInf = (i64)1 << 62;
 struct DevConst {
     int N, T, R, n_rc, ntp, ncp, nmb, nep;
     int S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
-    int delta_q, tau_linear, eta_q;
+    int delta_q, tau_linear, eta_q, uniform;
     double beta, kappa, chi, gamma, ovl_tp, ovl_cp, ovl_dp, capf;
     double alpha[3];
     double eta[HAP_MAX_TYPES], croute[HAP_MAX_TYPES], copt[HAP_MAX_TYPES];
@@ -738,6 +738,7 @@ __device__ __forceinline__ void dp_block_prologue(
             lo = a < 1 ? 1 : (int)a;
             hi = b > N - PP + 1 ? N - PP + 1 : (int)b;
         }
+        if (dc.uniform) { lo = N / PP; hi = (N + PP - 1) / PP; }      // ablation: uniform layer split only
         winT[threadIdx.x][0] = lo; winT[threadIdx.x][1] = hi;
     }
     __syncthreads();
@@ -891,7 +892,9 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                 sp.K += sP2P[hb][cls == HAP_CROSS ? 2 + ha : cls];
             }
         }
-        if (dc.delta_q >= 0) {
+        if (dc.uniform) {
+            if (lane < PP) { sp.nmin = N / PP; sp.nmax = (N + PP - 1) / PP; }
+        } else if (dc.delta_q >= 0) {
             if (multiset) {
                 if (lane < PP) { sp.nmin = winT[sp.mrow][0]; sp.nmax = winT[sp.mrow][1]; }   // homogeneous stage: its one type
             } else {

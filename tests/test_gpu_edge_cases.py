@@ -156,3 +156,34 @@ def test_heterogeneous_communication_pruning(hap, name, eta_q):
     fin = np.isfinite(got) & np.isfinite(cf)
     assert np.max(np.abs(got[fin] - cf[fin]) / cf[fin]) <= 1e-9
     hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small", "mixtral"])
+def test_uniform_partition_ablation(hap, name):
+    """HAP_OPT_UNIFORM (the paper's "non-uniform partitioning disabled" ablation): stages take floor/ceil(N/PP)
+    layers.  Parity with the oracle; the uniform optimum can never beat the non-uniform one when the window is off."""
+    pb = problems.make_problem(name)
+    pb.uniform = 1
+    o, costs = full_compare(hap, pb, tables_every=997)
+    for idx in range(0, o.n_cand, max(1, o.n_cand // 50)):
+        plan, _, _ = o.eval_index(idx)
+        if plan["T_iter"] < INF:
+            assert max(plan["n"]) - min(plan["n"]) <= 1
+    free = problems.make_problem(name)
+    free.delta_q = -1
+    best_free = Oracle(free).search_pconfs(0, 1, threads=8)[1]
+    assert costs.min() >= best_free
+    # the joint recurrence honours the same restriction
+    hp = hap.hap_problem_create(pb)
+    hap.hap_enumerate(hp)
+    jb = hap.hap_joint_bottleneck(hp).cpu().numpy()
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    bn = out["bottleneck"].cpu().numpy()
+    n_rc = len(pb.rc_masks)
+    for p in range(o.n_pconf):
+        if int(o.pconfs["mode"][p]) == 0:
+            off, nmap = int(o.pconfs["offset"][p]), int(o.pconfs["nmap"][p])
+            for rc in range(n_rc):
+                assert jb[p, rc] == bn[off + rc: off + nmap * n_rc: n_rc].min()
+    hap.hap_problem_destroy(hp)
