@@ -335,7 +335,7 @@ def main():
             clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"]),
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                      ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
-            gpu_launches=(4 + len(set(int(x) for x in pconfs["PP"]))) * args.steps,
+            gpu_launches=(4 + 2 * len(set(int(x) for x in pconfs["PP"]))) * args.steps,
             **extra_modes,
             joint_recurrence_ms=joint_ms,
             full_search_ms=statistics.median(search_ms),

@@ -579,6 +579,14 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         void *cvarg = f64 ? (void *)p->d_coeff : (void *)p->d_coef;
         void *args[] = {(void *)&p->dc, (void *)&its, (void *)&c2arg, (void *)&p->d_coef, (void *)&cvarg, (void *)&tab, (void *)&o, (void *)&nw, (void *)&used};
         CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
+        if (cl.has_tab && out.count > 1) {
+            // candidate decode (stage masks and link classes of every mapping of the class) is part of every pass,
+            // not a cached result of hap_enumerate; the one-candidate re-evaluation of a winner reuses the table
+            const WorkItem &rep = p->items[cl.item_lo];
+            const u64 nmap = p->pconfs[rep.p].nmap;
+            maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, rep.p, nmap, p->d_maptab + cl.map_base);
+            CUDA_TRY(p, cudaGetLastError());
+        }
         CUDA_TRY(p, cudaLaunchKernel(fn, dim3(blocks), dim3(cl.warps * 32), args, cl.smem, cl.stream));
         CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
         CUDA_TRY(p, cudaStreamWaitEvent(st, cl.done, 0));      // join
