@@ -251,6 +251,19 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     dc.act_coef[0] = p->act_coef[0]; dc.act_coef[1] = p->act_coef[1];
     for (int i = 0; i < pf->nep; ++i) dc.rho[i] = p->rho[i];
     for (int i = 0; i < so->n_rc; ++i) dc.rc_masks[i] = p->rc_masks[i];
+    {   // evaluation order of the policies: more allowed levels first (stable), and who contains whom
+        std::vector<int> order(so->n_rc);
+        for (int i = 0; i < so->n_rc; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+            return __builtin_popcount(p->rc_masks[a]) > __builtin_popcount(p->rc_masks[b]);
+        });
+        for (int j = 0; j < so->n_rc; ++j) {
+            dc.rc_order[j] = order[j];
+            dc.rc_sup[j] = 0;
+            for (int q = 0; q < j; ++q)
+                if ((p->rc_masks[order[q]] & p->rc_masks[order[j]]) == p->rc_masks[order[j]]) dc.rc_sup[j] |= 1u << q;
+        }
+    }
     dc.tau_linear = 1;
     for (int r = 0; r < pf->R; ++r) { dc.xi_q[r] = p->xi_q[r]; dc.tau_q[r] = p->tau_q[r]; if (p->tau_q[r] % 1024) dc.tau_linear = 0; }
     for (int l = 0; l < N; ++l) if (p->kind[l] == HAP_MOE) dc.kindbits[l >> 6] |= 1ull << (l & 63);
@@ -375,13 +388,15 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 if (resident > best_resident) { best_resident = resident; cl.warps = w; cl.smem = sm; }
             }
             if (!cl.warps) return fail(p, HAP_E_RANGE, "shared memory need of a PP=%d block exceeds the SM", PP);
-            const int slices = std::max(1, cl.warps / p->opts.n_rc);
-            const uint64_t chunk = 64ull * slices;
+            // a warp takes a slice of at most 64 consecutive mappings (one bit each in its infeasibility masks)
+            const uint64_t chunk_cap = 32ull * cl.warps;
             cl.item_lo = items.size();
             uint64_t nmap = 0;
             for (size_t pi = 0; pi < rows.size(); ++pi) {
                 if (rows[pi].PP != PP) continue;
                 nmap = rows[pi].nmap;
+                const uint64_t n_chunks = (nmap + chunk_cap - 1) / chunk_cap;
+                const uint64_t chunk = (nmap + n_chunks - 1) / n_chunks;          // balanced chunks
                 for (uint64_t lo = 0; lo < nmap; lo += chunk) {
                     WorkItem it; it.p = (uint32_t)pi; it.lo = lo; it.count = (uint32_t)std::min<uint64_t>(chunk, nmap - lo);
                     items.push_back(it);

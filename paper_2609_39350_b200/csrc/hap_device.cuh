@@ -46,6 +46,8 @@ struct DevConst {
     i64 P[HAP_MAX_TYPES], cap_eff[HAP_MAX_TYPES], m[HAP_MAX_TYPES];
     int node_size[HAP_MAX_TYPES];
     unsigned rc_masks[HAP_MAX_RC_MASKS];
+    int rc_order[HAP_MAX_RC_MASKS];   // policies from the most permissive to the most restrictive
+    unsigned rc_sup[HAP_MAX_RC_MASKS]; // per position in rc_order: earlier positions whose allowed levels are a superset
     int xi_q[HAP_MAX_RC], tau_q[HAP_MAX_RC];
     u64 kindbits[4];                  // bit l set: layer l is an MoE layer
     const double *tdf, *tdb, *tff, *tfb, *tpre, *tpost;
@@ -823,16 +825,21 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
     while (red0 < PP) red0 <<= 1;
     red0 >>= 1;
 
-    // warp -> (recompute policy, slice of consecutive mappings); consecutive mappings share a prefix of
-    // stage types, and the DP rows of a shared prefix are reused
-    const int slices = nwarps / n_rc > 0 ? nwarps / n_rc : 1;
-    const int my_rc = wib % n_rc, my_slice = wib / n_rc;
-    const bool active_warp = wib < slices * n_rc || n_rc > nwarps;
-    const u32 per_slice = (it.count + slices - 1) / slices;
-    for (int rc_idx = my_rc; rc_idx < n_rc && active_warp; rc_idx += nwarps) {
+    // warp -> slice of consecutive mappings, evaluated once per recompute policy.  Consecutive mappings share a
+    // prefix of stage types, and the DP rows of a shared prefix are reused.  Policies run from the most
+    // permissive to the most restrictive (dc.rc_order): a mapping that admits no feasible partition under a
+    // policy admits none under any policy whose allowed levels are a subset, so it is skipped there.
+    __shared__ u64 s_infeas[kDpWarps][HAP_MAX_RC_MASKS];
+    const u32 per_slice = (it.count + nwarps - 1) / nwarps;          // <= 64 (host chunking)
+    for (int rc_pos = 0; rc_pos < n_rc; ++rc_pos) {
+      const int rc_idx = dc.rc_order[rc_pos];
       const unsigned rc_mask = dc.rc_masks[rc_idx];
-      const u32 m_lo = (u32)my_slice * per_slice;
+      const u32 m_lo = (u32)wib * per_slice;
       const u32 m_hi = m_lo + per_slice < it.count ? m_lo + per_slice : it.count;
+      u64 known_infeasible = 0, infeasible_here = 0;
+      if (!COUNT && !want_tables)
+          for (int q = 0; q < rc_pos; ++q)
+              if ((dc.rc_sup[rc_pos] >> q) & 1u) known_infeasible |= s_infeas[wib][q];
       int valid_rows = 0;                  // DP rows of stages 1..valid_rows of the previous mapping are intact
       int dead_stage = 1 << 30;            // first of those stages whose row holds no finite value (none: large)
       int prev_mask = -1, prev_link = -1;
@@ -854,6 +861,23 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             mask = smap.mask; link = lane > 0 && lane < PP ? (smap.cls | (smap.ha << 2) | (smap.hb << 4)) : 0;
         }
         if (c < out.first || c >= out.first + out.count) { valid_rows = 0; dead_stage = 1 << 30; prev_mask = -1; continue; }
+        if ((known_infeasible >> (mi - m_lo)) & 1ull) {
+            // infeasible under a more permissive policy: infeasible here, nothing to compute
+            infeasible_here |= 1ull << (mi - m_lo);
+            valid_rows = 0; dead_stage = 1 << 30; prev_mask = -1;
+            if (SEARCH) n_eval++;
+            else {
+                const u64 o = c - out.first;
+                if (lane == 0) {
+                    if (out.cost) reinterpret_cast<VT *>(out.cost)[o] = vInf;
+                    if (out.bottleneck) reinterpret_cast<VT *>(out.bottleneck)[o] = vInf;
+                    if (out.detail) { VT *d = reinterpret_cast<VT *>(out.detail); d[o * 3] = vInf; d[o * 3 + 1] = 0; d[o * 3 + 2] = 0; }
+                }
+                if (out.partition) out.partition[o * HAP_MAX_PP + lane] = 0;
+                if (out.recompute) out.recompute[o * HAP_MAX_PP + lane] = 0;
+            }
+            continue;
+        }
         const unsigned differ = __ballot_sync(0xffffffffu, lane < PP && (mask != prev_mask || link != prev_link));
         int s0 = differ ? __ffs(differ) - 1 : PP;      // stages 1..s0 are shared with the previous mapping
         prev_mask = mask; prev_link = link;
@@ -864,6 +888,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         if (!COUNT && dead_stage <= s0) {
             // a shared stage prefix that already admits no feasible partition settles this mapping too
             valid_rows = s0;
+            infeasible_here |= 1ull << (mi - m_lo);
             if (SEARCH) n_eval++;
             else {
                 const u64 o = c - out.first;
@@ -1046,6 +1071,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         }
         __syncwarp();
 
+        if (!(bott < vInf)) infeasible_here |= 1ull << (mi - m_lo);
         int ref_a = 0, ref_b = 0;                          // refinement: this lane's stage span of the chosen partition
         if (REFINE && bott < vInf) {
             // ---- refinement: an additive recurrence over the same bands with a limit on the stage cost.
@@ -1212,6 +1238,8 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         }
         __syncwarp();
       }
+      if (lane == 0) s_infeas[wib][rc_pos] = infeasible_here;
+      __syncwarp();
     }
 
     if (out.counters) {
