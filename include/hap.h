@@ -130,6 +130,8 @@ typedef struct {
 
 /* hap_search_opts.flags */
 #define HAP_OPT_NO_MAPTAB 1   /* keep no table of decoded mappings on the device: the DP kernel unranks each mapping itself */
+#define HAP_OPT_NO_TRIE 16    /* keep no prefix tree of the mappings: every pass runs one warp per candidate (the tree form
+                                 shares the DP rows of common stage prefixes between all mappings of a configuration) */
 #define HAP_OPT_UNIFORM 8     /* ablation "non-uniform partitioning disabled" (Sec. 5.5): every stage takes floor(N/PP) or
                                  ceil(N/PP) layers; the load-balance window is ignored */
 #define HAP_OPT_EXACT 4       /* like HAP_OPT_REFINE, but the limit on the stage cost is then swept upward from the bottleneck over

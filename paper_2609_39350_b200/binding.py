@@ -141,6 +141,7 @@ OPT_NO_MAPTAB = 1
 OPT_REFINE = 2
 OPT_EXACT = 4
 OPT_UNIFORM = 8
+OPT_NO_TRIE = 16
 
 
 def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:

@@ -7,7 +7,7 @@ import subprocess
 _DIR = os.path.dirname(os.path.abspath(__file__))
 LIB = os.path.join(_DIR, "libhap.so")
 SOURCES = [os.path.join(_DIR, "csrc", "hap_api.cu")]
-HEADERS = [os.path.join(_DIR, "csrc", "hap_device.cuh"), os.path.join(os.path.dirname(_DIR), "include", "hap.h")]
+HEADERS = [os.path.join(_DIR, "csrc", "hap_device.cuh"), os.path.join(_DIR, "csrc", "hap_trie.cuh"), os.path.join(os.path.dirname(_DIR), "include", "hap.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "--fmad=false", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

@@ -2,6 +2,7 @@
 // work partitioning, kernel launches.  Every step of the hot path runs in the kernels of
 // hap_device.cuh; nothing here evaluates a cost.
 #include "hap_device.cuh"
+#include "hap_trie.cuh"
 
 #include <algorithm>
 #include <cstdarg>
@@ -33,7 +34,10 @@ struct hap_problem {
     std::vector<hap_pconf> pconfs;
     uint64_t n_cand = 0;
     std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
-    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; };
+    // prefix tree of a class's mappings (trie_dp_kernel); ok = false: the class runs in pipeline_dp_kernel only
+    struct Trie { bool ok; TrieMeta meta; unsigned char *d_blob; u32 *d_first_leaf; uint8_t *d_depth; TrieNode *d_nodes; TrieLeaf *d_leaves;
+                  u32 *d_plist; unsigned n_conf; u32 n_nodes; int threads; size_t smem; };
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     // device
@@ -119,7 +123,7 @@ static void release_device(hap_problem *p)
     cudaFree(p->d_range); cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); }
+    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist); }
 }
 
 extern "C" void hap_problem_destroy(hap_problem *p)
@@ -304,6 +308,171 @@ static uint64_t sequences_sat(const int *cnt, int T, uint64_t sat)
     return (uint64_t)r;
 }
 
+// Prefix tree of the decoded mappings of one PP class (host copy `tab`: nmap x PP x (mask, link) bytes).
+// A node is a distinct sequence of stage keys (types, link, load-balance window) of stages 1..d, d < PP;
+// mappings that are consecutive in enumeration order share the nodes of their common prefix.  The window
+// and the band of reachable end layers follow the same integer formulas as pipeline_dp_kernel; a node's
+// band is the union over the mappings below it, which only adds cells that hold their plain recurrence
+// value.  Returns false (and leaves the class on the general kernel) when the tree does not fit.
+static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, const std::vector<u32> &plist)
+{
+    const int N = p->model.N, PP = cl.PP, T = p->T, R = p->prof.R;
+    if (nmap == 0 || nmap > 65535 || plist.empty()) return false;
+    struct Key { uint8_t mask, link, nmin, nmax; };
+    struct HNode { u32 parent; Key k; int bl, bh; u32 first_leaf; };
+    std::vector<std::vector<HNode>> lv(PP + 1);               // lv[d], d = 1..PP-1
+    std::vector<TrieLeaf> leaves(nmap);
+    std::vector<u32> path(PP + 1, 0);
+    std::vector<Key> pkey(PP + 1);
+    bool have_prev = false;
+    i64 Pmin[1 << HAP_MAX_TYPES];
+    for (int mk = 1; mk < (1 << T); ++mk) {
+        i64 v = 0; bool seen = false;
+        for (int h = 0; h < T; ++h) if (mk >> h & 1) { if (!seen || p->P[h] < v) v = p->P[h]; seen = true; }
+        Pmin[mk] = v;
+    }
+    const int delta_q = p->opts.delta_q;
+    const bool uniform = (p->opts.flags & HAP_OPT_UNIFORM) != 0;
+    std::vector<int> nmin(PP + 1), nmax(PP + 1), bl(PP + 1), bh(PP + 1);
+    for (u64 m = 0; m < nmap; ++m) {
+        const uint8_t *row = tab + m * (u64)PP * 2;
+        i64 Ps = 0;
+        for (int s = 0; s < PP; ++s) {
+            const int mk = row[s * 2];
+            if (mk < 1 || mk >= (1 << T)) return false;
+            Ps += Pmin[mk];
+        }
+        for (int s = 1; s <= PP; ++s) {
+            int lo = 1, hi = N - PP + 1;
+            if (uniform) { lo = N / PP; hi = (N + PP - 1) / PP; }
+            else if (delta_q >= 0) {
+                const i64 Pm = Pmin[row[(s - 1) * 2]], den = 1024 * Ps;
+                i64 a = ((i64)(1024 - delta_q) * Pm * N) / den;
+                i64 b = ((i64)(1024 + delta_q) * Pm * N + den - 1) / den;
+                if (a < 1) a = 1;
+                if (b > N - PP + 1) b = N - PP + 1;
+                lo = (int)a; hi = (int)b;
+            }
+            if (lo < 0 || lo > 255 || hi < 0 || hi > 255) return false;
+            nmin[s] = lo; nmax[s] = hi;
+        }
+        int tmin = 0, tmax = 0;
+        for (int s = 1; s <= PP; ++s) { tmin += nmin[s]; tmax += nmax[s]; }
+        bool dead = false;
+        int smin = 0, smax = 0;
+        for (int s = 1; s <= PP; ++s) {
+            smin += nmin[s]; smax += nmax[s];
+            int lo = smin > s ? smin : s, hi = smax < N - PP + s ? smax : N - PP + s;
+            const int rl = N - (tmax - smax), rh = N - (tmin - smin);
+            lo = lo > rl ? lo : rl; hi = hi < rh ? hi : rh;
+            bl[s] = lo; bh[s] = hi;
+            if (lo > hi) dead = true;
+        }
+        TrieLeaf &lf = leaves[m];
+        std::memset(&lf, 0, sizeof(lf));
+        lf.mask = row[(PP - 1) * 2]; lf.link = row[(PP - 1) * 2 + 1];
+        lf.nmin = (uint8_t)nmin[PP]; lf.nmax = (uint8_t)nmax[PP];
+        lf.dead = dead ? 1 : 0;
+        if (dead) continue;
+        int d0 = 1;                                              // first depth at which a new node is needed
+        if (have_prev)
+            for (; d0 < PP; ++d0) {
+                const Key &k = pkey[d0];
+                if (k.mask != row[(d0 - 1) * 2] || k.link != row[(d0 - 1) * 2 + 1] || k.nmin != nmin[d0] || k.nmax != nmax[d0]) break;
+            }
+        for (int d = d0; d < PP; ++d) {
+            HNode nd;
+            nd.parent = d > 1 ? path[d - 1] : 0;
+            nd.k = Key{row[(d - 1) * 2], row[(d - 1) * 2 + 1], (uint8_t)nmin[d], (uint8_t)nmax[d]};
+            nd.bl = 1 << 20; nd.bh = -1; nd.first_leaf = (u32)m;
+            pkey[d] = nd.k;
+            path[d] = (u32)lv[d].size();
+            lv[d].push_back(nd);
+        }
+        have_prev = true;
+        for (int d = 1; d < PP; ++d) {
+            HNode &nd = lv[d][path[d]];
+            nd.bl = std::min(nd.bl, bl[d]); nd.bh = std::max(nd.bh, bh[d]);
+        }
+        lf.parent = PP > 1 ? (uint16_t)path[PP - 1] : 0;
+    }
+    // flat layout
+    hap_problem::Trie &tr = cl.trie;
+    TrieMeta &tm = tr.meta;
+    std::memset(&tm, 0, sizeof(tm));
+    tm.PP = PP; tm.nmap = (u32)nmap;
+    u32 n_nodes = 0, n_cells = 0, max_level = 0;
+    std::vector<std::vector<u32>> rowoff(PP + 1);
+    for (int d = 1; d < PP; ++d) {
+        if (lv[d].size() > 65535) return false;
+        tm.node_lo[d] = n_nodes; tm.cell_lo[d] = n_cells;
+        u32 c = 0;
+        rowoff[d].resize(lv[d].size());
+        for (size_t i = 0; i < lv[d].size(); ++i) { rowoff[d][i] = c; c += (u32)(lv[d][i].bh - lv[d][i].bl + 1); }
+        tm.buf_cells[d & 1] = std::max(tm.buf_cells[d & 1], c);
+        max_level = std::max(max_level, c);
+        n_nodes += (u32)lv[d].size(); n_cells += c;
+    }
+    for (int d = std::max(PP, 1); d <= HAP_MAX_PP; ++d) { tm.node_lo[d] = n_nodes; tm.cell_lo[d] = n_cells; }
+    tm.buf_cells[0] = (tm.buf_cells[0] + 1) / 2 * 2; tm.buf_cells[1] = (tm.buf_cells[1] + 1) / 2 * 2;
+    const size_t smem = trie_smem_bytes(N, PP, T, R, cl.multiset, tm.buf_cells[0], tm.buf_cells[1], n_cells);
+    if (smem > 220 * 1024) return false;
+    std::vector<TrieNode> nodes(n_nodes);
+    std::vector<uint16_t> parent(n_nodes), cell_node(n_cells);
+    std::vector<u32> first_leaf(n_nodes);
+    std::vector<uint8_t> depth(n_nodes);
+    for (int d = 1; d < PP; ++d)
+        for (size_t i = 0; i < lv[d].size(); ++i) {
+            const HNode &h = lv[d][i];
+            TrieNode &nd = nodes[tm.node_lo[d] + i];
+            nd.rowoff = rowoff[d][i];
+            nd.mask = h.k.mask; nd.link = h.k.link; nd.nmin = h.k.nmin; nd.nmax = h.k.nmax;
+            nd.bl = (uint8_t)h.bl; nd.bh = (uint8_t)h.bh;
+            if (d > 1) { const HNode &ph = lv[d - 1][h.parent]; nd.prowoff = rowoff[d - 1][h.parent]; nd.pbl = (uint8_t)ph.bl; nd.pbh = (uint8_t)ph.bh; }
+            else { nd.prowoff = 0; nd.pbl = 0; nd.pbh = 0; }
+            parent[tm.node_lo[d] + i] = (uint16_t)h.parent;
+            first_leaf[tm.node_lo[d] + i] = h.first_leaf;
+            depth[tm.node_lo[d] + i] = (uint8_t)d;
+            for (int j = h.bl; j <= h.bh; ++j) cell_node[tm.cell_lo[d] + rowoff[d][i] + (u32)(j - h.bl)] = (uint16_t)i;
+        }
+    for (u64 m = 0; m < nmap; ++m) {
+        TrieLeaf &lf = leaves[m];
+        if (lf.dead || PP == 1) { lf.prowoff = 0; lf.pbl = 0; lf.pbh = 0; continue; }
+        const HNode &ph = lv[PP - 1][lf.parent];
+        lf.prowoff = rowoff[PP - 1][lf.parent]; lf.pbl = (uint8_t)ph.bl; lf.pbh = (uint8_t)ph.bh;
+    }
+    // one allocation: nodes | leaves | first_leaf | parent | cell_node | depth
+    auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+    const size_t o_nodes = 0, o_leaves = up(o_nodes + (size_t)n_nodes * sizeof(TrieNode));
+    const size_t o_first = up(o_leaves + nmap * sizeof(TrieLeaf)), o_parent = up(o_first + (size_t)n_nodes * 4);
+    const size_t o_cell = up(o_parent + (size_t)n_nodes * 2), o_depth = up(o_cell + (size_t)n_cells * 2);
+    const size_t total = up(o_depth + n_nodes) + 256;
+    std::vector<unsigned char> blob(total, 0);
+    if (n_nodes) std::memcpy(blob.data() + o_nodes, nodes.data(), (size_t)n_nodes * sizeof(TrieNode));
+    std::memcpy(blob.data() + o_leaves, leaves.data(), nmap * sizeof(TrieLeaf));
+    if (n_nodes) std::memcpy(blob.data() + o_first, first_leaf.data(), (size_t)n_nodes * 4);
+    if (n_nodes) std::memcpy(blob.data() + o_parent, parent.data(), (size_t)n_nodes * 2);
+    if (n_cells) std::memcpy(blob.data() + o_cell, cell_node.data(), (size_t)n_cells * 2);
+    if (n_nodes) std::memcpy(blob.data() + o_depth, depth.data(), n_nodes);
+    if (cudaMalloc(&tr.d_blob, total) != cudaSuccess) { tr.d_blob = nullptr; cudaGetLastError(); return false; }
+    if (cudaMemcpy(tr.d_blob, blob.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    if (cudaMalloc(&tr.d_plist, plist.size() * sizeof(u32)) != cudaSuccess) { tr.d_plist = nullptr; cudaGetLastError(); return false; }
+    if (cudaMemcpy(tr.d_plist, plist.data(), plist.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    tr.d_nodes = reinterpret_cast<TrieNode *>(tr.d_blob + o_nodes);
+    tr.d_leaves = reinterpret_cast<TrieLeaf *>(tr.d_blob + o_leaves);
+    tr.d_first_leaf = reinterpret_cast<u32 *>(tr.d_blob + o_first);
+    tr.d_depth = tr.d_blob + o_depth;
+    tm.nodes = tr.d_nodes; tm.leaves = tr.d_leaves;
+    tm.parent = reinterpret_cast<const uint16_t *>(tr.d_blob + o_parent);
+    tm.cell_node = reinterpret_cast<const uint16_t *>(tr.d_blob + o_cell);
+    tr.n_conf = (unsigned)plist.size(); tr.n_nodes = n_nodes; tr.smem = smem;
+    const u32 want = std::max<u32>(max_level, (u32)nmap);
+    int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
+    tr.threads = std::min(1024, std::max(128, th));
+    tr.ok = true;
+    return true;
+}
+
 extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t *n_candidates)
 {
     if (!p) return HAP_E_INVALID;
@@ -458,6 +627,14 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 unsigned used = 0;
                 for (u64 e = 0; e < nmap * (u64)cl.PP; ++e) used |= 1u << tab[cl.map_base + e * 2];
                 cl.masks_used = used;
+                if (!(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear) {
+                    std::vector<u32> plist;
+                    for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == cl.PP) plist.push_back((u32)pi);
+                    if (!build_trie(p, cl, tab.data() + cl.map_base, nmap, plist)) {
+                        cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist);
+                        cl.trie = hap_problem::Trie{};
+                    }
+                }
             }
         }
         p->enumerated = true;
@@ -587,6 +764,35 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         DpOut o = out;
         o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0;
         if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
+        // plain integer passes over more than one candidate walk the class's prefix tree; tables, refinement,
+        // fp64, cell counting and the one-candidate re-evaluation stay in pipeline_dp_kernel
+        if (cl.trie.ok && !f64 && !out.count_only && !refine && lin && !out.dp_table && !out.choice && out.count > 1) {
+            const hap_problem::Trie &tr = cl.trie;
+            const void *tfn = search ? (const void *)trie_dp_kernel<true> : (const void *)trie_dp_kernel<false>;
+            static size_t trie_limit[64][2];
+            if (tr.smem > trie_limit[dev][search ? 1 : 0]) {
+                CUDA_TRY(p, cudaFuncSetAttribute(tfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tr.smem));
+                trie_limit[dev][search ? 1 : 0] = tr.smem;
+            }
+            CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
+            // candidate decode of this pass, then its stage bytes into the tree
+            const u64 nmap = tr.meta.nmap;
+            maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, p->items[cl.item_lo].p, nmap, p->d_maptab + cl.map_base);
+            CUDA_TRY(p, cudaGetLastError());
+            const u32 n_g = tr.n_nodes + (u32)nmap;
+            trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, tr.n_nodes, (u32)nmap, tr.d_first_leaf, tr.d_depth, tr.d_nodes, tr.d_leaves);
+            CUDA_TRY(p, cudaGetLastError());
+            unsigned n_active = tr.n_conf, used = cl.masks_used;
+            int ms = cl.multiset ? 1 : 0;
+            const u32 *plist = tr.d_plist;
+            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tr.meta,
+                             (void *)&o, (void *)&used, (void *)&ms};
+            const unsigned tblocks = search ? blocks : tr.n_conf;       // search: every partial slot of the class is written
+            CUDA_TRY(p, cudaLaunchKernel(tfn, dim3(tblocks), dim3(tr.threads), targs, tr.smem, cl.stream));
+            CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
+            CUDA_TRY(p, cudaStreamWaitEvent(st, cl.done, 0));
+            continue;
+        }
         const WorkItem *its = p->d_items + cl.item_lo;
         int nw = cl.warps;
         unsigned used = cl.masks_used;

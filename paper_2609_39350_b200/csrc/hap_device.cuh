@@ -595,13 +595,14 @@ struct MaskInfo {
 
 // Block prologue shared by the DP kernels: everything that depends on the configuration only.
 // All threads of the block call it; it ends with a barrier.
+// Part 1: stage-time prefix rows per type mask, byte prefixes, per-mask stage info, p2p coefficients.
 template <typename VT, bool LINEAR>
-__device__ __forceinline__ void dp_block_prologue(
-    const DevConst &dc, const hap_pconf &pc, unsigned p_index, const VT *c2, const i64 *coef, const VT *coefv,
+__device__ __forceinline__ void dp_prologue_rows(
+    const DevConst &dc, unsigned p_index, const VT *c2, const i64 *coef, const VT *coefv,
     bool multiset, int mrows, int RW, unsigned masks_used, int nwarps,
-    VT *sR, i64 *sW, i64 *sA, uint8_t *thr, uint8_t *sK, MaskInfo<VT> *minfo, VT (*sP2P)[6], VT *szero, int (*winT)[2])
+    VT *sR, i64 *sW, i64 *sA, uint8_t *sK, MaskInfo<VT> *minfo, VT (*sP2P)[6], VT *szero)
 {
-    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP;
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nmask = (1 << T) - 1;
     // ---- block prologue 1: rows of this configuration -----------------------------------
@@ -690,7 +691,16 @@ __device__ __forceinline__ void dp_block_prologue(
     }
     if (threadIdx.x == 0) szero[0] = 0;
     __syncthreads();
+}
 
+// Part 2: memory-threshold tables and the per-type load-balance window.
+template <typename VT>
+__device__ __forceinline__ void dp_prologue_thr(
+    const DevConst &dc, const hap_pconf &pc, unsigned p_index, const i64 *coef, bool multiset, int nwarps,
+    const i64 *sW, const i64 *sA, uint8_t *thr, const uint8_t *sK, int (*winT)[2])
+{
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP;
+    const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     // ---- block prologue 2: memory thresholds ----------------------------------------------
     // Feasibility of a span (k, j] is monotone: a shorter span needs no more memory, and the first
     // feasible k does not decrease with j.  One thread sweeps j for one (stage, capacity type, level).
@@ -744,7 +754,17 @@ __device__ __forceinline__ void dp_block_prologue(
         winT[threadIdx.x][0] = lo; winT[threadIdx.x][1] = hi;
     }
     __syncthreads();
+}
 
+template <typename VT, bool LINEAR>
+__device__ __forceinline__ void dp_block_prologue(
+    const DevConst &dc, const hap_pconf &pc, unsigned p_index, const VT *c2, const i64 *coef, const VT *coefv,
+    bool multiset, int mrows, int RW, unsigned masks_used, int nwarps,
+    VT *sR, i64 *sW, i64 *sA, uint8_t *thr, uint8_t *sK, MaskInfo<VT> *minfo, VT (*sP2P)[6], VT *szero, int (*winT)[2])
+{
+    dp_prologue_rows<VT, LINEAR>(dc, p_index, c2, coef, coefv, multiset, mrows, RW, masks_used, nwarps,
+                                 sR, sW, sA, sK, minfo, sP2P, szero);
+    dp_prologue_thr<VT>(dc, pc, p_index, coef, multiset, nwarps, sW, sA, thr, sK, winT);
 }
 
 // two blocks of up to 12 warps per SM: the register cap (85) keeps the occupancy independent of ptxas' heuristics

@@ -1,0 +1,354 @@
+// Prefix-tree form of the min-max pipeline recurrence (sm_100a).
+//
+// The DP row of stage d of a candidate depends only on the candidate's stages 1..d (their device
+// types, boundary links and load-balance windows), the configuration and the recomputation policy.
+// All mappings of a PP class therefore form a prefix tree whose nodes are distinct stage prefixes;
+// the tree, the band of reachable end layers of every node and the flat list of (node, end layer)
+// cells of every depth depend on the class alone and are built once on the host.
+//
+//   trie_dp_kernel   one block per configuration.  After the block prologue (stage rows, memory
+//                    thresholds) the block walks the tree depth by depth: one thread per cell
+//                    (node, j) runs the split loop over k against the parent node's row; rows of two
+//                    consecutive depths live in shared memory, split choices of all depths as bytes.
+//                    Then one thread per mapping evaluates the last stage's single cell (PP, N), walks
+//                    the split choices back through the node's ancestors and assembles Eq. 4.
+//                    Integer mode with level-combined rows only; every other mode runs in
+//                    pipeline_dp_kernel.
+#pragma once
+#include "hap_device.cuh"
+
+namespace hap {
+
+struct TrieNode {            // a distinct prefix of stages 1..d, d < PP               (16 bytes)
+    u32 rowoff;              // first cell of the node's row within its depth
+    u32 prowoff;             // the same for the parent node (depth d-1)
+    uint8_t mask, link;      // stage d: device types, boundary link into the stage
+    uint8_t nmin, nmax;      // stage d: load-balance window on the layer count
+    uint8_t bl, bh;          // band of end layers of stage d (union over the mappings below the node)
+    uint8_t pbl, pbh;        // the parent's band (stage 0: {0})
+};
+
+struct TrieLeaf {            // one mapping: its last stage                              (16 bytes)
+    u32 prowoff;             // row of the node of depth PP-1
+    uint16_t parent;         // that node's index within its depth
+    uint8_t mask, link, nmin, nmax, pbl, pbh;
+    uint8_t dead;            // the windows of this mapping cannot add up to N
+    uint8_t pad[3];
+};
+
+struct TrieMeta {
+    const TrieNode *nodes;          // grouped by depth
+    const uint16_t *parent;         // per node: index of its parent within depth d-1
+    const uint16_t *cell_node;      // per cell: index of its node within the depth
+    const TrieLeaf *leaves;         // [nmap]
+    u32 node_lo[HAP_MAX_PP + 1];    // nodes of depth d: [node_lo[d], node_lo[d+1]), d = 1..PP-1
+    u32 cell_lo[HAP_MAX_PP + 1];    // cells of depth d: [cell_lo[d], cell_lo[d+1])
+    u32 buf_cells[2];               // largest row storage of an even / odd depth, in cells
+    u32 nmap;
+    int PP;
+};
+
+__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, bool multiset, u32 buf_even, u32 buf_odd, u32 cells)
+{
+    const size_t n1 = (size_t)N + 1;
+    const size_t mrows = multiset ? (size_t)T : (size_t)((1 << T) - 1);
+    size_t b = mrows * (size_t)R * n1 * 8 + n1 * 16;
+    b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    b += (n1 + 15) / 16 * 16;
+    b += ((size_t)buf_even + buf_odd) * 8;
+    b += ((size_t)cells + 15) / 16 * 16;
+    return b + 32;
+}
+
+// Copies the stage bytes (device types, boundary link) that the decode of this pass produced into the
+// tree: node n of depth d takes stage d of the first mapping below it, leaf m the last stage of mapping m.
+__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 nmap,
+                                   const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
+                                   TrieNode *nodes, TrieLeaf *leaves)
+{
+    const u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g < n_nodes) {
+        const uint8_t *src = maptab + ((u64)first_leaf[g] * PP + (depth[g] - 1)) * 2;
+        nodes[g].mask = src[0]; nodes[g].link = src[1];
+    } else if (g < n_nodes + nmap) {
+        const u32 m = g - n_nodes;
+        const uint8_t *src = maptab + ((u64)m * PP + (PP - 1)) * 2;
+        leaves[m].mask = src[0]; leaves[m].link = src[1];
+    }
+}
+
+template <bool SEARCH>
+__global__ void __launch_bounds__(1024, 1)
+trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64 *c2, const i64 *coef,
+               const TrieMeta tm, DpOut out, unsigned masks_used, int multiset_i)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ MaskInfo<i64> minfo[kMaxMasks];
+    __shared__ i64 sP2P[HAP_MAX_TYPES][6];
+    __shared__ i64 szero[1];
+    __shared__ int winT[HAP_MAX_TYPES][2];
+    __shared__ i64 wcost[32];
+    __shared__ u64 widx[32];
+    __shared__ int s_skip;
+
+    const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, lane = tid & 31, wib = tid >> 5;
+    if (blockIdx.x >= n_active) {
+        if (SEARCH && tid == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
+        return;
+    }
+    const u32 p = plist[blockIdx.x];
+    const hap_pconf pc = dc.pconf[p];
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc;
+    const bool multiset = multiset_i != 0;
+    const u64 c_lo = pc.offset, c_hi = pc.offset + (u64)tm.nmap * n_rc;        // candidates of this configuration
+    const u64 w_lo = out.first, w_hi = out.first + out.count;                  // candidates that are wanted
+    if (c_hi <= w_lo || c_lo >= w_hi) {
+        if (SEARCH && tid == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
+        return;
+    }
+    if (SEARCH && out.prune) {
+        // T_iter >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on the summed stage time; one
+        // thread reads the moving incumbent and the block follows that reading as a whole
+        if (tid == 0) {
+            const i64 S = out.lb_sum[p];
+            const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
+            const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+            s_skip = (u64)lb > inc;
+            if (s_skip) {
+                out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
+                const u64 a = c_lo > w_lo ? c_lo : w_lo, b = c_hi < w_hi ? c_hi : w_hi;
+                atomicAdd(out.counters + 2, b - a);
+            }
+        }
+        __syncthreads();
+        if (s_skip) return;
+    }
+
+    const int nmask = (1 << T) - 1;
+    const int mrows = multiset ? T : nmask;
+    i64 *sR = reinterpret_cast<i64 *>(smem_raw);
+    i64 *sW = sR + (size_t)mrows * R * n1;
+    i64 *sA = sW + n1;
+    uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
+    const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    uint8_t *sK = thr + thr_bytes;
+    i64 *bufE = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);    // rows of the even depths
+    i64 *bufO = bufE + tm.buf_cells[0];                                        // rows of the odd depths
+    uint8_t *ch = reinterpret_cast<uint8_t *>(bufO + tm.buf_cells[1]);         // split choices, all depths
+
+    dp_prologue_rows<i64, true>(dc, p, c2, coef, coef, multiset, mrows, R, masks_used, nwarps, sR, sW, sA, sK, minfo, sP2P, szero);
+    const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
+
+    // writes "infeasible" for mapping m under policy rc_idx (non-search mode)
+    auto put_infeasible = [&](u64 c) {
+        const u64 o = c - out.first;
+        if (out.cost) out.cost[o] = kInf;
+        if (out.bottleneck) out.bottleneck[o] = kInf;
+        if (out.detail) { out.detail[o * 3] = kInf; out.detail[o * 3 + 1] = 0; out.detail[o * 3 + 2] = 0; }
+        if (out.partition) for (int s = 0; s < HAP_MAX_PP; ++s) out.partition[o * HAP_MAX_PP + s] = 0;
+        if (out.recompute) for (int s = 0; s < HAP_MAX_PP; ++s) out.recompute[o * HAP_MAX_PP + s] = 0;
+    };
+
+    i64 best_cost = kInf;
+    u64 best_index = ~0ull;
+    u64 n_eval = 0, n_feas = 0, n_cells = 0;
+    unsigned all_levels = 0;
+    for (int q = 0; q < n_rc; ++q) all_levels |= dc.rc_masks[q];
+
+    // ---- configurations whose first stage fits no device type at any level: nothing is feasible ----------
+    bool config_dead = false;
+    if (PP > 1) {
+        const u32 n_first = tm.node_lo[2] - tm.node_lo[1];
+        int fits = 0;
+        for (u32 e = tid; e < n_first * (u32)R; e += nthreads) {
+            const u32 nd_i = e / R; const int r = (int)(e % R);
+            if (!((all_levels >> r) & 1u)) continue;
+            const TrieNode nd = tm.nodes[tm.node_lo[1] + nd_i];
+            if (nd.bl > nd.bh) continue;
+            const int capt = minfo[nd.mask - 1].capt;
+            const i64 mstore = pc.M < PP ? pc.M : PP;
+            // feasibility is monotone in the span: the shortest span the band allows decides
+            fits |= span_fits(sW, sA, sK, cfp[HAP_MPRE], cfp[HAP_MX], mstore, dc.cap_eff[capt], dc.xi_q[r], 0, nd.bl);
+        }
+        config_dead = !__syncthreads_or(fits);
+    }
+    if (!config_dead) dp_prologue_thr<i64>(dc, pc, p, coef, multiset, nwarps, sW, sA, thr, sK, winT);
+
+    auto stage_K = [&](int d, int mask, int link) -> i64 {
+        i64 K = 0;
+        const MaskInfo<i64> &mi = minfo[mask - 1];
+        if (d == 1) K += mi.kpre;
+        if (d == PP) K += mi.kpost;
+        if (d > 1) { const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3; K += sP2P[hb][cls == HAP_CROSS ? 2 + ha : cls]; }
+        return K;
+    };
+
+    // one cell: min over k in [klo, khi] of max(prev[k], cost(k, j)), smallest k on ties; k runs downward over
+    // the level segments given by the memory thresholds (lowest allowed level that fits)
+    auto cell = [&](int d, int j, int mask, int link, int klo, int khi, const i64 *prev, unsigned rc_mask, i64 &best, int &arg) {
+        best = kInf; arg = 255;
+        if (klo > khi) return;
+        const int mrow = multiset ? __ffs(mask) - 1 : mask - 1;
+        const i64 K = stage_K(d, mask, link);
+        const i64 *rM = sR + (size_t)mrow * R * n1;
+        const uint8_t *th = thr + ((size_t)(d - 1) * T + minfo[mask - 1].capt) * R * n1;
+        int seg_hi = khi;
+        for (int r = 0; r < R && seg_hi >= klo; ++r) {
+            if (!((rc_mask >> r) & 1u)) continue;
+            int lo = th[(size_t)r * n1 + j];
+            if (lo < klo) lo = klo;
+            if (lo > seg_hi) continue;
+            n_cells += (u64)(seg_hi - lo + 1);
+            const i64 *rr = rM + (size_t)r * n1;
+            const i64 Cj = rr[j] + K;
+            for (int k = seg_hi; k >= lo; --k) {
+                const i64 pv = prev[k];
+                const i64 cst = Cj - rr[k];
+                const i64 v = pv > cst ? pv : cst;
+                if (v <= best && v < kInf) { best = v; arg = k; }
+            }
+            seg_hi = lo - 1;
+        }
+    };
+
+    unsigned policies_without_plan = 0;                      // positions in rc_order under which no mapping was feasible
+    for (int rc_pos = 0; rc_pos < n_rc; ++rc_pos) {
+        const int rc_idx = dc.rc_order[rc_pos];
+        const unsigned rc_mask = dc.rc_masks[rc_idx];
+        bool dead = config_dead || (dc.rc_sup[rc_pos] & policies_without_plan) != 0;
+
+        // ---- rows of the tree, depth by depth ------------------------------------------------
+        if (!dead) {
+            for (int d = 1; d < PP; ++d) {
+                const u32 ncell = tm.cell_lo[d + 1] - tm.cell_lo[d];
+                const TrieNode *nd_base = tm.nodes + tm.node_lo[d];
+                const uint16_t *cnode = tm.cell_node + tm.cell_lo[d];
+                uint8_t *chd = ch + tm.cell_lo[d];
+                i64 *cur = (d & 1) ? bufO : bufE;
+                const i64 *prevbuf = d == 1 ? szero : ((d & 1) ? bufE : bufO);
+                int alive = 0;
+                for (u32 e = tid; e < ncell; e += nthreads) {
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(nd_base + cnode[e]));
+                    const u32 rowoff = raw.x, prowoff = raw.y;
+                    const int mask = raw.z & 255, link = (raw.z >> 8) & 255, nmin = (raw.z >> 16) & 255, nmax = raw.z >> 24;
+                    const int bl = raw.w & 255, pbl = (raw.w >> 16) & 255, pbh = raw.w >> 24;
+                    const int j = bl + (int)(e - rowoff);
+                    int klo = j - nmax; if (klo < pbl) klo = pbl;
+                    int khi = j - nmin; if (khi > pbh) khi = pbh;
+                    i64 best; int arg;
+                    cell(d, j, mask, link, klo, khi, prevbuf + prowoff - pbl, rc_mask, best, arg);
+                    cur[e] = best;
+                    chd[e] = (uint8_t)arg;
+                    alive |= best < kInf;
+                }
+                if (!__syncthreads_or(alive)) { dead = true; break; }   // no cell of this depth is finite: nothing below is
+            }
+        }
+
+        // ---- one thread per mapping: cell (PP, N), backtrace, Eq. 4 ---------------------------------
+        int any_plan = 0;
+        const i64 *lastbuf = PP == 1 ? szero : (((PP - 1) & 1) ? bufO : bufE);
+        for (u32 m = tid; m < tm.nmap; m += nthreads) {
+            const u64 c = pc.offset + (u64)m * n_rc + (u64)rc_idx;
+            if (c < w_lo || c >= w_hi) continue;
+            i64 bott = kInf; int arg = 255;
+            TrieLeaf lf;
+            if (!dead) {
+                const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(tm.leaves + m));
+                lf.prowoff = raw.x; lf.parent = (uint16_t)(raw.y & 0xffff); lf.mask = (raw.y >> 16) & 255; lf.link = raw.y >> 24;
+                lf.nmin = raw.z & 255; lf.nmax = (raw.z >> 8) & 255; lf.pbl = (raw.z >> 16) & 255; lf.pbh = raw.z >> 24;
+                lf.dead = raw.w & 255;
+                if (!lf.dead) {
+                    int klo = N - lf.nmax; if (klo < lf.pbl) klo = lf.pbl;
+                    int khi = N - lf.nmin; if (khi > lf.pbh) khi = lf.pbh;
+                    cell(PP, N, lf.mask, lf.link, klo, khi, lastbuf + lf.prowoff - lf.pbl, rc_mask, bott, arg);
+                }
+            }
+            if (SEARCH) n_eval++;
+            if (!(bott < kInf)) {
+                if (!SEARCH) put_infeasible(c);
+                continue;
+            }
+            // backtrace from (PP, N) through the ancestors; per stage: level, cost, sync and optimizer terms
+            i64 sum = 0, mxc = 0, t_sync = 0, t_opt = 0, het = 0;
+            const u64 o = c - out.first;
+            int b = N, a = arg, mask = lf.mask, link = lf.link;
+            u32 node = lf.parent;
+            for (int d = PP; d >= 1; --d) {
+                const MaskInfo<i64> &mi = minfo[mask - 1];
+                const uint8_t *th = thr + ((size_t)(d - 1) * T + mi.capt) * R * n1;
+                int r = 0;
+                for (; r < R; ++r)
+                    if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b] <= a) break;
+                const int mrow = multiset ? __ffs(mask) - 1 : mask - 1;
+                const i64 *rr = sR + ((size_t)mrow * R + r) * n1;
+                const i64 cst = (rr[b] - rr[a]) + stage_K(d, mask, link);
+                sum += cst; mxc = cst > mxc ? cst : mxc;
+                const i64 n_moe = (i64)((int)sK[b] - (int)sK[a]), n_dense = (i64)(b - a) - n_moe;
+                const i64 sy = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
+                const i64 op = n_dense * mi.opt[0] + n_moe * mi.opt[1];
+                t_sync = sy > t_sync ? sy : t_sync; t_opt = op > t_opt ? op : t_opt;
+                if (dc.eta_q > 0 && d > 1 && (link & 3) == HAP_CROSS) het += sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
+                if (!SEARCH) {
+                    if (out.partition) out.partition[o * HAP_MAX_PP + d - 1] = (uint8_t)(b - a);
+                    if (out.recompute) out.recompute[o * HAP_MAX_PP + d - 1] = (uint8_t)r;
+                }
+                if (d > 1) {
+                    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(tm.nodes + tm.node_lo[d - 1] + node));
+                    const u32 parent = tm.parent[tm.node_lo[d - 1] + node];
+                    b = a;
+                    a = ch[tm.cell_lo[d - 1] + raw.x + (u32)(b - (int)(raw.w & 255))];
+                    mask = raw.z & 255; link = (raw.z >> 8) & 255;
+                    node = parent;
+                }
+            }
+            i64 T_pipe = sum + (i64)(pc.M - 1) * mxc;
+            i64 T_iter = T_pipe + t_sync + t_opt;
+            if (dc.eta_q > 0 && het * (i64)PP * 1024 > (i64)dc.eta_q * sum) { T_iter = kInf; T_pipe = kInf; }   // Pruning 3
+            if (SEARCH) {
+                if (T_iter < kInf) { n_feas++; any_plan = 1; }
+                if (T_iter < best_cost || (T_iter == best_cost && c < best_index)) { best_cost = T_iter; best_index = c; }
+            } else {
+                any_plan = 1;
+                if (out.cost) out.cost[o] = T_iter;
+                if (out.bottleneck) out.bottleneck[o] = bott;
+                if (out.detail) { out.detail[o * 3] = T_pipe; out.detail[o * 3 + 1] = t_sync; out.detail[o * 3 + 2] = t_opt; }
+                if (!(T_iter < kInf)) {
+                    if (out.partition) for (int s = 0; s < PP; ++s) out.partition[o * HAP_MAX_PP + s] = 0;
+                    if (out.recompute) for (int s = 0; s < PP; ++s) out.recompute[o * HAP_MAX_PP + s] = 0;
+                }
+                if (out.partition) for (int s = PP; s < HAP_MAX_PP; ++s) out.partition[o * HAP_MAX_PP + s] = 0;
+                if (out.recompute) for (int s = PP; s < HAP_MAX_PP; ++s) out.recompute[o * HAP_MAX_PP + s] = 0;
+            }
+        }
+        // the barrier also keeps the next policy from overwriting rows and choices that are still being read
+        const int bott_any = __syncthreads_or(any_plan);
+        // a policy under which no mapping of the WHOLE configuration has a feasible partition settles its subsets
+        if (!bott_any && c_lo >= w_lo && c_hi <= w_hi && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
+    }
+
+    if (out.counters) {
+        n_cells = (u64)warp_sum_i64((i64)n_cells);
+        if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
+    }
+    if (SEARCH) {
+        n_eval = (u64)warp_sum_i64((i64)n_eval); n_feas = (u64)warp_sum_i64((i64)n_feas);
+        warp_argmin(best_cost, best_index);
+        if (lane == 0) {
+            wcost[wib] = best_cost; widx[wib] = best_index;
+            if (n_eval) atomicAdd(out.counters + 0, n_eval);
+            if (n_feas) atomicAdd(out.counters + 1, n_feas);
+        }
+        __syncthreads();
+        if (tid == 0) {
+            i64 bc = wcost[0]; u64 bi = widx[0];
+            for (int q = 1; q < nwarps; ++q)
+                if (wcost[q] < bc || (wcost[q] == bc && widx[q] < bi)) { bc = wcost[q]; bi = widx[q]; }
+            out.partial_cost[blockIdx.x] = bc;
+            out.partial_index[blockIdx.x] = bi;
+            if (out.prune && bc < kInf) atomicMin(out.incumbent, (u64)bc);
+        }
+    }
+}
+
+}  // namespace hap

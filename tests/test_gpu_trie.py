@@ -1,0 +1,129 @@
+"""The prefix-tree form of the pipeline recurrence (trie_dp_kernel) against the oracle and against
+the one-warp-per-candidate kernel (HAP_OPT_NO_TRIE), through the C ABI.  Integer work: bit-exact."""
+import os
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from gen import problems  # noqa: E402
+from oracle import Oracle, INF  # noqa: E402
+
+NTHREADS = max(1, len(os.sched_getaffinity(0)))
+
+
+@pytest.fixture(scope="module")
+def hap():
+    import paper_2609_39350_b200 as hap
+    from paper_2609_39350_b200.build import build_library
+    build_library()
+    assert torch.cuda.is_available(), "the gpu tests need a CUDA device"
+    return hap
+
+
+def _pass(hap, pb, flags, first=0, count=None, partition=True):
+    hp = hap.hap_problem_create(pb, flags=flags)
+    hap.hap_enumerate(hp)
+    if count is None:
+        count = hp.n_cand - first
+    out = hap.hap_pipeline_dp(hp, first, count, partition=partition)
+    torch.cuda.synchronize()
+    res = {k: v.cpu().numpy() for k, v in out.items() if v is not None}
+    return hp, res
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("tiny", {"window": True}), ("small", {}), ("mixtral", {}), ("dsv2", {}), ("stress", {})])
+def test_both_kernels_agree_on_every_candidate(hap, name, kw):
+    """Costs, bottlenecks, partitions and recomputation levels of the whole candidate space."""
+    pb = problems.make_problem(name, **kw)
+    hp_t, tree = _pass(hap, pb, 0)
+    hp_w, warp = _pass(hap, pb, hap.OPT_NO_TRIE)
+    for key in ("cost", "bottleneck", "partition", "recompute"):
+        bad = np.nonzero((tree[key] != warp[key]).reshape(len(tree[key]), -1).any(axis=1))[0]
+        assert bad.size == 0, (key, bad[:8])
+    # and the oracle on a sample (the full comparison with the oracle runs in test_gpu_parity)
+    o = Oracle(pb)
+    rng = np.random.default_rng(11)
+    for idx in rng.integers(0, o.n_cand, 200).tolist():
+        plan, _, _ = o.eval_index(idx)
+        assert tree["cost"][idx] == plan["T_iter"] and tree["bottleneck"][idx] == plan["bottleneck"], idx
+        if plan["T_iter"] < INF:
+            PP = plan["PP"]
+            assert tree["partition"][idx, :PP].tolist() == plan["n"] and tree["recompute"][idx, :PP].tolist() == plan["r"], idx
+            assert not tree["partition"][idx, PP:].any()
+        else:
+            assert not tree["partition"][idx].any() and not tree["recompute"][idx].any()
+    # searches, with and without pruning, return the same plan
+    plan_t, st_t = hap.hap_search_best(hp_t)
+    plan_w, st_w = hap.hap_search_best(hp_w)
+    assert plan_t == plan_w
+    assert st_t["n_evaluated"] == st_w["n_evaluated"] == o.n_cand and st_t["n_feasible"] == st_w["n_feasible"]
+    am = int(np.argmin(tree["cost"]))
+    assert plan_t["index"] == am and plan_t["T_iter"] == int(tree["cost"][am])
+    hap.hap_problem_destroy(hp_t)
+    hap.hap_problem_destroy(hp_w)
+    hp_p = hap.hap_problem_create(pb, prune=1)
+    hap.hap_enumerate(hp_p)
+    plan_p, st_p = hap.hap_search_best(hp_p)
+    assert plan_p == plan_t and st_p["n_evaluated"] + st_p["n_pruned"] == o.n_cand
+    hap.hap_problem_destroy(hp_p)
+
+
+def test_ragged_ranges_across_configurations(hap):
+    """Ranges that start and end inside a configuration's candidates; everything outside stays untouched."""
+    pb = problems.small()
+    o = Oracle(pb)
+    costs, bn, best, feas = o.search(0, o.n_cand)
+    hp = hap.hap_problem_create(pb)
+    hap.hap_enumerate(hp)
+    rng = np.random.default_rng(5)
+    for first, count in [(0, 2), (1, 7), (o.n_cand - 3, 3)] + [(int(a), int(b)) for a, b in zip(rng.integers(0, o.n_cand - 5000, 6), rng.integers(2, 5000, 6))]:
+        out = hap.hap_pipeline_dp(hp, first, count, partition=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(out["cost"].cpu().numpy(), costs[first:first + count]), (first, count)
+        assert np.array_equal(out["bottleneck"].cpu().numpy(), bn[first:first + count]), (first, count)
+        sub = costs[first:first + count]
+        if sub.min() >= INF:
+            with pytest.raises(hap.HapError) as e:
+                hap.hap_search_range(hp, first, count)
+            assert e.value.name == "HAP_E_INFEASIBLE"
+            continue
+        plan, stats = hap.hap_search_range(hp, first, count)
+        assert plan["T_iter"] == int(sub.min()) and plan["index"] == first + int(np.argmin(sub))
+        assert stats["n_evaluated"] == count
+    hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_problems_with_tight_memory_and_windows(hap, seed):
+    """Small random problems (several types, tight capacities, general recomputation levels where the
+    level-combined rows exist) against the oracle, every candidate."""
+    pb = problems.random_small(20 + seed, N=8 + seed % 5, T=2 + seed % 2, nodes_per_type=((2, 2), (2, 1, 1))[seed % 2],
+                               node_size=2, window=(seed % 3 != 0), first_dense=(seed % 2 == 0))
+    if seed >= 3:       # three levels whose time factors are multiples of 1024, policies that skip a level
+        pb.xi_q = np.ascontiguousarray(np.array([1024, 512, 64], np.int32))
+        pb.tau_q = np.ascontiguousarray(np.array([0, 1024, 2048], np.int32))
+        pb.rc_masks = np.ascontiguousarray(np.array([0b001, 0b011, 0b111, 0b101], np.uint32))
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=NTHREADS, want_costs=True)
+    hp, tree = _pass(hap, pb, 0)
+    assert np.array_equal(tree["cost"], costs) and np.array_equal(tree["bottleneck"], bn)
+    for idx in range(0, o.n_cand, max(1, o.n_cand // 200)):
+        plan, _, _ = o.eval_index(idx)
+        if plan["T_iter"] < INF:
+            assert tree["partition"][idx, :plan["PP"]].tolist() == plan["n"] and tree["recompute"][idx, :plan["PP"]].tolist() == plan["r"], idx
+    hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("name,eta_q", [("tiny", 16), ("small", 24)])
+def test_heterogeneous_communication_rule_in_the_tree_kernel(hap, name, eta_q):
+    pb = problems.make_problem(name)
+    pb.eta_q = eta_q
+    o = Oracle(pb)
+    done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=NTHREADS, want_costs=True)
+    hp, tree = _pass(hap, pb, 0)
+    assert np.array_equal(tree["cost"], costs) and np.array_equal(tree["bottleneck"], bn)
+    assert (costs >= INF).sum() > (bn >= INF).sum()          # the rule dropped some candidates with a feasible partition
+    hap.hap_problem_destroy(hp)
