@@ -35,8 +35,8 @@ struct hap_problem {
     uint64_t n_cand = 0;
     std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
     // prefix tree of a class's mappings (trie_dp_kernel); ok = false: the class runs in pipeline_dp_kernel only
-    struct Trie { bool ok; TrieMeta meta; unsigned char *d_blob; u32 *d_first_leaf; uint8_t *d_depth; TrieNode *d_nodes; TrieLeaf *d_leaves;
-                  u32 *d_plist; unsigned n_conf; u32 n_nodes; int threads; size_t smem; };
+    struct Trie { bool ok; TrieMeta meta; unsigned char *d_blob; u32 *d_first_leaf, *d_gnode; uint8_t *d_depth; TrieNode *d_nodes; TrieLeaf *d_leaves;
+                  TrieCell *d_cells; u32 *d_plist; unsigned n_conf; u32 n_nodes, n_cells; int threads; size_t smem; };
     struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
@@ -331,6 +331,11 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
         for (int h = 0; h < T; ++h) if (mk >> h & 1) { if (!seen || p->P[h] < v) v = p->P[h]; seen = true; }
         Pmin[mk] = v;
     }
+    int capt_of[1 << HAP_MAX_TYPES] = {0};                      // type whose (smallest) memory binds a stage of these types
+    for (int mk = 1; mk < (1 << T); ++mk) {
+        i64 cap = 0; bool seen = false;
+        for (int h = 0; h < T; ++h) if (mk >> h & 1) { if (!seen || p->cap_eff[h] < cap) { cap = p->cap_eff[h]; capt_of[mk] = h; } seen = true; }
+    }
     const int delta_q = p->opts.delta_q;
     const bool uniform = (p->opts.flags & HAP_OPT_UNIFORM) != 0;
     std::vector<int> nmin(PP + 1), nmax(PP + 1), bl(PP + 1), bh(PP + 1);
@@ -373,6 +378,7 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
         lf.mask = row[(PP - 1) * 2]; lf.link = row[(PP - 1) * 2 + 1];
         lf.nmin = (uint8_t)nmin[PP]; lf.nmax = (uint8_t)nmax[PP];
         lf.dead = dead ? 1 : 0;
+        lf.capt = (uint8_t)capt_of[lf.mask];
         if (dead) continue;
         int d0 = 1;                                              // first depth at which a new node is needed
         if (have_prev)
@@ -417,8 +423,19 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     tm.buf_cells[0] = (tm.buf_cells[0] + 1) / 2 * 2; tm.buf_cells[1] = (tm.buf_cells[1] + 1) / 2 * 2;
     const size_t smem = trie_smem_bytes(N, PP, T, R, cl.multiset, tm.buf_cells[0], tm.buf_cells[1], n_cells);
     if (smem > 220 * 1024) return false;
+    if (n_cells >= (1u << 25)) return false;
     std::vector<TrieNode> nodes(n_nodes);
-    std::vector<uint16_t> parent(n_nodes), cell_node(n_cells);
+    std::vector<uint16_t> parent(n_nodes);
+    std::vector<TrieCell> cells(n_cells);
+    std::vector<u32> cell_gnode(n_cells);
+    int band_max = 1;
+    for (int d = 1; d <= PP; ++d) { tm.jlo[d] = 255; tm.jhi[d] = 0; tm.wmax[d] = 0; tm.tmask[d] = 0; tm.kmin[d] = 255; tm.kmax[d] = 0; }
+    tm.jlo[PP] = tm.jhi[PP] = (uint8_t)N;
+    for (u64 m = 0; m < nmap; ++m) {
+        if (leaves[m].dead) continue;
+        tm.wmax[PP] = std::max(tm.wmax[PP], leaves[m].nmax);
+        tm.tmask[PP] |= (uint8_t)(1u << leaves[m].capt);
+    }
     std::vector<u32> first_leaf(n_nodes);
     std::vector<uint8_t> depth(n_nodes);
     for (int d = 1; d < PP; ++d)
@@ -433,26 +450,47 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
             parent[tm.node_lo[d] + i] = (uint16_t)h.parent;
             first_leaf[tm.node_lo[d] + i] = h.first_leaf;
             depth[tm.node_lo[d] + i] = (uint8_t)d;
-            for (int j = h.bl; j <= h.bh; ++j) cell_node[tm.cell_lo[d] + rowoff[d][i] + (u32)(j - h.bl)] = (uint16_t)i;
+            tm.jlo[d] = std::min<uint8_t>(tm.jlo[d], nd.bl); tm.jhi[d] = std::max<uint8_t>(tm.jhi[d], nd.bh);
+            tm.wmax[d] = std::max(tm.wmax[d], nd.nmax);
+            tm.tmask[d] |= (uint8_t)(1u << capt_of[nd.mask]);
+            for (int j = h.bl; j <= h.bh; ++j) {
+                int klo = std::max(j - (int)nd.nmax, (int)nd.pbl), khi = std::min(j - (int)nd.nmin, (int)nd.pbh);
+                if (klo > khi) { klo = 1; khi = 0; }
+                else { tm.kmin[d] = std::min<uint8_t>(tm.kmin[d], (uint8_t)klo); tm.kmax[d] = std::max<uint8_t>(tm.kmax[d], (uint8_t)khi); }
+                const u32 c = tm.cell_lo[d] + rowoff[d][i] + (u32)(j - h.bl);
+                cells[c].x = (u32)((int)nd.prowoff - (int)nd.pbl + 256) | ((u32)nd.link << 26);
+                cells[c].y = (u32)j | ((u32)klo << 8) | ((u32)khi << 16) | ((u32)(nd.mask & 15) << 24) | ((u32)capt_of[nd.mask] << 28);
+                cell_gnode[c] = tm.node_lo[d] + (u32)i;
+            }
         }
+    for (int d = 1; d <= PP; ++d) if (tm.jlo[d] <= tm.jhi[d]) band_max = std::max(band_max, tm.jhi[d] - tm.jlo[d] + 1);
+    tm.band_max = band_max;
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];
         if (lf.dead || PP == 1) { lf.prowoff = 0; lf.pbl = 0; lf.pbh = 0; continue; }
         const HNode &ph = lv[PP - 1][lf.parent];
         lf.prowoff = rowoff[PP - 1][lf.parent]; lf.pbl = (uint8_t)ph.bl; lf.pbh = (uint8_t)ph.bh;
     }
-    // one allocation: nodes | leaves | first_leaf | parent | cell_node | depth
+    for (u64 m = 0; m < nmap; ++m) {
+        const TrieLeaf &lf = leaves[m];
+        if (lf.dead) continue;
+        const int klo = std::max(N - (int)lf.nmax, (int)lf.pbl), khi = std::min(N - (int)lf.nmin, (int)lf.pbh);
+        if (klo <= khi) { tm.kmin[PP] = std::min<uint8_t>(tm.kmin[PP], (uint8_t)klo); tm.kmax[PP] = std::max<uint8_t>(tm.kmax[PP], (uint8_t)khi); }
+    }
+    // one allocation: nodes | leaves | cells | first_leaf | cell_gnode | parent | depth
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
     const size_t o_nodes = 0, o_leaves = up(o_nodes + (size_t)n_nodes * sizeof(TrieNode));
-    const size_t o_first = up(o_leaves + nmap * sizeof(TrieLeaf)), o_parent = up(o_first + (size_t)n_nodes * 4);
-    const size_t o_cell = up(o_parent + (size_t)n_nodes * 2), o_depth = up(o_cell + (size_t)n_cells * 2);
+    const size_t o_cells = up(o_leaves + nmap * sizeof(TrieLeaf));
+    const size_t o_first = up(o_cells + (size_t)n_cells * sizeof(TrieCell)), o_gnode = up(o_first + (size_t)n_nodes * 4);
+    const size_t o_parent = up(o_gnode + (size_t)n_cells * 4), o_depth = up(o_parent + (size_t)n_nodes * 2);
     const size_t total = up(o_depth + n_nodes) + 256;
     std::vector<unsigned char> blob(total, 0);
     if (n_nodes) std::memcpy(blob.data() + o_nodes, nodes.data(), (size_t)n_nodes * sizeof(TrieNode));
     std::memcpy(blob.data() + o_leaves, leaves.data(), nmap * sizeof(TrieLeaf));
+    if (n_cells) std::memcpy(blob.data() + o_cells, cells.data(), (size_t)n_cells * sizeof(TrieCell));
     if (n_nodes) std::memcpy(blob.data() + o_first, first_leaf.data(), (size_t)n_nodes * 4);
+    if (n_cells) std::memcpy(blob.data() + o_gnode, cell_gnode.data(), (size_t)n_cells * 4);
     if (n_nodes) std::memcpy(blob.data() + o_parent, parent.data(), (size_t)n_nodes * 2);
-    if (n_cells) std::memcpy(blob.data() + o_cell, cell_node.data(), (size_t)n_cells * 2);
     if (n_nodes) std::memcpy(blob.data() + o_depth, depth.data(), n_nodes);
     if (cudaMalloc(&tr.d_blob, total) != cudaSuccess) { tr.d_blob = nullptr; cudaGetLastError(); return false; }
     if (cudaMemcpy(tr.d_blob, blob.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return false;
@@ -460,11 +498,13 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     if (cudaMemcpy(tr.d_plist, plist.data(), plist.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess) return false;
     tr.d_nodes = reinterpret_cast<TrieNode *>(tr.d_blob + o_nodes);
     tr.d_leaves = reinterpret_cast<TrieLeaf *>(tr.d_blob + o_leaves);
+    tr.d_cells = reinterpret_cast<TrieCell *>(tr.d_blob + o_cells);
     tr.d_first_leaf = reinterpret_cast<u32 *>(tr.d_blob + o_first);
+    tr.d_gnode = reinterpret_cast<u32 *>(tr.d_blob + o_gnode);
     tr.d_depth = tr.d_blob + o_depth;
-    tm.nodes = tr.d_nodes; tm.leaves = tr.d_leaves;
+    tm.nodes = tr.d_nodes; tm.leaves = tr.d_leaves; tm.cells = tr.d_cells;
     tm.parent = reinterpret_cast<const uint16_t *>(tr.d_blob + o_parent);
-    tm.cell_node = reinterpret_cast<const uint16_t *>(tr.d_blob + o_cell);
+    tr.n_cells = n_cells;
     tr.n_conf = (unsigned)plist.size(); tr.n_nodes = n_nodes; tr.smem = smem;
     const u32 want = std::max<u32>(max_level, (u32)nmap);
     int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
@@ -779,8 +819,9 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             const u64 nmap = tr.meta.nmap;
             maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, p->items[cl.item_lo].p, nmap, p->d_maptab + cl.map_base);
             CUDA_TRY(p, cudaGetLastError());
-            const u32 n_g = tr.n_nodes + (u32)nmap;
-            trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, tr.n_nodes, (u32)nmap, tr.d_first_leaf, tr.d_depth, tr.d_nodes, tr.d_leaves);
+            const u32 n_g = tr.n_nodes + tr.n_cells + (u32)nmap;
+            trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, tr.n_nodes, tr.n_cells, (u32)nmap, tr.d_first_leaf, tr.d_depth,
+                                                                          tr.d_gnode, tr.d_nodes, tr.d_cells, tr.d_leaves);
             CUDA_TRY(p, cudaGetLastError());
             unsigned n_active = tr.n_conf, used = cl.masks_used;
             int ms = cl.multiset ? 1 : 0;
@@ -1041,6 +1082,15 @@ extern "C" hap_status hap_get_timings(hap_problem *p, float *ms_layer_cost, floa
     if (cells) CUDA_TRY(p, cudaMemcpy(cells, p->d_counters + 4, sizeof(u64), cudaMemcpyDeviceToHost));
     return check_values(p);
 }
+
+#ifdef HAP_TRIE_TIMERS
+extern "C" hap_status hap_debug_counters(hap_problem *p, uint64_t *host8)
+{
+    CUDA_TRY(p, cudaDeviceSynchronize());
+    CUDA_TRY(p, cudaMemcpy(host8, p->d_counters, 8 * sizeof(u64), cudaMemcpyDeviceToHost));
+    return HAP_OK;
+}
+#endif
 
 static hap_status argmin_launch(hap_problem *p, const i64 *dev_cost, uint64_t count, i64 *dev_out, cudaStream_t st, i64 init)
 {

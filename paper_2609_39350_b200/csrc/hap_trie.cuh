@@ -33,19 +33,29 @@ struct TrieLeaf {            // one mapping: its last stage                     
     uint16_t parent;         // that node's index within its depth
     uint8_t mask, link, nmin, nmax, pbl, pbh;
     uint8_t dead;            // the windows of this mapping cannot add up to N
-    uint8_t pad[3];
+    uint8_t capt;            // device type whose memory binds the stage
+    uint8_t pad[2];
 };
+
+// One cell (node, end layer j) of a depth, everything its split loop needs in 8 bytes:
+//   x = (row origin of the parent in the previous depth's buffer, i.e. prowoff - pbl, + 256) | link << 26
+//   y = j | klo << 8 | khi << 16 | mask << 24 | capt << 28     (klo..khi: window of the stage within the parent's band)
+typedef uint2 TrieCell;
 
 struct TrieMeta {
     const TrieNode *nodes;          // grouped by depth
     const uint16_t *parent;         // per node: index of its parent within depth d-1
-    const uint16_t *cell_node;      // per cell: index of its node within the depth
+    const TrieCell *cells;          // grouped by depth
     const TrieLeaf *leaves;         // [nmap]
     u32 node_lo[HAP_MAX_PP + 1];    // nodes of depth d: [node_lo[d], node_lo[d+1]), d = 1..PP-1
     u32 cell_lo[HAP_MAX_PP + 1];    // cells of depth d: [cell_lo[d], cell_lo[d+1])
+    uint8_t jlo[HAP_MAX_PP + 1], jhi[HAP_MAX_PP + 1];   // end layers that occur at depth d (depth PP: N)
+    uint8_t wmax[HAP_MAX_PP + 1];   // widest window of a stage at depth d
+    uint8_t tmask[HAP_MAX_PP + 1];  // device types whose memory binds some stage of depth d
+    uint8_t kmin[HAP_MAX_PP + 1], kmax[HAP_MAX_PP + 1];   // smallest / largest split any cell of depth d looks at
     u32 buf_cells[2];               // largest row storage of an even / odd depth, in cells
     u32 nmap;
-    int PP;
+    int PP, band_max;               // band_max: most end layers of any depth
 };
 
 __host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, bool multiset, u32 buf_even, u32 buf_odd, u32 cells)
@@ -55,26 +65,168 @@ __host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, b
     size_t b = mrows * (size_t)R * n1 * 8 + n1 * 16;
     b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
     b += (n1 + 15) / 16 * 16;
+    b += (size_t)T * N * 16;                         // staged layer times of the configuration
     b += ((size_t)buf_even + buf_odd) * 8;
     b += ((size_t)cells + 15) / 16 * 16;
     return b + 32;
 }
 
 // Copies the stage bytes (device types, boundary link) that the decode of this pass produced into the
-// tree: node n of depth d takes stage d of the first mapping below it, leaf m the last stage of mapping m.
-__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 nmap,
+// tree: node n of depth d takes stage d of the first mapping below it, every cell of the node the same,
+// leaf m the last stage of mapping m.
+__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap,
                                    const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
-                                   TrieNode *nodes, TrieLeaf *leaves)
+                                   const u32 *__restrict__ cell_gnode, TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves)
 {
     const u32 g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g < n_nodes) {
         const uint8_t *src = maptab + ((u64)first_leaf[g] * PP + (depth[g] - 1)) * 2;
         nodes[g].mask = src[0]; nodes[g].link = src[1];
-    } else if (g < n_nodes + nmap) {
-        const u32 m = g - n_nodes;
+    } else if (g < n_nodes + n_cells) {
+        const u32 c = g - n_nodes, nd = cell_gnode[c];
+        const uint8_t *src = maptab + ((u64)first_leaf[nd] * PP + (depth[nd] - 1)) * 2;
+        TrieCell v = cells[c];
+        v.x = (v.x & 0x03ffffffu) | ((u32)src[1] << 26);
+        v.y = (v.y & 0xf0ffffffu) | ((u32)(src[0] & 15) << 24);
+        cells[c] = v;
+    } else if (g < n_nodes + n_cells + nmap) {
+        const u32 m = g - n_nodes - n_cells;
         const uint8_t *src = maptab + ((u64)m * PP + (PP - 1)) * 2;
         leaves[m].mask = src[0]; leaves[m].link = src[1];
     }
+}
+
+#ifdef HAP_TRIE_TIMERS
+#define HAP_TQ(x) x
+#else
+#define HAP_TQ(x)
+#endif
+
+// Block prologue, part 1: layer times of the configuration staged in shared memory, then per type mask the
+// prefix rows of the stage time at every recomputation level (fwd+bwd + (tau_r/1024) fwd), the weight and
+// activation byte prefixes, MoE prefix counts, per-mask stage info and p2p coefficients.
+__device__ __forceinline__ void trie_prologue_rows(
+    const DevConst &dc, unsigned p_index, const i64 *c2, const i64 *coef, bool multiset, int mrows, unsigned masks_used,
+    i64 *sC, i64 *sR, i64 *sW, i64 *sA, uint8_t *sK, MaskInfo<i64> *minfo, i64 (*sP2P)[6], i64 *szero)
+{
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
+    const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, wib = tid >> 5, lane = tid & 31;
+    const int nmask = (1 << T) - 1;
+    const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
+    {
+        const longlong2 *src = reinterpret_cast<const longlong2 *>(c2 + (size_t)p_index * T * N * 2);
+        longlong2 *dst = reinterpret_cast<longlong2 *>(sC);
+        for (int q = tid; q < T * N; q += nthreads) dst[q] = src[q];
+    }
+    for (int l = tid; l <= N; l += nthreads) sK[l] = (uint8_t)moe_before(dc, l);
+    if (tid < nmask) {
+        const int mk = tid + 1;
+        MaskInfo<i64> mi;
+        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
+        i64 cap = 0;
+        bool seen = false;
+        for (int h = 0; h < T; ++h)
+            if (mk >> h & 1) {
+                const i64 *row = cfp + h * HAP_NCOEF;
+                if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; mi.capt = h; }
+                if (!seen || dc.P[h] < mi.Pmin) mi.Pmin = dc.P[h];
+                if (!seen || row[HAP_KPRE] > mi.kpre) mi.kpre = row[HAP_KPRE];
+                if (!seen || row[HAP_KPOST] > mi.kpost) mi.kpost = row[HAP_KPOST];
+                if (!seen || row[HAP_SLAT] > mi.slat) mi.slat = row[HAP_SLAT];
+                if (!seen || row[HAP_SBW] > mi.sbw[0]) mi.sbw[0] = row[HAP_SBW];
+                if (!seen || row[HAP_SBW + 1] > mi.sbw[1]) mi.sbw[1] = row[HAP_SBW + 1];
+                if (!seen || row[HAP_OPT] > mi.opt[0]) mi.opt[0] = row[HAP_OPT];
+                if (!seen || row[HAP_OPT + 1] > mi.opt[1]) mi.opt[1] = row[HAP_OPT + 1];
+                seen = true;
+            }
+        minfo[tid] = mi;
+    }
+    if (tid >= 32 && tid < 32 + T * 6) {
+        const int q = tid - 32, h = q / 6, e = q % 6;
+        sP2P[h][e] = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
+    }
+    if (tid == 0) szero[0] = 0;
+    __syncthreads();
+    // rows: one warp per type mask (and one for the byte prefixes), inclusive warp scans over chunks of 32 layers
+    for (int mr = wib; mr <= mrows; mr += nwarps) {
+        const bool bytes = mr == mrows;
+        const int mk = bytes ? 0 : (multiset ? (1 << mr) : mr + 1);
+        if (!bytes && !((masks_used >> mk) & 1u)) continue;          // no mapping of this class has such a stage
+        i64 runA = 0, runB = 0;
+        for (int base = 0; base < N; base += 32) {
+            const int l = base + lane;
+            i64 vA = 0, vB = 0;                                      // times: fwd+bwd, fwd; bytes: weights, activations
+            if (l < N) {
+                if (bytes) { const int kd = layer_kind(dc, l); vA = cfp[HAP_MW + kd]; vB = cfp[HAP_MA + kd]; }
+                else {
+                    i64 F = 0, B = 0;
+                    for (int h = 0; h < T; ++h)
+                        if (mk >> h & 1) {
+                            const i64 qx = sC[((size_t)h * N + l) * 2], qy = sC[((size_t)h * N + l) * 2 + 1];
+                            F = qx > F ? qx : F;
+                            B = qy > B ? qy : B;
+                        }
+                    vA = F + B; vB = F;
+                }
+            }
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const i64 tA = __shfl_up_sync(0xffffffffu, vA, o), tB = __shfl_up_sync(0xffffffffu, vB, o);
+                if (lane >= o) { vA += tA; vB += tB; }
+            }
+            vA += runA; vB += runB;
+            if (l < N) {
+                if (bytes) { sW[l + 1] = vA; sA[l + 1] = vB; }
+                else for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = vA + (i64)(dc.tau_q[r] >> 10) * vB;
+            }
+            runA = shfl_i64(vA, 31); runB = shfl_i64(vB, 31);
+        }
+        if (lane == 0) {
+            if (bytes) { sW[0] = 0; sA[0] = 0; }
+            else for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1] = 0;
+        }
+    }
+    __syncthreads();
+}
+
+// Block prologue, part 2: thr[d-1][t][r][j] = first split k, among those a cell of depth d can look at, for which
+// layers (k, j] fit stage d on a device of type t at level r (one past the last such split if none), only for the
+// end layers, device types and levels that occur at depth d.
+// Feasibility is monotone in the span, so a thread sweeps a segment of eight end layers with a split pointer
+// that only moves forward.
+__device__ __forceinline__ void trie_prologue_thr(
+    const DevConst &dc, const hap_pconf &pc, const TrieMeta &tm, unsigned p_index, const i64 *coef, unsigned levels,
+    const i64 *sW, const i64 *sA, uint8_t *thr, const uint8_t *sK)
+{
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP;
+    const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
+    const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
+    constexpr int kSeg = 8;
+    const int nseg = (tm.band_max + kSeg - 1) / kSeg;
+    const int total = PP * T * R * nseg;
+    for (int e = threadIdx.x; e < total; e += blockDim.x) {
+        const int seg = e % nseg, q = e / nseg;
+        const int r = q % R, t = (q / R) % T, d = q / (R * T) + 1;
+        if (!((levels >> r) & 1u) || !((tm.tmask[d] >> t) & 1u)) continue;
+        const int j0 = tm.jlo[d] + seg * kSeg;
+        int j1 = j0 + kSeg - 1; if (j1 > tm.jhi[d]) j1 = tm.jhi[d];
+        if (j0 > j1) continue;
+        const i64 extra = (d == 1 ? mpre : 0) + (d == PP ? mpost : 0);
+        const int inflight = PP - d + 1;
+        const i64 mstore = pc.M < inflight ? pc.M : inflight;
+        const i64 cap = dc.cap_eff[t], xi = dc.xi_q[r];
+        const int wmax = tm.wmax[d];
+        uint8_t *row = thr + (size_t)q * n1;
+        int k = tm.kmin[d];
+        const int kmax = tm.kmax[d];
+        for (int j = j0; j <= j1; ++j) {
+            if (k < j - wmax) k = j - wmax;
+            const int kcap = kmax < j - 1 ? kmax : j - 1;           // no cell looks at a split beyond this
+            while (k <= kcap && !span_fits(sW, sA, sK, extra, mx, mstore, cap, xi, k, j)) ++k;
+            row[j] = (uint8_t)k;
+        }
+    }
+    __syncthreads();
 }
 
 template <bool SEARCH>
@@ -86,7 +238,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     __shared__ MaskInfo<i64> minfo[kMaxMasks];
     __shared__ i64 sP2P[HAP_MAX_TYPES][6];
     __shared__ i64 szero[1];
-    __shared__ int winT[HAP_MAX_TYPES][2];
     __shared__ i64 wcost[32];
     __shared__ u64 widx[32];
     __shared__ int s_skip;
@@ -129,17 +280,21 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     i64 *sR = reinterpret_cast<i64 *>(smem_raw);
     i64 *sW = sR + (size_t)mrows * R * n1;
     i64 *sA = sW + n1;
-    uint8_t *thr = reinterpret_cast<uint8_t *>(sA + n1);
+    const size_t thr_off = (((size_t)mrows * R + 2) * n1 * 8 + 15) / 16 * 16;  // keeps what follows 16-byte aligned
+    uint8_t *thr = smem_raw + thr_off;
     const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
     uint8_t *sK = thr + thr_bytes;
-    i64 *bufE = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);    // rows of the even depths
+    i64 *sC = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);      // staged layer times [T][N][2], 16-byte aligned
+    i64 *bufE = sC + (size_t)T * N * 2;                                        // rows of the even depths
     i64 *bufO = bufE + tm.buf_cells[0];                                        // rows of the odd depths
     uint8_t *ch = reinterpret_cast<uint8_t *>(bufO + tm.buf_cells[1]);         // split choices, all depths
 
-    dp_prologue_rows<i64, true>(dc, p, c2, coef, coef, multiset, mrows, R, masks_used, nwarps, sR, sW, sA, sK, minfo, sP2P, szero);
+    HAP_TQ(long long tq0 = clock64(); long long tq_lv = 0; long long tq_leaf = 0;)
+    trie_prologue_rows(dc, p, c2, coef, multiset, mrows, masks_used, sC, sR, sW, sA, sK, minfo, sP2P, szero);
+    HAP_TQ(long long tq1 = clock64();)
     const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
 
-    // writes "infeasible" for mapping m under policy rc_idx (non-search mode)
+    // writes "infeasible" for candidate c (non-search mode)
     auto put_infeasible = [&](u64 c) {
         const u64 o = c - out.first;
         if (out.cost) out.cost[o] = kInf;
@@ -172,7 +327,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         }
         config_dead = !__syncthreads_or(fits);
     }
-    if (!config_dead) dp_prologue_thr<i64>(dc, pc, p, coef, multiset, nwarps, sW, sA, thr, sK, winT);
+    if (!config_dead) trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
+    HAP_TQ(long long tq2 = clock64();)
 
     auto stage_K = [&](int d, int mask, int link) -> i64 {
         i64 K = 0;
@@ -184,31 +340,38 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     };
 
     // one cell: min over k in [klo, khi] of max(prev[k], cost(k, j)), smallest k on ties; k runs downward over
-    // the level segments given by the memory thresholds (lowest allowed level that fits)
-    auto cell = [&](int d, int j, int mask, int link, int klo, int khi, const i64 *prev, unsigned rc_mask, i64 &best, int &arg) {
-        best = kInf; arg = 255;
-        if (klo > khi) return;
-        const int mrow = multiset ? __ffs(mask) - 1 : mask - 1;
-        const i64 K = stage_K(d, mask, link);
-        const i64 *rM = sR + (size_t)mrow * R * n1;
-        const uint8_t *th = thr + ((size_t)(d - 1) * T + minfo[mask - 1].capt) * R * n1;
-        int seg_hi = khi;
-        for (int r = 0; r < R && seg_hi >= klo; ++r) {
-            if (!((rc_mask >> r) & 1u)) continue;
-            int lo = th[(size_t)r * n1 + j];
-            if (lo < klo) lo = klo;
-            if (lo > seg_hi) continue;
-            n_cells += (u64)(seg_hi - lo + 1);
-            const i64 *rr = rM + (size_t)r * n1;
-            const i64 Cj = rr[j] + K;
-            for (int k = seg_hi; k >= lo; --k) {
-                const i64 pv = prev[k];
-                const i64 cst = Cj - rr[k];
-                const i64 v = pv > cst ? pv : cst;
-                if (v <= best && v < kInf) { best = v; arg = k; }
+    // the level segments given by the memory thresholds (lowest allowed level that fits), two splits per step
+    // (an index below the segment is clamped to its lowest split, which re-evaluates that split: harmless)
+    auto cell = [&](int d, int j, int mask, int link, int capt, int klo, int khi, const i64 *prev, unsigned rc_mask, i64 &best_out, int &arg_out) {
+        i64 best = kInf - 1;                    // every finite value is below this, an unreachable one (= kInf) above
+        int arg = 255;
+        if (klo <= khi) {
+            const int mrow = multiset ? __ffs(mask) - 1 : mask - 1;
+            const i64 K = stage_K(d, mask, link);
+            const i64 *rM = sR + (size_t)mrow * R * n1;
+            const uint8_t *th = thr + ((size_t)(d - 1) * T + capt) * R * n1;
+            int seg_hi = khi;
+            for (int r = 0; r < R && seg_hi >= klo; ++r) {
+                if (!((rc_mask >> r) & 1u)) continue;
+                int lo = th[(size_t)r * n1 + j];
+                if (lo < klo) lo = klo;
+                if (lo > seg_hi) continue;
+                n_cells += (u64)(seg_hi - lo + 1);
+                const i64 *rr = rM + (size_t)r * n1;
+                const i64 Cj = rr[j] + K;
+                for (int k = seg_hi; k >= lo; k -= 2) {
+                    const int k1 = k - 1 > lo ? k - 1 : lo;
+                    const i64 p0 = prev[k], p1 = prev[k1];
+                    const i64 c0 = Cj - rr[k], c1 = Cj - rr[k1];
+                    const i64 v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
+                    if (v0 <= best) { best = v0; arg = k; }
+                    if (v1 <= best) { best = v1; arg = k1; }
+                }
+                seg_hi = lo - 1;
             }
-            seg_hi = lo - 1;
         }
+        best_out = arg == 255 ? kInf : best;
+        arg_out = arg;
     };
 
     unsigned policies_without_plan = 0;                      // positions in rc_order under which no mapping was feasible
@@ -217,26 +380,25 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         const unsigned rc_mask = dc.rc_masks[rc_idx];
         bool dead = config_dead || (dc.rc_sup[rc_pos] & policies_without_plan) != 0;
 
+        HAP_TQ(long long tq3 = clock64();)
         // ---- rows of the tree, depth by depth ------------------------------------------------
         if (!dead) {
             for (int d = 1; d < PP; ++d) {
                 const u32 ncell = tm.cell_lo[d + 1] - tm.cell_lo[d];
-                const TrieNode *nd_base = tm.nodes + tm.node_lo[d];
-                const uint16_t *cnode = tm.cell_node + tm.cell_lo[d];
+                const TrieCell *cells = tm.cells + tm.cell_lo[d];
                 uint8_t *chd = ch + tm.cell_lo[d];
                 i64 *cur = (d & 1) ? bufO : bufE;
-                const i64 *prevbuf = d == 1 ? szero : ((d & 1) ? bufE : bufO);
+                const i64 *prevbuf = (d == 1 ? szero : ((d & 1) ? bufE : bufO)) - 256;
                 int alive = 0;
+                TrieCell nxt = make_uint2(0, 0);
+                if ((u32)tid < ncell) nxt = __ldg(cells + tid);
                 for (u32 e = tid; e < ncell; e += nthreads) {
-                    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(nd_base + cnode[e]));
-                    const u32 rowoff = raw.x, prowoff = raw.y;
-                    const int mask = raw.z & 255, link = (raw.z >> 8) & 255, nmin = (raw.z >> 16) & 255, nmax = raw.z >> 24;
-                    const int bl = raw.w & 255, pbl = (raw.w >> 16) & 255, pbh = raw.w >> 24;
-                    const int j = bl + (int)(e - rowoff);
-                    int klo = j - nmax; if (klo < pbl) klo = pbl;
-                    int khi = j - nmin; if (khi > pbh) khi = pbh;
+                    const TrieCell rec = nxt;
+                    if (e + nthreads < ncell) nxt = __ldg(cells + e + nthreads);      // next record while this cell runs
+                    const int j = rec.y & 255, klo = (rec.y >> 8) & 255, khi = (rec.y >> 16) & 255;
+                    const int mask = (rec.y >> 24) & 15, capt = (rec.y >> 28) & 3, link = rec.x >> 26;
                     i64 best; int arg;
-                    cell(d, j, mask, link, klo, khi, prevbuf + prowoff - pbl, rc_mask, best, arg);
+                    cell(d, j, mask, link, capt, klo, khi, prevbuf + (rec.x & 0x03ffffffu) , rc_mask, best, arg);
                     cur[e] = best;
                     chd[e] = (uint8_t)arg;
                     alive |= best < kInf;
@@ -244,7 +406,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 if (!__syncthreads_or(alive)) { dead = true; break; }   // no cell of this depth is finite: nothing below is
             }
         }
-
+        HAP_TQ(long long tq4 = clock64(); tq_lv += tq4 - tq3;)
         // ---- one thread per mapping: cell (PP, N), backtrace, Eq. 4 ---------------------------------
         int any_plan = 0;
         const i64 *lastbuf = PP == 1 ? szero : (((PP - 1) & 1) ? bufO : bufE);
@@ -252,16 +414,18 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             const u64 c = pc.offset + (u64)m * n_rc + (u64)rc_idx;
             if (c < w_lo || c >= w_hi) continue;
             i64 bott = kInf; int arg = 255;
-            TrieLeaf lf;
+            int mask = 0, link = 0;
+            u32 node = 0;
             if (!dead) {
                 const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(tm.leaves + m));
-                lf.prowoff = raw.x; lf.parent = (uint16_t)(raw.y & 0xffff); lf.mask = (raw.y >> 16) & 255; lf.link = raw.y >> 24;
-                lf.nmin = raw.z & 255; lf.nmax = (raw.z >> 8) & 255; lf.pbl = (raw.z >> 16) & 255; lf.pbh = raw.z >> 24;
-                lf.dead = raw.w & 255;
-                if (!lf.dead) {
-                    int klo = N - lf.nmax; if (klo < lf.pbl) klo = lf.pbl;
-                    int khi = N - lf.nmin; if (khi > lf.pbh) khi = lf.pbh;
-                    cell(PP, N, lf.mask, lf.link, klo, khi, lastbuf + lf.prowoff - lf.pbl, rc_mask, bott, arg);
+                const u32 prowoff = raw.x;
+                node = raw.y & 0xffff; mask = (raw.y >> 16) & 255; link = raw.y >> 24;
+                const int nmin = raw.z & 255, nmax = (raw.z >> 8) & 255, pbl = (raw.z >> 16) & 255, pbh = raw.z >> 24;
+                const int ldead = raw.w & 255, capt = (raw.w >> 8) & 255;
+                if (!ldead) {
+                    int klo = N - nmax; if (klo < pbl) klo = pbl;
+                    int khi = N - nmin; if (khi > pbh) khi = pbh;
+                    cell(PP, N, mask, link, capt, klo, khi, lastbuf + prowoff - pbl, rc_mask, bott, arg);
                 }
             }
             if (SEARCH) n_eval++;
@@ -272,9 +436,15 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             // backtrace from (PP, N) through the ancestors; per stage: level, cost, sync and optimizer terms
             i64 sum = 0, mxc = 0, t_sync = 0, t_opt = 0, het = 0;
             const u64 o = c - out.first;
-            int b = N, a = arg, mask = lf.mask, link = lf.link;
-            u32 node = lf.parent;
+            int b = N, a = arg;
             for (int d = PP; d >= 1; --d) {
+                // the ancestor's record is fetched before this stage's arithmetic needs to wait for it
+                uint4 raw = make_uint4(0, 0, 0, 0);
+                u32 parent = 0;
+                if (d > 1) {
+                    raw = __ldg(reinterpret_cast<const uint4 *>(tm.nodes + tm.node_lo[d - 1] + node));
+                    parent = tm.parent[tm.node_lo[d - 1] + node];
+                }
                 const MaskInfo<i64> &mi = minfo[mask - 1];
                 const uint8_t *th = thr + ((size_t)(d - 1) * T + mi.capt) * R * n1;
                 int r = 0;
@@ -294,8 +464,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     if (out.recompute) out.recompute[o * HAP_MAX_PP + d - 1] = (uint8_t)r;
                 }
                 if (d > 1) {
-                    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(tm.nodes + tm.node_lo[d - 1] + node));
-                    const u32 parent = tm.parent[tm.node_lo[d - 1] + node];
                     b = a;
                     a = ch[tm.cell_lo[d - 1] + raw.x + (u32)(b - (int)(raw.w & 255))];
                     mask = raw.z & 255; link = (raw.z >> 8) & 255;
@@ -323,10 +491,19 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         }
         // the barrier also keeps the next policy from overwriting rows and choices that are still being read
         const int bott_any = __syncthreads_or(any_plan);
+        HAP_TQ(tq_leaf += clock64() - tq4;)
         // a policy under which no mapping of the WHOLE configuration has a feasible partition settles its subsets
         if (!bott_any && c_lo >= w_lo && c_hi <= w_hi && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
     }
 
+#ifdef HAP_TRIE_TIMERS
+    if (tid == 0 && out.counters && !SEARCH) {
+        // cycles per block: [5] rows prologue, [6] thresholds, [7] tree levels, [3] mappings, [2] whole block
+        atomicAdd(out.counters + 5, (u64)(tq1 - tq0)); atomicAdd(out.counters + 6, (u64)(tq2 - tq1));
+        atomicAdd(out.counters + 7, (u64)tq_lv); atomicAdd(out.counters + 3, (u64)tq_leaf);
+        atomicAdd(out.counters + 2, (u64)(clock64() - tq0));
+    }
+#endif
     if (out.counters) {
         n_cells = (u64)warp_sum_i64((i64)n_cells);
         if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
