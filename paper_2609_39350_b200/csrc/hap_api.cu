@@ -402,11 +402,33 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
         }
         lf.parent = PP > 1 ? (uint16_t)path[PP - 1] : 0;
     }
+    // nodes of a depth ordered by the width of their window (widest first, stable), so that the cells a warp works
+    // on have split loops of similar length
+    for (int d = 1; d < PP; ++d) {
+        std::vector<u32> ord(lv[d].size()), newidx(lv[d].size());
+        for (size_t i = 0; i < ord.size(); ++i) ord[i] = (u32)i;
+        std::stable_sort(ord.begin(), ord.end(), [&](u32 a, u32 b) {
+            return (int)lv[d][a].k.nmax - (int)lv[d][a].k.nmin > (int)lv[d][b].k.nmax - (int)lv[d][b].k.nmin; });
+        std::vector<HNode> sorted(lv[d].size());
+        for (size_t i = 0; i < ord.size(); ++i) { sorted[i] = lv[d][ord[i]]; newidx[ord[i]] = (u32)i; }
+        lv[d].swap(sorted);
+        if (d + 1 < PP) for (auto &ch : lv[d + 1]) ch.parent = newidx[ch.parent];
+        else for (u64 m = 0; m < nmap; ++m) if (!leaves[m].dead) leaves[m].parent = (uint16_t)newidx[leaves[m].parent];
+    }
     // flat layout
     hap_problem::Trie &tr = cl.trie;
     TrieMeta &tm = tr.meta;
     std::memset(&tm, 0, sizeof(tm));
     tm.PP = PP; tm.nmap = (u32)nmap;
+    // row groups of the time rows: one per type mask that some stage has
+    std::memset(tm.mrow_of, 255, sizeof(tm.mrow_of));
+    {
+        unsigned used = 0;
+        for (int d = 1; d < PP; ++d) for (const auto &h : lv[d]) used |= 1u << h.k.mask;
+        for (u64 m = 0; m < nmap; ++m) used |= 1u << leaves[m].mask;
+        for (int mk = 1; mk < (1 << T); ++mk)
+            if ((used >> mk) & 1u) { tm.mrow_of[mk] = (uint8_t)tm.n_mrows; tm.mask_of_row[tm.n_mrows] = (uint8_t)mk; tm.n_mrows++; }
+    }
     u32 n_nodes = 0, n_cells = 0, max_level = 0;
     std::vector<std::vector<u32>> rowoff(PP + 1);
     for (int d = 1; d < PP; ++d) {
@@ -421,8 +443,6 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     }
     for (int d = std::max(PP, 1); d <= HAP_MAX_PP; ++d) { tm.node_lo[d] = n_nodes; tm.cell_lo[d] = n_cells; }
     tm.buf_cells[0] = (tm.buf_cells[0] + 1) / 2 * 2; tm.buf_cells[1] = (tm.buf_cells[1] + 1) / 2 * 2;
-    const size_t smem = trie_smem_bytes(N, PP, T, R, cl.multiset, tm.buf_cells[0], tm.buf_cells[1], n_cells);
-    if (smem > 220 * 1024) return false;
     if (n_cells >= (1u << 25)) return false;
     std::vector<TrieNode> nodes(n_nodes);
     std::vector<uint16_t> parent(n_nodes);
@@ -458,13 +478,24 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
                 if (klo > khi) { klo = 1; khi = 0; }
                 else { tm.kmin[d] = std::min<uint8_t>(tm.kmin[d], (uint8_t)klo); tm.kmax[d] = std::max<uint8_t>(tm.kmax[d], (uint8_t)khi); }
                 const u32 c = tm.cell_lo[d] + rowoff[d][i] + (u32)(j - h.bl);
-                cells[c].x = (u32)((int)nd.prowoff - (int)nd.pbl + 256) | ((u32)nd.link << 26);
-                cells[c].y = (u32)j | ((u32)klo << 8) | ((u32)khi << 16) | ((u32)(nd.mask & 15) << 24) | ((u32)capt_of[nd.mask] << 28);
+                const int cls = nd.link & 3, ha = (nd.link >> 2) & 3, hb = (nd.link >> 4) & 3;
+                const u32 kidx = d == 1 ? tm.mrow_of[nd.mask] : 16 + hb * 6 + (cls == HAP_CROSS ? 2 + ha : cls);
+                cells[c].x = (u32)((int)nd.prowoff - (int)nd.pbl + 256) | (kidx << 26);
+                cells[c].y = (u32)j | ((u32)klo << 8) | ((u32)khi << 16);
+                cells[c].z = 0;                                   // threshold index: needs the depth's first end layer, set below
+                cells[c].w = (u32)tm.mrow_of[nd.mask] * (u32)(R * (N + 1));
                 cell_gnode[c] = tm.node_lo[d] + (u32)i;
             }
         }
     for (int d = 1; d <= PP; ++d) if (tm.jlo[d] <= tm.jhi[d]) band_max = std::max(band_max, tm.jhi[d] - tm.jlo[d] + 1);
+    for (u32 c = 0; c < n_cells; ++c) {
+        const u32 g = cell_gnode[c];
+        const int d = depth[g], j = (int)(cells[c].y & 255);
+        cells[c].z = (u32)((((d - 1) * T + capt_of[nodes[g].mask]) * R) * band_max + (j - (int)tm.jlo[d]));
+    }
     tm.band_max = band_max;
+    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, band_max, tm.buf_cells[0], tm.buf_cells[1], n_cells);
+    if (smem > 220 * 1024) return false;
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];
         if (lf.dead || PP == 1) { lf.prowoff = 0; lf.pbl = 0; lf.pbh = 0; continue; }
@@ -820,14 +851,14 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, p->items[cl.item_lo].p, nmap, p->d_maptab + cl.map_base);
             CUDA_TRY(p, cudaGetLastError());
             const u32 n_g = tr.n_nodes + tr.n_cells + (u32)nmap;
+            TrieRowMap rmap;
+            std::memcpy(rmap.mrow_of, tr.meta.mrow_of, sizeof(rmap.mrow_of));
             trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, tr.n_nodes, tr.n_cells, (u32)nmap, tr.d_first_leaf, tr.d_depth,
-                                                                          tr.d_gnode, tr.d_nodes, tr.d_cells, tr.d_leaves);
+                                                                          tr.d_gnode, rmap, tr.d_nodes, tr.d_cells, tr.d_leaves);
             CUDA_TRY(p, cudaGetLastError());
-            unsigned n_active = tr.n_conf, used = cl.masks_used;
-            int ms = cl.multiset ? 1 : 0;
+            unsigned n_active = tr.n_conf;
             const u32 *plist = tr.d_plist;
-            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tr.meta,
-                             (void *)&o, (void *)&used, (void *)&ms};
+            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tr.meta, (void *)&o};
             const unsigned tblocks = search ? blocks : tr.n_conf;       // search: every partial slot of the class is written
             CUDA_TRY(p, cudaLaunchKernel(tfn, dim3(tblocks), dim3(tr.threads), targs, tr.smem, cl.stream));
             CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));

@@ -37,10 +37,14 @@ struct TrieLeaf {            // one mapping: its last stage                     
     uint8_t pad[2];
 };
 
-// One cell (node, end layer j) of a depth, everything its split loop needs in 8 bytes:
-//   x = (row origin of the parent in the previous depth's buffer, i.e. prowoff - pbl, + 256) | link << 26
-//   y = j | klo << 8 | khi << 16 | mask << 24 | capt << 28     (klo..khi: window of the stage within the parent's band)
-typedef uint2 TrieCell;
+// One cell (node, end layer j) of a depth d < PP: everything its split loop needs, in 16 bytes.
+//   x = (row origin of the parent in the previous depth's buffer, i.e. prowoff - pbl, + 256) | kidx << 26
+//       kidx: entry of the block's table of stage constants (depth 1: pre-work of the stage's types;
+//       deeper: p2p transfer by receiving type and link class), filled from the decode of each pass
+//   y = j | klo << 8 | khi << 16          (klo..khi: window of the stage within the parent's band)
+//   z = index of the cell's level-0 memory threshold in the block's threshold table
+//   w = element offset of the level-0 time row of the stage's type mask
+typedef uint4 TrieCell;
 
 struct TrieMeta {
     const TrieNode *nodes;          // grouped by depth
@@ -53,30 +57,38 @@ struct TrieMeta {
     uint8_t wmax[HAP_MAX_PP + 1];   // widest window of a stage at depth d
     uint8_t tmask[HAP_MAX_PP + 1];  // device types whose memory binds some stage of depth d
     uint8_t kmin[HAP_MAX_PP + 1], kmax[HAP_MAX_PP + 1];   // smallest / largest split any cell of depth d looks at
+    uint8_t mrow_of[16];            // type mask -> its row group in the block's time rows (255: no stage has this mask)
+    uint8_t mask_of_row[16];        // the inverse
+    int n_mrows;
     u32 buf_cells[2];               // largest row storage of an even / odd depth, in cells
     u32 nmap;
     int PP, band_max;               // band_max: most end layers of any depth
 };
 
-__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, bool multiset, u32 buf_even, u32 buf_odd, u32 cells)
+constexpr int kTrieKtab = 16 + HAP_MAX_TYPES * 6;    // stage constants: [0,16) pre-work by row group, then p2p [type][6]
+
+__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, int n_mrows, int band_max, u32 buf_even, u32 buf_odd, u32 cells)
 {
     const size_t n1 = (size_t)N + 1;
-    const size_t mrows = multiset ? (size_t)T : (size_t)((1 << T) - 1);
-    size_t b = mrows * (size_t)R * n1 * 8 + n1 * 16;
-    b += ((size_t)PP * T * R * n1 + 15) / 16 * 16;
-    b += (n1 + 15) / 16 * 16;
-    b += (size_t)T * N * 16;                         // staged layer times of the configuration
+    size_t b = (((size_t)n_mrows * R + 2) * n1 * 8 + 15) / 16 * 16;      // time rows, weight and activation byte rows
+    b += ((size_t)PP * T * R * band_max + 15) / 16 * 16;                  // memory thresholds
+    b += (n1 + 15) / 16 * 16;                                              // MoE prefix counts
+    b += (size_t)T * N * 16;                                               // staged layer times of the configuration
+    b += (size_t)kTrieKtab * 8;
     b += ((size_t)buf_even + buf_odd) * 8;
     b += ((size_t)cells + 15) / 16 * 16;
     return b + 32;
 }
 
-// Copies the stage bytes (device types, boundary link) that the decode of this pass produced into the
-// tree: node n of depth d takes stage d of the first mapping below it, every cell of the node the same,
-// leaf m the last stage of mapping m.
+struct TrieRowMap { uint8_t mrow_of[16]; };
+
+// Copies what the decode of this pass produced into the tree: node n of depth d takes the stage bytes (device
+// types, boundary link) of stage d of the first mapping below it, every cell of the node the index of the stage
+// constant that follows from them, leaf m the last stage of mapping m.
 __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap,
                                    const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
-                                   const u32 *__restrict__ cell_gnode, TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves)
+                                   const u32 *__restrict__ cell_gnode, const TrieRowMap rm,
+                                   TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves)
 {
     const u32 g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g < n_nodes) {
@@ -84,11 +96,13 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
         nodes[g].mask = src[0]; nodes[g].link = src[1];
     } else if (g < n_nodes + n_cells) {
         const u32 c = g - n_nodes, nd = cell_gnode[c];
-        const uint8_t *src = maptab + ((u64)first_leaf[nd] * PP + (depth[nd] - 1)) * 2;
-        TrieCell v = cells[c];
-        v.x = (v.x & 0x03ffffffu) | ((u32)src[1] << 26);
-        v.y = (v.y & 0xf0ffffffu) | ((u32)(src[0] & 15) << 24);
-        cells[c] = v;
+        const int d = depth[nd];
+        const uint8_t *src = maptab + ((u64)first_leaf[nd] * PP + (d - 1)) * 2;
+        const int mask = src[0] & 15, link = src[1];
+        const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3;
+        const u32 kidx = d == 1 ? rm.mrow_of[mask] : 16 + hb * 6 + (cls == HAP_CROSS ? 2 + ha : cls);
+        u32 *x = reinterpret_cast<u32 *>(cells + c);
+        *x = (*x & 0x03ffffffu) | (kidx << 26);
     } else if (g < n_nodes + n_cells + nmap) {
         const u32 m = g - n_nodes - n_cells;
         const uint8_t *src = maptab + ((u64)m * PP + (PP - 1)) * 2;
@@ -102,16 +116,32 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
 #define HAP_TQ(x)
 #endif
 
-// Block prologue, part 1: layer times of the configuration staged in shared memory, then per type mask the
-// prefix rows of the stage time at every recomputation level (fwd+bwd + (tau_r/1024) fwd), the weight and
-// activation byte prefixes, MoE prefix counts, per-mask stage info and p2p coefficients.
+// shared-memory accesses by 32-bit address (the split loop walks two rows with plain address decrements)
+__device__ __forceinline__ u32 smem_u32(const void *p) { return (u32)__cvta_generic_to_shared(p); }
+template <int OFF> __device__ __forceinline__ i64 lds_i64(u32 a)
+{
+    i64 v;
+    asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(v) : "r"(a), "n"(OFF));
+    return v;
+}
+__device__ __forceinline__ int lds_u8(u32 a)
+{
+    u32 v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
+    return (int)v;
+}
+
+// Block prologue, part 1: layer times of the configuration staged in shared memory, then per type mask that
+// occurs in the class the prefix rows of the stage time at every recomputation level (fwd+bwd + (tau_r/1024) fwd),
+// the weight and activation byte prefixes, MoE prefix counts, per-mask stage info, p2p coefficients and the
+// table of stage constants.
 __device__ __forceinline__ void trie_prologue_rows(
-    const DevConst &dc, unsigned p_index, const i64 *c2, const i64 *coef, bool multiset, int mrows, unsigned masks_used,
-    i64 *sC, i64 *sR, i64 *sW, i64 *sA, uint8_t *sK, MaskInfo<i64> *minfo, i64 (*sP2P)[6], i64 *szero)
+    const DevConst &dc, const TrieMeta &tm, unsigned p_index, const i64 *c2, const i64 *coef,
+    i64 *sC, i64 *sR, i64 *sW, i64 *sA, uint8_t *sK, i64 *sKtab, MaskInfo<i64> *minfo, i64 (*sP2P)[6], i64 *szero)
 {
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, wib = tid >> 5, lane = tid & 31;
-    const int nmask = (1 << T) - 1;
+    const int nmask = (1 << T) - 1, mrows = tm.n_mrows;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     {
         const longlong2 *src = reinterpret_cast<const longlong2 *>(c2 + (size_t)p_index * T * N * 2);
@@ -140,18 +170,20 @@ __device__ __forceinline__ void trie_prologue_rows(
                 seen = true;
             }
         minfo[tid] = mi;
+        if (tm.mrow_of[mk] != 255) sKtab[tm.mrow_of[mk]] = mi.kpre;
     }
     if (tid >= 32 && tid < 32 + T * 6) {
         const int q = tid - 32, h = q / 6, e = q % 6;
-        sP2P[h][e] = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
+        const i64 v = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
+        sP2P[h][e] = v;
+        sKtab[16 + q] = v;
     }
     if (tid == 0) szero[0] = 0;
     __syncthreads();
     // rows: one warp per type mask (and one for the byte prefixes), inclusive warp scans over chunks of 32 layers
     for (int mr = wib; mr <= mrows; mr += nwarps) {
         const bool bytes = mr == mrows;
-        const int mk = bytes ? 0 : (multiset ? (1 << mr) : mr + 1);
-        if (!bytes && !((masks_used >> mk) & 1u)) continue;          // no mapping of this class has such a stage
+        const int mk = bytes ? 0 : tm.mask_of_row[mr];
         i64 runA = 0, runB = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
@@ -189,16 +221,21 @@ __device__ __forceinline__ void trie_prologue_rows(
     __syncthreads();
 }
 
-// Block prologue, part 2: thr[d-1][t][r][j] = first split k, among those a cell of depth d can look at, for which
+// index of the memory threshold of (stage d, capacity type t, level r, end layer j) in the block's table
+__device__ __forceinline__ u32 trie_thr_index(const TrieMeta &tm, int T, int R, int d, int t, int r, int j)
+{
+    return (u32)((((d - 1) * T + t) * R + r) * tm.band_max + (j - (int)tm.jlo[d]));
+}
+
+// Block prologue, part 2: threshold = first split k, among those a cell of depth d can look at, for which
 // layers (k, j] fit stage d on a device of type t at level r (one past the last such split if none), only for the
-// end layers, device types and levels that occur at depth d.
-// Feasibility is monotone in the span, so a thread sweeps a segment of eight end layers with a split pointer
-// that only moves forward.
+// end layers, device types and levels that occur at depth d.  Feasibility is monotone in the span, so a thread
+// sweeps a segment of eight end layers with a split pointer that only moves forward.
 __device__ __forceinline__ void trie_prologue_thr(
     const DevConst &dc, const hap_pconf &pc, const TrieMeta &tm, unsigned p_index, const i64 *coef, unsigned levels,
     const i64 *sW, const i64 *sA, uint8_t *thr, const uint8_t *sK)
 {
-    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP;
+    const int T = dc.T, R = dc.R, PP = pc.PP;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
     constexpr int kSeg = 8;
@@ -216,7 +253,7 @@ __device__ __forceinline__ void trie_prologue_thr(
         const i64 mstore = pc.M < inflight ? pc.M : inflight;
         const i64 cap = dc.cap_eff[t], xi = dc.xi_q[r];
         const int wmax = tm.wmax[d];
-        uint8_t *row = thr + (size_t)q * n1;
+        uint8_t *row = thr + (size_t)q * tm.band_max - tm.jlo[d];
         int k = tm.kmin[d];
         const int kmax = tm.kmax[d];
         for (int j = j0; j <= j1; ++j) {
@@ -232,7 +269,7 @@ __device__ __forceinline__ void trie_prologue_thr(
 template <bool SEARCH>
 __global__ void __launch_bounds__(1024, 1)
 trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64 *c2, const i64 *coef,
-               const TrieMeta tm, DpOut out, unsigned masks_used, int multiset_i)
+               const TrieMeta tm, DpOut out)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ MaskInfo<i64> minfo[kMaxMasks];
@@ -249,8 +286,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     }
     const u32 p = plist[blockIdx.x];
     const hap_pconf pc = dc.pconf[p];
-    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc;
-    const bool multiset = multiset_i != 0;
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.band_max;
     const u64 c_lo = pc.offset, c_hi = pc.offset + (u64)tm.nmap * n_rc;        // candidates of this configuration
     const u64 w_lo = out.first, w_hi = out.first + out.count;                  // candidates that are wanted
     if (c_hi <= w_lo || c_lo >= w_hi) {
@@ -275,22 +311,23 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         if (s_skip) return;
     }
 
-    const int nmask = (1 << T) - 1;
-    const int mrows = multiset ? T : nmask;
+    // shared memory: time rows | weight bytes | activation bytes | thresholds | MoE counts | staged layer times |
+    //                stage constants | rows of the even depths | rows of the odd depths | split choices
     i64 *sR = reinterpret_cast<i64 *>(smem_raw);
-    i64 *sW = sR + (size_t)mrows * R * n1;
+    i64 *sW = sR + (size_t)tm.n_mrows * R * n1;
     i64 *sA = sW + n1;
-    const size_t thr_off = (((size_t)mrows * R + 2) * n1 * 8 + 15) / 16 * 16;  // keeps what follows 16-byte aligned
+    const size_t thr_off = (((size_t)tm.n_mrows * R + 2) * n1 * 8 + 15) / 16 * 16;
     uint8_t *thr = smem_raw + thr_off;
-    const size_t thr_bytes = ((size_t)PP * T * R * n1 + 15) / 16 * 16;
+    const size_t thr_bytes = ((size_t)PP * T * R * bw + 15) / 16 * 16;
     uint8_t *sK = thr + thr_bytes;
-    i64 *sC = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);      // staged layer times [T][N][2], 16-byte aligned
-    i64 *bufE = sC + (size_t)T * N * 2;                                        // rows of the even depths
-    i64 *bufO = bufE + tm.buf_cells[0];                                        // rows of the odd depths
-    uint8_t *ch = reinterpret_cast<uint8_t *>(bufO + tm.buf_cells[1]);         // split choices, all depths
+    i64 *sC = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);      // [T][N][2], 16-byte aligned
+    i64 *sKtab = sC + (size_t)T * N * 2;
+    i64 *bufE = sKtab + kTrieKtab;
+    i64 *bufO = bufE + tm.buf_cells[0];
+    uint8_t *ch = reinterpret_cast<uint8_t *>(bufO + tm.buf_cells[1]);
 
     HAP_TQ(long long tq0 = clock64(); long long tq_lv = 0; long long tq_leaf = 0;)
-    trie_prologue_rows(dc, p, c2, coef, multiset, mrows, masks_used, sC, sR, sW, sA, sK, minfo, sP2P, szero);
+    trie_prologue_rows(dc, tm, p, c2, coef, sC, sR, sW, sA, sK, sKtab, minfo, sP2P, szero);
     HAP_TQ(long long tq1 = clock64();)
     const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
 
@@ -330,48 +367,45 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     if (!config_dead) trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
     HAP_TQ(long long tq2 = clock64();)
 
-    auto stage_K = [&](int d, int mask, int link) -> i64 {
-        i64 K = 0;
-        const MaskInfo<i64> &mi = minfo[mask - 1];
-        if (d == 1) K += mi.kpre;
-        if (d == PP) K += mi.kpost;
-        if (d > 1) { const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3; K += sP2P[hb][cls == HAP_CROSS ? 2 + ha : cls]; }
-        return K;
-    };
+    const u32 a_thr = smem_u32(thr), a_sR = smem_u32(sR);
 
-    // one cell: min over k in [klo, khi] of max(prev[k], cost(k, j)), smallest k on ties; k runs downward over
-    // the level segments given by the memory thresholds (lowest allowed level that fits), two splits per step
-    // (an index below the segment is clamped to its lowest split, which re-evaluates that split: harmless)
-    auto cell = [&](int d, int j, int mask, int link, int capt, int klo, int khi, const i64 *prev, unsigned rc_mask, i64 &best_out, int &arg_out) {
+    // One cell: min over k in [klo, khi] of max(prev[k], cost(k, j)), smallest k on ties.  k runs downward over the
+    // level segments given by the memory thresholds (lowest allowed level that fits); prev[k] and the time row
+    // entry of k are read through two addresses that step down together, two splits per step.
+    //   a_prev: address of prev[0]; a_th: address of the level-0 threshold of (stage, j); a_row: address of entry 0
+    //   of the level-0 time row of the stage's types; K: stage constant
+    auto cell = [&](u32 a_prev, int j, int klo, int khi, u32 a_th, u32 a_row, i64 K, unsigned rc_mask, i64 &best_out, int &arg_out) {
         i64 best = kInf - 1;                    // every finite value is below this, an unreachable one (= kInf) above
-        int arg = 255;
-        if (klo <= khi) {
-            const int mrow = multiset ? __ffs(mask) - 1 : mask - 1;
-            const i64 K = stage_K(d, mask, link);
-            const i64 *rM = sR + (size_t)mrow * R * n1;
-            const uint8_t *th = thr + ((size_t)(d - 1) * T + capt) * R * n1;
-            int seg_hi = khi;
-            for (int r = 0; r < R && seg_hi >= klo; ++r) {
-                if (!((rc_mask >> r) & 1u)) continue;
-                int lo = th[(size_t)r * n1 + j];
-                if (lo < klo) lo = klo;
-                if (lo > seg_hi) continue;
-                n_cells += (u64)(seg_hi - lo + 1);
-                const i64 *rr = rM + (size_t)r * n1;
-                const i64 Cj = rr[j] + K;
-                for (int k = seg_hi; k >= lo; k -= 2) {
-                    const int k1 = k - 1 > lo ? k - 1 : lo;
-                    const i64 p0 = prev[k], p1 = prev[k1];
-                    const i64 c0 = Cj - rr[k], c1 = Cj - rr[k1];
-                    const i64 v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
-                    if (v0 <= best) { best = v0; arg = k; }
-                    if (v1 <= best) { best = v1; arg = k1; }
-                }
-                seg_hi = lo - 1;
+        u32 a_arg = 0;
+        int seg_hi = khi;
+        for (int r = 0; r < R && seg_hi >= klo; ++r, a_th += (u32)bw, a_row += (u32)n1 * 8u) {
+            if (!((rc_mask >> r) & 1u)) continue;
+            int lo = lds_u8(a_th);
+            if (lo < klo) lo = klo;
+            if (lo > seg_hi) continue;
+            const int n = seg_hi - lo + 1;
+            n_cells += (u64)n;
+            const i64 Cj = lds_i64<0>(a_row + 8u * (u32)j) + K;
+            u32 pa = a_prev + 8u * (u32)seg_hi, ra = a_row + 8u * (u32)seg_hi;
+            const u32 pa_lo = a_prev + 8u * (u32)lo;
+            if (n & 1) {
+                const i64 p0 = lds_i64<0>(pa), c0 = Cj - lds_i64<0>(ra);
+                const i64 v0 = p0 > c0 ? p0 : c0;
+                if (v0 <= best) { best = v0; a_arg = pa; }
+                pa -= 8; ra -= 8;
             }
+            while ((int)(pa - pa_lo) > 0) {      // pa and pa - 8 are both inside the segment
+                const i64 p0 = lds_i64<0>(pa), p1 = lds_i64<-8>(pa);
+                const i64 c0 = Cj - lds_i64<0>(ra), c1 = Cj - lds_i64<-8>(ra);
+                const i64 v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
+                if (v0 <= best) { best = v0; a_arg = pa; }
+                if (v1 <= best) { best = v1; a_arg = pa - 8; }
+                pa -= 16; ra -= 16;
+            }
+            seg_hi = lo - 1;
         }
-        best_out = arg == 255 ? kInf : best;
-        arg_out = arg;
+        best_out = a_arg ? best : kInf;
+        arg_out = a_arg ? (int)((a_arg - a_prev) >> 3) : 255;
     };
 
     unsigned policies_without_plan = 0;                      // positions in rc_order under which no mapping was feasible
@@ -388,17 +422,17 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 const TrieCell *cells = tm.cells + tm.cell_lo[d];
                 uint8_t *chd = ch + tm.cell_lo[d];
                 i64 *cur = (d & 1) ? bufO : bufE;
-                const i64 *prevbuf = (d == 1 ? szero : ((d & 1) ? bufE : bufO)) - 256;
+                const u32 a_prevbuf = smem_u32(d == 1 ? szero : ((d & 1) ? bufE : bufO)) - 256u * 8u;
                 int alive = 0;
-                TrieCell nxt = make_uint2(0, 0);
+                TrieCell nxt = make_uint4(0, 0, 0, 0);
                 if ((u32)tid < ncell) nxt = __ldg(cells + tid);
                 for (u32 e = tid; e < ncell; e += nthreads) {
                     const TrieCell rec = nxt;
                     if (e + nthreads < ncell) nxt = __ldg(cells + e + nthreads);      // next record while this cell runs
                     const int j = rec.y & 255, klo = (rec.y >> 8) & 255, khi = (rec.y >> 16) & 255;
-                    const int mask = (rec.y >> 24) & 15, capt = (rec.y >> 28) & 3, link = rec.x >> 26;
+                    const i64 K = sKtab[rec.x >> 26];
                     i64 best; int arg;
-                    cell(d, j, mask, link, capt, klo, khi, prevbuf + (rec.x & 0x03ffffffu) , rc_mask, best, arg);
+                    cell(a_prevbuf + 8u * (rec.x & 0x03ffffffu), j, klo, khi, a_thr + rec.z, a_sR + 8u * rec.w, K, rc_mask, best, arg);
                     cur[e] = best;
                     chd[e] = (uint8_t)arg;
                     alive |= best < kInf;
@@ -408,8 +442,16 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         }
         HAP_TQ(long long tq4 = clock64(); tq_lv += tq4 - tq3;)
         // ---- one thread per mapping: cell (PP, N), backtrace, Eq. 4 ---------------------------------
+        auto stage_K = [&](int d, int mask, int link) -> i64 {
+            i64 K = 0;
+            const MaskInfo<i64> &mi = minfo[mask - 1];
+            if (d == 1) K += mi.kpre;
+            if (d == PP) K += mi.kpost;
+            if (d > 1) { const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3; K += sP2P[hb][cls == HAP_CROSS ? 2 + ha : cls]; }
+            return K;
+        };
         int any_plan = 0;
-        const i64 *lastbuf = PP == 1 ? szero : (((PP - 1) & 1) ? bufO : bufE);
+        const u32 a_last = smem_u32(PP == 1 ? szero : (((PP - 1) & 1) ? bufO : bufE));
         for (u32 m = tid; m < tm.nmap; m += nthreads) {
             const u64 c = pc.offset + (u64)m * n_rc + (u64)rc_idx;
             if (c < w_lo || c >= w_hi) continue;
@@ -425,7 +467,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 if (!ldead) {
                     int klo = N - nmax; if (klo < pbl) klo = pbl;
                     int khi = N - nmin; if (khi > pbh) khi = pbh;
-                    cell(PP, N, mask, link, capt, klo, khi, lastbuf + prowoff - pbl, rc_mask, bott, arg);
+                    cell(a_last + 8u * prowoff - 8u * (u32)pbl, N, klo, khi, a_thr + trie_thr_index(tm, T, R, PP, capt, 0, N),
+                         a_sR + 8u * (u32)tm.mrow_of[mask] * (u32)(R * n1), stage_K(PP, mask, link), rc_mask, bott, arg);
                 }
             }
             if (SEARCH) n_eval++;
@@ -446,12 +489,11 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     parent = tm.parent[tm.node_lo[d - 1] + node];
                 }
                 const MaskInfo<i64> &mi = minfo[mask - 1];
-                const uint8_t *th = thr + ((size_t)(d - 1) * T + mi.capt) * R * n1;
+                const uint8_t *th = thr + trie_thr_index(tm, T, R, d, mi.capt, 0, b);
                 int r = 0;
                 for (; r < R; ++r)
-                    if (((rc_mask >> r) & 1u) && th[(size_t)r * n1 + b] <= a) break;
-                const int mrow = multiset ? __ffs(mask) - 1 : mask - 1;
-                const i64 *rr = sR + ((size_t)mrow * R + r) * n1;
+                    if (((rc_mask >> r) & 1u) && th[r * bw] <= a) break;
+                const i64 *rr = sR + ((size_t)tm.mrow_of[mask] * R + r) * n1;
                 const i64 cst = (rr[b] - rr[a]) + stage_K(d, mask, link);
                 sum += cst; mxc = cst > mxc ? cst : mxc;
                 const i64 n_moe = (i64)((int)sK[b] - (int)sK[a]), n_dense = (i64)(b - a) - n_moe;
