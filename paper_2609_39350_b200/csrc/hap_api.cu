@@ -494,7 +494,7 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
         cells[c].z = (u32)((((d - 1) * T + capt_of[nodes[g].mask]) * R) * band_max + (j - (int)tm.jlo[d]));
     }
     tm.band_max = band_max;
-    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, band_max, tm.buf_cells[0], tm.buf_cells[1], n_cells);
+    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, band_max, tm.buf_cells[0], tm.buf_cells[1], n_cells, n_nodes);
     if (smem > 220 * 1024) return false;
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];
@@ -839,11 +839,15 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         // fp64, cell counting and the one-candidate re-evaluation stay in pipeline_dp_kernel
         if (cl.trie.ok && !f64 && !out.count_only && !refine && lin && !out.dp_table && !out.choice && out.count > 1) {
             const hap_problem::Trie &tr = cl.trie;
-            const void *tfn = search ? (const void *)trie_dp_kernel<true> : (const void *)trie_dp_kernel<false>;
-            static size_t trie_limit[64][2];
-            if (tr.smem > trie_limit[dev][search ? 1 : 0]) {
+            // 64 registers per thread in both shapes (measured: more warps per SM beat more registers per thread)
+            const int tv = tr.threads > 512 ? 0 : 1;
+            const void *tfn = search ? (tv == 0 ? (const void *)trie_dp_kernel<true, 1024, 1> : (const void *)trie_dp_kernel<true, 512, 2>)
+                                     : (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1> : (const void *)trie_dp_kernel<false, 512, 2>);
+            static size_t trie_limit[64][6];
+            const int vi = (search ? 3 : 0) + tv;
+            if (tr.smem > trie_limit[dev][vi]) {
                 CUDA_TRY(p, cudaFuncSetAttribute(tfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tr.smem));
-                trie_limit[dev][search ? 1 : 0] = tr.smem;
+                trie_limit[dev][vi] = tr.smem;
             }
             CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
             // candidate decode of this pass, then its stage bytes into the tree

@@ -67,7 +67,8 @@ struct TrieMeta {
 
 constexpr int kTrieKtab = 16 + HAP_MAX_TYPES * 6;    // stage constants: [0,16) pre-work by row group, then p2p [type][6]
 
-__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, int n_mrows, int band_max, u32 buf_even, u32 buf_odd, u32 cells)
+__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, int n_mrows, int band_max, u32 buf_even, u32 buf_odd, u32 cells,
+                                                  u32 n_nodes)
 {
     const size_t n1 = (size_t)N + 1;
     size_t b = (((size_t)n_mrows * R + 2) * n1 * 8 + 15) / 16 * 16;      // time rows, weight and activation byte rows
@@ -77,6 +78,7 @@ __host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, i
     b += (size_t)kTrieKtab * 8;
     b += ((size_t)buf_even + buf_odd) * 8;
     b += ((size_t)cells + 15) / 16 * 16;
+    b += (size_t)n_nodes * 16 + ((size_t)n_nodes * 2 + 15) / 16 * 16;      // node records and parent indices
     return b + 32;
 }
 
@@ -131,17 +133,17 @@ __device__ __forceinline__ int lds_u8(u32 a)
     return (int)v;
 }
 
-// Block prologue, part 1: layer times of the configuration staged in shared memory, then per type mask that
-// occurs in the class the prefix rows of the stage time at every recomputation level (fwd+bwd + (tau_r/1024) fwd),
-// the weight and activation byte prefixes, MoE prefix counts, per-mask stage info, p2p coefficients and the
-// table of stage constants.
+// Block prologue, part 1: layer times of the configuration staged in shared memory, the weight and activation
+// byte prefixes, MoE prefix counts, per-mask stage info, p2p coefficients, the table of stage constants and a
+// copy of the tree's node records: what decides whether any mapping of the configuration can be feasible.
 __device__ __forceinline__ void trie_prologue_rows(
     const DevConst &dc, const TrieMeta &tm, unsigned p_index, const i64 *c2, const i64 *coef,
-    i64 *sC, i64 *sR, i64 *sW, i64 *sA, uint8_t *sK, i64 *sKtab, MaskInfo<i64> *minfo, i64 (*sP2P)[6], i64 *szero)
+    i64 *sC, i64 *sW, i64 *sA, uint8_t *sK, i64 *sKtab, TrieNode *sNodes, uint16_t *sParent,
+    MaskInfo<i64> *minfo, i64 (*sP2P)[6], i64 *szero)
 {
-    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
+    const int N = dc.N, T = dc.T;
     const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, wib = tid >> 5, lane = tid & 31;
-    const int nmask = (1 << T) - 1, mrows = tm.n_mrows;
+    const int nmask = (1 << T) - 1;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     {
         const longlong2 *src = reinterpret_cast<const longlong2 *>(c2 + (size_t)p_index * T * N * 2);
@@ -179,27 +181,56 @@ __device__ __forceinline__ void trie_prologue_rows(
         sKtab[16 + q] = v;
     }
     if (tid == 0) szero[0] = 0;
-    __syncthreads();
-    // rows: one warp per type mask (and one for the byte prefixes), inclusive warp scans over chunks of 32 layers
-    for (int mr = wib; mr <= mrows; mr += nwarps) {
-        const bool bytes = mr == mrows;
-        const int mk = bytes ? 0 : tm.mask_of_row[mr];
+    // the tree's node records (for the walk back through a mapping's ancestors)
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(tm.nodes);
+        uint4 *dst = reinterpret_cast<uint4 *>(sNodes);
+        const u32 n_nodes = tm.node_lo[tm.PP];
+        for (u32 q = tid; q < n_nodes; q += nthreads) { dst[q] = src[q]; sParent[q] = tm.parent[q]; }
+    }
+    // weight and activation byte prefixes: one warp, inclusive scans over chunks of 32 layers
+    if (wib == nwarps - 1) {
         i64 runA = 0, runB = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
-            i64 vA = 0, vB = 0;                                      // times: fwd+bwd, fwd; bytes: weights, activations
+            i64 vA = 0, vB = 0;
+            if (l < N) { const int kd = layer_kind(dc, l); vA = cfp[HAP_MW + kd]; vB = cfp[HAP_MA + kd]; }
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const i64 tA = __shfl_up_sync(0xffffffffu, vA, o), tB = __shfl_up_sync(0xffffffffu, vB, o);
+                if (lane >= o) { vA += tA; vB += tB; }
+            }
+            vA += runA; vB += runB;
+            if (l < N) { sW[l + 1] = vA; sA[l + 1] = vB; }
+            runA = shfl_i64(vA, 31); runB = shfl_i64(vB, 31);
+        }
+        if (lane == 0) { sW[0] = 0; sA[0] = 0; }
+    }
+    __syncthreads();
+}
+
+// Block prologue, part 2 (configurations that can be feasible): per type mask that occurs in the class the prefix
+// rows of the stage time at every recomputation level, fwd+bwd + (tau_r/1024) fwd; one warp per mask, inclusive
+// warp scans over chunks of 32 layers.  No barrier: the threshold sweep that follows ends with one.
+__device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, const TrieMeta &tm, const i64 *sC, i64 *sR)
+{
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
+    const int nwarps = blockDim.x >> 5, wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int mr = wib; mr < tm.n_mrows; mr += nwarps) {
+        const int mk = tm.mask_of_row[mr];
+        i64 runA = 0, runB = 0;
+        for (int base = 0; base < N; base += 32) {
+            const int l = base + lane;
+            i64 vA = 0, vB = 0;                                      // fwd+bwd, fwd
             if (l < N) {
-                if (bytes) { const int kd = layer_kind(dc, l); vA = cfp[HAP_MW + kd]; vB = cfp[HAP_MA + kd]; }
-                else {
-                    i64 F = 0, B = 0;
-                    for (int h = 0; h < T; ++h)
-                        if (mk >> h & 1) {
-                            const i64 qx = sC[((size_t)h * N + l) * 2], qy = sC[((size_t)h * N + l) * 2 + 1];
-                            F = qx > F ? qx : F;
-                            B = qy > B ? qy : B;
-                        }
-                    vA = F + B; vB = F;
-                }
+                i64 F = 0, B = 0;
+                for (int h = 0; h < T; ++h)
+                    if (mk >> h & 1) {
+                        const i64 qx = sC[((size_t)h * N + l) * 2], qy = sC[((size_t)h * N + l) * 2 + 1];
+                        F = qx > F ? qx : F;
+                        B = qy > B ? qy : B;
+                    }
+                vA = F + B; vB = F;
             }
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -207,18 +238,11 @@ __device__ __forceinline__ void trie_prologue_rows(
                 if (lane >= o) { vA += tA; vB += tB; }
             }
             vA += runA; vB += runB;
-            if (l < N) {
-                if (bytes) { sW[l + 1] = vA; sA[l + 1] = vB; }
-                else for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = vA + (i64)(dc.tau_q[r] >> 10) * vB;
-            }
+            if (l < N) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = vA + (i64)(dc.tau_q[r] >> 10) * vB;
             runA = shfl_i64(vA, 31); runB = shfl_i64(vB, 31);
         }
-        if (lane == 0) {
-            if (bytes) { sW[0] = 0; sA[0] = 0; }
-            else for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1] = 0;
-        }
+        if (lane == 0) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1] = 0;
     }
-    __syncthreads();
 }
 
 // index of the memory threshold of (stage d, capacity type t, level r, end layer j) in the block's table
@@ -266,8 +290,8 @@ __device__ __forceinline__ void trie_prologue_thr(
     __syncthreads();
 }
 
-template <bool SEARCH>
-__global__ void __launch_bounds__(1024, 1)
+template <bool SEARCH, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB)
 trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64 *c2, const i64 *coef,
                const TrieMeta tm, DpOut out)
 {
@@ -325,9 +349,11 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     i64 *bufE = sKtab + kTrieKtab;
     i64 *bufO = bufE + tm.buf_cells[0];
     uint8_t *ch = reinterpret_cast<uint8_t *>(bufO + tm.buf_cells[1]);
+    TrieNode *sNodes = reinterpret_cast<TrieNode *>(ch + ((size_t)tm.cell_lo[PP] + 15) / 16 * 16);
+    uint16_t *sParent = reinterpret_cast<uint16_t *>(sNodes + tm.node_lo[PP]);
 
     HAP_TQ(long long tq0 = clock64(); long long tq_lv = 0; long long tq_leaf = 0;)
-    trie_prologue_rows(dc, tm, p, c2, coef, sC, sR, sW, sA, sK, sKtab, minfo, sP2P, szero);
+    trie_prologue_rows(dc, tm, p, c2, coef, sC, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
     HAP_TQ(long long tq1 = clock64();)
     const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
 
@@ -355,7 +381,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         for (u32 e = tid; e < n_first * (u32)R; e += nthreads) {
             const u32 nd_i = e / R; const int r = (int)(e % R);
             if (!((all_levels >> r) & 1u)) continue;
-            const TrieNode nd = tm.nodes[tm.node_lo[1] + nd_i];
+            const TrieNode nd = sNodes[tm.node_lo[1] + nd_i];
             if (nd.bl > nd.bh) continue;
             const int capt = minfo[nd.mask - 1].capt;
             const i64 mstore = pc.M < PP ? pc.M : PP;
@@ -364,7 +390,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         }
         config_dead = !__syncthreads_or(fits);
     }
-    if (!config_dead) trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
+    if (!config_dead) {
+        trie_prologue_time_rows(dc, tm, sC, sR);
+        trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
+    }
     HAP_TQ(long long tq2 = clock64();)
 
     const u32 a_thr = smem_u32(thr), a_sR = smem_u32(sR);
@@ -417,6 +446,9 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         HAP_TQ(long long tq3 = clock64();)
         // ---- rows of the tree, depth by depth ------------------------------------------------
         if (!dead) {
+            // a thread's first cell record of a depth is requested before the barrier that ends the previous depth
+            TrieCell nxt = make_uint4(0, 0, 0, 0);
+            if (PP > 1 && (u32)tid < tm.cell_lo[2] - tm.cell_lo[1]) nxt = __ldcs(tm.cells + tm.cell_lo[1] + tid);
             for (int d = 1; d < PP; ++d) {
                 const u32 ncell = tm.cell_lo[d + 1] - tm.cell_lo[d];
                 const TrieCell *cells = tm.cells + tm.cell_lo[d];
@@ -424,11 +456,9 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 i64 *cur = (d & 1) ? bufO : bufE;
                 const u32 a_prevbuf = smem_u32(d == 1 ? szero : ((d & 1) ? bufE : bufO)) - 256u * 8u;
                 int alive = 0;
-                TrieCell nxt = make_uint4(0, 0, 0, 0);
-                if ((u32)tid < ncell) nxt = __ldg(cells + tid);
                 for (u32 e = tid; e < ncell; e += nthreads) {
                     const TrieCell rec = nxt;
-                    if (e + nthreads < ncell) nxt = __ldg(cells + e + nthreads);      // next record while this cell runs
+                    if (e + nthreads < ncell) nxt = __ldcs(cells + e + nthreads);     // next record while this cell runs (streamed past L1)
                     const int j = rec.y & 255, klo = (rec.y >> 8) & 255, khi = (rec.y >> 16) & 255;
                     const i64 K = sKtab[rec.x >> 26];
                     i64 best; int arg;
@@ -437,6 +467,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     chd[e] = (uint8_t)arg;
                     alive |= best < kInf;
                 }
+                if (d + 1 < PP && (u32)tid < tm.cell_lo[d + 2] - tm.cell_lo[d + 1]) nxt = __ldcs(tm.cells + tm.cell_lo[d + 1] + tid);
                 if (!__syncthreads_or(alive)) { dead = true; break; }   // no cell of this depth is finite: nothing below is
             }
         }
@@ -485,8 +516,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 uint4 raw = make_uint4(0, 0, 0, 0);
                 u32 parent = 0;
                 if (d > 1) {
-                    raw = __ldg(reinterpret_cast<const uint4 *>(tm.nodes + tm.node_lo[d - 1] + node));
-                    parent = tm.parent[tm.node_lo[d - 1] + node];
+                    raw = *reinterpret_cast<const uint4 *>(sNodes + tm.node_lo[d - 1] + node);
+                    parent = sParent[tm.node_lo[d - 1] + node];
                 }
                 const MaskInfo<i64> &mi = minfo[mask - 1];
                 const uint8_t *th = thr + trie_thr_index(tm, T, R, d, mi.capt, 0, b);
