@@ -335,7 +335,8 @@ def main():
             clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"]),
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                      ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
-            gpu_launches=(4 + 2 * len(set(int(x) for x in pconfs["PP"]))) * args.steps,
+            # per step: type_const, layer_cost, per PP class (decode, tree gather, tree DP), argmin partial + final
+            gpu_launches=(4 + 3 * len(set(int(x) for x in pconfs["PP"]))) * args.steps,
             **extra_modes,
             joint_recurrence_ms=joint_ms,
             full_search_ms=statistics.median(search_ms),
@@ -343,15 +344,16 @@ def main():
                                     n_evaluated=stats_pr["n_evaluated"]),
             best=dict(cost=best[0], index=best[1], search_index=plan["index"]),
             kernels_ms=dict(layer_cost=lc_med, pipeline_dp=dp_med),
-            roofline=dict(bound="alu", kernel="pipeline_dp_kernel (one launch per PP class, concurrent streams)",
+            roofline=dict(bound="alu", kernel="trie_dp_kernel (one launch per PP class, concurrent streams)",
                           achieved=achieved, peak=alu_peak, unit="Tops/s", frac=achieved / alu_peak,
                           traffic=NCU_DP_TRAFFIC_BYTES.get(args.workload) if args.delta_q is None else None,
                           ops_per_cell=4, cells_finite_cost=cells_finite, cells_plain_recurrence=cells_plain,
                           cells_visited=cells, frac_plain_recurrence=4.0 * cells_plain / (dp_med * 1e-3) / 1e12 / alu_peak,
                           note="achieved = 4 ops x cells whose stage cost is finite (inside the load-balance window and "
                                "the memory limit), counted per candidate; the kernel visits fewer (cells_visited) because "
-                               "unreachable layers and stage prefixes shared by consecutive mappings are skipped, and the "
-                               "plain recurrence without the window would have cells_plain_recurrence",
+                               "unreachable layers are skipped and the rows of a stage prefix are computed once for all "
+                               "mappings that share it, and the plain recurrence without the window would have "
+                               "cells_plain_recurrence",
                           peak_source=f"{SM_COUNT} SMs x {SCHEDULERS_PER_SM} schedulers x {LANES} lanes x "
                           f"{peaks.get('sm_max_mhz', 1965.0)} MHz ({peak_kind} clock)", sm_mhz_seen=sm_mhz),
             roofline_layer_cost=dict(bound="hbm", kernel="layer_cost_kernel", achieved=lc_gbs, peak=peaks["hbm_gbs"],

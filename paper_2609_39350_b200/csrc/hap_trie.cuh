@@ -429,6 +429,9 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 const i64 v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
                 if (v0 <= best) { best = v0; a_arg = pa; }
                 if (v1 <= best) { best = v1; a_arg = pa - 8; }
+                // layer times are non-negative, so the stage cost only grows as k falls within a level: once it
+                // exceeds the best value no further split of this level can reach it
+                if (c1 > best) break;
                 pa -= 16; ra -= 16;
             }
             seg_hi = lo - 1;
