@@ -35,8 +35,10 @@ struct hap_problem {
     uint64_t n_cand = 0;
     std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
     // prefix tree of a class's mappings (trie_dp_kernel); ok = false: the class runs in pipeline_dp_kernel only
-    struct Trie { bool ok; TrieMeta meta; unsigned char *d_blob; u32 *d_first_leaf, *d_gnode; uint8_t *d_depth; TrieNode *d_nodes; TrieLeaf *d_leaves;
-                  TrieCell *d_cells; u32 *d_plist; unsigned n_conf; u32 n_nodes, n_cells; int threads; size_t smem; };
+    struct TriePartDev { TrieNode *d_nodes; TrieLeaf *d_leaves; TrieCell *d_cells; u32 *d_first_leaf, *d_gnode; uint8_t *d_depth;
+                         u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
+    struct Trie { bool ok = false; unsigned char *d_blob = nullptr; TrieMeta *d_metas = nullptr; u32 *d_plist = nullptr;
+                  std::vector<TriePartDev> parts; unsigned n_conf = 0; int threads = 0; size_t smem = 0; };
     struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
@@ -123,7 +125,7 @@ static void release_device(hap_problem *p)
     cudaFree(p->d_range); cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist); }
+    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist); cudaFree(cl.trie.d_metas); }
 }
 
 extern "C" void hap_problem_destroy(hap_problem *p)
@@ -314,10 +316,21 @@ static uint64_t sequences_sat(const int *cnt, int T, uint64_t sat)
 // and the band of reachable end layers follow the same integer formulas as pipeline_dp_kernel; a node's
 // band is the union over the mappings below it, which only adds cells that hold their plain recurrence
 // value.  Returns false (and leaves the class on the general kernel) when the tree does not fit.
-static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, const std::vector<u32> &plist)
+struct TriePartHost {
+    TrieMeta meta;                          // device pointers are filled in after the upload
+    std::vector<unsigned char> blob;        // nodes | leaves | cells | first_leaf | cell_gnode | parent | depth
+    size_t o_nodes, o_leaves, o_cells, o_first, o_gnode, o_parent, o_depth;
+    u32 n_nodes, n_cells, nmap, max_level;
+    size_t smem;
+};
+
+// the tree of mappings [m0, m1) of the class
+static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, const uint8_t *tab_all, u64 m0, u64 m1, TriePartHost &part)
 {
     const int N = p->model.N, PP = cl.PP, T = p->T, R = p->prof.R;
-    if (nmap == 0 || nmap > 65535 || plist.empty()) return false;
+    const u64 nmap = m1 - m0;
+    const uint8_t *tab = tab_all + m0 * (u64)PP * 2;
+    if (nmap == 0 || nmap > 65535) return false;
     struct Key { uint8_t mask, link, nmin, nmax; };
     struct HNode { u32 parent; Key k; int bl, bh; u32 first_leaf; };
     std::vector<std::vector<HNode>> lv(PP + 1);               // lv[d], d = 1..PP-1
@@ -390,7 +403,7 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
             HNode nd;
             nd.parent = d > 1 ? path[d - 1] : 0;
             nd.k = Key{row[(d - 1) * 2], row[(d - 1) * 2 + 1], (uint8_t)nmin[d], (uint8_t)nmax[d]};
-            nd.bl = 1 << 20; nd.bh = -1; nd.first_leaf = (u32)m;
+            nd.bl = 1 << 20; nd.bh = -1; nd.first_leaf = (u32)(m0 + m);
             pkey[d] = nd.k;
             path[d] = (u32)lv[d].size();
             lv[d].push_back(nd);
@@ -416,10 +429,9 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
         else for (u64 m = 0; m < nmap; ++m) if (!leaves[m].dead) leaves[m].parent = (uint16_t)newidx[leaves[m].parent];
     }
     // flat layout
-    hap_problem::Trie &tr = cl.trie;
-    TrieMeta &tm = tr.meta;
+    TrieMeta &tm = part.meta;
     std::memset(&tm, 0, sizeof(tm));
-    tm.PP = PP; tm.nmap = (u32)nmap;
+    tm.PP = PP; tm.nmap = (u32)nmap; tm.m_lo = (u32)m0;
     // row groups of the time rows: one per type mask that some stage has
     std::memset(tm.mrow_of, 255, sizeof(tm.mrow_of));
     {
@@ -508,38 +520,82 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
         const int klo = std::max(N - (int)lf.nmax, (int)lf.pbl), khi = std::min(N - (int)lf.nmin, (int)lf.pbh);
         if (klo <= khi) { tm.kmin[PP] = std::min<uint8_t>(tm.kmin[PP], (uint8_t)klo); tm.kmax[PP] = std::max<uint8_t>(tm.kmax[PP], (uint8_t)khi); }
     }
-    // one allocation: nodes | leaves | cells | first_leaf | cell_gnode | parent | depth
+    // one blob: nodes | leaves | cells | first_leaf | cell_gnode | parent | depth
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
-    const size_t o_nodes = 0, o_leaves = up(o_nodes + (size_t)n_nodes * sizeof(TrieNode));
-    const size_t o_cells = up(o_leaves + nmap * sizeof(TrieLeaf));
-    const size_t o_first = up(o_cells + (size_t)n_cells * sizeof(TrieCell)), o_gnode = up(o_first + (size_t)n_nodes * 4);
-    const size_t o_parent = up(o_gnode + (size_t)n_cells * 4), o_depth = up(o_parent + (size_t)n_nodes * 2);
-    const size_t total = up(o_depth + n_nodes) + 256;
-    std::vector<unsigned char> blob(total, 0);
-    if (n_nodes) std::memcpy(blob.data() + o_nodes, nodes.data(), (size_t)n_nodes * sizeof(TrieNode));
-    std::memcpy(blob.data() + o_leaves, leaves.data(), nmap * sizeof(TrieLeaf));
-    if (n_cells) std::memcpy(blob.data() + o_cells, cells.data(), (size_t)n_cells * sizeof(TrieCell));
-    if (n_nodes) std::memcpy(blob.data() + o_first, first_leaf.data(), (size_t)n_nodes * 4);
-    if (n_cells) std::memcpy(blob.data() + o_gnode, cell_gnode.data(), (size_t)n_cells * 4);
-    if (n_nodes) std::memcpy(blob.data() + o_parent, parent.data(), (size_t)n_nodes * 2);
-    if (n_nodes) std::memcpy(blob.data() + o_depth, depth.data(), n_nodes);
+    part.o_nodes = 0; part.o_leaves = up(part.o_nodes + (size_t)n_nodes * sizeof(TrieNode));
+    part.o_cells = up(part.o_leaves + nmap * sizeof(TrieLeaf));
+    part.o_first = up(part.o_cells + (size_t)n_cells * sizeof(TrieCell)); part.o_gnode = up(part.o_first + (size_t)n_nodes * 4);
+    part.o_parent = up(part.o_gnode + (size_t)n_cells * 4); part.o_depth = up(part.o_parent + (size_t)n_nodes * 2);
+    const size_t total = up(part.o_depth + n_nodes) + 256;
+    part.blob.assign(total, 0);
+    unsigned char *blob = part.blob.data();
+    if (n_nodes) std::memcpy(blob + part.o_nodes, nodes.data(), (size_t)n_nodes * sizeof(TrieNode));
+    std::memcpy(blob + part.o_leaves, leaves.data(), nmap * sizeof(TrieLeaf));
+    if (n_cells) std::memcpy(blob + part.o_cells, cells.data(), (size_t)n_cells * sizeof(TrieCell));
+    if (n_nodes) std::memcpy(blob + part.o_first, first_leaf.data(), (size_t)n_nodes * 4);
+    if (n_cells) std::memcpy(blob + part.o_gnode, cell_gnode.data(), (size_t)n_cells * 4);
+    if (n_nodes) std::memcpy(blob + part.o_parent, parent.data(), (size_t)n_nodes * 2);
+    if (n_nodes) std::memcpy(blob + part.o_depth, depth.data(), n_nodes);
+    part.n_nodes = n_nodes; part.n_cells = n_cells; part.nmap = (u32)nmap; part.max_level = max_level; part.smem = smem;
+    return true;
+}
+
+// Builds the class's tree, as one part or, when one part would leave room for only one block per SM, as up to
+// eight parts over contiguous ranges of mappings (the few nodes near the root that two parts share are computed by
+// both), and uploads it.  Returns false (the class stays on the general kernel) when nothing fits.
+static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, const std::vector<u32> &plist)
+{
+    if (nmap == 0 || plist.empty()) return false;
+    constexpr size_t kTwoPerSm = 108 * 1024;                 // dynamic shared memory that lets two blocks share an SM
+    const size_t slots = (cl.item_hi - cl.item_lo) / plist.size();       // partial-result slots per configuration
+    std::vector<TriePartHost> parts, whole;
+    for (int np : {1, 2, 3, 4, 6, 8}) {
+        if ((u64)np > nmap || (np > 1 && (size_t)np > slots)) break;
+        std::vector<TriePartHost> cand(np);
+        bool ok = true;
+        size_t worst = 0;
+        for (int q = 0; q < np && ok; ++q) {
+            const u64 m0 = nmap * q / np, m1 = nmap * (q + 1) / np;
+            ok = build_trie_part(p, cl, tab, m0, m1, cand[q]);
+            if (ok) worst = std::max(worst, cand[q].smem);
+        }
+        if (np == 1 && ok) whole = cand;
+        if (ok && worst <= kTwoPerSm) { parts.swap(cand); break; }
+    }
+    if (parts.empty()) parts.swap(whole);                    // one block per SM
+    if (parts.empty()) return false;
+    hap_problem::Trie &tr = cl.trie;
+    size_t total = 0, smem = 0;
+    u32 want = 0;
+    for (const auto &pt : parts) { total += pt.blob.size(); smem = std::max(smem, pt.smem); want = std::max(want, std::max(pt.max_level, pt.nmap)); }
     if (cudaMalloc(&tr.d_blob, total) != cudaSuccess) { tr.d_blob = nullptr; cudaGetLastError(); return false; }
-    if (cudaMemcpy(tr.d_blob, blob.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    if (cudaMalloc(&tr.d_metas, parts.size() * sizeof(TrieMeta)) != cudaSuccess) { tr.d_metas = nullptr; cudaGetLastError(); return false; }
     if (cudaMalloc(&tr.d_plist, plist.size() * sizeof(u32)) != cudaSuccess) { tr.d_plist = nullptr; cudaGetLastError(); return false; }
     if (cudaMemcpy(tr.d_plist, plist.data(), plist.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess) return false;
-    tr.d_nodes = reinterpret_cast<TrieNode *>(tr.d_blob + o_nodes);
-    tr.d_leaves = reinterpret_cast<TrieLeaf *>(tr.d_blob + o_leaves);
-    tr.d_cells = reinterpret_cast<TrieCell *>(tr.d_blob + o_cells);
-    tr.d_first_leaf = reinterpret_cast<u32 *>(tr.d_blob + o_first);
-    tr.d_gnode = reinterpret_cast<u32 *>(tr.d_blob + o_gnode);
-    tr.d_depth = tr.d_blob + o_depth;
-    tm.nodes = tr.d_nodes; tm.leaves = tr.d_leaves; tm.cells = tr.d_cells;
-    tm.parent = reinterpret_cast<const uint16_t *>(tr.d_blob + o_parent);
-    tr.n_cells = n_cells;
-    tr.n_conf = (unsigned)plist.size(); tr.n_nodes = n_nodes; tr.smem = smem;
-    const u32 want = std::max<u32>(max_level, (u32)nmap);
-    int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
-    tr.threads = std::min(1024, std::max(128, th));
+    size_t off = 0;
+    std::vector<TrieMeta> metas;
+    for (auto &pt : parts) {
+        unsigned char *base = tr.d_blob + off;
+        if (cudaMemcpy(base, pt.blob.data(), pt.blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) return false;
+        hap_problem::TriePartDev pd{};
+        pd.d_nodes = reinterpret_cast<TrieNode *>(base + pt.o_nodes);
+        pd.d_leaves = reinterpret_cast<TrieLeaf *>(base + pt.o_leaves);
+        pd.d_cells = reinterpret_cast<TrieCell *>(base + pt.o_cells);
+        pd.d_first_leaf = reinterpret_cast<u32 *>(base + pt.o_first);
+        pd.d_gnode = reinterpret_cast<u32 *>(base + pt.o_gnode);
+        pd.d_depth = base + pt.o_depth;
+        pd.n_nodes = pt.n_nodes; pd.n_cells = pt.n_cells; pd.nmap = pt.nmap; pd.m_lo = pt.meta.m_lo;
+        std::memcpy(pd.mrow_of, pt.meta.mrow_of, sizeof(pd.mrow_of));
+        pt.meta.nodes = pd.d_nodes; pt.meta.leaves = pd.d_leaves; pt.meta.cells = pd.d_cells;
+        pt.meta.parent = reinterpret_cast<const uint16_t *>(base + pt.o_parent);
+        tr.parts.push_back(pd);
+        metas.push_back(pt.meta);
+        off += pt.blob.size();
+    }
+    if (cudaMemcpy(tr.d_metas, metas.data(), metas.size() * sizeof(TrieMeta), cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    tr.n_conf = (unsigned)plist.size(); tr.smem = smem;
+    const int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
+    tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
     tr.ok = true;
     return true;
 }
@@ -698,11 +754,16 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 unsigned used = 0;
                 for (u64 e = 0; e < nmap * (u64)cl.PP; ++e) used |= 1u << tab[cl.map_base + e * 2];
                 cl.masks_used = used;
-                if (!(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear) {
+                // the tree kernel holds times as doubles: exact while every prefix row stays below 2^52, which the
+                // per-layer limit of 2^36 ns guarantees when N (2 + max tau) <= 2^16
+                int tau_max = 0;
+                for (int r = 0; r < p->prof.R; ++r) tau_max = std::max(tau_max, p->tau_q[r] >> 10);
+                const bool rows_exact = (int64_t)N * (2 + tau_max) <= 65536;
+                if (!(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear && rows_exact) {
                     std::vector<u32> plist;
                     for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == cl.PP) plist.push_back((u32)pi);
                     if (!build_trie(p, cl, tab.data() + cl.map_base, nmap, plist)) {
-                        cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist);
+                        cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist); cudaFree(cl.trie.d_metas);
                         cl.trie = hap_problem::Trie{};
                     }
                 }
@@ -851,19 +912,23 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             }
             CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
             // candidate decode of this pass, then its stage bytes into the tree
-            const u64 nmap = tr.meta.nmap;
+            const u64 nmap = p->pconfs[p->items[cl.item_lo].p].nmap;
             maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, p->items[cl.item_lo].p, nmap, p->d_maptab + cl.map_base);
             CUDA_TRY(p, cudaGetLastError());
-            const u32 n_g = tr.n_nodes + tr.n_cells + (u32)nmap;
-            TrieRowMap rmap;
-            std::memcpy(rmap.mrow_of, tr.meta.mrow_of, sizeof(rmap.mrow_of));
-            trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, tr.n_nodes, tr.n_cells, (u32)nmap, tr.d_first_leaf, tr.d_depth,
-                                                                          tr.d_gnode, rmap, tr.d_nodes, tr.d_cells, tr.d_leaves);
-            CUDA_TRY(p, cudaGetLastError());
-            unsigned n_active = tr.n_conf;
+            for (const auto &pd : tr.parts) {
+                const u32 n_g = pd.n_nodes + pd.n_cells + pd.nmap;
+                TrieRowMap rmap;
+                std::memcpy(rmap.mrow_of, pd.mrow_of, sizeof(rmap.mrow_of));
+                trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, pd.n_nodes, pd.n_cells, pd.nmap, pd.m_lo, pd.d_first_leaf,
+                                                                              pd.d_depth, pd.d_gnode, rmap, pd.d_nodes, pd.d_cells, pd.d_leaves);
+                CUDA_TRY(p, cudaGetLastError());
+            }
+            int n_parts = (int)tr.parts.size();
+            unsigned n_active = tr.n_conf * (unsigned)n_parts;
             const u32 *plist = tr.d_plist;
-            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&tr.meta, (void *)&o};
-            const unsigned tblocks = search ? blocks : tr.n_conf;       // search: every partial slot of the class is written
+            const TrieMeta *metas = tr.d_metas;
+            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&metas, (void *)&n_parts, (void *)&o};
+            const unsigned tblocks = search ? std::max(blocks, n_active) : n_active;       // search: every partial slot of the class is written
             CUDA_TRY(p, cudaLaunchKernel(tfn, dim3(tblocks), dim3(tr.threads), targs, tr.smem, cl.stream));
             CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
             CUDA_TRY(p, cudaStreamWaitEvent(st, cl.done, 0));

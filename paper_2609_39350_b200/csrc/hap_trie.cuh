@@ -61,7 +61,7 @@ struct TrieMeta {
     uint8_t mask_of_row[16];        // the inverse
     int n_mrows;
     u32 buf_cells[2];               // largest row storage of an even / odd depth, in cells
-    u32 nmap;
+    u32 nmap, m_lo;                 // the tree covers mappings [m_lo, m_lo + nmap) of the class
     int PP, band_max;               // band_max: most end layers of any depth
 };
 
@@ -87,7 +87,7 @@ struct TrieRowMap { uint8_t mrow_of[16]; };
 // Copies what the decode of this pass produced into the tree: node n of depth d takes the stage bytes (device
 // types, boundary link) of stage d of the first mapping below it, every cell of the node the index of the stage
 // constant that follows from them, leaf m the last stage of mapping m.
-__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap,
+__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap, u32 m_lo,
                                    const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
                                    const u32 *__restrict__ cell_gnode, const TrieRowMap rm,
                                    TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves)
@@ -107,7 +107,7 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
         *x = (*x & 0x03ffffffu) | (kidx << 26);
     } else if (g < n_nodes + n_cells + nmap) {
         const u32 m = g - n_nodes - n_cells;
-        const uint8_t *src = maptab + ((u64)m * PP + (PP - 1)) * 2;
+        const uint8_t *src = maptab + ((u64)(m_lo + m) * PP + (PP - 1)) * 2;
         leaves[m].mask = src[0]; leaves[m].link = src[1];
     }
 }
@@ -126,6 +126,12 @@ template <int OFF> __device__ __forceinline__ i64 lds_i64(u32 a)
     asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(v) : "r"(a), "n"(OFF));
     return v;
 }
+template <int OFF> __device__ __forceinline__ double lds_f64(u32 a)
+{
+    double v;
+    asm volatile("ld.shared.f64 %0, [%1+%2];" : "=d"(v) : "r"(a), "n"(OFF));
+    return v;
+}
 __device__ __forceinline__ int lds_u8(u32 a)
 {
     u32 v;
@@ -138,8 +144,8 @@ __device__ __forceinline__ int lds_u8(u32 a)
 // copy of the tree's node records: what decides whether any mapping of the configuration can be feasible.
 __device__ __forceinline__ void trie_prologue_rows(
     const DevConst &dc, const TrieMeta &tm, unsigned p_index, const i64 *c2, const i64 *coef,
-    i64 *sC, i64 *sW, i64 *sA, uint8_t *sK, i64 *sKtab, TrieNode *sNodes, uint16_t *sParent,
-    MaskInfo<i64> *minfo, i64 (*sP2P)[6], i64 *szero)
+    i64 *sC, i64 *sW, i64 *sA, uint8_t *sK, double *sKtab, TrieNode *sNodes, uint16_t *sParent,
+    MaskInfo<i64> *minfo, i64 (*sP2P)[6], double *szero)
 {
     const int N = dc.N, T = dc.T;
     const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, wib = tid >> 5, lane = tid & 31;
@@ -172,15 +178,15 @@ __device__ __forceinline__ void trie_prologue_rows(
                 seen = true;
             }
         minfo[tid] = mi;
-        if (tm.mrow_of[mk] != 255) sKtab[tm.mrow_of[mk]] = mi.kpre;
+        if (tm.mrow_of[mk] != 255) sKtab[tm.mrow_of[mk]] = (double)mi.kpre;
     }
     if (tid >= 32 && tid < 32 + T * 6) {
         const int q = tid - 32, h = q / 6, e = q % 6;
         const i64 v = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
         sP2P[h][e] = v;
-        sKtab[16 + q] = v;
+        sKtab[16 + q] = (double)v;
     }
-    if (tid == 0) szero[0] = 0;
+    if (tid == 0) szero[0] = 0.0;
     // the tree's node records (for the walk back through a mapping's ancestors)
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(tm.nodes);
@@ -212,7 +218,7 @@ __device__ __forceinline__ void trie_prologue_rows(
 // Block prologue, part 2 (configurations that can be feasible): per type mask that occurs in the class the prefix
 // rows of the stage time at every recomputation level, fwd+bwd + (tau_r/1024) fwd; one warp per mask, inclusive
 // warp scans over chunks of 32 layers.  No barrier: the threshold sweep that follows ends with one.
-__device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, const TrieMeta &tm, const i64 *sC, i64 *sR)
+__device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, const TrieMeta &tm, const i64 *sC, double *sR)
 {
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int nwarps = blockDim.x >> 5, wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -238,10 +244,10 @@ __device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, cons
                 if (lane >= o) { vA += tA; vB += tB; }
             }
             vA += runA; vB += runB;
-            if (l < N) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = vA + (i64)(dc.tau_q[r] >> 10) * vB;
+            if (l < N) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = (double)(vA + (i64)(dc.tau_q[r] >> 10) * vB);
             runA = shfl_i64(vA, 31); runB = shfl_i64(vB, 31);
         }
-        if (lane == 0) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1] = 0;
+        if (lane == 0) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1] = 0.0;
     }
 }
 
@@ -293,12 +299,12 @@ __device__ __forceinline__ void trie_prologue_thr(
 template <bool SEARCH, int MAXT, int MINB>
 __global__ void __launch_bounds__(MAXT, MINB)
 trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64 *c2, const i64 *coef,
-               const TrieMeta tm, DpOut out)
+               const TrieMeta *metas, int n_parts, DpOut out)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ MaskInfo<i64> minfo[kMaxMasks];
     __shared__ i64 sP2P[HAP_MAX_TYPES][6];
-    __shared__ i64 szero[1];
+    __shared__ double szero[1];
     __shared__ i64 wcost[32];
     __shared__ u64 widx[32];
     __shared__ int s_skip;
@@ -308,10 +314,18 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         if (SEARCH && tid == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
         return;
     }
-    const u32 p = plist[blockIdx.x];
+    // block -> (configuration, part of the class's tree); the part's description goes to shared memory
+    __shared__ TrieMeta tm;
+    {
+        const u32 *src = reinterpret_cast<const u32 *>(metas + blockIdx.x % (unsigned)n_parts);
+        u32 *dst = reinterpret_cast<u32 *>(&tm);
+        for (int q = tid; q < (int)(sizeof(TrieMeta) / 4); q += nthreads) dst[q] = src[q];
+    }
+    __syncthreads();
+    const u32 p = plist[blockIdx.x / (unsigned)n_parts];
     const hap_pconf pc = dc.pconf[p];
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.band_max;
-    const u64 c_lo = pc.offset, c_hi = pc.offset + (u64)tm.nmap * n_rc;        // candidates of this configuration
+    const u64 c_lo = pc.offset + (u64)tm.m_lo * n_rc, c_hi = c_lo + (u64)tm.nmap * n_rc;   // candidates of this block
     const u64 w_lo = out.first, w_hi = out.first + out.count;                  // candidates that are wanted
     if (c_hi <= w_lo || c_lo >= w_hi) {
         if (SEARCH && tid == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
@@ -337,17 +351,17 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
 
     // shared memory: time rows | weight bytes | activation bytes | thresholds | MoE counts | staged layer times |
     //                stage constants | rows of the even depths | rows of the odd depths | split choices
-    i64 *sR = reinterpret_cast<i64 *>(smem_raw);
-    i64 *sW = sR + (size_t)tm.n_mrows * R * n1;
+    double *sR = reinterpret_cast<double *>(smem_raw);
+    i64 *sW = reinterpret_cast<i64 *>(sR + (size_t)tm.n_mrows * R * n1);
     i64 *sA = sW + n1;
     const size_t thr_off = (((size_t)tm.n_mrows * R + 2) * n1 * 8 + 15) / 16 * 16;
     uint8_t *thr = smem_raw + thr_off;
     const size_t thr_bytes = ((size_t)PP * T * R * bw + 15) / 16 * 16;
     uint8_t *sK = thr + thr_bytes;
     i64 *sC = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);      // [T][N][2], 16-byte aligned
-    i64 *sKtab = sC + (size_t)T * N * 2;
-    i64 *bufE = sKtab + kTrieKtab;
-    i64 *bufO = bufE + tm.buf_cells[0];
+    double *sKtab = reinterpret_cast<double *>(sC + (size_t)T * N * 2);
+    double *bufE = sKtab + kTrieKtab;
+    double *bufO = bufE + tm.buf_cells[0];
     uint8_t *ch = reinterpret_cast<uint8_t *>(bufO + tm.buf_cells[1]);
     TrieNode *sNodes = reinterpret_cast<TrieNode *>(ch + ((size_t)tm.cell_lo[PP] + 15) / 16 * 16);
     uint16_t *sParent = reinterpret_cast<uint16_t *>(sNodes + tm.node_lo[PP]);
@@ -369,7 +383,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
 
     i64 best_cost = kInf;
     u64 best_index = ~0ull;
-    u64 n_eval = 0, n_feas = 0, n_cells = 0;
+    u64 n_eval = 0, n_feas = 0;
+    u32 n_cells32 = 0;                  // splits this thread evaluated
     unsigned all_levels = 0;
     for (int q = 0; q < n_rc; ++q) all_levels |= dc.rc_masks[q];
 
@@ -401,10 +416,13 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     // One cell: min over k in [klo, khi] of max(prev[k], cost(k, j)), smallest k on ties.  k runs downward over the
     // level segments given by the memory thresholds (lowest allowed level that fits); prev[k] and the time row
     // entry of k are read through two addresses that step down together, two splits per step.
+    // Times are integer ns below 2^53 held as doubles: every sum, difference and comparison is exact, and the
+    // subtraction and the two comparisons of a split run on the fp64 pipe instead of as int64 pairs on the ALU pipe.
     //   a_prev: address of prev[0]; a_th: address of the level-0 threshold of (stage, j); a_row: address of entry 0
     //   of the level-0 time row of the stage's types; K: stage constant
-    auto cell = [&](u32 a_prev, int j, int klo, int khi, u32 a_th, u32 a_row, i64 K, unsigned rc_mask, i64 &best_out, int &arg_out) {
-        i64 best = kInf - 1;                    // every finite value is below this, an unreachable one (= kInf) above
+    const double dInf = 4611686018427387904.0;             // 2^62, the integer INF
+    auto cell = [&](u32 a_prev, int j, int klo, int khi, u32 a_th, u32 a_row, double K, unsigned rc_mask, double &best_out, int &arg_out) {
+        double best = 2305843009213693952.0;   // 2^61: every finite value is below this, an unreachable one (2^62) above
         u32 a_arg = 0;
         int seg_hi = khi;
         for (int r = 0; r < R && seg_hi >= klo; ++r, a_th += (u32)bw, a_row += (u32)n1 * 8u) {
@@ -413,20 +431,20 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             if (lo < klo) lo = klo;
             if (lo > seg_hi) continue;
             const int n = seg_hi - lo + 1;
-            n_cells += (u64)n;
-            const i64 Cj = lds_i64<0>(a_row + 8u * (u32)j) + K;
+            n_cells32 += (u32)n;
+            const double Cj = lds_f64<0>(a_row + 8u * (u32)j) + K;
             u32 pa = a_prev + 8u * (u32)seg_hi, ra = a_row + 8u * (u32)seg_hi;
             const u32 pa_lo = a_prev + 8u * (u32)lo;
             if (n & 1) {
-                const i64 p0 = lds_i64<0>(pa), c0 = Cj - lds_i64<0>(ra);
-                const i64 v0 = p0 > c0 ? p0 : c0;
+                const double p0 = lds_f64<0>(pa), c0 = Cj - lds_f64<0>(ra);
+                const double v0 = p0 > c0 ? p0 : c0;
                 if (v0 <= best) { best = v0; a_arg = pa; }
                 pa -= 8; ra -= 8;
             }
             while ((int)(pa - pa_lo) > 0) {      // pa and pa - 8 are both inside the segment
-                const i64 p0 = lds_i64<0>(pa), p1 = lds_i64<-8>(pa);
-                const i64 c0 = Cj - lds_i64<0>(ra), c1 = Cj - lds_i64<-8>(ra);
-                const i64 v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
+                const double p0 = lds_f64<0>(pa), p1 = lds_f64<-8>(pa);
+                const double c0 = Cj - lds_f64<0>(ra), c1 = Cj - lds_f64<-8>(ra);
+                const double v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
                 if (v0 <= best) { best = v0; a_arg = pa; }
                 if (v1 <= best) { best = v1; a_arg = pa - 8; }
                 // layer times are non-negative, so the stage cost only grows as k falls within a level: once it
@@ -436,7 +454,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             }
             seg_hi = lo - 1;
         }
-        best_out = a_arg ? best : kInf;
+        best_out = a_arg ? best : dInf;
         arg_out = a_arg ? (int)((a_arg - a_prev) >> 3) : 255;
     };
 
@@ -456,19 +474,19 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 const u32 ncell = tm.cell_lo[d + 1] - tm.cell_lo[d];
                 const TrieCell *cells = tm.cells + tm.cell_lo[d];
                 uint8_t *chd = ch + tm.cell_lo[d];
-                i64 *cur = (d & 1) ? bufO : bufE;
+                double *cur = (d & 1) ? bufO : bufE;
                 const u32 a_prevbuf = smem_u32(d == 1 ? szero : ((d & 1) ? bufE : bufO)) - 256u * 8u;
                 int alive = 0;
                 for (u32 e = tid; e < ncell; e += nthreads) {
                     const TrieCell rec = nxt;
                     if (e + nthreads < ncell) nxt = __ldcs(cells + e + nthreads);     // next record while this cell runs (streamed past L1)
                     const int j = rec.y & 255, klo = (rec.y >> 8) & 255, khi = (rec.y >> 16) & 255;
-                    const i64 K = sKtab[rec.x >> 26];
-                    i64 best; int arg;
+                    const double K = sKtab[rec.x >> 26];
+                    double best; int arg;
                     cell(a_prevbuf + 8u * (rec.x & 0x03ffffffu), j, klo, khi, a_thr + rec.z, a_sR + 8u * rec.w, K, rc_mask, best, arg);
                     cur[e] = best;
                     chd[e] = (uint8_t)arg;
-                    alive |= best < kInf;
+                    alive |= best < dInf;
                 }
                 if (d + 1 < PP && (u32)tid < tm.cell_lo[d + 2] - tm.cell_lo[d + 1]) nxt = __ldcs(tm.cells + tm.cell_lo[d + 1] + tid);
                 if (!__syncthreads_or(alive)) { dead = true; break; }   // no cell of this depth is finite: nothing below is
@@ -487,9 +505,9 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         int any_plan = 0;
         const u32 a_last = smem_u32(PP == 1 ? szero : (((PP - 1) & 1) ? bufO : bufE));
         for (u32 m = tid; m < tm.nmap; m += nthreads) {
-            const u64 c = pc.offset + (u64)m * n_rc + (u64)rc_idx;
+            const u64 c = c_lo + (u64)m * n_rc + (u64)rc_idx;
             if (c < w_lo || c >= w_hi) continue;
-            i64 bott = kInf; int arg = 255;
+            double bott_d = dInf; int arg = 255;
             int mask = 0, link = 0;
             u32 node = 0;
             if (!dead) {
@@ -502,10 +520,11 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     int klo = N - nmax; if (klo < pbl) klo = pbl;
                     int khi = N - nmin; if (khi > pbh) khi = pbh;
                     cell(a_last + 8u * prowoff - 8u * (u32)pbl, N, klo, khi, a_thr + trie_thr_index(tm, T, R, PP, capt, 0, N),
-                         a_sR + 8u * (u32)tm.mrow_of[mask] * (u32)(R * n1), stage_K(PP, mask, link), rc_mask, bott, arg);
+                         a_sR + 8u * (u32)tm.mrow_of[mask] * (u32)(R * n1), (double)stage_K(PP, mask, link), rc_mask, bott_d, arg);
                 }
             }
             if (SEARCH) n_eval++;
+            const i64 bott = bott_d < dInf ? (i64)bott_d : kInf;
             if (!(bott < kInf)) {
                 if (!SEARCH) put_infeasible(c);
                 continue;
@@ -527,8 +546,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 int r = 0;
                 for (; r < R; ++r)
                     if (((rc_mask >> r) & 1u) && th[r * bw] <= a) break;
-                const i64 *rr = sR + ((size_t)tm.mrow_of[mask] * R + r) * n1;
-                const i64 cst = (rr[b] - rr[a]) + stage_K(d, mask, link);
+                const double *rr = sR + ((size_t)tm.mrow_of[mask] * R + r) * n1;
+                const i64 cst = (i64)(rr[b] - rr[a]) + stage_K(d, mask, link);
                 sum += cst; mxc = cst > mxc ? cst : mxc;
                 const i64 n_moe = (i64)((int)sK[b] - (int)sK[a]), n_dense = (i64)(b - a) - n_moe;
                 const i64 sy = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
@@ -568,7 +587,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         // the barrier also keeps the next policy from overwriting rows and choices that are still being read
         const int bott_any = __syncthreads_or(any_plan);
         HAP_TQ(tq_leaf += clock64() - tq4;)
-        // a policy under which no mapping of the WHOLE configuration has a feasible partition settles its subsets
+        // a policy under which none of the block's mappings has a feasible partition settles its subsets
         if (!bott_any && c_lo >= w_lo && c_hi <= w_hi && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
     }
 
@@ -581,7 +600,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     }
 #endif
     if (out.counters) {
-        n_cells = (u64)warp_sum_i64((i64)n_cells);
+        const u64 n_cells = (u64)warp_sum_i64((i64)n_cells32);
         if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
     }
     if (SEARCH) {
