@@ -37,11 +37,13 @@ struct hap_problem {
     // prefix tree of a class's mappings (trie_dp_kernel); ok = false: the class runs in pipeline_dp_kernel only
     struct TriePartDev { TrieNode *d_nodes; TrieLeaf *d_leaves; TrieCell *d_cells; u32 *d_first_leaf, *d_gnode; uint8_t *d_depth;
                          u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
-    struct Trie { bool ok = false; unsigned char *d_blob = nullptr; TrieMeta *d_metas = nullptr; u32 *d_plist = nullptr;
+    struct Trie { bool ok = false; TrieMeta *d_metas = nullptr; u32 *d_plist = nullptr;       // both inside d_trie_arena
                   std::vector<TriePartDev> parts; unsigned n_conf = 0; int threads = 0; size_t smem = 0; };
     struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
+    unsigned char *d_arena = nullptr;      // everything hap_enumerate sizes, in one allocation (the d_* pointers below point into it)
+    unsigned char *d_trie_arena = nullptr; // the prefix trees of all classes
     // device
     DevConst dc{};
     double *d_tables = nullptr;            // all six tables in one allocation
@@ -119,13 +121,13 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 
 static void release_device(hap_problem *p)
 {
-    cudaFree(p->d_tables); cudaFree(p->d_pconf); cudaFree(p->d_items); cudaFree(p->d_c2); cudaFree(p->d_coef);
+    cudaFree(p->d_tables); cudaFree(p->d_arena); cudaFree(p->d_trie_arena);
     cudaFree(p->d_joint_scratch);
     for (auto &j : p->joint) { cudaFree(j.d_ids); cudaFree(j.d_arrays); }
-    cudaFree(p->d_range); cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost); cudaFree(p->d_lb); cudaFree(p->d_tc); cudaFree(p->d_maptab); cudaFree(p->d_pcost); cudaFree(p->d_pindex); cudaFree(p->d_counters); cudaFree(p->d_best); cudaFree(p->d_single);
+    cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist); cudaFree(cl.trie.d_metas); }
+    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); }
 }
 
 extern "C" void hap_problem_destroy(hap_problem *p)
@@ -542,8 +544,10 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
 
 // Builds the class's tree, as one part or, when one part would leave room for only one block per SM, as up to
 // eight parts over contiguous ranges of mappings (the few nodes near the root that two parts share are computed by
-// both), and uploads it.  Returns false (the class stays on the general kernel) when nothing fits.
-static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, const std::vector<u32> &plist)
+// both).  Returns false (the class stays on the general kernel) when nothing fits.
+struct TrieClassHost { std::vector<TriePartHost> parts; std::vector<u32> plist; };
+
+static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, const std::vector<u32> &plist, TrieClassHost &out)
 {
     if (nmap == 0 || plist.empty()) return false;
     constexpr size_t kTwoPerSm = 108 * 1024;                 // dynamic shared memory that lets two blocks share an SM
@@ -564,39 +568,67 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     }
     if (parts.empty()) parts.swap(whole);                    // one block per SM
     if (parts.empty()) return false;
-    hap_problem::Trie &tr = cl.trie;
-    size_t total = 0, smem = 0;
-    u32 want = 0;
-    for (const auto &pt : parts) { total += pt.blob.size(); smem = std::max(smem, pt.smem); want = std::max(want, std::max(pt.max_level, pt.nmap)); }
-    if (cudaMalloc(&tr.d_blob, total) != cudaSuccess) { tr.d_blob = nullptr; cudaGetLastError(); return false; }
-    if (cudaMalloc(&tr.d_metas, parts.size() * sizeof(TrieMeta)) != cudaSuccess) { tr.d_metas = nullptr; cudaGetLastError(); return false; }
-    if (cudaMalloc(&tr.d_plist, plist.size() * sizeof(u32)) != cudaSuccess) { tr.d_plist = nullptr; cudaGetLastError(); return false; }
-    if (cudaMemcpy(tr.d_plist, plist.data(), plist.size() * sizeof(u32), cudaMemcpyHostToDevice) != cudaSuccess) return false;
-    size_t off = 0;
-    std::vector<TrieMeta> metas;
-    for (auto &pt : parts) {
-        unsigned char *base = tr.d_blob + off;
-        if (cudaMemcpy(base, pt.blob.data(), pt.blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) return false;
-        hap_problem::TriePartDev pd{};
-        pd.d_nodes = reinterpret_cast<TrieNode *>(base + pt.o_nodes);
-        pd.d_leaves = reinterpret_cast<TrieLeaf *>(base + pt.o_leaves);
-        pd.d_cells = reinterpret_cast<TrieCell *>(base + pt.o_cells);
-        pd.d_first_leaf = reinterpret_cast<u32 *>(base + pt.o_first);
-        pd.d_gnode = reinterpret_cast<u32 *>(base + pt.o_gnode);
-        pd.d_depth = base + pt.o_depth;
-        pd.n_nodes = pt.n_nodes; pd.n_cells = pt.n_cells; pd.nmap = pt.nmap; pd.m_lo = pt.meta.m_lo;
-        std::memcpy(pd.mrow_of, pt.meta.mrow_of, sizeof(pd.mrow_of));
-        pt.meta.nodes = pd.d_nodes; pt.meta.leaves = pd.d_leaves; pt.meta.cells = pd.d_cells;
-        pt.meta.parent = reinterpret_cast<const uint16_t *>(base + pt.o_parent);
-        tr.parts.push_back(pd);
-        metas.push_back(pt.meta);
-        off += pt.blob.size();
+    out.parts.swap(parts);
+    out.plist = plist;
+    return true;
+}
+
+// One allocation and one copy for the trees of all classes: per class its parts' blobs, the part descriptions
+// and the list of the class's configurations.
+static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpClass *, TrieClassHost>> &built)
+{
+    constexpr size_t kTwoPerSm = 108 * 1024;
+    auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+    size_t total = 0;
+    for (auto &bc : built) {
+        for (const auto &pt : bc.second.parts) total += up(pt.blob.size());
+        total += up(bc.second.parts.size() * sizeof(TrieMeta)) + up(bc.second.plist.size() * sizeof(u32));
     }
-    if (cudaMemcpy(tr.d_metas, metas.data(), metas.size() * sizeof(TrieMeta), cudaMemcpyHostToDevice) != cudaSuccess) return false;
-    tr.n_conf = (unsigned)plist.size(); tr.smem = smem;
-    const int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
-    tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
-    tr.ok = true;
+    if (!total) return true;
+    if (cudaMalloc(&p->d_trie_arena, total) != cudaSuccess) { p->d_trie_arena = nullptr; cudaGetLastError(); return false; }
+    std::vector<unsigned char> stage(total, 0);
+    size_t off = 0;
+    for (auto &bc : built) {
+        hap_problem::Trie &tr = bc.first->trie;
+        TrieClassHost &h = bc.second;
+        std::vector<TrieMeta> metas;
+        size_t smem = 0;
+        u32 want = 0;
+        for (auto &pt : h.parts) {
+            unsigned char *base = p->d_trie_arena + off;
+            std::memcpy(stage.data() + off, pt.blob.data(), pt.blob.size());
+            hap_problem::TriePartDev pd{};
+            pd.d_nodes = reinterpret_cast<TrieNode *>(base + pt.o_nodes);
+            pd.d_leaves = reinterpret_cast<TrieLeaf *>(base + pt.o_leaves);
+            pd.d_cells = reinterpret_cast<TrieCell *>(base + pt.o_cells);
+            pd.d_first_leaf = reinterpret_cast<u32 *>(base + pt.o_first);
+            pd.d_gnode = reinterpret_cast<u32 *>(base + pt.o_gnode);
+            pd.d_depth = base + pt.o_depth;
+            pd.n_nodes = pt.n_nodes; pd.n_cells = pt.n_cells; pd.nmap = pt.nmap; pd.m_lo = pt.meta.m_lo;
+            std::memcpy(pd.mrow_of, pt.meta.mrow_of, sizeof(pd.mrow_of));
+            pt.meta.nodes = pd.d_nodes; pt.meta.leaves = pd.d_leaves; pt.meta.cells = pd.d_cells;
+            pt.meta.parent = reinterpret_cast<const uint16_t *>(base + pt.o_parent);
+            tr.parts.push_back(pd);
+            metas.push_back(pt.meta);
+            smem = std::max(smem, pt.smem);
+            want = std::max(want, std::max(pt.max_level, pt.nmap));
+            off += up(pt.blob.size());
+        }
+        tr.d_metas = reinterpret_cast<TrieMeta *>(p->d_trie_arena + off);
+        std::memcpy(stage.data() + off, metas.data(), metas.size() * sizeof(TrieMeta));
+        off += up(metas.size() * sizeof(TrieMeta));
+        tr.d_plist = reinterpret_cast<u32 *>(p->d_trie_arena + off);
+        std::memcpy(stage.data() + off, h.plist.data(), h.plist.size() * sizeof(u32));
+        off += up(h.plist.size() * sizeof(u32));
+        tr.n_conf = (unsigned)h.plist.size(); tr.smem = smem;
+        const int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
+        tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
+        tr.ok = true;
+    }
+    if (cudaMemcpy(p->d_trie_arena, stage.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
+        for (auto &bc : built) bc.first->trie = hap_problem::Trie{};
+        return false;
+    }
     return true;
 }
 
@@ -712,22 +744,42 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         p->classes.swap(classes);
         p->n_cand = off;
         const size_t np = p->pconfs.size();
-        CUDA_TRY(p, cudaMalloc(&p->d_pconf, np * sizeof(hap_pconf)));
-        CUDA_TRY(p, cudaMemcpy(p->d_pconf, p->pconfs.data(), np * sizeof(hap_pconf), cudaMemcpyHostToDevice));
-        CUDA_TRY(p, cudaMalloc(&p->d_items, p->items.size() * sizeof(WorkItem)));
-        CUDA_TRY(p, cudaMemcpy(p->d_items, p->items.data(), p->items.size() * sizeof(WorkItem), cudaMemcpyHostToDevice));
-        CUDA_TRY(p, cudaMalloc(&p->d_c2, np * T * N * 2 * sizeof(i64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_coef, np * T * HAP_NCOEF * sizeof(i64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_tc, np * T * sizeof(TypeConst)));
-        CUDA_TRY(p, cudaMalloc(&p->d_lb, np * sizeof(i64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_range, sizeof(u64)));
-        CUDA_TRY(p, cudaMemset(p->d_range, 0, sizeof(u64)));
+        // one allocation for everything whose size the enumeration fixes (an allocation costs far more than the
+        // microseconds a pass takes): configuration table | work items | layer costs | coefficients | per-type
+        // constants | lower bounds | partial minima | mapping tables | small scalars
         p->n_partial = std::max<size_t>(p->items.size(), 1024);
-        CUDA_TRY(p, cudaMalloc(&p->d_pcost, p->n_partial * sizeof(i64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_pindex, p->n_partial * sizeof(u64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_counters, 8 * sizeof(u64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_best, 2 * sizeof(i64)));
-        CUDA_TRY(p, cudaMalloc(&p->d_single, sizeof(SingleOut)));
+        {
+            auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+            size_t o = 0;
+            const size_t o_pconf = o; o = up(o + np * sizeof(hap_pconf));
+            const size_t o_items = o; o = up(o + p->items.size() * sizeof(WorkItem));
+            const size_t o_c2 = o; o = up(o + np * T * N * 2 * sizeof(i64));
+            const size_t o_coef = o; o = up(o + np * T * HAP_NCOEF * sizeof(i64));
+            const size_t o_tc = o; o = up(o + np * T * sizeof(TypeConst));
+            const size_t o_lb = o; o = up(o + np * sizeof(i64));
+            const size_t o_pcost = o; o = up(o + p->n_partial * sizeof(i64));
+            const size_t o_pindex = o; o = up(o + p->n_partial * sizeof(u64));
+            const size_t o_maptab = o; o = up(o + tab_bytes);
+            const size_t o_range = o; o = up(o + sizeof(u64));
+            const size_t o_counters = o; o = up(o + 8 * sizeof(u64));
+            const size_t o_best = o; o = up(o + 2 * sizeof(i64));
+            const size_t o_single = o; o = up(o + sizeof(SingleOut));
+            CUDA_TRY(p, cudaMalloc(&p->d_arena, o));
+            unsigned char *base = p->d_arena;
+            p->d_pconf = reinterpret_cast<hap_pconf *>(base + o_pconf); p->d_items = reinterpret_cast<WorkItem *>(base + o_items);
+            p->d_c2 = reinterpret_cast<i64 *>(base + o_c2); p->d_coef = reinterpret_cast<i64 *>(base + o_coef);
+            p->d_tc = reinterpret_cast<TypeConst *>(base + o_tc); p->d_lb = reinterpret_cast<i64 *>(base + o_lb);
+            p->d_pcost = reinterpret_cast<i64 *>(base + o_pcost); p->d_pindex = reinterpret_cast<u64 *>(base + o_pindex);
+            p->d_maptab = tab_bytes ? base + o_maptab : nullptr;
+            p->d_range = reinterpret_cast<u64 *>(base + o_range); p->d_counters = reinterpret_cast<u64 *>(base + o_counters);
+            p->d_best = reinterpret_cast<i64 *>(base + o_best); p->d_single = base + o_single;
+            // configuration table and work items travel in one copy (they are adjacent up to padding)
+            std::vector<unsigned char> stage(o_c2, 0);
+            std::memcpy(stage.data() + o_pconf, p->pconfs.data(), np * sizeof(hap_pconf));
+            std::memcpy(stage.data() + o_items, p->items.data(), p->items.size() * sizeof(WorkItem));
+            CUDA_TRY(p, cudaMemcpy(base, stage.data(), o_c2, cudaMemcpyHostToDevice));
+            CUDA_TRY(p, cudaMemset(p->d_range, 0, sizeof(u64)));
+        }
         p->dc.pconf = p->d_pconf;
         p->dc.n_pconf = np;
         CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
@@ -736,7 +788,6 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             CUDA_TRY(p, cudaEventCreateWithFlags(&cl.done, cudaEventDisableTiming));
         }
         if (tab_bytes) {
-            CUDA_TRY(p, cudaMalloc(&p->d_maptab, tab_bytes));
             for (const auto &cl : p->classes) {
                 if (!cl.has_tab) continue;
                 const WorkItem &rep = p->items[cl.item_lo];
@@ -747,6 +798,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             CUDA_TRY(p, cudaDeviceSynchronize());
             // which type masks occur in a class: the DP kernel builds stage rows for those only
             std::vector<uint8_t> tab(tab_bytes);
+            std::vector<std::pair<hap_problem::PpClass *, TrieClassHost>> built;
             CUDA_TRY(p, cudaMemcpy(tab.data(), p->d_maptab, tab_bytes, cudaMemcpyDeviceToHost));
             for (auto &cl : p->classes) {
                 if (!cl.has_tab) continue;
@@ -762,12 +814,11 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 if (!(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear && rows_exact) {
                     std::vector<u32> plist;
                     for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == cl.PP) plist.push_back((u32)pi);
-                    if (!build_trie(p, cl, tab.data() + cl.map_base, nmap, plist)) {
-                        cudaFree(cl.trie.d_blob); cudaFree(cl.trie.d_plist); cudaFree(cl.trie.d_metas);
-                        cl.trie = hap_problem::Trie{};
-                    }
+                    TrieClassHost th;
+                    if (build_trie(p, cl, tab.data() + cl.map_base, nmap, plist, th)) built.emplace_back(&cl, std::move(th));
                 }
             }
+            upload_tries(p, built);
         }
         p->enumerated = true;
     }
