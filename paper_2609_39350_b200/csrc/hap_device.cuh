@@ -321,41 +321,50 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
     const int l = threadIdx.x;
     i64 lmin = 0;                       // min over device types of this layer's forward+backward time
     if (l < N) {
-    const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
-    const bool dense = layer_kind(dc, l) == HAP_DENSE;
-    double a[HAP_MAX_TYPES], ab[HAP_MAX_TYPES], f[HAP_MAX_TYPES], fb[HAP_MAX_TYPES];
+        const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
+        const bool dense = layer_kind(dc, l) == HAP_DENSE;
+        const size_t i5 = (size_t)tcs[0].row * N + l;                       // the same table row for every type
+        const double *pa = dc.tdf + i5, *pab = dc.tdb + i5, *pf = dc.tff + i5, *pfb = dc.tfb + i5;
+        double a[HAP_MAX_TYPES], ab[HAP_MAX_TYPES], f[HAP_MAX_TYPES], fb[HAP_MAX_TYPES];
 #pragma unroll
-    for (int h = 0; h < HAP_MAX_TYPES; ++h) {
-        if (h < T) {
-            const size_t i5 = (size_t)h * stride_h + (size_t)tcs[h].row * N + l;
-            a[h] = __ldg(dc.tdf + i5); ab[h] = __ldg(dc.tdb + i5);
-            f[h] = dense ? 0.0 : __ldg(dc.tff + i5); fb[h] = dense ? 0.0 : __ldg(dc.tfb + i5);
-        }
-    }
-#pragma unroll
-    for (int h = 0; h < HAP_MAX_TYPES; ++h) {
-        if (h < T) {
-            const TypeConst &tc = tcs[h];
-            double cf, cb;
-            if (dense) {
-                cf = a[h] + tc.commF[HAP_DENSE];
-                cb = ab[h] + tc.commB[HAP_DENSE];
-            } else {
-                const double xf = div_by(dc.kappa * f[h], tc.den, tc.rden);
-                const double mf = (xf + tc.disp2) * tc.imb;
-                cf = (((a[h] - f[h]) + mf) + tc.tr) + tc.commF[HAP_MOE];
-                const double xb = div_by(dc.kappa * fb[h], tc.den, tc.rden);
-                const double mb = (xb + tc.disp2) * tc.imb;
-                cb = (((ab[h] - fb[h]) + mb) + tc.tr2) + tc.commB[HAP_MOE];
-            }
-            store_pair<QUANT>(c2, c2f, (((size_t)p * T + h) * N + l) * 2, cf, cb);
-            if (!(cf < 6.8719e10 && cb < 6.8719e10) && range_flag) atomicOr(range_flag, 1ull);   // 2^36 ns per layer
-            if (QUANT) {
-                const i64 q = __double2ll_rn(cf) + __double2ll_rn(cb);
-                lmin = (h == 0 || q < lmin) ? q : lmin;
+        for (int h = 0; h < HAP_MAX_TYPES; ++h) {
+            if (h < T) {
+                a[h] = __ldg(pa + h * stride_h); ab[h] = __ldg(pab + h * stride_h);
+                f[h] = dense ? 0.0 : __ldg(pf + h * stride_h); fb[h] = dense ? 0.0 : __ldg(pfb + h * stride_h);
             }
         }
-    }
+        const size_t out0 = ((size_t)p * T * N + l) * 2, out_h = (size_t)N * 2;
+        bool bad = false;                                                    // a value left the supported range
+        const double kappa = dc.kappa;
+#pragma unroll
+        for (int h = 0; h < HAP_MAX_TYPES; ++h) {
+            if (h < T) {
+                const TypeConst &tc = tcs[h];
+                double cf, cb;
+                if (dense) {
+                    cf = a[h] + tc.commF[HAP_DENSE];
+                    cb = ab[h] + tc.commB[HAP_DENSE];
+                } else {
+                    const double xf = div_by(kappa * f[h], tc.den, tc.rden);
+                    const double mf = (xf + tc.disp2) * tc.imb;
+                    cf = (((a[h] - f[h]) + mf) + tc.tr) + tc.commF[HAP_MOE];
+                    const double xb = div_by(kappa * fb[h], tc.den, tc.rden);
+                    const double mb = (xb + tc.disp2) * tc.imb;
+                    cb = (((ab[h] - fb[h]) + mb) + tc.tr2) + tc.commB[HAP_MOE];
+                }
+                bad |= !(cf < 6.8719e10) | !(cb < 6.8719e10);                 // 2^36 ns per layer
+                if (QUANT) {
+                    longlong2 v; v.x = __double2ll_rn(cf); v.y = __double2ll_rn(cb);
+                    *reinterpret_cast<longlong2 *>(c2 + out0 + h * out_h) = v;
+                    const i64 q = v.x + v.y;
+                    lmin = (h == 0 || q < lmin) ? q : lmin;
+                } else {
+                    double2 v; v.x = cf; v.y = cb;
+                    *reinterpret_cast<double2 *>(c2f + out0 + h * out_h) = v;
+                }
+            }
+        }
+        if (bad && range_flag) atomicOr(range_flag, 1ull);
     }
     // every layer runs on some device type, so the sum over layers of the cheapest type's time bounds the
     // summed stage time of every candidate of this configuration from below (used by the search's pruning)

@@ -127,3 +127,31 @@ def test_heterogeneous_communication_rule_in_the_tree_kernel(hap, name, eta_q):
     assert np.array_equal(tree["cost"], costs) and np.array_equal(tree["bottleneck"], bn)
     assert (costs >= INF).sum() > (bn >= INF).sum()          # the rule dropped some candidates with a feasible partition
     hap.hap_problem_destroy(hp)
+
+
+def test_large_multiset_class(hap):
+    """12 870 distinct stage-type sequences per configuration (PP = 16 on the two-type cluster with no cap on the
+    enumeration): the tree is cut into parts or, where it does not fit, the class runs one warp per candidate;
+    either way the values are those of the oracle."""
+    pb = problems.mixtral()
+    pb.map_cap = 1 << 40
+    pb.pp_list = np.ascontiguousarray(np.array([16], np.int32))
+    pb.tp_list = pb.tp_list[:2]; pb.cp_list = pb.cp_list[:1]; pb.ep_list = pb.ep_list[:2]; pb.tpe_list = pb.tpe_list[:1]
+    pb.mb_list = pb.mb_list[:2]
+    for f in ("tdf", "tdb", "tff", "tfb"):
+        setattr(pb, f, np.ascontiguousarray(getattr(pb, f)[:, :2, :1, :2]))
+    pb.tpre = np.ascontiguousarray(pb.tpre[:, :2, :1, :2]); pb.tpost = np.ascontiguousarray(pb.tpost[:, :2, :1, :2])
+    pb.rho = pb.rho[:2].copy()
+    o = Oracle(pb)
+    assert int(o.pconfs["nmap"][0]) == 12870
+    done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=NTHREADS, want_costs=True)
+    hp, tree = _pass(hap, pb, 0)
+    assert np.array_equal(tree["cost"], costs) and np.array_equal(tree["bottleneck"], bn)
+    rng = np.random.default_rng(2)
+    for idx in rng.integers(0, o.n_cand, 100).tolist():
+        plan, _, _ = o.eval_index(idx)
+        if plan["T_iter"] < INF:
+            assert tree["partition"][idx, :16].tolist() == plan["n"] and tree["recompute"][idx, :16].tolist() == plan["r"], idx
+    plan, stats = hap.hap_search_best(hp)
+    assert (plan["T_iter"], plan["index"]) == (bc, bi)
+    hap.hap_problem_destroy(hp)
