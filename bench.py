@@ -31,8 +31,8 @@ UNIT = "candidates/s"
 SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of the DP launches of one pass, from the ncu capture summarised
-# in profiles/pipeline_dp_kernel_stress.md
-NCU_DP_TRAFFIC_BYTES = {"stress": 64.0e6}
+# in profiles/trie_dp_kernel_stress.md
+NCU_DP_TRAFFIC_BYTES = {"stress": 69.4e6}
 
 
 def read_peaks():
@@ -341,8 +341,8 @@ def main():
             clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"]),
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                      ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
-            # per step: type_const, layer_cost, per PP class (decode, tree gather, tree DP), argmin partial + final
-            gpu_launches=(4 + 3 * len(set(int(x) for x in pconfs["PP"]))) * args.steps,
+            # per step: type_const, layer_cost, per PP class (decode, tree gather per part, tree DP), argmin partial + final
+            gpu_launches=hap.hap_launches_per_pass(hp) * args.steps,
             **extra_modes,
             joint_recurrence_ms=joint_ms,
             full_search_ms=statistics.median(search_ms),

@@ -300,6 +300,11 @@ hap_status hap_count_cells(hap_problem *, uint64_t first, uint64_t count, uint64
  * call's kernels.  Any output may be NULL. */
 hap_status hap_get_timings(hap_problem *, float *ms_layer_cost, float *ms_dp, uint64_t *cells);
 
+/* Measurement aid: the number of kernels one hap_pipeline_dp call over the whole candidate space followed by
+ * one hap_argmin call launches (layer costs, per PP class the candidate decode and the dynamic program, the
+ * reduction).  Host value, no device work. */
+hap_status hap_launches_per_pass(hap_problem *, uint32_t *host_count);
+
 const char *hap_status_str(hap_status);
 const char *hap_last_error(const hap_problem *);
 

@@ -1243,6 +1243,21 @@ extern "C" hap_status hap_debug_counters(hap_problem *p, uint64_t *host8)
 }
 #endif
 
+extern "C" hap_status hap_launches_per_pass(hap_problem *p, uint32_t *host_count)
+{
+    if (!p || !host_count) return HAP_E_INVALID;
+    if (!p->enumerated) return fail(p, HAP_E_STATE, "hap_enumerate has not run");
+    const bool lin = p->dc.tau_linear != 0;
+    const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0;
+    uint32_t n = 2 + 2;                                     // type constants, layer costs; argmin partial and final
+    for (const auto &cl : p->classes) {
+        if (cl.trie.ok && lin && !refine) n += 1 + (uint32_t)cl.trie.parts.size() + 1;   // decode, tree gather per part, tree DP
+        else n += (cl.has_tab ? 1 : 0) + 1;                                            // decode table, one-warp-per-candidate DP
+    }
+    *host_count = n;
+    return HAP_OK;
+}
+
 static hap_status argmin_launch(hap_problem *p, const i64 *dev_cost, uint64_t count, i64 *dev_out, cudaStream_t st, i64 init)
 {
     const unsigned blocks = (unsigned)std::min<uint64_t>((count + 255) / 256, 1024);
