@@ -282,6 +282,15 @@ def main():
             extra_modes[mode_name]["latency_ratio_vs_non_uniform"] = ref_best[0] / best[0]
         hap.hap_problem_destroy(hp_ref)
 
+    # Appendix B's latency expression for the winning plan, beside the closed form the search minimises (context)
+    appb = None
+    if world == 1:
+        one = hap.hap_pipeline_dp(hp, best[1], 1, partition=True)
+        ab = hap.hap_eval_appendix_b(hp, best[1], 1, one["partition"], one["recompute"], detail=True)
+        torch.cuda.synchronize()
+        edge, middle, smax = (int(x) for x in ab["detail"][0].tolist())
+        appb = dict(T_iter_closed_form=best[0], T_iter_appendix_b=int(ab["t_iter"][0]), T_edge=edge, T_middle=middle, s_max=smax)
+
     # full search through the search entry point (pruning allowed), wall clock call to return
     search_ms, pruned_ms = [], []
     hp_pr = hap.hap_problem_create(pb, prune=1)
@@ -345,6 +354,7 @@ def main():
             gpu_launches=hap.hap_launches_per_pass(hp) * args.steps,
             **extra_modes,
             joint_recurrence_ms=joint_ms,
+            appendix_b_best_plan=appb,
             full_search_ms=statistics.median(search_ms),
             full_search_pruned=dict(ms=statistics.median(pruned_ms), n_pruned=stats_pr["n_pruned"],
                                     n_evaluated=stats_pr["n_evaluated"]),

@@ -300,6 +300,19 @@ hap_status hap_count_cells(hap_problem *, uint64_t first, uint64_t count, uint64
  * call's kernels.  Any output may be NULL. */
 hap_status hap_get_timings(hap_problem *, float *ms_layer_cost, float *ms_dp, uint64_t *cells);
 
+/* Appendix B: the iteration latency of GIVEN plans with the steady-state term written through the index s_max of
+ * the (first) bottleneck stage, T_iter = T_edge + T_middle + T_dp-sync + T_opt with T_edge = sum_i (t_f,i + t_b,i)
+ * (Eq. 4) and T_middle = sum_{i <= s_max} t_f,i + (M - s_max - 1) max_i (t_f,i + t_b,i), stages 1-based, the
+ * multiplier taken as 0 when negative.  t_f,i: forward time of the stage's layers (slowest member type per layer);
+ * t_b,i: the rest of the stage cost (backward time, recomputation at the stage's level, stage constant), so that
+ * t_f,i + t_b,i is the stage cost of the recurrence.  A post-hoc evaluator: it does not choose partitions.
+ * Candidates [first, first+count); dev_partition / dev_recompute: [count][HAP_MAX_PP] layers and levels per stage
+ * as hap_pipeline_dp wrote them for the same range; dev_t_iter: [count] out, HAP_INF where the layer counts do
+ * not partition the N layers (an infeasible candidate); dev_detail: [count][3] out, T_edge, T_middle, s_max
+ * (nullable).  Recomputes the layer costs into library-owned memory first.  Asynchronous on `stream`. */
+hap_status hap_eval_appendix_b(hap_problem *, uint64_t first, uint64_t count, const uint8_t *dev_partition,
+                               const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream);
+
 /* Measurement aid: the number of kernels one hap_pipeline_dp call over the whole candidate space followed by
  * one hap_argmin call launches (layer costs, per PP class the candidate decode and the dynamic program, the
  * reduction).  Host value, no device work. */

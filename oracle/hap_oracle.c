@@ -1323,3 +1323,65 @@ int64_t orc_joint_bottleneck(const orc_problem *pr, const orc_pconf *pc, uint32_
     free(D);
     return ans;
 }
+
+/* ------------------------------------------------------------------------------------ *
+ * Appendix B: the steady-state term written with the bottleneck stage's index s_max, evaluated for a
+ * given plan (layers and recomputation level per stage).  Plain loops over stages and layers.
+ * ------------------------------------------------------------------------------------ */
+int orc_appendix_b(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                   const int64_t *c2, const int64_t *coef, const uint8_t *n, const uint8_t *r, orc_appb_result *res)
+{
+    const int N = pr->N, PP = pc->PP;
+    memset(res, 0, sizeof(*res));
+    int total = 0;
+    for (int s = 0; s < PP; ++s) { if (n[s] == 0) total = -100000; total += n[s]; }
+    if (total != N) { res->T_iter = ORC_INF; return 1; }
+    int64_t edge = 0, cmax = -1, fsum = 0, f_upto_max = 0, tsync = 0, topt = 0;
+    int smax = 0, a = 0;
+    for (int s = 0; s < PP; ++s) {
+        const unsigned mask = mp->mask[s];
+        const int i = s + 1, b = a + n[s];
+        int64_t tf = 0, tb = 0;
+        for (int l = a; l < b; ++l) {
+            int64_t F = 0, Bk = 0;
+            int seen = 0;
+            for (int h = 0; h < pr->T; ++h)
+                if (mask & (1u << h)) {
+                    const int64_t qf = c2[((int64_t)h * N + l) * 2], qb = c2[((int64_t)h * N + l) * 2 + 1];
+                    if (!seen || qf > F) F = qf;
+                    if (!seen || qb > Bk) Bk = qb;
+                    seen = 1;
+                }
+            tf += F; tb += Bk;
+        }
+        tb += ((int64_t)pr->tau_q[r[s]] * tf) / 1024;                 /* forward work repeated in the backward pass */
+        if (i == 1) tb += mask_max(pr, mask, coef, ORC_KPRE);
+        if (i == PP) tb += mask_max(pr, mask, coef, ORC_KPOST);
+        if (i > 1) {
+            const int hb = mp->hb[s], ha = mp->ha[s];
+            if (mp->cls[s] == ORC_INTRA) tb += coef[hb * ORC_NCOEF + ORC_KP2P_INTRA];
+            else if (mp->cls[s] == ORC_INTER) tb += coef[hb * ORC_NCOEF + ORC_KP2P_INTER];
+            else tb += coef[hb * ORC_NCOEF + ORC_KP2P_CROSS + ha];
+        }
+        const int64_t c = tf + tb;
+        edge += c;
+        fsum += tf;
+        if (c > cmax) { cmax = c; smax = i; f_upto_max = fsum; }       /* strict: the first bottleneck stage */
+        int64_t sy = mask_max(pr, mask, coef, ORC_SLAT), op = 0;
+        for (int l = a; l < b; ++l) {
+            sy += mask_max(pr, mask, coef, ORC_SBW + pr->kind[l]);
+            op += mask_max(pr, mask, coef, ORC_OPT + pr->kind[l]);
+        }
+        if (sy > tsync) tsync = sy;
+        if (op > topt) topt = op;
+        a = b;
+    }
+    int64_t steady = (int64_t)pc->M - smax - 1;
+    if (steady < 0) steady = 0;
+    res->T_edge = edge;
+    res->T_middle = f_upto_max + steady * cmax;
+    res->T_sync = tsync; res->T_opt = topt;
+    res->s_max = smax;
+    res->T_iter = res->T_edge + res->T_middle + tsync + topt;
+    return 0;
+}

@@ -4,8 +4,8 @@
  * A plain, slow, single-threaded restatement of what the planner computes: the 6-D
  * enumeration, the MoE-aware layer cost (Eq. 2, Eq. 3, load-imbalance scaling), the stage
  * memory model with minimal feasible recomputation, the per-candidate min-max pipeline
- * partitioning recurrence, the 1F1B closed-form iteration latency (Eq. 4) and the global
- * argmin (Eq. 1).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+ * partitioning recurrence, the 1F1B closed-form iteration latency (Eq. 4), the appendix's
+ * steady-state expression for given plans and the global argmin (Eq. 1).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
  * call it.  It shares no code with the CUDA library.
  *
  * Parity status: every function below is pinned by tests that do not go through this file's
@@ -153,4 +153,20 @@ int orc_candidate_f64(const orc_problem *pr, const orc_pconf *pc, const orc_mapp
                       const double *c2f, const int64_t *coef, const double *coeff, orc_result_f *res);
 int orc_search_pconfs_f64(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
                           uint64_t p_stride, uint64_t *n_done, double *costs, double *bottlenecks, uint8_t *parts);
+/* Iteration latency of a GIVEN plan by the appendix's steady-state expression (Appendix B, with Eq. 4):
+ *   T_iter = T_edge + T_middle + T_dp-sync + T_opt,  T_edge = sum_i (t_f,i + t_b,i),
+ *   s_max = the (first) stage with the largest t_f,i + t_b,i,
+ *   T_middle = sum_{i <= s_max} t_f,i + (M - s_max - 1) * max_i (t_f,i + t_b,i),
+ * stages 1-based.  t_f,i is the forward time of the stage's layers (slowest member type per layer); t_b,i is
+ * everything else of the stage cost (backward time, recomputation at the stage's level r_i, the stage constant),
+ * so t_f,i + t_b,i is the stage cost of the min-max recurrence.  The multiplier of the steady-state term is taken
+ * as max(0, M - s_max - 1).  n: layers per stage (sum N), r: recomputation level per stage.  Returns 0, or 1 and
+ * T_iter = ORC_INF when n does not partition the N layers. */
+typedef struct {
+    int64_t T_iter, T_edge, T_middle, T_sync, T_opt;
+    int32_t s_max, pad;
+} orc_appb_result;
+int orc_appendix_b(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                   const int64_t *c2, const int64_t *coef, const uint8_t *n, const uint8_t *r, orc_appb_result *res);
+
 #endif

@@ -77,6 +77,11 @@ class ResultF(C.Structure):
                 ("r", C.c_uint8 * MAX_PP), ("c", C.c_double * MAX_PP)]
 
 
+class AppBResult(C.Structure):
+    _fields_ = [("T_iter", C.c_int64), ("T_edge", C.c_int64), ("T_middle", C.c_int64), ("T_sync", C.c_int64),
+                ("T_opt", C.c_int64), ("s_max", C.c_int32), ("pad", C.c_int32)]
+
+
 class Plan(C.Structure):
     _fields_ = [("index", C.c_uint64), ("pc", PConf), ("map", Mapping), ("rc_mask", C.c_uint32), ("res", Result)]
 
@@ -210,6 +215,14 @@ class Oracle:
         self.L.orc_candidate(C.byref(self.s), self._pc(p), C.byref(mp), C.c_uint32(rc_mask), _ptr(c2), _ptr(coef),
                              C.byref(res), _ptr(dp) if tables else None, _ptr(ch) if tables else None)
         return res, dp, ch
+
+    def appendix_b(self, p, mp, c2, coef, n, r) -> AppBResult:
+        """Appendix B's iteration latency of a given plan (layers n and recomputation levels r per stage)."""
+        res = AppBResult()
+        na = np.zeros(MAX_PP, np.uint8); ra = np.zeros(MAX_PP, np.uint8)
+        na[:len(n)] = n; ra[:len(r)] = r
+        self.L.orc_appendix_b(C.byref(self.s), self._pc(p), C.byref(mp), _ptr(c2), _ptr(coef), _ptr(na), _ptr(ra), C.byref(res))
+        return res
 
     def bruteforce(self, p, mp, rc_mask, c2, coef, i, j):
         cnt = C.c_uint64()

@@ -16,6 +16,7 @@
 //                       Instantiated on int64 (exact) and double (fp64 mode).
 //   joint_dp_kernel     recurrence over the device-group state: minimum bottleneck over all
 //                       stage-type sequences of a configuration.
+//   appendix_b_kernel   iteration latency of given plans by the appendix's steady-state expression.
 //   argmin kernels      lexicographic (cost, index) minimum, block partials then one block.
 #pragma once
 #include <cuda_runtime.h>
@@ -516,6 +517,97 @@ __global__ void decode_kernel(const DevConst dc, u64 first, u64 count, hap_candi
     }
     o->mask[lane] = lane < pc.PP ? (uint8_t)sm.mask : 0;
     o->link[lane] = (lane < pc.PP && lane > 0) ? (uint8_t)(sm.cls | (sm.ha << 2) | (sm.hb << 4)) : 0;
+}
+
+// ------------------------------------------------------------------------------------------
+// Appendix B: iteration latency of GIVEN plans with the steady-state term written through the bottleneck
+// stage's index, T_middle = sum_{i <= s_max} t_f,i + max(0, M - s_max - 1) max_i (t_f,i + t_b,i), T_edge = the
+// summed stage cost (Eq. 4).  t_f,i is the forward time of the stage's layers (slowest member type per layer);
+// recomputation, backward time and the stage constant make up t_b,i.  One warp per candidate, lane s = stage s+1;
+// partition / recompute: [count][HAP_MAX_PP] layers and levels per stage as written by the DP kernels.
+// t_iter: [count]; detail: [count][3] T_edge, T_middle, s_max (nullable).
+// ------------------------------------------------------------------------------------------
+__global__ void appendix_b_kernel(const DevConst dc, u64 first, u64 count, const i64 *__restrict__ c2,
+                                  const i64 *__restrict__ coef, const uint8_t *__restrict__ partition,
+                                  const uint8_t *__restrict__ recompute, i64 *t_iter, i64 *detail)
+{
+    const u64 w = ((u64)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= count) return;
+    const u64 c = first + w;
+    const u64 p = find_pconf(dc, c);
+    const hap_pconf pc = dc.pconf[p];
+    const int PP = pc.PP, N = dc.N, T = dc.T;
+    const u64 map_idx = (c - pc.offset) / (u64)dc.n_rc;
+    const StageMap sm = decode_stage(dc, pc, map_idx, lane);
+    const bool on = lane < PP;
+    const int n_me = on ? partition[w * HAP_MAX_PP + lane] : 0;
+    const int r_me = on ? recompute[w * HAP_MAX_PP + lane] : 0;
+    int b_me = n_me;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, b_me, o); if (lane >= o) b_me += t; }
+    const int total = __shfl_sync(0xffffffffu, b_me, PP - 1);
+    const bool ok = total == N && !__any_sync(0xffffffffu, on && n_me == 0) && !__any_sync(0xffffffffu, on && r_me >= dc.R);
+    if (!ok) {
+        if (lane == 0) {
+            t_iter[w] = kInf;
+            if (detail) { detail[w * 3] = kInf; detail[w * 3 + 1] = kInf; detail[w * 3 + 2] = 0; }
+        }
+        return;
+    }
+    i64 tf = 0, cst = 0, sy = 0, op = 0;
+    if (on) {
+        const int a_me = b_me - n_me;
+        const i64 *c2p = c2 + (size_t)p * T * N * 2;
+        const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
+        i64 tb = 0;
+        for (int l = a_me; l < b_me; ++l) {
+            i64 F = 0, B = 0;
+            for (int h = 0; h < T; ++h)
+                if (sm.mask >> h & 1) {
+                    const i64 qx = c2p[((size_t)h * N + l) * 2], qy = c2p[((size_t)h * N + l) * 2 + 1];
+                    F = qx > F ? qx : F;
+                    B = qy > B ? qy : B;
+                }
+            tf += F; tb += B;
+        }
+        // coefficients of a stage of several types: the slowest member's
+        i64 kpre = 0, kpost = 0, slat = 0, sbw[2] = {0, 0}, opt[2] = {0, 0};
+        for (int h = 0; h < T; ++h)
+            if (sm.mask >> h & 1) {
+                const i64 *row = cfp + h * HAP_NCOEF;
+                kpre = row[HAP_KPRE] > kpre ? row[HAP_KPRE] : kpre;
+                kpost = row[HAP_KPOST] > kpost ? row[HAP_KPOST] : kpost;
+                slat = row[HAP_SLAT] > slat ? row[HAP_SLAT] : slat;
+                for (int kd = 0; kd < 2; ++kd) {
+                    sbw[kd] = row[HAP_SBW + kd] > sbw[kd] ? row[HAP_SBW + kd] : sbw[kd];
+                    opt[kd] = row[HAP_OPT + kd] > opt[kd] ? row[HAP_OPT + kd] : opt[kd];
+                }
+            }
+        tb += ((i64)dc.tau_q[r_me] * tf) >> 10;              // forward work repeated in the backward pass
+        if (lane == 0) tb += kpre;
+        if (lane == PP - 1) tb += kpost;
+        if (lane > 0) tb += cfp[sm.hb * HAP_NCOEF + (sm.cls == HAP_CROSS ? HAP_KP2P_CROSS + sm.ha : HAP_KP2P_INTRA + sm.cls)];
+        cst = tf + tb;
+        const i64 n_moe = (i64)(moe_before(dc, b_me) - moe_before(dc, a_me)), n_dense = (i64)n_me - n_moe;
+        sy = slat + n_dense * sbw[0] + n_moe * sbw[1];
+        op = n_dense * opt[0] + n_moe * opt[1];
+    }
+    const i64 edge = warp_sum_i64(cst), cmax = warp_max_i64(cst);
+    const i64 t_sync = warp_max_i64(sy), t_opt = warp_max_i64(op);
+    const unsigned at_max = __ballot_sync(0xffffffffu, on && cst == cmax);
+    const int s_lane = __ffs(at_max) - 1;                      // the first bottleneck stage
+    i64 fpre = tf;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const i64 t = __shfl_up_sync(0xffffffffu, fpre, o); if (lane >= o) fpre += t; }
+    const i64 f_upto = shfl_i64(fpre, s_lane);
+    i64 steady = (i64)pc.M - (s_lane + 1) - 1;
+    if (steady < 0) steady = 0;
+    if (lane == 0) {
+        const i64 middle = f_upto + steady * cmax;
+        t_iter[w] = edge + middle + t_sync + t_opt;
+        if (detail) { detail[w * 3] = edge; detail[w * 3 + 1] = middle; detail[w * 3 + 2] = s_lane + 1; }
+    }
 }
 
 // ------------------------------------------------------------------------------------------

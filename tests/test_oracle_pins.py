@@ -739,3 +739,71 @@ def test_limit_sweep_reaches_the_exhaustive_optimum_of_the_pipeline_term(make, s
         swept += ex["passes"] > 2
     if pb.name == "tiny":
         assert improved > 0 and swept > 0
+
+
+# --------------------------------------------------------------------------------------
+# Appendix B: steady-state term with the bottleneck stage's index
+# --------------------------------------------------------------------------------------
+def test_appendix_b_hand_values_on_the_two_device_example():
+    g = gold("e5_appendix_b.json")["expect"]
+    o = Oracle(e1_problem())
+    c2, _, coef, _ = o.layer_costs(0)
+    for idx, key in ((0, "map_AB"), (1, "map_BA")):
+        plan, _, _ = o.eval_index(idx)
+        assert plan["n"] == g[key]["n"]
+        r = o.appendix_b(0, o.decode(0, idx), c2, coef, plan["n"], plan["r"])
+        assert (r.s_max, r.T_edge, r.T_middle, r.T_iter) == (g[key]["s_max"], g[key]["T_edge"], g[key]["T_middle"], g[key]["T_iter"])
+        assert r.T_edge == sum(plan["c"])                  # T_edge is the summed stage cost of the recurrence
+    # fewer micro-batches than the bottleneck's index + 1: no steady-state repetitions are left
+    pb = e1_problem()
+    pb.GB = 2
+    o2 = Oracle(pb)
+    assert int(o2.pconfs["M"][0]) == 2
+    c2, _, coef, _ = o2.layer_costs(0)
+    r = o2.appendix_b(0, o2.decode(0, 1), c2, coef, [1, 3], [0, 0])
+    assert (r.T_middle, r.T_iter) == (g["map_BA_M2"]["T_middle"], g["map_BA_M2"]["T_iter"])
+    # a layer vector that does not cover the N layers is rejected
+    assert o.appendix_b(0, o.decode(0, 0), c2, coef, [2, 1], [0, 0]).T_iter == INF
+    assert o.appendix_b(0, o.decode(0, 0), c2, coef, [4, 0], [0, 0]).T_iter == INF
+
+
+def test_appendix_b_against_the_closed_form_and_the_schedule_simulation():
+    """Identities that hold for every plan: with s = s_max and M >= s + 1,
+    T_appB = closed form - s * max_i c_i + sum_{i <= s} t_f,i (so it never exceeds the closed form);
+    for uniform stages (f, b per micro-batch) it is (M + PP - 2)(f + b) + f, i.e. exactly b below the
+    simulated 1F1B makespan (M + PP - 1)(f + b): the appendix's expression and the schedule differ by one
+    backward pass of the bottleneck stage."""
+    pb = problems.tiny()
+    o = Oracle(pb)
+    rng = np.random.default_rng(4)
+    checked = 0
+    for idx in rng.integers(0, o.n_cand, 400).tolist():
+        plan, _, _ = o.eval_index(int(idx))
+        if plan["T_iter"] >= INF:
+            continue
+        p = o.find_pconf(int(idx))
+        c2, _, coef, _ = o.layer_costs(p)
+        mp = o.decode(p, (int(idx) - int(o.pconfs["offset"][p])) // len(pb.rc_masks))
+        r = o.appendix_b(p, mp, c2, coef, plan["n"], plan["r"])
+        c = plan["c"]
+        M, s = plan["M"], r.s_max
+        assert r.T_edge == sum(c) and c[s - 1] == max(c) and all(x < max(c) for x in c[:s - 1])
+        a = sum(plan["n"][:s])
+        # forward time of stages 1..s: slowest member type per layer
+        tf = 0
+        lo = 0
+        for st in range(s):
+            types = [h for h in range(pb.T) if plan["mask"][st] >> h & 1]
+            tf += sum(max(int(c2[h, l, 0]) for h in types) for l in range(lo, lo + plan["n"][st]))
+            lo += plan["n"][st]
+        assert lo == a
+        assert r.T_middle == tf + max(0, M - s - 1) * max(c)
+        assert (r.T_sync, r.T_opt) == (plan["T_sync"], plan["T_opt"])
+        if M >= s + 1:
+            assert r.T_iter == plan["T_iter"] - s * max(c) + tf and r.T_iter <= plan["T_iter"]
+        checked += 1
+    assert checked > 50
+    for PP, M, f, b in ((4, 8, 3.0, 6.0), (2, 5, 1.0, 1.0), (8, 12, 2.0, 5.0)):
+        appb = PP * (f + b) + f + (M - 1 - 1) * (f + b)           # s_max = 1 for identical stages
+        assert appb == (M + PP - 2) * (f + b) + f
+        assert _simulate_1f1b([f] * PP, [b] * PP, M) - appb == b
