@@ -1234,15 +1234,6 @@ extern "C" hap_status hap_get_timings(hap_problem *p, float *ms_layer_cost, floa
     return check_values(p);
 }
 
-#ifdef HAP_TRIE_TIMERS
-extern "C" hap_status hap_debug_counters(hap_problem *p, uint64_t *host8)
-{
-    CUDA_TRY(p, cudaDeviceSynchronize());
-    CUDA_TRY(p, cudaMemcpy(host8, p->d_counters, 8 * sizeof(u64), cudaMemcpyDeviceToHost));
-    return HAP_OK;
-}
-#endif
-
 extern "C" hap_status hap_eval_appendix_b(hap_problem *p, uint64_t first, uint64_t count, const uint8_t *dev_partition,
                                           const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream)
 {

@@ -7,7 +7,7 @@
 //   layer_cost_kernel   per (configuration, type, layer): Eq. 2 with imbalance scaling, rounding,
 //                       one block per configuration, one thread per layer.
 //   decode_kernel       candidate index -> stage type masks and boundary link classes;
-//   maptab_kernel       the same for every mapping of one PP class, once per problem.
+//   maptab_kernel       the same for every mapping of one PP class (every pass).
 //   pipeline_dp_kernel  one warp per candidate: stage rows and memory-threshold tables in shared
 //                       memory (built once per block for the block's configuration), min-max
 //                       recurrence with lanes over the end layer j, optional refinement pass,
@@ -612,7 +612,8 @@ __global__ void appendix_b_kernel(const DevConst dc, u64 first, u64 count, const
 
 // ------------------------------------------------------------------------------------------
 // mapping table: decoded (mask, link) byte pairs per stage for every mapping of one PP class,
-// built once per problem so that the DP kernel does not unrank per candidate
+// built in every pass (and once at enumeration, for the host-side tree) so that the DP kernels do not
+// unrank per candidate
 // ------------------------------------------------------------------------------------------
 __global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *tab)
 {

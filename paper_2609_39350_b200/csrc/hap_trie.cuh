@@ -112,12 +112,6 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
     }
 }
 
-#ifdef HAP_TRIE_TIMERS
-#define HAP_TQ(x) x
-#else
-#define HAP_TQ(x)
-#endif
-
 // shared-memory accesses by 32-bit address (the split loop walks two rows with plain address decrements)
 __device__ __forceinline__ u32 smem_u32(const void *p) { return (u32)__cvta_generic_to_shared(p); }
 template <int OFF> __device__ __forceinline__ i64 lds_i64(u32 a)
@@ -366,9 +360,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     TrieNode *sNodes = reinterpret_cast<TrieNode *>(ch + ((size_t)tm.cell_lo[PP] + 15) / 16 * 16);
     uint16_t *sParent = reinterpret_cast<uint16_t *>(sNodes + tm.node_lo[PP]);
 
-    HAP_TQ(long long tq0 = clock64(); long long tq_lv = 0; long long tq_leaf = 0;)
     trie_prologue_rows(dc, tm, p, c2, coef, sC, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
-    HAP_TQ(long long tq1 = clock64();)
     const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
 
     // writes "infeasible" for candidate c (non-search mode)
@@ -409,7 +401,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         trie_prologue_time_rows(dc, tm, sC, sR);
         trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
     }
-    HAP_TQ(long long tq2 = clock64();)
 
     const u32 a_thr = smem_u32(thr), a_sR = smem_u32(sR);
 
@@ -464,7 +455,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         const unsigned rc_mask = dc.rc_masks[rc_idx];
         bool dead = config_dead || (dc.rc_sup[rc_pos] & policies_without_plan) != 0;
 
-        HAP_TQ(long long tq3 = clock64();)
         // ---- rows of the tree, depth by depth ------------------------------------------------
         if (!dead) {
             // a thread's first cell record of a depth is requested before the barrier that ends the previous depth
@@ -492,7 +482,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 if (!__syncthreads_or(alive)) { dead = true; break; }   // no cell of this depth is finite: nothing below is
             }
         }
-        HAP_TQ(long long tq4 = clock64(); tq_lv += tq4 - tq3;)
         // ---- one thread per mapping: cell (PP, N), backtrace, Eq. 4 ---------------------------------
         auto stage_K = [&](int d, int mask, int link) -> i64 {
             i64 K = 0;
@@ -586,19 +575,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         }
         // the barrier also keeps the next policy from overwriting rows and choices that are still being read
         const int bott_any = __syncthreads_or(any_plan);
-        HAP_TQ(tq_leaf += clock64() - tq4;)
         // a policy under which none of the block's mappings has a feasible partition settles its subsets
         if (!bott_any && c_lo >= w_lo && c_hi <= w_hi && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
     }
 
-#ifdef HAP_TRIE_TIMERS
-    if (tid == 0 && out.counters && !SEARCH) {
-        // cycles per block: [5] rows prologue, [6] thresholds, [7] tree levels, [3] mappings, [2] whole block
-        atomicAdd(out.counters + 5, (u64)(tq1 - tq0)); atomicAdd(out.counters + 6, (u64)(tq2 - tq1));
-        atomicAdd(out.counters + 7, (u64)tq_lv); atomicAdd(out.counters + 3, (u64)tq_leaf);
-        atomicAdd(out.counters + 2, (u64)(clock64() - tq0));
-    }
-#endif
     if (out.counters) {
         const u64 n_cells = (u64)warp_sum_i64((i64)n_cells32);
         if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
