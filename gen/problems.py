@@ -104,6 +104,9 @@ class Problem:
     extra: Dict[str, np.ndarray] = field(default_factory=dict)
     uniform: int = 0     # ablation: 1 = uniform layer split only (non-uniform partitioning disabled)
     eta_q: int = 0       # Pruning 3 threshold eta in 1/1024 (2048 = the paper's default 2); <= 0 disables it
+    # communication-primitive table: link efficiency by message size (empty: efficiency 1 everywhere)
+    fsize: np.ndarray = field(default_factory=lambda: np.zeros(0, np.float64))     # [n] bytes, ascending
+    feff: np.ndarray = field(default_factory=lambda: np.zeros((3, 0), np.float64))  # [3][n] INTRA, INTER, CROSS
 
     @property
     def T(self) -> int:
@@ -352,3 +355,20 @@ def blank(*, N, S, H, E, k, GB, P_tf, C_gb, node_size, nodes_per_type, tp_list=(
         pp_list=_i32(pp_list), tpe_list=_i32(tpe_list), tp_max=max(list(tp_list) + list(tpe_list)),
         delta_q=-1, map_cap=1 << 40, rc_masks=np.ascontiguousarray(np.asarray([(1 << R) - 1], np.uint32)),
     )
+
+
+def with_link_efficiency_table(pb: Problem, seed: int = 7, n: int = 8) -> Problem:
+    """The same problem with a synthetic communication-primitive table: link efficiency rising with the
+    message size (64 KiB .. 8 GiB, factor 8 between sizes) towards 0.75-0.97, lower for slower link classes,
+    with a seeded wiggle so that the interpolation segments have different slopes."""
+    rng = SplitMix64(0xF00D ^ (seed * 104729))
+    out = pb.copy()
+    out.fsize = np.ascontiguousarray(np.array([65536.0 * 8.0 ** i for i in range(n)], np.float64))
+    top = [0.97, 0.9, 0.75]
+    eff = np.zeros((3, n), np.float64)
+    for c in range(3):
+        for i in range(n):
+            ramp = (i + 1.0) / (n + 1.0)
+            eff[c, i] = min(1.0, max(0.05, top[c] * (0.35 + 0.65 * ramp) + 0.03 * (rng.u() - 0.5)))
+    out.feff = np.ascontiguousarray(eff)
+    return out

@@ -126,6 +126,13 @@ typedef struct {
     int32_t R;                   /* recomputation levels, 1..HAP_MAX_RC; level 0 = none */
     const int32_t *xi_q;         /* [R] activation-memory factor xi(r) in 1/1024 */
     const int32_t *tau_q;        /* [R] fraction of the forward pass re-executed, in 1/1024 */
+    /* Communication-primitive table (Sec. 3.4, "f_prim across link types"): the profiled efficiency of a link by
+     * message size.  The volume term of every primitive (ring collectives, all-to-all / all-gather dispatch, p2p,
+     * gradient sync), volume / bandwidth, is divided by the efficiency of its link class at its volume, piecewise
+     * linear between the profiled sizes and constant outside them.  n_fsize = 0: no table, efficiency 1. */
+    int32_t n_fsize;             /* 0..HAP_MAX_LIST profiled message sizes */
+    const double *fsize;         /* [n_fsize] bytes, > 0, strictly ascending */
+    const double *feff;          /* [3][n_fsize] efficiency in (0, 1] for HAP_INTRA / HAP_INTER / HAP_CROSS links */
 } hap_profile;
 
 /* hap_search_opts.flags */

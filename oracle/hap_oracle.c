@@ -237,6 +237,28 @@ typedef struct { const orc_problem *pr; int h; double bw_inter; } linkctx;
 static int link_cls(const linkctx *lc, int64_t ext) { return ext <= lc->pr->node_size[lc->h] ? ORC_INTRA : ORC_INTER; }
 static double link_bw(const linkctx *lc, int cls) { return cls == ORC_INTRA ? lc->pr->bw_intra[lc->h] : lc->bw_inter; }
 
+/* Volume term of a communication primitive (the communication-primitive table of Sec. 3.4): the time to move
+ * `vol` bytes over a link of class c with nominal bandwidth bw is vol / bw divided by the link's profiled
+ * efficiency at that message size, piecewise linear between the profiled sizes and constant outside them.
+ * Without a table the efficiency is 1 and the term is vol / bw. */
+static double link_eff(const orc_problem *pr, int c, double vol)
+{
+    const int n = pr->n_fsize;
+    const double *sz = pr->fsize, *e = pr->feff + (size_t)c * n;
+    if (vol <= sz[0]) return e[0];
+    if (vol >= sz[n - 1]) return e[n - 1];
+    int i = 0;
+    while (vol >= sz[i + 1]) ++i;
+    return e[i] + (vol - sz[i]) * ((e[i + 1] - e[i]) / (sz[i + 1] - sz[i]));
+}
+
+static double xfer(const orc_problem *pr, int c, double vol, double bw)
+{
+    const double t = vol / bw;
+    if (pr->n_fsize <= 0) return t;
+    return t / link_eff(pr, c, vol);
+}
+
 /* ring-style collective over w ranks spanning `ext` devices moving D bytes */
 static double coll(const linkctx *lc, int64_t w, int64_t ext, double D)
 {
@@ -244,7 +266,7 @@ static double coll(const linkctx *lc, int64_t w, int64_t ext, double D)
     int c = link_cls(lc, ext);
     double lat = lc->pr->alpha[c] * (double)(w - 1);
     double vol = (D * (double)(w - 1)) / (double)w;
-    return lat + vol / link_bw(lc, c);
+    return lat + xfer(lc->pr, c, vol, link_bw(lc, c));
 }
 
 int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, double *c2f,
@@ -271,8 +293,8 @@ int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, dou
             double Dmoe = ((thb * pr->beta) * (double)pr->k) * (1.0 - 1.0 / (double)EP);
             double Dag = (thb * pr->beta) * (double)(EP - 1);
             int c = link_cls(&lc, (int64_t)EP * TPE);
-            double fa = pr->alpha[c] * (double)(EP - 1) + Dmoe / link_bw(&lc, c);
-            double fg = pr->alpha[c] * (double)(EP - 1) + Dag / link_bw(&lc, c);
+            double fa = pr->alpha[c] * (double)(EP - 1) + xfer(pr, c, Dmoe, link_bw(&lc, c));
+            double fg = pr->alpha[c] * (double)(EP - 1) + xfer(pr, c, Dag, link_bw(&lc, c));
             tdisp = (fa <= fg) ? fa : fg;
         }
         const double ttpA = 2.0 * coll(&lc, TP, TP, Dtp);
@@ -312,12 +334,12 @@ int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, dou
         double v[ORC_NCOEF];
         v[ORC_KPRE] = pr->tpre[i4];
         v[ORC_KPOST] = pr->tpost[i4];
-        v[ORC_KP2P_INTRA] = 2.0 * (pr->alpha[ORC_INTRA] + (Dtp / (double)TP) / pr->bw_intra[h]);
-        v[ORC_KP2P_INTER] = 2.0 * (pr->alpha[ORC_INTER] + (Dtp / (double)TP) / bwi[h]);
+        v[ORC_KP2P_INTRA] = 2.0 * (pr->alpha[ORC_INTRA] + xfer(pr, ORC_INTRA, Dtp / (double)TP, pr->bw_intra[h]));
+        v[ORC_KP2P_INTER] = 2.0 * (pr->alpha[ORC_INTER] + xfer(pr, ORC_INTER, Dtp / (double)TP, bwi[h]));
         for (int h2 = 0; h2 < ORC_MAX_TYPES; ++h2) {
             double bo = h2 < T ? bwi[h2] : bwi[h];
             double bmin = bwi[h] < bo ? bwi[h] : bo;
-            v[ORC_KP2P_CROSS + h2] = 2.0 * (pr->alpha[ORC_CROSS] + (Dtp / (double)TP) / (bmin * pr->chi));
+            v[ORC_KP2P_CROSS + h2] = 2.0 * (pr->alpha[ORC_CROSS] + xfer(pr, ORC_CROSS, Dtp / (double)TP, bmin * pr->chi));
         }
         const double shd = 6.0 + 12.0 / (double)((int64_t)DP * CP);
         const double she = 6.0 + 12.0 / (double)EDP;
@@ -342,8 +364,8 @@ int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, dou
         for (int kd = 0; kd < 2; ++kd) {
             const int64_t Pdd = Pd[kd] + (kd == ORC_MOE ? Prt : 0);
             const double Pel = kd == ORC_MOE ? (double)Pe / (double)TPE : 0.0;
-            v[ORC_SBW + kd] = pr->ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG)
-                                            + (((6.0 * Pel) * vfe) / bwG));
+            v[ORC_SBW + kd] = pr->ovl_dp * (xfer(pr, cG, (6.0 * ((double)Pdd / (double)TP)) * vfd, bwG)
+                                            + xfer(pr, cG, (6.0 * Pel) * vfe, bwG));
             v[ORC_OPT + kd] = pr->copt[h] * ((double)Pdd / (double)((int64_t)TP * DP * CP) + Pel / (double)EDP);
         }
         v[ORC_SLAT] = pr->ovl_dp * (pr->alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));

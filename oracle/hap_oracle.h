@@ -72,6 +72,10 @@ typedef struct {
     const uint32_t *rc_masks;
     int32_t eta_q;      /* Pruning 3 threshold eta in 1/1024; <= 0: off */
     int32_t uniform;    /* ablation: uniform layer split only (floor/ceil of N/PP layers per stage) */
+    /* communication-primitive table: link efficiency by message size (0 sizes: efficiency 1 everywhere) */
+    int32_t n_fsize, pad_f;
+    const double *fsize;    /* [n_fsize] bytes, ascending */
+    const double *feff;     /* [3][n_fsize] efficiency in (0, 1] of an intra-node / inter-node / cross-type link */
 } orc_problem;
 
 typedef struct {

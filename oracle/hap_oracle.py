@@ -51,6 +51,7 @@ class _Problem(C.Structure):
         ("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
         ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64),
         ("n_rc", C.c_int32), ("rc_masks", C.c_void_p), ("eta_q", C.c_int32), ("uniform", C.c_int32),
+        ("n_fsize", C.c_int32), ("pad_f", C.c_int32), ("fsize", C.c_void_p), ("feff", C.c_void_p),
     ]
 
 
@@ -159,6 +160,11 @@ class Oracle:
         s.rc_masks = arr("rc_masks", np.uint32)
         s.eta_q = int(getattr(pb, "eta_q", 0))
         s.uniform = int(getattr(pb, "uniform", 0))
+        fsize = np.ascontiguousarray(np.asarray(getattr(pb, "fsize", []), dtype=np.float64))
+        feff = np.ascontiguousarray(np.asarray(getattr(pb, "feff", []), dtype=np.float64))
+        keep["fsize"], keep["feff"] = fsize, feff
+        s.n_fsize = int(fsize.shape[0])
+        s.fsize, s.feff = (_ptr(fsize), _ptr(feff)) if s.n_fsize else (None, None)
         self._keep = keep
         self.s = s
         self.N, self.T = int(pb.N), s.T

@@ -45,7 +45,8 @@ class _Profile(C.Structure):
                 ("kappa", C.c_double), ("alpha", C.c_void_p), ("chi", C.c_double), ("rho", C.c_void_p),
                 ("gamma", C.c_double), ("ovl_tp", C.c_double), ("ovl_cp", C.c_double), ("ovl_dp", C.c_double),
                 ("act_coef", C.c_void_p), ("capf", C.c_double), ("copt", C.c_void_p), ("cap_eff", C.c_void_p),
-                ("R", C.c_int32), ("xi_q", C.c_void_p), ("tau_q", C.c_void_p)]
+                ("R", C.c_int32), ("xi_q", C.c_void_p), ("tau_q", C.c_void_p),
+                ("n_fsize", C.c_int32), ("fsize", C.c_void_p), ("feff", C.c_void_p)]
 
 
 class _Opts(C.Structure):
@@ -175,6 +176,11 @@ def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
         setattr(pf, n, float(getattr(pb, n)))
     pf.cap_eff = arr("cap_eff", np.int64)
     pf.R = len(pb.xi_q)
+    fsize = np.ascontiguousarray(np.asarray(getattr(pb, "fsize", []), dtype=np.float64))
+    feff = np.ascontiguousarray(np.asarray(getattr(pb, "feff", []), dtype=np.float64))
+    keep += [fsize, feff]
+    pf.n_fsize = int(fsize.shape[0])
+    pf.fsize, pf.feff = (_ptr(fsize), _ptr(feff)) if pf.n_fsize else (None, None)
     so = _Opts()
     so.npp, so.ntpe = len(pb.pp_list), len(pb.tpe_list)
     so.pp_list, so.tpe_list = arr("pp_list", np.int32), arr("tpe_list", np.int32)

@@ -222,6 +222,11 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
         !(pf->ovl_dp >= 0.0) || !(pf->capf >= 0.0))
         return HAP_E_INVALID;
     for (double r : p->rho) if (!(r >= 1.0)) return HAP_E_INVALID;
+    if (pf->n_fsize < 0 || pf->n_fsize > HAP_MAX_LIST || (pf->n_fsize > 0 && (!pf->fsize || !pf->feff))) return HAP_E_INVALID;
+    for (int i = 0; i < pf->n_fsize; ++i) {
+        if (!(pf->fsize[i] > 0.0) || !std::isfinite(pf->fsize[i]) || (i > 0 && !(pf->fsize[i] > pf->fsize[i - 1]))) return HAP_E_INVALID;
+        for (int c = 0; c < 3; ++c) { const double e = pf->feff[c * pf->n_fsize + i]; if (!(e > 0.0 && e <= 1.0)) return HAP_E_INVALID; }
+    }
 
     const size_t n4 = (size_t)T * pf->ntp * pf->ncp * pf->nmb, n5 = n4 * N;
     std::vector<double> tables(4 * n5 + 2 * n4);
@@ -271,6 +276,11 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
             for (int q = 0; q < j; ++q)
                 if ((p->rc_masks[order[q]] & p->rc_masks[order[j]]) == p->rc_masks[order[j]]) dc.rc_sup[j] |= 1u << q;
         }
+    }
+    dc.n_fsize = pf->n_fsize;
+    for (int i = 0; i < pf->n_fsize; ++i) {
+        dc.fsize[i] = pf->fsize[i];
+        for (int c = 0; c < 3; ++c) dc.feff[c][i] = pf->feff[c * pf->n_fsize + i];
     }
     dc.tau_linear = 1;
     for (int r = 0; r < pf->R; ++r) { dc.xi_q[r] = p->xi_q[r]; dc.tau_q[r] = p->tau_q[r]; if (p->tau_q[r] % 1024) dc.tau_linear = 0; }

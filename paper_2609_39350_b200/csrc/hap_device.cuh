@@ -46,6 +46,8 @@ struct DevConst {
     double rho[HAP_MAX_LIST];
     i64 P[HAP_MAX_TYPES], cap_eff[HAP_MAX_TYPES], m[HAP_MAX_TYPES];
     int node_size[HAP_MAX_TYPES];
+    int n_fsize;                      // communication-primitive table: link efficiency by message size (0: none)
+    double fsize[HAP_MAX_LIST], feff[3][HAP_MAX_LIST];
     unsigned rc_masks[HAP_MAX_RC_MASKS];
     int rc_order[HAP_MAX_RC_MASKS];   // policies from the most permissive to the most restrictive
     unsigned rc_sup[HAP_MAX_RC_MASKS]; // per position in rc_order: earlier positions whose allowed levels are a superset
@@ -139,6 +141,26 @@ struct LinkCtx { double bw_intra, bw_inter; int node_size; };
 __device__ __forceinline__ int link_class(const LinkCtx &lc, i64 ext) { return ext <= lc.node_size ? HAP_INTRA : HAP_INTER; }
 __device__ __forceinline__ double link_bw(const LinkCtx &lc, int cls) { return cls == HAP_INTRA ? lc.bw_intra : lc.bw_inter; }
 
+// Volume term of a communication primitive (the communication-primitive table of Sec. 3.4): vol bytes over a link
+// of class cls with nominal bandwidth bw take vol / bw divided by the link's profiled efficiency at that message
+// size, piecewise linear between the profiled sizes and constant outside them; no table: efficiency 1.
+__device__ __forceinline__ double link_eff(const DevConst &dc, int cls, double vol)
+{
+    const int n = dc.n_fsize;
+    if (vol <= dc.fsize[0]) return dc.feff[cls][0];
+    if (vol >= dc.fsize[n - 1]) return dc.feff[cls][n - 1];
+    int i = 0;
+    while (vol >= dc.fsize[i + 1]) ++i;
+    return dc.feff[cls][i] + (vol - dc.fsize[i]) * ((dc.feff[cls][i + 1] - dc.feff[cls][i]) / (dc.fsize[i + 1] - dc.fsize[i]));
+}
+
+__device__ __forceinline__ double xfer_ns(const DevConst &dc, int cls, double vol, double bw)
+{
+    const double t = vol / bw;
+    if (dc.n_fsize <= 0) return t;
+    return t / link_eff(dc, cls, vol);
+}
+
 // collective over w ranks that span `ext` consecutive devices, D bytes per rank
 __device__ __forceinline__ double collective_ns(const DevConst &dc, const LinkCtx &lc, i64 w, i64 ext, double D)
 {
@@ -146,7 +168,7 @@ __device__ __forceinline__ double collective_ns(const DevConst &dc, const LinkCt
     const int cls = link_class(lc, ext);
     const double lat = dc.alpha[cls] * (double)(w - 1);
     const double vol = (D * (double)(w - 1)) / (double)w;
-    return lat + vol / link_bw(lc, cls);
+    return lat + xfer_ns(dc, cls, vol, link_bw(lc, cls));
 }
 
 struct TypeConst {      // per (configuration, type) values used by every layer
@@ -225,8 +247,8 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
             const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
             const double Dag = (thb * dc.beta) * (double)(EP - 1);
             const int cls = link_class(lc, (i64)EP * TPE);
-            const double fa = dc.alpha[cls] * (double)(EP - 1) + Dmoe / link_bw(lc, cls);
-            const double fg = dc.alpha[cls] * (double)(EP - 1) + Dag / link_bw(lc, cls);
+            const double fa = dc.alpha[cls] * (double)(EP - 1) + xfer_ns(dc, cls, Dmoe, link_bw(lc, cls));
+            const double fg = dc.alpha[cls] * (double)(EP - 1) + xfer_ns(dc, cls, Dag, link_bw(lc, cls));
             tdisp = (fa <= fg) ? fa : fg;
         }
         tc.disp2 = 2.0 * tdisp;
@@ -250,13 +272,13 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
         bad |= put_coef<QUANT>(coef, coeff, at, HAP_KPRE, dc.tpre[i4]);
         bad |= put_coef<QUANT>(coef, coeff, at, HAP_KPOST, dc.tpost[i4]);
         const double Dp = Dtp / (double)TP;
-        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_INTRA, 2.0 * (dc.alpha[HAP_INTRA] + Dp / dc.bw_intra[h]));
-        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_INTER, 2.0 * (dc.alpha[HAP_INTER] + Dp / dc.bw_inter[h]));
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_INTRA, 2.0 * (dc.alpha[HAP_INTRA] + xfer_ns(dc, HAP_INTRA, Dp, dc.bw_intra[h])));
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_INTER, 2.0 * (dc.alpha[HAP_INTER] + xfer_ns(dc, HAP_INTER, Dp, dc.bw_inter[h])));
 #pragma unroll
         for (int h2 = 0; h2 < HAP_MAX_TYPES; ++h2) {
             const double bo = h2 < T ? dc.bw_inter[h2] : dc.bw_inter[h];
             const double bmin = dc.bw_inter[h] < bo ? dc.bw_inter[h] : bo;
-            bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_CROSS + h2, 2.0 * (dc.alpha[HAP_CROSS] + Dp / (bmin * dc.chi)));
+            bad |= put_coef<QUANT>(coef, coeff, at, HAP_KP2P_CROSS + h2, 2.0 * (dc.alpha[HAP_CROSS] + xfer_ns(dc, HAP_CROSS, Dp, bmin * dc.chi)));
         }
         const i64 wd = (i64)DP * CP;
         const double shd = 6.0 + 12.0 / (double)wd;
@@ -291,7 +313,7 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
             const i64 Pdd = Pd[kd] + (kd == HAP_MOE ? Prt : 0);
             const double Pel = kd == HAP_MOE ? PeT : 0.0;
             bad |= put_coef<QUANT>(coef, coeff, at, HAP_SBW + kd,
-                                   dc.ovl_dp * ((((6.0 * ((double)Pdd / (double)TP)) * vfd) / bwG) + (((6.0 * Pel) * vfe) / bwG)));
+                                   dc.ovl_dp * (xfer_ns(dc, cG, (6.0 * ((double)Pdd / (double)TP)) * vfd, bwG) + xfer_ns(dc, cG, (6.0 * Pel) * vfe, bwG)));
             bad |= put_coef<QUANT>(coef, coeff, at, HAP_OPT + kd,
                                    dc.copt[h] * ((double)Pdd / (double)((i64)TP * DP * CP) + Pel / (double)EDP));
         }

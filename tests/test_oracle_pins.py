@@ -807,3 +807,48 @@ def test_appendix_b_against_the_closed_form_and_the_schedule_simulation():
         appb = PP * (f + b) + f + (M - 1 - 1) * (f + b)           # s_max = 1 for identical stages
         assert appb == (M + PP - 2) * (f + b) + f
         assert _simulate_1f1b([f] * PP, [b] * PP, M) - appb == b
+
+
+# --------------------------------------------------------------------------------------
+# communication-primitive table: link efficiency by message size
+# --------------------------------------------------------------------------------------
+def _e1_with_table(sizes, intra, inter, cross):
+    pb = e1_problem()
+    pb.fsize = np.ascontiguousarray(np.array(sizes, np.float64))
+    pb.feff = np.ascontiguousarray(np.array([intra, inter, cross], np.float64))
+    return pb
+
+
+def test_link_efficiency_table_hand_values():
+    g = gold("e6_link_efficiency.json")["expect"]
+    _, _, coef0, _ = Oracle(e1_problem()).layer_costs(0)
+    assert coef0[0, COEF["KP2P_INTRA"]] == g["kp2p_intra_no_table"]            # 2 * (2000 + 10485.76)
+    _, _, coef, _ = Oracle(_e1_with_table([1e6, 1e7], [0.5, 0.9], [0.45, 0.85], [0.4, 0.8])).layer_costs(0)
+    assert coef[0, COEF["KP2P_INTRA"]] == g["kp2p_intra"]
+    assert coef[1, COEF["KP2P_CROSS"] + 0] == g["kp2p_cross"] and coef[0, COEF["KP2P_CROSS"] + 1] == g["kp2p_cross"]
+    _, _, coef, _ = Oracle(_e1_with_table([1e7, 1e8], [0.5, 0.9], [0.45, 0.85], [0.4, 0.8])).layer_costs(0)
+    assert coef[0, COEF["KP2P_INTRA"]] == g["kp2p_intra_below"]
+    _, _, coef, _ = Oracle(_e1_with_table([1e5, 1e6], [0.5, 0.9], [0.45, 0.85], [0.4, 0.8])).layer_costs(0)
+    assert coef[0, COEF["KP2P_INTRA"]] == g["kp2p_intra_above"]
+
+
+def test_link_efficiency_table_limits_and_monotonicity():
+    """Efficiency 1 everywhere is the model without a table, bit for bit; a lower efficiency never lowers a layer
+    time or a communication coefficient, and leaves the memory coefficients alone."""
+    pb = problems.small()
+    o0 = Oracle(pb)
+    ones = problems.with_link_efficiency_table(pb)
+    ones.feff = np.ones_like(ones.feff)
+    o1 = Oracle(ones)
+    ot = Oracle(problems.with_link_efficiency_table(pb))
+    comm = [COEF[k] for k in ("KP2P_INTRA", "KP2P_INTER", "SBW")] + [COEF["KP2P_CROSS"] + q for q in range(4)] + [COEF["SBW"] + 1]
+    mem = [COEF["MW"], COEF["MW"] + 1, COEF["MA"], COEF["MA"] + 1, COEF["MX"], COEF["MPRE"], COEF["MPOST"], COEF["OPT"], COEF["SLAT"]]
+    grew = 0
+    for p in range(0, o0.n_pconf, 37):
+        a, af, ac, _ = o0.layer_costs(p)
+        b, bf, bc, _ = o1.layer_costs(p)
+        c, cf, cc, _ = ot.layer_costs(p)
+        assert np.array_equal(a, b) and np.array_equal(af, bf) and np.array_equal(ac, bc)
+        assert (c >= a).all() and (cc[:, comm] >= ac[:, comm]).all() and np.array_equal(cc[:, mem], ac[:, mem])
+        grew += int((c > a).any())
+    assert grew > 0
