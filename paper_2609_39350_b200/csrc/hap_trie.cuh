@@ -254,7 +254,7 @@ __device__ __forceinline__ u32 trie_thr_index(const TrieMeta &tm, int T, int R, 
 // Block prologue, part 2: threshold = first split k, among those a cell of depth d can look at, for which
 // layers (k, j] fit stage d on a device of type t at level r (one past the last such split if none), only for the
 // end layers, device types and levels that occur at depth d.  Feasibility is monotone in the span, so a thread
-// sweeps a segment of eight end layers with a split pointer that only moves forward.
+// sweeps the end layers of a row with a split pointer that only moves forward.
 __device__ __forceinline__ void trie_prologue_thr(
     const DevConst &dc, const hap_pconf &pc, const TrieMeta &tm, unsigned p_index, const i64 *coef, unsigned levels,
     const i64 *sW, const i64 *sA, uint8_t *thr, const uint8_t *sK)
@@ -262,7 +262,9 @@ __device__ __forceinline__ void trie_prologue_thr(
     const int T = dc.T, R = dc.R, PP = pc.PP;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
-    constexpr int kSeg = 8;
+    // end layers per thread: a whole row (fewest evaluations: the pointer never restarts) when the rows alone keep
+    // half the block busy, segments of eight otherwise
+    const int kSeg = PP * T * R * 2 >= (int)blockDim.x ? 32 : 8;
     const int nseg = (tm.band_max + kSeg - 1) / kSeg;
     const int total = PP * T * R * nseg;
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
@@ -283,7 +285,15 @@ __device__ __forceinline__ void trie_prologue_thr(
         for (int j = j0; j <= j1; ++j) {
             if (k < j - wmax) k = j - wmax;
             const int kcap = kmax < j - 1 ? kmax : j - 1;           // no cell looks at a split beyond this
-            while (k <= kcap && !span_fits(sW, sA, sK, extra, mx, mstore, cap, xi, k, j)) ++k;
+            // span (k, j] fits: weights + extra (+ MoE buffers if it holds an MoE layer) + xi * stored activations / 1024
+            const i64 Wj = sW[j] + extra, Aj = sA[j];
+            const int Kj = sK[j];
+            while (k <= kcap) {
+                const i64 Wb = (Wj - sW[k]) + (Kj != sK[k] ? mx : 0);
+                const i64 A = mstore * (Aj - sA[k]);
+                if (Wb + ((xi * A) >> 10) <= cap) break;
+                ++k;
+            }
             row[j] = (uint8_t)k;
         }
     }
