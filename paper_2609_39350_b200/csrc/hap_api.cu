@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -80,6 +81,18 @@ struct SingleOut {
     hap_candidate cand;
 };
 
+// The side streams the PP classes run on are shared by all problems of a device and live until the process ends:
+// creating half a dozen streams costs more than a whole search.  Index = position of the class in the problem.
+static cudaStream_t pooled_stream(int device, size_t index)
+{
+    static std::mutex mu;
+    static cudaStream_t pool[64][HAP_MAX_PP + 1];
+    std::lock_guard<std::mutex> lock(mu);
+    cudaStream_t &s = pool[device & 63][index % (HAP_MAX_PP + 1)];
+    if (!s && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) s = nullptr;
+    return s;
+}
+
 static hap_status fail(hap_problem *p, hap_status s, const char *fmt, ...)
 {
     if (p) {
@@ -127,7 +140,7 @@ static void release_device(hap_problem *p)
     cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-    for (auto &cl : p->classes) { if (cl.stream) cudaStreamDestroy(cl.stream); if (cl.done) cudaEventDestroy(cl.done); }
+    for (auto &cl : p->classes) { if (cl.done) cudaEventDestroy(cl.done); }      // the class streams belong to the pool
 }
 
 extern "C" void hap_problem_destroy(hap_problem *p)
@@ -337,7 +350,9 @@ struct TriePartHost {
 };
 
 // the tree of mappings [m0, m1) of the class
-static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, const uint8_t *tab_all, u64 m0, u64 m1, TriePartHost &part)
+// `limit`: largest acceptable dynamic shared memory; a tree that needs more is abandoned before its records are written
+static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, const uint8_t *tab_all, u64 m0, u64 m1, size_t limit,
+                            TriePartHost &part)
 {
     const int N = p->model.N, PP = cl.PP, T = p->T, R = p->prof.R;
     const u64 nmap = m1 - m0;
@@ -466,6 +481,17 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
         n_nodes += (u32)lv[d].size(); n_cells += c;
     }
     for (int d = std::max(PP, 1); d <= HAP_MAX_PP; ++d) { tm.node_lo[d] = n_nodes; tm.cell_lo[d] = n_cells; }
+    {   // the shared memory the tree needs is known from the node bands: stop here if it is too much
+        int widest = 1;
+        for (int d = 1; d < PP; ++d) {
+            int lo = 1 << 20, hi = -1;
+            for (const auto &h : lv[d]) { lo = std::min(lo, h.bl); hi = std::max(hi, h.bh); }
+            if (hi >= lo) widest = std::max(widest, hi - lo + 1);
+        }
+        const u32 be = (tm.buf_cells[0] + 1) / 2 * 2, bo = (tm.buf_cells[1] + 1) / 2 * 2;
+        part.smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, widest, be, bo, n_cells, n_nodes);
+        if (part.smem > limit) return false;
+    }
     tm.buf_cells[0] = (tm.buf_cells[0] + 1) / 2 * 2; tm.buf_cells[1] = (tm.buf_cells[1] + 1) / 2 * 2;
     if (n_cells >= (1u << 25)) return false;
     std::vector<TrieNode> nodes(n_nodes);
@@ -519,7 +545,7 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
     }
     tm.band_max = band_max;
     const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, band_max, tm.buf_cells[0], tm.buf_cells[1], n_cells, n_nodes);
-    if (smem > 220 * 1024) return false;
+    if (smem > limit) return false;
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];
         if (lf.dead || PP == 1) { lf.prowoff = 0; lf.pbl = 0; lf.pbh = 0; continue; }
@@ -562,21 +588,18 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     if (nmap == 0 || plist.empty()) return false;
     constexpr size_t kTwoPerSm = 108 * 1024;                 // dynamic shared memory that lets two blocks share an SM
     const size_t slots = (cl.item_hi - cl.item_lo) / plist.size();       // partial-result slots per configuration
-    std::vector<TriePartHost> parts, whole;
+    std::vector<TriePartHost> parts;
     for (int np : {1, 2, 3, 4, 6, 8}) {
         if ((u64)np > nmap || (np > 1 && (size_t)np > slots)) break;
         std::vector<TriePartHost> cand(np);
         bool ok = true;
-        size_t worst = 0;
-        for (int q = 0; q < np && ok; ++q) {
-            const u64 m0 = nmap * q / np, m1 = nmap * (q + 1) / np;
-            ok = build_trie_part(p, cl, tab, m0, m1, cand[q]);
-            if (ok) worst = std::max(worst, cand[q].smem);
-        }
-        if (np == 1 && ok) whole = cand;
-        if (ok && worst <= kTwoPerSm) { parts.swap(cand); break; }
+        for (int q = 0; q < np && ok; ++q) ok = build_trie_part(p, cl, tab, nmap * q / np, nmap * (q + 1) / np, kTwoPerSm, cand[q]);
+        if (ok) { parts.swap(cand); break; }
     }
-    if (parts.empty()) parts.swap(whole);                    // one block per SM
+    if (parts.empty()) {                                     // no split lets two blocks share an SM: one block per SM
+        parts.resize(1);
+        if (!build_trie_part(p, cl, tab, 0, nmap, 220 * 1024, parts[0])) parts.clear();
+    }
     if (parts.empty()) return false;
     out.parts.swap(parts);
     out.plist = plist;
@@ -793,8 +816,10 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         p->dc.pconf = p->d_pconf;
         p->dc.n_pconf = np;
         CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
-        for (auto &cl : p->classes) {
-            CUDA_TRY(p, cudaStreamCreateWithFlags(&cl.stream, cudaStreamNonBlocking));
+        for (size_t ci = 0; ci < p->classes.size(); ++ci) {
+            auto &cl = p->classes[ci];
+            cl.stream = pooled_stream(p->device, ci);
+            if (!cl.stream) return fail(p, HAP_E_CUDA, "cudaStreamCreateWithFlags");
             CUDA_TRY(p, cudaEventCreateWithFlags(&cl.done, cudaEventDisableTiming));
         }
         if (tab_bytes) {
