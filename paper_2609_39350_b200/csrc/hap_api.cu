@@ -654,7 +654,8 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
         std::memcpy(stage.data() + off, h.plist.data(), h.plist.size() * sizeof(u32));
         off += up(h.plist.size() * sizeof(u32));
         tr.n_conf = (unsigned)h.plist.size(); tr.smem = smem;
-        const int th = (int)(((want + 1) / 2 + 31) / 32 * 32);
+        // a thread takes about four cells of the widest depth (measured: smaller blocks, more of them per SM)
+        const int th = (int)(((want + 3) / 4 + 31) / 32 * 32);
         tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
         tr.ok = true;
     }
