@@ -155,3 +155,37 @@ def test_large_multiset_class(hap):
     plan, stats = hap.hap_search_best(hp)
     assert (plan["T_iter"], plan["index"]) == (bc, bi)
     hap.hap_problem_destroy(hp)
+
+
+def test_many_random_problems_agree_between_the_two_kernels(hap):
+    """Differential test without the oracle in the loop: forty random problems (two to four device types, window on
+    and off, one to three recomputation levels, several policies, dense first layer or not, uniform-split ablation,
+    heterogeneous-communication rule) through both kernels; every output must be identical."""
+    shapes = [((2, 2), 2), ((2, 1, 1), 3), ((1, 1, 1, 1), 4), ((4, 2, 2), 3), ((3, 1), 2)]
+    n_checked = 0
+    for seed in range(40):
+        nodes, T = shapes[seed % len(shapes)]
+        pb = problems.random_small(100 + seed, N=6 + (seed * 7) % 19, T=T, nodes_per_type=nodes, node_size=2,
+                                   window=(seed % 3 != 1), first_dense=(seed % 4 == 0))
+        if seed % 5 == 2:
+            pb.xi_q = np.ascontiguousarray(np.array([1024, 512, 64], np.int32))
+            pb.tau_q = np.ascontiguousarray(np.array([0, 1024, 3072], np.int32))
+            pb.rc_masks = np.ascontiguousarray(np.array([0b001, 0b011, 0b111, 0b101, 0b100], np.uint32))
+        if seed % 5 == 3:
+            pb.rc_masks = np.ascontiguousarray(np.array([0b01], np.uint32))
+        if seed % 7 == 6:
+            pb.uniform = 1
+        if seed % 6 == 5:
+            pb.eta_q = 40
+        if seed % 8 == 7:
+            pb.map_cap = 4                                  # forces block orderings with mixed stages
+        hp_t, tree = _pass(hap, pb, 0)
+        hp_w, warp = _pass(hap, pb, hap.OPT_NO_TRIE)
+        for key in ("cost", "bottleneck", "partition", "recompute"):
+            assert np.array_equal(tree[key], warp[key]), (seed, key)
+        if (tree["cost"] < INF).any():
+            assert hap.hap_search_best(hp_t)[0] == hap.hap_search_best(hp_w)[0], seed
+        n_checked += len(tree["cost"])
+        hap.hap_problem_destroy(hp_t)
+        hap.hap_problem_destroy(hp_w)
+    assert n_checked > 20000
