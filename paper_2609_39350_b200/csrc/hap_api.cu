@@ -298,6 +298,8 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     dc.tau_linear = 1;
     for (int r = 0; r < pf->R; ++r) { dc.xi_q[r] = p->xi_q[r]; dc.tau_q[r] = p->tau_q[r]; if (p->tau_q[r] % 1024) dc.tau_linear = 0; }
     for (int l = 0; l < N; ++l) if (p->kind[l] == HAP_MOE) dc.kindbits[l >> 6] |= 1ull << (l & 63);
+    dc.kind_uniform = 1;
+    for (int l = 1; l < N; ++l) if (p->kind[l] != p->kind[0]) dc.kind_uniform = 0;
     dc.tdf = p->d_tables; dc.tdb = dc.tdf + n5; dc.tff = dc.tdb + n5; dc.tfb = dc.tff + n5;
     dc.tpre = dc.tfb + n5; dc.tpost = dc.tpre + n4;
 

@@ -41,6 +41,7 @@ struct DevConst {
     int N, T, R, n_rc, ntp, ncp, nmb, nep;
     int S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
     int delta_q, tau_linear, eta_q, uniform;
+    int kind_uniform;                 // every layer is of one kind (all MoE or all dense): a span's memory depends on its length only
     double beta, kappa, chi, gamma, ovl_tp, ovl_cp, ovl_dp, capf;
     double alpha[3];
     double eta[HAP_MAX_TYPES], croute[HAP_MAX_TYPES], copt[HAP_MAX_TYPES];

@@ -262,6 +262,42 @@ __device__ __forceinline__ void trie_prologue_thr(
     const int T = dc.T, R = dc.R, PP = pc.PP;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
+    if (dc.kind_uniform) {
+        // All layers of one kind: the memory of a span depends on its length alone, so a row is settled by the longest
+        // span that fits (a search over the lengths a window of this depth allows), threshold(j) = j - that length.
+        __shared__ uint8_t s_nfit[HAP_MAX_PP * HAP_MAX_TYPES * HAP_MAX_RC];
+        const int rows = PP * T * R;
+        for (int q = threadIdx.x; q < rows; q += blockDim.x) {
+            const int r = q % R, t = (q / R) % T, d = q / (R * T) + 1;
+            int fit = 0;
+            if (((levels >> r) & 1u) && ((tm.tmask[d] >> t) & 1u)) {
+                const i64 extra = (d == 1 ? mpre : 0) + (d == PP ? mpost : 0);
+                const int inflight = PP - d + 1;
+                const i64 mstore = pc.M < inflight ? pc.M : inflight;
+                int lo = 0, hi = tm.wmax[d];                 // invariant: lengths <= lo fit (0: trivially), lengths > hi do not
+                while (lo < hi) {
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (span_fits(sW, sA, sK, extra, mx, mstore, dc.cap_eff[t], dc.xi_q[r], 0, mid)) lo = mid; else hi = mid - 1;
+                }
+                fit = lo;
+            }
+            s_nfit[q] = (uint8_t)fit;
+        }
+        __syncthreads();
+        const int bw = tm.band_max;
+        for (int e = threadIdx.x; e < rows * bw; e += blockDim.x) {
+            const int q = e / bw, d = q / (R * T) + 1, j = tm.jlo[d] + (e - q * bw);
+            if (j > tm.jhi[d]) continue;
+            const int start = j - (int)tm.wmax[d] > (int)tm.kmin[d] ? j - (int)tm.wmax[d] : (int)tm.kmin[d];
+            const int kcap = (int)tm.kmax[d] < j - 1 ? (int)tm.kmax[d] : j - 1;   // no cell looks at a split beyond this
+            const int fit = s_nfit[q];
+            int k = j - fit > start ? j - fit : start;
+            if (fit == 0 || k > kcap) k = kcap + 1;
+            thr[e] = (uint8_t)(k < 0 ? 0 : k);
+        }
+        __syncthreads();
+        return;
+    }
     // end layers per thread: a whole row (fewest evaluations: the pointer never restarts) when the rows alone keep
     // half the block busy, segments of eight otherwise
     const int kSeg = PP * T * R * 2 >= (int)blockDim.x ? 32 : 8;
