@@ -491,7 +491,7 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
             if (hi >= lo) widest = std::max(widest, hi - lo + 1);
         }
         const u32 be = (tm.buf_cells[0] + 1) / 2 * 2, bo = (tm.buf_cells[1] + 1) / 2 * 2;
-        part.smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, widest, be, bo, n_cells, n_nodes);
+        part.smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, p->dc.kind_uniform ? 1 : widest, be, bo, n_cells, n_nodes);
         if (part.smem > limit) return false;
     }
     tm.buf_cells[0] = (tm.buf_cells[0] + 1) / 2 * 2; tm.buf_cells[1] = (tm.buf_cells[1] + 1) / 2 * 2;
@@ -540,13 +540,15 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
             }
         }
     for (int d = 1; d <= PP; ++d) if (tm.jlo[d] <= tm.jhi[d]) band_max = std::max(band_max, tm.jhi[d] - tm.jlo[d] + 1);
+    const int thr_w = p->dc.kind_uniform ? 1 : band_max;        // one threshold per row when a span's memory depends on its length only
+    tm.thr_w = thr_w;
     for (u32 c = 0; c < n_cells; ++c) {
         const u32 g = cell_gnode[c];
         const int d = depth[g], j = (int)(cells[c].y & 255);
-        cells[c].z = (u32)((((d - 1) * T + capt_of[nodes[g].mask]) * R) * band_max + (j - (int)tm.jlo[d]));
+        cells[c].z = (u32)((((d - 1) * T + capt_of[nodes[g].mask]) * R) * thr_w + (thr_w == 1 ? 0 : j - (int)tm.jlo[d]));
     }
     tm.band_max = band_max;
-    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, band_max, tm.buf_cells[0], tm.buf_cells[1], n_cells, n_nodes);
+    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, thr_w, tm.buf_cells[0], tm.buf_cells[1], n_cells, n_nodes);
     if (smem > limit) return false;
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];

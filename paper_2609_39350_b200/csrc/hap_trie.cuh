@@ -63,16 +63,17 @@ struct TrieMeta {
     u32 buf_cells[2];               // largest row storage of an even / odd depth, in cells
     u32 nmap, m_lo;                 // the tree covers mappings [m_lo, m_lo + nmap) of the class
     int PP, band_max;               // band_max: most end layers of any depth
+    int thr_w;                      // entries per row of the threshold table: band_max, or 1 when all layers are of one kind
 };
 
 constexpr int kTrieKtab = 16 + HAP_MAX_TYPES * 6;    // stage constants: [0,16) pre-work by row group, then p2p [type][6]
 
-__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, int n_mrows, int band_max, u32 buf_even, u32 buf_odd, u32 cells,
+__host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, int n_mrows, int thr_w, u32 buf_even, u32 buf_odd, u32 cells,
                                                   u32 n_nodes)
 {
     const size_t n1 = (size_t)N + 1;
     size_t b = (((size_t)n_mrows * R + 2) * n1 * 8 + 15) / 16 * 16;      // time rows, weight and activation byte rows
-    b += ((size_t)PP * T * R * band_max + 15) / 16 * 16;                  // memory thresholds
+    b += ((size_t)PP * T * R * thr_w + 15) / 16 * 16;                     // memory thresholds
     b += (n1 + 15) / 16 * 16;                                              // MoE prefix counts
     b += (size_t)T * N * 16;                                               // staged layer times of the configuration
     b += (size_t)kTrieKtab * 8;
@@ -248,12 +249,12 @@ __device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, cons
 // index of the memory threshold of (stage d, capacity type t, level r, end layer j) in the block's table
 __device__ __forceinline__ u32 trie_thr_index(const TrieMeta &tm, int T, int R, int d, int t, int r, int j)
 {
-    return (u32)((((d - 1) * T + t) * R + r) * tm.band_max + (j - (int)tm.jlo[d]));
+    return (u32)((((d - 1) * T + t) * R + r) * tm.thr_w + (tm.thr_w == 1 ? 0 : j - (int)tm.jlo[d]));
 }
 
-// Block prologue, part 2: threshold = first split k, among those a cell of depth d can look at, for which
-// layers (k, j] fit stage d on a device of type t at level r (one past the last such split if none), only for the
-// end layers, device types and levels that occur at depth d.  Feasibility is monotone in the span, so a thread
+// Block prologue, part 3: threshold table: for stage d on a device of type t at level r, the length of the longest
+// span ending at layer j that fits (among the splits a cell of depth d can look at; 0: none), only for the end
+// layers, device types and levels that occur at depth d; one entry per row when all layers are of one kind.  Feasibility is monotone in the span, so a thread
 // sweeps the end layers of a row with a split pointer that only moves forward.
 __device__ __forceinline__ void trie_prologue_thr(
     const DevConst &dc, const hap_pconf &pc, const TrieMeta &tm, unsigned p_index, const i64 *coef, unsigned levels,
@@ -263,9 +264,8 @@ __device__ __forceinline__ void trie_prologue_thr(
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
     if (dc.kind_uniform) {
-        // All layers of one kind: the memory of a span depends on its length alone, so a row is settled by the longest
-        // span that fits (a search over the lengths a window of this depth allows), threshold(j) = j - that length.
-        __shared__ uint8_t s_nfit[HAP_MAX_PP * HAP_MAX_TYPES * HAP_MAX_RC];
+        // All layers of one kind: the memory of a span depends on its length alone, so a row is one number, the
+        // longest span that fits (a search over the lengths a window of this depth allows).
         const int rows = PP * T * R;
         for (int q = threadIdx.x; q < rows; q += blockDim.x) {
             const int r = q % R, t = (q / R) % T, d = q / (R * T) + 1;
@@ -281,19 +281,7 @@ __device__ __forceinline__ void trie_prologue_thr(
                 }
                 fit = lo;
             }
-            s_nfit[q] = (uint8_t)fit;
-        }
-        __syncthreads();
-        const int bw = tm.band_max;
-        for (int e = threadIdx.x; e < rows * bw; e += blockDim.x) {
-            const int q = e / bw, d = q / (R * T) + 1, j = tm.jlo[d] + (e - q * bw);
-            if (j > tm.jhi[d]) continue;
-            const int start = j - (int)tm.wmax[d] > (int)tm.kmin[d] ? j - (int)tm.wmax[d] : (int)tm.kmin[d];
-            const int kcap = (int)tm.kmax[d] < j - 1 ? (int)tm.kmax[d] : j - 1;   // no cell looks at a split beyond this
-            const int fit = s_nfit[q];
-            int k = j - fit > start ? j - fit : start;
-            if (fit == 0 || k > kcap) k = kcap + 1;
-            thr[e] = (uint8_t)(k < 0 ? 0 : k);
+            thr[q] = (uint8_t)fit;
         }
         __syncthreads();
         return;
@@ -330,7 +318,7 @@ __device__ __forceinline__ void trie_prologue_thr(
                 if (Wb + ((xi * A) >> 10) <= cap) break;
                 ++k;
             }
-            row[j] = (uint8_t)k;
+            row[j] = (uint8_t)(k <= kcap ? j - k : 0);              // the longest span ending at j that fits (0: none)
         }
     }
     __syncthreads();
@@ -364,7 +352,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     __syncthreads();
     const u32 p = plist[blockIdx.x / (unsigned)n_parts];
     const hap_pconf pc = dc.pconf[p];
-    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.band_max;
+    const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.thr_w;
     const u64 c_lo = pc.offset + (u64)tm.m_lo * n_rc, c_hi = c_lo + (u64)tm.nmap * n_rc;   // candidates of this block
     const u64 w_lo = out.first, w_hi = out.first + out.count;                  // candidates that are wanted
     if (c_hi <= w_lo || c_lo >= w_hi) {
@@ -464,7 +452,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         int seg_hi = khi;
         for (int r = 0; r < R && seg_hi >= klo; ++r, a_th += (u32)bw, a_row += (u32)n1 * 8u) {
             if (!((rc_mask >> r) & 1u)) continue;
-            int lo = lds_u8(a_th);
+            int lo = j - lds_u8(a_th);           // first split of this level: end layer minus the longest span that fits
             if (lo < klo) lo = klo;
             if (lo > seg_hi) continue;
             const int n = seg_hi - lo + 1;
@@ -580,7 +568,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 const uint8_t *th = thr + trie_thr_index(tm, T, R, d, mi.capt, 0, b);
                 int r = 0;
                 for (; r < R; ++r)
-                    if (((rc_mask >> r) & 1u) && th[r * bw] <= a) break;
+                    if (((rc_mask >> r) & 1u) && b - (int)th[r * bw] <= a) break;
                 const double *rr = sR + ((size_t)tm.mrow_of[mask] * R + r) * n1;
                 const i64 cst = (i64)(rr[b] - rr[a]) + stage_K(d, mask, link);
                 sum += cst; mxc = cst > mxc ? cst : mxc;
