@@ -207,7 +207,14 @@ typedef struct hap_problem hap_problem;
  * tables to the current device.  *out is NULL on failure. */
 hap_status hap_problem_create(const hap_model *, const hap_cluster *, const hap_profile *,
                               const hap_search_opts *, hap_problem **out);
+/* Waits for the problem's device work and releases it.  Its device memory is not returned to the driver but kept
+ * (up to 24 blocks and 4 GiB per process) for the next hap_problem_create / hap_enumerate of the same device, which
+ * reuse a block that fits with at most a quarter to spare: allocating and freeing a problem's arenas costs about as
+ * much as a whole search.  No counterpart in the paper (resource management of this library). */
 void hap_problem_destroy(hap_problem *);
+/* Returns every idle block of that cache, on every device, to the driver (cudaFree).  Blocks of live problems are
+ * not touched.  HAP_E_CUDA if a free failed. */
+hap_status hap_release_cached_memory(void);
 
 /* Sec. 3.5 / 5.1 "searches the 6D parallel space": enumerates every (PP,TP,CP,DP,EP,TPE) with
  * PP*TP*CP*DP = #devices, EP*TPE | TP*CP*DP, EP | E, x micro-batch size, in a fixed

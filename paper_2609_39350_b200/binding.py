@@ -17,7 +17,7 @@ STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE",
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
            "hap_search_range", "hap_search_range_f64",
-           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_release_cached_memory", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -357,6 +357,13 @@ def hap_eval_appendix_b(hp: HapProblem, first: int, count: int, partition, recom
     hp.check(load_library().hap_eval_appendix_b(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(partition), _dev(recompute),
                                                 _dev(t), _dev(d), _stream(stream)))
     return {"t_iter": t, "detail": d}
+
+
+def hap_release_cached_memory() -> None:
+    """Returns the device memory the library keeps from destroyed problems to the driver."""
+    st = load_library().hap_release_cached_memory()
+    if st != 0:
+        raise HapError(st, "hap_release_cached_memory")
 
 
 def hap_launches_per_pass(hp: HapProblem) -> int:

@@ -12,6 +12,7 @@
 #include <mutex>
 #include <new>
 #include <string>
+#include <unordered_map>
 #include <vector>
 
 using namespace hap;
@@ -40,7 +41,8 @@ struct hap_problem {
                          u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
     struct Trie { bool ok = false; TrieMeta *d_metas = nullptr; u32 *d_plist = nullptr;       // both inside d_trie_arena
                   std::vector<TriePartDev> parts; unsigned n_conf = 0; int threads = 0; size_t smem = 0; };
-    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie;
+                     mutable bool decoded = false; };       // this pass's candidate decode is already queued on `stream`
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     unsigned char *d_arena = nullptr;      // everything hap_enumerate sizes, in one allocation (the d_* pointers below point into it)
@@ -71,6 +73,7 @@ struct hap_problem {
     bool timed = false;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_fork = nullptr;          // classes run on their own streams between this event and their `done` events
+    cudaEvent_t ev_pre = nullptr;           // start of a pass: the candidate decode of the classes waits for this one only
     std::string err;
 };
 
@@ -91,6 +94,87 @@ static cudaStream_t pooled_stream(int device, size_t index)
     cudaStream_t &s = pool[device & 63][index % (HAP_MAX_PP + 1)];
     if (!s && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) s = nullptr;
     return s;
+}
+
+// Device memory of destroyed problems is kept for the next problem of the process: allocating and freeing the
+// three arenas of a problem costs about as much as the search itself.  A freed block serves a later request
+// of its device that it fits with at most a quarter (plus 1 MiB) to spare.  At most kCacheBlocks blocks and kCacheBytes
+// bytes are held; hap_release_cached_memory() returns everything to the driver.
+namespace {
+struct CachedBlock { int device; size_t bytes; void *ptr; };
+struct MemCache {
+    std::mutex mu;
+    std::vector<CachedBlock> idle;
+    std::unordered_map<void *, CachedBlock> live;
+    size_t idle_bytes = 0;
+};
+constexpr size_t kCacheBlocks = 24;
+constexpr size_t kCacheBytes = 4ull << 30;
+MemCache &mem_cache() { static MemCache *c = new MemCache(); return *c; }     // never destroyed: outlives static teardown
+}  // namespace
+
+static cudaError_t cached_malloc(int device, void **out, size_t bytes)
+{
+    MemCache &mc = mem_cache();
+    bytes = (std::max<size_t>(bytes, 1) + 0xffff) & ~(size_t)0xffff;
+    std::lock_guard<std::mutex> lock(mc.mu);
+    size_t best = mc.idle.size();
+    for (size_t i = 0; i < mc.idle.size(); ++i) {
+        const CachedBlock &b = mc.idle[i];
+        if (b.device != device || b.bytes < bytes || b.bytes > bytes + bytes / 4 + (1u << 20)) continue;
+        if (best == mc.idle.size() || b.bytes < mc.idle[best].bytes) best = i;
+    }
+    if (best != mc.idle.size()) {
+        const CachedBlock b = mc.idle[best];
+        mc.idle.erase(mc.idle.begin() + (long)best);
+        mc.idle_bytes -= b.bytes;
+        mc.live[b.ptr] = b;
+        *out = b.ptr;
+        return cudaSuccess;
+    }
+    void *ptr = nullptr;
+    cudaError_t e = cudaMalloc(&ptr, bytes);
+    if (e == cudaErrorMemoryAllocation) {           // give the idle blocks of this device back and try once more
+        cudaGetLastError();
+        for (size_t i = mc.idle.size(); i-- > 0;)
+            if (mc.idle[i].device == device) { cudaFree(mc.idle[i].ptr); mc.idle_bytes -= mc.idle[i].bytes; mc.idle.erase(mc.idle.begin() + (long)i); }
+        e = cudaMalloc(&ptr, bytes);
+    }
+    if (e != cudaSuccess) { *out = nullptr; return e; }
+    mc.live[ptr] = CachedBlock{device, bytes, ptr};
+    *out = ptr;
+    return cudaSuccess;
+}
+
+// The caller has made sure that no work that touches the block is still in flight.
+static void cached_free(void *ptr)
+{
+    if (!ptr) return;
+    MemCache &mc = mem_cache();
+    std::lock_guard<std::mutex> lock(mc.mu);
+    auto it = mc.live.find(ptr);
+    if (it == mc.live.end()) { cudaFree(ptr); return; }
+    const CachedBlock b = it->second;
+    mc.live.erase(it);
+    if (mc.idle.size() >= kCacheBlocks || mc.idle_bytes + b.bytes > kCacheBytes) { cudaFree(ptr); return; }
+    mc.idle.push_back(b);
+    mc.idle_bytes += b.bytes;
+}
+
+extern "C" hap_status hap_release_cached_memory(void)
+{
+    MemCache &mc = mem_cache();
+    std::lock_guard<std::mutex> lock(mc.mu);
+    int prev = 0;
+    const bool have_prev = cudaGetDevice(&prev) == cudaSuccess;
+    hap_status st = HAP_OK;
+    for (const CachedBlock &b : mc.idle)
+        if (cudaSetDevice(b.device) != cudaSuccess || cudaFree(b.ptr) != cudaSuccess) st = HAP_E_CUDA;
+    mc.idle.clear();
+    mc.idle_bytes = 0;
+    if (have_prev) cudaSetDevice(prev);
+    if (st != HAP_OK) cudaGetLastError();
+    return st;
 }
 
 static hap_status fail(hap_problem *p, hap_status s, const char *fmt, ...)
@@ -134,12 +218,15 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 
 static void release_device(hap_problem *p)
 {
-    cudaFree(p->d_tables); cudaFree(p->d_arena); cudaFree(p->d_trie_arena);
-    cudaFree(p->d_joint_scratch);
-    for (auto &j : p->joint) { cudaFree(j.d_ids); cudaFree(j.d_arrays); }
-    cudaFree(p->d_c2f); cudaFree(p->d_coeff); cudaFree(p->d_fcost);
+    // nothing of this problem may still be running when its memory goes back to the cache
+    if (p->d_tables || p->d_arena) cudaDeviceSynchronize();
+    cached_free(p->d_tables); cached_free(p->d_arena); cached_free(p->d_trie_arena);
+    cached_free(p->d_joint_scratch);
+    for (auto &j : p->joint) { cached_free(j.d_ids); cached_free(j.d_arrays); }
+    cached_free(p->d_c2f); cached_free(p->d_coeff); cached_free(p->d_fcost);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+    if (p->ev_pre) cudaEventDestroy(p->ev_pre);
     for (auto &cl : p->classes) { if (cl.done) cudaEventDestroy(cl.done); }      // the class streams belong to the pool
 }
 
@@ -256,7 +343,7 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
 
     // ---- device ------------------------------------------------------------------------------
     if (cudaGetDevice(&p->device) != cudaSuccess) return HAP_E_CUDA;
-    if (cudaMalloc(&p->d_tables, tables.size() * sizeof(double)) != cudaSuccess) return HAP_E_NOMEM;
+    if (cached_malloc(p->device, (void **)&p->d_tables, tables.size() * sizeof(double)) != cudaSuccess) return HAP_E_NOMEM;
     if (cudaMemcpy(p->d_tables, tables.data(), tables.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess)
         return HAP_E_CUDA;
     for (auto &e : p->ev) if (cudaEventCreate(&e) != cudaSuccess) return HAP_E_CUDA;
@@ -622,7 +709,7 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
         total += up(bc.second.parts.size() * sizeof(TrieMeta)) + up(bc.second.plist.size() * sizeof(u32));
     }
     if (!total) return true;
-    if (cudaMalloc(&p->d_trie_arena, total) != cudaSuccess) { p->d_trie_arena = nullptr; cudaGetLastError(); return false; }
+    if (cached_malloc(p->device, (void **)&p->d_trie_arena, total) != cudaSuccess) { p->d_trie_arena = nullptr; cudaGetLastError(); return false; }
     std::vector<unsigned char> stage(total, 0);
     size_t off = 0;
     for (auto &bc : built) {
@@ -802,7 +889,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             const size_t o_counters = o; o = up(o + 8 * sizeof(u64));
             const size_t o_best = o; o = up(o + 2 * sizeof(i64));
             const size_t o_single = o; o = up(o + sizeof(SingleOut));
-            CUDA_TRY(p, cudaMalloc(&p->d_arena, o));
+            CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_arena, o));
             unsigned char *base = p->d_arena;
             p->d_pconf = reinterpret_cast<hap_pconf *>(base + o_pconf); p->d_items = reinterpret_cast<WorkItem *>(base + o_items);
             p->d_c2 = reinterpret_cast<i64 *>(base + o_c2); p->d_coef = reinterpret_cast<i64 *>(base + o_coef);
@@ -821,6 +908,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         p->dc.pconf = p->d_pconf;
         p->dc.n_pconf = np;
         CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
+        CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_pre, cudaEventDisableTiming));
         for (size_t ci = 0; ci < p->classes.size(); ++ci) {
             auto &cl = p->classes[ci];
             cl.stream = pooled_stream(p->device, ci);
@@ -923,8 +1011,17 @@ static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double 
     if ((quant && c2) || (!quant && c2f)) {
         const unsigned b2 = (unsigned)p->pconfs.size();
         const unsigned thr = (unsigned)((p->model.N + 31) / 32 * 32);
-        if (quant) layer_cost_kernel<true><<<b2, thr, 0, st>>>(p->dc, p->d_tc, c2, nullptr, lb_sum, p->d_range);
-        else layer_cost_kernel<false><<<b2, thr, 0, st>>>(p->dc, p->d_tc, nullptr, c2f, nullptr, p->d_range);
+        // programmatic dependent launch: the blocks start while type_const_kernel drains and wait inside the kernel
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(b2); cfg.blockDim = dim3(thr); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        const TypeConst *tcg = p->d_tc;
+        i64 *no_i = nullptr; double *no_d = nullptr;
+        if (quant) CUDA_TRY(p, cudaLaunchKernelEx(&cfg, layer_cost_kernel<true>, p->dc, tcg, c2, no_d, lb_sum, p->d_range));
+        else CUDA_TRY(p, cudaLaunchKernelEx(&cfg, layer_cost_kernel<false>, p->dc, tcg, no_i, c2f, no_i, p->d_range));
     }
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
@@ -946,6 +1043,59 @@ extern "C" hap_status hap_eval_layer_costs_f64(hap_problem *p, double *dev_c2, d
     return launch_layer_costs(p, nullptr, nullptr, dev_c2, dev_coef, false, (cudaStream_t)stream);
 }
 
+// whether all candidates of the class lie outside the range the pass writes
+static bool class_outside(const hap_problem *p, const hap_problem::PpClass &cl, const DpOut &out)
+{
+    const WorkItem &a = p->items[cl.item_lo], &b = p->items[cl.item_hi - 1];
+    const u64 c0 = p->pconfs[a.p].offset, c1 = p->pconfs[b.p].offset + p->pconfs[b.p].nmap * (u64)p->opts.n_rc;
+    return c1 <= out.first || c0 >= out.first + out.count;
+}
+
+// plain integer passes over more than one candidate walk the class's prefix tree; tables, refinement, fp64, cell
+// counting and the one-candidate re-evaluation stay in pipeline_dp_kernel
+static bool pass_uses_trie(const hap_problem *p, const hap_problem::PpClass &cl, const DpOut &out, bool f64)
+{
+    const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
+    return cl.trie.ok && !f64 && !out.count_only && !refine && p->dc.tau_linear != 0 && !out.dp_table && !out.choice && out.count > 1;
+}
+
+// candidate decode of a class for this pass, then its stage bytes into the class's tree
+static hap_status launch_class_decode(hap_problem *p, const hap_problem::PpClass &cl)
+{
+    const hap_problem::Trie &tr = cl.trie;
+    const uint8_t *tab = p->d_maptab + cl.map_base;
+    const u64 nmap = p->pconfs[p->items[cl.item_lo].p].nmap;
+    maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, p->items[cl.item_lo].p, nmap, p->d_maptab + cl.map_base);
+    CUDA_TRY(p, cudaGetLastError());
+    for (const auto &pd : tr.parts) {
+        const u32 n_g = pd.n_nodes + pd.n_cells + pd.nmap;
+        TrieRowMap rmap;
+        std::memcpy(rmap.mrow_of, pd.mrow_of, sizeof(rmap.mrow_of));
+        trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, pd.n_nodes, pd.n_cells, pd.nmap, pd.m_lo, pd.d_first_leaf,
+                                                                      pd.d_depth, pd.d_gnode, rmap, pd.d_nodes, pd.d_cells, pd.d_leaves);
+        CUDA_TRY(p, cudaGetLastError());
+    }
+    return HAP_OK;
+}
+
+// The candidate decode reads nothing the layer-cost kernels write: a pass queues it on the class streams first, so
+// that it runs beside the layer costs instead of between them and the recurrence.
+static hap_status launch_decode_early(hap_problem *p, const DpOut &out, bool search, cudaStream_t st)
+{
+    bool any = false;
+    for (const auto &cl : p->classes) any |= pass_uses_trie(p, cl, out, false) && (search || !class_outside(p, cl, out));
+    if (!any) return HAP_OK;
+    CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
+    for (const auto &cl : p->classes) {
+        if (!pass_uses_trie(p, cl, out, false) || (!search && class_outside(p, cl, out))) continue;
+        CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_pre, 0));
+        hap_status s = launch_class_decode(p, cl);
+        if (s != HAP_OK) return s;
+        cl.decoded = true;
+    }
+    return HAP_OK;
+}
+
 // One launch per PP class (each has its own block shape); every block clips to the candidate range.
 static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaStream_t st, bool f64 = false)
 {
@@ -964,10 +1114,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     for (const hap_problem::PpClass *clp : order) {
         const hap_problem::PpClass &cl = *clp;
         // skip classes whose candidates all lie outside the range
-        const WorkItem &a = p->items[cl.item_lo], &b = p->items[cl.item_hi - 1];
-        const u64 c0 = p->pconfs[a.p].offset, c1 = p->pconfs[b.p].offset + p->pconfs[b.p].nmap * (u64)p->opts.n_rc;
-        const bool outside = c1 <= out.first || c0 >= out.first + out.count;
-        if (outside && !search) continue;
+        if (!search && class_outside(p, cl, out)) continue;
         const bool lin = p->dc.tau_linear != 0;
         const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
         const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (refine ? 8 : 0) + (search ? 2 : 0) + (lin ? 1 : 0);
@@ -987,9 +1134,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         DpOut o = out;
         o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0;
         if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
-        // plain integer passes over more than one candidate walk the class's prefix tree; tables, refinement,
-        // fp64, cell counting and the one-candidate re-evaluation stay in pipeline_dp_kernel
-        if (cl.trie.ok && !f64 && !out.count_only && !refine && lin && !out.dp_table && !out.choice && out.count > 1) {
+        if (pass_uses_trie(p, cl, out, f64)) {
             const hap_problem::Trie &tr = cl.trie;
             // 64 registers per thread in both shapes (measured: more warps per SM beat more registers per thread)
             const int tv = tr.threads > 512 ? 0 : 1;
@@ -1002,18 +1147,11 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
                 trie_limit[dev][vi] = tr.smem;
             }
             CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
-            // candidate decode of this pass, then its stage bytes into the tree
-            const u64 nmap = p->pconfs[p->items[cl.item_lo].p].nmap;
-            maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, p->items[cl.item_lo].p, nmap, p->d_maptab + cl.map_base);
-            CUDA_TRY(p, cudaGetLastError());
-            for (const auto &pd : tr.parts) {
-                const u32 n_g = pd.n_nodes + pd.n_cells + pd.nmap;
-                TrieRowMap rmap;
-                std::memcpy(rmap.mrow_of, pd.mrow_of, sizeof(rmap.mrow_of));
-                trie_gather_kernel<<<(n_g + 255) / 256, 256, 0, cl.stream>>>(tab, cl.PP, pd.n_nodes, pd.n_cells, pd.nmap, pd.m_lo, pd.d_first_leaf,
-                                                                              pd.d_depth, pd.d_gnode, rmap, pd.d_nodes, pd.d_cells, pd.d_leaves);
-                CUDA_TRY(p, cudaGetLastError());
+            if (!cl.decoded) {                      // not queued ahead of the layer costs by this pass
+                hap_status sd = launch_class_decode(p, cl);
+                if (sd != HAP_OK) return sd;
             }
+            cl.decoded = false;
             int n_parts = (int)tr.parts.size();
             unsigned n_active = tr.n_conf * (unsigned)n_parts;
             const u32 *plist = tr.d_plist;
@@ -1058,13 +1196,14 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     cudaStream_t st = (cudaStream_t)stream;
     CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
     CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
-    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
-    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     DpOut out{};
     out.counters = p->d_counters;
     out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
     out.recompute = dev_recompute; out.dp_table = (i64 *)dev_dp_table; out.choice = dev_choice;
     out.first = first; out.count = count;
+    if ((s = launch_decode_early(p, out, false, st)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
@@ -1074,8 +1213,8 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
 static hap_status ensure_f64_buffers(hap_problem *p)
 {
     const size_t np = p->pconfs.size();
-    if (!p->d_c2f) CUDA_TRY(p, cudaMalloc(&p->d_c2f, np * p->T * p->model.N * 2 * sizeof(double)));
-    if (!p->d_coeff) CUDA_TRY(p, cudaMalloc(&p->d_coeff, np * p->T * HAP_NCOEF * sizeof(double)));
+    if (!p->d_c2f) CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_c2f, np * p->T * p->model.N * 2 * sizeof(double)));
+    if (!p->d_coeff) CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_coeff, np * p->T * HAP_NCOEF * sizeof(double)));
     return HAP_OK;
 }
 
@@ -1115,7 +1254,7 @@ extern "C" hap_status hap_search_range_f64(hap_problem *p, uint64_t first, uint6
     if ((s = check_range(p, first, count)) != HAP_OK) return s;
     if (count == 0) return fail(p, HAP_E_RANGE, "empty candidate range");
     cudaStream_t st = (cudaStream_t)stream;
-    if (!p->d_fcost) CUDA_TRY(p, cudaMalloc(&p->d_fcost, (size_t)p->n_cand * sizeof(i64)));
+    if (!p->d_fcost) CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_fcost, (size_t)p->n_cand * sizeof(i64)));
     if ((s = hap_pipeline_dp_f64(p, first, count, (double *)p->d_fcost, nullptr, nullptr, nullptr, stream)) != HAP_OK) return s;
     // non-negative doubles order like their bit patterns read as int64 (+inf is the largest), so the integer
     // (cost, index) argmin serves the fp64 costs unchanged
@@ -1195,11 +1334,11 @@ static hap_status joint_setup(hap_problem *p)
         arrays.insert(arrays.end(), lvl_off.begin(), lvl_off.end());
         arrays.insert(arrays.end(), st_idx.begin(), st_idx.end());
         arrays.insert(arrays.end(), slot.begin(), slot.end());
-        CUDA_TRY(p, cudaMalloc(&jh.d_arrays, arrays.size() * sizeof(int)));
+        CUDA_TRY(p, cached_malloc(p->device, (void **)&jh.d_arrays, arrays.size() * sizeof(int)));
         CUDA_TRY(p, cudaMemcpy(jh.d_arrays, arrays.data(), arrays.size() * sizeof(int), cudaMemcpyHostToDevice));
         jc.lvl_off = jh.d_arrays; jc.st_idx = jh.d_arrays + (PP + 2); jc.slot = jc.st_idx + S;
         for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == PP) jh.ids.push_back((unsigned)pi);
-        CUDA_TRY(p, cudaMalloc(&jh.d_ids, jh.ids.size() * sizeof(unsigned)));
+        CUDA_TRY(p, cached_malloc(p->device, (void **)&jh.d_ids, jh.ids.size() * sizeof(unsigned)));
         CUDA_TRY(p, cudaMemcpy(jh.d_ids, jh.ids.data(), jh.ids.size() * sizeof(unsigned), cudaMemcpyHostToDevice));
         jh.smem = joint_smem_bytes(N, PP, T, p->prof.R, p->dc.tau_linear != 0);
         if (jh.smem > 227 * 1024) return fail(p, HAP_E_RANGE, "shared memory need of the joint recurrence exceeds the SM");
@@ -1208,7 +1347,7 @@ static hap_status joint_setup(hap_problem *p)
     p->joint_grid = 2 * 148;
     if (lmax_all) {
         const size_t bytes = (size_t)p->joint_grid * 2 * lmax_all * T * (N + 1) * sizeof(i64);
-        CUDA_TRY(p, cudaMalloc(&p->d_joint_scratch, bytes));
+        CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_joint_scratch, bytes));
     }
     p->joint_ready = true;
     return HAP_OK;
@@ -1338,13 +1477,14 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     const u64 init_counters[8] = {0, 0, 0, (u64)kInf, 0, 0, 0, 0};           // [3] = incumbent starts at +INF
     CUDA_TRY(p, cudaMemcpyAsync(p->d_counters, init_counters, sizeof(init_counters), cudaMemcpyHostToDevice, st));
     CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
-    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st, p->d_lb)) != HAP_OK) return s;
-    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     DpOut out{};
     out.lb_sum = p->d_lb;
     out.first = first; out.count = count; out.prune = p->opts.prune;
     out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
     out.incumbent = p->d_counters + 3;
+    if ((s = launch_decode_early(p, out, true, st)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st, p->d_lb)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
     argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best, kInf);
     CUDA_TRY(p, cudaGetLastError());

@@ -223,6 +223,8 @@ template <bool QUANT>
 __global__ void __launch_bounds__(kLcThreads)
 type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u64 *range_flag)
 {
+    // the layer-cost kernel behind this one may start its table reads now (programmatic dependent launch)
+    asm volatile("griddepcontrol.launch_dependents;");
     const int T = dc.T;
     const int role = blockIdx.y;
     const i64 H = dc.H;
@@ -338,21 +340,17 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
     __shared__ i64 s_lb[8];
     const int N = dc.N, T = dc.T;
     const unsigned p = blockIdx.x;
-    {   // stage the configuration's per-type constants (11 doubles each) in shared memory
-        constexpr int W = sizeof(TypeConst) / 8;
-        const double *src = reinterpret_cast<const double *>(tcg + (size_t)p * T);
-        double *dst = reinterpret_cast<double *>(tcs);
-        for (int q = threadIdx.x; q < T * W; q += blockDim.x) dst[q] = src[q];
-    }
-    __syncthreads();
     const int l = threadIdx.x;
-    i64 lmin = 0;                       // min over device types of this layer's forward+backward time
+    const bool dense = l < N && layer_kind(dc, l) == HAP_DENSE;
+    double a[HAP_MAX_TYPES], ab[HAP_MAX_TYPES], f[HAP_MAX_TYPES], fb[HAP_MAX_TYPES];
     if (l < N) {
+        // the profiled table entries depend on the kernel's inputs only: they are requested before the wait for
+        // the per-type constants of the preceding kernel
+        const hap_pconf *pcf = dc.pconf + p;
+        const size_t row = ((size_t)pcf->itp * dc.ncp + pcf->icp) * dc.nmb + pcf->ib;   // the same table row for every type
         const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
-        const bool dense = layer_kind(dc, l) == HAP_DENSE;
-        const size_t i5 = (size_t)tcs[0].row * N + l;                       // the same table row for every type
+        const size_t i5 = row * N + l;
         const double *pa = dc.tdf + i5, *pab = dc.tdb + i5, *pf = dc.tff + i5, *pfb = dc.tfb + i5;
-        double a[HAP_MAX_TYPES], ab[HAP_MAX_TYPES], f[HAP_MAX_TYPES], fb[HAP_MAX_TYPES];
 #pragma unroll
         for (int h = 0; h < HAP_MAX_TYPES; ++h) {
             if (h < T) {
@@ -360,6 +358,19 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
                 f[h] = dense ? 0.0 : __ldg(pf + h * stride_h); fb[h] = dense ? 0.0 : __ldg(pfb + h * stride_h);
             }
         }
+    }
+    // launched as a programmatic dependent of type_const_kernel: everything above overlaps that kernel's tail;
+    // its results are visible after this wait (a no-op in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    {   // stage the configuration's per-type constants (11 doubles each) in shared memory
+        constexpr int W = sizeof(TypeConst) / 8;
+        const double *src = reinterpret_cast<const double *>(tcg + (size_t)p * T);
+        double *dst = reinterpret_cast<double *>(tcs);
+        for (int q = threadIdx.x; q < T * W; q += blockDim.x) dst[q] = src[q];
+    }
+    __syncthreads();
+    i64 lmin = 0;                       // min over device types of this layer's forward+backward time
+    if (l < N) {
         const size_t out0 = ((size_t)p * T * N + l) * 2, out_h = (size_t)N * 2;
         bool bad = false;                                                    // a value left the supported range
         const double kappa = dc.kappa;

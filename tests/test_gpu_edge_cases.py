@@ -187,3 +187,32 @@ def test_uniform_partition_ablation(hap, name):
             for rc in range(n_rc):
                 assert jb[p, rc] == bn[off + rc: off + nmap * n_rc: n_rc].min()
     hap.hap_problem_destroy(hp)
+
+
+def test_device_memory_of_destroyed_problems_is_reused(hap):
+    """Problems created one after another (different sizes in between) give the oracle's plan every time: a
+    recycled, dirty arena must not leak anything of its previous owner into the next problem; releasing the
+    cache returns the memory to the driver."""
+    torch.cuda.synchronize()
+    hap.hap_release_cached_memory()
+    expected = {}
+    for name in ("small", "tiny", "small", "mixtral", "small", "tiny"):
+        pb = problems.make_problem(name)
+        if name not in expected:
+            o = Oracle(pb)
+            done, bc, bi, costs, bn = o.search_pconfs(0, 1, threads=8, want_costs=True)
+            expected[name] = (bc, bi, costs)
+        bc, bi, costs = expected[name]
+        hp = hap.hap_problem_create(pb)
+        hap.hap_enumerate(hp)
+        plan, stats = hap.hap_search_best(hp)
+        assert (plan["T_iter"], plan["index"]) == (bc, bi), name
+        out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+        torch.cuda.synchronize()
+        assert np.array_equal(out["cost"].cpu().numpy(), costs), name
+        hap.hap_problem_destroy(hp)
+    free_cached, _ = torch.cuda.mem_get_info()
+    hap.hap_release_cached_memory()
+    free_released, _ = torch.cuda.mem_get_info()
+    assert free_released > free_cached           # idle blocks went back to the driver
+    hap.hap_release_cached_memory()              # nothing left: a no-op
