@@ -1407,3 +1407,98 @@ int orc_appendix_b(const orc_problem *pr, const orc_pconf *pc, const orc_mapping
     res->T_iter = res->T_edge + res->T_middle + tsync + topt;
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Event simulation of the 1F1B schedule for a GIVEN plan (Sec. 3.3: "the end-to-end iteration
+ * latency under the 1F1B pipeline schedule", which Eq. 4 and Appendix B put in closed form).
+ * Stage i (1-based) runs, strictly in this order: min(PP - i, M) warm-up forward passes, then
+ * forward / backward pairs while forwards remain, then the backward passes that are left.
+ * F(i, m) starts when stage i is free and F(i-1, m) has finished; B(i, m) starts when stage i is
+ * free and B(i+1, m) has finished (on the last stage: when its own F(i, m) has).  A forward pass of
+ * stage i takes t_f,i, a backward pass t_b,i, split as in Appendix B: t_f,i is the forward time of
+ * the stage's layers (slowest member type per layer), t_b,i everything else of the stage cost
+ * (backward time, recomputation at the stage's level, the stage constant with its transfer term), so
+ * transfers take no time of their own.  T_pipe_sim is the time the last backward pass ends,
+ * T_iter = T_pipe_sim + T_sync + T_opt; T_pipe_closed = sum_i c_i + (M-1) max_i c_i is Eq. 4's
+ * pipeline term for the same plan.  Returns 1 and T_iter = ORC_INF when n does not partition the layers.
+ * ------------------------------------------------------------------------------------------ */
+int orc_simulate_1f1b(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                      const int64_t *c2, const int64_t *coef, const uint8_t *n, const uint8_t *r, orc_sim_result *res)
+{
+    const int N = pr->N, PP = pc->PP, M = pc->M;
+    memset(res, 0, sizeof(*res));
+    int total = 0;
+    for (int s = 0; s < PP; ++s) { if (n[s] == 0) total = -100000; total += n[s]; }
+    if (total != N || M < 1) { res->T_iter = ORC_INF; return 1; }
+    int64_t tf[ORC_MAX_PP], tb[ORC_MAX_PP], csum = 0, cmax = 0, tsync = 0, topt = 0;
+    int a = 0;
+    for (int s = 0; s < PP; ++s) {
+        const unsigned mask = mp->mask[s];
+        const int i = s + 1, b = a + n[s];
+        int64_t F = 0, B = 0;
+        for (int l = a; l < b; ++l) {
+            int64_t fl = 0, bl = 0;
+            for (int h = 0; h < pr->T; ++h)
+                if (mask & (1u << h)) {
+                    const int64_t qf = c2[((int64_t)h * N + l) * 2], qb = c2[((int64_t)h * N + l) * 2 + 1];
+                    if (qf > fl) fl = qf;
+                    if (qb > bl) bl = qb;
+                }
+            F += fl; B += bl;
+        }
+        B += ((int64_t)pr->tau_q[r[s]] * F) / 1024;
+        if (i == 1) B += mask_max(pr, mask, coef, ORC_KPRE);
+        if (i == PP) B += mask_max(pr, mask, coef, ORC_KPOST);
+        if (i > 1) {
+            const int hb = mp->hb[s], ha = mp->ha[s];
+            B += coef[hb * ORC_NCOEF + (mp->cls[s] == ORC_CROSS ? ORC_KP2P_CROSS + ha : (mp->cls[s] == ORC_INTER ? ORC_KP2P_INTER : ORC_KP2P_INTRA))];
+        }
+        tf[s] = F; tb[s] = B;
+        csum += F + B;
+        if (F + B > cmax) cmax = F + B;
+        int64_t sy = mask_max(pr, mask, coef, ORC_SLAT), op = 0;
+        for (int l = a; l < b; ++l) {
+            sy += mask_max(pr, mask, coef, ORC_SBW + pr->kind[l]);
+            op += mask_max(pr, mask, coef, ORC_OPT + pr->kind[l]);
+        }
+        if (sy > tsync) tsync = sy;
+        if (op > topt) topt = op;
+        a = b;
+    }
+    /* finish times of every pass; -1: not run yet */
+    int64_t *Fd = (int64_t *)malloc(sizeof(int64_t) * (size_t)PP * M * 2), *Bd = Fd + (size_t)PP * M;
+    if (!Fd) { res->T_iter = ORC_INF; return 1; }
+    for (size_t q = 0; q < (size_t)PP * M * 2; ++q) Fd[q] = -1;
+    int nf[ORC_MAX_PP], nb[ORC_MAX_PP];
+    int64_t t_free[ORC_MAX_PP];
+    for (int s = 0; s < PP; ++s) { nf[s] = nb[s] = 0; t_free[s] = 0; }
+    long remaining = 2L * PP * M;
+    while (remaining > 0) {
+        long before = remaining;
+        for (int s = 0; s < PP; ++s) {
+            const int warm = PP - 1 - s < M ? PP - 1 - s : M;
+            for (;;) {
+                if (nb[s] == M) break;
+                /* the stage's next pass in its fixed order */
+                const int fwd = nf[s] < M && (nf[s] < warm || nf[s] - nb[s] == warm);
+                int64_t dep;
+                if (fwd) dep = s == 0 ? 0 : Fd[(size_t)(s - 1) * M + nf[s]];
+                else dep = s == PP - 1 ? Fd[(size_t)s * M + nb[s]] : Bd[(size_t)(s + 1) * M + nb[s]];
+                if (dep < 0) break;                                        /* its input has not been produced yet */
+                const int64_t start = t_free[s] > dep ? t_free[s] : dep;
+                if (fwd) { t_free[s] = start + tf[s]; Fd[(size_t)s * M + nf[s]] = t_free[s]; nf[s]++; }
+                else { t_free[s] = start + tb[s]; Bd[(size_t)s * M + nb[s]] = t_free[s]; nb[s]++; }
+                remaining--;
+            }
+        }
+        if (remaining == before) { free(Fd); res->T_iter = ORC_INF; return 1; }   /* cannot happen: the schedule has no cycle */
+    }
+    int64_t end = 0;
+    for (int s = 0; s < PP; ++s) if (t_free[s] > end) end = t_free[s];
+    free(Fd);
+    res->T_pipe_sim = end;
+    res->T_pipe_closed = csum + (int64_t)(M - 1) * cmax;
+    res->T_sync = tsync; res->T_opt = topt;
+    res->T_iter = end + tsync + topt;
+    return 0;
+}

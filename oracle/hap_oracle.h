@@ -5,7 +5,7 @@
  * enumeration, the MoE-aware layer cost (Eq. 2, Eq. 3, load-imbalance scaling), the stage
  * memory model with minimal feasible recomputation, the per-candidate min-max pipeline
  * partitioning recurrence, the 1F1B closed-form iteration latency (Eq. 4), the appendix's
- * steady-state expression for given plans and the global argmin (Eq. 1).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+ * steady-state expression and an event simulation of the 1F1B schedule for given plans, and the global argmin (Eq. 1).  Only the tests, the smoke check and the benchmark's CPU-baseline leg may
  * call it.  It shares no code with the CUDA library.
  *
  * Parity status: every function below is pinned by tests that do not go through this file's
@@ -172,5 +172,15 @@ typedef struct {
 } orc_appb_result;
 int orc_appendix_b(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
                    const int64_t *c2, const int64_t *coef, const uint8_t *n, const uint8_t *r, orc_appb_result *res);
+
+/* Event simulation of the 1F1B schedule for a GIVEN plan (the schedule Eq. 4 and Appendix B put in closed form): the
+ * time at which the last backward pass ends when every stage runs its passes in the 1F1B order (min(PP - i, M)
+ * warm-up forwards, forward / backward pairs, remaining backwards), a forward pass of stage i taking t_f,i and a
+ * backward pass t_b,i (split as for orc_appendix_b).  T_pipe_closed is Eq. 4's pipeline term for the same plan. */
+typedef struct {
+    int64_t T_iter, T_pipe_sim, T_pipe_closed, T_sync, T_opt;
+} orc_sim_result;
+int orc_simulate_1f1b(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
+                      const int64_t *c2, const int64_t *coef, const uint8_t *n, const uint8_t *r, orc_sim_result *res);
 
 #endif

@@ -83,6 +83,11 @@ class AppBResult(C.Structure):
                 ("T_opt", C.c_int64), ("s_max", C.c_int32), ("pad", C.c_int32)]
 
 
+class SimResult(C.Structure):
+    _fields_ = [("T_iter", C.c_int64), ("T_pipe_sim", C.c_int64), ("T_pipe_closed", C.c_int64), ("T_sync", C.c_int64),
+                ("T_opt", C.c_int64)]
+
+
 class Plan(C.Structure):
     _fields_ = [("index", C.c_uint64), ("pc", PConf), ("map", Mapping), ("rc_mask", C.c_uint32), ("res", Result)]
 
@@ -228,6 +233,14 @@ class Oracle:
         na = np.zeros(MAX_PP, np.uint8); ra = np.zeros(MAX_PP, np.uint8)
         na[:len(n)] = n; ra[:len(r)] = r
         self.L.orc_appendix_b(C.byref(self.s), self._pc(p), C.byref(mp), _ptr(c2), _ptr(coef), _ptr(na), _ptr(ra), C.byref(res))
+        return res
+
+    def simulate_1f1b(self, p, mp, c2, coef, n, r) -> SimResult:
+        """Event simulation of the 1F1B schedule for a given plan (layers n and recomputation levels r per stage)."""
+        res = SimResult()
+        na = np.zeros(MAX_PP, np.uint8); ra = np.zeros(MAX_PP, np.uint8)
+        na[:len(n)] = n; ra[:len(r)] = r
+        self.L.orc_simulate_1f1b(C.byref(self.s), self._pc(p), C.byref(mp), _ptr(c2), _ptr(coef), _ptr(na), _ptr(ra), C.byref(res))
         return res
 
     def bruteforce(self, p, mp, rc_mask, c2, coef, i, j):

@@ -852,3 +852,118 @@ def test_link_efficiency_table_limits_and_monotonicity():
         assert (c >= a).all() and (cc[:, comm] >= ac[:, comm]).all() and np.array_equal(cc[:, mem], ac[:, mem])
         grew += int((c > a).any())
     assert grew > 0
+
+
+# --------------------------------------------------------------------------------------
+# event simulation of the 1F1B schedule for given plans
+# --------------------------------------------------------------------------------------
+def _longest_path_1f1b(f, b, M):
+    """The same schedule as a precedence graph: a pass ends at its duration plus the latest end among the pass
+    before it on its stage and the pass that produces its input; evaluated by memoised recursion (no event loop)."""
+    import functools
+    import sys
+    PP = len(f)
+    prev_on_stage = {}
+    for s in range(PP):
+        warm = min(PP - s - 1, M)
+        ops = [("F", m) for m in range(warm)]
+        nf, nb = warm, 0
+        while nb < M:
+            if nf < M:
+                ops.append(("F", nf)); nf += 1
+            ops.append(("B", nb)); nb += 1
+        for a, c in zip([None] + ops[:-1], ops):
+            prev_on_stage[(c[0], s, c[1])] = None if a is None else (a[0], s, a[1])
+    sys.setrecursionlimit(max(10000, 8 * PP * M + 1000))
+
+    @functools.lru_cache(maxsize=None)
+    def end(kind, s, m):
+        t = 0
+        p = prev_on_stage[(kind, s, m)]
+        if p is not None:
+            t = max(t, end(*p))
+        if kind == "F" and s > 0:
+            t = max(t, end("F", s - 1, m))
+        if kind == "B":
+            t = max(t, end("B", s + 1, m) if s < PP - 1 else end("F", s, m))
+        return t + (f[s] if kind == "F" else b[s])
+    return max(end("B", s, M - 1) for s in range(PP))
+
+
+def test_1f1b_schedule_worked_examples_and_two_formulations_agree():
+    g = gold("e7_1f1b_schedule.json")
+    for case in g["cases"]:
+        assert _simulate_1f1b(case["f"], case["b"], case["M"]) == case["makespan"], case["name"]
+        assert _longest_path_1f1b(tuple(case["f"]), tuple(case["b"]), case["M"]) == case["makespan"], case["name"]
+        c = [x + y for x, y in zip(case["f"], case["b"])]
+        assert sum(c) + (case["M"] - 1) * max(c) == case["closed_form_sum_plus_M_minus_1_max"]
+    rng = np.random.default_rng(12)
+    for _ in range(60):
+        PP, M = int(rng.integers(1, 9)), int(rng.integers(1, 12))
+        f = tuple(int(x) for x in rng.integers(1, 20, PP)); b = tuple(int(x) for x in rng.integers(1, 40, PP))
+        sim = _simulate_1f1b(list(f), list(b), M)
+        assert sim == _longest_path_1f1b(f, b, M)
+        c = [x + y for x, y in zip(f, b)]
+        # the bottleneck stage alone and one trip through the pipeline bound the makespan from below, running every
+        # pass one after another from above.  Eq. 4's pipeline term is neither: with unequal stages the schedule
+        # can end a little after it (c = (27, 28, 42, 9), M = 8 below) as well as before it.
+        assert max(M * max(c), sum(c)) <= sim <= M * sum(c)
+        if PP == 1:
+            assert sim == M * c[0]
+        if M == 1:
+            assert sim == sum(c)
+    # Eq. 4's pipeline term is not an upper bound of the schedule
+    f, b = (16, 11, 6, 7), (11, 17, 36, 2)
+    assert [x + y for x, y in zip(f, b)] == [27, 28, 42, 9]
+    assert _simulate_1f1b(list(f), list(b), 8) == _longest_path_1f1b(f, b, 8) == 401 > 106 + 7 * 42
+
+
+def test_oracle_1f1b_simulation_hand_example_and_closed_forms():
+    g = gold("e7_1f1b_schedule.json")["oracle_case"]
+    o = Oracle(_uniform_problem(g["N"], (g["PP"],), g["PP"], g["GB"]))
+    c2, _, coef, _ = o.layer_costs(0)
+    r = o.simulate_1f1b(0, o.decode(0, 0), c2, coef, g["n"], [0] * g["PP"])
+    assert (r.T_pipe_sim, r.T_pipe_closed) == (g["T_pipe_sim_ns"], g["T_pipe_closed_ns"])
+    assert r.T_iter == r.T_pipe_sim + r.T_sync + r.T_opt
+    # identical stages: the simulated schedule takes exactly Eq. 4's (M + PP - 1) c
+    for N, PP, GB in ((12, 4, 8), (16, 8, 8), (9, 3, 5), (6, 1, 4), (8, 8, 1)):
+        o = Oracle(_uniform_problem(N, (PP,), PP, GB))
+        c2, _, coef, _ = o.layer_costs(0)
+        r = o.simulate_1f1b(0, o.decode(0, 0), c2, coef, [N // PP] * PP, [0] * PP)
+        c = (N // PP) * 15000
+        assert r.T_pipe_sim == (GB + PP - 1) * c == r.T_pipe_closed
+    # a layer vector that does not cover the N layers is rejected
+    assert o.simulate_1f1b(0, o.decode(0, 0), c2, coef, [2] + [1] * 7, [0] * 8).T_iter == INF
+    assert o.simulate_1f1b(0, o.decode(0, 0), c2, coef, [0] + [1] * 6 + [2], [0] * 8).T_iter == INF
+
+
+def test_oracle_1f1b_simulation_against_the_python_schedule_on_searched_plans():
+    """Plans the search returns for tiny and small (several types per stage, recomputation, transfer constants):
+    the oracle's simulation equals the two Python formulations fed with the plan's own per-stage forward and
+    backward times, respects the bounds that hold for every schedule, and shares T_sync / T_opt with Eq. 4."""
+    checked = 0
+    for pb in (problems.tiny(), problems.small()):
+        o = Oracle(pb)
+        rng = np.random.default_rng(8)
+        for idx in rng.integers(0, o.n_cand, 300).tolist():
+            plan, _, _ = o.eval_index(int(idx))
+            if plan["T_iter"] >= INF or plan["M"] > 64:
+                continue
+            p = o.find_pconf(int(idx))
+            c2, _, coef, _ = o.layer_costs(p)
+            mp = o.decode(p, (int(idx) - int(o.pconfs["offset"][p])) // len(pb.rc_masks))
+            r = o.simulate_1f1b(p, mp, c2, coef, plan["n"], plan["r"])
+            tf, lo = [], 0
+            for st in range(plan["PP"]):
+                types = [h for h in range(pb.T) if plan["mask"][st] >> h & 1]
+                tf.append(sum(max(int(c2[h, l, 0]) for h in types) for l in range(lo, lo + plan["n"][st])))
+                lo += plan["n"][st]
+            tb = [c - x for c, x in zip(plan["c"], tf)]
+            assert all(x >= 0 for x in tb)
+            sim = _simulate_1f1b(tf, tb, plan["M"])
+            assert r.T_pipe_sim == sim == _longest_path_1f1b(tuple(tf), tuple(tb), plan["M"]), idx
+            assert r.T_pipe_closed == plan["T_pipe"] and (r.T_sync, r.T_opt) == (plan["T_sync"], plan["T_opt"])
+            assert max(plan["M"] * max(plan["c"]), sum(plan["c"])) <= r.T_pipe_sim <= plan["M"] * sum(plan["c"])
+            assert r.T_iter == r.T_pipe_sim + r.T_sync + r.T_opt
+            checked += 1
+    assert checked > 80
