@@ -306,6 +306,11 @@ def main():
         torch.cuda.synchronize()
         edge, middle, smax = (int(x) for x in ab["detail"][0].tolist())
         appb = dict(T_iter_closed_form=best[0], T_iter_appendix_b=int(ab["t_iter"][0]), T_edge=edge, T_middle=middle, s_max=smax)
+        # ... and the 1F1B schedule itself run for that plan (context: what the closed form leaves out)
+        sim = hap.hap_simulate_1f1b(hp, best[1], 1, one["partition"], one["recompute"], detail=True)
+        torch.cuda.synchronize()
+        appb["T_iter_simulated_1f1b"] = int(sim["t_iter"][0])
+        appb["T_pipe_simulated_1f1b"], appb["T_pipe_closed_form"] = (int(x) for x in sim["detail"][0].tolist())
 
     # full search through the search entry point (pruning allowed), wall clock call to return
     search_ms, pruned_ms = [], []

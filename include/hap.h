@@ -327,6 +327,21 @@ hap_status hap_get_timings(hap_problem *, float *ms_layer_cost, float *ms_dp, ui
 hap_status hap_eval_appendix_b(hap_problem *, uint64_t first, uint64_t count, const uint8_t *dev_partition,
                                const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream);
 
+/* Sec. 3.3 names the 1F1B schedule; Eq. 4 and Appendix B put its iteration latency in closed form.  This entry
+ * point runs the schedule itself for GIVEN plans, to measure what the closed forms leave out on unequal stages:
+ * stage i of PP runs min(PP - i, M) warm-up forward passes, then forward / backward pairs while forwards remain,
+ * then the remaining backward passes; F(i, m) starts when the stage is free and F(i-1, m) has ended, B(i, m) when
+ * the stage is free and B(i+1, m) has ended (last stage: its own F(i, m)); a forward pass of stage i takes t_f,i,
+ * a backward pass t_b,i (the split of hap_eval_appendix_b, so transfers are part of the passes).
+ * Candidates [first, first+count); dev_partition / dev_recompute: [count][HAP_MAX_PP] as hap_pipeline_dp wrote
+ * them for the same range; dev_t_iter: [count] out, time the last backward pass ends + T_sync + T_opt, HAP_INF
+ * where the layer counts do not partition the N layers; dev_detail: [count][2] out, the simulated pipeline time
+ * and Eq. 4's pipeline term sum_i c_i + (M-1) max_i c_i of the same plan (nullable).  A post-hoc evaluator: one
+ * warp per plan and about 2 (M + PP) rounds each, meant for chosen plans, not for the whole candidate space.
+ * Recomputes the layer costs into library-owned memory first.  Asynchronous on `stream`. */
+hap_status hap_simulate_1f1b(hap_problem *, uint64_t first, uint64_t count, const uint8_t *dev_partition,
+                             const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream);
+
 /* Measurement aid: the number of kernels one hap_pipeline_dp call over the whole candidate space followed by
  * one hap_argmin call launches (layer costs, per PP class the candidate decode and the dynamic program, the
  * reduction).  Host value, no device work. */

@@ -17,7 +17,7 @@ STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE",
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
            "hap_search_range", "hap_search_range_f64",
-           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_release_cached_memory", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_simulate_1f1b", "hap_release_cached_memory", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -356,6 +356,18 @@ def hap_eval_appendix_b(hp: HapProblem, first: int, count: int, partition, recom
     d = torch.empty((count, 3), dtype=torch.int64, device="cuda") if detail else None
     hp.check(load_library().hap_eval_appendix_b(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(partition), _dev(recompute),
                                                 _dev(t), _dev(d), _stream(stream)))
+    return {"t_iter": t, "detail": d}
+
+
+def hap_simulate_1f1b(hp: HapProblem, first: int, count: int, partition, recompute, *, detail=False, stream=None):
+    """Iteration latency of the plans by an event simulation of the 1F1B schedule (partition, recompute as returned
+    by hap_pipeline_dp for the same range).  Returns {"t_iter": [count] int64, "detail": [count][2] (simulated
+    pipeline time, Eq. 4's pipeline term) or None}."""
+    import torch
+    t = torch.empty(count, dtype=torch.int64, device="cuda")
+    d = torch.empty((count, 2), dtype=torch.int64, device="cuda") if detail else None
+    hp.check(load_library().hap_simulate_1f1b(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(partition), _dev(recompute),
+                                              _dev(t), _dev(d), _stream(stream)))
     return {"t_iter": t, "detail": d}
 
 

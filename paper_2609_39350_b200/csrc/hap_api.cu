@@ -1431,6 +1431,23 @@ extern "C" hap_status hap_eval_appendix_b(hap_problem *p, uint64_t first, uint64
     return HAP_OK;
 }
 
+extern "C" hap_status hap_simulate_1f1b(hap_problem *p, uint64_t first, uint64_t count, const uint8_t *dev_partition,
+                                        const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream)
+{
+    hap_status s = enter(p);
+    if (s != HAP_OK) return s;
+    if ((s = check_range(p, first, count)) != HAP_OK) return s;
+    if (count == 0) return HAP_OK;
+    if (!dev_partition || !dev_recompute || !dev_t_iter) return HAP_E_INVALID;
+    if (count > 0x7fffffffull) return fail(p, HAP_E_RANGE, "count too large for one launch");
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    simulate_1f1b_kernel<<<(unsigned)count, 32, 0, st>>>(p->dc, first, count, p->d_c2, p->d_coef, dev_partition, dev_recompute,
+                                                         (i64 *)dev_t_iter, (i64 *)dev_detail);
+    CUDA_TRY(p, cudaGetLastError());
+    return HAP_OK;
+}
+
 extern "C" hap_status hap_launches_per_pass(hap_problem *p, uint32_t *host_count)
 {
     if (!p || !host_count) return HAP_E_INVALID;

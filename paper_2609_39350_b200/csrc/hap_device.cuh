@@ -20,6 +20,7 @@
 //   joint_dp_kernel     recurrence over the device-group state: minimum bottleneck over all
 //                       stage-type sequences of a configuration.
 //   appendix_b_kernel   iteration latency of given plans by the appendix's steady-state expression.
+//   simulate_1f1b_kernel  iteration latency of given plans by an event simulation of the 1F1B schedule.
 //   argmin kernels      lexicographic (cost, index) minimum, block partials then one block.
 #pragma once
 #include <cuda_runtime.h>
@@ -556,6 +557,52 @@ __global__ void decode_kernel(const DevConst dc, u64 first, u64 count, hap_candi
     o->link[lane] = (lane < pc.PP && lane > 0) ? (uint8_t)(sm.cls | (sm.ha << 2) | (sm.hb << 4)) : 0;
 }
 
+// Terms of one stage of a GIVEN plan (layers [a, b) at recomputation level r on the stage's device types): t_f, the
+// forward time of its layers (slowest member type per layer); the stage cost c = t_f + t_b with t_b the backward
+// time, the recomputed forward work and the stage constant (pre / post-processing, the transfer into the stage);
+// the stage's gradient-synchronisation and optimizer times.  `stage` is 0-based.
+__device__ __forceinline__ void plan_stage_terms(const DevConst &dc, u64 p, int PP, const StageMap &sm, int stage, int a, int b, int r,
+                                                 const i64 *__restrict__ c2, const i64 *__restrict__ coef,
+                                                 i64 &tf, i64 &cst, i64 &sy, i64 &op)
+{
+    const int N = dc.N, T = dc.T;
+    const i64 *c2p = c2 + (size_t)p * T * N * 2;
+    const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
+    i64 tb = 0;
+    tf = 0;
+    for (int l = a; l < b; ++l) {
+        i64 F = 0, B = 0;
+        for (int h = 0; h < T; ++h)
+            if (sm.mask >> h & 1) {
+                const i64 qx = c2p[((size_t)h * N + l) * 2], qy = c2p[((size_t)h * N + l) * 2 + 1];
+                F = qx > F ? qx : F;
+                B = qy > B ? qy : B;
+            }
+        tf += F; tb += B;
+    }
+    // coefficients of a stage of several types: the slowest member's
+    i64 kpre = 0, kpost = 0, slat = 0, sbw[2] = {0, 0}, opt[2] = {0, 0};
+    for (int h = 0; h < T; ++h)
+        if (sm.mask >> h & 1) {
+            const i64 *row = cfp + h * HAP_NCOEF;
+            kpre = row[HAP_KPRE] > kpre ? row[HAP_KPRE] : kpre;
+            kpost = row[HAP_KPOST] > kpost ? row[HAP_KPOST] : kpost;
+            slat = row[HAP_SLAT] > slat ? row[HAP_SLAT] : slat;
+            for (int kd = 0; kd < 2; ++kd) {
+                sbw[kd] = row[HAP_SBW + kd] > sbw[kd] ? row[HAP_SBW + kd] : sbw[kd];
+                opt[kd] = row[HAP_OPT + kd] > opt[kd] ? row[HAP_OPT + kd] : opt[kd];
+            }
+        }
+    tb += ((i64)dc.tau_q[r] * tf) >> 10;              // forward work repeated in the backward pass
+    if (stage == 0) tb += kpre;
+    if (stage == PP - 1) tb += kpost;
+    if (stage > 0) tb += cfp[sm.hb * HAP_NCOEF + (sm.cls == HAP_CROSS ? HAP_KP2P_CROSS + sm.ha : HAP_KP2P_INTRA + sm.cls)];
+    cst = tf + tb;
+    const i64 n_moe = (i64)(moe_before(dc, b) - moe_before(dc, a)), n_dense = (i64)(b - a) - n_moe;
+    sy = slat + n_dense * sbw[0] + n_moe * sbw[1];
+    op = n_dense * opt[0] + n_moe * opt[1];
+}
+
 // ------------------------------------------------------------------------------------------
 // Appendix B: iteration latency of GIVEN plans with the steady-state term written through the bottleneck
 // stage's index, T_middle = sum_{i <= s_max} t_f,i + max(0, M - s_max - 1) max_i (t_f,i + t_b,i), T_edge = the
@@ -574,7 +621,7 @@ __global__ void appendix_b_kernel(const DevConst dc, u64 first, u64 count, const
     const u64 c = first + w;
     const u64 p = find_pconf(dc, c);
     const hap_pconf pc = dc.pconf[p];
-    const int PP = pc.PP, N = dc.N, T = dc.T;
+    const int PP = pc.PP, N = dc.N;
     const u64 map_idx = (c - pc.offset) / (u64)dc.n_rc;
     const StageMap sm = decode_stage(dc, pc, map_idx, lane);
     const bool on = lane < PP;
@@ -593,43 +640,7 @@ __global__ void appendix_b_kernel(const DevConst dc, u64 first, u64 count, const
         return;
     }
     i64 tf = 0, cst = 0, sy = 0, op = 0;
-    if (on) {
-        const int a_me = b_me - n_me;
-        const i64 *c2p = c2 + (size_t)p * T * N * 2;
-        const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
-        i64 tb = 0;
-        for (int l = a_me; l < b_me; ++l) {
-            i64 F = 0, B = 0;
-            for (int h = 0; h < T; ++h)
-                if (sm.mask >> h & 1) {
-                    const i64 qx = c2p[((size_t)h * N + l) * 2], qy = c2p[((size_t)h * N + l) * 2 + 1];
-                    F = qx > F ? qx : F;
-                    B = qy > B ? qy : B;
-                }
-            tf += F; tb += B;
-        }
-        // coefficients of a stage of several types: the slowest member's
-        i64 kpre = 0, kpost = 0, slat = 0, sbw[2] = {0, 0}, opt[2] = {0, 0};
-        for (int h = 0; h < T; ++h)
-            if (sm.mask >> h & 1) {
-                const i64 *row = cfp + h * HAP_NCOEF;
-                kpre = row[HAP_KPRE] > kpre ? row[HAP_KPRE] : kpre;
-                kpost = row[HAP_KPOST] > kpost ? row[HAP_KPOST] : kpost;
-                slat = row[HAP_SLAT] > slat ? row[HAP_SLAT] : slat;
-                for (int kd = 0; kd < 2; ++kd) {
-                    sbw[kd] = row[HAP_SBW + kd] > sbw[kd] ? row[HAP_SBW + kd] : sbw[kd];
-                    opt[kd] = row[HAP_OPT + kd] > opt[kd] ? row[HAP_OPT + kd] : opt[kd];
-                }
-            }
-        tb += ((i64)dc.tau_q[r_me] * tf) >> 10;              // forward work repeated in the backward pass
-        if (lane == 0) tb += kpre;
-        if (lane == PP - 1) tb += kpost;
-        if (lane > 0) tb += cfp[sm.hb * HAP_NCOEF + (sm.cls == HAP_CROSS ? HAP_KP2P_CROSS + sm.ha : HAP_KP2P_INTRA + sm.cls)];
-        cst = tf + tb;
-        const i64 n_moe = (i64)(moe_before(dc, b_me) - moe_before(dc, a_me)), n_dense = (i64)n_me - n_moe;
-        sy = slat + n_dense * sbw[0] + n_moe * sbw[1];
-        op = n_dense * opt[0] + n_moe * opt[1];
-    }
+    if (on) plan_stage_terms(dc, p, PP, sm, lane, b_me - n_me, b_me, r_me, c2, coef, tf, cst, sy, op);
     const i64 edge = warp_sum_i64(cst), cmax = warp_max_i64(cst);
     const i64 t_sync = warp_max_i64(sy), t_opt = warp_max_i64(op);
     const unsigned at_max = __ballot_sync(0xffffffffu, on && cst == cmax);
@@ -644,6 +655,96 @@ __global__ void appendix_b_kernel(const DevConst dc, u64 first, u64 count, const
         const i64 middle = f_upto + steady * cmax;
         t_iter[w] = edge + middle + t_sync + t_opt;
         if (detail) { detail[w * 3] = edge; detail[w * 3 + 1] = middle; detail[w * 3 + 2] = s_lane + 1; }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// Event simulation of the 1F1B schedule for GIVEN plans (the schedule whose iteration latency Eq. 4 and Appendix B
+// put in closed form).  Stage i of PP (1-based) runs, in this order, min(PP - i, M) warm-up forward passes, then
+// forward / backward pairs while forwards remain, then the backward passes that are left; F(i, m) starts when the
+// stage is free and F(i-1, m) has ended, B(i, m) when the stage is free and B(i+1, m) has ended (last stage: its
+// own F(i, m)).  A forward pass of stage i takes t_f,i, a backward pass t_b,i = c_i - t_f,i (the split of
+// Appendix B), so transfers are part of the passes.  One warp per candidate, lane = stage: every round each lane runs
+// its next pass if that pass's input exists; end times travel between neighbouring stages through a ring of the
+// last kSimRing passes per stage and direction (a stage is at most PP passes ahead of its consumer).
+// t_iter: [count] simulated pipeline time + T_sync + T_opt; detail: [count][2] simulated pipeline time and Eq. 4's
+// pipeline term sum_i c_i + (M-1) max_i c_i of the same plan (nullable).
+// ------------------------------------------------------------------------------------------
+constexpr int kSimRing = 64;
+
+__global__ void __launch_bounds__(32)
+simulate_1f1b_kernel(const DevConst dc, u64 first, u64 count, const i64 *__restrict__ c2, const i64 *__restrict__ coef,
+                     const uint8_t *__restrict__ partition, const uint8_t *__restrict__ recompute, i64 *t_iter, i64 *detail)
+{
+    __shared__ i64 ringF[HAP_MAX_PP][kSimRing], ringB[HAP_MAX_PP][kSimRing];
+    const u64 w = blockIdx.x;
+    const int lane = threadIdx.x;
+    if (w >= count) return;
+    const u64 c = first + w;
+    const u64 p = find_pconf(dc, c);
+    const hap_pconf pc = dc.pconf[p];
+    const int PP = pc.PP, N = dc.N, M = pc.M;
+    const u64 map_idx = (c - pc.offset) / (u64)dc.n_rc;
+    const StageMap sm = decode_stage(dc, pc, map_idx, lane);
+    const bool on = lane < PP;
+    const int n_me = on ? partition[w * HAP_MAX_PP + lane] : 0;
+    const int r_me = on ? recompute[w * HAP_MAX_PP + lane] : 0;
+    int b_me = n_me;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, b_me, o); if (lane >= o) b_me += t; }
+    const int total = __shfl_sync(0xffffffffu, b_me, PP - 1);
+    const bool ok = total == N && M >= 1 && !__any_sync(0xffffffffu, on && n_me == 0) && !__any_sync(0xffffffffu, on && r_me >= dc.R);
+    if (!ok) {
+        if (lane == 0) {
+            t_iter[w] = kInf;
+            if (detail) { detail[w * 2] = kInf; detail[w * 2 + 1] = kInf; }
+        }
+        return;
+    }
+    i64 tf = 0, cst = 0, sy = 0, op = 0;
+    if (on) plan_stage_terms(dc, p, PP, sm, lane, b_me - n_me, b_me, r_me, c2, coef, tf, cst, sy, op);
+    const i64 tb = cst - tf;
+    const i64 csum = warp_sum_i64(cst), cmax = warp_max_i64(cst);
+    const i64 t_sync = warp_max_i64(sy), t_opt = warp_max_i64(op);
+
+    const int warm = PP - 1 - lane < M ? PP - 1 - lane : M;
+    int nf = 0, nb = 0;                     // forward / backward passes this stage has run
+    i64 t_free = 0;
+    // every round at least one stage runs a pass (the schedule has no cycle); the longest chain of passes is
+    // 2 (M + PP), which bounds the rounds
+    const int max_rounds = 4 * (M + PP) + 16;
+    bool stuck = true;
+    for (int round = 0; round < max_rounds; ++round) {
+        const int nf_prev = __shfl_up_sync(0xffffffffu, nf, 1), nb_next = __shfl_down_sync(0xffffffffu, nb, 1);
+        const bool active = on && nb < M;
+        if (!__any_sync(0xffffffffu, active)) { stuck = false; break; }
+        if (active) {
+            const bool fwd = nf < M && (nf < warm || nf - nb == warm);       // the stage's next pass in its fixed order
+            bool ready;
+            i64 dep = 0;
+            if (fwd) {
+                ready = lane == 0 || nf_prev > nf;
+                if (ready && lane > 0) dep = ringF[lane - 1][nf & (kSimRing - 1)];
+            } else if (lane == PP - 1) {
+                ready = true;                                                 // its own forward pass of the micro-batch came just before
+                dep = ringF[lane][nb & (kSimRing - 1)];
+            } else {
+                ready = nb_next > nb;
+                if (ready) dep = ringB[lane + 1][nb & (kSimRing - 1)];
+            }
+            if (ready) {
+                const i64 start = t_free > dep ? t_free : dep;
+                if (fwd) { t_free = start + tf; ringF[lane][nf & (kSimRing - 1)] = t_free; ++nf; }
+                else { t_free = start + tb; ringB[lane][nb & (kSimRing - 1)] = t_free; ++nb; }
+            }
+        }
+        __syncwarp();
+    }
+    const i64 end = warp_max_i64(on ? t_free : 0);
+    if (lane == 0) {
+        const i64 sim = stuck ? kInf : end;
+        t_iter[w] = stuck ? kInf : end + t_sync + t_opt;
+        if (detail) { detail[w * 2] = sim; detail[w * 2 + 1] = csum + (i64)(M - 1) * cmax; }
     }
 }
 
