@@ -32,7 +32,7 @@ SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of the DP launches of one pass, from the ncu capture summarised
 # in profiles/trie_dp_kernel_stress.md
-NCU_DP_TRAFFIC_BYTES = {"stress": 69.4e6}
+NCU_DP_TRAFFIC_BYTES = {"stress": 54.6e6}
 
 
 def read_peaks():

@@ -1468,8 +1468,14 @@ static hap_status argmin_launch(hap_problem *p, const i64 *dev_cost, uint64_t co
     const unsigned blocks = (unsigned)std::min<uint64_t>((count + 255) / 256, 1024);
     argmin_partial_kernel<<<blocks, 256, 0, st>>>(dev_cost, count, p->d_pcost, p->d_pindex, init);
     CUDA_TRY(p, cudaGetLastError());
-    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, blocks, dev_out, init);
-    CUDA_TRY(p, cudaGetLastError());
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(1); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const i64 *pc = p->d_pcost; const u64 *pi = p->d_pindex; const u64 nb = blocks;
+    CUDA_TRY(p, cudaLaunchKernelEx(&cfg, argmin_final_kernel, pc, pi, nb, dev_out, init));
     return HAP_OK;
 }
 

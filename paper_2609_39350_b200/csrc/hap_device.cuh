@@ -1664,6 +1664,7 @@ argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex, i64 i
 {
     // `init` is the value reported when nothing is smaller: HAP_INF for integer costs, INT64_MAX when the
     // array holds the bit patterns of non-negative doubles (which order like the doubles themselves)
+    asm volatile("griddepcontrol.launch_dependents;");      // the one-block second stage may be brought up meanwhile
     i64 bc = init; u64 bi = ~0ull;
     for (u64 i = (u64)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (u64)gridDim.x * blockDim.x) {
         const i64 v = cost[i];
@@ -1683,6 +1684,9 @@ argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex, i64 i
 __global__ void __launch_bounds__(256)
 argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2, i64 init)
 {
+    // launched as a programmatic dependent of the first stage where it follows one directly: the partials are
+    // complete and visible after this wait (a no-op in an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     i64 bc = init; u64 bi = ~0ull;
     for (u64 i = threadIdx.x; i < n; i += blockDim.x) {
         const i64 v = pcost[i]; const u64 ix = pindex[i];
