@@ -258,6 +258,19 @@ def main():
         if it >= 3:
             lc_alone.append(a.elapsed_time(b))
     lc_alone_ms = statistics.median(lc_alone)
+    # yardstick, not part of the path: a plain fill of the same c2 buffer under the same timing (what a kernel that
+    # does nothing but write these bytes reaches at this size, launch latency included)
+    fill_ms = []
+    for it in range(8):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        c2_buf.zero_()
+        b.record(stream)
+        b.synchronize()
+        if it >= 3:
+            fill_ms.append(a.elapsed_time(b))
+    fill_same_bytes_ms = statistics.median(fill_ms)
     del c2_buf, coef_buf
 
     # joint recurrence over the device state (all stage-type sequences at once), second call timed
@@ -397,6 +410,7 @@ def main():
                                      achieved=lc_gbs, peak=peaks["hbm_gbs"],
                                      unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=None,
                                      bytes_per_launch=16 * units, ms_alone=lc_alone_ms, ms_in_pass=lc_med,
+                                     ms_plain_fill_of_the_same_bytes=fill_same_bytes_ms,
                                      peak_source=f"hbm_gbs ({peak_kind})"),
             wall_s=t_wall,
         )

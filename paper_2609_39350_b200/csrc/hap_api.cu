@@ -329,17 +329,17 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     }
 
     const size_t n4 = (size_t)T * pf->ntp * pf->ncp * pf->nmb, n5 = n4 * N;
+    // device layout: the four per-layer tables interleaved entry by entry (one 32-byte record per (type, row, layer):
+    // the layer-cost kernel reads a record with two 16-byte loads), then tpre, then tpost
     std::vector<double> tables(4 * n5 + 2 * n4);
-    const double *srcs[6] = {pf->tdf, pf->tdb, pf->tff, pf->tfb, pf->tpre, pf->tpost};
-    size_t at = 0;
-    for (int t = 0; t < 6; ++t) {
-        const size_t n = t < 4 ? n5 : n4;
-        std::memcpy(tables.data() + at, srcs[t], n * sizeof(double));
-        at += n;
+    for (size_t i = 0; i < n5; ++i) {
+        double *rec = tables.data() + 4 * i;
+        rec[0] = pf->tdf[i]; rec[1] = pf->tdb[i]; rec[2] = pf->tff[i]; rec[3] = pf->tfb[i];
+        if (rec[0] < rec[2] || rec[1] < rec[3]) return HAP_E_INVALID;                // t_dense includes its FFN
     }
+    std::memcpy(tables.data() + 4 * n5, pf->tpre, n4 * sizeof(double));
+    std::memcpy(tables.data() + 4 * n5 + n4, pf->tpost, n4 * sizeof(double));
     for (double x : tables) if (!(x >= 0.0) || x > 1e15) return HAP_E_INVALID;   // finite, non-negative, < 2^50 ns
-    for (size_t i = 0; i < n5; ++i)                                              // t_dense includes its FFN
-        if (tables[i] < tables[2 * n5 + i] || tables[n5 + i] < tables[3 * n5 + i]) return HAP_E_INVALID;
 
     // ---- device ------------------------------------------------------------------------------
     if (cudaGetDevice(&p->device) != cudaSuccess) return HAP_E_CUDA;
@@ -387,8 +387,8 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     for (int l = 0; l < N; ++l) if (p->kind[l] == HAP_MOE) dc.kindbits[l >> 6] |= 1ull << (l & 63);
     dc.kind_uniform = 1;
     for (int l = 1; l < N; ++l) if (p->kind[l] != p->kind[0]) dc.kind_uniform = 0;
-    dc.tdf = p->d_tables; dc.tdb = dc.tdf + n5; dc.tff = dc.tdb + n5; dc.tfb = dc.tff + n5;
-    dc.tpre = dc.tfb + n5; dc.tpost = dc.tpre + n4;
+    dc.tab4 = p->d_tables;
+    dc.tpre = dc.tab4 + 4 * n5; dc.tpost = dc.tpre + n4;
 
     guard.keep = true;
     *out = p;
@@ -1020,8 +1020,19 @@ static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double 
         cfg.attrs = attr; cfg.numAttrs = 1;
         const TypeConst *tcg = p->d_tc;
         i64 *no_i = nullptr; double *no_d = nullptr;
-        if (quant) CUDA_TRY(p, cudaLaunchKernelEx(&cfg, layer_cost_kernel<true>, p->dc, tcg, c2, no_d, lb_sum, p->d_range));
-        else CUDA_TRY(p, cudaLaunchKernelEx(&cfg, layer_cost_kernel<false>, p->dc, tcg, no_i, c2f, no_i, p->d_range));
+        // layer kinds: 0 all dense, 1 all MoE (uniform branch compiled away), 2 mixed
+        const int kind = !p->dc.kind_uniform ? 2 : (p->kind[0] == HAP_MOE ? 1 : 0);
+        if (quant) {
+            using Fn = void (*)(const DevConst, const TypeConst *, i64 *, double *, i64 *, u64 *);
+            static const Fn fns[3][2] = {{layer_cost_kernel<true, 0, false>, layer_cost_kernel<true, 0, true>},
+                                         {layer_cost_kernel<true, 1, false>, layer_cost_kernel<true, 1, true>},
+                                         {layer_cost_kernel<true, 2, false>, layer_cost_kernel<true, 2, true>}};
+            CUDA_TRY(p, cudaLaunchKernelEx(&cfg, fns[kind][lb_sum ? 1 : 0], p->dc, tcg, c2, no_d, lb_sum, p->d_range));
+        } else {
+            using Fn = void (*)(const DevConst, const TypeConst *, i64 *, double *, i64 *, u64 *);
+            static const Fn fns[3] = {layer_cost_kernel<false, 0, false>, layer_cost_kernel<false, 1, false>, layer_cost_kernel<false, 2, false>};
+            CUDA_TRY(p, cudaLaunchKernelEx(&cfg, fns[kind], p->dc, tcg, no_i, c2f, no_i, p->d_range));
+        }
     }
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;

@@ -58,7 +58,8 @@ struct DevConst {
     unsigned rc_sup[HAP_MAX_RC_MASKS]; // per position in rc_order: earlier positions whose allowed levels are a superset
     int xi_q[HAP_MAX_RC], tau_q[HAP_MAX_RC];
     u64 kindbits[4];                  // bit l set: layer l is an MoE layer
-    const double *tdf, *tdb, *tff, *tfb, *tpre, *tpost;
+    const double *tab4;               // [type][tp][cp][mb][layer] x (t_dense fwd, t_dense bwd, t_ffn fwd, t_ffn bwd), 32-byte records
+    const double *tpre, *tpost;
     const hap_pconf *pconf;           // device copy of the configuration table
     u64 n_pconf;
 };
@@ -176,9 +177,13 @@ __device__ __forceinline__ double collective_ns(const DevConst &dc, const LinkCt
     return lat + xfer_ns(dc, cls, vol, link_bw(lc, cls));
 }
 
-struct TypeConst {      // per (configuration, type) values used by every layer
-    double disp2, imb, den, rden, tr, tr2, commF[2], commB[2];
-    long long row;          // table row (itp, icp, ib) of the configuration
+struct __align__(16) TypeConst {      // per (configuration, type) values used by every layer, in the pairs the layer kernel reads
+    double den, rden;               // expert-term divisor (Eq. 3) and its correctly rounded reciprocal
+    double disp2, imb;              // twice the dispatch time, load-imbalance factor
+    double tr, tr2;                 // router term, forward and backward
+    double commF_moe, commB_moe;    // exposed collective time of an MoE layer, forward and backward
+    double commF_dense, commB_dense;
+    long long row, pad;             // table row (itp, icp, ib) of the configuration
 };
 
 template <bool QUANT>
@@ -266,13 +271,14 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
         const double tcp = collective_ns(dc, lc, CP, (i64)TP * CP, Dkv);
         tc.tr = dc.croute[h] * thb;
         tc.tr2 = 2.0 * tc.tr;
-        tc.commF[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
-        tc.commB[HAP_DENSE] = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
-        tc.commF[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
-        tc.commB[HAP_MOE] = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
+        tc.commF_dense = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * tcp;
+        tc.commB_dense = dc.ovl_tp * (ttpA + ttpD) + dc.ovl_cp * (2.0 * tcp);
+        tc.commF_moe = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * tcp;
+        tc.commB_moe = dc.ovl_tp * (ttpA + ttpM) + dc.ovl_cp * (2.0 * tcp);
         tc.den = (dc.eta[h] * (double)EP) * (double)TPE;
         tc.rden = 1.0 / tc.den;
         tc.row = (pc.itp * dc.ncp + pc.icp) * dc.nmb + pc.ib;
+        tc.pad = 0;
         tcg[p * T + h] = tc;
     } else if (role == 1) {
         const size_t i4 = (((size_t)h * dc.ntp + pc.itp) * dc.ncp + pc.icp) * dc.nmb + pc.ib;
@@ -331,8 +337,10 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
 }
 
 // one block per configuration, one thread per layer; a thread handles its layer for every device type, so
-// that up to 16 table reads are in flight per thread before the first result is needed
-template <bool QUANT>
+// that up to 8 table reads of 16 bytes are in flight per thread before the first result is needed.
+// KIND: 0 every layer dense, 1 every layer MoE (the branch on the layer kind is then uniform and compiled away),
+// 2 mixed.  WANT_LB: also the per-configuration lower bound the search prunes with.
+template <bool QUANT, int KIND, bool WANT_LB>
 __global__ void __launch_bounds__(256)
 layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__restrict__ c2, double *__restrict__ c2f,
                   i64 *__restrict__ lb_sum, u64 *range_flag)
@@ -342,64 +350,71 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
     const int N = dc.N, T = dc.T;
     const unsigned p = blockIdx.x;
     const int l = threadIdx.x;
-    const bool dense = l < N && layer_kind(dc, l) == HAP_DENSE;
-    double a[HAP_MAX_TYPES], ab[HAP_MAX_TYPES], f[HAP_MAX_TYPES], fb[HAP_MAX_TYPES];
+    const bool dense = KIND == 0 || (KIND == 2 && l < N && layer_kind(dc, l) == HAP_DENSE);
+    double2 ta[HAP_MAX_TYPES], tf[HAP_MAX_TYPES];           // (t_dense fwd, bwd), (t_ffn fwd, bwd) of the layer per type
     if (l < N) {
         // the profiled table entries depend on the kernel's inputs only: they are requested before the wait for
         // the per-type constants of the preceding kernel
         const hap_pconf *pcf = dc.pconf + p;
         const size_t row = ((size_t)pcf->itp * dc.ncp + pcf->icp) * dc.nmb + pcf->ib;   // the same table row for every type
-        const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N;      // table stride between device types
-        const size_t i5 = row * N + l;
-        const double *pa = dc.tdf + i5, *pab = dc.tdb + i5, *pf = dc.tff + i5, *pfb = dc.tfb + i5;
+        const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N * 2;                // double2 pairs between device types
+        const double2 *tp = reinterpret_cast<const double2 *>(dc.tab4) + (row * N + l) * 2;
 #pragma unroll
         for (int h = 0; h < HAP_MAX_TYPES; ++h) {
             if (h < T) {
-                a[h] = __ldg(pa + h * stride_h); ab[h] = __ldg(pab + h * stride_h);
-                f[h] = dense ? 0.0 : __ldg(pf + h * stride_h); fb[h] = dense ? 0.0 : __ldg(pfb + h * stride_h);
+                ta[h] = __ldg(tp);
+                if (!dense) tf[h] = __ldg(tp + 1);
+                tp += stride_h;
             }
         }
     }
     // launched as a programmatic dependent of type_const_kernel: everything above overlaps that kernel's tail;
     // its results are visible after this wait (a no-op in an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    {   // stage the configuration's per-type constants (11 doubles each) in shared memory
-        constexpr int W = sizeof(TypeConst) / 8;
-        const double *src = reinterpret_cast<const double *>(tcg + (size_t)p * T);
-        double *dst = reinterpret_cast<double *>(tcs);
+    {   // stage the configuration's per-type constants (12 doubles each) in shared memory
+        constexpr int W = sizeof(TypeConst) / 16;
+        const double2 *src = reinterpret_cast<const double2 *>(tcg + (size_t)p * T);
+        double2 *dst = reinterpret_cast<double2 *>(tcs);
         for (int q = threadIdx.x; q < T * W; q += blockDim.x) dst[q] = src[q];
     }
     __syncthreads();
     i64 lmin = 0;                       // min over device types of this layer's forward+backward time
     if (l < N) {
-        const size_t out0 = ((size_t)p * T * N + l) * 2, out_h = (size_t)N * 2;
         bool bad = false;                                                    // a value left the supported range
         const double kappa = dc.kappa;
+        i64 *o_i = c2 + ((size_t)p * T * N + l) * 2;
+        double *o_d = c2f + ((size_t)p * T * N + l) * 2;
 #pragma unroll
         for (int h = 0; h < HAP_MAX_TYPES; ++h) {
             if (h < T) {
-                const TypeConst &tc = tcs[h];
+                const double2 *tc = reinterpret_cast<const double2 *>(&tcs[h]);
                 double cf, cb;
                 if (dense) {
-                    cf = a[h] + tc.commF[HAP_DENSE];
-                    cb = ab[h] + tc.commB[HAP_DENSE];
+                    const double2 cm = tc[4];                                // commF_dense, commB_dense
+                    cf = ta[h].x + cm.x;
+                    cb = ta[h].y + cm.y;
                 } else {
-                    const double xf = div_by(kappa * f[h], tc.den, tc.rden);
-                    const double mf = (xf + tc.disp2) * tc.imb;
-                    cf = (((a[h] - f[h]) + mf) + tc.tr) + tc.commF[HAP_MOE];
-                    const double xb = div_by(kappa * fb[h], tc.den, tc.rden);
-                    const double mb = (xb + tc.disp2) * tc.imb;
-                    cb = (((ab[h] - fb[h]) + mb) + tc.tr2) + tc.commB[HAP_MOE];
+                    const double2 dn = tc[0], di = tc[1], tr = tc[2], cm = tc[3];
+                    const double xf = div_by(kappa * tf[h].x, dn.x, dn.y);
+                    const double mf = (xf + di.x) * di.y;
+                    cf = (((ta[h].x - tf[h].x) + mf) + tr.x) + cm.x;
+                    const double xb = div_by(kappa * tf[h].y, dn.x, dn.y);
+                    const double mb = (xb + di.x) * di.y;
+                    cb = (((ta[h].y - tf[h].y) + mb) + tr.y) + cm.y;
                 }
                 bad |= !(cf < 6.8719e10) | !(cb < 6.8719e10);                 // 2^36 ns per layer
                 if (QUANT) {
                     longlong2 v; v.x = __double2ll_rn(cf); v.y = __double2ll_rn(cb);
-                    *reinterpret_cast<longlong2 *>(c2 + out0 + h * out_h) = v;
-                    const i64 q = v.x + v.y;
-                    lmin = (h == 0 || q < lmin) ? q : lmin;
+                    *reinterpret_cast<longlong2 *>(o_i) = v;
+                    o_i += (size_t)N * 2;
+                    if (WANT_LB) {
+                        const i64 q = v.x + v.y;
+                        lmin = (h == 0 || q < lmin) ? q : lmin;
+                    }
                 } else {
                     double2 v; v.x = cf; v.y = cb;
-                    *reinterpret_cast<double2 *>(c2f + out0 + h * out_h) = v;
+                    *reinterpret_cast<double2 *>(o_d) = v;
+                    o_d += (size_t)N * 2;
                 }
             }
         }
@@ -407,7 +422,7 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
     }
     // every layer runs on some device type, so the sum over layers of the cheapest type's time bounds the
     // summed stage time of every candidate of this configuration from below (used by the search's pruning)
-    if (QUANT && lb_sum) {
+    if (QUANT && WANT_LB) {
         lmin = warp_sum_i64(lmin);
         if ((threadIdx.x & 31) == 0) s_lb[threadIdx.x >> 5] = lmin;
         __syncthreads();
