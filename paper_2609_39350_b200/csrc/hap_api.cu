@@ -385,8 +385,9 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     dc.tau_linear = 1;
     for (int r = 0; r < pf->R; ++r) { dc.xi_q[r] = p->xi_q[r]; dc.tau_q[r] = p->tau_q[r]; if (p->tau_q[r] % 1024) dc.tau_linear = 0; }
     for (int l = 0; l < N; ++l) if (p->kind[l] == HAP_MOE) dc.kindbits[l >> 6] |= 1ull << (l & 63);
-    dc.kind_uniform = 1;
-    for (int l = 1; l < N; ++l) if (p->kind[l] != p->kind[0]) dc.kind_uniform = 0;
+    dc.kind_uniform_from = N - 1;
+    while (dc.kind_uniform_from > 0 && p->kind[dc.kind_uniform_from - 1] == p->kind[N - 1]) --dc.kind_uniform_from;
+    dc.kind_uniform = dc.kind_uniform_from == 0;
     dc.tab4 = p->d_tables;
     dc.tpre = dc.tab4 + 4 * n5; dc.tpost = dc.tpre + n4;
 
@@ -627,16 +628,6 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
             }
         }
     for (int d = 1; d <= PP; ++d) if (tm.jlo[d] <= tm.jhi[d]) band_max = std::max(band_max, tm.jhi[d] - tm.jlo[d] + 1);
-    const int thr_w = p->dc.kind_uniform ? 1 : band_max;        // one threshold per row when a span's memory depends on its length only
-    tm.thr_w = thr_w;
-    for (u32 c = 0; c < n_cells; ++c) {
-        const u32 g = cell_gnode[c];
-        const int d = depth[g], j = (int)(cells[c].y & 255);
-        cells[c].z = (u32)((((d - 1) * T + capt_of[nodes[g].mask]) * R) * thr_w + (thr_w == 1 ? 0 : j - (int)tm.jlo[d]));
-    }
-    tm.band_max = band_max;
-    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, thr_w, tm.buf_cells[0], tm.buf_cells[1], n_cells, n_nodes);
-    if (smem > limit) return false;
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];
         if (lf.dead || PP == 1) { lf.prowoff = 0; lf.pbl = 0; lf.pbh = 0; continue; }
@@ -649,6 +640,25 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
         const int klo = std::max(N - (int)lf.nmax, (int)lf.pbl), khi = std::min(N - (int)lf.nmin, (int)lf.pbh);
         if (klo <= khi) { tm.kmin[PP] = std::min<uint8_t>(tm.kmin[PP], (uint8_t)klo); tm.kmax[PP] = std::max<uint8_t>(tm.kmax[PP], (uint8_t)khi); }
     }
+    // A depth whose cells only look at splits behind the last change of layer kind sees spans of one kind only:
+    // their memory depends on the length alone and a threshold row of that depth is one number.  All depths of a
+    // model whose layers are all of one kind; every depth but the first few of a model with a dense prefix.
+    bool all_flat = true;
+    for (int d = 1; d <= PP; ++d) {
+        tm.flat[d] = (tm.kmin[d] > tm.kmax[d] || (int)tm.kmin[d] >= p->dc.kind_uniform_from) ? 1 : 0;
+        all_flat = all_flat && tm.flat[d];
+    }
+    tm.all_flat = all_flat ? 1 : 0;
+    const int thr_w = all_flat ? 1 : band_max;
+    tm.thr_w = thr_w;
+    for (u32 c = 0; c < n_cells; ++c) {
+        const u32 g = cell_gnode[c];
+        const int d = depth[g], j = (int)(cells[c].y & 255);
+        cells[c].z = (u32)((((d - 1) * T + capt_of[nodes[g].mask]) * R) * thr_w + ((thr_w == 1 || tm.flat[d]) ? 0 : j - (int)tm.jlo[d]));
+    }
+    tm.band_max = band_max;
+    const size_t smem = trie_smem_bytes(N, PP, T, R, tm.n_mrows, thr_w, tm.buf_cells[0], tm.buf_cells[1], n_cells, n_nodes);
+    if (smem > limit) return false;
     // one blob: nodes | leaves | cells | first_leaf | cell_gnode | parent | depth
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
     part.o_nodes = 0; part.o_leaves = up(part.o_nodes + (size_t)n_nodes * sizeof(TrieNode));

@@ -43,6 +43,7 @@ struct DevConst {
     int S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
     int delta_q, tau_linear, eta_q, uniform;
     int kind_uniform;                 // every layer is of one kind (all MoE or all dense): a span's memory depends on its length only
+    int kind_uniform_from;            // first layer u such that layers u..N-1 are all of one kind (0 when kind_uniform)
     double beta, kappa, chi, gamma, ovl_tp, ovl_cp, ovl_dp, capf;
     double alpha[3];
     double eta[HAP_MAX_TYPES], croute[HAP_MAX_TYPES], copt[HAP_MAX_TYPES];

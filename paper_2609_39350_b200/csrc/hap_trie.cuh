@@ -6,7 +6,7 @@
 // the tree, the band of reachable end layers of every node and the flat list of (node, end layer)
 // cells of every depth depend on the class alone and are built once on the host.
 //
-//   trie_dp_kernel   one block per configuration.  After the block prologue (stage rows, memory
+//   trie_dp_kernel   one block per (configuration, part of the tree).  After the block prologue (stage rows, memory
 //                    thresholds) the block walks the tree depth by depth: one thread per cell
 //                    (node, j) runs the split loop over k against the parent node's row; rows of two
 //                    consecutive depths live in shared memory, split choices of all depths as bytes.
@@ -63,7 +63,10 @@ struct TrieMeta {
     u32 buf_cells[2];               // largest row storage of an even / odd depth, in cells
     u32 nmap, m_lo;                 // the tree covers mappings [m_lo, m_lo + nmap) of the class
     int PP, band_max;               // band_max: most end layers of any depth
-    int thr_w;                      // entries per row of the threshold table: band_max, or 1 when all layers are of one kind
+    int thr_w;                      // entries per row of the threshold table: band_max, or 1 when every depth is flat
+    uint8_t flat[HAP_MAX_PP + 1];   // depth d sees spans of one layer kind only: its threshold rows hold one entry (column 0)
+    uint8_t all_flat;               // every depth is
+    uint8_t pad_flat[2];
 };
 
 constexpr int kTrieKtab = 16 + HAP_MAX_TYPES * 6;    // stage constants: [0,16) pre-work by row group, then p2p [type][6]
@@ -249,13 +252,14 @@ __device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, cons
 // index of the memory threshold of (stage d, capacity type t, level r, end layer j) in the block's table
 __device__ __forceinline__ u32 trie_thr_index(const TrieMeta &tm, int T, int R, int d, int t, int r, int j)
 {
-    return (u32)((((d - 1) * T + t) * R + r) * tm.thr_w + (tm.thr_w == 1 ? 0 : j - (int)tm.jlo[d]));
+    return (u32)((((d - 1) * T + t) * R + r) * tm.thr_w + ((tm.thr_w == 1 || tm.flat[d]) ? 0 : j - (int)tm.jlo[d]));
 }
 
 // Block prologue, part 3: threshold table: for stage d on a device of type t at level r, the length of the longest
 // span ending at layer j that fits (among the splits a cell of depth d can look at; 0: none), only for the end
-// layers, device types and levels that occur at depth d; one entry per row when all layers are of one kind.  Feasibility is monotone in the span, so a thread
-// sweeps the end layers of a row with a split pointer that only moves forward.
+// layers, device types and levels that occur at depth d; one entry per row at the depths whose spans are of one layer
+// kind.  Feasibility is monotone in the span, so for the other depths a thread sweeps the end layers of a row with a
+// split pointer that only moves forward.
 __device__ __forceinline__ void trie_prologue_thr(
     const DevConst &dc, const hap_pconf &pc, const TrieMeta &tm, unsigned p_index, const i64 *coef, unsigned levels,
     const i64 *sW, const i64 *sA, uint8_t *thr, const uint8_t *sK)
@@ -263,28 +267,30 @@ __device__ __forceinline__ void trie_prologue_thr(
     const int T = dc.T, R = dc.R, PP = pc.PP;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
     const i64 mx = cfp[HAP_MX], mpre = cfp[HAP_MPRE], mpost = cfp[HAP_MPOST];
-    if (dc.kind_uniform) {
-        // All layers of one kind: the memory of a span depends on its length alone, so a row is one number, the
-        // longest span that fits (a search over the lengths a window of this depth allows).
-        const int rows = PP * T * R;
+    {
+        // Flat depths (every span a cell of the depth can look at lies behind the last change of layer kind): the
+        // memory of a span depends on its length alone, so a row is one number, the longest span that fits (a
+        // search over the lengths a window of this depth allows, on spans that end at the last layer).
+        const int N = dc.N, rows = PP * T * R;
+        const int len_cap = N - dc.kind_uniform_from;
         for (int q = threadIdx.x; q < rows; q += blockDim.x) {
             const int r = q % R, t = (q / R) % T, d = q / (R * T) + 1;
+            if (!tm.flat[d]) continue;
             int fit = 0;
             if (((levels >> r) & 1u) && ((tm.tmask[d] >> t) & 1u)) {
                 const i64 extra = (d == 1 ? mpre : 0) + (d == PP ? mpost : 0);
                 const int inflight = PP - d + 1;
                 const i64 mstore = pc.M < inflight ? pc.M : inflight;
-                int lo = 0, hi = tm.wmax[d];                 // invariant: lengths <= lo fit (0: trivially), lengths > hi do not
+                int lo = 0, hi = tm.wmax[d] < len_cap ? tm.wmax[d] : len_cap;   // invariant: lengths <= lo fit (0: trivially), lengths > hi do not
                 while (lo < hi) {
                     const int mid = (lo + hi + 1) >> 1;
-                    if (span_fits(sW, sA, sK, extra, mx, mstore, dc.cap_eff[t], dc.xi_q[r], 0, mid)) lo = mid; else hi = mid - 1;
+                    if (span_fits(sW, sA, sK, extra, mx, mstore, dc.cap_eff[t], dc.xi_q[r], N - mid, N)) lo = mid; else hi = mid - 1;
                 }
                 fit = lo;
             }
-            thr[q] = (uint8_t)fit;
+            thr[(size_t)q * tm.thr_w] = (uint8_t)fit;
         }
-        __syncthreads();
-        return;
+        if (tm.all_flat) { __syncthreads(); return; }
     }
     // end layers per thread: a whole row (fewest evaluations: the pointer never restarts) when the rows alone keep
     // half the block busy, segments of eight otherwise
@@ -294,7 +300,7 @@ __device__ __forceinline__ void trie_prologue_thr(
     for (int e = threadIdx.x; e < total; e += blockDim.x) {
         const int seg = e % nseg, q = e / nseg;
         const int r = q % R, t = (q / R) % T, d = q / (R * T) + 1;
-        if (!((levels >> r) & 1u) || !((tm.tmask[d] >> t) & 1u)) continue;
+        if (tm.flat[d] || !((levels >> r) & 1u) || !((tm.tmask[d] >> t) & 1u)) continue;
         const int j0 = tm.jlo[d] + seg * kSeg;
         int j1 = j0 + kSeg - 1; if (j1 > tm.jhi[d]) j1 = tm.jhi[d];
         if (j0 > j1) continue;
