@@ -436,6 +436,15 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             fits |= span_fits(sW, sA, sK, cfp[HAP_MPRE], cfp[HAP_MX], mstore, dc.cap_eff[capt], dc.xi_q[r], 0, nd.bl);
         }
         config_dead = !__syncthreads_or(fits);
+    } else {
+        // a single stage holds all N layers with the pre- and post-processing state: on some type, at some level?
+        int fits = 0;
+        for (int e = tid; e < T * R; e += nthreads) {
+            const int t = e / R, r = e % R;
+            if (!((all_levels >> r) & 1u) || !((tm.tmask[1] >> t) & 1u)) continue;
+            fits |= span_fits(sW, sA, sK, cfp[HAP_MPRE] + cfp[HAP_MPOST], cfp[HAP_MX], pc.M < 1 ? pc.M : 1, dc.cap_eff[t], dc.xi_q[r], 0, N);
+        }
+        config_dead = !__syncthreads_or(fits);
     }
     if (!config_dead) {
         trie_prologue_time_rows(dc, tm, sC, sR);
