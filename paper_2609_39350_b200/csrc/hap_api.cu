@@ -469,6 +469,10 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
     const int delta_q = p->opts.delta_q;
     const bool uniform = (p->opts.flags & HAP_OPT_UNIFORM) != 0;
     std::vector<int> nmin(PP + 1), nmax(PP + 1), bl(PP + 1), bh(PP + 1);
+    // the window of a stage depends on its type mask and on the mapping's summed compute power only: the two
+    // divisions are done once per mask while that sum stays the same (it does for all sequences of a multiset)
+    i64 win_Ps = -1;
+    int win_lo[1 << HAP_MAX_TYPES], win_hi[1 << HAP_MAX_TYPES];
     for (u64 m = 0; m < nmap; ++m) {
         const uint8_t *row = tab + m * (u64)PP * 2;
         i64 Ps = 0;
@@ -477,17 +481,21 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
             if (mk < 1 || mk >= (1 << T)) return false;
             Ps += Pmin[mk];
         }
+        if (!uniform && delta_q >= 0 && Ps != win_Ps) {
+            const i64 den = 1024 * Ps;
+            for (int mk = 1; mk < (1 << T); ++mk) {
+                i64 a = ((i64)(1024 - delta_q) * Pmin[mk] * N) / den;
+                i64 b = ((i64)(1024 + delta_q) * Pmin[mk] * N + den - 1) / den;
+                if (a < 1) a = 1;
+                if (b > N - PP + 1) b = N - PP + 1;
+                win_lo[mk] = (int)a; win_hi[mk] = (int)b;
+            }
+            win_Ps = Ps;
+        }
         for (int s = 1; s <= PP; ++s) {
             int lo = 1, hi = N - PP + 1;
             if (uniform) { lo = N / PP; hi = (N + PP - 1) / PP; }
-            else if (delta_q >= 0) {
-                const i64 Pm = Pmin[row[(s - 1) * 2]], den = 1024 * Ps;
-                i64 a = ((i64)(1024 - delta_q) * Pm * N) / den;
-                i64 b = ((i64)(1024 + delta_q) * Pm * N + den - 1) / den;
-                if (a < 1) a = 1;
-                if (b > N - PP + 1) b = N - PP + 1;
-                lo = (int)a; hi = (int)b;
-            }
+            else if (delta_q >= 0) { lo = win_lo[row[(s - 1) * 2]]; hi = win_hi[row[(s - 1) * 2]]; }
             if (lo < 0 || lo > 255 || hi < 0 || hi > 255) return false;
             nmin[s] = lo; nmax[s] = hi;
         }
@@ -775,6 +783,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         const hap_model &mo = p->model;
         const int N = mo.N, T = p->T;
         std::vector<hap_pconf> rows;
+        rows.reserve(p->pp_list.size() * p->tp_list.size() * p->cp_list.size() * p->ep_list.size() * p->tpe_list.size() * p->mb_list.size() / 4 + 16);
         uint64_t off = 0;
         const uint64_t SAT = 1ull << 62;
         for (int PP : p->pp_list) {
@@ -827,6 +836,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         for (const auto &r : rows) if (std::find(pps.begin(), pps.end(), r.PP) == pps.end()) pps.push_back(r.PP);
         std::sort(pps.begin(), pps.end(), [](int a, int b) { return a > b; });
         std::vector<WorkItem> items;
+        items.reserve(rows.size() * 2);
         std::vector<hap_problem::PpClass> classes;
         u64 tab_bytes = 0;
         for (int PP : pps) {
