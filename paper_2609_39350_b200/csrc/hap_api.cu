@@ -1365,9 +1365,16 @@ static hap_status joint_setup(hap_problem *p)
         arrays.insert(arrays.end(), lvl_off.begin(), lvl_off.end());
         arrays.insert(arrays.end(), st_idx.begin(), st_idx.end());
         arrays.insert(arrays.end(), slot.begin(), slot.end());
+        for (int pos = 0; pos < S; ++pos) {                      // stage counts per type of the states, in level order
+            int dg = 0;
+            for (int h = 0; h < HAP_MAX_TYPES; ++h) dg |= ((st_idx[pos] / jc.stride[h]) % (jc.cnt[h] + 1)) << (8 * h);
+            arrays.push_back(dg);
+        }
+        arrays.insert(arrays.end(), (size_t)S, 0);               // band table, filled by the kernel
         CUDA_TRY(p, cached_malloc(p->device, (void **)&jh.d_arrays, arrays.size() * sizeof(int)));
         CUDA_TRY(p, cudaMemcpy(jh.d_arrays, arrays.data(), arrays.size() * sizeof(int), cudaMemcpyHostToDevice));
         jc.lvl_off = jh.d_arrays; jc.st_idx = jh.d_arrays + (PP + 2); jc.slot = jc.st_idx + S;
+        jc.dig = jc.slot + S; jc.band = jh.d_arrays + (PP + 2) + 3 * (size_t)S;
         for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == PP) jh.ids.push_back((unsigned)pi);
         CUDA_TRY(p, cached_malloc(p->device, (void **)&jh.d_ids, jh.ids.size() * sizeof(unsigned)));
         CUDA_TRY(p, cudaMemcpy(jh.d_ids, jh.ids.data(), jh.ids.size() * sizeof(unsigned), cudaMemcpyHostToDevice));

@@ -1556,6 +1556,8 @@ struct JointClass {
     const int *lvl_off;           // [PP+2] offsets of each level in st_idx
     const int *st_idx;            // [S] state indices ordered by level
     const int *slot;              // [S] rank of a state within its level
+    const int *dig;               // [S] in level order: the state's stage counts per type, one byte each
+    int *band;                    // [S] in level order: reachable end layers of the state, lo | hi << 8 (filled by the kernel)
 };
 
 __host__ __device__ inline size_t joint_smem_bytes(int N, int PP, int T, int R, bool linear)
@@ -1596,20 +1598,42 @@ joint_dp_kernel(const DevConst dc, const unsigned *pconf_ids, unsigned n_ids, co
         __syncthreads();                                  // the previous configuration's tables are no longer read
         dp_block_prologue<VT, LINEAR>(dc, pc, p, c2, coef, coef, true, T, RW, 0xffffffffu, nwarps,
                                       sR, sW, sA, thr, sK, minfo, sP2P, szero, winT);
+        if (w == blockIdx.x) {
+            // End layers a state can have: the stages placed so far and the stages still to place each hold a number
+            // of layers inside their type's window (the same for every configuration of the class); a cell outside
+            // the band is on no complete partition.  Every block fills the whole table with the same values and
+            // reads what it wrote itself.
+            for (int pos = threadIdx.x; pos < jc.S; pos += blockDim.x) {
+                const int dg = jc.dig[pos];
+                int lvl = 0, smin = 0, smax = 0, rmin = 0, rmax = 0;
+                for (int h = 0; h < T; ++h) {
+                    const int uh = (dg >> (8 * h)) & 255, rh = jc.cnt[h] - uh;
+                    lvl += uh;
+                    smin += uh * winT[h][0]; smax += uh * winT[h][1];
+                    rmin += rh * winT[h][0]; rmax += rh * winT[h][1];
+                }
+                int bl = smin > N - rmax ? smin : N - rmax, bh = smax < N - rmin ? smax : N - rmin;
+                if (bl < lvl) bl = lvl;
+                if (bh > N - PP + lvl) bh = N - PP + lvl;
+                if (bl > bh || bl < 0) { bl = 255; bh = 0; }
+                jc.band[pos] = bl | (bh << 8);
+            }
+            __threadfence_block();
+            __syncthreads();
+        }
         for (int rc_idx = 0; rc_idx < n_rc; ++rc_idx) {
             const unsigned rc_mask = dc.rc_masks[rc_idx];
             for (int i = 1; i <= PP; ++i) {
                 i64 *cur = (i & 1) ? buf1 : buf0;
                 const i64 *prv = (i & 1) ? buf0 : buf1;
                 const int l0 = jc.lvl_off[i], l1 = jc.lvl_off[i + 1];
-                const int jlo = i, jhi = N - PP + i;
                 for (int pr = wib; pr < (l1 - l0) * T; pr += nwarps) {
                     const int sl = pr / T, t = pr - sl * T;
-                    const int ui = jc.st_idx[l0 + sl];
-                    const int ut = (ui / jc.stride[t]) % (jc.cnt[t] + 1);
+                    const int dg = jc.dig[l0 + sl];
+                    const int ut = (dg >> (8 * t)) & 255;
                     i64 *row = cur + ((size_t)sl * T + t) * n1;
                     if (ut == 0) continue;                  // no stage of type t placed: rows of such pairs are never read
-                    const int up = ui - jc.stride[t];
+                    const int up = jc.st_idx[l0 + sl] - jc.stride[t];
                     const int slot_up = i > 1 ? jc.slot[up] : 0;
                     const int nmin = winT[t][0], nmax = winT[t][1];
                     const uint8_t *th = thr + ((size_t)(i - 1) * T + t) * R * n1;
@@ -1619,44 +1643,60 @@ joint_dp_kernel(const DevConst dc, const unsigned *pconf_ids, unsigned n_ids, co
                     // the q-th stage of its type starts at device q*G of the type's device line
                     const i64 first = (i64)(ut - 1) * pc.G;
                     const int same_cls = ((first - 1) / dc.node_size[t] == first / dc.node_size[t]) ? HAP_INTRA : HAP_INTER;
-                    for (int j = lane; j <= N; j += 32) {
+                    const int bb = jc.band[l0 + sl];
+                    const int bl = bb & 255, bh = bb >> 8;
+                    // the band of the state before this stage (one stage of type t fewer): its rows hold nothing
+                    // outside it, so the splits are clipped to it
+                    int pbl = 0, pbh = 0;
+                    if (i > 1) {
+                        const int pb = jc.band[jc.lvl_off[i - 1] + slot_up];
+                        pbl = pb & 255; pbh = pb >> 8;
+                    }
+                    // four lanes per end layer, one per type of the stage before (T <= 4); the lane's type is fixed
+                    const int tp = lane & 3;
+                    bool tp_ok = i == 1 ? tp == 0 : tp < T;
+                    const VT *prow = szero;
+                    VT K = Kbase;
+                    if (i > 1 && tp_ok) {
+                        const int utp = ((dg >> (8 * tp)) & 255) - (tp == t ? 1 : 0);
+                        tp_ok = utp != 0;                      // the prefix contains type tp
+                        prow = prv + ((size_t)slot_up * T + tp) * n1;
+                        K += tp != t ? sP2P[t][2 + tp] : sP2P[t][same_cls];
+                    }
+                    const int cells4 = (bh - bl + 1) * 4;
+                    for (int base = 0; base < cells4; base += 32) {
+                        const int idx = base + lane, j = bl + (idx >> 2);
                         VT best = kInf;
-                        if (j >= jlo && j <= jhi) {
-                            int klo = j - nmax; if (klo < i - 1) klo = i - 1;
-                            int khi = j - nmin; if (khi > jhi - 1) khi = jhi - 1;
-                            const int ntp = i == 1 ? 1 : T;
-                            for (int tp = 0; tp < ntp; ++tp) {
-                                const VT *prow = szero;
-                                VT K = Kbase;
-                                int kl = klo, kh = khi;
-                                if (i > 1) {
-                                    const int utp = (up / jc.stride[tp]) % (jc.cnt[tp] + 1);
-                                    if (utp == 0) continue;     // the prefix does not contain type tp
-                                    prow = prv + ((size_t)slot_up * T + tp) * n1;
-                                    K += tp != t ? sP2P[t][2 + tp] : sP2P[t][same_cls];
-                                } else {
-                                    kh = kh < 0 ? kh : 0;       // the first stage starts at layer 0
+                        if (idx < cells4 && tp_ok) {
+                            int kl = j - nmax; if (kl < pbl) kl = pbl;
+                            int kh = j - nmin; if (kh > pbh) kh = pbh;
+                            int seg_hi = kh;
+                            for (int r = 0; r < R && seg_hi >= kl; ++r) {
+                                if (!((rc_mask >> r) & 1u)) continue;
+                                int lo = th[(size_t)r * n1 + j];
+                                if (lo < kl) lo = kl;
+                                if (lo > seg_hi) continue;
+                                const VT Cj = LINEAR ? rM[(size_t)r * n1 + j] + K : 0;
+                                for (int k = seg_hi; k >= lo; --k) {
+                                    VT cst;
+                                    if (LINEAR) cst = Cj - rM[(size_t)r * n1 + k];
+                                    else cst = ((rM[j] - rM[k]) + tau_term((i64)dc.tau_q[r], rM[n1 + j] - rM[n1 + k])) + K;
+                                    const VT pv = prow[k];
+                                    const VT v = pv > cst ? pv : cst;
+                                    best = v < best ? v : best;
+                                    // layer times are non-negative: the stage cost only grows as k falls within
+                                    // a level, so nothing further down this level can beat the best value
+                                    if (cst > best) break;
                                 }
-                                int seg_hi = kh;
-                                for (int r = 0; r < R && seg_hi >= kl; ++r) {
-                                    if (!((rc_mask >> r) & 1u)) continue;
-                                    int lo = th[(size_t)r * n1 + j];
-                                    if (lo < kl) lo = kl;
-                                    if (lo > seg_hi) continue;
-                                    for (int k = seg_hi; k >= lo; --k) {
-                                        VT cst;
-                                        if (LINEAR) cst = (rM[(size_t)r * n1 + j] - rM[(size_t)r * n1 + k]) + K;
-                                        else cst = ((rM[j] - rM[k]) + tau_term((i64)dc.tau_q[r], rM[n1 + j] - rM[n1 + k])) + K;
-                                        const VT pv = prow[k];
-                                        const VT v = pv > cst ? pv : cst;
-                                        best = v < best ? v : best;
-                                    }
-                                    seg_hi = lo - 1;
-                                }
+                                seg_hi = lo - 1;
                             }
                         }
-                        row[j] = best;
+                        VT o = shfl_i64(best, lane ^ 1); best = o < best ? o : best;
+                        o = shfl_i64(best, lane ^ 2); best = o < best ? o : best;
+                        if (idx < cells4 && tp == 0) row[j] = best;
                     }
+                    // the answer is read at (all stages placed, N): make sure that cell exists
+                    if (i == PP && lane == 0 && (N < bl || N > bh)) row[N] = kInf;
                 }
                 __syncthreads();
             }
