@@ -342,6 +342,15 @@ hap_status hap_eval_appendix_b(hap_problem *, uint64_t first, uint64_t count, co
 hap_status hap_simulate_1f1b(hap_problem *, uint64_t first, uint64_t count, const uint8_t *dev_partition,
                              const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream);
 
+/* Self-checking build (no counterpart in the paper).  A library compiled with -DHAP_CHECKED
+ * (paper_2609_39350_b200.build.build_library(checked=True) -> libhap_checked.so) compares the indices and
+ * shared-memory addresses its kernels form from tables (tree records, row origins, threshold indices, output slots,
+ * ring slots of the schedule simulation) with their bounds before use; a violation sets a bit per check site in a
+ * device word and skips the access, so nothing faults.  hap_self_check waits for the current device, returns the
+ * sites that fired since the last call in *host_sites (0: none) and clears the word.  In the normal build the checks
+ * are compiled away and the call returns HAP_E_STATE with *host_sites = 0. */
+hap_status hap_self_check(uint64_t *host_sites);
+
 /* Measurement aid: the number of kernels one hap_pipeline_dp call over the whole candidate space followed by
  * one hap_argmin call launches (layer costs, per PP class the candidate decode and the dynamic program, the
  * reduction).  Host value, no device work. */

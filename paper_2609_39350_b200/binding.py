@@ -7,7 +7,7 @@ from typing import Optional
 
 import numpy as np
 
-from .build import LIB
+from .build import LIB, LIB_CHECKED
 
 MAX_TYPES, MAX_PP, MAX_LAYERS, NCOEF = 4, 32, 255, 20
 INF = 1 << 62
@@ -17,7 +17,7 @@ STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE",
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
            "hap_search_range", "hap_search_range_f64",
-           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_simulate_1f1b", "hap_release_cached_memory", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_simulate_1f1b", "hap_release_cached_memory", "hap_self_check", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -82,9 +82,11 @@ def load_library():
     """Loads libhap.so; raises if it has not been built (there is no fallback)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB):
-            raise HapError(5, f"{LIB} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
-        L = C.CDLL(LIB)
+        # HAP_LIBRARY=checked selects the self-checking build of the same sources (libhap_checked.so)
+        path = LIB_CHECKED if os.environ.get("HAP_LIBRARY") == "checked" else LIB
+        if not os.path.exists(path):
+            raise HapError(5, f"{path} is missing: run __graft_entry__.build() (nvcc, sm_100a) first")
+        L = C.CDLL(path)
         L.hap_status_str.restype = C.c_char_p
         L.hap_last_error.restype = C.c_char_p
         L.hap_last_error.argtypes = [C.c_void_p]
@@ -369,6 +371,16 @@ def hap_simulate_1f1b(hp: HapProblem, first: int, count: int, partition, recompu
     hp.check(load_library().hap_simulate_1f1b(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(partition), _dev(recompute),
                                               _dev(t), _dev(d), _stream(stream)))
     return {"t_iter": t, "detail": d}
+
+
+def hap_self_check() -> int:
+    """Check sites that fired since the last call (bit per site, 0: none); raises HAP_E_STATE unless the loaded
+    library is the self-checking build."""
+    sites = C.c_uint64()
+    st = load_library().hap_self_check(C.byref(sites))
+    if st != 0:
+        raise HapError(st, "hap_self_check")
+    return int(sites.value)
 
 
 def hap_release_cached_memory() -> None:

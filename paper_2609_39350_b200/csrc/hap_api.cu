@@ -1486,6 +1486,22 @@ extern "C" hap_status hap_simulate_1f1b(hap_problem *p, uint64_t first, uint64_t
     return HAP_OK;
 }
 
+extern "C" hap_status hap_self_check(uint64_t *host_sites)
+{
+    if (!host_sites) return HAP_E_INVALID;
+    *host_sites = 0;
+#ifdef HAP_CHECKED
+    if (cudaDeviceSynchronize() != cudaSuccess) return HAP_E_CUDA;
+    unsigned long long sites = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&sites, hap::g_hap_check_sites, sizeof(sites)) != cudaSuccess) return HAP_E_CUDA;
+    if (cudaMemcpyToSymbol(hap::g_hap_check_sites, &zero, sizeof(zero)) != cudaSuccess) return HAP_E_CUDA;
+    *host_sites = sites;
+    return HAP_OK;
+#else
+    return HAP_E_STATE;                     // the checks are compiled away in this build
+#endif
+}
+
 extern "C" hap_status hap_launches_per_pass(hap_problem *p, uint32_t *host_count)
 {
     if (!p || !host_count) return HAP_E_INVALID;

@@ -33,6 +33,21 @@ typedef long long i64;
 typedef unsigned long long u64;
 typedef unsigned int u32;
 
+// Self-checking build (-DHAP_CHECKED): what a memory checker would do from outside, done by the kernels themselves.
+// Indices and shared-memory addresses that a kernel forms from tables (tree records, row origins, threshold
+// indices, output slots) are compared with their bounds before use; a violation sets the site's bit in a device
+// word and the access is skipped: nothing traps, the launch completes, hap_self_check() returns the word.
+// The normal build compiles every check away.
+//   site 0 shared-memory address outside the block's allocation or misaligned    1 row-buffer slot
+//        2 split-choice slot    3 output slot    4 tree node    5 split index read back    6 threshold index
+//        7 configuration index  8 decoded-mapping table    9 ring slot of the schedule simulation
+#ifdef HAP_CHECKED
+__device__ unsigned long long g_hap_check_sites;
+#define HAP_CHECK_OK(site, cond) ((cond) ? true : (atomicOr(&hap::g_hap_check_sites, 1ull << (site)), false))
+#else
+#define HAP_CHECK_OK(site, cond) (true)
+#endif
+
 constexpr int kMaxMasks = (1 << HAP_MAX_TYPES) - 1;
 constexpr int kDpWarps = 12;          // most warps per block of the DP kernel
 constexpr i64 kInf = (i64)1 << 62;
@@ -734,6 +749,12 @@ simulate_1f1b_kernel(const DevConst dc, u64 first, u64 count, const i64 *__restr
         const int nf_prev = __shfl_up_sync(0xffffffffu, nf, 1), nb_next = __shfl_down_sync(0xffffffffu, nb, 1);
         const bool active = on && nb < M;
         if (!__any_sync(0xffffffffu, active)) { stuck = false; break; }
+        {   // a stage is never a whole ring of passes ahead of the neighbour that consumes them
+            const int nf_next = __shfl_down_sync(0xffffffffu, nf, 1), nb_prev = __shfl_up_sync(0xffffffffu, nb, 1);
+            (void)HAP_CHECK_OK(9, !(on && lane + 1 < PP) || nf - nf_next < kSimRing);
+            (void)HAP_CHECK_OK(9, !(on && lane > 0) || nb - nb_prev < kSimRing);
+            (void)nf_next; (void)nb_prev;
+        }
         if (active) {
             const bool fwd = nf < M && (nf < warm || nf - nb == warm);       // the stage's next pass in its fixed order
             bool ready;

@@ -102,7 +102,9 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
         nodes[g].mask = src[0]; nodes[g].link = src[1];
     } else if (g < n_nodes + n_cells) {
         const u32 c = g - n_nodes, nd = cell_gnode[c];
+        if (!HAP_CHECK_OK(8, nd < n_nodes)) return;
         const int d = depth[nd];
+        if (!HAP_CHECK_OK(8, d >= 1 && d < PP)) return;
         const uint8_t *src = maptab + ((u64)first_leaf[nd] * PP + (d - 1)) * 2;
         const int mask = src[0] & 15, link = src[1];
         const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3;
@@ -118,20 +120,35 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
 
 // shared-memory accesses by 32-bit address (the split loop walks two rows with plain address decrements)
 __device__ __forceinline__ u32 smem_u32(const void *p) { return (u32)__cvta_generic_to_shared(p); }
+#ifdef HAP_CHECKED
+__device__ __forceinline__ bool smem_addr_ok(u32 a, u32 bytes)
+{
+    // the dynamic part lies behind the static variables of the kernel: nothing is addressable past its end
+    extern __shared__ __align__(16) unsigned char dyn_smem_base[];
+    u32 dyn;
+    asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn));
+    return HAP_CHECK_OK(0, a % bytes == 0 && a + bytes <= smem_u32(dyn_smem_base) + dyn);
+}
+#else
+__device__ __forceinline__ bool smem_addr_ok(u32, u32) { return true; }
+#endif
 template <int OFF> __device__ __forceinline__ i64 lds_i64(u32 a)
 {
+    if (!smem_addr_ok(a + (u32)OFF, 8)) return 0;
     i64 v;
     asm volatile("ld.shared.b64 %0, [%1+%2];" : "=l"(v) : "r"(a), "n"(OFF));
     return v;
 }
 template <int OFF> __device__ __forceinline__ double lds_f64(u32 a)
 {
+    if (!smem_addr_ok(a + (u32)OFF, 8)) return 0.0;
     double v;
     asm volatile("ld.shared.f64 %0, [%1+%2];" : "=d"(v) : "r"(a), "n"(OFF));
     return v;
 }
 __device__ __forceinline__ int lds_u8(u32 a)
 {
+    if (!smem_addr_ok(a, 1)) return 0;
     u32 v;
     asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a));
     return (int)v;
@@ -357,6 +374,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     }
     __syncthreads();
     const u32 p = plist[blockIdx.x / (unsigned)n_parts];
+    if (!HAP_CHECK_OK(7, (u64)p < dc.n_pconf)) return;
     const hap_pconf pc = dc.pconf[p];
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.thr_w;
     const u64 c_lo = pc.offset + (u64)tm.m_lo * n_rc, c_hi = c_lo + (u64)tm.nmap * n_rc;   // candidates of this block
@@ -522,9 +540,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     const int j = rec.y & 255, klo = (rec.y >> 8) & 255, khi = (rec.y >> 16) & 255;
                     const double K = sKtab[rec.x >> 26];
                     double best; int arg;
+                    (void)HAP_CHECK_OK(6, rec.z + (u32)(R - 1) * (u32)bw < (u32)thr_bytes);
                     cell(a_prevbuf + 8u * (rec.x & 0x03ffffffu), j, klo, khi, a_thr + rec.z, a_sR + 8u * rec.w, K, rc_mask, best, arg);
-                    cur[e] = best;
-                    chd[e] = (uint8_t)arg;
+                    if (HAP_CHECK_OK(1, e < tm.buf_cells[d & 1])) cur[e] = best;
+                    if (HAP_CHECK_OK(2, tm.cell_lo[d] + e < tm.cell_lo[PP])) chd[e] = (uint8_t)arg;
                     alive |= best < dInf;
                 }
                 if (d + 1 < PP && (u32)tid < tm.cell_lo[d + 2] - tm.cell_lo[d + 1]) nxt = __ldcs(tm.cells + tm.cell_lo[d + 1] + tid);
@@ -545,6 +564,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         for (u32 m = tid; m < tm.nmap; m += nthreads) {
             const u64 c = c_lo + (u64)m * n_rc + (u64)rc_idx;
             if (c < w_lo || c >= w_hi) continue;
+            if (!HAP_CHECK_OK(3, c - out.first < out.count)) continue;
             double bott_d = dInf; int arg = 255;
             int mask = 0, link = 0;
             u32 node = 0;
@@ -576,10 +596,13 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 uint4 raw = make_uint4(0, 0, 0, 0);
                 u32 parent = 0;
                 if (d > 1) {
+                    if (!HAP_CHECK_OK(4, node < tm.node_lo[d] - tm.node_lo[d - 1])) break;
                     raw = *reinterpret_cast<const uint4 *>(sNodes + tm.node_lo[d - 1] + node);
                     parent = sParent[tm.node_lo[d - 1] + node];
                 }
+                if (!HAP_CHECK_OK(5, a >= 0 && a < b && b <= N && mask >= 1 && mask <= kMaxMasks)) break;
                 const MaskInfo<i64> &mi = minfo[mask - 1];
+                if (!HAP_CHECK_OK(6, trie_thr_index(tm, T, R, d, mi.capt, 0, b) + (u32)(R - 1) * (u32)bw < (u32)thr_bytes)) break;
                 const uint8_t *th = thr + trie_thr_index(tm, T, R, d, mi.capt, 0, b);
                 int r = 0;
                 for (; r < R; ++r)
@@ -598,6 +621,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 }
                 if (d > 1) {
                     b = a;
+                    if (!HAP_CHECK_OK(2, b >= (int)(raw.w & 255) && raw.x + (u32)(b - (int)(raw.w & 255)) < tm.cell_lo[d] - tm.cell_lo[d - 1])) break;
                     a = ch[tm.cell_lo[d - 1] + raw.x + (u32)(b - (int)(raw.w & 255))];
                     mask = raw.z & 255; link = (raw.z >> 8) & 255;
                     node = parent;
