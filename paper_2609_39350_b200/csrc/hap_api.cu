@@ -1087,7 +1087,8 @@ static bool class_outside(const hap_problem *p, const hap_problem::PpClass &cl, 
 static bool pass_uses_trie(const hap_problem *p, const hap_problem::PpClass &cl, const DpOut &out, bool f64)
 {
     const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
-    return cl.trie.ok && !f64 && !out.count_only && !refine && p->dc.tau_linear != 0 && !out.dp_table && !out.choice && out.count > 1;
+    (void)f64;                                  // both value types walk the tree
+    return cl.trie.ok && !out.count_only && !refine && p->dc.tau_linear != 0 && !out.dp_table && !out.choice && out.count > 1;
 }
 
 // candidate decode of a class for this pass, then its stage bytes into the class's tree
@@ -1169,10 +1170,12 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             const hap_problem::Trie &tr = cl.trie;
             // 64 registers per thread in both shapes (measured: more warps per SM beat more registers per thread)
             const int tv = tr.threads > 512 ? 0 : 1;
-            const void *tfn = search ? (tv == 0 ? (const void *)trie_dp_kernel<true, 1024, 1> : (const void *)trie_dp_kernel<true, 512, 2>)
+            if (search && f64) return fail(p, HAP_E_STATE, "the fp64 search reduces a cost array");
+            const void *tfn = f64 ? (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1, double> : (const void *)trie_dp_kernel<false, 512, 2, double>)
+                            : search ? (tv == 0 ? (const void *)trie_dp_kernel<true, 1024, 1> : (const void *)trie_dp_kernel<true, 512, 2>)
                                      : (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1> : (const void *)trie_dp_kernel<false, 512, 2>);
             static size_t trie_limit[64][6];
-            const int vi = (search ? 3 : 0) + tv;
+            const int vi = (f64 ? 4 : search ? 2 : 0) + tv;
             if (tr.smem > trie_limit[dev][vi]) {
                 CUDA_TRY(p, cudaFuncSetAttribute(tfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tr.smem));
                 trie_limit[dev][vi] = tr.smem;
@@ -1187,7 +1190,8 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             unsigned n_active = tr.n_conf * (unsigned)n_parts;
             const u32 *plist = tr.d_plist;
             const TrieMeta *metas = tr.d_metas;
-            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&p->d_c2, (void *)&p->d_coef, (void *)&metas, (void *)&n_parts, (void *)&o};
+            void *c2v = f64 ? (void *)p->d_c2f : (void *)p->d_c2, *coefv = f64 ? (void *)p->d_coeff : (void *)p->d_coef;
+            void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&c2v, (void *)&p->d_coef, (void *)&coefv, (void *)&metas, (void *)&n_parts, (void *)&o};
             const unsigned tblocks = search ? std::max(blocks, n_active) : n_active;       // search: every partial slot of the class is written
             CUDA_TRY(p, cudaLaunchKernel(tfn, dim3(tblocks), dim3(tr.threads), targs, tr.smem, cl.stream));
             CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));

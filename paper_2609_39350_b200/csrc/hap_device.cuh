@@ -10,7 +10,7 @@
 //   maptab_kernel       the same for every mapping of one PP class (every pass).
 //   trie_dp_kernel      (hap_trie.cuh) the default dynamic program: all mappings of a configuration
 //                       together through the prefix tree of their stage sequences.
-//   pipeline_dp_kernel  the general form (DP tables on request, refinement / exact modes, fp64 mode, classes
+//   pipeline_dp_kernel  the general form (DP tables on request, refinement / exact modes, classes
 //                       without a tree): one warp per candidate, stage rows and memory-threshold tables in shared
 //                       memory (built once per block for the block's configuration), min-max
 //                       recurrence with lanes over the end layer j, optional refinement pass,

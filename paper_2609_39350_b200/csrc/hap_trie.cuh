@@ -12,8 +12,8 @@
 //                    consecutive depths live in shared memory, split choices of all depths as bytes.
 //                    Then one thread per mapping evaluates the last stage's single cell (PP, N), walks
 //                    the split choices back through the node's ancestors and assembles Eq. 4.
-//                    Integer mode with level-combined rows only; every other mode runs in
-//                    pipeline_dp_kernel.
+//                    Integer and fp64 mode, level-combined rows only (recomputation factors that are
+//                    multiples of 1024); DP tables and the refinement modes run in pipeline_dp_kernel.
 #pragma once
 #include "hap_device.cuh"
 
@@ -157,15 +157,17 @@ __device__ __forceinline__ int lds_u8(u32 a)
 // Block prologue, part 1: layer times of the configuration staged in shared memory, the weight and activation
 // byte prefixes, MoE prefix counts, per-mask stage info, p2p coefficients, the table of stage constants and a
 // copy of the tree's node records: what decides whether any mapping of the configuration can be feasible.
+template <typename VT>
 __device__ __forceinline__ void trie_prologue_rows(
-    const DevConst &dc, const TrieMeta &tm, unsigned p_index, const i64 *c2, const i64 *coef,
-    i64 *sC, i64 *sW, i64 *sA, uint8_t *sK, double *sKtab, TrieNode *sNodes, uint16_t *sParent,
-    MaskInfo<i64> *minfo, i64 (*sP2P)[6], double *szero)
+    const DevConst &dc, const TrieMeta &tm, unsigned p_index, const VT *c2, const i64 *coef, const VT *coefv,
+    VT *sC, i64 *sW, i64 *sA, uint8_t *sK, double *sKtab, TrieNode *sNodes, uint16_t *sParent,
+    MaskInfo<VT> *minfo, VT (*sP2P)[6], double *szero)
 {
     const int N = dc.N, T = dc.T;
     const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, wib = tid >> 5, lane = tid & 31;
     const int nmask = (1 << T) - 1;
-    const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;
+    const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;         // byte coefficients: integers in both modes
+    const VT *cvp = coefv + (size_t)p_index * T * HAP_NCOEF;         // time coefficients
     {
         const longlong2 *src = reinterpret_cast<const longlong2 *>(c2 + (size_t)p_index * T * N * 2);
         longlong2 *dst = reinterpret_cast<longlong2 *>(sC);
@@ -174,13 +176,13 @@ __device__ __forceinline__ void trie_prologue_rows(
     for (int l = tid; l <= N; l += nthreads) sK[l] = (uint8_t)moe_before(dc, l);
     if (tid < nmask) {
         const int mk = tid + 1;
-        MaskInfo<i64> mi;
+        MaskInfo<VT> mi;
         mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
         i64 cap = 0;
         bool seen = false;
         for (int h = 0; h < T; ++h)
             if (mk >> h & 1) {
-                const i64 *row = cfp + h * HAP_NCOEF;
+                const VT *row = cvp + h * HAP_NCOEF;
                 if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; mi.capt = h; }
                 if (!seen || dc.P[h] < mi.Pmin) mi.Pmin = dc.P[h];
                 if (!seen || row[HAP_KPRE] > mi.kpre) mi.kpre = row[HAP_KPRE];
@@ -197,7 +199,7 @@ __device__ __forceinline__ void trie_prologue_rows(
     }
     if (tid >= 32 && tid < 32 + T * 6) {
         const int q = tid - 32, h = q / 6, e = q % 6;
-        const i64 v = cfp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];      // intra, inter, cross[0..3] are consecutive columns
+        const VT v = cvp[h * HAP_NCOEF + HAP_KP2P_INTRA + e];       // intra, inter, cross[0..3] are consecutive columns
         sP2P[h][e] = v;
         sKtab[16 + q] = (double)v;
     }
@@ -233,21 +235,22 @@ __device__ __forceinline__ void trie_prologue_rows(
 // Block prologue, part 2 (configurations that can be feasible): per type mask that occurs in the class the prefix
 // rows of the stage time at every recomputation level, fwd+bwd + (tau_r/1024) fwd; one warp per mask, inclusive
 // warp scans over chunks of 32 layers.  No barrier: the threshold sweep that follows ends with one.
-__device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, const TrieMeta &tm, const i64 *sC, double *sR)
+template <typename VT>
+__device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, const TrieMeta &tm, const VT *sC, double *sR)
 {
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int nwarps = blockDim.x >> 5, wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int mr = wib; mr < tm.n_mrows; mr += nwarps) {
         const int mk = tm.mask_of_row[mr];
-        i64 runA = 0, runB = 0;
+        VT runA = 0, runB = 0;
         for (int base = 0; base < N; base += 32) {
             const int l = base + lane;
-            i64 vA = 0, vB = 0;                                      // fwd+bwd, fwd
+            VT vA = 0, vB = 0;                                       // fwd+bwd, fwd
             if (l < N) {
-                i64 F = 0, B = 0;
+                VT F = 0, B = 0;
                 for (int h = 0; h < T; ++h)
                     if (mk >> h & 1) {
-                        const i64 qx = sC[((size_t)h * N + l) * 2], qy = sC[((size_t)h * N + l) * 2 + 1];
+                        const VT qx = sC[((size_t)h * N + l) * 2], qy = sC[((size_t)h * N + l) * 2 + 1];
                         F = qx > F ? qx : F;
                         B = qy > B ? qy : B;
                     }
@@ -255,12 +258,12 @@ __device__ __forceinline__ void trie_prologue_time_rows(const DevConst &dc, cons
             }
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const i64 tA = __shfl_up_sync(0xffffffffu, vA, o), tB = __shfl_up_sync(0xffffffffu, vB, o);
+                const VT tA = __shfl_up_sync(0xffffffffu, vA, o), tB = __shfl_up_sync(0xffffffffu, vB, o);
                 if (lane >= o) { vA += tA; vB += tB; }
             }
             vA += runA; vB += runB;
-            if (l < N) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = (double)(vA + (i64)(dc.tau_q[r] >> 10) * vB);
-            runA = shfl_i64(vA, 31); runB = shfl_i64(vB, 31);
+            if (l < N) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1 + l + 1] = (double)(vA + (VT)(dc.tau_q[r] >> 10) * vB);
+            runA = shfl_v(vA, 31); runB = shfl_v(vB, 31);
         }
         if (lane == 0) for (int r = 0; r < R; ++r) sR[((size_t)mr * R + r) * n1] = 0.0;
     }
@@ -347,14 +350,21 @@ __device__ __forceinline__ void trie_prologue_thr(
     __syncthreads();
 }
 
-template <bool SEARCH, int MAXT, int MINB>
+template <typename T> struct IsF64 { static constexpr bool value = false; };
+template <> struct IsF64<double> { static constexpr bool value = true; };
+
+// VT: i64 (times rounded to integer ns: every operation below is exact) or double (fp64 mode: unrounded times,
+// the same steps in floating point; not instantiated for SEARCH).
+template <bool SEARCH, int MAXT, int MINB, typename VT = i64>
 __global__ void __launch_bounds__(MAXT, MINB)
-trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64 *c2, const i64 *coef,
+trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT *c2, const i64 *coef, const VT *coefv,
                const TrieMeta *metas, int n_parts, DpOut out)
 {
+    constexpr bool F64 = IsF64<VT>::value;
+    static_assert(!(SEARCH && F64), "the fp64 search reduces a cost array; the tree kernel only fills it");
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    __shared__ MaskInfo<i64> minfo[kMaxMasks];
-    __shared__ i64 sP2P[HAP_MAX_TYPES][6];
+    __shared__ MaskInfo<VT> minfo[kMaxMasks];
+    __shared__ VT sP2P[HAP_MAX_TYPES][6];
     __shared__ double szero[1];
     __shared__ i64 wcost[32];
     __shared__ u64 widx[32];
@@ -410,7 +420,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     uint8_t *thr = smem_raw + thr_off;
     const size_t thr_bytes = ((size_t)PP * T * R * bw + 15) / 16 * 16;
     uint8_t *sK = thr + thr_bytes;
-    i64 *sC = reinterpret_cast<i64 *>(sK + ((size_t)n1 + 15) / 16 * 16);      // [T][N][2], 16-byte aligned
+    VT *sC = reinterpret_cast<VT *>(sK + ((size_t)n1 + 15) / 16 * 16);        // [T][N][2], 16-byte aligned
     double *sKtab = reinterpret_cast<double *>(sC + (size_t)T * N * 2);
     double *bufE = sKtab + kTrieKtab;
     double *bufO = bufE + tm.buf_cells[0];
@@ -418,15 +428,16 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
     TrieNode *sNodes = reinterpret_cast<TrieNode *>(ch + ((size_t)tm.cell_lo[PP] + 15) / 16 * 16);
     uint16_t *sParent = reinterpret_cast<uint16_t *>(sNodes + tm.node_lo[PP]);
 
-    trie_prologue_rows(dc, tm, p, c2, coef, sC, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
+    trie_prologue_rows<VT>(dc, tm, p, c2, coef, coefv, sC, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
     const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
 
     // writes "infeasible" for candidate c (non-search mode)
+    const VT vInf = ValInf<VT>::get();
     auto put_infeasible = [&](u64 c) {
         const u64 o = c - out.first;
-        if (out.cost) out.cost[o] = kInf;
-        if (out.bottleneck) out.bottleneck[o] = kInf;
-        if (out.detail) { out.detail[o * 3] = kInf; out.detail[o * 3 + 1] = 0; out.detail[o * 3 + 2] = 0; }
+        if (out.cost) reinterpret_cast<VT *>(out.cost)[o] = vInf;
+        if (out.bottleneck) reinterpret_cast<VT *>(out.bottleneck)[o] = vInf;
+        if (out.detail) { VT *dt = reinterpret_cast<VT *>(out.detail); dt[o * 3] = vInf; dt[o * 3 + 1] = 0; dt[o * 3 + 2] = 0; }
         if (out.partition) for (int s = 0; s < HAP_MAX_PP; ++s) out.partition[o * HAP_MAX_PP + s] = 0;
         if (out.recompute) for (int s = 0; s < HAP_MAX_PP; ++s) out.recompute[o * HAP_MAX_PP + s] = 0;
     };
@@ -465,7 +476,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
         config_dead = !__syncthreads_or(fits);
     }
     if (!config_dead) {
-        trie_prologue_time_rows(dc, tm, sC, sR);
+        trie_prologue_time_rows<VT>(dc, tm, sC, sR);
         trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
     }
 
@@ -490,18 +501,22 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             if (lo > seg_hi) continue;
             const int n = seg_hi - lo + 1;
             n_cells32 += (u32)n;
-            const double Cj = lds_f64<0>(a_row + 8u * (u32)j) + K;
+            // integer mode: (row[j] + K) - row[k], exact in any order; fp64 mode keeps the order (row[j] - row[k]) + K
+            const double Rj = lds_f64<0>(a_row + 8u * (u32)j);
+            const double Cj = F64 ? Rj : Rj + K;
+            const double Kadd = F64 ? K : 0.0;
             u32 pa = a_prev + 8u * (u32)seg_hi, ra = a_row + 8u * (u32)seg_hi;
             const u32 pa_lo = a_prev + 8u * (u32)lo;
             if (n & 1) {
-                const double p0 = lds_f64<0>(pa), c0 = Cj - lds_f64<0>(ra);
+                const double p0 = lds_f64<0>(pa), c0 = F64 ? (Cj - lds_f64<0>(ra)) + Kadd : Cj - lds_f64<0>(ra);
                 const double v0 = p0 > c0 ? p0 : c0;
                 if (v0 <= best) { best = v0; a_arg = pa; }
                 pa -= 8; ra -= 8;
             }
             while ((int)(pa - pa_lo) > 0) {      // pa and pa - 8 are both inside the segment
                 const double p0 = lds_f64<0>(pa), p1 = lds_f64<-8>(pa);
-                const double c0 = Cj - lds_f64<0>(ra), c1 = Cj - lds_f64<-8>(ra);
+                const double c0 = F64 ? (Cj - lds_f64<0>(ra)) + Kadd : Cj - lds_f64<0>(ra);
+                const double c1 = F64 ? (Cj - lds_f64<-8>(ra)) + Kadd : Cj - lds_f64<-8>(ra);
                 const double v0 = p0 > c0 ? p0 : c0, v1 = p1 > c1 ? p1 : c1;
                 if (v0 <= best) { best = v0; a_arg = pa; }
                 if (v1 <= best) { best = v1; a_arg = pa - 8; }
@@ -551,9 +566,9 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
             }
         }
         // ---- one thread per mapping: cell (PP, N), backtrace, Eq. 4 ---------------------------------
-        auto stage_K = [&](int d, int mask, int link) -> i64 {
-            i64 K = 0;
-            const MaskInfo<i64> &mi = minfo[mask - 1];
+        auto stage_K = [&](int d, int mask, int link) -> VT {
+            VT K = 0;
+            const MaskInfo<VT> &mi = minfo[mask - 1];
             if (d == 1) K += mi.kpre;
             if (d == PP) K += mi.kpost;
             if (d > 1) { const int cls = link & 3, ha = (link >> 2) & 3, hb = (link >> 4) & 3; K += sP2P[hb][cls == HAP_CROSS ? 2 + ha : cls]; }
@@ -582,13 +597,13 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                 }
             }
             if (SEARCH) n_eval++;
-            const i64 bott = bott_d < dInf ? (i64)bott_d : kInf;
-            if (!(bott < kInf)) {
+            const VT bott = bott_d < dInf ? (VT)bott_d : vInf;
+            if (!(bott < vInf)) {
                 if (!SEARCH) put_infeasible(c);
                 continue;
             }
             // backtrace from (PP, N) through the ancestors; per stage: level, cost, sync and optimizer terms
-            i64 sum = 0, mxc = 0, t_sync = 0, t_opt = 0, het = 0;
+            VT sum = 0, mxc = 0, t_sync = 0, t_opt = 0, het = 0;
             const u64 o = c - out.first;
             int b = N, a = arg;
             for (int d = PP; d >= 1; --d) {
@@ -601,18 +616,18 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     parent = sParent[tm.node_lo[d - 1] + node];
                 }
                 if (!HAP_CHECK_OK(5, a >= 0 && a < b && b <= N && mask >= 1 && mask <= kMaxMasks)) break;
-                const MaskInfo<i64> &mi = minfo[mask - 1];
+                const MaskInfo<VT> &mi = minfo[mask - 1];
                 if (!HAP_CHECK_OK(6, trie_thr_index(tm, T, R, d, mi.capt, 0, b) + (u32)(R - 1) * (u32)bw < (u32)thr_bytes)) break;
                 const uint8_t *th = thr + trie_thr_index(tm, T, R, d, mi.capt, 0, b);
                 int r = 0;
                 for (; r < R; ++r)
                     if (((rc_mask >> r) & 1u) && b - (int)th[r * bw] <= a) break;
                 const double *rr = sR + ((size_t)tm.mrow_of[mask] * R + r) * n1;
-                const i64 cst = (i64)(rr[b] - rr[a]) + stage_K(d, mask, link);
+                const VT cst = (VT)(rr[b] - rr[a]) + stage_K(d, mask, link);
                 sum += cst; mxc = cst > mxc ? cst : mxc;
-                const i64 n_moe = (i64)((int)sK[b] - (int)sK[a]), n_dense = (i64)(b - a) - n_moe;
-                const i64 sy = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
-                const i64 op = n_dense * mi.opt[0] + n_moe * mi.opt[1];
+                const VT n_moe = (VT)((int)sK[b] - (int)sK[a]), n_dense = (VT)(b - a) - n_moe;
+                const VT sy = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
+                const VT op = n_dense * mi.opt[0] + n_moe * mi.opt[1];
                 t_sync = sy > t_sync ? sy : t_sync; t_opt = op > t_opt ? op : t_opt;
                 if (dc.eta_q > 0 && d > 1 && (link & 3) == HAP_CROSS) het += sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
                 if (!SEARCH) {
@@ -627,18 +642,18 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const i64
                     node = parent;
                 }
             }
-            i64 T_pipe = sum + (i64)(pc.M - 1) * mxc;
-            i64 T_iter = T_pipe + t_sync + t_opt;
-            if (dc.eta_q > 0 && het * (i64)PP * 1024 > (i64)dc.eta_q * sum) { T_iter = kInf; T_pipe = kInf; }   // Pruning 3
+            VT T_pipe = sum + (VT)(pc.M - 1) * mxc;
+            VT T_iter = T_pipe + t_sync + t_opt;
+            if (dc.eta_q > 0 && het * (VT)PP * (VT)1024 > (VT)dc.eta_q * sum) { T_iter = vInf; T_pipe = vInf; }   // Pruning 3
             if (SEARCH) {
-                if (T_iter < kInf) { n_feas++; any_plan = 1; }
-                if (T_iter < best_cost || (T_iter == best_cost && c < best_index)) { best_cost = T_iter; best_index = c; }
+                if (T_iter < vInf) { n_feas++; any_plan = 1; }
+                if ((i64)T_iter < best_cost || ((i64)T_iter == best_cost && c < best_index)) { best_cost = (i64)T_iter; best_index = c; }
             } else {
                 any_plan = 1;
-                if (out.cost) out.cost[o] = T_iter;
-                if (out.bottleneck) out.bottleneck[o] = bott;
-                if (out.detail) { out.detail[o * 3] = T_pipe; out.detail[o * 3 + 1] = t_sync; out.detail[o * 3 + 2] = t_opt; }
-                if (!(T_iter < kInf)) {
+                if (out.cost) reinterpret_cast<VT *>(out.cost)[o] = T_iter;
+                if (out.bottleneck) reinterpret_cast<VT *>(out.bottleneck)[o] = bott;
+                if (out.detail) { VT *dt = reinterpret_cast<VT *>(out.detail); dt[o * 3] = T_pipe; dt[o * 3 + 1] = t_sync; dt[o * 3 + 2] = t_opt; }
+                if (!(T_iter < vInf)) {
                     if (out.partition) for (int s = 0; s < PP; ++s) out.partition[o * HAP_MAX_PP + s] = 0;
                     if (out.recompute) for (int s = 0; s < PP; ++s) out.recompute[o * HAP_MAX_PP + s] = 0;
                 }
