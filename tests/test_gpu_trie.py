@@ -189,3 +189,28 @@ def test_many_random_problems_agree_between_the_two_kernels(hap):
         hap.hap_problem_destroy(hp_t)
         hap.hap_problem_destroy(hp_w)
     assert n_checked > 20000
+
+
+@pytest.mark.parametrize("name", ["tiny", "small", "dsv2"])
+def test_fp64_mode_agrees_between_the_two_kernels(hap, name):
+    """fp64 mode: the tree kernel and the one-warp-per-candidate kernel follow the same steps up to the order of a
+    few additions (stage constants, the sum over the stages of a plan); feasibility agrees exactly, costs and
+    bottlenecks to rounding, partitions except where two splits tie to the last bits."""
+    pb = problems.make_problem(name)
+    res = {}
+    for flags in (0, hap.OPT_NO_TRIE):
+        hp = hap.hap_problem_create(pb, flags=flags)
+        hap.hap_enumerate(hp)
+        out = hap.hap_pipeline_dp_f64(hp, 0, hp.n_cand, partition=True)
+        torch.cuda.synchronize()
+        res[flags] = {k: v.cpu().numpy() for k, v in out.items()}
+        hap.hap_problem_destroy(hp)
+    a, b = res[0], res[hap.OPT_NO_TRIE]
+    fin = np.isfinite(a["cost"])
+    assert np.array_equal(fin, np.isfinite(b["cost"])) and fin.any()
+    assert np.allclose(a["bottleneck"][fin], b["bottleneck"][fin], rtol=1e-13, atol=0.0)
+    same_part = (a["partition"] == b["partition"]).all(axis=1)
+    assert same_part[fin].mean() > 0.999
+    both = fin & same_part
+    assert np.allclose(a["cost"][both], b["cost"][both], rtol=1e-13, atol=0.0)
+    assert np.array_equal(a["recompute"][both], b["recompute"][both])
