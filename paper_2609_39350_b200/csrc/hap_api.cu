@@ -41,8 +41,7 @@ struct hap_problem {
                          u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
     struct Trie { bool ok = false; TrieMeta *d_metas = nullptr; u32 *d_plist = nullptr;       // both inside d_trie_arena
                   std::vector<TriePartDev> parts; unsigned n_conf = 0; int threads = 0; size_t smem = 0; };
-    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie;
-                     mutable bool decoded = false; };       // this pass's candidate decode is already queued on `stream`
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     unsigned char *d_arena = nullptr;      // everything hap_enumerate sizes, in one allocation (the d_* pointers below point into it)
@@ -74,6 +73,12 @@ struct hap_problem {
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_fork = nullptr;          // classes run on their own streams between this event and their `done` events
     cudaEvent_t ev_pre = nullptr;           // start of a pass: the candidate decode of the classes waits for this one only
+    cudaEvent_t ev_dec = nullptr;           // the merged candidate decode of a pass has finished
+    DecodeJobs decode_jobs{};               // classes that walk a prefix tree: one merged decode launch per pass
+    GatherJob *d_gather_jobs = nullptr;     // inside d_trie_arena: one entry per part of every tree
+    int n_gather_jobs = 0;
+    unsigned gather_blocks = 0;
+    bool decoded_all = false;               // this pass's merged decode is already queued
     std::string err;
 };
 
@@ -227,6 +232,7 @@ static void release_device(hap_problem *p)
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_pre) cudaEventDestroy(p->ev_pre);
+    if (p->ev_dec) cudaEventDestroy(p->ev_dec);
     for (auto &cl : p->classes) { if (cl.done) cudaEventDestroy(cl.done); }      // the class streams belong to the pool
 }
 
@@ -721,12 +727,18 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
 {
     constexpr size_t kTwoPerSm = 108 * 1024;
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
-    size_t total = 0;
+    size_t total = 0, n_parts_all = 0;
     for (auto &bc : built) {
         for (const auto &pt : bc.second.parts) total += up(pt.blob.size());
         total += up(bc.second.parts.size() * sizeof(TrieMeta)) + up(bc.second.plist.size() * sizeof(u32));
+        n_parts_all += bc.second.parts.size();
     }
     if (!total) return true;
+    const size_t o_jobs = total;
+    total += up(n_parts_all * sizeof(GatherJob));
+    std::vector<GatherJob> gjobs;
+    DecodeJobs dj{};
+    unsigned dblk = 0, gblk = 0;
     if (cached_malloc(p->device, (void **)&p->d_trie_arena, total) != cudaSuccess) { p->d_trie_arena = nullptr; cudaGetLastError(); return false; }
     std::vector<unsigned char> stage(total, 0);
     size_t off = 0;
@@ -752,6 +764,14 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
             pt.meta.parent = reinterpret_cast<const uint16_t *>(base + pt.o_parent);
             tr.parts.push_back(pd);
             metas.push_back(pt.meta);
+            GatherJob gj{};
+            gj.first_leaf = pd.d_first_leaf; gj.gnode = pd.d_gnode; gj.depth = pd.d_depth;
+            gj.nodes = pd.d_nodes; gj.cells = pd.d_cells; gj.leaves = pd.d_leaves;
+            gj.tab_off = bc.first->map_base; gj.n_nodes = pd.n_nodes; gj.n_cells = pd.n_cells; gj.nmap = pd.nmap; gj.m_lo = pd.m_lo;
+            gj.blk_lo = gblk; gj.PP = bc.first->PP;
+            std::memcpy(gj.rm.mrow_of, pd.mrow_of, sizeof(gj.rm.mrow_of));
+            gblk += (pd.n_nodes + pd.n_cells + pd.nmap + 255) / 256;
+            gjobs.push_back(gj);
             smem = std::max(smem, pt.smem);
             want = std::max(want, std::max(pt.max_level, pt.nmap));
             off += up(pt.blob.size());
@@ -763,15 +783,29 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
         std::memcpy(stage.data() + off, h.plist.data(), h.plist.size() * sizeof(u32));
         off += up(h.plist.size() * sizeof(u32));
         tr.n_conf = (unsigned)h.plist.size(); tr.smem = smem;
+        if (dj.n <= HAP_MAX_PP) {
+            const hap_problem::PpClass &cl = *bc.first;
+            const u32 rep = p->items[cl.item_lo].p;
+            const u64 nmap_cl = p->pconfs[rep].nmap;
+            dj.blk_lo[dj.n] = dblk; dj.p_rep[dj.n] = rep; dj.nmap[dj.n] = (u32)nmap_cl; dj.tab_off[dj.n] = cl.map_base;
+            dblk += (unsigned)((nmap_cl + 3) / 4);
+            dj.n++;
+            dj.blk_lo[dj.n] = dblk;
+        }
         // a thread takes about four cells of the widest depth (measured: smaller blocks, more of them per SM)
         const int th = (int)(((want + 3) / 4 + 31) / 32 * 32);
         tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
         tr.ok = true;
     }
+    std::memcpy(stage.data() + o_jobs, gjobs.data(), gjobs.size() * sizeof(GatherJob));
     if (cudaMemcpy(p->d_trie_arena, stage.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
         for (auto &bc : built) bc.first->trie = hap_problem::Trie{};
         return false;
     }
+    p->decode_jobs = dj;
+    p->d_gather_jobs = reinterpret_cast<GatherJob *>(p->d_trie_arena + o_jobs);
+    p->n_gather_jobs = (int)gjobs.size();
+    p->gather_blocks = gblk;
     return true;
 }
 
@@ -929,6 +963,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         p->dc.n_pconf = np;
         CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming));
         CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_pre, cudaEventDisableTiming));
+        CUDA_TRY(p, cudaEventCreateWithFlags(&p->ev_dec, cudaEventDisableTiming));
         for (size_t ci = 0; ci < p->classes.size(); ++ci) {
             auto &cl = p->classes[ci];
             cl.stream = pooled_stream(p->device, ci);
@@ -1110,21 +1145,30 @@ static hap_status launch_class_decode(hap_problem *p, const hap_problem::PpClass
     return HAP_OK;
 }
 
-// The candidate decode reads nothing the layer-cost kernels write: a pass queues it on the class streams first, so
-// that it runs beside the layer costs instead of between them and the recurrence.
-static hap_status launch_decode_early(hap_problem *p, const DpOut &out, bool search, cudaStream_t st)
+// The candidate decode reads nothing the layer-cost kernels write: it waits only for the start of the pass (ev_pre,
+// recorded before the layer-cost launches) and runs on the class streams beside the layer costs instead of between
+// them and the recurrence.  On the host it is issued after the layer-cost launches, so that those reach an idle GPU
+// without waiting for a dozen other launches to be queued.
+static hap_status launch_decode_early(hap_problem *p, const DpOut &out, bool search)
 {
-    bool any = false;
-    for (const auto &cl : p->classes) any |= pass_uses_trie(p, cl, out, false) && (search || !class_outside(p, cl, out));
-    if (!any) return HAP_OK;
-    CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
+    (void)search;
+    bool any = false, all = true;
     for (const auto &cl : p->classes) {
-        if (!pass_uses_trie(p, cl, out, false) || (!search && class_outside(p, cl, out))) continue;
-        CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_pre, 0));
-        hap_status s = launch_class_decode(p, cl);
-        if (s != HAP_OK) return s;
-        cl.decoded = true;
+        const bool uses = pass_uses_trie(p, cl, out, false);
+        any |= uses;
+        if (cl.trie.ok && !uses) all = false;
     }
+    if (!any || !all || !p->n_gather_jobs || p->decode_jobs.n == 0) return HAP_OK;
+    // one decode launch and one gather launch for all classes and parts, on the first class's stream
+    cudaStream_t sx = p->classes[0].stream;
+    CUDA_TRY(p, cudaStreamWaitEvent(sx, p->ev_pre, 0));
+    const DecodeJobs &dj = p->decode_jobs;
+    maptab_all_kernel<<<dj.blk_lo[dj.n], 128, 0, sx>>>(p->dc, dj, p->d_maptab);
+    CUDA_TRY(p, cudaGetLastError());
+    trie_gather_all_kernel<<<p->gather_blocks, 256, 0, sx>>>(p->d_gather_jobs, p->n_gather_jobs, p->d_maptab);
+    CUDA_TRY(p, cudaGetLastError());
+    CUDA_TRY(p, cudaEventRecord(p->ev_dec, sx));
+    p->decoded_all = true;
     return HAP_OK;
 }
 
@@ -1135,7 +1179,11 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     // process: raise it (never lower it) before a launch that needs more
     static size_t smem_limit[64][12];
     const int dev = p->device & 63;
-    // fork: every PP class runs on its own stream so that the tail of one class overlaps the next
+    // fork: every PP class runs on its own stream so that the tail of one class overlaps the next; a merged
+    // candidate decode queued earlier in this pass joins first, so that the fork event covers it
+    const bool decoded_all = p->decoded_all;
+    p->decoded_all = false;
+    if (decoded_all) CUDA_TRY(p, cudaStreamWaitEvent(st, p->ev_dec, 0));
     CUDA_TRY(p, cudaEventRecord(p->ev_fork, st));
     // the class with the most work goes first; the others fill the SMs it leaves free and its tail
     std::vector<const hap_problem::PpClass *> order;
@@ -1143,6 +1191,8 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     std::stable_sort(order.begin(), order.end(), [](const hap_problem::PpClass *a, const hap_problem::PpClass *b) {
         return (a->item_hi - a->item_lo) * (size_t)a->PP > (b->item_hi - b->item_lo) * (size_t)b->PP;
     });
+    // a pruning search wants an incumbent early: the light classes go first, their minimum then prunes the heavy ones
+    if (search && out.prune) std::reverse(order.begin(), order.end());
     for (const hap_problem::PpClass *clp : order) {
         const hap_problem::PpClass &cl = *clp;
         // skip classes whose candidates all lie outside the range
@@ -1181,11 +1231,10 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
                 trie_limit[dev][vi] = tr.smem;
             }
             CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
-            if (!cl.decoded) {                      // not queued ahead of the layer costs by this pass
+            if (!decoded_all) {                     // not queued beside the layer costs by this pass
                 hap_status sd = launch_class_decode(p, cl);
                 if (sd != HAP_OK) return sd;
             }
-            cl.decoded = false;
             int n_parts = (int)tr.parts.size();
             unsigned n_active = tr.n_conf * (unsigned)n_parts;
             const u32 *plist = tr.d_plist;
@@ -1236,9 +1285,10 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
     out.recompute = dev_recompute; out.dp_table = (i64 *)dev_dp_table; out.choice = dev_choice;
     out.first = first; out.count = count;
-    if ((s = launch_decode_early(p, out, false, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
     if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
+    if ((s = launch_decode_early(p, out, false)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
@@ -1513,8 +1563,11 @@ extern "C" hap_status hap_launches_per_pass(hap_problem *p, uint32_t *host_count
     const bool lin = p->dc.tau_linear != 0;
     const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0;
     uint32_t n = 2 + 2;                                     // type constants, layer costs; argmin partial and final
+    bool all_trees = p->n_gather_jobs > 0;
+    for (const auto &cl : p->classes) if (cl.trie.ok && !(lin && !refine)) all_trees = false;
+    if (all_trees) n += 2;                                  // one decode and one tree-gather launch for all classes
     for (const auto &cl : p->classes) {
-        if (cl.trie.ok && lin && !refine) n += 1 + (uint32_t)cl.trie.parts.size() + 1;   // decode, tree gather per part, tree DP
+        if (cl.trie.ok && lin && !refine) n += all_trees ? 1 : 1 + (uint32_t)cl.trie.parts.size() + 1;   // (decode, gather per part,) tree DP
         else n += (cl.has_tab ? 1 : 0) + 1;                                            // decode table, one-warp-per-candidate DP
     }
     *host_count = n;
@@ -1563,9 +1616,10 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     out.first = first; out.count = count; out.prune = p->opts.prune;
     out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
     out.incumbent = p->d_counters + 3;
-    if ((s = launch_decode_early(p, out, true, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
     if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st, p->d_lb)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
+    if ((s = launch_decode_early(p, out, true)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
     argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best, kInf);
     CUDA_TRY(p, cudaGetLastError());

@@ -790,10 +790,8 @@ simulate_1f1b_kernel(const DevConst dc, u64 first, u64 count, const i64 *__restr
 // built in every pass (and once at enumeration, for the host-side tree) so that the DP kernels do not
 // unrank per candidate
 // ------------------------------------------------------------------------------------------
-__global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *tab)
+__device__ __forceinline__ void maptab_one(const DevConst &dc, u64 p_rep, u64 nmap, uint8_t *tab, u64 w, int lane)
 {
-    const u64 w = ((u64)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
     if (w >= nmap) return;
     const hap_pconf pc = dc.pconf[p_rep];
     const StageMap sm = decode_stage(dc, pc, w, lane);
@@ -802,6 +800,29 @@ __global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *t
         o[0] = (uint8_t)sm.mask;
         o[1] = (uint8_t)(lane > 0 ? (sm.cls | (sm.ha << 2) | (sm.hb << 4)) : 0);
     }
+}
+
+__global__ void maptab_kernel(const DevConst dc, u64 p_rep, u64 nmap, uint8_t *tab)
+{
+    maptab_one(dc, p_rep, nmap, tab, ((u64)blockIdx.x * blockDim.x + threadIdx.x) >> 5, threadIdx.x & 31);
+}
+
+// The same for several PP classes in one launch (a pass decodes all classes that walk a prefix tree this way):
+// class q owns blocks [blk_lo[q], blk_lo[q+1]) of 128 threads, four mappings per block.
+struct DecodeJobs {
+    int n;
+    u32 blk_lo[HAP_MAX_PP + 2];
+    u32 p_rep[HAP_MAX_PP + 1];
+    u32 nmap[HAP_MAX_PP + 1];
+    u64 tab_off[HAP_MAX_PP + 1];            // byte offset of the class's table
+};
+
+__global__ void __launch_bounds__(128) maptab_all_kernel(const DevConst dc, const DecodeJobs jobs, uint8_t *tab_base)
+{
+    int q = 0;
+    while (q + 1 < jobs.n && blockIdx.x >= jobs.blk_lo[q + 1]) ++q;
+    const u64 w = ((u64)(blockIdx.x - jobs.blk_lo[q]) * blockDim.x + threadIdx.x) >> 5;
+    maptab_one(dc, jobs.p_rep[q], jobs.nmap[q], tab_base + jobs.tab_off[q], w, threadIdx.x & 31);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -91,12 +91,11 @@ struct TrieRowMap { uint8_t mrow_of[16]; };
 // Copies what the decode of this pass produced into the tree: node n of depth d takes the stage bytes (device
 // types, boundary link) of stage d of the first mapping below it, every cell of the node the index of the stage
 // constant that follows from them, leaf m the last stage of mapping m.
-__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap, u32 m_lo,
-                                   const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
-                                   const u32 *__restrict__ cell_gnode, const TrieRowMap rm,
-                                   TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves)
+__device__ __forceinline__ void trie_gather_one(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap, u32 m_lo,
+                                                const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
+                                                const u32 *__restrict__ cell_gnode, const TrieRowMap &rm,
+                                                TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves, u32 g)
 {
-    const u32 g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g < n_nodes) {
         const uint8_t *src = maptab + ((u64)first_leaf[g] * PP + (depth[g] - 1)) * 2;
         nodes[g].mask = src[0]; nodes[g].link = src[1];
@@ -116,6 +115,38 @@ __global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u
         const uint8_t *src = maptab + ((u64)(m_lo + m) * PP + (PP - 1)) * 2;
         leaves[m].mask = src[0]; leaves[m].link = src[1];
     }
+}
+
+__global__ void trie_gather_kernel(const uint8_t *__restrict__ maptab, int PP, u32 n_nodes, u32 n_cells, u32 nmap, u32 m_lo,
+                                   const u32 *__restrict__ first_leaf, const uint8_t *__restrict__ depth,
+                                   const u32 *__restrict__ cell_gnode, const TrieRowMap rm,
+                                   TrieNode *nodes, TrieCell *cells, TrieLeaf *leaves)
+{
+    trie_gather_one(maptab, PP, n_nodes, n_cells, nmap, m_lo, first_leaf, depth, cell_gnode, rm, nodes, cells, leaves,
+                    blockIdx.x * blockDim.x + threadIdx.x);
+}
+
+// The same for every part of every class's tree in one launch: part q owns blocks [blk_lo, blk_lo + blocks) of 256
+// threads (the job list lives in device memory: it is fixed once the trees are built).
+struct GatherJob {
+    const u32 *first_leaf, *gnode;
+    const uint8_t *depth;
+    TrieNode *nodes;
+    TrieCell *cells;
+    TrieLeaf *leaves;
+    u64 tab_off;                 // byte offset of the class's decoded-mapping table
+    u32 n_nodes, n_cells, nmap, m_lo, blk_lo;
+    int PP;
+    TrieRowMap rm;
+};
+
+__global__ void __launch_bounds__(256) trie_gather_all_kernel(const GatherJob *__restrict__ jobs, int n_jobs, const uint8_t *__restrict__ tab_base)
+{
+    int q = 0;
+    while (q + 1 < n_jobs && blockIdx.x >= jobs[q + 1].blk_lo) ++q;
+    const GatherJob &jb = jobs[q];
+    trie_gather_one(tab_base + jb.tab_off, jb.PP, jb.n_nodes, jb.n_cells, jb.nmap, jb.m_lo, jb.first_leaf, jb.depth, jb.gnode, jb.rm,
+                    jb.nodes, jb.cells, jb.leaves, (blockIdx.x - jb.blk_lo) * blockDim.x + threadIdx.x);
 }
 
 // shared-memory accesses by 32-bit address (the split loop walks two rows with plain address decrements)
