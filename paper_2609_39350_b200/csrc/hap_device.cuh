@@ -7,7 +7,8 @@
 //   layer_cost_kernel   per (configuration, type, layer): Eq. 2 with imbalance scaling, rounding,
 //                       one block per configuration, one thread per layer.
 //   decode_kernel       candidate index -> stage type masks and boundary link classes;
-//   maptab_kernel       the same for every mapping of one PP class (every pass).
+//   maptab_kernel       the same for every mapping of one PP class; maptab_all_kernel for all classes in one
+//                       launch (every pass).
 //   trie_dp_kernel      (hap_trie.cuh) the default dynamic program: all mappings of a configuration
 //                       together through the prefix tree of their stage sequences.
 //   pipeline_dp_kernel  the general form (DP tables on request, refinement / exact modes, classes
