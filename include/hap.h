@@ -342,6 +342,19 @@ hap_status hap_eval_appendix_b(hap_problem *, uint64_t first, uint64_t count, co
 hap_status hap_simulate_1f1b(hap_problem *, uint64_t first, uint64_t count, const uint8_t *dev_partition,
                              const uint8_t *dev_recompute, int64_t *dev_t_iter, int64_t *dev_detail, void *stream);
 
+/* Sec. 4 caches the profiled tables between planner runs; these two calls do that for a whole planning problem.
+ * hap_problem_save writes everything hap_problem_create was given (model, cluster, tables, coefficients, search
+ * options; the tables are read back from the device) as one self-describing blob into host_buf and sets *host_need
+ * to its size; with host_buf = NULL it only reports the size, with cap < size it writes nothing and returns
+ * HAP_E_RANGE.  hap_problem_load validates a blob (magic, length, every array length) and hands its content to
+ * hap_problem_create on the current device; a blob that is truncated, altered in size or of another version gives
+ * HAP_E_INVALID.  The blob is host-endian and tied to this header's limits; it carries no results. */
+hap_status hap_problem_save(hap_problem *, void *host_buf, uint64_t cap, uint64_t *host_need);
+hap_status hap_problem_load(const void *host_buf, uint64_t len, hap_problem **out);
+/* Layers, device types and recomputation policies of a problem (what a caller needs to size the outputs of a loaded
+ * problem); any pointer may be NULL. */
+hap_status hap_problem_dims(const hap_problem *, int32_t *host_N, int32_t *host_T, int32_t *host_n_rc);
+
 /* Self-checking build (no counterpart in the paper).  A library compiled with -DHAP_CHECKED
  * (paper_2609_39350_b200.build.build_library(checked=True) -> libhap_checked.so) compares the indices and
  * shared-memory addresses its kernels form from tables (tree records, row origins, threshold indices, output slots,

@@ -17,7 +17,7 @@ STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE",
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
            "hap_search_range", "hap_search_range_f64",
-           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_simulate_1f1b", "hap_release_cached_memory", "hap_self_check", "hap_status_str", "hap_last_error"]
+           "hap_search_best", "hap_argmin", "hap_argmin_static", "hap_joint_bottleneck", "hap_count_cells", "hap_get_timings", "hap_launches_per_pass", "hap_eval_appendix_b", "hap_simulate_1f1b", "hap_release_cached_memory", "hap_self_check", "hap_problem_save", "hap_problem_load", "hap_problem_dims", "hap_status_str", "hap_last_error"]
 
 
 class HapError(RuntimeError):
@@ -117,10 +117,14 @@ def _stream(stream) -> C.c_void_p:
 class HapProblem:
     """Owner of a hap_problem* handle."""
 
-    def __init__(self, handle: int, pb):
+    def __init__(self, handle: int, pb=None):
         self.h = C.c_void_p(handle)
-        self.N, self.T = int(pb.N), int(pb.P.shape[0])
-        self.n_rc = len(pb.rc_masks)
+        if pb is not None:
+            self.N, self.T, self.n_rc = int(pb.N), int(pb.P.shape[0]), len(pb.rc_masks)
+        else:                               # a loaded problem: ask the library
+            n, t, r = C.c_int32(), C.c_int32(), C.c_int32()
+            self.check(load_library().hap_problem_dims(self.h, C.byref(n), C.byref(t), C.byref(r)))
+            self.N, self.T, self.n_rc = int(n.value), int(t.value), int(r.value)
         self.n_pconf = self.n_cand = None
 
     def check(self, status: int):
@@ -371,6 +375,29 @@ def hap_simulate_1f1b(hp: HapProblem, first: int, count: int, partition, recompu
     hp.check(load_library().hap_simulate_1f1b(hp.h, C.c_uint64(first), C.c_uint64(count), _dev(partition), _dev(recompute),
                                               _dev(t), _dev(d), _stream(stream)))
     return {"t_iter": t, "detail": d}
+
+
+def hap_problem_dims(hp: HapProblem):
+    """(layers, device types, recomputation policies) of a problem."""
+    return hp.N, hp.T, hp.n_rc
+
+
+def hap_problem_save(hp: HapProblem) -> bytes:
+    """The problem's inputs (model, cluster, tables, coefficients, search options) as one blob."""
+    need = C.c_uint64()
+    hp.check(load_library().hap_problem_save(hp.h, None, C.c_uint64(0), C.byref(need)))
+    buf = C.create_string_buffer(int(need.value))
+    hp.check(load_library().hap_problem_save(hp.h, buf, C.c_uint64(need.value), C.byref(need)))
+    return buf.raw[:int(need.value)]
+
+
+def hap_problem_load(blob: bytes) -> HapProblem:
+    """A new problem on the current device from a blob written by hap_problem_save."""
+    h = C.c_void_p()
+    st = load_library().hap_problem_load(blob, C.c_uint64(len(blob)), C.byref(h))
+    if st != 0:
+        raise HapError(st, "hap_problem_load")
+    return HapProblem(h.value)
 
 
 def hap_self_check() -> int:

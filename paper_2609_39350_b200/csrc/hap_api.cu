@@ -1540,6 +1540,138 @@ extern "C" hap_status hap_simulate_1f1b(hap_problem *p, uint64_t first, uint64_t
     return HAP_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// hap_problem_save / hap_problem_load: the planner's inputs as one flat blob (the profiled tables are the
+// expensive part of a planning problem: Sec. 4 caches them between runs)
+// ------------------------------------------------------------------------------------------
+namespace {
+constexpr uint64_t kBlobMagic = 0x31424f4c42504148ull;        // "HAPBLOB1"
+struct BlobWriter {
+    unsigned char *buf; uint64_t cap, at = 0;
+    void bytes(const void *src, uint64_t n) { if (buf && at + n <= cap) std::memcpy(buf + at, src, n); at += n; }
+    template <class T> void pod(const T &v) { bytes(&v, sizeof(T)); }
+    template <class T> void vec(const std::vector<T> &v) { pod<uint64_t>(v.size()); if (!v.empty()) bytes(v.data(), v.size() * sizeof(T)); }
+};
+struct BlobReader {
+    const unsigned char *buf; uint64_t len, at = 0; bool ok = true;
+    void bytes(void *dst, uint64_t n) { if (!ok || n > len - at) { ok = false; return; } std::memcpy(dst, buf + at, n); at += n; }
+    template <class T> void pod(T &v) { bytes(&v, sizeof(T)); }
+    template <class T> void vec(std::vector<T> &v, uint64_t max_n)
+    {
+        uint64_t n = 0; pod(n);
+        if (!ok || n > max_n || n * sizeof(T) > len - at) { ok = false; return; }
+        v.resize(n);
+        if (n) bytes(v.data(), n * sizeof(T));
+    }
+};
+}  // namespace
+
+extern "C" hap_status hap_problem_save(hap_problem *p, void *host_buf, uint64_t cap, uint64_t *host_need)
+{
+    if (!p || !host_need) return HAP_E_INVALID;
+    if (cudaSetDevice(p->device) != cudaSuccess) return fail(p, HAP_E_CUDA, "cudaSetDevice");
+    const int N = p->model.N, T = p->T;
+    const hap_profile &pf = p->prof;
+    const size_t n4 = (size_t)T * pf.ntp * pf.ncp * pf.nmb, n5 = n4 * N;
+    // the tables live on the device only (per-layer ones interleaved entry by entry): read them back in the caller's layout
+    std::vector<double> dev(4 * n5 + 2 * n4), tab[4];
+    CUDA_TRY(p, cudaMemcpy(dev.data(), p->d_tables, dev.size() * sizeof(double), cudaMemcpyDeviceToHost));
+    for (int t = 0; t < 4; ++t) { tab[t].resize(n5); for (size_t i = 0; i < n5; ++i) tab[t][i] = dev[4 * i + t]; }
+    std::vector<double> tpre(dev.begin() + 4 * n5, dev.begin() + 4 * n5 + n4), tpost(dev.begin() + 4 * n5 + n4, dev.end());
+    std::vector<double> fsize(p->dc.fsize, p->dc.fsize + pf.n_fsize), feff;
+    for (int c = 0; c < 3; ++c) feff.insert(feff.end(), p->dc.feff[c], p->dc.feff[c] + pf.n_fsize);
+    BlobWriter w{static_cast<unsigned char *>(host_buf), host_buf ? cap : 0};
+    w.pod(kBlobMagic); w.pod<uint64_t>(0);                         // total size, patched below
+    hap_model mo = p->model; mo.kind = nullptr;
+    w.pod(mo); w.vec(p->kind);
+    w.pod<int32_t>(T);
+    w.vec(p->P); w.vec(p->C); w.vec(p->node_size); w.vec(p->bw_intra); w.vec(p->node_type); w.vec(p->node_bw_inter);
+    w.vec(p->tp_list); w.vec(p->cp_list); w.vec(p->mb_list); w.vec(p->ep_list);
+    for (int t = 0; t < 4; ++t) w.vec(tab[t]);
+    w.vec(tpre); w.vec(tpost);
+    w.vec(p->eta); w.vec(p->croute); w.vec(p->alpha); w.vec(p->rho); w.vec(p->act_coef); w.vec(p->copt); w.vec(p->cap_eff);
+    w.vec(p->xi_q); w.vec(p->tau_q); w.vec(fsize); w.vec(feff);
+    const double scal[7] = {pf.kappa, pf.chi, pf.gamma, pf.ovl_tp, pf.ovl_cp, pf.ovl_dp, pf.capf};
+    w.bytes(scal, sizeof(scal));
+    w.vec(p->pp_list); w.vec(p->tpe_list); w.vec(p->rc_masks);
+    const hap_search_opts &so = p->opts;
+    const int64_t oi[6] = {so.tp_max, so.delta_q, (int64_t)so.map_cap, so.prune, so.flags, so.eta_q};
+    w.bytes(oi, sizeof(oi));
+    *host_need = w.at;
+    if (!host_buf || cap < w.at) return host_buf ? fail(p, HAP_E_RANGE, "the blob needs %llu bytes", (unsigned long long)w.at) : HAP_OK;
+    std::memcpy(static_cast<unsigned char *>(host_buf) + 8, &w.at, 8);
+    return HAP_OK;
+}
+
+extern "C" hap_status hap_problem_load(const void *host_buf, uint64_t len, hap_problem **out)
+{
+    if (!out) return HAP_E_INVALID;
+    *out = nullptr;
+    if (!host_buf || len < 16) return HAP_E_INVALID;
+    BlobReader r{static_cast<const unsigned char *>(host_buf), len};
+    uint64_t magic = 0, total = 0;
+    r.pod(magic); r.pod(total);
+    if (!r.ok || magic != kBlobMagic || total != len) return HAP_E_INVALID;
+    constexpr uint64_t kMaxTab = 1ull << 28;
+    hap_model mo{}; std::vector<uint8_t> kind;
+    int32_t T = 0;
+    std::vector<int64_t> P, C, cap_eff;
+    std::vector<int32_t> node_size, node_type, tp, cp, mb, ep, xi, tau, pp, tpe;
+    std::vector<double> bw_intra, node_bw, tab[4], tpre, tpost, eta, croute, alpha, rho, act, copt, fsize, feff;
+    std::vector<uint32_t> rc;
+    r.pod(mo); r.vec(kind, HAP_MAX_LAYERS);
+    r.pod(T);
+    r.vec(P, HAP_MAX_TYPES); r.vec(C, HAP_MAX_TYPES); r.vec(node_size, HAP_MAX_TYPES); r.vec(bw_intra, HAP_MAX_TYPES);
+    r.vec(node_type, 1u << 20); r.vec(node_bw, 1u << 20);
+    r.vec(tp, HAP_MAX_LIST); r.vec(cp, HAP_MAX_LIST); r.vec(mb, HAP_MAX_LIST); r.vec(ep, HAP_MAX_LIST);
+    for (int t = 0; t < 4; ++t) r.vec(tab[t], kMaxTab);
+    r.vec(tpre, kMaxTab); r.vec(tpost, kMaxTab);
+    r.vec(eta, HAP_MAX_TYPES); r.vec(croute, HAP_MAX_TYPES); r.vec(alpha, 3); r.vec(rho, HAP_MAX_LIST); r.vec(act, 2);
+    r.vec(copt, HAP_MAX_TYPES); r.vec(cap_eff, HAP_MAX_TYPES);
+    r.vec(xi, HAP_MAX_RC); r.vec(tau, HAP_MAX_RC); r.vec(fsize, HAP_MAX_LIST); r.vec(feff, 3 * HAP_MAX_LIST);
+    double scal[7] = {0}; r.bytes(scal, sizeof(scal));
+    r.vec(pp, HAP_MAX_LIST); r.vec(tpe, HAP_MAX_LIST); r.vec(rc, HAP_MAX_RC_MASKS);
+    int64_t oi[6] = {0}; r.bytes(oi, sizeof(oi));
+    if (!r.ok || r.at != len) return HAP_E_INVALID;
+    // sizes that hap_problem_create takes on trust from the pointers it is given
+    if (T < 1 || T > HAP_MAX_TYPES || mo.N < 1 || (int64_t)kind.size() != mo.N || (int)P.size() != T || (int)C.size() != T ||
+        (int)node_size.size() != T || (int)bw_intra.size() != T || node_type.size() != node_bw.size() || (int)eta.size() != T ||
+        (int)croute.size() != T || alpha.size() != 3 || rho.size() != ep.size() || act.size() != 2 || (int)copt.size() != T ||
+        (int)cap_eff.size() != T || xi.size() != tau.size() || xi.empty() || feff.size() != 3 * fsize.size())
+        return HAP_E_INVALID;
+    const size_t n4 = (size_t)T * tp.size() * cp.size() * mb.size(), n5 = n4 * (size_t)mo.N;
+    for (int t = 0; t < 4; ++t) if (tab[t].size() != n5) return HAP_E_INVALID;
+    if (tpre.size() != n4 || tpost.size() != n4) return HAP_E_INVALID;
+    mo.kind = kind.data();
+    hap_cluster cl{};
+    cl.n_types = T; cl.P = P.data(); cl.C = C.data(); cl.node_size = node_size.data(); cl.bw_intra = bw_intra.data();
+    cl.n_nodes = (int32_t)node_type.size(); cl.node_type = node_type.data(); cl.node_bw_inter = node_bw.data();
+    hap_profile pf{};
+    pf.ntp = (int32_t)tp.size(); pf.ncp = (int32_t)cp.size(); pf.nmb = (int32_t)mb.size(); pf.nep = (int32_t)ep.size();
+    pf.tp_list = tp.data(); pf.cp_list = cp.data(); pf.mb_list = mb.data(); pf.ep_list = ep.data();
+    pf.tdf = tab[0].data(); pf.tdb = tab[1].data(); pf.tff = tab[2].data(); pf.tfb = tab[3].data();
+    pf.tpre = tpre.data(); pf.tpost = tpost.data();
+    pf.eta = eta.data(); pf.croute = croute.data(); pf.kappa = scal[0]; pf.alpha = alpha.data(); pf.chi = scal[1];
+    pf.rho = rho.data(); pf.gamma = scal[2]; pf.ovl_tp = scal[3]; pf.ovl_cp = scal[4]; pf.ovl_dp = scal[5];
+    pf.act_coef = act.data(); pf.capf = scal[6]; pf.copt = copt.data(); pf.cap_eff = cap_eff.data();
+    pf.R = (int32_t)xi.size(); pf.xi_q = xi.data(); pf.tau_q = tau.data();
+    pf.n_fsize = (int32_t)fsize.size(); pf.fsize = fsize.empty() ? nullptr : fsize.data(); pf.feff = feff.empty() ? nullptr : feff.data();
+    hap_search_opts so{};
+    so.npp = (int32_t)pp.size(); so.ntpe = (int32_t)tpe.size(); so.pp_list = pp.data(); so.tpe_list = tpe.data();
+    so.tp_max = (int32_t)oi[0]; so.delta_q = (int32_t)oi[1]; so.map_cap = (uint64_t)oi[2]; so.n_rc = (int32_t)rc.size();
+    so.rc_masks = rc.data(); so.prune = (int32_t)oi[3]; so.flags = (int32_t)oi[4]; so.eta_q = (int32_t)oi[5];
+    return hap_problem_create(&mo, &cl, &pf, &so, out);
+}
+
+extern "C" hap_status hap_problem_dims(const hap_problem *p, int32_t *host_N, int32_t *host_T, int32_t *host_n_rc)
+{
+    if (!p) return HAP_E_INVALID;
+    if (host_N) *host_N = p->model.N;
+    if (host_T) *host_T = p->T;
+    if (host_n_rc) *host_n_rc = p->opts.n_rc;
+    return HAP_OK;
+}
+
 extern "C" hap_status hap_self_check(uint64_t *host_sites)
 {
     if (!host_sites) return HAP_E_INVALID;

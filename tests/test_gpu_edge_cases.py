@@ -216,3 +216,38 @@ def test_device_memory_of_destroyed_problems_is_reused(hap):
     free_released, _ = torch.cuda.mem_get_info()
     assert free_released > free_cached           # idle blocks went back to the driver
     hap.hap_release_cached_memory()              # nothing left: a no-op
+
+
+@pytest.mark.parametrize("make", [lambda: problems.tiny(), lambda: problems.with_link_efficiency_table(problems.small(), seed=3),
+                                  lambda: problems.random_small(23, N=12, T=3, nodes_per_type=(2, 1, 1), node_size=2, window=True, first_dense=True)])
+def test_saved_problem_loads_into_an_identical_one(hap, make):
+    """hap_problem_save / hap_problem_load: the blob carries every input; the loaded problem enumerates the same
+    space and gives the same costs and plan.  Damaged blobs are refused."""
+    pb = make()
+    hp = hap.hap_problem_create(pb)
+    blob = hap.hap_problem_save(hp)
+    hap.hap_enumerate(hp)
+    ref = hap.hap_pipeline_dp(hp, 0, hp.n_cand, partition=True)
+    plan, _ = hap.hap_search_best(hp)
+    assert hap.hap_problem_save(hp) == blob                       # saving is repeatable and independent of the state
+    hp2 = hap.hap_problem_load(blob)
+    assert (hp2.N, hp2.T, hp2.n_rc) == (hp.N, hp.T, hp.n_rc)
+    assert hap.hap_enumerate(hp2) == (hp.n_pconf, hp.n_cand)
+    out = hap.hap_pipeline_dp(hp2, 0, hp2.n_cand, partition=True)
+    plan2, _ = hap.hap_search_best(hp2)
+    torch.cuda.synchronize()
+    for key in ("cost", "bottleneck", "partition", "recompute"):
+        assert torch.equal(out[key], ref[key]), key
+    assert plan2 == plan
+    assert hap.hap_problem_save(hp2) == blob
+    hap.hap_problem_destroy(hp)
+    hap.hap_problem_destroy(hp2)
+    for bad in (blob[:-1], blob[:40], b"", blob + b"\0", b"X" + blob[1:], blob[:8] + (len(blob) + 8).to_bytes(8, "little") + blob[16:]):
+        with pytest.raises(hap.HapError) as e:
+            hap.hap_problem_load(bad)
+        assert e.value.name == "HAP_E_INVALID"
+    # a length field inside the blob that points past its end
+    cut = bytearray(blob)
+    cut[16 + 64 + 0:16 + 64 + 8] = (1 << 40).to_bytes(8, "little")
+    with pytest.raises(hap.HapError):
+        hap.hap_problem_load(bytes(cut))
