@@ -35,6 +35,12 @@ def test_status_strings_and_null_arguments():
     assert lib.hap_problem_create(None, None, None, None, ctypes.byref(out)) == 1 and not out.value
     assert lib.hap_enumerate(None, None, None) == 1
     lib.hap_problem_destroy(None)
+    # blobs are validated before any device work: garbage is refused without a GPU
+    for blob in (b"", b"not a blob at all....", b"HAPBLOB1" + (24).to_bytes(8, "little") + b"\0" * 8):
+        out = ctypes.c_void_p(0)
+        assert lib.hap_problem_load(blob, ctypes.c_uint64(len(blob)), ctypes.byref(out)) == 1 and not out.value
+    sites = ctypes.c_uint64(7)
+    assert lib.hap_self_check(ctypes.byref(sites)) == 5 and sites.value == 0      # HAP_E_STATE: not the self-checking build
 
 
 def test_layouts_match_the_header_sizes():
