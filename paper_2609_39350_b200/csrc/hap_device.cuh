@@ -1345,6 +1345,9 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                                     const VT cst = Cj - rr[k];
                                     const VT v = pv > cst ? pv : cst;
                                     if (v <= best && v < vInf) { best = v; arg = k; }   // descending k, <=: smallest k wins
+                                    // layer times are non-negative: the stage cost only grows as k falls within a
+                                    // level, so no further split of this level can reach the best value
+                                    if (cst > best) break;
                                 }
                             } else {
                                 const VT *rC = rM, *rF = rM + n1;
@@ -1355,6 +1358,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
                                     const VT cst = (Cj - rC[k]) + tau_term(tau, Fj - rF[k]);   // forward sums are non-negative
                                     const VT v = pv > cst ? pv : cst;
                                     if (v <= best && v < vInf) { best = v; arg = k; }
+                                    if (cst > best) break;
                                 }
                             }
                             seg_hi = lo - 1;
