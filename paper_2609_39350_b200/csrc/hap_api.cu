@@ -9,6 +9,8 @@
 #include <cstdio>
 #include <cmath>
 #include <cstring>
+#include <array>
+#include <map>
 #include <mutex>
 #include <new>
 #include <string>
@@ -704,13 +706,30 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     constexpr size_t kTwoPerSm = 108 * 1024;                 // dynamic shared memory that lets two blocks share an SM
     const size_t slots = (cl.item_hi - cl.item_lo) / plist.size();       // partial-result slots per configuration
     std::vector<TriePartHost> parts;
-    for (int np : {1, 2, 3, 4, 6, 8}) {
-        if ((u64)np > nmap || (np > 1 && (size_t)np > slots)) break;
+    // The number of parts that worked for a class of this shape before is tried first (a hint kept per process: a
+    // wrong hint costs one failed attempt, the sequence below then runs as usual).
+    static std::mutex hint_mu;
+    static std::map<std::array<long long, 6>, int> hint;
+    const std::array<long long, 6> key = {cl.PP, (long long)nmap, p->model.N, p->T * 16 + p->prof.R, p->opts.delta_q, (long long)(p->opts.flags & HAP_OPT_UNIFORM)};
+    int first_np = 0;
+    { std::lock_guard<std::mutex> lock(hint_mu); auto it = hint.find(key); if (it != hint.end()) first_np = it->second; }
+    auto attempt = [&](int np) {
+        if ((u64)np > nmap || (np > 1 && (size_t)np > slots)) return false;
         std::vector<TriePartHost> cand(np);
         bool ok = true;
         for (int q = 0; q < np && ok; ++q) ok = build_trie_part(p, cl, tab, nmap * q / np, nmap * (q + 1) / np, kTwoPerSm, cand[q]);
-        if (ok) { parts.swap(cand); break; }
-    }
+        if (ok) parts.swap(cand);
+        return ok;
+    };
+    int used_np = 0;
+    if (first_np > 1 && attempt(first_np)) used_np = first_np;
+    if (!used_np)
+        for (int np : {1, 2, 3, 4, 6, 8}) {
+            if ((u64)np > nmap || (np > 1 && (size_t)np > slots)) break;
+            if (np == first_np) continue;
+            if (attempt(np)) { used_np = np; break; }
+        }
+    if (used_np) { std::lock_guard<std::mutex> lock(hint_mu); hint[key] = used_np; }
     if (parts.empty()) {                                     // no split lets two blocks share an SM: one block per SM
         parts.resize(1);
         if (!build_trie_part(p, cl, tab, 0, nmap, 220 * 1024, parts[0])) parts.clear();
