@@ -1210,8 +1210,10 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     std::stable_sort(order.begin(), order.end(), [](const hap_problem::PpClass *a, const hap_problem::PpClass *b) {
         return (a->item_hi - a->item_lo) * (size_t)a->PP > (b->item_hi - b->item_lo) * (size_t)b->PP;
     });
-    // a pruning search wants an incumbent early: the light classes go first, their minimum then prunes the heavy ones
-    if (search && out.prune) std::reverse(order.begin(), order.end());
+    // a pruning search wants a good incumbent early: the lower bound S + (M-1) ceil(S / PP) falls with PP, so the
+    // deepest pipelines are the likeliest to hold the best plan and go first
+    if (search && out.prune)
+        std::stable_sort(order.begin(), order.end(), [](const hap_problem::PpClass *a, const hap_problem::PpClass *b) { return a->PP > b->PP; });
     for (const hap_problem::PpClass *clp : order) {
         const hap_problem::PpClass &cl = *clp;
         // skip classes whose candidates all lie outside the range
