@@ -365,8 +365,9 @@ hap_status hap_problem_dims(const hap_problem *, int32_t *host_N, int32_t *host_
 hap_status hap_self_check(uint64_t *host_sites);
 
 /* Measurement aid: the number of kernels one hap_pipeline_dp call over the whole candidate space followed by
- * one hap_argmin call launches (layer costs, per PP class the candidate decode and the dynamic program, the
- * reduction).  Host value, no device work. */
+ * one hap_argmin call launches (the two layer-cost kernels, the candidate decode and the tree gather - one launch
+ * each for all PP classes when every class walks its prefix tree, else per class -, the dynamic program per PP
+ * class, the two reduction kernels).  Host value, no device work. */
 hap_status hap_launches_per_pass(hap_problem *, uint32_t *host_count);
 
 const char *hap_status_str(hap_status);
