@@ -92,14 +92,24 @@ struct SingleOut {
 };
 
 // The side streams the PP classes run on are shared by all problems of a device and live until the process ends:
-// creating half a dozen streams costs more than a whole search.  Index = position of the class in the problem.
+// creating half a dozen streams costs more than a whole search.  Index = position of the class in the problem,
+// classes ordered from the deepest pipeline down.  A block of a deep class is a long chain of short steps (one
+// barrier-separated depth of its tree per stage and policy) that leaves most issue slots idle, a block of the class
+// with the most mappings keeps them busy but fills an SM's registers: the deep classes' blocks should be resident
+// first and the busy class should fill in behind them, so the streams get priorities in class order (measured at the
+// Stress workload: DP phase 0.46 -> 0.42 ms and the same time in every pass instead of 0.44-0.50).
 static cudaStream_t pooled_stream(int device, size_t index)
 {
     static std::mutex mu;
     static cudaStream_t pool[64][HAP_MAX_PP + 1];
     std::lock_guard<std::mutex> lock(mu);
     cudaStream_t &s = pool[device & 63][index % (HAP_MAX_PP + 1)];
-    if (!s && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) s = nullptr;
+    if (!s) {
+        int least = 0, greatest = 0;                    // numerically: greatest priority <= least priority
+        if (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess) { least = greatest = 0; cudaGetLastError(); }
+        const int pr = std::min(least, greatest + (int)(index % (HAP_MAX_PP + 1)));
+        if (cudaStreamCreateWithPriority(&s, cudaStreamNonBlocking, pr) != cudaSuccess) s = nullptr;
+    }
     return s;
 }
 
