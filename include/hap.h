@@ -152,7 +152,7 @@ typedef struct {
 
 typedef struct {
     int32_t npp, ntpe;
-    const int32_t *pp_list, *tpe_list;  /* pipeline and expert-TP degrees to try (ascending) */
+    const int32_t *pp_list, *tpe_list;  /* pipeline and expert-TP degrees to try (ascending; pp_list without repeats) */
     int32_t tp_max;                      /* TP and TPE are limited to this */
     int32_t delta_q;                     /* load-balance window delta in 1/1024 (Pruning 1); < 0 disables */
     uint64_t map_cap;                    /* enumerate all distinct stage-type sequences only up to this count (<= 2^56) */

@@ -330,6 +330,8 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     }
     for (int h = 0; h < T; ++h) { if (!has[h]) return HAP_E_INVALID; p->W += p->m[h]; }
     auto positive = [](const std::vector<int32_t> &v) { for (int x : v) if (x < 1) return false; return true; };
+    for (size_t i = 0; i < p->pp_list.size(); ++i)                   // a repeated PP would enumerate its configurations twice
+        for (size_t j = 0; j < i; ++j) if (p->pp_list[i] == p->pp_list[j]) return HAP_E_INVALID;
     if (!positive(p->tp_list) || !positive(p->cp_list) || !positive(p->mb_list) || !positive(p->ep_list) ||
         !positive(p->pp_list) || !positive(p->tpe_list))
         return HAP_E_INVALID;
@@ -908,11 +910,15 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             cl.masks_used = 0xffffffffu;
             cl.stream = nullptr; cl.done = nullptr;
             cl.warps = 0;
-            for (const auto &r : rows) if (r.PP == PP) { cl.multiset = r.mode == HAP_MAP_MULTISET; break; }
+            // the rows of a PP value are contiguous (PP is the outermost loop of the enumeration)
+            size_t row_lo = 0;
+            while (row_lo < rows.size() && rows[row_lo].PP != PP) ++row_lo;
+            size_t row_hi = row_lo;
+            while (row_hi < rows.size() && rows[row_hi].PP == PP) ++row_hi;
+            cl.multiset = rows[row_lo].mode == HAP_MAP_MULTISET;
             // most warps per SM: try block shapes from large to small, keep the one with the most resident warps
             int best_resident = 0;
-            uint64_t class_nmap = 0;
-            for (const auto &r : rows) if (r.PP == PP) { class_nmap = r.nmap; break; }
+            const uint64_t class_nmap = rows[row_lo].nmap;
             const uint64_t per_pconf = class_nmap * (uint64_t)p->opts.n_rc;     // candidates a block can have at most
             for (int w : {12, 8, 6, 4, 2, 1}) {
                 if ((uint64_t)w * 8 > per_pconf && w > 2) continue;             // keep about 8 candidates per warp
@@ -928,8 +934,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             const uint64_t chunk_cap = 32ull * cl.warps;
             cl.item_lo = items.size();
             uint64_t nmap = 0;
-            for (size_t pi = 0; pi < rows.size(); ++pi) {
-                if (rows[pi].PP != PP) continue;
+            for (size_t pi = row_lo; pi < row_hi; ++pi) {
                 nmap = rows[pi].nmap;
                 const uint64_t n_chunks = (nmap + chunk_cap - 1) / chunk_cap;
                 const uint64_t chunk = (nmap + n_chunks - 1) / n_chunks;          // balanced chunks
