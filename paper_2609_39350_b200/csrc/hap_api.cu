@@ -1030,7 +1030,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 const bool rows_exact = (int64_t)N * (2 + tau_max) <= 65536;
                 if (!(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear && rows_exact) {
                     std::vector<u32> plist;
-                    for (size_t pi = 0; pi < p->pconfs.size(); ++pi) if (p->pconfs[pi].PP == cl.PP) plist.push_back((u32)pi);
+                    for (size_t pi = p->items[cl.item_lo].p; pi <= p->items[cl.item_hi - 1].p; ++pi) plist.push_back((u32)pi);   // contiguous
                     TrieClassHost th;
                     if (build_trie(p, cl, tab.data() + cl.map_base, nmap, plist, th)) built.emplace_back(&cl, std::move(th));
                 }
