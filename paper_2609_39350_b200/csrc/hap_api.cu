@@ -1084,7 +1084,7 @@ extern "C" hap_status hap_decode(hap_problem *p, uint64_t first, uint64_t count,
     if (!dev_out) return HAP_E_INVALID;
     const uint64_t blocks = (count + 3) / 4;
     if (blocks > 0x7fffffffull) return fail(p, HAP_E_RANGE, "count too large for one launch");
-    decode_kernel<<<(unsigned)blocks, 128, 0, (cudaStream_t)stream>>>(p->dc, first, count, dev_out);
+    decode_kernel<<<(unsigned)blocks, 128, 0, (cudaStream_t)stream>>>(p->dc, first, count, dev_out, nullptr);
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
 }
@@ -1232,7 +1232,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     for (const hap_problem::PpClass *clp : order) {
         const hap_problem::PpClass &cl = *clp;
         // skip classes whose candidates all lie outside the range
-        if (!search && class_outside(p, cl, out)) continue;
+        if (!search && !out.first_dev && class_outside(p, cl, out)) continue;     // (a range that starts at a device-side index: every class looks)
         const bool lin = p->dc.tau_linear != 0;
         const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
         const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (refine ? 8 : 0) + (search ? 2 : 0) + (lin ? 1 : 0);
@@ -1393,7 +1393,7 @@ extern "C" hap_status hap_search_range_f64(hap_problem *p, uint64_t first, uint6
     one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
     one.recompute = d1->rec; one.first = win; one.count = 1;
     if ((s = launch_dp(p, one, false, st, true)) != HAP_OK) return s;
-    decode_kernel<<<1, 32, 0, st>>>(p->dc, win, 1, &d1->cand);
+    decode_kernel<<<1, 32, 0, st>>>(p->dc, win, 1, &d1->cand, nullptr);
     CUDA_TRY(p, cudaGetLastError());
     SingleOut h1;
     CUDA_TRY(p, cudaMemcpyAsync(&h1, d1, sizeof(h1), cudaMemcpyDeviceToHost, st));
@@ -1793,10 +1793,22 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     CUDA_TRY(p, cudaGetLastError());
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
+    // the winner is evaluated once more alone, for its partition and recomputation levels; its index stays on the
+    // device (every class's kernel looks whether the index is its own), so the host waits only once
+    SingleOut *d1 = (SingleOut *)p->d_single;
+    DpOut one{};
+    one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
+    one.recompute = d1->rec; one.first = 0; one.count = 1; one.first_dev = p->d_best + 1;
+    if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
+    decode_kernel<<<1, 32, 0, st>>>(p->dc, 0, 1, &d1->cand, p->d_best + 1);
+    CUDA_TRY(p, cudaGetLastError());
     i64 best[2];
-    u64 counters[4];
+    u64 counters[4], flag = 0;
+    SingleOut h1;
     CUDA_TRY(p, cudaMemcpyAsync(best, p->d_best, sizeof(best), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(p, cudaMemcpyAsync(counters, p->d_counters, sizeof(counters), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaMemcpyAsync(&flag, p->d_range, sizeof(flag), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaMemcpyAsync(&h1, d1, sizeof(h1), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(p, cudaStreamSynchronize(st));
     if (host_stats) {
         std::memset(host_stats, 0, sizeof(*host_stats));
@@ -1806,23 +1818,11 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
         cudaEventElapsedTime(&host_stats->ms_dp, p->ev[1], p->ev[2]);
         host_stats->ms_total = host_stats->ms_layer_cost + host_stats->ms_dp;
     }
-    if ((s = check_values(p)) != HAP_OK) return s;
+    if (flag) return fail(p, HAP_E_RANGE, "a layer time or stage coefficient exceeds the supported range (see hap.h)");
     if (best[0] >= kInf) return fail(p, HAP_E_INFEASIBLE, "no candidate satisfies the memory constraint");
-
-    // re-evaluate the winner alone to obtain its partition and recomputation levels
     const u64 win = (u64)best[1];
-    SingleOut *d1 = (SingleOut *)p->d_single;
-    DpOut one{};
-    one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
-    one.recompute = d1->rec; one.first = win; one.count = 1;
-    if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
-    decode_kernel<<<1, 32, 0, st>>>(p->dc, win, 1, &d1->cand);
-    CUDA_TRY(p, cudaGetLastError());
-    SingleOut h1;
-    CUDA_TRY(p, cudaMemcpyAsync(&h1, d1, sizeof(h1), cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(p, cudaStreamSynchronize(st));
     const hap_candidate &hc = h1.cand;
-    if (h1.cost != best[0]) return fail(p, HAP_E_CUDA, "winner re-evaluation disagrees with the search");
+    if (h1.cost != best[0] || hc.index != win) return fail(p, HAP_E_CUDA, "winner re-evaluation disagrees with the search");
     const hap_pconf &pc = p->pconfs[hc.pconf];
     host_out->index = win;
     host_out->PP = pc.PP; host_out->TP = pc.TP; host_out->CP = pc.CP; host_out->DP = pc.DP; host_out->EP = pc.EP;

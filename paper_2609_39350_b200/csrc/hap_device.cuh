@@ -95,6 +95,7 @@ struct DpOut {
     uint8_t *choice;
     i64 *detail;                      // [count][3] T_pipe, T_sync, T_opt (nullable)
     u64 first, count;                 // global candidate range that is written
+    const i64 *first_dev;             // if set: `first` is read from here by the kernel (a negative value: nothing is written)
     // search mode
     i64 *partial_cost;                // [gridDim.x]
     u64 *partial_index;               // [gridDim.x]
@@ -567,11 +568,16 @@ __device__ __forceinline__ u64 find_pconf(const DevConst &dc, u64 c)
     return lo;
 }
 
-__global__ void decode_kernel(const DevConst dc, u64 first, u64 count, hap_candidate *out)
+__global__ void decode_kernel(const DevConst dc, u64 first, u64 count, hap_candidate *out, const i64 *first_dev)
 {
     const u64 w = ((u64)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (w >= count) return;
+    if (first_dev) {                    // the index a preceding kernel left in device memory (negative: none)
+        const i64 f = *first_dev;
+        if (f < 0) return;
+        first = (u64)f;
+    }
     const u64 c = first + w;
     const u64 p = find_pconf(dc, c);
     const hap_pconf pc = dc.pconf[p];
@@ -1075,6 +1081,11 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
     // c2: layer times; coef: integer coefficients (memory bytes); coefv: time coefficients in the value type
     // (the same array as coef in integer mode)
     const VT vInf = ValInf<VT>::get();
+    if (out.first_dev) {
+        // the range starts at an index a preceding kernel left in device memory (the winner of a search)
+        const i64 f = *out.first_dev;
+        out.first = f < 0 ? (~0ull >> 1) : (u64)f;
+    }
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1;
     const int wib = threadIdx.x >> 5, lane = threadIdx.x & 31;
