@@ -285,6 +285,21 @@ def main():
         b.synchronize()
         joint_ms = a.elapsed_time(b)
 
+    # the same pass in fp64 mode (unrounded times; context, the bench line is the integer mode)
+    fp64_ms = None
+    if world == 1:
+        ts = []
+        for it in range(5):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            hap.hap_pipeline_dp_f64(hp, first, count)
+            b.record(stream)
+            b.synchronize()
+            if it >= 2:
+                ts.append(a.elapsed_time(b))
+        fp64_ms = statistics.median(ts)
+
     # the same pass with the refinement (smallest stage-cost sum among the bottleneck-optimal partitions) and with
     # the exact optimisation of sum + (M-1) max (limit sweep); untimed extras
     extra_modes = {}
@@ -388,6 +403,7 @@ def main():
             gpu_launches=hap.hap_launches_per_pass(hp) * args.steps,
             **extra_modes,
             joint_recurrence_ms=joint_ms,
+            fp64_mode_pass_ms=fp64_ms,
             appendix_b_best_plan=appb,
             full_search_ms=statistics.median(search_ms),
             full_search_pruned=dict(ms=statistics.median(pruned_ms), n_pruned=stats_pr["n_pruned"],
