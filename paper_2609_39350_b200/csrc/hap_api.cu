@@ -1802,14 +1802,21 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
     decode_kernel<<<1, 32, 0, st>>>(p->dc, 0, 1, &d1->cand, p->d_best + 1);
     CUDA_TRY(p, cudaGetLastError());
+    // range flag, counters, minimum and the re-evaluated winner sit in consecutive 256-byte slots at the end of the
+    // arena: one copy brings all four back
+    alignas(16) unsigned char tail[3 * 256 + sizeof(SingleOut)];
+    if ((unsigned char *)p->d_counters - (unsigned char *)p->d_range != 256 || (unsigned char *)p->d_best - (unsigned char *)p->d_range != 512 ||
+        (unsigned char *)p->d_single - (unsigned char *)p->d_range != 768)
+        return fail(p, HAP_E_STATE, "result slots are not adjacent");
+    CUDA_TRY(p, cudaMemcpyAsync(tail, p->d_range, sizeof(tail), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(p, cudaStreamSynchronize(st));
     i64 best[2];
     u64 counters[4], flag = 0;
     SingleOut h1;
-    CUDA_TRY(p, cudaMemcpyAsync(best, p->d_best, sizeof(best), cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(p, cudaMemcpyAsync(counters, p->d_counters, sizeof(counters), cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(p, cudaMemcpyAsync(&flag, p->d_range, sizeof(flag), cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(p, cudaMemcpyAsync(&h1, d1, sizeof(h1), cudaMemcpyDeviceToHost, st));
-    CUDA_TRY(p, cudaStreamSynchronize(st));
+    std::memcpy(&flag, tail, sizeof(flag));
+    std::memcpy(counters, tail + 256, sizeof(counters));
+    std::memcpy(best, tail + 512, sizeof(best));
+    std::memcpy(&h1, tail + 768, sizeof(h1));
     if (host_stats) {
         std::memset(host_stats, 0, sizeof(*host_stats));
         host_stats->n_pconf = p->pconfs.size(); host_stats->n_candidates = p->n_cand;
