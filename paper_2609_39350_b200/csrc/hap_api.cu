@@ -626,35 +626,52 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
     }
     std::vector<u32> first_leaf(n_nodes);
     std::vector<uint8_t> depth(n_nodes);
-    for (int d = 1; d < PP; ++d)
+    for (int d = 1; d < PP; ++d) {
+        // per-depth extremes are gathered in locals (the description's byte fields alias everything the loop writes)
+        int d_jlo = 255, d_jhi = 0, d_wmax = 0, d_kmin = 255, d_kmax = 0;
+        unsigned d_tmask = 0;
+        const u32 node_lo = tm.node_lo[d], cell_lo = tm.cell_lo[d];
+        const u32 *ro = rowoff[d].data();
+        TrieCell *cd = cells.data();
+        u32 *gn = cell_gnode.data();
         for (size_t i = 0; i < lv[d].size(); ++i) {
             const HNode &h = lv[d][i];
-            TrieNode &nd = nodes[tm.node_lo[d] + i];
-            nd.rowoff = rowoff[d][i];
+            TrieNode nd{};
+            nd.rowoff = ro[i];
             nd.mask = h.k.mask; nd.link = h.k.link; nd.nmin = h.k.nmin; nd.nmax = h.k.nmax;
             nd.bl = (uint8_t)h.bl; nd.bh = (uint8_t)h.bh;
             if (d > 1) { const HNode &ph = lv[d - 1][h.parent]; nd.prowoff = rowoff[d - 1][h.parent]; nd.pbl = (uint8_t)ph.bl; nd.pbh = (uint8_t)ph.bh; }
             else { nd.prowoff = 0; nd.pbl = 0; nd.pbh = 0; }
-            parent[tm.node_lo[d] + i] = (uint16_t)h.parent;
-            first_leaf[tm.node_lo[d] + i] = h.first_leaf;
-            depth[tm.node_lo[d] + i] = (uint8_t)d;
-            tm.jlo[d] = std::min<uint8_t>(tm.jlo[d], nd.bl); tm.jhi[d] = std::max<uint8_t>(tm.jhi[d], nd.bh);
-            tm.wmax[d] = std::max(tm.wmax[d], nd.nmax);
-            tm.tmask[d] |= (uint8_t)(1u << capt_of[nd.mask]);
-            for (int j = h.bl; j <= h.bh; ++j) {
-                int klo = std::max(j - (int)nd.nmax, (int)nd.pbl), khi = std::min(j - (int)nd.nmin, (int)nd.pbh);
+            nodes[node_lo + i] = nd;
+            parent[node_lo + i] = (uint16_t)h.parent;
+            first_leaf[node_lo + i] = h.first_leaf;
+            depth[node_lo + i] = (uint8_t)d;
+            d_jlo = std::min<int>(d_jlo, nd.bl); d_jhi = std::max<int>(d_jhi, nd.bh);
+            d_wmax = std::max<int>(d_wmax, nd.nmax);
+            d_tmask |= 1u << capt_of[nd.mask];
+            const int cls = nd.link & 3, ha = (nd.link >> 2) & 3, hb = (nd.link >> 4) & 3;
+            const u32 kidx = d == 1 ? tm.mrow_of[nd.mask] : 16 + hb * 6 + (cls == HAP_CROSS ? 2 + ha : cls);
+            const u32 cx = (u32)((int)nd.prowoff - (int)nd.pbl + 256) | (kidx << 26);
+            const u32 cw = (u32)tm.mrow_of[nd.mask] * (u32)(R * (N + 1));
+            const u32 g = node_lo + (u32)i;
+            const int nmx = nd.nmax, nmn = nd.nmin, pbl = nd.pbl, pbh = nd.pbh;
+            u32 c = cell_lo + ro[i];
+            for (int j = h.bl; j <= h.bh; ++j, ++c) {
+                int klo = std::max(j - nmx, pbl), khi = std::min(j - nmn, pbh);
                 if (klo > khi) { klo = 1; khi = 0; }
-                else { tm.kmin[d] = std::min<uint8_t>(tm.kmin[d], (uint8_t)klo); tm.kmax[d] = std::max<uint8_t>(tm.kmax[d], (uint8_t)khi); }
-                const u32 c = tm.cell_lo[d] + rowoff[d][i] + (u32)(j - h.bl);
-                const int cls = nd.link & 3, ha = (nd.link >> 2) & 3, hb = (nd.link >> 4) & 3;
-                const u32 kidx = d == 1 ? tm.mrow_of[nd.mask] : 16 + hb * 6 + (cls == HAP_CROSS ? 2 + ha : cls);
-                cells[c].x = (u32)((int)nd.prowoff - (int)nd.pbl + 256) | (kidx << 26);
-                cells[c].y = (u32)j | ((u32)klo << 8) | ((u32)khi << 16);
-                cells[c].z = 0;                                   // threshold index: needs the depth's first end layer, set below
-                cells[c].w = (u32)tm.mrow_of[nd.mask] * (u32)(R * (N + 1));
-                cell_gnode[c] = tm.node_lo[d] + (u32)i;
+                else { d_kmin = std::min(d_kmin, klo); d_kmax = std::max(d_kmax, khi); }
+                TrieCell cc;
+                cc.x = cx;
+                cc.y = (u32)j | ((u32)klo << 8) | ((u32)khi << 16);
+                cc.z = 0;                                         // threshold index: needs the depth's first end layer, set below
+                cc.w = cw;
+                cd[c] = cc;
+                gn[c] = g;
             }
         }
+        tm.jlo[d] = (uint8_t)d_jlo; tm.jhi[d] = (uint8_t)d_jhi; tm.wmax[d] = (uint8_t)d_wmax;
+        tm.tmask[d] = (uint8_t)d_tmask; tm.kmin[d] = (uint8_t)d_kmin; tm.kmax[d] = (uint8_t)d_kmax;
+    }
     for (int d = 1; d <= PP; ++d) if (tm.jlo[d] <= tm.jhi[d]) band_max = std::max(band_max, tm.jhi[d] - tm.jlo[d] + 1);
     for (u64 m = 0; m < nmap; ++m) {
         TrieLeaf &lf = leaves[m];
