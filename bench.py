@@ -33,6 +33,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}
 # dram__bytes_read.sum + dram__bytes_write.sum of the DP launches of one pass, from the ncu capture summarised
 # in profiles/trie_dp_kernel_stress.md
 NCU_DP_TRAFFIC_BYTES = {"stress": 54.6e6}
+# the same for type_const_kernel + layer_cost_kernel (profiles/layer_cost_kernel_stress.md): 0.68 + 4.2 MB read and
+# 0.31 MB written while they run; the 47.8 MB of layer costs they produce are still in L2 when they end
+NCU_LC_TRAFFIC_BYTES = {"stress": 5.2e6}
 
 
 def read_peaks():
@@ -424,7 +427,7 @@ def main():
                           f"{peaks.get('sm_max_mhz', 1965.0)} MHz ({peak_kind} clock)", sm_mhz_seen=sm_mhz),
             roofline_layer_cost=dict(bound="hbm", kernel="type_const_kernel + layer_cost_kernel (hap_eval_layer_costs alone)",
                                      achieved=lc_gbs, peak=peaks["hbm_gbs"],
-                                     unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=None,
+                                     unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=NCU_LC_TRAFFIC_BYTES.get(args.workload),
                                      bytes_per_launch=16 * units, ms_alone=lc_alone_ms, ms_in_pass=lc_med,
                                      ms_plain_fill_of_the_same_bytes=fill_same_bytes_ms,
                                      peak_source=f"hbm_gbs ({peak_kind})"),
