@@ -11,6 +11,7 @@ import pytest
 from gen import problems
 from gen.problems import DENSE, MOE
 from oracle import Oracle, INF, COEF, NCOEF, Mapping
+from hand_examples import e8_problem, e9_problem
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -967,3 +968,102 @@ def test_oracle_1f1b_simulation_against_the_python_schedule_on_searched_plans():
             assert r.T_iter == r.T_pipe_sim + r.T_sync + r.T_opt
             checked += 1
     assert checked > 80
+
+
+# --------------------------------------------------------------------------------------
+# Eq. 4's synchronisation and optimizer terms over the stages; stages that span two device types
+# --------------------------------------------------------------------------------------
+def _check_plan(o, index, want):
+    pl, _, _ = o.eval_index(index)
+    for key in ("n", "c", "bottleneck", "T_pipe", "T_sync", "T_opt", "T_iter"):
+        assert pl[key] == want[key], (index, key, pl[key], want[key])
+    if "r" in want:
+        assert pl["r"] == want["r"]
+    return pl
+
+
+def test_e8_sync_and_optimizer_terms_are_the_slowest_stage_of_each():
+    g = gold("e8_sync_opt_assembly.json")["expect"]
+    o = Oracle(e8_problem())
+    assert (o.n_pconf, o.n_cand) == (1, 6)
+    assert [int(o.pconfs[k][0]) for k in ("PP", "DP", "EDP", "M", "G")] == [3, 4, 4, 4, 4]
+    _, _, coef, _ = o.layer_costs(0)
+    for h, name in enumerate("ABC"):
+        assert [coef[h, COEF["SBW"]], coef[h, COEF["SBW"] + 1]] == g["coef"]["sbw"][name]
+        assert [coef[h, COEF["OPT"]], coef[h, COEF["OPT"] + 1]] == g["coef"]["opt"][name]
+        assert coef[h, COEF["SLAT"]] == g["coef"]["slat"]
+        assert all(coef[h, COEF["KP2P_CROSS"] + h2] == g["coef"]["kp2p_cross"] for h2 in range(3))
+    for name in ("ABC", "BAC"):
+        want = g[name]
+        mp = o.decode(0, want["map_idx"])
+        assert [int(m).bit_length() - 1 for m in mp.mask[:3]] == ["ABC".index(ch) for ch in name]
+        _check_plan(o, want["map_idx"], want)
+    # the three terms are decided by three different stages in the first mapping, so none of the plausible
+    # mistakes (sum over stages, the bottleneck stage's own terms, one stage for both terms) reproduces it
+    a = g["ABC"]
+    assert a["T_iter"] == a["T_pipe"] + a["T_sync"] + a["T_opt"]
+    assert a["c"].index(a["bottleneck"]) == 0 and a["T_sync"] == 12000 + 2 * 660741 and a["T_opt"] == 3 * 352395
+
+
+def test_e9_stage_spanning_two_device_types():
+    g = gold("e9_mixed_type_stage.json")["expect"]
+    o = Oracle(e9_problem())
+    assert (o.n_pconf, o.n_cand) == (1, 2)
+    assert int(o.pconfs["nmap"][0]) == 2 and int(o.pconfs["G"][0]) == 4 and int(o.pconfs["M"][0]) == 4
+    c2, _, coef, _ = o.layer_costs(0)
+    m = g["mem_coef"]
+    assert coef[0, COEF["MW"] + MOE] == m["mw"] and coef[0, COEF["MA"] + MOE] == m["ma"]
+    assert coef[0, COEF["MX"]] == m["mx"] and coef[0, COEF["MPRE"]] == m["mpre"] == coef[0, COEF["MPOST"]]
+    for name in ("AB", "BA"):
+        want = g[name]
+        mp = o.decode(0, want["map_idx"])
+        assert [int(x) for x in mp.mask[:2]] == g["masks"][name]
+        assert int(mp.cls[1]) == 0                      # the boundary lies inside type A's node
+        lo, hi = o.window(0, mp)
+        assert [[int(lo[s]), int(hi[s])] for s in range(2)] == g["window"][name]
+        pl = _check_plan(o, want["map_idx"], want)
+        assert pl["mask"] == g["masks"][name]
+    mp = o.decode(0, 0)
+    for n2, (cost, level) in g["stage2_AB_spans"].items():
+        assert o.stage_cost(0, mp, 0b11, c2, coef, 2, 8 - int(n2), 8) == (cost, level)
+    # without recomputation the mixed stage holds one layer only (B's 2 GiB), which the window still allows
+    assert o.stage_cost(0, mp, 0b01, c2, coef, 2, 6, 8)[0] == INF
+    assert o.stage_cost(0, mp, 0b01, c2, coef, 2, 7, 8) == (1314486, 0)
+    costs, _, best, _ = o.search()
+    assert costs.tolist() == [g["AB"]["T_iter"], g["BA"]["T_iter"]] and best["index"] == g["best_index"]
+
+
+@pytest.mark.parametrize("make, gname, names", [(e8_problem, "e8_sync_opt_assembly.json", ("ABC", "BAC")),
+                                                (e9_problem, "e9_mixed_type_stage.json", ("AB", "BA"))])
+def test_every_objective_variant_assembles_sync_and_optimizer_terms_alike(make, gname, names):
+    """The hand examples have one optimal partition under every objective (smallest bottleneck, smallest sum under
+    it, exact pipeline term), so the refinement, the exact sweep, the fp64 mode and the post-hoc evaluators must
+    report the hand-computed T_sync and T_opt as well."""
+    g = gold(gname)["expect"]
+    o = Oracle(make())
+    c2, _, coef, _ = o.layer_costs(0)
+    for name in names:
+        want = g[name]
+        for got in (o.eval_index_refined(want["map_idx"]), o.eval_index_exact(want["map_idx"])):
+            for key in ("n", "c", "bottleneck", "T_pipe", "T_sync", "T_opt", "T_iter"):
+                assert got[key] == want[key], (name, key)
+        mp = o.decode(0, want["map_idx"])
+        r = want.get("r", [0] * len(want["n"]))
+        for res in (o.appendix_b(0, mp, c2, coef, want["n"], r), o.simulate_1f1b(0, mp, c2, coef, want["n"], r)):
+            assert (int(res.T_sync), int(res.T_opt)) == (want["T_sync"], want["T_opt"])
+        f = o.eval_index_f64(want["map_idx"])
+        assert f["n"] == want["n"]
+        for key in ("T_sync", "T_opt", "T_pipe", "T_iter"):      # fp64 mode keeps the coefficients unrounded
+            assert abs(f[key] - want[key]) <= 1.0 * (len(want["n"]) + 8), (name, key, f[key])
+
+
+def test_e8_fp64_mode_hand_values():
+    # unrounded terms of the first mapping: sync 12000 + 2*660741.12, optimizer 3*352395.264,
+    # transfers 503349.0285714...; T_pipe = 9e6 + (6e6 + x) + (7.2e6 + x) + 3*9e6 with x the transfer
+    o = Oracle(e8_problem())
+    f = o.eval_index_f64(0)
+    x = 2.0 * (12000.0 + 4194304.0 / 17.5)
+    assert f["T_sync"] == pytest.approx(1333482.24, rel=1e-13)
+    assert f["T_opt"] == pytest.approx(1057185.792, rel=1e-13)
+    assert f["T_pipe"] == pytest.approx(49200000.0 + 2.0 * x, rel=1e-13)
+    assert f["T_iter"] == pytest.approx(49200000.0 + 2.0 * x + 1333482.24 + 1057185.792, rel=1e-13)
