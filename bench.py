@@ -30,13 +30,6 @@ METRIC = "candidate_plans_per_second"
 UNIT = "candidates/s"
 SM_COUNT, SCHEDULERS_PER_SM, LANES = 148, 4, 32
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of the DP launches of one pass, from the ncu capture summarised
-# in profiles/trie_dp_kernel_stress.md
-NCU_DP_TRAFFIC_BYTES = {"stress": 54.6e6}
-# the same for type_const_kernel + layer_cost_kernel (profiles/layer_cost_kernel_stress.md): 0.68 + 4.2 MB read and
-# 0.31 MB written while they run; the 47.8 MB of layer costs they produce are still in L2 when they end
-NCU_LC_TRAFFIC_BYTES = {"stress": 5.2e6}
-
 
 def read_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -246,6 +239,13 @@ def main():
     value = n_cand * args.steps / (total_ms * 1e-3)
 
     cells_finite = hap.hap_count_cells(hp, first, count)        # untimed instrumentation launch
+    # untimed: the same pass through the counting form of the kernels -> splits evaluated after all early exits
+    hp_cnt = hap.hap_problem_create(pb, flags=hap.OPT_COUNT_SPLITS)
+    hap.hap_enumerate(hp_cnt)
+    hap.hap_pipeline_dp(hp_cnt, first, count, out=out)
+    torch.cuda.synchronize()
+    cells = hap.hap_get_timings(hp_cnt)[2]
+    hap.hap_problem_destroy(hp_cnt)
 
     # the layer-cost kernels alone (inside a pass the candidate decode of the classes runs beside them on other
     # streams, so the pass's own phase time is not the kernels' time), L2 flushed, CUDA events on the launching stream
@@ -375,6 +375,15 @@ def main():
         plan2, _ = hap.hap_search_range(hp2, first, count)
         e2e_ms.append(1e3 * (time.perf_counter() - t0))
         hap.hap_problem_destroy(hp2)
+    # the same once more with the library's cache of device memory emptied first (the allocations are then the driver's)
+    hap.hap_release_cached_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    hp2 = hap.hap_problem_create(pb)
+    hap.hap_enumerate(hp2)
+    hap.hap_search_range(hp2, first, count)
+    e2e_uncached_ms = 1e3 * (time.perf_counter() - t0)
+    hap.hap_problem_destroy(hp2)
     e2e_t = torch.tensor([statistics.median(e2e_ms)], dtype=torch.float64, device=xdev)
     if world > 1:
         dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
@@ -384,11 +393,16 @@ def main():
         peaks, peak_kind = read_peaks()
         dp_med, lc_med = statistics.median(dp_ms), statistics.median(lc_ms)
         sm_mhz = clocks["sm_mhz"] or peaks.get("sm_max_mhz", 1965.0)
-        alu_peak = SM_COUNT * SCHEDULERS_PER_SM * LANES * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
-        # algorithmic work of the DP kernel: 4 semiring operations (prefix difference, max, min, arg-select) per
-        # cell update of the plain recurrence, 2w + (PP-2)w(w+1)/2 cells per candidate with w = N-PP+1
+        # issue-slot peak at the clock sampled during the timed region
+        alu_peak = SM_COUNT * SCHEDULERS_PER_SM * LANES * float(sm_mhz) * 1e6 / 1e12
+        # Work of the DP phase, three ways, all at 4 semiring operations (prefix difference, max, min, arg-select)
+        # per split: `executed` = the splits the kernels evaluated (counted by the kernels, after windows, bands,
+        # shared stage prefixes and early exits) -- this is what the fraction reports; `finite` = the splits of the
+        # recurrence whose stage cost is finite, per candidate, nothing shared; `plain` = the recurrence without
+        # the window, 2w + (PP-2)w(w+1)/2 per candidate with w = N-PP+1.  The last two say how much work the tree
+        # form avoids; they are not utilisation figures.
         cells_plain = float(sum(recurrence_cells(pb.N, int(r["PP"])) * int(r["nmap"]) * len(pb.rc_masks) for r in pconfs))
-        achieved = 4.0 * cells_finite / (dp_med * 1e-3) / 1e12
+        achieved = 4.0 * cells / (dp_med * 1e-3) / 1e12
         units = n_pconf * hp.T * pb.N
         lc_gbs = 16.0 * units / (lc_alone_ms * 1e-3) / 1e9
         line = dict(
@@ -401,8 +415,10 @@ def main():
                         parallelism=f"candidate ranges over {world} gpu(s)"),
             clocks=dict(sm_mhz=clocks["sm_mhz"], sm_max_mhz=clocks["sm_max_mhz"], reasons=clocks["reasons"]),
             e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-                     ms=float(e2e_t.item()), what="hap_problem_create + hap_enumerate + hap_search_best from host buffers"),
-            # per step: type_const, layer_cost, per PP class (decode, tree gather per part, tree DP), argmin partial + final
+                     ms=float(e2e_t.item()), ms_without_cached_device_memory=e2e_uncached_ms,
+                     what="hap_problem_create + hap_enumerate + hap_search_best from host buffers (median of 3; the "
+                          "process keeps freed device memory and the classes' prefix trees between problems)"),
+            # per step: type_const, one decode and one tree-gather launch, one tree DP launch per PP class, argmin partial + final
             gpu_launches=hap.hap_launches_per_pass(hp) * args.steps,
             **extra_modes,
             joint_recurrence_ms=joint_ms,
@@ -412,24 +428,26 @@ def main():
             full_search_pruned=dict(ms=statistics.median(pruned_ms), n_pruned=stats_pr["n_pruned"],
                                     n_evaluated=stats_pr["n_evaluated"]),
             best=dict(cost=best[0], index=best[1], search_index=plan["index"]),
-            kernels_ms=dict(layer_cost=lc_med, pipeline_dp=dp_med),
+            kernels_ms=dict(type_constants=lc_med, pipeline_dp=dp_med),
             roofline=dict(bound="alu", kernel="trie_dp_kernel (one launch per PP class, concurrent streams)",
                           achieved=achieved, peak=alu_peak, unit="Tops/s", frac=achieved / alu_peak,
-                          traffic=NCU_DP_TRAFFIC_BYTES.get(args.workload) if args.delta_q is None else None,
-                          ops_per_cell=4, cells_finite_cost=cells_finite, cells_plain_recurrence=cells_plain,
-                          cells_visited=cells, frac_plain_recurrence=4.0 * cells_plain / (dp_med * 1e-3) / 1e12 / alu_peak,
-                          note="achieved = 4 ops x cells whose stage cost is finite (inside the load-balance window and "
-                               "the memory limit), counted per candidate; the kernel visits fewer (cells_visited) because "
-                               "unreachable layers are skipped and the rows of a stage prefix are computed once for all "
-                               "mappings that share it, and the plain recurrence without the window would have "
-                               "cells_plain_recurrence",
+                          traffic=None, ops_per_split=4, splits_executed=cells,
+                          effective_finite=dict(cells=cells_finite, tops=4.0 * cells_finite / (dp_med * 1e-3) / 1e12),
+                          effective_plain_recurrence=dict(cells=cells_plain, tops=4.0 * cells_plain / (dp_med * 1e-3) / 1e12),
+                          note="achieved = 4 ops x splits the kernels evaluated / CUDA-event time of the DP phase; the "
+                               "effective_* figures divide the work of the per-candidate recurrence (finite-cost splits; "
+                               "every split without the window) by the same time and measure what the shared prefix tree, "
+                               "bands and early exits avoid, not utilisation; traffic: not measured by this run",
                           peak_source=f"{SM_COUNT} SMs x {SCHEDULERS_PER_SM} schedulers x {LANES} lanes x "
-                          f"{peaks.get('sm_max_mhz', 1965.0)} MHz ({peak_kind} clock)", sm_mhz_seen=sm_mhz),
-            roofline_layer_cost=dict(bound="hbm", kernel="type_const_kernel + layer_cost_kernel (hap_eval_layer_costs alone)",
+                          f"{sm_mhz} MHz (clock sampled during the timed region)", sm_mhz_seen=sm_mhz),
+            roofline_layer_cost=dict(bound="hbm", kernel="type_const_kernel + layer_cost_kernel (hap_eval_layer_costs alone; "
+                                     "the pass itself computes layer costs inside the DP blocks and writes none)",
                                      achieved=lc_gbs, peak=peaks["hbm_gbs"],
-                                     unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=NCU_LC_TRAFFIC_BYTES.get(args.workload),
-                                     bytes_per_launch=16 * units, ms_alone=lc_alone_ms, ms_in_pass=lc_med,
+                                     unit="GB/s", frac=lc_gbs / peaks["hbm_gbs"], traffic=None,
+                                     bytes_per_launch=16 * units, ms_alone=lc_alone_ms, ms_before_dp_in_pass=lc_med,
                                      ms_plain_fill_of_the_same_bytes=fill_same_bytes_ms,
+                                     note="achieved = 16 B per (configuration, type, layer) unit written / time of the call "
+                                          "alone after an L2 flush; the output may still sit in L2 when the call ends",
                                      peak_source=f"hbm_gbs ({peak_kind})"),
             wall_s=t_wall,
         )

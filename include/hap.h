@@ -139,6 +139,11 @@ typedef struct {
 #define HAP_OPT_NO_MAPTAB 1   /* keep no table of decoded mappings on the device: the DP kernel unranks each mapping itself */
 #define HAP_OPT_NO_TRIE 16    /* keep no prefix tree of the mappings: every pass runs one warp per candidate (the tree form
                                  shares the DP rows of common stage prefixes between all mappings of a configuration) */
+#define HAP_OPT_NO_FUSE 32    /* passes that walk the prefix trees let every block compute the layer times of its configuration itself
+                                 (Eq. 2) instead of reading an array that a layer-cost launch wrote before; this flag keeps the
+                                 separate launch (identical results) */
+#define HAP_OPT_COUNT_SPLITS 64 /* instrumentation: hap_pipeline_dp passes of this problem also count the splits (k, j) their kernels
+                                 evaluate, after all early exits, for hap_get_timings; costs a few percent of the pass */
 #define HAP_OPT_UNIFORM 8     /* ablation "non-uniform partitioning disabled" (Sec. 5.5): every stage takes floor(N/PP) or
                                  ceil(N/PP) layers; the load-balance window is ignored */
 #define HAP_OPT_EXACT 4       /* like HAP_OPT_REFINE, but the limit on the stage cost is then swept upward from the bottleneck over
@@ -309,9 +314,12 @@ hap_status hap_joint_bottleneck(hap_problem *, int64_t *dev_out, void *stream);
 hap_status hap_count_cells(hap_problem *, uint64_t first, uint64_t count, uint64_t *host_cells, void *stream);
 
 /* Measurement aid: CUDA-event durations (ms) of the layer-cost kernel and of the dynamic-program
- * kernel of the most recent hap_pipeline_dp / hap_search_* call, and the number of recurrence cell
- * updates (k, j pairs inside the window and the memory limit) that launch evaluated.  Waits for that
- * call's kernels.  Any output may be NULL. */
+ * kernel of the most recent hap_pipeline_dp / hap_search_* call, and -- for a problem created with
+ * HAP_OPT_COUNT_SPLITS, 0 otherwise -- the number of splits (k, j pairs inside the window and the memory limit) that
+ * a hap_pipeline_dp launch evaluated, counted after its early exits: the work executed, as opposed to
+ * hap_count_cells, the work the recurrence defines.  ms_layer_cost covers what precedes the
+ * dynamic program in the pass (the per-type constants and stage coefficients, and the layer-cost launch when the
+ * pass has one).  Waits for that call's kernels.  Any output may be NULL. */
 hap_status hap_get_timings(hap_problem *, float *ms_layer_cost, float *ms_dp, uint64_t *cells);
 
 /* Appendix B: the iteration latency of GIVEN plans with the steady-state term written through the index s_max of

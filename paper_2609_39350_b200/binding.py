@@ -149,6 +149,8 @@ OPT_REFINE = 2
 OPT_EXACT = 4
 OPT_UNIFORM = 8
 OPT_NO_TRIE = 16
+OPT_NO_FUSE = 32
+OPT_COUNT_SPLITS = 64
 
 
 def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:

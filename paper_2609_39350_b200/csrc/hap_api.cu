@@ -11,6 +11,7 @@
 #include <cstring>
 #include <array>
 #include <map>
+#include <memory>
 #include <mutex>
 #include <new>
 #include <string>
@@ -43,7 +44,9 @@ struct hap_problem {
                          u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
     struct Trie { bool ok = false; TrieMeta *d_metas = nullptr; u32 *d_plist = nullptr;       // both inside d_trie_arena
                   std::vector<TriePartDev> parts; unsigned n_conf = 0; int threads = 0; size_t smem = 0; };
-    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie; };
+    struct PpClass { int PP; int warps; size_t smem; size_t item_lo, item_hi; u64 map_base; bool has_tab; bool multiset; unsigned masks_used; cudaStream_t stream; cudaEvent_t done; Trie trie;
+                     mutable bool tab_valid = false;        // the device table of decoded mappings of this class has been filled
+                     size_t pslot_lo = 0, pslot_n = 0; };   // the class's slots in the per-block partial minima of a search
     std::vector<PpClass> classes;
     uint8_t *d_maptab = nullptr;           // decoded mappings of every class that is small enough
     unsigned char *d_arena = nullptr;      // everything hap_enumerate sizes, in one allocation (the d_* pointers below point into it)
@@ -70,7 +73,8 @@ struct hap_problem {
     u64 *d_counters = nullptr;             // [0] evaluated [1] feasible [2] pruned [3] incumbent
     i64 *d_best = nullptr;                 // (cost, index) of the search
     void *d_single = nullptr;              // outputs of the one-candidate re-evaluation
-    size_t n_partial = 0;
+    size_t n_partial = 0;                  // allocated slots of the partial minima
+    size_t n_pslots = 0;                   // slots a search pass writes and reduces (sum of the classes' pslot_n)
     bool timed = false;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     cudaEvent_t ev_fork = nullptr;          // classes run on their own streams between this event and their `done` events
@@ -727,13 +731,15 @@ static bool build_trie_part(hap_problem *p, const hap_problem::PpClass &cl, cons
 // Builds the class's tree, as one part or, when one part would leave room for only one block per SM, as up to
 // eight parts over contiguous ranges of mappings (the few nodes near the root that two parts share are computed by
 // both).  Returns false (the class stays on the general kernel) when nothing fits.
-struct TrieClassHost { std::vector<TriePartHost> parts; std::vector<u32> plist; };
+struct TrieClassHost { std::vector<TriePartHost> parts; unsigned masks_used = 0xffffffffu; };
+// what upload_tries gets per class: the class, its (shared) host tree and the class's configurations
+struct TrieBuilt { hap_problem::PpClass *cl; std::shared_ptr<const TrieClassHost> tree; std::vector<u32> plist; };
 
-static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, const std::vector<u32> &plist, TrieClassHost &out)
+static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *tab, u64 nmap, size_t n_conf, TrieClassHost &out)
 {
-    if (nmap == 0 || plist.empty()) return false;
+    if (nmap == 0 || n_conf == 0) return false;
     constexpr size_t kTwoPerSm = 108 * 1024;                 // dynamic shared memory that lets two blocks share an SM
-    const size_t slots = (cl.item_hi - cl.item_lo) / plist.size();       // partial-result slots per configuration
+    const size_t slots = (cl.item_hi - cl.item_lo) / n_conf;             // work items per configuration
     std::vector<TriePartHost> parts;
     // The number of parts that worked for a class of this shape before is tried first (a hint kept per process: a
     // wrong hint costs one failed attempt, the sequence below then runs as usual).
@@ -765,21 +771,20 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     }
     if (parts.empty()) return false;
     out.parts.swap(parts);
-    out.plist = plist;
     return true;
 }
 
 // One allocation and one copy for the trees of all classes: per class its parts' blobs, the part descriptions
 // and the list of the class's configurations.
-static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpClass *, TrieClassHost>> &built)
+static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
 {
     constexpr size_t kTwoPerSm = 108 * 1024;
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
     size_t total = 0, n_parts_all = 0;
     for (auto &bc : built) {
-        for (const auto &pt : bc.second.parts) total += up(pt.blob.size());
-        total += up(bc.second.parts.size() * sizeof(TrieMeta)) + up(bc.second.plist.size() * sizeof(u32));
-        n_parts_all += bc.second.parts.size();
+        for (const auto &pt : bc.tree->parts) total += up(pt.blob.size());
+        total += up(bc.tree->parts.size() * sizeof(TrieMeta)) + up(bc.plist.size() * sizeof(u32));
+        n_parts_all += bc.tree->parts.size();
     }
     if (!total) return true;
     const size_t o_jobs = total;
@@ -791,12 +796,12 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
     std::vector<unsigned char> stage(total, 0);
     size_t off = 0;
     for (auto &bc : built) {
-        hap_problem::Trie &tr = bc.first->trie;
-        TrieClassHost &h = bc.second;
+        hap_problem::Trie &tr = bc.cl->trie;
+        const TrieClassHost &h = *bc.tree;
         std::vector<TrieMeta> metas;
         size_t smem = 0;
         u32 want = 0;
-        for (auto &pt : h.parts) {
+        for (const auto &pt : h.parts) {
             unsigned char *base = p->d_trie_arena + off;
             std::memcpy(stage.data() + off, pt.blob.data(), pt.blob.size());
             hap_problem::TriePartDev pd{};
@@ -808,15 +813,16 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
             pd.d_depth = base + pt.o_depth;
             pd.n_nodes = pt.n_nodes; pd.n_cells = pt.n_cells; pd.nmap = pt.nmap; pd.m_lo = pt.meta.m_lo;
             std::memcpy(pd.mrow_of, pt.meta.mrow_of, sizeof(pd.mrow_of));
-            pt.meta.nodes = pd.d_nodes; pt.meta.leaves = pd.d_leaves; pt.meta.cells = pd.d_cells;
-            pt.meta.parent = reinterpret_cast<const uint16_t *>(base + pt.o_parent);
+            TrieMeta meta = pt.meta;                 // the host tree is shared between problems: the device pointers go into a copy
+            meta.nodes = pd.d_nodes; meta.leaves = pd.d_leaves; meta.cells = pd.d_cells;
+            meta.parent = reinterpret_cast<const uint16_t *>(base + pt.o_parent);
             tr.parts.push_back(pd);
-            metas.push_back(pt.meta);
+            metas.push_back(meta);
             GatherJob gj{};
             gj.first_leaf = pd.d_first_leaf; gj.gnode = pd.d_gnode; gj.depth = pd.d_depth;
             gj.nodes = pd.d_nodes; gj.cells = pd.d_cells; gj.leaves = pd.d_leaves;
-            gj.tab_off = bc.first->map_base; gj.n_nodes = pd.n_nodes; gj.n_cells = pd.n_cells; gj.nmap = pd.nmap; gj.m_lo = pd.m_lo;
-            gj.blk_lo = gblk; gj.PP = bc.first->PP;
+            gj.tab_off = bc.cl->map_base; gj.n_nodes = pd.n_nodes; gj.n_cells = pd.n_cells; gj.nmap = pd.nmap; gj.m_lo = pd.m_lo;
+            gj.blk_lo = gblk; gj.PP = bc.cl->PP;
             std::memcpy(gj.rm.mrow_of, pd.mrow_of, sizeof(gj.rm.mrow_of));
             gblk += (pd.n_nodes + pd.n_cells + pd.nmap + 255) / 256;
             gjobs.push_back(gj);
@@ -828,11 +834,11 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
         std::memcpy(stage.data() + off, metas.data(), metas.size() * sizeof(TrieMeta));
         off += up(metas.size() * sizeof(TrieMeta));
         tr.d_plist = reinterpret_cast<u32 *>(p->d_trie_arena + off);
-        std::memcpy(stage.data() + off, h.plist.data(), h.plist.size() * sizeof(u32));
-        off += up(h.plist.size() * sizeof(u32));
-        tr.n_conf = (unsigned)h.plist.size(); tr.smem = smem;
+        std::memcpy(stage.data() + off, bc.plist.data(), bc.plist.size() * sizeof(u32));
+        off += up(bc.plist.size() * sizeof(u32));
+        tr.n_conf = (unsigned)bc.plist.size(); tr.smem = smem;
         if (dj.n <= HAP_MAX_PP) {
-            const hap_problem::PpClass &cl = *bc.first;
+            const hap_problem::PpClass &cl = *bc.cl;
             const u32 rep = p->items[cl.item_lo].p;
             const u64 nmap_cl = p->pconfs[rep].nmap;
             dj.blk_lo[dj.n] = dblk; dj.p_rep[dj.n] = rep; dj.nmap[dj.n] = (u32)nmap_cl; dj.tab_off[dj.n] = cl.map_base;
@@ -847,7 +853,7 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
     }
     std::memcpy(stage.data() + o_jobs, gjobs.data(), gjobs.size() * sizeof(GatherJob));
     if (cudaMemcpy(p->d_trie_arena, stage.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
-        for (auto &bc : built) bc.first->trie = hap_problem::Trie{};
+        for (auto &bc : built) bc.cl->trie = hap_problem::Trie{};
         return false;
     }
     p->decode_jobs = dj;
@@ -855,6 +861,51 @@ static bool upload_tries(hap_problem *p, std::vector<std::pair<hap_problem::PpCl
     p->n_gather_jobs = (int)gjobs.size();
     p->gather_blocks = gblk;
     return true;
+}
+
+// ---- per-process cache of the classes' prefix trees ------------------------------------------------------
+namespace {
+std::mutex g_trie_cache_mu;
+std::map<std::string, std::shared_ptr<const TrieClassHost>> g_trie_cache;
+constexpr size_t kTrieCacheEntries = 256;
+}
+
+template <class V> static void key_put(std::string &k, const V &v) { k.append(reinterpret_cast<const char *>(&v), sizeof(v)); }
+
+// everything the decoded mappings, the windows, the bands, the cell records and the split into parts depend on
+static std::string trie_cache_key(const hap_problem *p, const hap_problem::PpClass &cl)
+{
+    std::string k("hap-trie-1");
+    const hap_pconf &rep = p->pconfs[p->items[cl.item_lo].p];
+    const size_t n_conf = p->items[cl.item_hi - 1].p - p->items[cl.item_lo].p + 1;
+    const int32_t head[] = {p->model.N, p->T, p->prof.R, cl.PP, rep.G, rep.mode, p->opts.delta_q, (int32_t)(p->opts.flags & HAP_OPT_UNIFORM),
+                            p->dc.kind_uniform, p->dc.kind_uniform_from, (int32_t)((cl.item_hi - cl.item_lo) / n_conf)};
+    key_put(k, head);
+    key_put(k, rep.nmap);
+    for (int h = 0; h < p->T; ++h) { key_put(k, p->P[h]); key_put(k, p->cap_eff[h]); key_put(k, p->dc.m[h]); key_put(k, p->dc.node_size[h]); }
+    return k;
+}
+
+static std::shared_ptr<const TrieClassHost> trie_cache_find(const std::string &key)
+{
+    std::lock_guard<std::mutex> lock(g_trie_cache_mu);
+    auto it = g_trie_cache.find(key);
+    return it == g_trie_cache.end() ? nullptr : it->second;
+}
+
+static void trie_cache_insert(const std::string &key, std::shared_ptr<const TrieClassHost> tree)
+{
+    std::lock_guard<std::mutex> lock(g_trie_cache_mu);
+    if (g_trie_cache.size() >= kTrieCacheEntries) g_trie_cache.clear();
+    g_trie_cache[key] = std::move(tree);
+}
+
+// the configurations of a class (contiguous: PP is the outermost loop of the enumeration)
+static std::vector<u32> class_plist(const hap_problem *p, const hap_problem::PpClass &cl)
+{
+    std::vector<u32> plist;
+    for (size_t pi = p->items[cl.item_lo].p; pi <= p->items[cl.item_hi - 1].p; ++pi) plist.push_back((u32)pi);
+    return plist;
 }
 
 extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t *n_candidates)
@@ -977,7 +1028,13 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
         // one allocation for everything whose size the enumeration fixes (an allocation costs far more than the
         // microseconds a pass takes): configuration table | work items | layer costs | coefficients | per-type
         // constants | lower bounds | partial minima | mapping tables | small scalars
-        p->n_partial = std::max<size_t>(p->items.size(), 1024);
+        // partial minima of a search: one slot per block; a class's tree kernel may run up to 8 parts per configuration
+        // (the exact count is fixed below, once the trees are built)
+        p->n_partial = 1024;
+        for (const auto &cl : p->classes) {
+            const size_t n_conf = p->items[cl.item_hi - 1].p - p->items[cl.item_lo].p + 1;
+            p->n_partial += std::max(cl.item_hi - cl.item_lo, n_conf * 8);
+        }
         {
             auto up = [](size_t v) { return (v + 255) / 256 * 256; };
             size_t o = 0;
@@ -1022,38 +1079,68 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             CUDA_TRY(p, cudaEventCreateWithFlags(&cl.done, cudaEventDisableTiming));
         }
         if (tab_bytes) {
-            for (const auto &cl : p->classes) {
+            // The prefix tree of a class depends on the cluster, the stage count, the model's layer kinds and the
+            // window, not on the profiled tables: trees are kept per process under a key of exactly those inputs, so
+            // that planning again on the same cluster (new tables, new batch) neither decodes the mappings for the
+            // host nor rebuilds a tree.
+            // the tree kernel holds times as doubles: exact while every prefix row stays below 2^52, which the
+            // per-layer limit of 2^36 ns guarantees when N (2 + max tau) <= 2^16
+            int tau_max = 0;
+            for (int r = 0; r < p->prof.R; ++r) tau_max = std::max(tau_max, p->tau_q[r] >> 10);
+            const bool rows_exact = (int64_t)N * (2 + tau_max) <= 65536;
+            const bool want_trees = !(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear && rows_exact;
+            std::vector<TrieBuilt> built;
+            std::vector<hap_problem::PpClass *> missing;
+            std::vector<std::string> keys(p->classes.size());
+            for (size_t ci = 0; ci < p->classes.size(); ++ci) {
+                auto &cl = p->classes[ci];
                 if (!cl.has_tab) continue;
-                const WorkItem &rep = p->items[cl.item_lo];
-                const u64 nmap = p->pconfs[rep.p].nmap;
-                maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128>>>(p->dc, rep.p, nmap, p->d_maptab + cl.map_base);
-                CUDA_TRY(p, cudaGetLastError());
+                keys[ci] = trie_cache_key(p, cl);
+                std::shared_ptr<const TrieClassHost> hit = trie_cache_find(keys[ci]);
+                if (!hit) { missing.push_back(&cl); continue; }
+                cl.masks_used = hit->masks_used;
+                if (want_trees && !hit->parts.empty()) built.push_back(TrieBuilt{&cl, hit, class_plist(p, cl)});
             }
-            CUDA_TRY(p, cudaDeviceSynchronize());
-            // which type masks occur in a class: the DP kernel builds stage rows for those only
-            std::vector<uint8_t> tab(tab_bytes);
-            std::vector<std::pair<hap_problem::PpClass *, TrieClassHost>> built;
-            CUDA_TRY(p, cudaMemcpy(tab.data(), p->d_maptab, tab_bytes, cudaMemcpyDeviceToHost));
-            for (auto &cl : p->classes) {
-                if (!cl.has_tab) continue;
-                const u64 nmap = p->pconfs[p->items[cl.item_lo].p].nmap;
-                unsigned used = 0;
-                for (u64 e = 0; e < nmap * (u64)cl.PP; ++e) used |= 1u << tab[cl.map_base + e * 2];
-                cl.masks_used = used;
-                // the tree kernel holds times as doubles: exact while every prefix row stays below 2^52, which the
-                // per-layer limit of 2^36 ns guarantees when N (2 + max tau) <= 2^16
-                int tau_max = 0;
-                for (int r = 0; r < p->prof.R; ++r) tau_max = std::max(tau_max, p->tau_q[r] >> 10);
-                const bool rows_exact = (int64_t)N * (2 + tau_max) <= 65536;
-                if (!(p->opts.flags & HAP_OPT_NO_TRIE) && p->dc.tau_linear && rows_exact) {
-                    std::vector<u32> plist;
-                    for (size_t pi = p->items[cl.item_lo].p; pi <= p->items[cl.item_hi - 1].p; ++pi) plist.push_back((u32)pi);   // contiguous
-                    TrieClassHost th;
-                    if (build_trie(p, cl, tab.data() + cl.map_base, nmap, plist, th)) built.emplace_back(&cl, std::move(th));
+            if (!missing.empty()) {
+                for (const hap_problem::PpClass *cl : missing) {
+                    const WorkItem &rep = p->items[cl->item_lo];
+                    const u64 nmap = p->pconfs[rep.p].nmap;
+                    maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128>>>(p->dc, rep.p, nmap, p->d_maptab + cl->map_base);
+                    CUDA_TRY(p, cudaGetLastError());
+                    cl->tab_valid = true;
+                }
+                CUDA_TRY(p, cudaDeviceSynchronize());
+                std::vector<uint8_t> tab(tab_bytes);
+                CUDA_TRY(p, cudaMemcpy(tab.data(), p->d_maptab, tab_bytes, cudaMemcpyDeviceToHost));
+                for (hap_problem::PpClass *clp : missing) {
+                    auto &cl = *clp;
+                    const u64 nmap = p->pconfs[p->items[cl.item_lo].p].nmap;
+                    auto th = std::make_shared<TrieClassHost>();
+                    // which type masks occur in a class: the DP kernel builds stage rows for those only
+                    unsigned used = 0;
+                    for (u64 e = 0; e < nmap * (u64)cl.PP; ++e) used |= 1u << tab[cl.map_base + e * 2];
+                    th->masks_used = used;
+                    cl.masks_used = used;
+                    const std::vector<u32> plist = class_plist(p, cl);
+                    const bool ok = want_trees && build_trie(p, cl, tab.data() + cl.map_base, nmap, plist.size(), *th);
+                    if (!ok) th->parts.clear();
+                    // a class whose tree was not wanted this time is not remembered as "has no tree"
+                    if (want_trees) trie_cache_insert(keys[clp - p->classes.data()], th);
+                    if (ok) built.push_back(TrieBuilt{&cl, th, plist});
                 }
             }
+            // the launch order of the merged decode / gather jobs follows the class order
+            std::sort(built.begin(), built.end(), [](const TrieBuilt &x, const TrieBuilt &y) { return x.cl < y.cl; });
             upload_tries(p, built);
         }
+        p->n_pslots = 0;
+        for (auto &cl : p->classes) {
+            cl.pslot_lo = p->n_pslots;
+            cl.pslot_n = cl.item_hi - cl.item_lo;
+            if (cl.trie.ok) cl.pslot_n = std::max(cl.pslot_n, (size_t)cl.trie.n_conf * cl.trie.parts.size());
+            p->n_pslots += cl.pslot_n;
+        }
+        if (p->n_pslots > p->n_partial) return fail(p, HAP_E_STATE, "partial-minimum slots exceed their allocation");
         p->enumerated = true;
     }
     if (n_pconf) *n_pconf = p->pconfs.size();
@@ -1106,6 +1193,36 @@ extern "C" hap_status hap_decode(hap_problem *p, uint64_t first, uint64_t count,
     return HAP_OK;
 }
 
+// per (configuration, type) constants and stage coefficients, then the layer costs of `n_conf` configurations from
+// `p_first` on (all by default); index_dev: of the one configuration that owns the candidate index stored there
+static hap_status launch_layer_kernel(hap_problem *p, i64 *c2, double *c2f, bool quant, cudaStream_t st, i64 *lb_sum,
+                                      const i64 *index_dev, unsigned p_first, unsigned n_conf, bool dependent)
+{
+    const unsigned thr = (unsigned)((p->model.N + 31) / 32 * 32);
+    // programmatic dependent launch: the blocks start while type_const_kernel drains and wait inside the kernel
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(n_conf); cfg.blockDim = dim3(thr); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = dependent ? 1 : 0;
+    const TypeConst *tcg = p->d_tc;
+    i64 *no_i = nullptr; double *no_d = nullptr;
+    // layer kinds: 0 all dense, 1 all MoE (uniform branch compiled away), 2 mixed
+    const int kind = !p->dc.kind_uniform ? 2 : (p->kind[0] == HAP_MOE ? 1 : 0);
+    using Fn = void (*)(const DevConst, const TypeConst *, i64 *, double *, i64 *, u64 *, const i64 *, unsigned);
+    if (quant) {
+        static const Fn fns[3][2] = {{layer_cost_kernel<true, 0, false>, layer_cost_kernel<true, 0, true>},
+                                     {layer_cost_kernel<true, 1, false>, layer_cost_kernel<true, 1, true>},
+                                     {layer_cost_kernel<true, 2, false>, layer_cost_kernel<true, 2, true>}};
+        CUDA_TRY(p, cudaLaunchKernelEx(&cfg, fns[kind][lb_sum ? 1 : 0], p->dc, tcg, c2, no_d, lb_sum, p->d_range, index_dev, p_first));
+    } else {
+        static const Fn fns[3] = {layer_cost_kernel<false, 0, false>, layer_cost_kernel<false, 1, false>, layer_cost_kernel<false, 2, false>};
+        CUDA_TRY(p, cudaLaunchKernelEx(&cfg, fns[kind], p->dc, tcg, no_i, c2f, no_i, p->d_range, index_dev, p_first));
+    }
+    return HAP_OK;
+}
+
 static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st,
                                      i64 *lb_sum = nullptr)
 {
@@ -1115,30 +1232,8 @@ static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double 
     else type_const_kernel<false><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff, p->d_range);
     CUDA_TRY(p, cudaGetLastError());
     if ((quant && c2) || (!quant && c2f)) {
-        const unsigned b2 = (unsigned)p->pconfs.size();
-        const unsigned thr = (unsigned)((p->model.N + 31) / 32 * 32);
-        // programmatic dependent launch: the blocks start while type_const_kernel drains and wait inside the kernel
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(b2); cfg.blockDim = dim3(thr); cfg.dynamicSmemBytes = 0; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        const TypeConst *tcg = p->d_tc;
-        i64 *no_i = nullptr; double *no_d = nullptr;
-        // layer kinds: 0 all dense, 1 all MoE (uniform branch compiled away), 2 mixed
-        const int kind = !p->dc.kind_uniform ? 2 : (p->kind[0] == HAP_MOE ? 1 : 0);
-        if (quant) {
-            using Fn = void (*)(const DevConst, const TypeConst *, i64 *, double *, i64 *, u64 *);
-            static const Fn fns[3][2] = {{layer_cost_kernel<true, 0, false>, layer_cost_kernel<true, 0, true>},
-                                         {layer_cost_kernel<true, 1, false>, layer_cost_kernel<true, 1, true>},
-                                         {layer_cost_kernel<true, 2, false>, layer_cost_kernel<true, 2, true>}};
-            CUDA_TRY(p, cudaLaunchKernelEx(&cfg, fns[kind][lb_sum ? 1 : 0], p->dc, tcg, c2, no_d, lb_sum, p->d_range));
-        } else {
-            using Fn = void (*)(const DevConst, const TypeConst *, i64 *, double *, i64 *, u64 *);
-            static const Fn fns[3] = {layer_cost_kernel<false, 0, false>, layer_cost_kernel<false, 1, false>, layer_cost_kernel<false, 2, false>};
-            CUDA_TRY(p, cudaLaunchKernelEx(&cfg, fns[kind], p->dc, tcg, no_i, c2f, no_i, p->d_range));
-        }
+        hap_status s = launch_layer_kernel(p, c2, c2f, quant, st, lb_sum, nullptr, 0, (unsigned)p->pconfs.size(), true);
+        if (s != HAP_OK) return s;
     }
     CUDA_TRY(p, cudaGetLastError());
     return HAP_OK;
@@ -1175,6 +1270,21 @@ static bool pass_uses_trie(const hap_problem *p, const hap_problem::PpClass &cl,
     const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
     (void)f64;                                  // both value types walk the tree
     return cl.trie.ok && !out.count_only && !refine && p->dc.tau_linear != 0 && !out.dp_table && !out.choice && out.count > 1;
+}
+
+// Whether every class the pass touches walks its prefix tree: then the blocks of the tree kernel compute the layer
+// times of their configuration themselves (Eq. 2 from the profiled tables and the per-type constants) and the pass
+// neither writes nor reads the layer-cost array.
+static bool pass_fuses_layer_costs(const hap_problem *p, const DpOut &out, bool search)
+{
+    if (p->opts.flags & HAP_OPT_NO_FUSE) return false;
+    bool any = false;
+    for (const auto &cl : p->classes) {
+        if (!search && !out.first_dev && class_outside(p, cl, out)) continue;
+        if (!pass_uses_trie(p, cl, out, false)) return false;
+        any = true;
+    }
+    return any;
 }
 
 // candidate decode of a class for this pass, then its stage bytes into the class's tree
@@ -1220,6 +1330,7 @@ static hap_status launch_decode_early(hap_problem *p, const DpOut &out, bool sea
     CUDA_TRY(p, cudaGetLastError());
     CUDA_TRY(p, cudaEventRecord(p->ev_dec, sx));
     p->decoded_all = true;
+    for (const auto &cl : p->classes) if (cl.trie.ok) cl.tab_valid = true;
     return HAP_OK;
 }
 
@@ -1268,17 +1379,19 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const uint8_t *tab = cl.has_tab ? p->d_maptab + cl.map_base : nullptr;
         DpOut o = out;
         o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0;
-        if (search) { o.partial_cost += cl.item_lo; o.partial_index += cl.item_lo; }
+        if (search) { o.partial_cost += cl.pslot_lo; o.partial_index += cl.pslot_lo; }
         if (pass_uses_trie(p, cl, out, f64)) {
             const hap_problem::Trie &tr = cl.trie;
             // 64 registers per thread in both shapes (measured: more warps per SM beat more registers per thread)
             const int tv = tr.threads > 512 ? 0 : 1;
             if (search && f64) return fail(p, HAP_E_STATE, "the fp64 search reduces a cost array");
+            const bool counting = (p->opts.flags & HAP_OPT_COUNT_SPLITS) && !f64 && !search;
             const void *tfn = f64 ? (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1, double> : (const void *)trie_dp_kernel<false, 512, 2, double>)
                             : search ? (tv == 0 ? (const void *)trie_dp_kernel<true, 1024, 1> : (const void *)trie_dp_kernel<true, 512, 2>)
-                                     : (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1> : (const void *)trie_dp_kernel<false, 512, 2>);
-            static size_t trie_limit[64][6];
-            const int vi = (f64 ? 4 : search ? 2 : 0) + tv;
+                            : counting ? (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1, i64, true> : (const void *)trie_dp_kernel<false, 512, 2, i64, true>)
+                                       : (tv == 0 ? (const void *)trie_dp_kernel<false, 1024, 1> : (const void *)trie_dp_kernel<false, 512, 2>);
+            static size_t trie_limit[64][8];
+            const int vi = (f64 ? 4 : search ? 2 : counting ? 6 : 0) + tv;
             if (tr.smem > trie_limit[dev][vi]) {
                 CUDA_TRY(p, cudaFuncSetAttribute(tfn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)tr.smem));
                 trie_limit[dev][vi] = tr.smem;
@@ -1286,6 +1399,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
             if (!decoded_all) {                     // not queued beside the layer costs by this pass
                 hap_status sd = launch_class_decode(p, cl);
+                cl.tab_valid = true;
                 if (sd != HAP_OK) return sd;
             }
             int n_parts = (int)tr.parts.size();
@@ -1294,7 +1408,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
             const TrieMeta *metas = tr.d_metas;
             void *c2v = f64 ? (void *)p->d_c2f : (void *)p->d_c2, *coefv = f64 ? (void *)p->d_coeff : (void *)p->d_coef;
             void *targs[] = {(void *)&p->dc, (void *)&plist, (void *)&n_active, (void *)&c2v, (void *)&p->d_coef, (void *)&coefv, (void *)&metas, (void *)&n_parts, (void *)&o};
-            const unsigned tblocks = search ? std::max(blocks, n_active) : n_active;       // search: every partial slot of the class is written
+            const unsigned tblocks = search ? (unsigned)cl.pslot_n : n_active;             // search: every partial slot of the class is written
             CUDA_TRY(p, cudaLaunchKernel(tfn, dim3(tblocks), dim3(tr.threads), targs, tr.smem, cl.stream));
             CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
             CUDA_TRY(p, cudaStreamWaitEvent(st, cl.done, 0));
@@ -1307,15 +1421,21 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         void *cvarg = f64 ? (void *)p->d_coeff : (void *)p->d_coef;
         void *args[] = {(void *)&p->dc, (void *)&its, (void *)&c2arg, (void *)&p->d_coef, (void *)&cvarg, (void *)&tab, (void *)&o, (void *)&nw, (void *)&used};
         CUDA_TRY(p, cudaStreamWaitEvent(cl.stream, p->ev_fork, 0));
-        if (cl.has_tab && out.count > 1) {
+        if (cl.has_tab && (out.count > 1 || !cl.tab_valid)) {        // (a single candidate reuses a table that some pass has filled)
             // candidate decode (stage masks and link classes of every mapping of the class) is part of every pass,
             // not a cached result of hap_enumerate; the one-candidate re-evaluation of a winner reuses the table
             const WorkItem &rep = p->items[cl.item_lo];
             const u64 nmap = p->pconfs[rep.p].nmap;
             maptab_kernel<<<(unsigned)((nmap + 3) / 4), 128, 0, cl.stream>>>(p->dc, rep.p, nmap, p->d_maptab + cl.map_base);
             CUDA_TRY(p, cudaGetLastError());
+            cl.tab_valid = true;
         }
         CUDA_TRY(p, cudaLaunchKernel(fn, dim3(blocks), dim3(cl.warps * 32), args, cl.smem, cl.stream));
+        if (search && cl.pslot_n > blocks) {       // slots that only the class's tree kernel would write
+            const unsigned extra = (unsigned)(cl.pslot_n - blocks);
+            fill_partials_kernel<<<(extra + 255) / 256, 256, 0, cl.stream>>>(o.partial_cost + blocks, o.partial_index + blocks, extra);
+            CUDA_TRY(p, cudaGetLastError());
+        }
         CUDA_TRY(p, cudaEventRecord(cl.done, cl.stream));
         CUDA_TRY(p, cudaStreamWaitEvent(st, cl.done, 0));      // join
     }
@@ -1338,8 +1458,10 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
     out.recompute = dev_recompute; out.dp_table = (i64 *)dev_dp_table; out.choice = dev_choice;
     out.first = first; out.count = count;
+    const bool fused = pass_fuses_layer_costs(p, out, false);
+    out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
     CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
-    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_decode_early(p, out, false)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
@@ -1370,13 +1492,15 @@ extern "C" hap_status hap_pipeline_dp_f64(hap_problem *p, uint64_t first, uint64
     CUDA_TRY(p, cudaMemsetAsync(p->d_counters, 0, 8 * sizeof(u64), st));
     CUDA_TRY(p, cudaEventRecord(p->ev[0], st));
     // the memory model stays on the integer byte coefficients; times stay unrounded
-    if ((s = launch_layer_costs(p, nullptr, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
-    if ((s = launch_layer_costs(p, nullptr, nullptr, p->d_c2f, p->d_coeff, false, st)) != HAP_OK) return s;
-    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     DpOut out{};
     out.counters = p->d_counters;
     out.cost = (i64 *)dev_cost; out.bottleneck = (i64 *)dev_bottleneck; out.partition = dev_partition;
     out.recompute = dev_recompute; out.first = first; out.count = count;
+    const bool fused = pass_fuses_layer_costs(p, out, false);
+    out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
+    if ((s = launch_layer_costs(p, nullptr, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, nullptr, nullptr, fused ? nullptr : p->d_c2f, p->d_coeff, false, st)) != HAP_OK) return s;
+    CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_dp(p, out, false, st, true)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
@@ -1409,6 +1533,11 @@ extern "C" hap_status hap_search_range_f64(hap_problem *p, uint64_t first, uint6
     DpOut one{};
     one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
     one.recompute = d1->rec; one.first = win; one.count = 1;
+    {   // the pass may have left the layer-cost array untouched: the winner's configuration is evaluated here
+        size_t lo = 0, hi = p->pconfs.size();
+        while (hi - lo > 1) { const size_t mid = (lo + hi) / 2; if (p->pconfs[mid].offset <= win) lo = mid; else hi = mid; }
+        if ((s = launch_layer_kernel(p, nullptr, p->d_c2f, false, st, nullptr, nullptr, (unsigned)lo, 1, false)) != HAP_OK) return s;
+    }
     if ((s = launch_dp(p, one, false, st, true)) != HAP_OK) return s;
     decode_kernel<<<1, 32, 0, st>>>(p->dc, win, 1, &d1->cand, nullptr);
     CUDA_TRY(p, cudaGetLastError());
@@ -1750,6 +1879,9 @@ extern "C" hap_status hap_launches_per_pass(hap_problem *p, uint32_t *host_count
     uint32_t n = 2 + 2;                                     // type constants, layer costs; argmin partial and final
     bool all_trees = p->n_gather_jobs > 0;
     for (const auto &cl : p->classes) if (cl.trie.ok && !(lin && !refine)) all_trees = false;
+    bool fused = !(p->opts.flags & HAP_OPT_NO_FUSE) && lin && !refine && !p->classes.empty();
+    for (const auto &cl : p->classes) if (!cl.trie.ok) fused = false;
+    if (fused) n -= 1;                                      // the tree blocks compute the layer costs themselves
     if (all_trees) n += 2;                                  // one decode and one tree-gather launch for all classes
     for (const auto &cl : p->classes) {
         if (cl.trie.ok && lin && !refine) n += all_trees ? 1 : 1 + (uint32_t)cl.trie.parts.size() + 1;   // (decode, gather per part,) tree DP
@@ -1801,12 +1933,14 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     out.first = first; out.count = count; out.prune = p->opts.prune;
     out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
     out.incumbent = p->d_counters + 3;
+    const bool fused = pass_fuses_layer_costs(p, out, true);
+    out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
     CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
-    if ((s = launch_layer_costs(p, p->d_c2, p->d_coef, nullptr, nullptr, true, st, p->d_lb)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st, fused ? nullptr : p->d_lb)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_decode_early(p, out, true)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
-    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->items.size(), p->d_best, kInf);
+    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->n_pslots, p->d_best, kInf);
     CUDA_TRY(p, cudaGetLastError());
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
@@ -1816,6 +1950,7 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     DpOut one{};
     one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
     one.recompute = d1->rec; one.first = 0; one.count = 1; one.first_dev = p->d_best + 1;
+    if (fused && (s = launch_layer_kernel(p, p->d_c2, nullptr, true, st, nullptr, p->d_best + 1, 0, 1, false)) != HAP_OK) return s;
     if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
     decode_kernel<<<1, 32, 0, st>>>(p->dc, 0, 1, &d1->cand, p->d_best + 1);
     CUDA_TRY(p, cudaGetLastError());

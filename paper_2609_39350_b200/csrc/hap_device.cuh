@@ -105,6 +105,10 @@ struct DpOut {
     int prune;                        // search mode: skip blocks whose lower bound exceeds the incumbent
     int exact;                        // refinement kernels: sweep the stage-cost limit for the optimum of sum + (M-1) max
     int count_only;                   // instrumentation: count the finite-cost cells of each candidate, run no recurrence
+    // layer costs computed by the DP blocks themselves (prefix-tree kernel): per (configuration, type) constants of
+    // Eq. 2; null: the blocks read the layer-cost array.  range_flag: set when a layer time leaves the supported range
+    const struct TypeConst *tcg;
+    u64 *range_flag;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -217,6 +221,28 @@ __device__ __forceinline__ void store_pair(i64 *qi, double *qd, size_t at, doubl
 }
 
 constexpr int kLcThreads = 128;
+
+// Eq. 2 for one (configuration, device type, layer): forward and backward time of the layer from its table entries
+// ta = (t_dense fwd, bwd), tf = (t_ffn fwd, bwd) and the per-(configuration, type) constants tc (a TypeConst read as
+// 16-byte pairs).  One IEEE operation per operator, in the order the formulas are written.
+__device__ __forceinline__ double div_by(double a, double b, double y);
+__device__ __forceinline__ u64 find_pconf(const DevConst &dc, u64 c);
+__device__ __forceinline__ void layer_cost_pair(const double2 *tc, double2 ta, double2 tf, bool dense, double kappa, double &cf, double &cb)
+{
+    if (dense) {
+        const double2 cm = tc[4];                                // commF_dense, commB_dense
+        cf = ta.x + cm.x;
+        cb = ta.y + cm.y;
+    } else {
+        const double2 dn = tc[0], di = tc[1], tr = tc[2], cm = tc[3];
+        const double xf = div_by(kappa * tf.x, dn.x, dn.y);
+        const double mf = (xf + di.x) * di.y;
+        cf = (((ta.x - tf.x) + mf) + tr.x) + cm.x;
+        const double xb = div_by(kappa * tf.y, dn.x, dn.y);
+        const double mb = (xb + di.x) * di.y;
+        cb = (((ta.y - tf.y) + mb) + tr.y) + cm.y;
+    }
+}
 
 // a / b for a divisor whose correctly rounded reciprocal y = RN(1/b) is known: q0 = RN(a*y), the exact
 // residual r = a - b*q0 (one fused operation) and q = RN(q0 + r*y) give the correctly rounded quotient
@@ -361,12 +387,19 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
 template <bool QUANT, int KIND, bool WANT_LB>
 __global__ void __launch_bounds__(256)
 layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__restrict__ c2, double *__restrict__ c2f,
-                  i64 *__restrict__ lb_sum, u64 *range_flag)
+                  i64 *__restrict__ lb_sum, u64 *range_flag, const i64 *index_dev, unsigned p_first)
 {
     __shared__ TypeConst tcs[HAP_MAX_TYPES];
     __shared__ i64 s_lb[8];
     const int N = dc.N, T = dc.T;
-    const unsigned p = blockIdx.x;
+    // block b works on configuration p_first + b; or, when a preceding kernel left a candidate index in device
+    // memory, on the configuration that owns it (negative: none)
+    unsigned p = p_first + blockIdx.x;
+    if (index_dev) {
+        const i64 f = *index_dev;
+        if (f < 0) return;
+        p = (unsigned)find_pconf(dc, (u64)f);
+    }
     const int l = threadIdx.x;
     const bool dense = KIND == 0 || (KIND == 2 && l < N && layer_kind(dc, l) == HAP_DENSE);
     double2 ta[HAP_MAX_TYPES], tf[HAP_MAX_TYPES];           // (t_dense fwd, bwd), (t_ffn fwd, bwd) of the layer per type
@@ -381,7 +414,7 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
         for (int h = 0; h < HAP_MAX_TYPES; ++h) {
             if (h < T) {
                 ta[h] = __ldg(tp);
-                if (!dense) tf[h] = __ldg(tp + 1);
+                tf[h] = dense ? make_double2(0.0, 0.0) : __ldg(tp + 1);
                 tp += stride_h;
             }
         }
@@ -405,21 +438,8 @@ layer_cost_kernel(const DevConst dc, const TypeConst *__restrict__ tcg, i64 *__r
 #pragma unroll
         for (int h = 0; h < HAP_MAX_TYPES; ++h) {
             if (h < T) {
-                const double2 *tc = reinterpret_cast<const double2 *>(&tcs[h]);
                 double cf, cb;
-                if (dense) {
-                    const double2 cm = tc[4];                                // commF_dense, commB_dense
-                    cf = ta[h].x + cm.x;
-                    cb = ta[h].y + cm.y;
-                } else {
-                    const double2 dn = tc[0], di = tc[1], tr = tc[2], cm = tc[3];
-                    const double xf = div_by(kappa * tf[h].x, dn.x, dn.y);
-                    const double mf = (xf + di.x) * di.y;
-                    cf = (((ta[h].x - tf[h].x) + mf) + tr.x) + cm.x;
-                    const double xb = div_by(kappa * tf[h].y, dn.x, dn.y);
-                    const double mb = (xb + di.x) * di.y;
-                    cb = (((ta[h].y - tf[h].y) + mb) + tr.y) + cm.y;
-                }
+                layer_cost_pair(reinterpret_cast<const double2 *>(&tcs[h]), ta[h], tf[h], dense, kappa, cf, cb);
                 bad |= !(cf < 6.8719e10) | !(cb < 6.8719e10);                 // 2^36 ns per layer
                 if (QUANT) {
                     longlong2 v; v.x = __double2ll_rn(cf); v.y = __double2ll_rn(cb);
@@ -1773,6 +1793,13 @@ joint_dp_kernel(const DevConst dc, const unsigned *pconf_ids, unsigned n_ids, co
 // ------------------------------------------------------------------------------------------
 // argmin: stage 1 reduces a slice per block, stage 2 (one block) reduces the partials
 // ------------------------------------------------------------------------------------------
+// "no candidate" into partial-minimum slots that no block of the pass writes
+__global__ void fill_partials_kernel(i64 *pcost, u64 *pindex, unsigned n)
+{
+    const unsigned q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q < n) { pcost[q] = kInf; pindex[q] = ~0ull; }
+}
+
 __global__ void __launch_bounds__(256)
 argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex, i64 init)
 {

@@ -88,6 +88,9 @@ __host__ __device__ inline size_t trie_smem_bytes(int N, int PP, int T, int R, i
 
 struct TrieRowMap { uint8_t mrow_of[16]; };
 
+template <typename T> struct IsF64 { static constexpr bool value = false; };
+template <> struct IsF64<double> { static constexpr bool value = true; };
+
 // Copies what the decode of this pass produced into the tree: node n of depth d takes the stage bytes (device
 // types, boundary link) of stage d of the first mapping below it, every cell of the node the index of the stage
 // constant that follows from them, leaf m the last stage of mapping m.
@@ -185,13 +188,55 @@ __device__ __forceinline__ int lds_u8(u32 a)
     return (int)v;
 }
 
-// Block prologue, part 1: layer times of the configuration staged in shared memory, the weight and activation
-// byte prefixes, MoE prefix counts, per-mask stage info, p2p coefficients, the table of stage constants and a
-// copy of the tree's node records: what decides whether any mapping of the configuration can be feasible.
+// Layer times of the configuration into shared memory, computed from the profiled tables and the per-(configuration,
+// type) constants of Eq. 2: one thread per (type, layer), with the arithmetic of layer_cost_kernel (same function,
+// same bits).  Kept out of line (it runs once per block and would otherwise raise the register pressure of the split
+// loop); takes scalars, not the by-value constant block, so that nothing is copied to local memory.  No barrier.
+template <typename VT>
+__device__ __noinline__ void trie_compute_costs(const double2 *tab, size_t stride_h, int N, int T, double kappa, u64 kb0, u64 kb1,
+                                                u64 kb2, u64 kb3, const TypeConst *tcp, u64 *range_flag, VT *sC)
+{
+    bool bad = false;
+    for (int q = threadIdx.x; q < T * N; q += blockDim.x) {
+        const int h = q / N, l = q - h * N;
+        const u64 kb = l < 64 ? kb0 : l < 128 ? kb1 : l < 192 ? kb2 : kb3;
+        const bool dense = ((kb >> (l & 63)) & 1ull) == (u64)HAP_DENSE;
+        const double2 *tp = tab + (size_t)h * stride_h + (size_t)l * 2;
+        const double2 ta = __ldg(tp);
+        const double2 tf = dense ? make_double2(0.0, 0.0) : __ldg(tp + 1);
+        double cf, cb;
+        layer_cost_pair(reinterpret_cast<const double2 *>(tcp + h), ta, tf, dense, kappa, cf, cb);
+        bad |= !(cf < 6.8719e10) | !(cb < 6.8719e10);                                 // 2^36 ns per layer
+        if (IsF64<VT>::value) { sC[(size_t)q * 2] = (VT)cf; sC[(size_t)q * 2 + 1] = (VT)cb; }
+        else { sC[(size_t)q * 2] = (VT)__double2ll_rn(cf); sC[(size_t)q * 2 + 1] = (VT)__double2ll_rn(cb); }
+    }
+    if (bad && range_flag) atomicOr(range_flag, 1ull);
+}
+
+// The same from the layer-cost array of a preceding launch, or computed here when the pass hands the constants instead.
+template <typename VT>
+__device__ __forceinline__ void trie_stage_costs(const DevConst &dc, const hap_pconf &pc, unsigned p_index, const VT *c2,
+                                                 const TypeConst *tcg, u64 *range_flag, VT *sC)
+{
+    const int N = dc.N, T = dc.T, tid = threadIdx.x, nthreads = blockDim.x;
+    if (!tcg) {
+        const longlong2 *src = reinterpret_cast<const longlong2 *>(c2 + (size_t)p_index * T * N * 2);
+        longlong2 *dst = reinterpret_cast<longlong2 *>(sC);
+        for (int q = tid; q < T * N; q += nthreads) dst[q] = src[q];
+        return;
+    }
+    const size_t row = ((size_t)pc.itp * dc.ncp + pc.icp) * dc.nmb + pc.ib;            // the same table row for every type
+    const size_t stride_h = (size_t)dc.ntp * dc.ncp * dc.nmb * N * 2;                   // 16-byte pairs between device types
+    trie_compute_costs<VT>(reinterpret_cast<const double2 *>(dc.tab4) + row * N * 2, stride_h, N, T, dc.kappa, dc.kindbits[0],
+                           dc.kindbits[1], dc.kindbits[2], dc.kindbits[3], tcg + (size_t)p_index * T, range_flag, sC);
+}
+
+// Block prologue, part 1: the weight and activation byte prefixes, MoE prefix counts, per-mask stage info, p2p
+// coefficients, the table of stage constants and a copy of the tree's node records.
 template <typename VT>
 __device__ __forceinline__ void trie_prologue_rows(
-    const DevConst &dc, const TrieMeta &tm, unsigned p_index, const VT *c2, const i64 *coef, const VT *coefv,
-    VT *sC, i64 *sW, i64 *sA, uint8_t *sK, double *sKtab, TrieNode *sNodes, uint16_t *sParent,
+    const DevConst &dc, const TrieMeta &tm, unsigned p_index, const i64 *coef, const VT *coefv,
+    i64 *sW, i64 *sA, uint8_t *sK, double *sKtab, TrieNode *sNodes, uint16_t *sParent,
     MaskInfo<VT> *minfo, VT (*sP2P)[6], double *szero)
 {
     const int N = dc.N, T = dc.T;
@@ -199,11 +244,6 @@ __device__ __forceinline__ void trie_prologue_rows(
     const int nmask = (1 << T) - 1;
     const i64 *cfp = coef + (size_t)p_index * T * HAP_NCOEF;         // byte coefficients: integers in both modes
     const VT *cvp = coefv + (size_t)p_index * T * HAP_NCOEF;         // time coefficients
-    {
-        const longlong2 *src = reinterpret_cast<const longlong2 *>(c2 + (size_t)p_index * T * N * 2);
-        longlong2 *dst = reinterpret_cast<longlong2 *>(sC);
-        for (int q = tid; q < T * N; q += nthreads) dst[q] = src[q];
-    }
     for (int l = tid; l <= N; l += nthreads) sK[l] = (uint8_t)moe_before(dc, l);
     if (tid < nmask) {
         const int mk = tid + 1;
@@ -381,12 +421,11 @@ __device__ __forceinline__ void trie_prologue_thr(
     __syncthreads();
 }
 
-template <typename T> struct IsF64 { static constexpr bool value = false; };
-template <> struct IsF64<double> { static constexpr bool value = true; };
-
 // VT: i64 (times rounded to integer ns: every operation below is exact) or double (fp64 mode: unrounded times,
 // the same steps in floating point; not instantiated for SEARCH).
-template <bool SEARCH, int MAXT, int MINB, typename VT = i64>
+// COUNT: also count the splits the block evaluates (after its early exits) into out.counters[4]; the counting costs a
+// few percent, so only passes of a problem created with HAP_OPT_COUNT_SPLITS run this form.
+template <bool SEARCH, int MAXT, int MINB, typename VT = i64, bool COUNT = false>
 __global__ void __launch_bounds__(MAXT, MINB)
 trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT *c2, const i64 *coef, const VT *coefv,
                const TrieMeta *metas, int n_parts, DpOut out)
@@ -400,6 +439,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     __shared__ i64 wcost[32];
     __shared__ u64 widx[32];
     __shared__ int s_skip;
+    __shared__ unsigned long long s_lb;
 
     const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, lane = tid & 31, wib = tid >> 5;
     if (blockIdx.x >= n_active) {
@@ -420,13 +460,19 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.thr_w;
     const u64 c_lo = pc.offset + (u64)tm.m_lo * n_rc, c_hi = c_lo + (u64)tm.nmap * n_rc;   // candidates of this block
     const u64 w_lo = out.first, w_hi = out.first + out.count;                  // candidates that are wanted
+    // how many wanted candidates this block stands for
+    auto block_candidates = [&]() -> u64 {
+        const u64 a = c_lo > w_lo ? c_lo : w_lo, b = c_hi < w_hi ? c_hi : w_hi;
+        return b > a ? b - a : 0;
+    };
     if (c_hi <= w_lo || c_lo >= w_hi) {
         if (SEARCH && tid == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
         return;
     }
-    if (SEARCH && out.prune) {
-        // T_iter >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on the summed stage time; one
-        // thread reads the moving incumbent and the block follows that reading as a whole
+    // T_iter >= S + (M-1) ceil(S / PP) with S the configuration's lower bound on the summed stage time (the sum over
+    // layers of the cheapest device type's time); one thread reads the moving incumbent and the block follows that
+    // reading as a whole.  S comes from the layer-cost kernel, or from this block's own layer times further down.
+    if (SEARCH && out.prune && !out.tcg) {
         if (tid == 0) {
             const i64 S = out.lb_sum[p];
             const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
@@ -434,8 +480,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
             s_skip = (u64)lb > inc;
             if (s_skip) {
                 out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
-                const u64 a = c_lo > w_lo ? c_lo : w_lo, b = c_hi < w_hi ? c_hi : w_hi;
-                atomicAdd(out.counters + 2, b - a);
+                atomicAdd(out.counters + 2, block_candidates());
             }
         }
         __syncthreads();
@@ -459,7 +504,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     TrieNode *sNodes = reinterpret_cast<TrieNode *>(ch + ((size_t)tm.cell_lo[PP] + 15) / 16 * 16);
     uint16_t *sParent = reinterpret_cast<uint16_t *>(sNodes + tm.node_lo[PP]);
 
-    trie_prologue_rows<VT>(dc, tm, p, c2, coef, coefv, sC, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
     const i64 *cfp = coef + (size_t)p * T * HAP_NCOEF;
 
     // writes "infeasible" for candidate c (non-search mode)
@@ -476,36 +520,88 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     i64 best_cost = kInf;
     u64 best_index = ~0ull;
     u64 n_eval = 0, n_feas = 0;
-    u32 n_cells32 = 0;                  // splits this thread evaluated
+    u32 n_cells32 = 0;                  // splits this thread evaluated (after the early exits)
     unsigned all_levels = 0;
     for (int q = 0; q < n_rc; ++q) all_levels |= dc.rc_masks[q];
 
     // ---- configurations whose first stage fits no device type at any level: nothing is feasible ----------
-    bool config_dead = false;
-    if (PP > 1) {
-        const u32 n_first = tm.node_lo[2] - tm.node_lo[1];
+    // Decided before anything is staged, from the byte coefficients alone: the memory of a span is its numbers of
+    // dense and MoE layers times the per-kind bytes.  Feasibility is monotone in the span, so the shortest first
+    // stage the band of a depth-1 node allows decides (PP = 1: the one stage holds all N layers).
+    {
+        const i64 mw0 = cfp[HAP_MW], mw1 = cfp[HAP_MW + 1], ma0 = cfp[HAP_MA], ma1 = cfp[HAP_MA + 1];
+        const i64 extra = cfp[HAP_MPRE] + (PP == 1 ? cfp[HAP_MPOST] : 0), mx = cfp[HAP_MX];
+        const i64 mstore = pc.M < PP ? pc.M : PP;
+        auto first_fits = [&](int b, i64 cap, int r) {
+            const i64 nm = moe_before(dc, b), nd = (i64)b - nm;
+            const i64 Wb = nd * mw0 + nm * mw1 + extra + (nm ? mx : 0);
+            const i64 A = mstore * (nd * ma0 + nm * ma1);
+            return Wb + (((i64)dc.xi_q[r] * A) >> 10) <= cap;
+        };
         int fits = 0;
-        for (u32 e = tid; e < n_first * (u32)R; e += nthreads) {
-            const u32 nd_i = e / R; const int r = (int)(e % R);
-            if (!((all_levels >> r) & 1u)) continue;
-            const TrieNode nd = sNodes[tm.node_lo[1] + nd_i];
-            if (nd.bl > nd.bh) continue;
-            const int capt = minfo[nd.mask - 1].capt;
-            const i64 mstore = pc.M < PP ? pc.M : PP;
-            // feasibility is monotone in the span: the shortest span the band allows decides
-            fits |= span_fits(sW, sA, sK, cfp[HAP_MPRE], cfp[HAP_MX], mstore, dc.cap_eff[capt], dc.xi_q[r], 0, nd.bl);
+        if (PP > 1) {
+            const u32 n_first = tm.node_lo[2] - tm.node_lo[1];
+            for (u32 e = tid; e < n_first * (u32)R; e += nthreads) {
+                const u32 nd_i = e / R; const int r = (int)(e % R);
+                if (!((all_levels >> r) & 1u)) continue;
+                const TrieNode nd = tm.nodes[tm.node_lo[1] + nd_i];
+                if (nd.bl > nd.bh) continue;
+                i64 cap = 0; bool seen = false;
+                for (int h = 0; h < T; ++h)
+                    if (nd.mask >> h & 1) { if (!seen || dc.cap_eff[h] < cap) cap = dc.cap_eff[h]; seen = true; }
+                fits |= first_fits(nd.bl, cap, r);
+            }
+        } else {
+            for (int e = tid; e < T * R; e += nthreads) {
+                const int t = e / R, r = e % R;
+                if (!((all_levels >> r) & 1u) || !((tm.tmask[1] >> t) & 1u)) continue;
+                fits |= first_fits(N, dc.cap_eff[t], r);
+            }
         }
-        config_dead = !__syncthreads_or(fits);
-    } else {
-        // a single stage holds all N layers with the pre- and post-processing state: on some type, at some level?
-        int fits = 0;
-        for (int e = tid; e < T * R; e += nthreads) {
-            const int t = e / R, r = e % R;
-            if (!((all_levels >> r) & 1u) || !((tm.tmask[1] >> t) & 1u)) continue;
-            fits |= span_fits(sW, sA, sK, cfp[HAP_MPRE] + cfp[HAP_MPOST], cfp[HAP_MX], pc.M < 1 ? pc.M : 1, dc.cap_eff[t], dc.xi_q[r], 0, N);
+        if (!__syncthreads_or(fits)) {
+            // every candidate of the block is infeasible: say so and leave
+            if (SEARCH) {
+                if (tid == 0) {
+                    out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
+                    atomicAdd(out.counters + 0, block_candidates());
+                }
+            } else {
+                const u64 a = c_lo > w_lo ? c_lo : w_lo, b = c_hi < w_hi ? c_hi : w_hi;
+                for (u64 c = a + tid; c < b; c += nthreads) put_infeasible(c);
+            }
+            return;
         }
-        config_dead = !__syncthreads_or(fits);
     }
+    const bool config_dead = false;
+
+    // ---- layer times of the configuration; in a pruning search whose blocks compute them, the lower bound too ----
+    trie_stage_costs<VT>(dc, pc, p, c2, out.tcg, out.range_flag, sC);
+    if (SEARCH && out.prune && out.tcg) {
+        if (tid == 0) s_lb = 0;
+        __syncthreads();
+        i64 lmin = 0;
+        for (int l = tid; l < N; l += nthreads) {
+            i64 m = 0;
+            for (int h = 0; h < T; ++h) { const i64 q = (i64)sC[((size_t)h * N + l) * 2] + (i64)sC[((size_t)h * N + l) * 2 + 1]; m = (h == 0 || q < m) ? q : m; }
+            lmin += m;
+        }
+        lmin = warp_sum_i64(lmin);
+        if (lane == 0 && lmin) atomicAdd(&s_lb, (unsigned long long)lmin);
+        __syncthreads();
+        if (tid == 0) {
+            const i64 S = (i64)s_lb;
+            const i64 lb = S + (i64)(pc.M - 1) * ((S + PP - 1) / PP);
+            const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+            s_skip = (u64)lb > inc;
+            if (s_skip) {
+                out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull;
+                atomicAdd(out.counters + 2, block_candidates());
+            }
+        }
+        __syncthreads();
+        if (s_skip) return;
+    }
+    trie_prologue_rows<VT>(dc, tm, p, coef, coefv, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
     if (!config_dead) {
         trie_prologue_time_rows<VT>(dc, tm, sC, sR);
         trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
@@ -531,7 +627,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
             if (lo < klo) lo = klo;
             if (lo > seg_hi) continue;
             const int n = seg_hi - lo + 1;
-            n_cells32 += (u32)n;
             // integer mode: (row[j] + K) - row[k], exact in any order; fp64 mode keeps the order (row[j] - row[k]) + K
             const double Rj = lds_f64<0>(a_row + 8u * (u32)j);
             const double Cj = F64 ? Rj : Rj + K;
@@ -553,9 +648,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
                 if (v1 <= best) { best = v1; a_arg = pa - 8; }
                 // layer times are non-negative, so the stage cost only grows as k falls within a level: once it
                 // exceeds the best value no further split of this level can reach it
-                if (c1 > best) break;
+                if (c1 > best) { if (COUNT) pa -= 16; break; }
                 pa -= 16; ra -= 16;
             }
+            if (COUNT) n_cells32 += ((a_prev + 8u * (u32)seg_hi) - pa) >> 3;      // splits evaluated (pa has stepped past them)
             seg_hi = lo - 1;
         }
         best_out = a_arg ? best : dInf;
@@ -698,7 +794,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
         if (!bott_any && c_lo >= w_lo && c_hi <= w_hi && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
     }
 
-    if (out.counters) {
+    if (COUNT && out.counters) {
         const u64 n_cells = (u64)warp_sum_i64((i64)n_cells32);
         if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
     }

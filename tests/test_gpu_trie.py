@@ -214,3 +214,35 @@ def test_fp64_mode_agrees_between_the_two_kernels(hap, name):
     both = fin & same_part
     assert np.allclose(a["cost"][both], b["cost"][both], rtol=1e-13, atol=0.0)
     assert np.array_equal(a["recompute"][both], b["recompute"][both])
+
+
+@pytest.mark.parametrize("name", ["tiny", "small", "dsv2", "stress"])
+def test_layer_costs_computed_inside_the_tree_blocks_equal_the_separate_launch(hap, name):
+    """By default the blocks of the tree kernel compute Eq. 2 for their configuration themselves; HAP_OPT_NO_FUSE keeps
+    the separate layer-cost launch.  Same arithmetic, so every output is identical, in both value types, and so are
+    the searches (with pruning: the lower bound then comes from the block's own layer times)."""
+    pb = problems.make_problem(name)
+    hp_f, fused = _pass(hap, pb, 0)
+    hp_s, sep = _pass(hap, pb, hap.OPT_NO_FUSE)
+    for key in ("cost", "bottleneck", "partition", "recompute"):
+        assert np.array_equal(fused[key], sep[key]), key
+    out_f = hap.hap_pipeline_dp_f64(hp_f, 0, hp_f.n_cand)
+    out_s = hap.hap_pipeline_dp_f64(hp_s, 0, hp_s.n_cand)
+    torch.cuda.synchronize()
+    assert np.array_equal(out_f["cost"].cpu().numpy(), out_s["cost"].cpu().numpy())
+    assert hap.hap_search_best(hp_f)[0] == hap.hap_search_best(hp_s)[0]
+    assert hap.hap_launches_per_pass(hp_f) + 1 == hap.hap_launches_per_pass(hp_s)
+    hap.hap_problem_destroy(hp_f)
+    hap.hap_problem_destroy(hp_s)
+    plans = []
+    for flags in (0, hap.OPT_NO_FUSE):
+        hp = hap.hap_problem_create(pb, prune=1, flags=flags)
+        hap.hap_enumerate(hp)
+        plan, stats = hap.hap_search_best(hp)
+        assert stats["n_evaluated"] + stats["n_pruned"] == hp.n_cand
+        plans.append(plan)
+        if name in ("small", "dsv2"):
+            plan64 = hap.hap_search_range_f64(hp, 0, hp.n_cand)
+            assert plan64["index"] == plan["index"] and plan64["n"] == plan["n"]
+        hap.hap_problem_destroy(hp)
+    assert plans[0] == plans[1]
