@@ -67,6 +67,7 @@ struct hap_problem {
     int joint_grid = 0;
     bool joint_ready = false;
     i64 *d_lb = nullptr;                    // scratch: per-configuration lower bound on the summed stage time
+    i64 *d_cand_lb = nullptr;               // scratch of the refinement searches: per-candidate bottleneck, then lower bound (first use)
     TypeConst *d_tc = nullptr;              // scratch: per (configuration, type) constants of the layer-cost kernels
     i64 *d_pcost = nullptr;                // per-block partial minima
     u64 *d_pindex = nullptr;
@@ -244,7 +245,7 @@ static void release_device(hap_problem *p)
     cached_free(p->d_tables); cached_free(p->d_arena); cached_free(p->d_trie_arena);
     cached_free(p->d_joint_scratch);
     for (auto &j : p->joint) { cached_free(j.d_ids); cached_free(j.d_arrays); }
-    cached_free(p->d_c2f); cached_free(p->d_coeff); cached_free(p->d_fcost);
+    cached_free(p->d_c2f); cached_free(p->d_coeff); cached_free(p->d_fcost); cached_free(p->d_cand_lb);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_pre) cudaEventDestroy(p->ev_pre);
@@ -1267,7 +1268,7 @@ static bool class_outside(const hap_problem *p, const hap_problem::PpClass &cl, 
 // counting and the one-candidate re-evaluation stay in pipeline_dp_kernel
 static bool pass_uses_trie(const hap_problem *p, const hap_problem::PpClass &cl, const DpOut &out, bool f64)
 {
-    const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
+    const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only && !out.force_plain;
     (void)f64;                                  // both value types walk the tree
     return cl.trie.ok && !out.count_only && !refine && p->dc.tau_linear != 0 && !out.dp_table && !out.choice && out.count > 1;
 }
@@ -1362,7 +1363,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         // skip classes whose candidates all lie outside the range
         if (!search && !out.first_dev && class_outside(p, cl, out)) continue;     // (a range that starts at a device-side index: every class looks)
         const bool lin = p->dc.tau_linear != 0;
-        const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only;
+        const bool refine = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0 && !out.count_only && !out.force_plain;
         const int variant = f64 ? 6 + (lin ? 1 : 0) : out.count_only ? 4 + (lin ? 1 : 0) : (refine ? 8 : 0) + (search ? 2 : 0) + (lin ? 1 : 0);
         const void *fn;
         if (f64) fn = lin ? (const void *)pipeline_dp_kernel<false, true, false, double> : (const void *)pipeline_dp_kernel<false, false, false, double>;
@@ -1378,7 +1379,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const unsigned blocks = (unsigned)(cl.item_hi - cl.item_lo);
         const uint8_t *tab = cl.has_tab ? p->d_maptab + cl.map_base : nullptr;
         DpOut o = out;
-        o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0;
+        o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0 && !out.force_plain;
         if (search) { o.partial_cost += cl.pslot_lo; o.partial_index += cl.pslot_lo; }
         if (pass_uses_trie(p, cl, out, f64)) {
             const hap_problem::Trie &tr = cl.trie;
@@ -1933,11 +1934,37 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     out.first = first; out.count = count; out.prune = p->opts.prune;
     out.partial_cost = p->d_pcost; out.partial_index = p->d_pindex; out.counters = p->d_counters;
     out.incumbent = p->d_counters + 3;
+    const bool refine_mode = (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0;
     const bool fused = pass_fuses_layer_costs(p, out, true);
     out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
     CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
     if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st, fused ? nullptr : p->d_lb)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
+    if (refine_mode && count > 1) {
+        // The refinement and the exact sweep cost one warp per candidate and up to dozens of passes each, so they run
+        // only where they can matter.  A plain pass over the prefix trees leaves every candidate's bottleneck B*; with
+        // S the configuration's lower bound on the stage-cost sum, no partition of the candidate gets below
+        // S + (M-1) B* (sync and optimizer terms only add).  The candidate with the smallest bound is evaluated first
+        // and its cost starts the incumbent; the refinement kernels then skip every candidate whose bound exceeds the
+        // incumbent (strict, so the (cost, index) minimum is unchanged).
+        if (!p->d_cand_lb) CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_cand_lb, (size_t)p->n_cand * sizeof(i64)));
+        DpOut plain{};
+        plain.bottleneck = p->d_cand_lb + first;         // the kernels index outputs by candidate - first: entry c of the array
+        plain.first = first; plain.count = count; plain.force_plain = 1; plain.range_flag = p->d_range;
+        if ((s = launch_decode_early(p, plain, false)) != HAP_OK) return s;
+        if ((s = launch_dp(p, plain, false, st)) != HAP_OK) return s;
+        cand_bound_kernel<<<(unsigned)p->pconfs.size(), 128, 0, st>>>(p->dc, p->d_lb, p->d_cand_lb, first, count);
+        CUDA_TRY(p, cudaGetLastError());
+        if ((s = argmin_launch(p, p->d_cand_lb + first, count, p->d_best, st, kInf)) != HAP_OK) return s;
+        offset_index_kernel<<<1, 32, 0, st>>>(p->d_best + 1, (i64)first);
+        SingleOut *d0 = (SingleOut *)p->d_single;
+        DpOut seed{};
+        seed.cost = &d0->cost; seed.first = 0; seed.count = 1; seed.first_dev = p->d_best + 1;
+        if ((s = launch_dp(p, seed, false, st)) != HAP_OK) return s;
+        set_incumbent_kernel<<<1, 32, 0, st>>>(p->d_counters + 3, &d0->cost, p->d_best + 1);
+        CUDA_TRY(p, cudaGetLastError());
+        out.cand_lb = p->d_cand_lb;
+    }
     if ((s = launch_decode_early(p, out, true)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
     argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->n_pslots, p->d_best, kInf);

@@ -109,6 +109,11 @@ struct DpOut {
     // Eq. 2; null: the blocks read the layer-cost array.  range_flag: set when a layer time leaves the supported range
     const struct TypeConst *tcg;
     u64 *range_flag;
+    // search with the refinement / exact objective: per-candidate lower bounds on T_iter from a preceding plain pass,
+    // indexed by the global candidate index (HAP_INF: the candidate has no feasible partition); a candidate whose
+    // bound exceeds the incumbent is skipped
+    const i64 *cand_lb;
+    int force_plain;                  // run the plain min-max pass although the problem asks for a refinement mode
 };
 
 // ------------------------------------------------------------------------------------------
@@ -1141,6 +1146,29 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
         __syncthreads();
         if (s_skip) return;
     }
+    if (SEARCH && out.cand_lb) {
+        // bounds of the block's candidates against the incumbent: when none can win, the block leaves before its prologue
+        const u64 c0 = pc.offset + it.lo * (u64)n_rc, c1 = c0 + (u64)it.count * n_rc;
+        const u64 a = c0 > out.first ? c0 : out.first, b = c1 < out.first + out.count ? c1 : out.first + out.count;
+        const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+        int alive = 0;
+        u64 n_inf = 0, n_cut = 0;
+        for (u64 c = a + threadIdx.x; c < b; c += blockDim.x) {
+            const i64 lb = out.cand_lb[c];
+            if (lb >= kInf) n_inf++;
+            else if ((u64)lb > inc) n_cut++;
+            else alive = 1;
+        }
+        if (!__syncthreads_or(alive)) {
+            n_inf = (u64)warp_sum_i64((i64)n_inf); n_cut = (u64)warp_sum_i64((i64)n_cut);
+            if (lane == 0) {
+                if (n_inf) atomicAdd(out.counters + 0, n_inf);
+                if (n_cut) atomicAdd(out.counters + 2, n_cut);
+            }
+            if (threadIdx.x == 0) { out.partial_cost[blockIdx.x] = kInf; out.partial_index[blockIdx.x] = ~0ull; }
+            return;
+        }
+    }
     const bool multiset = pc.mode == HAP_MAP_MULTISET;
     const int nmask = (1 << T) - 1;
     const int mrows = multiset ? T : nmask;
@@ -1211,6 +1239,17 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             mask = smap.mask; link = lane > 0 && lane < PP ? (smap.cls | (smap.ha << 2) | (smap.hb << 4)) : 0;
         }
         if (c < out.first || c >= out.first + out.count) { valid_rows = 0; dead_stage = 1 << 30; prev_mask = -1; continue; }
+        if (SEARCH && out.cand_lb) {
+            // the candidate's lower bound from the plain pass (one address for the whole warp, so one reading)
+            const i64 lb = out.cand_lb[c];
+            const u64 inc = *reinterpret_cast<volatile const u64 *>(out.incumbent);
+            if (lb >= kInf || (u64)lb > inc) {
+                valid_rows = 0; dead_stage = 1 << 30; prev_mask = -1;
+                if (lb >= kInf) n_eval++;
+                else if (lane == 0) atomicAdd(out.counters + 2, 1ull);
+                continue;
+            }
+        }
         if ((known_infeasible >> (mi - m_lo)) & 1ull) {
             // infeasible under a more permissive policy: infeasible here, nothing to compute
             infeasible_here |= 1ull << (mi - m_lo);
@@ -1575,7 +1614,7 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             if (T_iter < vInf) n_feas++;
             if (T_iter < best_cost || (T_iter == best_cost && c < best_index)) {
                 best_cost = T_iter; best_index = c;
-                if (out.prune && lane == 0) atomicMin(out.incumbent, (u64)(i64)T_iter);
+                if ((out.prune || out.cand_lb) && lane == 0) atomicMin(out.incumbent, (u64)(i64)T_iter);
             }
         } else {
             const u64 o = c - out.first;
@@ -1793,6 +1832,35 @@ joint_dp_kernel(const DevConst dc, const unsigned *pconf_ids, unsigned n_ids, co
 // ------------------------------------------------------------------------------------------
 // argmin: stage 1 reduces a slice per block, stage 2 (one block) reduces the partials
 // ------------------------------------------------------------------------------------------
+// Lower bounds on T_iter of the candidates of one configuration per block, from the bottlenecks a plain pass left in
+// `bound` (in place): any partition of candidate c has a largest stage cost >= B*(c) and a stage-cost sum >= S, the sum
+// over layers of the cheapest device type's time, so sum + (M-1) max >= S + (M-1) B*(c); infeasible stays HAP_INF.
+__global__ void cand_bound_kernel(const DevConst dc, const i64 *__restrict__ lb_sum, i64 *bound, u64 first, u64 count)
+{
+    const u64 p = blockIdx.x;
+    const hap_pconf pc = dc.pconf[p];
+    const u64 c0 = pc.offset, c1 = c0 + pc.nmap * (u64)dc.n_rc;
+    const u64 a = c0 > first ? c0 : first, b = c1 < first + count ? c1 : first + count;
+    const i64 S = lb_sum[p], m1 = (i64)pc.M - 1;
+    for (u64 c = a + threadIdx.x; c < b; c += blockDim.x) {
+        const i64 bott = bound[c];
+        bound[c] = bott >= kInf ? kInf : S + m1 * bott;
+    }
+}
+
+// an index relative to a range start becomes a global candidate index (negative: none, stays negative)
+__global__ void offset_index_kernel(i64 *index, i64 first)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0 && *index >= 0) *index += first;
+}
+
+// the incumbent of a search starts at the cost of one evaluated candidate
+// (index < 0: no candidate was evaluated, the incumbent stays at +INF)
+__global__ void set_incumbent_kernel(u64 *incumbent, const i64 *cost, const i64 *index)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) { const i64 c = *index < 0 ? kInf : *cost; *incumbent = c < kInf ? (u64)c : (u64)kInf; }
+}
+
 // "no candidate" into partial-minimum slots that no block of the pass writes
 __global__ void fill_partials_kernel(i64 *pcost, u64 *pindex, unsigned n)
 {

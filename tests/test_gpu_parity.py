@@ -439,3 +439,47 @@ def test_exact_mode_on_random_problems(hap, seed):
         if ex["T_iter"] < INF:
             assert ex["T_pipe"] == ex["brute_pipe"]
     hap.hap_problem_destroy(hp)
+
+
+def _configs_sampled(o, stride):
+    """Candidate index ranges of every `stride`-th configuration (what search_pconfs(0, stride) evaluates)."""
+    n_rc = o.n_cand and len(o.pb.rc_masks)
+    return [(int(o.pconfs["offset"][p]), int(o.pconfs["nmap"][p]) * n_rc) for p in range(0, o.n_pconf, stride)]
+
+
+@pytest.mark.parametrize("mode,stride", [("refine", 5), ("exact", 23)])
+def test_refinement_modes_on_the_stress_workload(hap, mode, stride):
+    """The refinement and the exact pipeline term at the benchmark's size: every candidate of every `stride`-th
+    configuration against the oracle; the bounded search (plain pass, per-candidate lower bounds, refinement only
+    where the bound can still win) returns the minimum of the unbounded pass over all candidates."""
+    pb = problems.stress()
+    o = Oracle(pb)
+    flag = hap.OPT_REFINE if mode == "refine" else hap.OPT_EXACT
+    search = o.search_pconfs_refined if mode == "refine" else o.search_pconfs_exact
+    done, _, _, costs, bn = search(0, stride, threads=NTHREADS)
+    hp = hap.hap_problem_create(pb, flags=flag)
+    hap.hap_enumerate(hp)
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    got, gotb = out["cost"].cpu().numpy(), out["bottleneck"].cpu().numpy()
+    n = 0
+    for off, cnt in _configs_sampled(o, stride):
+        assert np.array_equal(got[off:off + cnt], costs[off:off + cnt]), off
+        assert np.array_equal(gotb[off:off + cnt], bn[off:off + cnt]), off
+        n += cnt
+    assert n == done and (costs[costs >= 0] < INF).any()
+    plan, stats = hap.hap_search_best(hp)
+    am = int(np.argmin(got))
+    assert (plan["T_iter"], plan["index"]) == (int(got[am]), am)
+    # candidates without a feasible partition count as evaluated; nearly all others are cut by their bound
+    assert stats["n_evaluated"] + stats["n_pruned"] == hp.n_cand and stats["n_pruned"] > 0.9 * int((got < INF).sum())
+    # a range that does not hold the global optimum, and pruning by the configuration-level bound on top
+    first, count = hp.n_cand // 4, hp.n_cand // 3
+    sub, _ = hap.hap_search_range(hp, first, count)
+    am = int(np.argmin(got[first:first + count]))
+    assert (sub["T_iter"], sub["index"]) == (int(got[first + am]), first + am)
+    hap.hap_problem_destroy(hp)
+    hp = hap.hap_problem_create(pb, prune=1, flags=flag)
+    hap.hap_enumerate(hp)
+    assert hap.hap_search_best(hp)[0] == plan
+    hap.hap_problem_destroy(hp)
