@@ -154,7 +154,7 @@ def main():
     import torch
     import torch.distributed as dist
     import paper_2609_39350_b200 as hap
-    from paper_2609_39350_b200.sharding import shard_ranges, exchange_minimum, recurrence_cells
+    from paper_2609_39350_b200.sharding import shard_ranges, exchange_minimum_tensor, recurrence_cells, NO_CANDIDATE
     from gen import problems
 
     rank = int(os.environ.get("RANK", "0"))
@@ -212,8 +212,10 @@ def main():
         a.record(stream)
         am = step()
         if world > 1:
-            c, i = (int(x) for x in am.tolist())
-            best = exchange_minimum(c, i + first, device=xdev)
+            # one (cost, index) pair per rank, gathered and reduced on the device the backend talks on: no host
+            # round trip inside the step (gloo has no device path: the pair goes through the host there)
+            pair = am if am is not None else torch.tensor(NO_CANDIDATE, dtype=torch.int64, device="cuda")
+            best_t = exchange_minimum_tensor(pair if xdev == "cuda" else pair.cpu(), first)
         b.record(stream)
         b.synchronize()
         lc, dpk, cells = hap.hap_get_timings(hp)
@@ -229,6 +231,8 @@ def main():
     if world == 1:
         c, i = (int(x) for x in am.tolist())
         best = (c, i + first)
+    else:
+        best = tuple(int(x) for x in best_t.tolist())
 
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device=xdev)

@@ -979,6 +979,16 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
                       uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
                       int64_t *costs, int64_t *bottlenecks)
 {
+    return orc_search_pconfs_plans(pr, pcs, n_pconf, p_first, p_stride, n_done, best_cost, best_index, costs, bottlenecks,
+                                   NULL, NULL);
+}
+
+/* the same, also returning every candidate's partition (layers per stage) and recomputation levels,
+ * [n_cand][ORC_MAX_PP] each, zero for infeasible candidates */
+int orc_search_pconfs_plans(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
+                            uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
+                            int64_t *costs, int64_t *bottlenecks, uint8_t *parts, uint8_t *levels)
+{
     int64_t gbest = ORC_INF;
     uint64_t gidx = UINT64_MAX, done = 0;
     if (p_stride == 0) p_stride = 1;
@@ -1003,6 +1013,8 @@ int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pc
                 uint64_t idx = pc->offset + map_idx * (uint64_t)pr->n_rc + (uint64_t)rc;
                 if (costs) costs[idx] = res.T_iter;              /* indexed by candidate, whole space */
                 if (bottlenecks) bottlenecks[idx] = res.bottleneck;
+                if (parts) memcpy(parts + idx * ORC_MAX_PP, res.n, ORC_MAX_PP);
+                if (levels) memcpy(levels + idx * ORC_MAX_PP, res.r, ORC_MAX_PP);
                 if (res.T_iter < lbest) { lbest = res.T_iter; lidx = idx; }
                 done++;
             }

@@ -130,6 +130,9 @@ int orc_search(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, ui
 int orc_search_pconfs(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
                       uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
                       int64_t *costs, int64_t *bottlenecks);
+int orc_search_pconfs_plans(const orc_problem *pr, const orc_pconf *pcs, uint64_t n_pconf, uint64_t p_first,
+                            uint64_t p_stride, uint64_t *n_done, int64_t *best_cost, uint64_t *best_index,
+                            int64_t *costs, int64_t *bottlenecks, uint8_t *parts, uint8_t *levels);
 
 /* refinement: smallest sum of stage costs among the bottleneck-optimal partitions */
 int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, uint32_t rc_mask,

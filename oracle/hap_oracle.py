@@ -304,6 +304,21 @@ class Oracle:
             return int(done.value), int(bc.value), int(bi.value), costs, bn
         return int(done.value), int(bc.value), int(bi.value)
 
+    def search_pconfs_plans(self, p_first: int = 0, p_stride: int = 1, threads: int = 1):
+        """search_pconfs with every candidate's partition and recomputation levels ([n_cand][MAX_PP] uint8 each;
+        rows of candidates outside the selected configurations stay zero)."""
+        done = C.c_uint64(); bc = C.c_int64(); bi = C.c_uint64()
+        costs = np.full(self.n_cand, -1, np.int64); bn = np.full(self.n_cand, -1, np.int64)
+        parts = np.zeros((self.n_cand, MAX_PP), np.uint8); levels = np.zeros((self.n_cand, MAX_PP), np.uint8)
+        try:
+            C.CDLL("libgomp.so.1").omp_set_num_threads(C.c_int(threads))
+        except OSError:
+            pass
+        self.L.orc_search_pconfs_plans(C.byref(self.s), _ptr(self.pconfs), C.c_uint64(self.n_pconf), C.c_uint64(p_first),
+                                       C.c_uint64(p_stride), C.byref(done), C.byref(bc), C.byref(bi), _ptr(costs), _ptr(bn),
+                                       _ptr(parts), _ptr(levels))
+        return int(done.value), costs, bn, parts, levels
+
     # ---- refinement --------------------------------------------------------------------
     def candidate_refined(self, p, mp, rc_mask, c2, coef) -> Result:
         res = Result()

@@ -334,15 +334,28 @@ def hap_count_cells(hp: HapProblem, first: int, count: int, stream=None) -> int:
 ARGMIN_STATIC_MAX_COUNT = 1 << 26
 
 
+def _check_cost_tensor(cost):
+    import torch
+    if not (cost.is_cuda and cost.dtype == torch.int64 and cost.is_contiguous() and cost.numel() > 0):
+        raise HapError(1, "the cost array must be a non-empty contiguous int64 CUDA tensor")
+    if cost.device.index is not None and cost.device.index != torch.cuda.current_device():
+        raise HapError(1, "the cost array must live on the current CUDA device")
+
+
 def hap_argmin_static(cost, out=None, stream=None, count=None):
     """(cost, index) minimum of an int64 CUDA tensor through the entry point that allocates nothing
     inside the library: no problem handle, scratch in the library image.  `out` is a 2-element int64
     CUDA tensor (made here with torch if not given; pass your own when the caller must not allocate).
     `count` defaults to cost.numel()."""
     import torch
+    _check_cost_tensor(cost)
     if out is None:
         out = torch.empty(2, dtype=torch.int64, device=cost.device)
-    n = cost.numel() if count is None else count
+    if not (out.is_cuda and out.dtype == torch.int64 and out.is_contiguous() and out.numel() >= 2 and out.device == cost.device):
+        raise HapError(1, "hap_argmin_static: out must be a contiguous int64 CUDA tensor of 2 elements on the cost tensor's device")
+    n = cost.numel() if count is None else int(count)
+    if n < 1 or n > cost.numel():
+        raise HapError(4, f"hap_argmin_static: count {n} outside [1, {cost.numel()}] (the tensor's size)")
     st = load_library().hap_argmin_static(_dev(cost), C.c_uint64(n), _dev(out), _stream(stream))
     if st != 0:
         raise HapError(st, "hap_argmin_static: count must be in [1, 2^26] and the pointers non-null" if st in (1, 4) else "hap_argmin_static")
@@ -429,6 +442,7 @@ def hap_launches_per_pass(hp: HapProblem) -> int:
 def hap_argmin(hp: HapProblem, cost, stream=None):
     """(cost, index) minimum of an int64 CUDA tensor, lowest index on ties; returns a 2-element CUDA tensor."""
     import torch
-    out = torch.empty(2, dtype=torch.int64, device="cuda")
+    _check_cost_tensor(cost)
+    out = torch.empty(2, dtype=torch.int64, device=cost.device)
     hp.check(load_library().hap_argmin(hp.h, _dev(cost), C.c_uint64(cost.numel()), _dev(out), _stream(stream)))
     return out

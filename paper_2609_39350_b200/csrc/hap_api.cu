@@ -1224,16 +1224,33 @@ static hap_status launch_layer_kernel(hap_problem *p, i64 *c2, double *c2f, bool
     return HAP_OK;
 }
 
-static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st,
-                                     i64 *lb_sum = nullptr)
+// configurations that own candidates of [first, first + count): a contiguous range [lo, hi)
+static void configs_of_range(const hap_problem *p, u64 first, u64 count, unsigned &lo, unsigned &hi)
 {
-    const u64 nph = (u64)p->pconfs.size() * HAP_MAX_TYPES;
+    auto owner = [&](u64 c) {
+        size_t a = 0, b = p->pconfs.size();
+        while (b - a > 1) { const size_t mid = (a + b) / 2; if (p->pconfs[mid].offset <= c) a = mid; else b = mid; }
+        return (unsigned)a;
+    };
+    if (count == 0 || p->pconfs.empty()) { lo = hi = 0; return; }
+    lo = owner(first); hi = owner(first + count - 1) + 1;
+}
+
+// Per-type constants and stage coefficients, then (where an output array is given) the layer costs, of the
+// configurations [p_lo, p_hi): a pass over a candidate range touches only the configurations that own its candidates.
+static hap_status launch_layer_costs(hap_problem *p, i64 *c2, i64 *coef, double *c2f, double *coeff, bool quant, cudaStream_t st,
+                                     i64 *lb_sum = nullptr, unsigned p_lo = 0, unsigned p_hi = ~0u)
+{
+    if (p_hi > p->pconfs.size()) p_hi = (unsigned)p->pconfs.size();
+    if (p_lo >= p_hi) return HAP_OK;
+    const unsigned n_conf = p_hi - p_lo;
+    const u64 nph = (u64)n_conf * HAP_MAX_TYPES;
     const unsigned b1 = (unsigned)((nph + kLcThreads - 1) / kLcThreads);
-    if (quant) type_const_kernel<true><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr, p->d_range);
-    else type_const_kernel<false><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff, p->d_range);
+    if (quant) type_const_kernel<true><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, coef, nullptr, p->d_range, p_lo, n_conf);
+    else type_const_kernel<false><<<dim3(b1, 3), kLcThreads, 0, st>>>(p->dc, p->d_tc, nullptr, coeff, p->d_range, p_lo, n_conf);
     CUDA_TRY(p, cudaGetLastError());
     if ((quant && c2) || (!quant && c2f)) {
-        hap_status s = launch_layer_kernel(p, c2, c2f, quant, st, lb_sum, nullptr, 0, (unsigned)p->pconfs.size(), true);
+        hap_status s = launch_layer_kernel(p, c2, c2f, quant, st, lb_sum, nullptr, p_lo, n_conf, true);
         if (s != HAP_OK) return s;
     }
     CUDA_TRY(p, cudaGetLastError());
@@ -1341,6 +1358,8 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
     // the dynamic shared memory limit is a per-kernel, per-device attribute shared by every problem of the
     // process: raise it (never lower it) before a launch that needs more
     static size_t smem_limit[64][12];
+    static std::mutex limit_mu;                 // both tables of raised limits, for problems used from several host threads
+    std::lock_guard<std::mutex> limit_lock(limit_mu);
     const int dev = p->device & 63;
     // fork: every PP class runs on its own stream so that the tail of one class overlaps the next; a merged
     // candidate decode queued earlier in this pass joins first, so that the fork event covers it
@@ -1462,7 +1481,9 @@ extern "C" hap_status hap_pipeline_dp(hap_problem *p, uint64_t first, uint64_t c
     const bool fused = pass_fuses_layer_costs(p, out, false);
     out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
     CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
-    if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
+    unsigned p_lo, p_hi;
+    configs_of_range(p, first, count, p_lo, p_hi);
+    if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st, nullptr, p_lo, p_hi)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_decode_early(p, out, false)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, false, st)) != HAP_OK) return s;
@@ -1499,8 +1520,10 @@ extern "C" hap_status hap_pipeline_dp_f64(hap_problem *p, uint64_t first, uint64
     out.recompute = dev_recompute; out.first = first; out.count = count;
     const bool fused = pass_fuses_layer_costs(p, out, false);
     out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
-    if ((s = launch_layer_costs(p, nullptr, p->d_coef, nullptr, nullptr, true, st)) != HAP_OK) return s;
-    if ((s = launch_layer_costs(p, nullptr, nullptr, fused ? nullptr : p->d_c2f, p->d_coeff, false, st)) != HAP_OK) return s;
+    unsigned p_lo, p_hi;
+    configs_of_range(p, first, count, p_lo, p_hi);
+    if ((s = launch_layer_costs(p, nullptr, p->d_coef, nullptr, nullptr, true, st, nullptr, p_lo, p_hi)) != HAP_OK) return s;
+    if ((s = launch_layer_costs(p, nullptr, nullptr, fused ? nullptr : p->d_c2f, p->d_coeff, false, st, nullptr, p_lo, p_hi)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if ((s = launch_dp(p, out, false, st, true)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
@@ -1938,7 +1961,10 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
     const bool fused = pass_fuses_layer_costs(p, out, true);
     out.tcg = fused ? p->d_tc : nullptr; out.range_flag = p->d_range;
     CUDA_TRY(p, cudaEventRecord(p->ev_pre, st));
-    if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st, fused ? nullptr : p->d_lb)) != HAP_OK) return s;
+    unsigned p_lo, p_hi;
+    configs_of_range(p, first, count, p_lo, p_hi);
+    if (refine_mode && count > 1) { p_lo = 0; p_hi = ~0u; }          // (the bounds kernel below reads every configuration's S)
+    if ((s = launch_layer_costs(p, fused ? nullptr : p->d_c2, p->d_coef, nullptr, nullptr, true, st, fused ? nullptr : p->d_lb, p_lo, p_hi)) != HAP_OK) return s;
     CUDA_TRY(p, cudaEventRecord(p->ev[1], st));
     if (refine_mode && count > 1) {
         // The refinement and the exact sweep cost one warp per candidate and up to dozens of passes each, so they run
@@ -2039,8 +2065,11 @@ static __device__ __align__(256) unsigned char g_argmin_static_scratch[kStaticAr
 
 // In host code the name above is only a handle for the runtime, not an address a kernel can use.
 // The device address is looked up once per device (with that device current) and cached here.
+// The entry point has no handle, so it is the one most likely to be called from several host threads: the lookup
+// is serialised (a lock per call costs nothing beside two kernel launches).
 static void *g_argmin_static_ptr[64];
 static bool g_argmin_static_ready[64];
+static std::mutex g_argmin_static_mu;
 
 extern "C" hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count, int64_t *dev_out, void *stream)
 {
@@ -2049,13 +2078,23 @@ extern "C" hap_status hap_argmin_static(const int64_t *dev_cost, uint64_t count,
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return HAP_E_CUDA;
     if (dev < 0 || dev >= 64) return HAP_E_RANGE;
-    if (!g_argmin_static_ready[dev]) {
-        void *ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_argmin_static_scratch) != cudaSuccess || !ptr) return HAP_E_CUDA;
-        g_argmin_static_ptr[dev] = ptr;
-        g_argmin_static_ready[dev] = true;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_argmin_static_mu);
+        if (!g_argmin_static_ready[dev]) {
+            void *ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_argmin_static_scratch) != cudaSuccess || !ptr) return HAP_E_CUDA;
+            g_argmin_static_ptr[dev] = ptr;
+            g_argmin_static_ready[dev] = true;
+        }
+        scratch = g_argmin_static_ptr[dev];
     }
-    i64 *pcost = reinterpret_cast<i64 *>(g_argmin_static_ptr[dev]);
+    {   // the cost array must live on the current device (the scratch and the launches do)
+        cudaPointerAttributes at{};
+        if (cudaPointerGetAttributes(&at, dev_cost) != cudaSuccess) { cudaGetLastError(); return HAP_E_INVALID; }
+        if (at.type == cudaMemoryTypeDevice && at.device != dev) return HAP_E_INVALID;
+    }
+    i64 *pcost = reinterpret_cast<i64 *>(scratch);
     u64 *pindex = reinterpret_cast<u64 *>(pcost + kStaticArgminBlocks);
     cudaStream_t st = (cudaStream_t)stream;
     const unsigned blocks = (unsigned)((count + kStaticArgminTile - 1) / kStaticArgminTile);

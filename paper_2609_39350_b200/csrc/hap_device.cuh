@@ -276,7 +276,7 @@ __device__ __forceinline__ bool put_coef(i64 *coef, double *coeff, size_t at, in
 
 template <bool QUANT>
 __global__ void __launch_bounds__(kLcThreads)
-type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u64 *range_flag)
+type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u64 *range_flag, unsigned p_first, unsigned n_conf)
 {
     // the layer-cost kernel behind this one may start its table reads now (programmatic dependent launch)
     asm volatile("griddepcontrol.launch_dependents;");
@@ -284,9 +284,9 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
     const int role = blockIdx.y;
     const i64 H = dc.H;
     const u64 gid = (u64)blockIdx.x * kLcThreads + threadIdx.x;
-    const u64 p = gid / HAP_MAX_TYPES;
+    const u64 p = (u64)p_first + gid / HAP_MAX_TYPES;          // configurations [p_first, p_first + n_conf)
     const int h = (int)(gid % HAP_MAX_TYPES);
-    if (p >= dc.n_pconf || h >= T) return;
+    if (gid / HAP_MAX_TYPES >= n_conf || p >= dc.n_pconf || h >= T) return;
     const bool want_coef = (QUANT && coef) || (!QUANT && coeff);
     if (role != 0 && !want_coef) return;
     const hap_pconf pc = dc.pconf[p];

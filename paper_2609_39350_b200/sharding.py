@@ -59,3 +59,26 @@ def exchange_minimum(cost: int, index: int, device=None) -> Tuple[int, int]:
     gathered = [torch.empty_like(mine) for _ in range(dist.get_world_size())]
     dist.all_gather(gathered, mine)
     return combine_minima([(int(g[0]), int(g[1])) for g in gathered])
+
+
+NO_CANDIDATE = (1 << 62, (1 << 63) - 1)      # what a rank with an empty range contributes
+
+
+def exchange_minimum_tensor(pair, first: int):
+    """The same exchange without a host round trip: `pair` is the rank's (cost, index within its range) as a
+    2-element int64 tensor on the device the process group communicates on (what hap_argmin returns; NO_CANDIDATE for
+    an empty range); `first` is the start of the rank's range.  Returns the global (cost, index) as a tensor on that
+    device; nothing is read back here, so the caller decides when to synchronise."""
+    import torch
+    import torch.distributed as dist
+    mine = pair.clone()
+    mine[1] = torch.where(mine[0] < NO_CANDIDATE[0], mine[1] + first, mine[1])      # "no candidate" keeps its index
+    if not dist.is_available() or not dist.is_initialized() or dist.get_world_size() == 1:
+        return mine
+    world = dist.get_world_size()
+    gathered = torch.empty((world, 2), dtype=torch.int64, device=mine.device)
+    dist.all_gather_into_tensor(gathered, mine.reshape(1, 2))
+    cost = gathered[:, 0]
+    best = cost.min()
+    index = torch.where(cost == best, gathered[:, 1], torch.full_like(cost, NO_CANDIDATE[1])).min()
+    return torch.stack([best, index])

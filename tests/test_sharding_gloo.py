@@ -9,7 +9,8 @@ import pytest
 
 from gen import problems
 from oracle import Oracle
-from paper_2609_39350_b200.sharding import shard_ranges, combine_minima, exchange_minimum, recurrence_cells
+from paper_2609_39350_b200.sharding import (shard_ranges, combine_minima, exchange_minimum, exchange_minimum_tensor,
+                                            recurrence_cells, NO_CANDIDATE)
 
 
 def test_recurrence_cell_count_matches_the_loop_nest():
@@ -62,7 +63,8 @@ def _free_port():
     return port
 
 
-def _rank_main(rank, world, port, name, q):
+def _rank_main(rank, world, port, name, q, ranges):
+    import torch
     import torch.distributed as dist
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
@@ -70,30 +72,57 @@ def _rank_main(rank, world, port, name, q):
     try:
         pb = problems.make_problem(name)
         o = Oracle(pb)
-        first, count = shard_ranges(o.pconfs, len(pb.rc_masks), pb.N, world)[rank]
-        costs, _, best, _ = o.search(first, count)
-        mine = (best["T_iter"], best["index"]) if best is not None else (1 << 62, (1 << 63) - 1)
-        q.put((rank, mine, exchange_minimum(mine[0], mine[1])))
+        first, count = (ranges or shard_ranges(o.pconfs, len(pb.rc_masks), pb.N, world))[rank]
+        best = o.search(first, count)[2] if count else None
+        mine = (best["T_iter"], best["index"]) if best is not None else NO_CANDIDATE
+        # the tensor form takes the index relative to the range start, as hap_argmin returns it
+        local = torch.tensor([mine[0], mine[1] - first if best is not None else mine[1]], dtype=torch.int64)
+        combined_t = exchange_minimum_tensor(local, first if best is not None else 0)
+        q.put((rank, mine, exchange_minimum(mine[0], mine[1]), tuple(int(x) for x in combined_t.tolist())))
     finally:
         dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("name", ["tiny", "small"])
-def test_two_rank_search_over_gloo_equals_the_single_rank_search(name):
+def _run_ranks(name, world, ranges=None):
     import torch.multiprocessing as mp
-    world = 2
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
     port = _free_port()
-    procs = [ctx.Process(target=_rank_main, args=(r, world, port, name, q)) for r in range(world)]
+    procs = [ctx.Process(target=_rank_main, args=(r, world, port, name, q, ranges)) for r in range(world)]
     for p in procs:
         p.start()
-    got = [q.get(timeout=180) for _ in range(world)]
+    got = [q.get(timeout=300) for _ in range(world)]
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
+    return got
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_two_rank_search_over_gloo_equals_the_single_rank_search(name):
+    got = _run_ranks(name, 2)
     o = Oracle(problems.make_problem(name))
     _, _, best, _ = o.search()
-    for rank, mine, combined in got:
-        assert combined == (best["T_iter"], best["index"]), (rank, mine, combined)
-    assert len({m for _, m, _ in got}) == 2            # the two ranks really searched different ranges
+    for rank, mine, combined, combined_t in got:
+        assert combined == combined_t == (best["T_iter"], best["index"]), (rank, mine, combined, combined_t)
+    assert len({m for _, m, _, _ in got}) == 2            # the two ranks really searched different ranges
+
+
+@pytest.mark.parametrize("world", [3, 8])
+def test_more_ranks_and_an_empty_shard(world):
+    """World sizes 3 and 8 on the Tiny space; the last rank gets an empty range and contributes "no candidate"."""
+    pb = problems.tiny()
+    o = Oracle(pb)
+    ranges = shard_ranges(o.pconfs, len(pb.rc_masks), pb.N, world - 1) + [(o.n_cand, 0)]
+    assert sum(c for _, c in ranges) == o.n_cand
+    got = _run_ranks("tiny", world, ranges)
+    _, _, best, _ = o.search()
+    for rank, mine, combined, combined_t in got:
+        assert combined == combined_t == (best["T_iter"], best["index"]), (rank, mine, combined, combined_t)
+    assert [m for r, m, _, _ in got if r == world - 1] == [NO_CANDIDATE]
+
+
+def test_all_shards_empty_or_infeasible_yield_no_candidate():
+    import torch
+    t = exchange_minimum_tensor(torch.tensor(list(NO_CANDIDATE), dtype=torch.int64), 0)
+    assert tuple(int(x) for x in t.tolist()) == NO_CANDIDATE
