@@ -909,6 +909,48 @@ static std::vector<u32> class_plist(const hap_problem *p, const hap_problem::PpC
     return plist;
 }
 
+// ---- per-process cache of enumerations -----------------------------------------------------------------------
+struct EnumResult {
+    std::vector<hap_pconf> rows;
+    std::vector<WorkItem> items;
+    std::vector<hap_problem::PpClass> classes;       // streams, events and trees are per problem: empty here
+    uint64_t n_cand = 0;
+    u64 tab_bytes = 0;
+};
+namespace {
+std::mutex g_enum_cache_mu;
+std::map<std::string, std::shared_ptr<const EnumResult>> g_enum_cache;
+constexpr size_t kEnumCacheEntries = 64;
+}
+
+// every input of the enumeration loop nest and of the block shapes of the classes
+static std::string enum_cache_key(const hap_problem *p)
+{
+    std::string k("hap-enum-1");
+    const hap_model &mo = p->model;
+    const int64_t head[] = {mo.N, mo.S, mo.E, mo.GB, mo.nq, mo.nkv, p->T, p->W, p->prof.R, p->dc.tau_linear, p->opts.tp_max,
+                            p->opts.n_rc, (int64_t)p->opts.map_cap, (int64_t)(p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT | HAP_OPT_NO_MAPTAB))};
+    key_put(k, head);
+    for (int h = 0; h < p->T; ++h) key_put(k, p->m[h]);
+    auto put_list = [&](const std::vector<int> &v) { const int64_t n = (int64_t)v.size(); key_put(k, n); for (int x : v) key_put(k, x); };
+    put_list(p->pp_list); put_list(p->tp_list); put_list(p->cp_list); put_list(p->ep_list); put_list(p->tpe_list); put_list(p->mb_list);
+    return k;
+}
+
+static std::shared_ptr<const EnumResult> enum_cache_find(const std::string &key)
+{
+    std::lock_guard<std::mutex> lock(g_enum_cache_mu);
+    auto it = g_enum_cache.find(key);
+    return it == g_enum_cache.end() ? nullptr : it->second;
+}
+
+static void enum_cache_insert(const std::string &key, std::shared_ptr<const EnumResult> r)
+{
+    std::lock_guard<std::mutex> lock(g_enum_cache_mu);
+    if (g_enum_cache.size() >= kEnumCacheEntries) g_enum_cache.clear();
+    g_enum_cache[key] = std::move(r);
+}
+
 extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t *n_candidates)
 {
     if (!p) return HAP_E_INVALID;
@@ -916,114 +958,132 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
     if (!p->enumerated) {
         const hap_model &mo = p->model;
         const int N = mo.N, T = p->T;
+        // The configuration table, the work items and the PP classes are a function of the model's dimensions, the
+        // cluster inventory and the search options -- not of the profiled tables: they are kept per process, so that
+        // planning again for the same cluster and lists copies them instead of running the loop nest.
+        const std::string ekey = enum_cache_key(p);
+        std::shared_ptr<const EnumResult> er = enum_cache_find(ekey);
+        if (!er) {
+            auto fresh = std::make_shared<EnumResult>();
+            hap_status es = [&]() -> hap_status {
         std::vector<hap_pconf> rows;
-        rows.reserve(p->pp_list.size() * p->tp_list.size() * p->cp_list.size() * p->ep_list.size() * p->tpe_list.size() * p->mb_list.size() / 4 + 16);
-        uint64_t off = 0;
-        const uint64_t SAT = 1ull << 62;
-        for (int PP : p->pp_list) {
-            if (PP > N || PP > HAP_MAX_PP || p->W % PP) continue;
-            const int64_t G = p->W / PP;
-            if (G > 0x7fffffffll) continue;
-            bool homog = true;
-            int cnt[HAP_MAX_TYPES] = {0, 0, 0, 0};
-            for (int h = 0; h < T; ++h) { if (p->m[h] % G) homog = false; cnt[h] = (int)(p->m[h] / G); }
-            const uint64_t nms = homog ? sequences_sat(cnt, T, SAT) : 0;
-            const int mode = (homog && nms <= p->opts.map_cap) ? HAP_MAP_MULTISET : HAP_MAP_BLOCK;
-            uint64_t nmap = nms;
-            if (mode == HAP_MAP_BLOCK) { nmap = 1; for (int i = 2; i <= T; ++i) nmap *= (uint64_t)i; }
-            for (int itp = 0; itp < (int)p->tp_list.size(); ++itp) {
-                const int TP = p->tp_list[itp];
-                if (G % TP || TP > p->opts.tp_max || mo.nq % TP || mo.nkv % TP) continue;
-                for (int icp = 0; icp < (int)p->cp_list.size(); ++icp) {
-                    const int CP = p->cp_list[icp];
-                    if (G % ((int64_t)TP * CP) || mo.S % (2 * CP)) continue;
-                    const int64_t DP = G / ((int64_t)TP * CP);
-                    for (int iep = 0; iep < (int)p->ep_list.size(); ++iep) {
-                        const int EP = p->ep_list[iep];
-                        if (mo.E % EP || G % EP) continue;
-                        for (int TPE : p->tpe_list) {
-                            if (G % ((int64_t)EP * TPE) || TPE > p->opts.tp_max) continue;
-                            const int64_t EDP = G / ((int64_t)EP * TPE);
-                            for (int ib = 0; ib < (int)p->mb_list.size(); ++ib) {
-                                const int b = p->mb_list[ib];
-                                if (mo.GB % (DP * b)) continue;
-                                hap_pconf q{};
-                                q.PP = PP; q.TP = TP; q.CP = CP; q.DP = (int)DP; q.EP = EP; q.TPE = TPE; q.b = b;
-                                q.M = (int)(mo.GB / (DP * b)); q.EDP = (int)EDP; q.G = (int)G;
-                                q.itp = itp; q.icp = icp; q.ib = ib; q.iep = iep; q.mode = mode; q.reserved = 0;
-                                q.nmap = nmap; q.offset = off;
-                                if (nmap > (SAT - off) / (uint64_t)p->opts.n_rc) return fail(p, HAP_E_RANGE, "candidate space overflows 2^62");
-                                off += nmap * (uint64_t)p->opts.n_rc;
-                                rows.push_back(q);
+            rows.reserve(p->pp_list.size() * p->tp_list.size() * p->cp_list.size() * p->ep_list.size() * p->tpe_list.size() * p->mb_list.size() / 4 + 16);
+            uint64_t off = 0;
+            const uint64_t SAT = 1ull << 62;
+            for (int PP : p->pp_list) {
+                if (PP > N || PP > HAP_MAX_PP || p->W % PP) continue;
+                const int64_t G = p->W / PP;
+                if (G > 0x7fffffffll) continue;
+                bool homog = true;
+                int cnt[HAP_MAX_TYPES] = {0, 0, 0, 0};
+                for (int h = 0; h < T; ++h) { if (p->m[h] % G) homog = false; cnt[h] = (int)(p->m[h] / G); }
+                const uint64_t nms = homog ? sequences_sat(cnt, T, SAT) : 0;
+                const int mode = (homog && nms <= p->opts.map_cap) ? HAP_MAP_MULTISET : HAP_MAP_BLOCK;
+                uint64_t nmap = nms;
+                if (mode == HAP_MAP_BLOCK) { nmap = 1; for (int i = 2; i <= T; ++i) nmap *= (uint64_t)i; }
+                for (int itp = 0; itp < (int)p->tp_list.size(); ++itp) {
+                    const int TP = p->tp_list[itp];
+                    if (G % TP || TP > p->opts.tp_max || mo.nq % TP || mo.nkv % TP) continue;
+                    for (int icp = 0; icp < (int)p->cp_list.size(); ++icp) {
+                        const int CP = p->cp_list[icp];
+                        if (G % ((int64_t)TP * CP) || mo.S % (2 * CP)) continue;
+                        const int64_t DP = G / ((int64_t)TP * CP);
+                        for (int iep = 0; iep < (int)p->ep_list.size(); ++iep) {
+                            const int EP = p->ep_list[iep];
+                            if (mo.E % EP || G % EP) continue;
+                            for (int TPE : p->tpe_list) {
+                                if (G % ((int64_t)EP * TPE) || TPE > p->opts.tp_max) continue;
+                                const int64_t EDP = G / ((int64_t)EP * TPE);
+                                for (int ib = 0; ib < (int)p->mb_list.size(); ++ib) {
+                                    const int b = p->mb_list[ib];
+                                    if (mo.GB % (DP * b)) continue;
+                                    hap_pconf q{};
+                                    q.PP = PP; q.TP = TP; q.CP = CP; q.DP = (int)DP; q.EP = EP; q.TPE = TPE; q.b = b;
+                                    q.M = (int)(mo.GB / (DP * b)); q.EDP = (int)EDP; q.G = (int)G;
+                                    q.itp = itp; q.icp = icp; q.ib = ib; q.iep = iep; q.mode = mode; q.reserved = 0;
+                                    q.nmap = nmap; q.offset = off;
+                                    if (nmap > (SAT - off) / (uint64_t)p->opts.n_rc) return fail(p, HAP_E_RANGE, "candidate space overflows 2^62");
+                                    off += nmap * (uint64_t)p->opts.n_rc;
+                                    rows.push_back(q);
+                                }
                             }
                         }
                     }
                 }
             }
-        }
-        if (rows.empty()) return fail(p, HAP_E_INFEASIBLE, "no parallel configuration divides the cluster");
-        if (rows.size() > 0xffffffffull) return fail(p, HAP_E_RANGE, "too many configurations");
+            if (rows.empty()) return fail(p, HAP_E_INFEASIBLE, "no parallel configuration divides the cluster");
+            if (rows.size() > 0xffffffffull) return fail(p, HAP_E_RANGE, "too many configurations");
 
-        // PP classes (heaviest first).  Each class is one launch with its own block shape; a class keeps a
-        // table of its decoded mappings when that table is small.
-        std::vector<int> pps;
-        for (const auto &r : rows) if (std::find(pps.begin(), pps.end(), r.PP) == pps.end()) pps.push_back(r.PP);
-        std::sort(pps.begin(), pps.end(), [](int a, int b) { return a > b; });
-        std::vector<WorkItem> items;
-        items.reserve(rows.size() * 2);
-        std::vector<hap_problem::PpClass> classes;
-        u64 tab_bytes = 0;
-        for (int PP : pps) {
-            hap_problem::PpClass cl{};
-            cl.PP = PP;
-            cl.masks_used = 0xffffffffu;
-            cl.stream = nullptr; cl.done = nullptr;
-            cl.warps = 0;
-            // the rows of a PP value are contiguous (PP is the outermost loop of the enumeration)
-            size_t row_lo = 0;
-            while (row_lo < rows.size() && rows[row_lo].PP != PP) ++row_lo;
-            size_t row_hi = row_lo;
-            while (row_hi < rows.size() && rows[row_hi].PP == PP) ++row_hi;
-            cl.multiset = rows[row_lo].mode == HAP_MAP_MULTISET;
-            // most warps per SM: try block shapes from large to small, keep the one with the most resident warps
-            int best_resident = 0;
-            const uint64_t class_nmap = rows[row_lo].nmap;
-            const uint64_t per_pconf = class_nmap * (uint64_t)p->opts.n_rc;     // candidates a block can have at most
-            for (int w : {12, 8, 6, 4, 2, 1}) {
-                if ((uint64_t)w * 8 > per_pconf && w > 2) continue;             // keep about 8 candidates per warp
-                const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0,
-                                                (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0);
-                if (sm > 227 * 1024) continue;
-                const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), std::min(32, 64 / w));
-                const int resident = std::min(per_sm * w, 24);           // registers allow about 24 warps per SM
-                if (resident > best_resident) { best_resident = resident; cl.warps = w; cl.smem = sm; }
-            }
-            if (!cl.warps) return fail(p, HAP_E_RANGE, "shared memory need of a PP=%d block exceeds the SM", PP);
-            // a warp takes a slice of at most 64 consecutive mappings (one bit each in its infeasibility masks)
-            const uint64_t chunk_cap = 32ull * cl.warps;
-            cl.item_lo = items.size();
-            uint64_t nmap = 0;
-            for (size_t pi = row_lo; pi < row_hi; ++pi) {
-                nmap = rows[pi].nmap;
-                const uint64_t n_chunks = (nmap + chunk_cap - 1) / chunk_cap;
-                const uint64_t chunk = (nmap + n_chunks - 1) / n_chunks;          // balanced chunks
-                for (uint64_t lo = 0; lo < nmap; lo += chunk) {
-                    WorkItem it; it.p = (uint32_t)pi; it.lo = lo; it.count = (uint32_t)std::min<uint64_t>(chunk, nmap - lo);
-                    items.push_back(it);
+            // PP classes (heaviest first).  Each class is one launch with its own block shape; a class keeps a
+            // table of its decoded mappings when that table is small.
+            std::vector<int> pps;
+            for (const auto &r : rows) if (std::find(pps.begin(), pps.end(), r.PP) == pps.end()) pps.push_back(r.PP);
+            std::sort(pps.begin(), pps.end(), [](int a, int b) { return a > b; });
+            std::vector<WorkItem> items;
+            items.reserve(rows.size() * 2);
+            std::vector<hap_problem::PpClass> classes;
+            u64 tab_bytes = 0;
+            for (int PP : pps) {
+                hap_problem::PpClass cl{};
+                cl.PP = PP;
+                cl.masks_used = 0xffffffffu;
+                cl.stream = nullptr; cl.done = nullptr;
+                cl.warps = 0;
+                // the rows of a PP value are contiguous (PP is the outermost loop of the enumeration)
+                size_t row_lo = 0;
+                while (row_lo < rows.size() && rows[row_lo].PP != PP) ++row_lo;
+                size_t row_hi = row_lo;
+                while (row_hi < rows.size() && rows[row_hi].PP == PP) ++row_hi;
+                cl.multiset = rows[row_lo].mode == HAP_MAP_MULTISET;
+                // most warps per SM: try block shapes from large to small, keep the one with the most resident warps
+                int best_resident = 0;
+                const uint64_t class_nmap = rows[row_lo].nmap;
+                const uint64_t per_pconf = class_nmap * (uint64_t)p->opts.n_rc;     // candidates a block can have at most
+                for (int w : {12, 8, 6, 4, 2, 1}) {
+                    if ((uint64_t)w * 8 > per_pconf && w > 2) continue;             // keep about 8 candidates per warp
+                    const size_t sm = dp_smem_bytes(N, PP, T, p->prof.R, w, cl.multiset, p->dc.tau_linear != 0,
+                                                    (p->opts.flags & (HAP_OPT_REFINE | HAP_OPT_EXACT)) != 0);
+                    if (sm > 227 * 1024) continue;
+                    const int per_sm = std::min<int>((int)((227 * 1024) / (sm + 1024)), std::min(32, 64 / w));
+                    const int resident = std::min(per_sm * w, 24);           // registers allow about 24 warps per SM
+                    if (resident > best_resident) { best_resident = resident; cl.warps = w; cl.smem = sm; }
                 }
+                if (!cl.warps) return fail(p, HAP_E_RANGE, "shared memory need of a PP=%d block exceeds the SM", PP);
+                // a warp takes a slice of at most 64 consecutive mappings (one bit each in its infeasibility masks)
+                const uint64_t chunk_cap = 32ull * cl.warps;
+                cl.item_lo = items.size();
+                uint64_t nmap = 0;
+                for (size_t pi = row_lo; pi < row_hi; ++pi) {
+                    nmap = rows[pi].nmap;
+                    const uint64_t n_chunks = (nmap + chunk_cap - 1) / chunk_cap;
+                    const uint64_t chunk = (nmap + n_chunks - 1) / n_chunks;          // balanced chunks
+                    for (uint64_t lo = 0; lo < nmap; lo += chunk) {
+                        WorkItem it; it.p = (uint32_t)pi; it.lo = lo; it.count = (uint32_t)std::min<uint64_t>(chunk, nmap - lo);
+                        items.push_back(it);
+                    }
+                }
+                cl.item_hi = items.size();
+                cl.has_tab = !(p->opts.flags & HAP_OPT_NO_MAPTAB) && nmap * (uint64_t)PP * 2 <= (64ull << 20) &&
+                             tab_bytes + nmap * PP * 2 <= (256ull << 20);
+                cl.map_base = tab_bytes;
+                if (cl.has_tab) tab_bytes += (nmap * (uint64_t)PP * 2 + 255) / 256 * 256;
+                classes.push_back(cl);
             }
-            cl.item_hi = items.size();
-            cl.has_tab = !(p->opts.flags & HAP_OPT_NO_MAPTAB) && nmap * (uint64_t)PP * 2 <= (64ull << 20) &&
-                         tab_bytes + nmap * PP * 2 <= (256ull << 20);
-            cl.map_base = tab_bytes;
-            if (cl.has_tab) tab_bytes += (nmap * (uint64_t)PP * 2 + 255) / 256 * 256;
-            classes.push_back(cl);
-        }
-        if (items.size() > 0x7fffffffull) return fail(p, HAP_E_RANGE, "too many work items");
+            if (items.size() > 0x7fffffffull) return fail(p, HAP_E_RANGE, "too many work items");
 
-        p->pconfs.swap(rows);
-        p->items.swap(items);
-        p->classes.swap(classes);
+            fresh->rows.swap(rows); fresh->items.swap(items); fresh->classes.swap(classes);
+            fresh->n_cand = off; fresh->tab_bytes = tab_bytes;
+            return HAP_OK;
+            }();
+            if (es != HAP_OK) return es;
+            enum_cache_insert(ekey, fresh);
+            er = fresh;
+        }
+        p->pconfs = er->rows;
+        p->items = er->items;
+        p->classes = er->classes;
+        const uint64_t off = er->n_cand;
+        const u64 tab_bytes = er->tab_bytes;
         p->n_cand = off;
         const size_t np = p->pconfs.size();
         // one allocation for everything whose size the enumeration fixes (an allocation costs far more than the
