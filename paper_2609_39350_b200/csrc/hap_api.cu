@@ -101,8 +101,8 @@ struct SingleOut {
 // classes ordered from the deepest pipeline down.  A block of a deep class is a long chain of short steps (one
 // barrier-separated depth of its tree per stage and policy) that leaves most issue slots idle, a block of the class
 // with the most mappings keeps them busy but fills an SM's registers: the deep classes' blocks should be resident
-// first and the busy class should fill in behind them, so the streams get priorities in class order (measured at the
-// Stress workload: DP phase 0.46 -> 0.42 ms and the same time in every pass instead of 0.44-0.50).
+// first and the busy class should fill in behind them, so the streams get priorities in class order: the phase is
+// shorter and takes the same time in every pass.
 static cudaStream_t pooled_stream(int device, size_t index)
 {
     static std::mutex mu;

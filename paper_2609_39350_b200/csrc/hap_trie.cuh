@@ -608,6 +608,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     }
 
     const u32 a_thr = smem_u32(thr), a_sR = smem_u32(sR);
+    const bool all_flat = tm.all_flat != 0;
+    const int kind0 = layer_kind(dc, 0);
 
     // One cell: min over k in [klo, khi] of max(prev[k], cost(k, j)), smallest k on ties.  k runs downward over the
     // level segments given by the memory thresholds (lowest allowed level that fits); prev[k] and the time row
@@ -733,6 +735,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
             VT sum = 0, mxc = 0, t_sync = 0, t_opt = 0, het = 0;
             const u64 o = c - out.first;
             int b = N, a = arg;
+            double Kd = (double)stage_K(PP, mask, link);          // stage constant of the stage at hand (exact in a double)
             for (int d = PP; d >= 1; --d) {
                 // the ancestor's record is fetched before this stage's arithmetic needs to wait for it
                 uint4 raw = make_uint4(0, 0, 0, 0);
@@ -744,17 +747,25 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
                 }
                 if (!HAP_CHECK_OK(5, a >= 0 && a < b && b <= N && mask >= 1 && mask <= kMaxMasks)) break;
                 const MaskInfo<VT> &mi = minfo[mask - 1];
-                if (!HAP_CHECK_OK(6, trie_thr_index(tm, T, R, d, mi.capt, 0, b) + (u32)(R - 1) * (u32)bw < (u32)thr_bytes)) break;
-                const uint8_t *th = thr + trie_thr_index(tm, T, R, d, mi.capt, 0, b);
+                const u32 ti = all_flat ? (u32)(((d - 1) * T + mi.capt) * R) : trie_thr_index(tm, T, R, d, mi.capt, 0, b);
+                if (!HAP_CHECK_OK(6, ti + (u32)(R - 1) * (u32)bw < (u32)thr_bytes)) break;
+                const uint8_t *th = thr + ti;
                 int r = 0;
                 for (; r < R; ++r)
                     if (((rc_mask >> r) & 1u) && b - (int)th[r * bw] <= a) break;
-                const double *rr = sR + ((size_t)tm.mrow_of[mask] * R + r) * n1;
-                const VT cst = (VT)(rr[b] - rr[a]) + stage_K(d, mask, link);
+                const int mrow = tm.mrow_of[mask];
+                const double *rr = sR + ((size_t)mrow * R + r) * n1;
+                const VT cst = (VT)((rr[b] - rr[a]) + Kd);
                 sum += cst; mxc = cst > mxc ? cst : mxc;
-                const VT n_moe = (VT)((int)sK[b] - (int)sK[a]), n_dense = (VT)(b - a) - n_moe;
-                const VT sy = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
-                const VT op = n_dense * mi.opt[0] + n_moe * mi.opt[1];
+                VT sy, op;
+                if (dc.kind_uniform) {                               // one layer kind: the terms are a count times a coefficient
+                    const VT n = (VT)(b - a);
+                    sy = mi.slat + n * mi.sbw[kind0]; op = n * mi.opt[kind0];
+                } else {
+                    const VT n_moe = (VT)((int)sK[b] - (int)sK[a]), n_dense = (VT)(b - a) - n_moe;
+                    sy = mi.slat + n_dense * mi.sbw[0] + n_moe * mi.sbw[1];
+                    op = n_dense * mi.opt[0] + n_moe * mi.opt[1];
+                }
                 t_sync = sy > t_sync ? sy : t_sync; t_opt = op > t_opt ? op : t_opt;
                 if (dc.eta_q > 0 && d > 1 && (link & 3) == HAP_CROSS) het += sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
                 if (!SEARCH) {
@@ -767,6 +778,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
                     a = ch[tm.cell_lo[d - 1] + raw.x + (u32)(b - (int)(raw.w & 255))];
                     mask = raw.z & 255; link = (raw.z >> 8) & 255;
                     node = parent;
+                    // the stage constant of stage d-1 from the block's table: pre-work of a first stage by row group,
+                    // transfer into a later stage by receiving type and link class (the entries the cells use)
+                    const int cls = link & 3;
+                    Kd = sKtab[d == 2 ? (int)tm.mrow_of[mask] : 16 + ((link >> 4) & 3) * 6 + (cls == HAP_CROSS ? 2 + ((link >> 2) & 3) : cls)];
                 }
             }
             VT T_pipe = sum + (VT)(pc.M - 1) * mxc;
