@@ -143,6 +143,8 @@ def main():
     ap.add_argument("--workload", default="stress")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="run the warm-up and the timed steps and stop (for profiler captures): prints a reduced line")
     ap.add_argument("--delta-q", type=int, default=None, help="override the load-balance window (1/1024; <0 = off)")
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
                     help="torch.distributed backend of the (cost, index) exchange when launched with several ranks")
@@ -235,6 +237,15 @@ def main():
         best = tuple(int(x) for x in best_t.tolist())
 
     step_ms = [a.elapsed_time(b) for a, b in ev]
+    if args.timed_only:
+        if rank == 0:
+            print(json.dumps(dict(metric=METRIC, unit=UNIT, value=n_cand * args.steps / (sum(step_ms) * 1e-3), n_gpus=world,
+                                  steps=args.steps, warmup=warmup, ms_per_step=sum(step_ms) / args.steps,
+                                  config=dict(workload=args.workload), note="timed region only (--timed-only)")))
+        hap.hap_problem_destroy(hp)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     total_ms = torch.tensor([sum(step_ms)], dtype=torch.float64, device=xdev)
     if world > 1:
         dist.all_reduce(total_ms, op=dist.ReduceOp.MAX)

@@ -190,10 +190,9 @@ __device__ __forceinline__ int lds_u8(u32 a)
 
 // Layer times of the configuration into shared memory, computed from the profiled tables and the per-(configuration,
 // type) constants of Eq. 2: one thread per (type, layer), with the arithmetic of layer_cost_kernel (same function,
-// same bits).  Kept out of line (it runs once per block and would otherwise raise the register pressure of the split
-// loop); takes scalars, not the by-value constant block, so that nothing is copied to local memory.  No barrier.
+// same bits).  No barrier.
 template <typename VT>
-__device__ __noinline__ void trie_compute_costs(const double2 *tab, size_t stride_h, int N, int T, double kappa, u64 kb0, u64 kb1,
+__device__ __forceinline__ void trie_compute_costs(const double2 *tab, size_t stride_h, int N, int T, double kappa, u64 kb0, u64 kb1,
                                                 u64 kb2, u64 kb3, const TypeConst *tcp, u64 *range_flag, VT *sC)
 {
     bool bad = false;
@@ -439,6 +438,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     __shared__ i64 wcost[32];
     __shared__ u64 widx[32];
     __shared__ int s_skip;
+    __shared__ u64 s_clo;               // first candidate of the block
+    __shared__ int s_whole;             // every candidate of the block is wanted
     __shared__ unsigned long long s_lb;
 
     const int tid = threadIdx.x, nthreads = blockDim.x, nwarps = nthreads >> 5, lane = tid & 31, wib = tid >> 5;
@@ -460,6 +461,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     const int N = dc.N, T = dc.T, R = dc.R, n1 = N + 1, PP = pc.PP, n_rc = dc.n_rc, bw = tm.thr_w;
     const u64 c_lo = pc.offset + (u64)tm.m_lo * n_rc, c_hi = c_lo + (u64)tm.nmap * n_rc;   // candidates of this block
     const u64 w_lo = out.first, w_hi = out.first + out.count;                  // candidates that are wanted
+    // (the phases after the prologue read the block's range from shared memory: fewer live registers in the split loop)
+    if (tid == 0) { s_clo = c_lo; s_whole = c_lo >= w_lo && c_hi <= w_hi; }
     // how many wanted candidates this block stands for
     auto block_candidates = [&]() -> u64 {
         const u64 a = c_lo > w_lo ? c_lo : w_lo, b = c_hi < w_hi ? c_hi : w_hi;
@@ -706,8 +709,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
         int any_plan = 0;
         const u32 a_last = smem_u32(PP == 1 ? szero : (((PP - 1) & 1) ? bufO : bufE));
         for (u32 m = tid; m < tm.nmap; m += nthreads) {
-            const u64 c = c_lo + (u64)m * n_rc + (u64)rc_idx;
-            if (c < w_lo || c >= w_hi) continue;
+            const u64 c = s_clo + (u64)m * n_rc + (u64)rc_idx;
+            if (c < out.first || c >= out.first + out.count) continue;
             if (!HAP_CHECK_OK(3, c - out.first < out.count)) continue;
             double bott_d = dInf; int arg = 255;
             int mask = 0, link = 0;
@@ -806,7 +809,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
         // the barrier also keeps the next policy from overwriting rows and choices that are still being read
         const int bott_any = __syncthreads_or(any_plan);
         // a policy under which none of the block's mappings has a feasible partition settles its subsets
-        if (!bott_any && c_lo >= w_lo && c_hi <= w_hi && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
+        if (!bott_any && s_whole && dc.eta_q <= 0) policies_without_plan |= 1u << rc_pos;
     }
 
     if (COUNT && out.counters) {
