@@ -223,7 +223,11 @@ hap_status hap_release_cached_memory(void);
 
 /* Sec. 3.5 / 5.1 "searches the 6D parallel space": enumerates every (PP,TP,CP,DP,EP,TPE) with
  * PP*TP*CP*DP = #devices, EP*TPE | TP*CP*DP, EP | E, x micro-batch size, in a fixed
- * lexicographic order, counts the stage mappings of each and builds the device-side tables. */
+ * lexicographic order, counts the stage mappings of each and builds the device-side tables.
+ * What depends on the model's dimensions, the cluster and the search options only -- the configuration table, the
+ * work items and the prefix trees of the classes' stage mappings -- is kept per process (host memory, at most a few
+ * hundred entries, keyed by exactly those inputs) and copied when a later problem has the same key: planning again on
+ * the same cluster with new profiled tables skips the loop nest and the tree build. */
 hap_status hap_enumerate(hap_problem *, uint64_t *n_pconf, uint64_t *n_candidates);
 hap_status hap_get_pconfs(const hap_problem *, hap_pconf *host_out, uint64_t cap);
 
@@ -241,7 +245,9 @@ hap_status hap_eval_layer_costs_f64(hap_problem *, double *dev_c2, double *dev_c
 /* Sec. 3.5 (non-uniform layer assignment, Pruning 1 and 2) with the min-max recurrence
  * DP[i][j] = min_k max(DP[i-1][k], cost_i(k,j)), backtrace, and Eq. 4 in the closed form
  * sum_i c_i + (M-1) max_i c_i + T_dp-sync + T_opt, for candidates [first, first+count).
- * Recomputes the layer costs into library-owned memory first.  No candidate is skipped.
+ * The layer costs (Eq. 2) are recomputed first: inside the blocks of the dynamic program where the pass walks the
+ * classes' prefix trees (the default), into library-owned memory by a separate launch otherwise.  No candidate is
+ * skipped.
  * dev_cost, dev_bottleneck: [count] (HAP_INF when infeasible)
  * dev_partition, dev_recompute: [count][HAP_MAX_PP] (nullable; zero when infeasible)
  * dev_dp_table: [count][HAP_MAX_PP+1][N+1] int64, rows 0..PP written (nullable)
@@ -266,7 +272,13 @@ hap_status hap_search_range_f64(hap_problem *, uint64_t first, uint64_t count, h
 
 /* Eq. 1: layer costs, dynamic program and argmin over candidates [first, first+count) with
  * ties going to the lowest index; writes the plan to host memory.  Synchronises `stream`.
- * host_stats is nullable.  Returns HAP_E_INFEASIBLE when no candidate is feasible. */
+ * host_stats is nullable.  Returns HAP_E_INFEASIBLE when no candidate is feasible.
+ * With opts.prune, blocks whose configuration-level lower bound exceeds the incumbent are skipped (strict bound:
+ * same plan).  Under HAP_OPT_REFINE / HAP_OPT_EXACT a plain pass first bounds every candidate from below by
+ * S + (M-1) B* (B* its bottleneck, S the configuration's sum over layers of the cheapest type's time) and the
+ * refinement runs only for candidates whose bound does not exceed the incumbent; host_stats->n_pruned counts the
+ * candidates cut this way, candidates without a feasible partition count as evaluated.  The first such call
+ * allocates 8 bytes per candidate of scratch. */
 hap_status hap_search_range(hap_problem *, uint64_t first, uint64_t count, hap_plan *host_out,
                             hap_search_stats *host_stats, void *stream);
 /* The whole candidate space. */

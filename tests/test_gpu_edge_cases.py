@@ -1,5 +1,7 @@
 """Edge cases of the CUDA path against the oracle: maximum sizes, degenerate sizes, one device type,
 many recomputation levels and policies, in-kernel unranking instead of the mapping table, value limits."""
+import os
+
 import numpy as np
 import pytest
 
@@ -251,3 +253,34 @@ def test_saved_problem_loads_into_an_identical_one(hap, make):
     cut[16 + 64 + 0:16 + 64 + 8] = (1 << 40).to_bytes(8, "little")
     with pytest.raises(hap.HapError):
         hap.hap_problem_load(bytes(cut))
+
+
+def test_enumeration_and_trees_reused_across_problems_of_the_process(hap):
+    """Problems on the same cluster with different profiled tables share the cached enumeration and prefix trees;
+    a problem that differs in anything the trees depend on (capacities order, window, compute rates) must not.
+    Every variant is checked against the oracle, in one process, interleaved."""
+    base = problems.small()
+    variants = []
+    faster = base.copy()
+    faster.tdf *= 0.7; faster.tdb *= 0.7; faster.tff *= 0.7; faster.tfb *= 0.7            # new tables, same cluster
+    variants.append(faster)
+    caps = base.copy()
+    caps.cap_eff = np.ascontiguousarray(base.cap_eff[::-1].copy())                         # another type binds the memory
+    variants.append(caps)
+    win = base.copy()
+    win.delta_q = 100                                                                      # narrower window
+    variants.append(win)
+    rates = base.copy()
+    rates.P = np.ascontiguousarray(base.P[::-1].copy())                                    # other window shares
+    variants.append(rates)
+    for pb in [base] + variants + [base, faster]:
+        hp = hap.hap_problem_create(pb)
+        hap.hap_enumerate(hp)
+        o = Oracle(pb)
+        assert (hp.n_pconf, hp.n_cand) == (o.n_pconf, o.n_cand)
+        out = hap.hap_pipeline_dp(hp, 0, hp.n_cand, partition=True)
+        torch.cuda.synchronize()
+        done, costs, bn, parts, levels = o.search_pconfs_plans(0, 1, threads=max(1, len(os.sched_getaffinity(0))))
+        assert np.array_equal(out["cost"].cpu().numpy(), costs)
+        assert np.array_equal(out["partition"].cpu().numpy(), parts) and np.array_equal(out["recompute"].cpu().numpy(), levels)
+        hap.hap_problem_destroy(hp)

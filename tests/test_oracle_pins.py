@@ -1067,3 +1067,18 @@ def test_e8_fp64_mode_hand_values():
     assert f["T_opt"] == pytest.approx(1057185.792, rel=1e-13)
     assert f["T_pipe"] == pytest.approx(49200000.0 + 2.0 * x, rel=1e-13)
     assert f["T_iter"] == pytest.approx(49200000.0 + 2.0 * x + 1333482.24 + 1057185.792, rel=1e-13)
+
+
+def test_bulk_search_with_plans_agrees_with_single_candidate_evaluation():
+    """Plumbing of the bulk search that also returns partitions and levels: same values as eval_index."""
+    o = Oracle(problems.tiny(window=True))
+    done, costs, bn, parts, levels = o.search_pconfs_plans(0, 1, threads=2)
+    assert done == o.n_cand
+    for idx in range(0, o.n_cand, 13):
+        pl, _, _ = o.eval_index(idx)
+        assert costs[idx] == pl["T_iter"] and bn[idx] == pl["bottleneck"]
+        if pl["T_iter"] < INF:
+            assert parts[idx, :pl["PP"]].tolist() == pl["n"] and levels[idx, :pl["PP"]].tolist() == pl["r"]
+            assert not parts[idx, pl["PP"]:].any()
+        else:
+            assert not parts[idx].any() and not levels[idx].any()
