@@ -78,6 +78,8 @@ struct hap_problem {
     size_t n_pslots = 0;                   // slots a search pass writes and reduces (sum of the classes' pslot_n)
     bool timed = false;
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    cudaEvent_t ev_upload = nullptr;       // the last host-to-device upload of this problem (tables, configuration table, trees)
+    bool upload_pending = false;           // that upload has not been waited for yet
     cudaEvent_t ev_fork = nullptr;          // classes run on their own streams between this event and their `done` events
     cudaEvent_t ev_pre = nullptr;           // start of a pass: the candidate decode of the classes waits for this one only
     cudaEvent_t ev_dec = nullptr;           // the merged candidate decode of a pass has finished
@@ -116,6 +118,90 @@ static cudaStream_t pooled_stream(int device, size_t index)
         if (cudaStreamCreateWithPriority(&s, cudaStreamNonBlocking, pr) != cudaSuccess) s = nullptr;
     }
     return s;
+}
+
+// Uploads (profiled tables, configuration table, prefix trees) go through page-locked staging buffers and an
+// upload stream of their own, asynchronously: the host builds the next thing while the copy runs, and the first call
+// that uses the data waits for the upload's event.  The staging buffers are kept per process (a page-locked
+// allocation costs more than a search); a buffer is reused once the copy that last read it has completed.
+namespace {
+struct PinnedBuf { void *ptr = nullptr; size_t cap = 0; cudaEvent_t done = nullptr; int device = -1; };
+struct UploadState {
+    std::mutex mu;
+    std::vector<PinnedBuf> bufs;
+    cudaStream_t stream[64] = {};
+};
+UploadState &upload_state() { static UploadState *u = new UploadState(); return *u; }      // never destroyed
+constexpr size_t kPinnedBufs = 8;
+}  // namespace
+
+static cudaStream_t upload_stream(int device)
+{
+    UploadState &u = upload_state();
+    std::lock_guard<std::mutex> lock(u.mu);
+    cudaStream_t &s = u.stream[device & 63];
+    if (!s && cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) s = nullptr;
+    return s;
+}
+
+// a page-locked buffer of at least `bytes` whose previous copy (if any) has completed; nullptr: use pageable memory
+static PinnedBuf *pinned_get(int device, size_t bytes)
+{
+    UploadState &u = upload_state();
+    std::lock_guard<std::mutex> lock(u.mu);
+    for (auto &b : u.bufs)
+        if (b.device == device && b.cap >= bytes && cudaEventQuery(b.done) == cudaSuccess) return &b;
+    cudaGetLastError();                                  // cudaErrorNotReady of a busy buffer is not an error
+    if (u.bufs.size() >= kPinnedBufs) {                  // reuse the oldest buffer of the device: wait for it, regrow it
+        for (auto &b : u.bufs)
+            if (b.device == device) {
+                cudaEventSynchronize(b.done);
+                if (b.cap >= bytes) return &b;
+                cudaFreeHost(b.ptr); b.ptr = nullptr; b.cap = 0;
+                if (cudaHostAlloc(&b.ptr, bytes, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); b.ptr = nullptr; return nullptr; }
+                b.cap = bytes;
+                return &b;
+            }
+        return nullptr;
+    }
+    u.bufs.reserve(kPinnedBufs);                          // pointers into the vector stay valid
+    PinnedBuf b;
+    b.device = device;
+    b.cap = std::max<size_t>(bytes, 1 << 20);
+    if (cudaHostAlloc(&b.ptr, b.cap, cudaHostAllocDefault) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    if (cudaEventCreateWithFlags(&b.done, cudaEventDisableTiming) != cudaSuccess) { cudaFreeHost(b.ptr); cudaGetLastError(); return nullptr; }
+    u.bufs.push_back(b);
+    return &u.bufs.back();
+}
+
+// host -> device copy of `bytes` that `fill` writes into a staging buffer; asynchronous when a page-locked buffer
+// and the upload stream are available (the problem's upload event then marks its completion), synchronous otherwise
+template <class Fill>
+static cudaError_t upload(hap_problem *p, void *dst, size_t bytes, Fill fill)
+{
+    cudaStream_t us = upload_stream(p->device);
+    PinnedBuf *pb = us ? pinned_get(p->device, bytes) : nullptr;
+    if (!pb) {
+        std::vector<unsigned char> stage(bytes, 0);
+        if (!fill(stage.data())) return cudaErrorInvalidValue;
+        return cudaMemcpy(dst, stage.data(), bytes, cudaMemcpyHostToDevice);
+    }
+    if (!fill(static_cast<unsigned char *>(pb->ptr))) return cudaErrorInvalidValue;
+    cudaError_t e = cudaMemcpyAsync(dst, pb->ptr, bytes, cudaMemcpyHostToDevice, us);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaEventRecord(pb->done, us)) != cudaSuccess) return e;
+    if (!p->ev_upload && (e = cudaEventCreateWithFlags(&p->ev_upload, cudaEventDisableTiming)) != cudaSuccess) return e;
+    if ((e = cudaEventRecord(p->ev_upload, us)) != cudaSuccess) return e;
+    p->upload_pending = true;
+    return cudaSuccess;
+}
+
+// the first use of uploaded data waits for the upload (on the host: by then the copy has long finished)
+static cudaError_t uploads_done(hap_problem *p)
+{
+    if (!p->upload_pending) return cudaSuccess;
+    p->upload_pending = false;
+    return cudaEventSynchronize(p->ev_upload);
 }
 
 // Device memory of destroyed problems is kept for the next problem of the process: allocating and freeing the
@@ -241,6 +327,7 @@ extern "C" const char *hap_last_error(const hap_problem *p) { return p ? p->err.
 static void release_device(hap_problem *p)
 {
     // nothing of this problem may still be running when its memory goes back to the cache
+    if (p->upload_pending) { cudaEventSynchronize(p->ev_upload); p->upload_pending = false; }
     if (p->d_tables || p->d_arena) cudaDeviceSynchronize();
     cached_free(p->d_tables); cached_free(p->d_arena); cached_free(p->d_trie_arena);
     cached_free(p->d_joint_scratch);
@@ -250,6 +337,7 @@ static void release_device(hap_problem *p)
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_pre) cudaEventDestroy(p->ev_pre);
     if (p->ev_dec) cudaEventDestroy(p->ev_dec);
+    if (p->ev_upload) cudaEventDestroy(p->ev_upload);
     for (auto &cl : p->classes) { if (cl.done) cudaEventDestroy(cl.done); }      // the class streams belong to the pool
 }
 
@@ -356,21 +444,33 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     const size_t n4 = (size_t)T * pf->ntp * pf->ncp * pf->nmb, n5 = n4 * N;
     // device layout: the four per-layer tables interleaved entry by entry (one 32-byte record per (type, row, layer):
     // the layer-cost kernel reads a record with two 16-byte loads), then tpre, then tpost
-    std::vector<double> tables(4 * n5 + 2 * n4);
-    for (size_t i = 0; i < n5; ++i) {
-        double *rec = tables.data() + 4 * i;
-        rec[0] = pf->tdf[i]; rec[1] = pf->tdb[i]; rec[2] = pf->tff[i]; rec[3] = pf->tfb[i];
-        if (rec[0] < rec[2] || rec[1] < rec[3]) return HAP_E_INVALID;                // t_dense includes its FFN
-    }
-    std::memcpy(tables.data() + 4 * n5, pf->tpre, n4 * sizeof(double));
-    std::memcpy(tables.data() + 4 * n5 + n4, pf->tpost, n4 * sizeof(double));
-    for (double x : tables) if (!(x >= 0.0) || x > 1e15) return HAP_E_INVALID;   // finite, non-negative, < 2^50 ns
+    const size_t n_tab = 4 * n5 + 2 * n4;
+    auto fill_tables = [&](unsigned char *dst) -> bool {
+        double *tables = reinterpret_cast<double *>(dst);
+        bool ok = true;
+        for (size_t i = 0; i < n5; ++i) {
+            const double a = pf->tdf[i], b = pf->tdb[i], c = pf->tff[i], d = pf->tfb[i];
+            double *rec = tables + 4 * i;
+            rec[0] = a; rec[1] = b; rec[2] = c; rec[3] = d;
+            // t_dense includes its FFN; every entry finite, non-negative, < 2^50 ns (NaN fails every comparison)
+            ok &= (a >= c) & (b >= d) & (c >= 0.0) & (d >= 0.0) & (a <= 1e15) & (b <= 1e15);
+        }
+        for (size_t i = 0; i < n4; ++i) {
+            const double a = pf->tpre[i], b = pf->tpost[i];
+            tables[4 * n5 + i] = a; tables[4 * n5 + n4 + i] = b;
+            ok &= (a >= 0.0) & (b >= 0.0) & (a <= 1e15) & (b <= 1e15);
+        }
+        return ok;
+    };
 
     // ---- device ------------------------------------------------------------------------------
     if (cudaGetDevice(&p->device) != cudaSuccess) return HAP_E_CUDA;
-    if (cached_malloc(p->device, (void **)&p->d_tables, tables.size() * sizeof(double)) != cudaSuccess) return HAP_E_NOMEM;
-    if (cudaMemcpy(p->d_tables, tables.data(), tables.size() * sizeof(double), cudaMemcpyHostToDevice) != cudaSuccess)
-        return HAP_E_CUDA;
+    if (cached_malloc(p->device, (void **)&p->d_tables, n_tab * sizeof(double)) != cudaSuccess) return HAP_E_NOMEM;
+    {
+        const cudaError_t e = upload(p, p->d_tables, n_tab * sizeof(double), fill_tables);
+        if (e == cudaErrorInvalidValue) { cudaGetLastError(); return HAP_E_INVALID; }
+        if (e != cudaSuccess) return HAP_E_CUDA;
+    }
     for (auto &e : p->ev) if (cudaEventCreate(&e) != cudaSuccess) return HAP_E_CUDA;
 
     DevConst &dc = p->dc;
@@ -794,7 +894,7 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
     DecodeJobs dj{};
     unsigned dblk = 0, gblk = 0;
     if (cached_malloc(p->device, (void **)&p->d_trie_arena, total) != cudaSuccess) { p->d_trie_arena = nullptr; cudaGetLastError(); return false; }
-    std::vector<unsigned char> stage(total, 0);
+    auto fill = [&](unsigned char *stage) -> bool {          // (gaps between the pieces are padding that nothing reads)
     size_t off = 0;
     for (auto &bc : built) {
         hap_problem::Trie &tr = bc.cl->trie;
@@ -804,7 +904,7 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
         u32 want = 0;
         for (const auto &pt : h.parts) {
             unsigned char *base = p->d_trie_arena + off;
-            std::memcpy(stage.data() + off, pt.blob.data(), pt.blob.size());
+            std::memcpy(stage + off, pt.blob.data(), pt.blob.size());
             hap_problem::TriePartDev pd{};
             pd.d_nodes = reinterpret_cast<TrieNode *>(base + pt.o_nodes);
             pd.d_leaves = reinterpret_cast<TrieLeaf *>(base + pt.o_leaves);
@@ -832,10 +932,10 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
             off += up(pt.blob.size());
         }
         tr.d_metas = reinterpret_cast<TrieMeta *>(p->d_trie_arena + off);
-        std::memcpy(stage.data() + off, metas.data(), metas.size() * sizeof(TrieMeta));
+        std::memcpy(stage + off, metas.data(), metas.size() * sizeof(TrieMeta));
         off += up(metas.size() * sizeof(TrieMeta));
         tr.d_plist = reinterpret_cast<u32 *>(p->d_trie_arena + off);
-        std::memcpy(stage.data() + off, bc.plist.data(), bc.plist.size() * sizeof(u32));
+        std::memcpy(stage + off, bc.plist.data(), bc.plist.size() * sizeof(u32));
         off += up(bc.plist.size() * sizeof(u32));
         tr.n_conf = (unsigned)bc.plist.size(); tr.smem = smem;
         if (dj.n <= HAP_MAX_PP) {
@@ -852,8 +952,11 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
         tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
         tr.ok = true;
     }
-    std::memcpy(stage.data() + o_jobs, gjobs.data(), gjobs.size() * sizeof(GatherJob));
-    if (cudaMemcpy(p->d_trie_arena, stage.data(), total, cudaMemcpyHostToDevice) != cudaSuccess) {
+    std::memcpy(stage + o_jobs, gjobs.data(), gjobs.size() * sizeof(GatherJob));
+    return true;
+    };
+    if (upload(p, p->d_trie_arena, total, fill) != cudaSuccess) {
+        cudaGetLastError();
         for (auto &bc : built) bc.cl->trie = hap_problem::Trie{};
         return false;
     }
@@ -1122,11 +1225,15 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             p->d_range = reinterpret_cast<u64 *>(base + o_range); p->d_counters = reinterpret_cast<u64 *>(base + o_counters);
             p->d_best = reinterpret_cast<i64 *>(base + o_best); p->d_single = base + o_single;
             // configuration table and work items travel in one copy (they are adjacent up to padding)
-            std::vector<unsigned char> stage(o_c2, 0);
-            std::memcpy(stage.data() + o_pconf, p->pconfs.data(), np * sizeof(hap_pconf));
-            std::memcpy(stage.data() + o_items, p->items.data(), p->items.size() * sizeof(WorkItem));
-            CUDA_TRY(p, cudaMemcpy(base, stage.data(), o_c2, cudaMemcpyHostToDevice));
-            CUDA_TRY(p, cudaMemset(p->d_range, 0, sizeof(u64)));
+            CUDA_TRY(p, upload(p, base, o_c2, [&](unsigned char *stage) {
+                std::memcpy(stage + o_pconf, p->pconfs.data(), np * sizeof(hap_pconf));
+                std::memcpy(stage + o_items, p->items.data(), p->items.size() * sizeof(WorkItem));
+                return true; }));
+            if (p->upload_pending) {
+                cudaStream_t us = upload_stream(p->device);
+                CUDA_TRY(p, cudaMemsetAsync(p->d_range, 0, sizeof(u64), us));
+                CUDA_TRY(p, cudaEventRecord(p->ev_upload, us));
+            } else CUDA_TRY(p, cudaMemset(p->d_range, 0, sizeof(u64)));
         }
         p->dc.pconf = p->d_pconf;
         p->dc.n_pconf = np;
@@ -1163,6 +1270,7 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
                 if (want_trees && !hit->parts.empty()) built.push_back(TrieBuilt{&cl, hit, class_plist(p, cl)});
             }
             if (!missing.empty()) {
+                CUDA_TRY(p, uploads_done(p));                 // the decode below reads the configuration table
                 for (const hap_problem::PpClass *cl : missing) {
                     const WorkItem &rep = p->items[cl->item_lo];
                     const u64 nmap = p->pconfs[rep.p].nmap;
@@ -1223,6 +1331,7 @@ static hap_status enter(hap_problem *p)
     if (!p) return HAP_E_INVALID;
     if (!p->enumerated) return fail(p, HAP_E_STATE, "hap_enumerate has not run");
     if (cudaSetDevice(p->device) != cudaSuccess) return fail(p, HAP_E_CUDA, "cudaSetDevice");
+    if (uploads_done(p) != cudaSuccess) return fail(p, HAP_E_CUDA, "upload of the problem's tables");
     return HAP_OK;
 }
 
@@ -1841,6 +1950,7 @@ extern "C" hap_status hap_problem_save(hap_problem *p, void *host_buf, uint64_t 
     const size_t n4 = (size_t)T * pf.ntp * pf.ncp * pf.nmb, n5 = n4 * N;
     // the tables live on the device only (per-layer ones interleaved entry by entry): read them back in the caller's layout
     std::vector<double> dev(4 * n5 + 2 * n4), tab[4];
+    CUDA_TRY(p, uploads_done(p));
     CUDA_TRY(p, cudaMemcpy(dev.data(), p->d_tables, dev.size() * sizeof(double), cudaMemcpyDeviceToHost));
     for (int t = 0; t < 4; ++t) { tab[t].resize(n5); for (size_t i = 0; i < n5; ++i) tab[t][i] = dev[4 * i + t]; }
     std::vector<double> tpre(dev.begin() + 4 * n5, dev.begin() + 4 * n5 + n4), tpost(dev.begin() + 4 * n5 + n4, dev.end());
