@@ -521,8 +521,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     };
 
     i64 best_cost = kInf;
-    u64 best_index = ~0ull;
-    u64 n_eval = 0, n_feas = 0;
+    u32 best_local = ~0u;               // the best candidate's offset from the block's first candidate
+    u32 n_eval = 0, n_feas = 0;         // (a thread evaluates far fewer than 2^32 candidates)
     u32 n_cells32 = 0;                  // splits this thread evaluated (after the early exits)
     unsigned all_levels = 0;
     for (int q = 0; q < n_rc; ++q) all_levels |= dc.rc_masks[q];
@@ -792,7 +792,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
             if (dc.eta_q > 0 && het * (VT)PP * (VT)1024 > (VT)dc.eta_q * sum) { T_iter = vInf; T_pipe = vInf; }   // Pruning 3
             if (SEARCH) {
                 if (T_iter < vInf) { n_feas++; any_plan = 1; }
-                if ((i64)T_iter < best_cost || ((i64)T_iter == best_cost && c < best_index)) { best_cost = (i64)T_iter; best_index = c; }
+                {   // (offsets grow with the candidate index, so the smaller offset is the smaller index)
+                    const u32 loc = m * (u32)n_rc + (u32)rc_idx;
+                    if ((i64)T_iter < best_cost || ((i64)T_iter == best_cost && loc < best_local)) { best_cost = (i64)T_iter; best_local = loc; }
+                }
             } else {
                 any_plan = 1;
                 if (out.cost) reinterpret_cast<VT *>(out.cost)[o] = T_iter;
@@ -817,12 +820,13 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
         if (lane == 0 && n_cells) atomicAdd(out.counters + 4, n_cells);
     }
     if (SEARCH) {
-        n_eval = (u64)warp_sum_i64((i64)n_eval); n_feas = (u64)warp_sum_i64((i64)n_feas);
+        const u64 n_eval_w = (u64)warp_sum_i64((i64)n_eval), n_feas_w = (u64)warp_sum_i64((i64)n_feas);
+        u64 best_index = best_local == ~0u ? ~0ull : s_clo + (u64)best_local;
         warp_argmin(best_cost, best_index);
         if (lane == 0) {
             wcost[wib] = best_cost; widx[wib] = best_index;
-            if (n_eval) atomicAdd(out.counters + 0, n_eval);
-            if (n_feas) atomicAdd(out.counters + 1, n_feas);
+            if (n_eval_w) atomicAdd(out.counters + 0, n_eval_w);
+            if (n_feas_w) atomicAdd(out.counters + 1, n_feas_w);
         }
         __syncthreads();
         if (tid == 0) {
