@@ -103,6 +103,7 @@ class Problem:
     # ---- extras that are not inputs of the method (kept for inspection)
     extra: Dict[str, np.ndarray] = field(default_factory=dict)
     uniform: int = 0     # ablation: 1 = uniform layer split only (non-uniform partitioning disabled)
+    het_coll: int = 0    # Pruning 3 also counts the dispatch / combine traffic of stages that span device types
     eta_q: int = 0       # Pruning 3 threshold eta in 1/1024 (2048 = the paper's default 2); <= 0 disables it
     # communication-primitive table: link efficiency by message size (empty: efficiency 1 everywhere)
     fsize: np.ndarray = field(default_factory=lambda: np.zeros(0, np.float64))     # [n] bytes, ascending

@@ -369,6 +369,18 @@ int orc_layer_costs(const orc_problem *pr, const orc_pconf *pc, int64_t *c2, dou
             v[ORC_OPT + kd] = pr->copt[h] * ((double)Pdd / (double)((int64_t)TP * DP * CP) + Pel / (double)EDP);
         }
         v[ORC_SLAT] = pr->ovl_dp * (pr->alpha[cG] * (2.0 * (double)(wd - 1) + 2.0 * (double)(EDP - 1)));
+        /* dispatch and combine of one MoE layer, forward and backward (the 2 t_disp per direction of Eq. 2, with
+         * its imbalance factor), when the expert-parallel group spans device types: Eq. 3's volumes over the
+         * cross-type link class at chi times this type's inter-node bandwidth.  Used by Pruning 3 only. */
+        if (EP == 1) v[ORC_KXD] = 0.0;
+        else {
+            double Dmoe = ((thb * pr->beta) * (double)pr->k) * (1.0 - 1.0 / (double)EP);
+            double Dag = (thb * pr->beta) * (double)(EP - 1);
+            double bx = bwi[h] * pr->chi;
+            double fa = pr->alpha[ORC_CROSS] * (double)(EP - 1) + xfer(pr, ORC_CROSS, Dmoe, bx);
+            double fg = pr->alpha[ORC_CROSS] * (double)(EP - 1) + xfer(pr, ORC_CROSS, Dag, bx);
+            v[ORC_KXD] = (4.0 * ((fa <= fg) ? fa : fg)) * imb;
+        }
         for (int q = 0; q < ORC_NCOEF; ++q) {
             if (coeff) coeff[h * ORC_NCOEF + q] = v[q];
             if (coef) coef[h * ORC_NCOEF + q] = llrint(v[q]);
@@ -537,22 +549,40 @@ int64_t orc_stage_cost(const orc_problem *pr, const orc_pconf *pc, const orc_map
 
 
 /* Pruning 3 (heterogeneous communication): the candidate is dropped when its cross-type communication time
- * per micro-batch -- here the stage-to-stage transfers over cross-type links, the only cross-type traffic
- * the model carries -- exceeds eta times the mean stage time, T_hetero > eta * (1/PP) * sum_i c_i.
- * eta is given in 1/1024 (eta_q = 2048 is the paper's default eta = 2); eta_q <= 0 switches the rule off. */
-static int64_t hetero_comm(const orc_pconf *pc, const orc_mapping *mp, const int64_t *coef)
+ * per micro-batch exceeds eta times the mean stage time, T_hetero > eta * (1/PP) * sum_i c_i.
+ * T_hetero is the stage-to-stage transfers over cross-type links; with het_coll set it also holds, for every
+ * stage whose devices are of more than one type (its expert-parallel groups leave a homogeneous sub-cluster,
+ * the case Sec. 3.5 names), the dispatch and combine traffic of the stage's MoE layers re-timed on the
+ * cross-type link: n_moe(stage) times the slowest member type's coefficient ORC_KXD.  The stage times
+ * themselves are not changed by the option.
+ * eta is given in 1/1024 (eta_q = 2048 is the paper's default eta = 2); eta_q <= 0 switches the rule off.
+ * n[s] = layers of stage s of the chosen partition. */
+static int64_t hetero_comm(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp, const int64_t *coef,
+                           const uint8_t *n)
 {
     int64_t t = 0;
     for (int s = 1; s < pc->PP; ++s)
         if (mp->cls[s] == ORC_CROSS) t += coef[mp->hb[s] * ORC_NCOEF + ORC_KP2P_CROSS + mp->ha[s]];
+    if (pr->het_coll) {
+        int a = 0;
+        for (int s = 0; s < pc->PP; ++s) {
+            const unsigned mask = mp->mask[s];
+            if (mask & (mask - 1)) {                       /* more than one device type in the stage */
+                int64_t n_moe = 0;
+                for (int l = a; l < a + n[s]; ++l) n_moe += pr->kind[l] == ORC_MOE;
+                t += n_moe * mask_max(pr, mask, coef, ORC_KXD);
+            }
+            a += n[s];
+        }
+    }
     return t;
 }
 
 static int pruned_by_hetero_comm(const orc_problem *pr, const orc_pconf *pc, const orc_mapping *mp,
-                                 const int64_t *coef, int64_t sum_stage)
+                                 const int64_t *coef, int64_t sum_stage, const uint8_t *n)
 {
     if (pr->eta_q <= 0) return 0;
-    return hetero_comm(pc, mp, coef) * (int64_t)pc->PP * 1024 > (int64_t)pr->eta_q * sum_stage;
+    return hetero_comm(pr, pc, mp, coef, n) * (int64_t)pc->PP * 1024 > (int64_t)pr->eta_q * sum_stage;
 }
 
 /* ------------------------------------------------------------------------------------ *
@@ -617,7 +647,7 @@ int orc_candidate(const orc_problem *pr, const orc_pconf *pc, const orc_mapping 
     res->T_sync = tsync;
     res->T_opt = topt;
     res->T_iter = res->T_pipe + tsync + topt;
-    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum)) res->T_iter = res->T_pipe = ORC_INF;   /* Pruning 3 */
+    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum, res->n)) res->T_iter = res->T_pipe = ORC_INF;   /* Pruning 3 */
     free(DPt); free(CH); free(cx);
 #undef DPAT
 #undef CHAT
@@ -683,7 +713,7 @@ int orc_candidate_refined(const orc_problem *pr, const orc_pconf *pc, const orc_
     res->T_sync = tsync;
     res->T_opt = topt;
     res->T_iter = res->T_pipe + tsync + topt;
-    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum)) res->T_iter = res->T_pipe = ORC_INF;   /* Pruning 3 */
+    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum, res->n)) res->T_iter = res->T_pipe = ORC_INF;   /* Pruning 3 */
     free(D); free(CH); free(cx);
 #undef DAT
 #undef CHAT
@@ -792,7 +822,7 @@ int orc_candidate_exact(const orc_problem *pr, const orc_pconf *pc, const orc_ma
     res->T_sync = tsync;
     res->T_opt = topt;
     res->T_iter = res->T_pipe + tsync + topt;
-    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum)) res->T_iter = res->T_pipe = ORC_INF;
+    if (pruned_by_hetero_comm(pr, pc, mp, coef, sum, res->n)) res->T_iter = res->T_pipe = ORC_INF;
     free(D); free(CH); free(cx);
     return 0;
 }
@@ -1193,6 +1223,18 @@ int orc_candidate_f64(const orc_problem *pr, const orc_pconf *pc, const orc_mapp
         double th = 0.0;
         for (int st = 1; st < PP; ++st)
             if (mp->cls[st] == ORC_CROSS) th += coeff[mp->hb[st] * ORC_NCOEF + ORC_KP2P_CROSS + mp->ha[st]];
+        if (pr->het_coll) {                                /* mixed-type stages: dispatch and combine on the cross-type link */
+            int a = 0;
+            for (int st = 0; st < PP; ++st) {
+                const unsigned mask = mp->mask[st];
+                if (mask & (mask - 1)) {
+                    int n_moe = 0;
+                    for (int l = a; l < a + res->n[st]; ++l) n_moe += pr->kind[l] == ORC_MOE;
+                    th += (double)n_moe * mask_max_f(pr, mask, coeff, ORC_KXD);
+                }
+                a += res->n[st];
+            }
+        }
         if (th * (double)PP * 1024.0 > (double)pr->eta_q * sum) res->T_iter = res->T_pipe = INFINITY;
     }
     free(DPt); free(CH); free(cx);

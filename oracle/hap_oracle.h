@@ -32,7 +32,8 @@ enum {
     ORC_KP2P_CROSS = 4, /* +h' for the sending type, 4 entries */
     ORC_SLAT = 8, ORC_SBW = 9, /* +kind */ ORC_OPT = 11, /* +kind */
     ORC_MW = 13, /* +kind */ ORC_MA = 15, /* +kind */ ORC_MX = 17, ORC_MPRE = 18, ORC_MPOST = 19,
-    ORC_NCOEF = 20
+    ORC_KXD = 20, /* dispatch + combine of an MoE layer over the cross-type link (Pruning 3 with het_coll) */
+    ORC_NCOEF = 21
 };
 
 typedef struct {
@@ -73,7 +74,8 @@ typedef struct {
     int32_t eta_q;      /* Pruning 3 threshold eta in 1/1024; <= 0: off */
     int32_t uniform;    /* ablation: uniform layer split only (floor/ceil of N/PP layers per stage) */
     /* communication-primitive table: link efficiency by message size (0 sizes: efficiency 1 everywhere) */
-    int32_t n_fsize, pad_f;
+    int32_t n_fsize;
+    int32_t het_coll;   /* Pruning 3 also counts the dispatch / combine traffic of stages that span device types */
     const double *fsize;    /* [n_fsize] bytes, ascending */
     const double *feff;     /* [3][n_fsize] efficiency in (0, 1] of an intra-node / inter-node / cross-type link */
 } orc_problem;

@@ -17,10 +17,10 @@ _DIR = os.path.dirname(os.path.abspath(__file__))
 _SO = os.path.join(_DIR, "libhap_oracle.so")
 _SRC = [os.path.join(_DIR, "hap_oracle.c"), os.path.join(_DIR, "hap_oracle.h")]
 
-MAX_TYPES, MAX_PP, MAX_N, NCOEF = 4, 32, 255, 20
+MAX_TYPES, MAX_PP, MAX_N, NCOEF = 4, 32, 255, 21
 INF = 1 << 62
 COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, SBW=9, OPT=11,
-            MW=13, MA=15, MX=17, MPRE=18, MPOST=19)
+            MW=13, MA=15, MX=17, MPRE=18, MPOST=19, KXD=20)
 
 
 def build_oracle(force: bool = False) -> str:
@@ -51,7 +51,7 @@ class _Problem(C.Structure):
         ("npp", C.c_int32), ("ntpe", C.c_int32), ("pp_list", C.c_void_p), ("tpe_list", C.c_void_p),
         ("tp_max", C.c_int32), ("delta_q", C.c_int32), ("map_cap", C.c_uint64),
         ("n_rc", C.c_int32), ("rc_masks", C.c_void_p), ("eta_q", C.c_int32), ("uniform", C.c_int32),
-        ("n_fsize", C.c_int32), ("pad_f", C.c_int32), ("fsize", C.c_void_p), ("feff", C.c_void_p),
+        ("n_fsize", C.c_int32), ("het_coll", C.c_int32), ("fsize", C.c_void_p), ("feff", C.c_void_p),
     ]
 
 
@@ -165,6 +165,7 @@ class Oracle:
         s.rc_masks = arr("rc_masks", np.uint32)
         s.eta_q = int(getattr(pb, "eta_q", 0))
         s.uniform = int(getattr(pb, "uniform", 0))
+        s.het_coll = int(getattr(pb, "het_coll", 0))
         fsize = np.ascontiguousarray(np.asarray(getattr(pb, "fsize", []), dtype=np.float64))
         feff = np.ascontiguousarray(np.asarray(getattr(pb, "feff", []), dtype=np.float64))
         keep["fsize"], keep["feff"] = fsize, feff

@@ -42,3 +42,21 @@ def e9_problem():
     pb.delta_q = 205
     assert pb.cap_eff.tolist() == [100 << 30, 2 << 30]
     return pb
+
+
+def e10_problem():
+    pb = problems.blank(N=4, S=1024, H=1024, E=4, k=2, GB=16, P_tf=[300, 100], C_gb=[100000, 100000], node_size=[6, 2],
+                        nodes_per_type=[1, 1], pp_list=(2,), ep_list=(2,), kind=[DENSE, MOE, MOE, MOE], F_exp=1024)
+    for h, (d, m) in enumerate(((300000.0, 400000.0), (380000.0, 500000.0))):
+        row = np.array([d, m, m, m])
+        pb.tdf[h, 0, 0, 0] = row
+        pb.tdb[h, 0, 0, 0] = 2 * row
+        pb.tff[h, 0, 0, 0] = row / 2
+        pb.tfb[h, 0, 0, 0] = row
+    pb.alpha[:] = [2000.0, 8000.0, 12000.0]
+    pb.bw_intra[:] = [400.0, 200.0]
+    pb.node_bw_inter[:] = [25.0, 50.0]
+    pb.chi, pb.gamma, pb.ovl_dp = 0.7, 0.5, 0.0
+    pb.rho[:] = 1.5
+    pb.het_coll = 1
+    return pb

@@ -11,7 +11,7 @@ import pytest
 from gen import problems
 from gen.problems import DENSE, MOE
 from oracle import Oracle, INF, COEF, NCOEF, Mapping
-from hand_examples import e8_problem, e9_problem
+from hand_examples import e8_problem, e9_problem, e10_problem
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 
@@ -1031,6 +1031,43 @@ def test_e9_stage_spanning_two_device_types():
     assert o.stage_cost(0, mp, 0b01, c2, coef, 2, 7, 8) == (1314486, 0)
     costs, _, best, _ = o.search()
     assert costs.tolist() == [g["AB"]["T_iter"], g["BA"]["T_iter"]] and best["index"] == g["best_index"]
+
+
+def test_e10_dispatch_of_mixed_type_stages_in_the_heterogeneous_communication_rule():
+    """Pruning 3 with the dispatch / combine traffic of stages that span device types: the coefficient, which
+    stages and layers count, and the decisions around the hand-computed thresholds."""
+    g = gold("e10_hetero_dispatch.json")["expect"]
+    o = Oracle(e10_problem())
+    assert (o.n_pconf, o.n_cand) == (1, 2)
+    assert [int(o.pconfs[k][0]) for k in ("EP", "EDP", "M", "G")] == [2, 2, 4, 4]
+    c2, c2f, coef, coeff = o.layer_costs(0)
+    assert coef[:, COEF["KXD"]].tolist() == g["kxd"]
+    assert coeff[:, COEF["KXD"]].tolist() == pytest.approx(g["kxd_f64"], rel=1e-14)
+    assert c2.sum(axis=2).tolist() == [g["layer_sum"]["A"], g["layer_sum"]["B"]]
+    for name in ("AB", "BA"):
+        mp = o.decode(0, g[name]["map_idx"])
+        assert [int(x) for x in mp.mask[:2]] == g["masks"][name] and int(mp.cls[1]) == 0
+    for eta_q, want in g["pruned"].items():
+        for variant in ("plain", "refined", "exact", "f64"):
+            pb = e10_problem()
+            pb.eta_q = int(eta_q)
+            ov = Oracle(pb)
+            for name, dropped in zip(("AB", "BA"), want):
+                idx = g[name]["map_idx"]
+                got = {"plain": lambda: ov.eval_index(idx)[0], "refined": lambda: ov.eval_index_refined(idx),
+                       "exact": lambda: ov.eval_index_exact(idx), "f64": lambda: ov.eval_index_f64(idx)}[variant]()
+                assert got["n"] == g[name]["n"], (eta_q, variant, name)
+                if variant == "f64":
+                    assert (got["T_iter"] == float("inf")) == dropped, (eta_q, variant, name)
+                else:
+                    assert got["bottleneck"] == g[name]["bottleneck"]
+                    assert got["T_iter"] == (INF if dropped else g[name]["T_iter"]), (eta_q, variant, name)
+    # the narrow reading sees no cross-type traffic here: nothing is dropped, whatever eta
+    for eta_q, want in g["pruned_without_option"].items():
+        pb = e10_problem()
+        pb.eta_q, pb.het_coll = int(eta_q), 0
+        costs, _, best, feas = Oracle(pb).search()
+        assert costs.tolist() == [g["AB"]["T_iter"], g["BA"]["T_iter"]] and feas == 2 and best["index"] == 1
 
 
 @pytest.mark.parametrize("make, gname, names", [(e8_problem, "e8_sync_opt_assembly.json", ("ABC", "BAC")),
