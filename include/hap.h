@@ -69,7 +69,11 @@ enum {
     HAP_MX = 17,         /* M_moe-extra of a stage that holds at least one MoE layer, bytes */
     HAP_MPRE = 18,       /* embedding weights on the first stage, bytes */
     HAP_MPOST = 19,      /* LM head weights on the last stage, bytes */
-    HAP_NCOEF = 20
+    HAP_KXD = 20,        /* dispatch + combine of one MoE layer, forward and backward, when the expert-parallel group spans
+                            device types: Eq. 3's volumes over the cross-type link class at chi x the type's inter-node
+                            bandwidth, with the imbalance factor of Eq. 2, ns; read by Pruning 3 under
+                            HAP_OPT_HETERO_DISPATCH only */
+    HAP_NCOEF = 21
 };
 
 /* Model and training hyper-parameters (Sec. 3.2 "Input": N, S, H, E, k, batch sizes). */
@@ -144,6 +148,11 @@ typedef struct {
                                  separate launch (identical results) */
 #define HAP_OPT_COUNT_SPLITS 64 /* instrumentation: hap_pipeline_dp passes of this problem also count the splits (k, j) their kernels
                                  evaluate, after all early exits, for hap_get_timings; costs a few percent of the pass */
+#define HAP_OPT_HETERO_DISPATCH 128 /* Pruning 3 (Sec. 3.5 (3)) also counts, for every stage whose devices are of more than one
+                                  type (its expert-parallel groups leave a homogeneous sub-cluster), the dispatch and combine
+                                  traffic of the stage's MoE layers on the cross-type link: the number of MoE layers of the
+                                  stage x the largest HAP_KXD among the stage's types is added to the cross-type transfer
+                                  time the rule compares with eta x the mean stage time.  Stage times are not changed. */
 #define HAP_OPT_UNIFORM 8     /* ablation "non-uniform partitioning disabled" (Sec. 5.5): every stage takes floor(N/PP) or
                                  ceil(N/PP) layers; the load-balance window is ignored */
 #define HAP_OPT_EXACT 4       /* like HAP_OPT_REFINE, but the limit on the stage cost is then swept upward from the bottleneck over

@@ -9,4 +9,5 @@ from .binding import (HapError, HapProblem, hap_problem_create, hap_enumerate, h
                       hap_eval_layer_costs, hap_eval_layer_costs_f64, hap_pipeline_dp, hap_pipeline_dp_f64, hap_search_best,
                       hap_search_range_f64,
                       hap_search_range, hap_argmin, hap_argmin_static, hap_joint_bottleneck, hap_count_cells, hap_get_timings, hap_launches_per_pass, hap_eval_appendix_b, hap_simulate_1f1b, hap_release_cached_memory, hap_self_check, hap_problem_save, hap_problem_load, hap_problem_dims, hap_problem_destroy, load_library, EXPORTS, INF, COEF,
-                      NCOEF, MAX_PP, OPT_NO_MAPTAB, OPT_REFINE, OPT_EXACT, OPT_UNIFORM, OPT_NO_TRIE, OPT_NO_FUSE, OPT_COUNT_SPLITS)
+                      NCOEF, MAX_PP, OPT_NO_MAPTAB, OPT_REFINE, OPT_EXACT, OPT_UNIFORM, OPT_NO_TRIE, OPT_NO_FUSE, OPT_COUNT_SPLITS,
+                      OPT_HETERO_DISPATCH)

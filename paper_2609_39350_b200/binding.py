@@ -9,10 +9,10 @@ import numpy as np
 
 from .build import LIB, LIB_CHECKED
 
-MAX_TYPES, MAX_PP, MAX_LAYERS, NCOEF = 4, 32, 255, 20
+MAX_TYPES, MAX_PP, MAX_LAYERS, NCOEF = 4, 32, 255, 21
 INF = 1 << 62
 COEF = dict(KPRE=0, KPOST=1, KP2P_INTRA=2, KP2P_INTER=3, KP2P_CROSS=4, SLAT=8, SBW=9, OPT=11,
-            MW=13, MA=15, MX=17, MPRE=18, MPOST=19)
+            MW=13, MA=15, MX=17, MPRE=18, MPOST=19, KXD=20)
 STATUS = ["HAP_OK", "HAP_E_INVALID", "HAP_E_NOMEM", "HAP_E_CUDA", "HAP_E_RANGE", "HAP_E_STATE", "HAP_E_INFEASIBLE"]
 EXPORTS = ["hap_problem_create", "hap_problem_destroy", "hap_enumerate", "hap_get_pconfs", "hap_decode",
            "hap_eval_layer_costs", "hap_eval_layer_costs_f64", "hap_pipeline_dp", "hap_pipeline_dp_f64",
@@ -148,6 +148,7 @@ OPT_NO_MAPTAB = 1
 OPT_REFINE = 2
 OPT_EXACT = 4
 OPT_UNIFORM = 8
+OPT_HETERO_DISPATCH = 128
 OPT_NO_TRIE = 16
 OPT_NO_FUSE = 32
 OPT_COUNT_SPLITS = 64
@@ -196,7 +197,8 @@ def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     so.n_rc = len(pb.rc_masks)
     so.rc_masks = arr("rc_masks", np.uint32)
     so.prune = int(prune)
-    so.flags = int(flags) | (OPT_UNIFORM if int(getattr(pb, "uniform", 0)) else 0)
+    so.flags = (int(flags) | (OPT_UNIFORM if int(getattr(pb, "uniform", 0)) else 0)
+                | (OPT_HETERO_DISPATCH if int(getattr(pb, "het_coll", 0)) else 0))
     so.eta_q = int(getattr(pb, "eta_q", 0))
     out = C.c_void_p(0)
     st = L.hap_problem_create(C.byref(mo), C.byref(cl), C.byref(pf), C.byref(so), C.byref(out))

@@ -478,6 +478,7 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     dc.N = N; dc.T = T; dc.R = pf->R; dc.n_rc = so->n_rc; dc.ntp = pf->ntp; dc.ncp = pf->ncp; dc.nmb = pf->nmb; dc.nep = pf->nep;
     dc.S = mo->S; dc.H = mo->H; dc.E = mo->E; dc.k = mo->k; dc.n_shared = mo->n_shared; dc.F_dense = mo->F_dense;
     dc.F_exp = mo->F_exp; dc.nq = mo->nq; dc.nkv = mo->nkv; dc.V = mo->V; dc.GB = mo->GB; dc.delta_q = so->delta_q; dc.eta_q = so->eta_q; dc.uniform = (so->flags & HAP_OPT_UNIFORM) != 0;
+    dc.het_dispatch = (so->flags & HAP_OPT_HETERO_DISPATCH) != 0;
     dc.beta = mo->beta; dc.kappa = pf->kappa; dc.chi = pf->chi; dc.gamma = pf->gamma; dc.ovl_tp = pf->ovl_tp;
     dc.ovl_cp = pf->ovl_cp; dc.ovl_dp = pf->ovl_dp; dc.capf = pf->capf;
     for (int i = 0; i < 3; ++i) dc.alpha[i] = p->alpha[i];

@@ -1,7 +1,7 @@
 // Device-side data layout and kernels of libhap (sm_100a).
 //
 // Kernels
-//   type_const_kernel   per (configuration, type): constants of Eq. 2 / Eq. 3 and the 20 stage
+//   type_const_kernel   per (configuration, type): constants of Eq. 2 / Eq. 3 and the 21 stage
 //                       coefficients, fp64 with one IEEE operation per operator (the translation
 //                       unit is compiled with --fmad=false), three independent roles per pair.
 //   layer_cost_kernel   per (configuration, type, layer): Eq. 2 with imbalance scaling, rounding,
@@ -58,6 +58,7 @@ struct DevConst {
     int N, T, R, n_rc, ntp, ncp, nmb, nep;
     int S, H, E, k, n_shared, F_dense, F_exp, nq, nkv, V, GB;
     int delta_q, tau_linear, eta_q, uniform;
+    int het_dispatch;                 // Pruning 3 also counts the dispatch / combine traffic of stages that span device types
     int kind_uniform;                 // every layer is of one kind (all MoE or all dense): a span's memory depends on its length only
     int kind_uniform_from;            // first layer u such that layers u..N-1 are all of one kind (0 when kind_uniform)
     double beta, kappa, chi, gamma, ovl_tp, ovl_cp, ovl_dp, capf;
@@ -260,7 +261,7 @@ __device__ __forceinline__ double div_by(double a, double b, double y)
 }
 
 // Phase 1 (type_const_kernel): per (configuration, type) the constants of Eq. 2 / Eq. 3 (into a scratch array)
-// and the 20 stage coefficients.  The work of one (configuration, type) is a chain of about 40 fp64 divisions,
+// and the 21 stage coefficients.  The work of one (configuration, type) is a chain of about 40 fp64 divisions,
 // so it is cut into three independent roles (blockIdx.y: layer constants; p2p / activation / extra-memory
 // coefficients; weight / sync / optimizer coefficients), one thread per (configuration, type) and role.
 // Phase 2 (layer_cost_kernel): one block per configuration, one thread per layer.
@@ -270,7 +271,7 @@ __device__ __forceinline__ bool put_coef(i64 *coef, double *coeff, size_t at, in
     if (QUANT) coef[at + q] = __double2ll_rn(v);
     else coeff[at + q] = v;
     // time coefficients must stay below 2^40 ns (per-layer ones below 2^36), bytes below 2^50
-    const double lim = q <= HAP_SLAT ? 1.0995e12 : (q < HAP_MW ? 6.8719e10 : 1.1259e15);
+    const double lim = (q <= HAP_SLAT || q == HAP_KXD) ? 1.0995e12 : (q < HAP_MW ? 6.8719e10 : 1.1259e15);
     return !(v < lim);
 }
 
@@ -352,6 +353,18 @@ type_const_kernel(const DevConst dc, TypeConst *tcg, i64 *coef, double *coeff, u
         const double mpre = (((double)dc.V * (double)H) / (double)TP) * shd;
         bad |= put_coef<QUANT>(coef, coeff, at, HAP_MPRE, mpre);
         bad |= put_coef<QUANT>(coef, coeff, at, HAP_MPOST, mpre);
+        // dispatch + combine of one MoE layer (forward and backward, with the imbalance factor of Eq. 2) when the
+        // expert-parallel group spans device types: Eq. 3's volumes over the cross-type link
+        double kxd = 0.0;
+        if (EP != 1) {
+            const double Dmoe = ((thb * dc.beta) * (double)dc.k) * (1.0 - 1.0 / (double)EP);
+            const double Dag = (thb * dc.beta) * (double)(EP - 1);
+            const double bx = dc.bw_inter[h] * dc.chi;
+            const double fa = dc.alpha[HAP_CROSS] * (double)(EP - 1) + xfer_ns(dc, HAP_CROSS, Dmoe, bx);
+            const double fg = dc.alpha[HAP_CROSS] * (double)(EP - 1) + xfer_ns(dc, HAP_CROSS, Dag, bx);
+            kxd = (4.0 * ((fa <= fg) ? fa : fg)) * (1.0 + dc.gamma * (dc.rho[pc.iep] - 1.0));
+        }
+        bad |= put_coef<QUANT>(coef, coeff, at, HAP_KXD, kxd);
     } else {
         const i64 wd = (i64)DP * CP;
         const double shd = 6.0 + 12.0 / (double)wd;
@@ -919,6 +932,7 @@ __device__ __forceinline__ double tau_term(i64 tau, double F) { return ((double)
 template <typename VT>
 struct MaskInfo {
     VT kpre, kpost, slat, sbw[2], opt[2];
+    VT kxd;             // what an MoE layer of a stage with these types adds to the cross-type time of Pruning 3 (0: one type, or option off)
     i64 Pmin;
     int capt, pad;
 };
@@ -996,12 +1010,14 @@ __device__ __forceinline__ void dp_prologue_rows(
     if (threadIdx.x < nmask) {
         const int mk = threadIdx.x + 1;
         MaskInfo<VT> mi;
-        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
+        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.kxd = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
         i64 cap = 0;
         bool seen = false;
+        const bool het_stage = dc.het_dispatch && (mk & (mk - 1)) != 0;      // more than one device type
         for (int h = 0; h < T; ++h)
             if (mk >> h & 1) {
                 const VT *row = cvp + h * HAP_NCOEF;
+                if (het_stage && row[HAP_KXD] > mi.kxd) mi.kxd = row[HAP_KXD];
                 if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; mi.capt = h; }
                 if (!seen || dc.P[h] < mi.Pmin) mi.Pmin = dc.P[h];
                 if (!seen || row[HAP_KPRE] > mi.kpre) mi.kpre = row[HAP_KPRE];
@@ -1592,6 +1608,8 @@ pipeline_dp_kernel(const DevConst dc, const WorkItem *items, const VT *c2, const
             }
             VT het_me = 0;                                  // cross-type transfer into this lane's stage (Pruning 3)
             if (dc.eta_q > 0 && lane > 0 && lane < PP && (link & 3) == HAP_CROSS) het_me = sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
+            // ... and, when asked for, the dispatch / combine traffic of the MoE layers of a stage that spans device types
+            if (dc.eta_q > 0 && lane < PP) het_me += (VT)((int)sK[b_me] - (int)sK[a_me]) * minfo[mask - 1].kxd;
             VT sum = c_me, mxc = c_me;
             for (int o = red0; o > 0; o >>= 1) {          // lanes >= PP hold zeros
                 const VT t1 = __shfl_xor_sync(0xffffffffu, sum, o), t2 = __shfl_xor_sync(0xffffffffu, mxc, o);

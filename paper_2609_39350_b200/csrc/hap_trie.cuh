@@ -247,12 +247,14 @@ __device__ __forceinline__ void trie_prologue_rows(
     if (tid < nmask) {
         const int mk = tid + 1;
         MaskInfo<VT> mi;
-        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
+        mi.kpre = mi.kpost = mi.slat = mi.sbw[0] = mi.sbw[1] = mi.opt[0] = mi.opt[1] = 0; mi.kxd = 0; mi.Pmin = 0; mi.capt = 0; mi.pad = 0;
         i64 cap = 0;
         bool seen = false;
+        const bool het_stage = dc.het_dispatch && (mk & (mk - 1)) != 0;      // more than one device type
         for (int h = 0; h < T; ++h)
             if (mk >> h & 1) {
                 const VT *row = cvp + h * HAP_NCOEF;
+                if (het_stage && row[HAP_KXD] > mi.kxd) mi.kxd = row[HAP_KXD];
                 if (!seen || dc.cap_eff[h] < cap) { cap = dc.cap_eff[h]; mi.capt = h; }
                 if (!seen || dc.P[h] < mi.Pmin) mi.Pmin = dc.P[h];
                 if (!seen || row[HAP_KPRE] > mi.kpre) mi.kpre = row[HAP_KPRE];
@@ -770,7 +772,10 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
                     op = n_dense * mi.opt[0] + n_moe * mi.opt[1];
                 }
                 t_sync = sy > t_sync ? sy : t_sync; t_opt = op > t_opt ? op : t_opt;
-                if (dc.eta_q > 0 && d > 1 && (link & 3) == HAP_CROSS) het += sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
+                if (dc.eta_q > 0) {                                  // Pruning 3: cross-type transfer into the stage; dispatch of a mixed-type stage
+                    if (d > 1 && (link & 3) == HAP_CROSS) het += sP2P[(link >> 4) & 3][2 + ((link >> 2) & 3)];
+                    het += (VT)((int)sK[b] - (int)sK[a]) * mi.kxd;
+                }
                 if (!SEARCH) {
                     if (out.partition) out.partition[o * HAP_MAX_PP + d - 1] = (uint8_t)(b - a);
                     if (out.recompute) out.recompute[o * HAP_MAX_PP + d - 1] = (uint8_t)r;

@@ -136,6 +136,42 @@ def test_value_limits_are_reported(hap):
     assert e.value.name == "HAP_E_RANGE"
 
 
+# flags: default, one warp per candidate, refinement, exact sweep (the refinement modes on one threshold per workload)
+@pytest.mark.parametrize("name,eta_q,flags", [(n, e, f) for n, e in (("tiny", 2048), ("tiny", 128), ("small", 2048), ("small", 24), ("mixtral", 512))
+                                              for f in (0, 16, 2, 4) if f < 2 or n == "tiny" or e == 2048])
+def test_heterogeneous_communication_pruning_with_dispatch_of_mixed_stages(hap, name, eta_q, flags):
+    """The wider reading of Pruning 3: the dispatch and combine traffic of stages that span device types counts as
+    cross-type communication, so candidates are dropped that the narrow reading keeps (already at the paper's eta = 2)."""
+    pb = problems.make_problem(name)
+    pb.eta_q = eta_q
+    o_narrow = Oracle(pb)
+    narrow = {0: o_narrow.search_pconfs, 16: o_narrow.search_pconfs, 2: o_narrow.search_pconfs_refined,
+              4: o_narrow.search_pconfs_exact}[flags](0, 1, threads=8, want_costs=True)[3]
+    pb.het_coll = 1
+    o = Oracle(pb)
+    search = {0: o.search_pconfs, 16: o.search_pconfs, 2: o.search_pconfs_refined, 4: o.search_pconfs_exact}[flags]
+    done, bc, bi, costs, bn = search(0, 1, threads=8, want_costs=True)
+    assert ((costs >= INF) & (narrow < INF)).sum() > 0 and not ((costs < INF) & (narrow >= INF)).any()
+    hp = hap.hap_problem_create(pb, flags=flags)
+    hap.hap_enumerate(hp)
+    out = hap.hap_pipeline_dp(hp, 0, hp.n_cand)
+    torch.cuda.synchronize()
+    assert np.array_equal(out["cost"].cpu().numpy(), costs) and np.array_equal(out["bottleneck"].cpu().numpy(), bn)
+    for prune in (0, 1):
+        hq = hap.hap_problem_create(pb, flags=flags, prune=prune)
+        hap.hap_enumerate(hq)
+        plan, stats = hap.hap_search_best(hq)
+        assert (plan["T_iter"], plan["index"]) == (bc, bi)
+        hap.hap_problem_destroy(hq)
+    if flags == 0:
+        got = hap.hap_pipeline_dp_f64(hp, 0, hp.n_cand)["cost"].cpu().numpy()
+        cf = o.search_pconfs_f64(0, 1, threads=8)[1]
+        assert (np.isfinite(got) == np.isfinite(cf)).mean() > 0.9999       # a candidate exactly at the threshold may fall either way
+        fin = np.isfinite(got) & np.isfinite(cf)
+        assert np.max(np.abs(got[fin] - cf[fin]) / cf[fin]) <= 1e-9
+    hap.hap_problem_destroy(hp)
+
+
 @pytest.mark.parametrize("name,eta_q", [("tiny", 64), ("tiny", 16), ("small", 2048), ("small", 24), ("mixtral", 12)])
 def test_heterogeneous_communication_pruning(hap, name, eta_q):
     """Pruning 3: candidates whose cross-type transfer time exceeds eta x the mean stage time cost +INF."""

@@ -3,7 +3,8 @@ by hand there (not with the oracle), so a mistake that the oracle and the kernel
 
 e8: Eq. 4's gradient-synchronisation and optimizer terms, each decided by a different stage than the bottleneck.
 e9: a stage whose device group spans two device types (per-layer slowest member, smallest member's memory,
-    slowest member's share in the load-balance window)."""
+    slowest member's share in the load-balance window).
+e10: Pruning 3 with the dispatch / combine traffic of stages that span device types."""
 import json
 import os
 
@@ -13,7 +14,7 @@ import pytest
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
-from hand_examples import e8_problem, e9_problem  # noqa: E402
+from hand_examples import e8_problem, e9_problem, e10_problem  # noqa: E402
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
 INF = 1 << 62
@@ -110,4 +111,44 @@ def test_fp64_mode_tracks_the_hand_values(hap, make, gname, names):
         PP = len(want["n"])
         assert abs(cost[want["map_idx"]] - want["T_iter"]) <= PP + 8        # unrounded coefficients: < 1 ns per term
         assert part[want["map_idx"], :PP].tolist() == want["n"]
+    hap.hap_problem_destroy(hp)
+
+
+@pytest.mark.parametrize("flags", [0, 16, 2, 4, 1])     # default, no prefix tree, refinement, exact sweep, no mapping table
+def test_hand_values_of_the_wider_heterogeneous_communication_rule(hap, flags):
+    g = gold("e10_hetero_dispatch.json")
+    cases = [(k, v, 1) for k, v in g["pruned"].items()] + [(k, v, 0) for k, v in g["pruned_without_option"].items()]
+    for eta_q, want, option in cases:
+        pb = e10_problem()
+        pb.eta_q, pb.het_coll = int(eta_q), option
+        hp = hap.hap_problem_create(pb, flags=flags)
+        n_pconf, n_cand = hap.hap_enumerate(hp)
+        assert (n_pconf, n_cand) == (1, 2)
+        out = hap.hap_pipeline_dp(hp, 0, n_cand, partition=True)
+        torch.cuda.synchronize()
+        cost, bott = out["cost"].cpu().numpy(), out["bottleneck"].cpu().numpy()
+        for name, dropped in zip(("AB", "BA"), want):
+            i = g[name]["map_idx"]
+            assert int(bott[i]) == g[name]["bottleneck"]
+            assert int(cost[i]) == (INF if dropped else g[name]["T_iter"]), (eta_q, name, int(cost[i]))
+        if not all(want):
+            plan, stats = hap.hap_search_best(hp)
+            assert plan["index"] == (1 if not want[1] else 0) and stats["n_feasible"] == want.count(False)
+        if flags == 0:
+            fo = hap.hap_pipeline_dp_f64(hp, 0, n_cand)
+            torch.cuda.synchronize()
+            assert [not np.isfinite(x) for x in fo["cost"].cpu().numpy()] == want
+        hap.hap_problem_destroy(hp)
+
+
+def test_hand_values_of_the_cross_type_dispatch_coefficient(hap):
+    g = gold("e10_hetero_dispatch.json")
+    hp = hap.hap_problem_create(e10_problem())
+    hap.hap_enumerate(hp)
+    c2, coef = hap.hap_eval_layer_costs(hp)
+    c2f, coeff = hap.hap_eval_layer_costs_f64(hp)
+    torch.cuda.synchronize()
+    assert coef.cpu().numpy()[0, :, hap.COEF["KXD"]].tolist() == g["kxd"]
+    assert np.allclose(coeff.cpu().numpy()[0, :, hap.COEF["KXD"]], g["kxd_f64"], rtol=1e-14, atol=0)
+    assert c2.cpu().numpy()[0].sum(axis=2).tolist() == [g["layer_sum"]["A"], g["layer_sum"]["B"]]
     hap.hap_problem_destroy(hp)
