@@ -67,6 +67,7 @@ struct hap_problem {
     int joint_grid = 0;
     bool joint_ready = false;
     i64 *d_lb = nullptr;                    // scratch: per-configuration lower bound on the summed stage time
+    PlanSlot *d_plans = nullptr;            // per partial-minimum slot the plan of the block's best candidate (searches over the prefix trees; first use)
     i64 *d_cand_lb = nullptr;               // scratch of the refinement searches: per-candidate bottleneck, then lower bound (first use)
     TypeConst *d_tc = nullptr;              // scratch: per (configuration, type) constants of the layer-cost kernels
     i64 *d_pcost = nullptr;                // per-block partial minima
@@ -332,7 +333,7 @@ static void release_device(hap_problem *p)
     cached_free(p->d_tables); cached_free(p->d_arena); cached_free(p->d_trie_arena);
     cached_free(p->d_joint_scratch);
     for (auto &j : p->joint) { cached_free(j.d_ids); cached_free(j.d_arrays); }
-    cached_free(p->d_c2f); cached_free(p->d_coeff); cached_free(p->d_fcost); cached_free(p->d_cand_lb);
+    cached_free(p->d_c2f); cached_free(p->d_coeff); cached_free(p->d_fcost); cached_free(p->d_cand_lb); cached_free(p->d_plans);
     for (auto &e : p->ev) if (e) cudaEventDestroy(e);
     if (p->ev_fork) cudaEventDestroy(p->ev_fork);
     if (p->ev_pre) cudaEventDestroy(p->ev_pre);
@@ -1569,7 +1570,7 @@ static hap_status launch_dp(hap_problem *p, const DpOut &out, bool search, cudaS
         const uint8_t *tab = cl.has_tab ? p->d_maptab + cl.map_base : nullptr;
         DpOut o = out;
         o.exact = (p->opts.flags & HAP_OPT_EXACT) != 0 && !out.force_plain;
-        if (search) { o.partial_cost += cl.pslot_lo; o.partial_index += cl.pslot_lo; }
+        if (search) { o.partial_cost += cl.pslot_lo; o.partial_index += cl.pslot_lo; if (o.block_plan) o.block_plan += cl.pslot_lo; }
         if (pass_uses_trie(p, cl, out, f64)) {
             const hap_problem::Trie &tr = cl.trie;
             // 64 registers per thread in both shapes (measured: more warps per SM beat more registers per thread)
@@ -2098,7 +2099,8 @@ static hap_status argmin_launch(hap_problem *p, const i64 *dev_cost, uint64_t co
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     const i64 *pc = p->d_pcost; const u64 *pi = p->d_pindex; const u64 nb = blocks;
-    CUDA_TRY(p, cudaLaunchKernelEx(&cfg, argmin_final_kernel, pc, pi, nb, dev_out, init));
+    const PlanSlot *no_plans = nullptr; i64 *no_vals = nullptr; uint8_t *no_bytes = nullptr;
+    CUDA_TRY(p, cudaLaunchKernelEx(&cfg, argmin_final_kernel, pc, pi, nb, dev_out, init, no_plans, no_vals, no_bytes, no_bytes));
     return HAP_OK;
 }
 
@@ -2162,20 +2164,32 @@ extern "C" hap_status hap_search_range(hap_problem *p, uint64_t first, uint64_t 
         CUDA_TRY(p, cudaGetLastError());
         out.cand_lb = p->d_cand_lb;
     }
+    // When every class of the search walks its prefix tree, each block also leaves the plan of its best candidate
+    // (partition, levels, the terms of Eq. 4) and the final reduction copies the winner's: nothing is evaluated twice.
+    bool plans = count > 1;
+    for (const auto &cl : p->classes) plans = plans && pass_uses_trie(p, cl, out, false);
+    SingleOut *d1 = (SingleOut *)p->d_single;
+    if (plans) {
+        if (!p->d_plans) CUDA_TRY(p, cached_malloc(p->device, (void **)&p->d_plans, p->n_pslots * sizeof(PlanSlot)));
+        out.block_plan = p->d_plans;
+    }
     if ((s = launch_decode_early(p, out, true)) != HAP_OK) return s;
     if ((s = launch_dp(p, out, true, st)) != HAP_OK) return s;
-    argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->n_pslots, p->d_best, kInf);
+    static_assert(offsetof(SingleOut, bott) == 8 && offsetof(SingleOut, detail) == 16, "the final reduction writes cost, bottleneck and the three terms in a row");
+    if (plans) argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->n_pslots, p->d_best, kInf, p->d_plans, &d1->cost, d1->part, d1->rec);
+    else argmin_final_kernel<<<1, 256, 0, st>>>(p->d_pcost, p->d_pindex, p->n_pslots, p->d_best, kInf);
     CUDA_TRY(p, cudaGetLastError());
     CUDA_TRY(p, cudaEventRecord(p->ev[2], st));
     p->timed = true;
-    // the winner is evaluated once more alone, for its partition and recomputation levels; its index stays on the
-    // device (every class's kernel looks whether the index is its own), so the host waits only once
-    SingleOut *d1 = (SingleOut *)p->d_single;
-    DpOut one{};
-    one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
-    one.recompute = d1->rec; one.first = 0; one.count = 1; one.first_dev = p->d_best + 1;
-    if (fused && (s = launch_layer_kernel(p, p->d_c2, nullptr, true, st, nullptr, p->d_best + 1, 0, 1, false)) != HAP_OK) return s;
-    if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
+    if (!plans) {
+        // the winner is evaluated once more alone, for its partition and recomputation levels; its index stays on the
+        // device (every class's kernel looks whether the index is its own), so the host waits only once
+        DpOut one{};
+        one.cost = &d1->cost; one.bottleneck = &d1->bott; one.detail = d1->detail; one.partition = d1->part;
+        one.recompute = d1->rec; one.first = 0; one.count = 1; one.first_dev = p->d_best + 1;
+        if (fused && (s = launch_layer_kernel(p, p->d_c2, nullptr, true, st, nullptr, p->d_best + 1, 0, 1, false)) != HAP_OK) return s;
+        if ((s = launch_dp(p, one, false, st)) != HAP_OK) return s;
+    }
     decode_kernel<<<1, 32, 0, st>>>(p->dc, 0, 1, &d1->cand, p->d_best + 1);
     CUDA_TRY(p, cudaGetLastError());
     // range flag, counters, minimum and the re-evaluated winner sit in consecutive 256-byte slots at the end of the

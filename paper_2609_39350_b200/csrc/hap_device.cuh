@@ -89,6 +89,14 @@ struct WorkItem {
     u64 lo;
 };
 
+// What a block of a search leaves beside its (cost, index) minimum when it can: the plan of that candidate.
+struct __align__(16) PlanSlot {
+    i64 bott, T_pipe, T_sync, T_opt;
+    uint8_t n[HAP_MAX_PP], r[HAP_MAX_PP];     // layers and recomputation level of stages 1..PP (the rest is not written)
+    int PP, pad[3];
+};
+static_assert(HAP_MAX_PP == 32 && sizeof(PlanSlot) % 16 == 0, "the plan bytes move as 16-byte pieces");
+
 struct DpOut {
     i64 *cost, *bottleneck;
     uint8_t *partition, *recompute;
@@ -114,6 +122,7 @@ struct DpOut {
     // indexed by the global candidate index (HAP_INF: the candidate has no feasible partition); a candidate whose
     // bound exceeds the incumbent is skipped
     const i64 *cand_lb;
+    PlanSlot *block_plan;             // search over the prefix trees: per block the plan of its best candidate (nullable)
     int force_plain;                  // run the plain min-max pass although the problem asks for a refinement mode
 };
 
@@ -1909,7 +1918,8 @@ argmin_partial_kernel(const i64 *cost, u64 count, i64 *pcost, u64 *pindex, i64 i
 }
 
 __global__ void __launch_bounds__(256)
-argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2, i64 init)
+argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2, i64 init, const PlanSlot *plans = nullptr,
+                    i64 *w_vals = nullptr, uint8_t *w_part = nullptr, uint8_t *w_rec = nullptr)
 {
     // launched as a programmatic dependent of the first stage where it follows one directly: the partials are
     // complete and visible after this wait (a no-op in an ordinary launch)
@@ -1927,7 +1937,21 @@ argmin_final_kernel(const i64 *pcost, const u64 *pindex, u64 n, i64 *out2, i64 i
     if (threadIdx.x == 0) {
         for (int q = 1; q < 8; ++q) if (sc[q] < bc || (sc[q] == bc && si[q] < bi)) { bc = sc[q]; bi = si[q]; }
         out2[0] = bc; out2[1] = (i64)bi;
+        sc[0] = bc; si[0] = bi;
+        if (plans) w_vals[0] = init;             // (a winner whose plan is not found below shows as a cost that differs)
     }
+    if (!plans) return;
+    // the block that reported the minimum also left the candidate's plan: copy it beside the minimum
+    // (w_vals: cost, bottleneck, T_pipe, T_sync, T_opt)
+    __syncthreads();
+    bc = sc[0]; bi = si[0];
+    if (!(bc < init)) return;
+    for (u64 i = threadIdx.x; i < n; i += blockDim.x)
+        if (pindex[i] == bi && pcost[i] == bc) {
+            const PlanSlot ps = plans[i];
+            w_vals[0] = bc; w_vals[1] = ps.bott; w_vals[2] = ps.T_pipe; w_vals[3] = ps.T_sync; w_vals[4] = ps.T_opt;
+            for (int q = 0; q < HAP_MAX_PP; ++q) { w_part[q] = q < ps.PP ? ps.n[q] : 0; w_rec[q] = q < ps.PP ? ps.r[q] : 0; }
+        }
 }
 
 }  // namespace hap

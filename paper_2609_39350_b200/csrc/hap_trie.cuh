@@ -526,6 +526,11 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     u32 best_local = ~0u;               // the best candidate's offset from the block's first candidate
     u32 n_eval = 0, n_feas = 0;         // (a thread evaluates far fewer than 2^32 candidates)
     u32 n_cells32 = 0;                  // splits this thread evaluated (after the early exits)
+    // A search that records plans: the partition and levels of the candidate at hand go to one of two places in local
+    // memory (stores that nothing waits for), the other one holds those of the thread's best candidate so far.
+    __align__(16) uint8_t plan_n[2][HAP_MAX_PP], plan_r[2][HAP_MAX_PP];    // per stage: layers, level
+    i64 plan_val[2][4];                 // bottleneck, T_pipe, T_sync, T_opt
+    u32 plan_cur = 0;
     unsigned all_levels = 0;
     for (int q = 0; q < n_rc; ++q) all_levels |= dc.rc_masks[q];
 
@@ -779,7 +784,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
                 if (!SEARCH) {
                     if (out.partition) out.partition[o * HAP_MAX_PP + d - 1] = (uint8_t)(b - a);
                     if (out.recompute) out.recompute[o * HAP_MAX_PP + d - 1] = (uint8_t)r;
-                }
+                } else if (out.block_plan) { plan_n[plan_cur][d - 1] = (uint8_t)(b - a); plan_r[plan_cur][d - 1] = (uint8_t)r; }
                 if (d > 1) {
                     b = a;
                     if (!HAP_CHECK_OK(2, b >= (int)(raw.w & 255) && raw.x + (u32)(b - (int)(raw.w & 255)) < tm.cell_lo[d] - tm.cell_lo[d - 1])) break;
@@ -799,7 +804,14 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
                 if (T_iter < vInf) { n_feas++; any_plan = 1; }
                 {   // (offsets grow with the candidate index, so the smaller offset is the smaller index)
                     const u32 loc = m * (u32)n_rc + (u32)rc_idx;
-                    if ((i64)T_iter < best_cost || ((i64)T_iter == best_cost && loc < best_local)) { best_cost = (i64)T_iter; best_local = loc; }
+                    if ((i64)T_iter < best_cost || ((i64)T_iter == best_cost && loc < best_local)) {
+                        best_cost = (i64)T_iter; best_local = loc;
+                        if (out.block_plan) {
+                            plan_val[plan_cur][0] = (i64)bott; plan_val[plan_cur][1] = (i64)T_pipe;
+                            plan_val[plan_cur][2] = (i64)t_sync; plan_val[plan_cur][3] = (i64)t_opt;
+                            plan_cur ^= 1u;                  // the place just filled is kept, the other one is written next
+                        }
+                    }
                 }
             } else {
                 any_plan = 1;
@@ -841,6 +853,21 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
             out.partial_cost[blockIdx.x] = bc;
             out.partial_index[blockIdx.x] = bi;
             if (out.prune && bc < kInf) atomicMin(out.incumbent, (u64)bc);
+            wcost[0] = bc; widx[0] = bi;
+        }
+        if (out.block_plan) {
+            // the thread that evaluated the block's best candidate writes its plan to the block's slot
+            __syncthreads();
+            if (wcost[0] < kInf && best_local != ~0u && s_clo + (u64)best_local == widx[0]) {
+                PlanSlot *ps = out.block_plan + blockIdx.x;
+                const u32 keep = plan_cur ^ 1u;
+                ps->bott = plan_val[keep][0]; ps->T_pipe = plan_val[keep][1]; ps->T_sync = plan_val[keep][2]; ps->T_opt = plan_val[keep][3];
+                ps->PP = PP;                                  // (entries of later stages are whatever the thread's memory held)
+                const uint4 *sn = reinterpret_cast<const uint4 *>(plan_n[keep]), *sr = reinterpret_cast<const uint4 *>(plan_r[keep]);
+                uint4 *dn = reinterpret_cast<uint4 *>(ps->n), *dr = reinterpret_cast<uint4 *>(ps->r);
+                dn[0] = sn[0]; dr[0] = sr[0];
+                if (PP > 16) { dn[1] = sn[1]; dr[1] = sr[1]; }
+            }
         }
     }
 }
