@@ -582,7 +582,6 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
             return;
         }
     }
-    const bool config_dead = false;
 
     // ---- layer times of the configuration; in a pruning search whose blocks compute them, the lower bound too ----
     trie_stage_costs<VT>(dc, pc, p, c2, out.tcg, out.range_flag, sC);
@@ -612,10 +611,8 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
         if (s_skip) return;
     }
     trie_prologue_rows<VT>(dc, tm, p, coef, coefv, sW, sA, sK, sKtab, sNodes, sParent, minfo, sP2P, szero);
-    if (!config_dead) {
-        trie_prologue_time_rows<VT>(dc, tm, sC, sR);
-        trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
-    }
+    trie_prologue_time_rows<VT>(dc, tm, sC, sR);
+    trie_prologue_thr(dc, pc, tm, p, coef, all_levels, sW, sA, thr, sK);
 
     const u32 a_thr = smem_u32(thr), a_sR = smem_u32(sR);
     const bool all_flat = tm.all_flat != 0;
@@ -674,7 +671,7 @@ trie_dp_kernel(const DevConst dc, const u32 *plist, unsigned n_active, const VT 
     for (int rc_pos = 0; rc_pos < n_rc; ++rc_pos) {
         const int rc_idx = dc.rc_order[rc_pos];
         const unsigned rc_mask = dc.rc_masks[rc_idx];
-        bool dead = config_dead || (dc.rc_sup[rc_pos] & policies_without_plan) != 0;
+        bool dead = (dc.rc_sup[rc_pos] & policies_without_plan) != 0;
 
         // ---- rows of the tree, depth by depth ------------------------------------------------
         if (!dead) {
