@@ -2,6 +2,7 @@
 from __future__ import annotations
 
 import ctypes as C
+import weakref
 import os
 from typing import Optional
 
@@ -154,15 +155,44 @@ OPT_NO_FUSE = 32
 OPT_COUNT_SPLITS = 64
 
 
+_ADDRESSES = {}          # id(problem) -> (weak reference to it, {field: (array as given, array as passed, address)})
+
+
+def _address_memo(pb) -> dict:
+    key = id(pb)
+    hit = _ADDRESSES.get(key)
+    if hit is not None and hit[0]() is pb:
+        return hit[1]
+    try:
+        ref = weakref.ref(pb, lambda _r, key=key: _ADDRESSES.pop(key, None))
+    except TypeError:                       # an object that cannot be referenced weakly: nothing is remembered
+        return {}
+    _ADDRESSES[key] = (ref, {})
+    return _ADDRESSES[key][1]
+
+
 def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     """Marshals a plain-data problem (see gen.problems.Problem) into the C descriptors."""
     L = load_library()
     keep = []
 
+    # addresses of the problem's arrays, remembered per problem object and field for as long as the field holds the
+    # same array object (looking an address up costs more than everything else here); kept beside the object, not in
+    # it, so that copies of the problem start empty
+    memo = _address_memo(pb)
+
     def arr(name, dtype):
-        a = np.ascontiguousarray(np.asarray(getattr(pb, name), dtype=dtype))
-        keep.append(a)
-        return _ptr(a)
+        a = getattr(pb, name)
+        hit = memo.get(name)
+        if hit is not None and hit[0] is a:
+            keep.append(hit[1])
+            return hit[2]
+        c = a
+        if not (type(c) is np.ndarray and c.dtype == dtype and c.flags.c_contiguous):     # (no copy in the usual case)
+            c = np.ascontiguousarray(np.asarray(c, dtype=dtype))
+        keep.append(c)
+        memo[name] = (a, c, c.ctypes.data)
+        return memo[name][2]
 
     mo = _Model()
     for n in ("N", "S", "H", "E", "k", "n_shared", "F_dense", "F_exp", "nq", "nkv", "V", "GB"):

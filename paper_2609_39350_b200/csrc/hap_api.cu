@@ -20,6 +20,18 @@
 
 using namespace hap;
 
+// read-only view of a vector that someone else keeps alive
+template <typename E> struct View {
+    const E *ptr = nullptr;
+    size_t n = 0;
+    size_t size() const { return n; }
+    bool empty() const { return n == 0; }
+    const E *data() const { return ptr; }
+    const E &operator[](size_t i) const { return ptr[i]; }
+    const E *begin() const { return ptr; }
+    const E *end() const { return ptr + n; }
+};
+
 struct hap_problem {
     int device = 0;
     // host copies
@@ -34,11 +46,13 @@ struct hap_problem {
     hap_search_opts opts{};
     int64_t m[HAP_MAX_TYPES] = {0, 0, 0, 0};
     int64_t W = 0;
-    // enumeration
+    // enumeration: the configuration table and the work items belong to the per-process enumeration result that
+    // `enum_ref` keeps alive (problems with the same lists share one)
     bool enumerated = false;
-    std::vector<hap_pconf> pconfs;
+    View<hap_pconf> pconfs;
     uint64_t n_cand = 0;
-    std::vector<WorkItem> items;           // grouped by PP class, heaviest class first
+    View<WorkItem> items;                  // grouped by PP class, heaviest class first
+    std::shared_ptr<const void> enum_ref;
     // prefix tree of a class's mappings (trie_dp_kernel); ok = false: the class runs in pipeline_dp_kernel only
     struct TriePartDev { TrieNode *d_nodes; TrieLeaf *d_leaves; TrieCell *d_cells; u32 *d_first_leaf, *d_gnode; uint8_t *d_depth;
                          u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
@@ -1184,8 +1198,9 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             enum_cache_insert(ekey, fresh);
             er = fresh;
         }
-        p->pconfs = er->rows;
-        p->items = er->items;
+        p->enum_ref = er;
+        p->pconfs.ptr = er->rows.data(); p->pconfs.n = er->rows.size();
+        p->items.ptr = er->items.data(); p->items.n = er->items.size();
         p->classes = er->classes;
         const uint64_t off = er->n_cand;
         const u64 tab_bytes = er->tab_bytes;
