@@ -17,6 +17,9 @@
 #include <string>
 #include <unordered_map>
 #include <vector>
+#if defined(__SSE2__)
+#include <emmintrin.h>
+#endif
 
 using namespace hap;
 
@@ -461,13 +464,32 @@ extern "C" hap_status hap_problem_create(const hap_model *mo, const hap_cluster 
     // the layer-cost kernel reads a record with two 16-byte loads), then tpre, then tpost
     const size_t n_tab = 4 * n5 + 2 * n4;
     auto fill_tables = [&](unsigned char *dst) -> bool {
-        double *tables = reinterpret_cast<double *>(dst);
+        double *__restrict__ tables = reinterpret_cast<double *>(dst);
+        const double *__restrict__ A = pf->tdf, *__restrict__ B = pf->tdb, *__restrict__ F = pf->tff, *__restrict__ G = pf->tfb;
         bool ok = true;
-        for (size_t i = 0; i < n5; ++i) {
-            const double a = pf->tdf[i], b = pf->tdb[i], c = pf->tff[i], d = pf->tfb[i];
+        size_t i = 0;
+        // t_dense includes its FFN; every entry finite, non-negative, < 2^50 ns (NaN fails every comparison)
+#if defined(__SSE2__)
+        {   // two entries per step: the records are the 2 x 2 transposes of the four streams
+            const __m128d zero = _mm_setzero_pd(), big = _mm_set1_pd(1e15);
+            __m128d okv = _mm_castsi128_pd(_mm_set1_epi32(-1));
+            for (; i + 2 <= n5; i += 2) {
+                const __m128d a = _mm_loadu_pd(A + i), b = _mm_loadu_pd(B + i), c = _mm_loadu_pd(F + i), d = _mm_loadu_pd(G + i);
+                double *rec = tables + 4 * i;
+                _mm_storeu_pd(rec, _mm_unpacklo_pd(a, b)); _mm_storeu_pd(rec + 2, _mm_unpacklo_pd(c, d));
+                _mm_storeu_pd(rec + 4, _mm_unpackhi_pd(a, b)); _mm_storeu_pd(rec + 6, _mm_unpackhi_pd(c, d));
+                __m128d v = _mm_and_pd(_mm_cmpge_pd(a, c), _mm_cmpge_pd(b, d));
+                v = _mm_and_pd(v, _mm_and_pd(_mm_cmpge_pd(c, zero), _mm_cmpge_pd(d, zero)));
+                v = _mm_and_pd(v, _mm_and_pd(_mm_cmple_pd(a, big), _mm_cmple_pd(b, big)));
+                okv = _mm_and_pd(okv, v);
+            }
+            ok = _mm_movemask_pd(okv) == 3;
+        }
+#endif
+        for (; i < n5; ++i) {
+            const double a = A[i], b = B[i], c = F[i], d = G[i];
             double *rec = tables + 4 * i;
             rec[0] = a; rec[1] = b; rec[2] = c; rec[3] = d;
-            // t_dense includes its FFN; every entry finite, non-negative, < 2^50 ns (NaN fails every comparison)
             ok &= (a >= c) & (b >= d) & (c >= 0.0) & (d >= 0.0) & (a <= 1e15) & (b <= 1e15);
         }
         for (size_t i = 0; i < n4; ++i) {
