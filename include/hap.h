@@ -235,8 +235,10 @@ hap_status hap_release_cached_memory(void);
  * lexicographic order, counts the stage mappings of each and builds the device-side tables.
  * What depends on the model's dimensions, the cluster and the search options only -- the configuration table, the
  * work items and the prefix trees of the classes' stage mappings -- is kept per process (host memory, at most a few
- * hundred entries, keyed by exactly those inputs) and copied when a later problem has the same key: planning again on
- * the same cluster with new profiled tables skips the loop nest and the tree build. */
+ * hundred entries, keyed by exactly those inputs) and reused when a later problem has the same key: planning again on
+ * the same cluster with new profiled tables skips the loop nest and the tree build.  The device copies are still the
+ * problem's own; the table and the address-free part of the trees are uploaded straight from page-locked images of
+ * them (one per key, the tree images at most 16 per process). */
 hap_status hap_enumerate(hap_problem *, uint64_t *n_pconf, uint64_t *n_candidates);
 hap_status hap_get_pconfs(const hap_problem *, hap_pconf *host_out, uint64_t cap);
 

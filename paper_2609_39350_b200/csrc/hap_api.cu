@@ -56,6 +56,7 @@ struct hap_problem {
     uint64_t n_cand = 0;
     View<WorkItem> items;                  // grouped by PP class, heaviest class first
     std::shared_ptr<const void> enum_ref;
+    std::shared_ptr<const void> tree_image;      // the page-locked image the trees were uploaded from (kept until the copy is known to be done)
     // prefix tree of a class's mappings (trie_dp_kernel); ok = false: the class runs in pipeline_dp_kernel only
     struct TriePartDev { TrieNode *d_nodes; TrieLeaf *d_leaves; TrieCell *d_cells; u32 *d_first_leaf, *d_gnode; uint8_t *d_depth;
                          u32 n_nodes, n_cells, nmap, m_lo; uint8_t mrow_of[16]; };
@@ -208,6 +209,39 @@ static cudaError_t upload(hap_problem *p, void *dst, size_t bytes, Fill fill)
     cudaError_t e = cudaMemcpyAsync(dst, pb->ptr, bytes, cudaMemcpyHostToDevice, us);
     if (e != cudaSuccess) return e;
     if ((e = cudaEventRecord(pb->done, us)) != cudaSuccess) return e;
+    if (!p->ev_upload && (e = cudaEventCreateWithFlags(&p->ev_upload, cudaEventDisableTiming)) != cudaSuccess) return e;
+    if ((e = cudaEventRecord(p->ev_upload, us)) != cudaSuccess) return e;
+    p->upload_pending = true;
+    return cudaSuccess;
+}
+
+// A host image in page-locked memory that uploads read directly, without the pass through a staging buffer: what is
+// derived from the lists and the cluster alone (configuration table, prefix trees) is laid out once per process.
+struct PinnedImage {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+    PinnedImage() = default;
+    PinnedImage(const PinnedImage &) = delete;
+    PinnedImage &operator=(const PinnedImage &) = delete;
+    ~PinnedImage() { if (ptr) { cudaFreeHost(ptr); cudaGetLastError(); } }
+};
+
+static std::shared_ptr<PinnedImage> pinned_image(size_t bytes)
+{
+    auto im = std::make_shared<PinnedImage>();
+    if (cudaHostAlloc(&im->ptr, std::max<size_t>(bytes, 1), cudaHostAllocPortable) != cudaSuccess) { cudaGetLastError(); im->ptr = nullptr; return nullptr; }
+    im->bytes = bytes;
+    return im;
+}
+
+// host -> device copy straight from such an image (the problem holds a reference to it until it is destroyed, which
+// waits for the copy)
+static cudaError_t upload_image(hap_problem *p, void *dst, const PinnedImage &im, size_t bytes)
+{
+    cudaStream_t us = upload_stream(p->device);
+    if (!us) return cudaMemcpy(dst, im.ptr, bytes, cudaMemcpyHostToDevice);
+    cudaError_t e = cudaMemcpyAsync(dst, im.ptr, bytes, cudaMemcpyHostToDevice, us);
+    if (e != cudaSuccess) return e;
     if (!p->ev_upload && (e = cudaEventCreateWithFlags(&p->ev_upload, cudaEventDisableTiming)) != cudaSuccess) return e;
     if ((e = cudaEventRecord(p->ev_upload, us)) != cudaSuccess) return e;
     p->upload_pending = true;
@@ -913,27 +947,49 @@ static bool build_trie(hap_problem *p, hap_problem::PpClass &cl, const uint8_t *
     return true;
 }
 
-// One allocation and one copy for the trees of all classes: per class its parts' blobs, the part descriptions
-// and the list of the class's configurations.
-static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
+// One allocation for the trees of all classes.  Its head holds what does not depend on where it lies -- per class the
+// parts' blobs and the list of the class's configurations -- and is copied from an image kept per process under
+// `image_key` (the classes' tree keys and the enumeration's key); behind it lie the part descriptions and the job
+// list of the gather kernel, which hold device addresses and are staged for every problem.
+namespace {
+std::mutex g_tree_image_mu;
+std::map<std::string, std::shared_ptr<PinnedImage>> g_tree_images;
+constexpr size_t kTreeImages = 16;
+}
+
+static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built, const std::string &image_key)
 {
     constexpr size_t kTwoPerSm = 108 * 1024;
     auto up = [](size_t v) { return (v + 255) / 256 * 256; };
-    size_t total = 0, n_parts_all = 0;
+    size_t head = 0, tail = 0, n_parts_all = 0;
     for (auto &bc : built) {
-        for (const auto &pt : bc.tree->parts) total += up(pt.blob.size());
-        total += up(bc.tree->parts.size() * sizeof(TrieMeta)) + up(bc.plist.size() * sizeof(u32));
+        for (const auto &pt : bc.tree->parts) head += up(pt.blob.size());
+        head += up(bc.plist.size() * sizeof(u32));
+        tail += up(bc.tree->parts.size() * sizeof(TrieMeta));
         n_parts_all += bc.tree->parts.size();
     }
-    if (!total) return true;
-    const size_t o_jobs = total;
-    total += up(n_parts_all * sizeof(GatherJob));
+    if (!head) return true;
+    const size_t o_jobs = head + tail;
+    const size_t total = o_jobs + up(n_parts_all * sizeof(GatherJob));
     std::vector<GatherJob> gjobs;
     DecodeJobs dj{};
     unsigned dblk = 0, gblk = 0;
     if (cached_malloc(p->device, (void **)&p->d_trie_arena, total) != cudaSuccess) { p->d_trie_arena = nullptr; cudaGetLastError(); return false; }
-    auto fill = [&](unsigned char *stage) -> bool {          // (gaps between the pieces are padding that nothing reads)
-    size_t off = 0;
+    // the head: blobs and configuration lists (`stage` may be null: only the offsets are wanted then)
+    auto fill_head = [&](unsigned char *stage) {
+        size_t off = 0;
+        for (auto &bc : built) {
+            for (const auto &pt : bc.tree->parts) {
+                if (stage) std::memcpy(stage + off, pt.blob.data(), pt.blob.size());
+                off += up(pt.blob.size());
+            }
+            if (stage) std::memcpy(stage + off, bc.plist.data(), bc.plist.size() * sizeof(u32));
+            off += up(bc.plist.size() * sizeof(u32));
+        }
+    };
+    // the tail: part descriptions and gather jobs, with this arena's addresses; also fills the per-class records
+    auto fill_tail = [&](unsigned char *stage) -> bool {          // (stage = start of the tail)
+    size_t off = 0, toff = 0;
     for (auto &bc : built) {
         hap_problem::Trie &tr = bc.cl->trie;
         const TrieClassHost &h = *bc.tree;
@@ -942,7 +998,6 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
         u32 want = 0;
         for (const auto &pt : h.parts) {
             unsigned char *base = p->d_trie_arena + off;
-            std::memcpy(stage + off, pt.blob.data(), pt.blob.size());
             hap_problem::TriePartDev pd{};
             pd.d_nodes = reinterpret_cast<TrieNode *>(base + pt.o_nodes);
             pd.d_leaves = reinterpret_cast<TrieLeaf *>(base + pt.o_leaves);
@@ -969,12 +1024,11 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
             want = std::max(want, std::max(pt.max_level, pt.nmap));
             off += up(pt.blob.size());
         }
-        tr.d_metas = reinterpret_cast<TrieMeta *>(p->d_trie_arena + off);
-        std::memcpy(stage + off, metas.data(), metas.size() * sizeof(TrieMeta));
-        off += up(metas.size() * sizeof(TrieMeta));
         tr.d_plist = reinterpret_cast<u32 *>(p->d_trie_arena + off);
-        std::memcpy(stage + off, bc.plist.data(), bc.plist.size() * sizeof(u32));
         off += up(bc.plist.size() * sizeof(u32));
+        tr.d_metas = reinterpret_cast<TrieMeta *>(p->d_trie_arena + head + toff);
+        std::memcpy(stage + toff, metas.data(), metas.size() * sizeof(TrieMeta));
+        toff += up(metas.size() * sizeof(TrieMeta));
         tr.n_conf = (unsigned)bc.plist.size(); tr.smem = smem;
         if (dj.n <= HAP_MAX_PP) {
             const hap_problem::PpClass &cl = *bc.cl;
@@ -990,14 +1044,31 @@ static bool upload_tries(hap_problem *p, std::vector<TrieBuilt> &built)
         tr.threads = std::min(smem <= kTwoPerSm ? 512 : 1024, std::max(128, th));
         tr.ok = true;
     }
-    std::memcpy(stage + o_jobs, gjobs.data(), gjobs.size() * sizeof(GatherJob));
+    std::memcpy(stage + tail, gjobs.data(), gjobs.size() * sizeof(GatherJob));
     return true;
     };
-    if (upload(p, p->d_trie_arena, total, fill) != cudaSuccess) {
+    // head: from the process's image of these trees when there is one (made on first use)
+    std::shared_ptr<PinnedImage> image;
+    if (upload_stream(p->device)) {
+        std::lock_guard<std::mutex> lock(g_tree_image_mu);
+        auto it = g_tree_images.find(image_key);
+        if (it != g_tree_images.end() && it->second->bytes == head) image = it->second;
+        else if ((image = pinned_image(head))) {
+            std::memset(image->ptr, 0, head);
+            fill_head(static_cast<unsigned char *>(image->ptr));
+            if (g_tree_images.size() >= kTreeImages) g_tree_images.clear();
+            g_tree_images[image_key] = image;
+        }
+    }
+    cudaError_t e = image ? upload_image(p, p->d_trie_arena, *image, head)
+                          : upload(p, p->d_trie_arena, head, [&](unsigned char *stage) { fill_head(stage); return true; });
+    if (e == cudaSuccess) e = upload(p, p->d_trie_arena + head, total - head, fill_tail);
+    if (e != cudaSuccess) {
         cudaGetLastError();
         for (auto &bc : built) bc.cl->trie = hap_problem::Trie{};
         return false;
     }
+    p->tree_image = image;
     p->decode_jobs = dj;
     p->d_gather_jobs = reinterpret_cast<GatherJob *>(p->d_trie_arena + o_jobs);
     p->n_gather_jobs = (int)gjobs.size();
@@ -1057,6 +1128,7 @@ struct EnumResult {
     std::vector<hap_problem::PpClass> classes;       // streams, events and trees are per problem: empty here
     uint64_t n_cand = 0;
     u64 tab_bytes = 0;
+    std::shared_ptr<PinnedImage> image;             // rows | padding to 256 bytes | items | padding: the head of a problem's arena (may be null)
 };
 namespace {
 std::mutex g_enum_cache_mu;
@@ -1214,6 +1286,17 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
 
             fresh->rows.swap(rows); fresh->items.swap(items); fresh->classes.swap(classes);
             fresh->n_cand = off; fresh->tab_bytes = tab_bytes;
+            {   // the table and the items as every problem with these lists uploads them
+                auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+                const size_t o_items = up(fresh->rows.size() * sizeof(hap_pconf)), total = up(o_items + fresh->items.size() * sizeof(WorkItem));
+                fresh->image = pinned_image(total);
+                if (fresh->image) {
+                    unsigned char *im = static_cast<unsigned char *>(fresh->image->ptr);
+                    std::memset(im, 0, total);
+                    std::memcpy(im, fresh->rows.data(), fresh->rows.size() * sizeof(hap_pconf));
+                    std::memcpy(im + o_items, fresh->items.data(), fresh->items.size() * sizeof(WorkItem));
+                }
+            }
             return HAP_OK;
             }();
             if (es != HAP_OK) return es;
@@ -1264,7 +1347,8 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             p->d_range = reinterpret_cast<u64 *>(base + o_range); p->d_counters = reinterpret_cast<u64 *>(base + o_counters);
             p->d_best = reinterpret_cast<i64 *>(base + o_best); p->d_single = base + o_single;
             // configuration table and work items travel in one copy (they are adjacent up to padding)
-            CUDA_TRY(p, upload(p, base, o_c2, [&](unsigned char *stage) {
+            if (er->image && er->image->bytes == o_c2) CUDA_TRY(p, upload_image(p, base, *er->image, o_c2));
+            else CUDA_TRY(p, upload(p, base, o_c2, [&](unsigned char *stage) {
                 std::memcpy(stage + o_pconf, p->pconfs.data(), np * sizeof(hap_pconf));
                 std::memcpy(stage + o_items, p->items.data(), p->items.size() * sizeof(WorkItem));
                 return true; }));
@@ -1339,7 +1423,9 @@ extern "C" hap_status hap_enumerate(hap_problem *p, uint64_t *n_pconf, uint64_t 
             }
             // the launch order of the merged decode / gather jobs follows the class order
             std::sort(built.begin(), built.end(), [](const TrieBuilt &x, const TrieBuilt &y) { return x.cl < y.cl; });
-            upload_tries(p, built);
+            std::string image_key = ekey;
+            for (const auto &bc : built) image_key += keys[bc.cl - p->classes.data()];
+            upload_tries(p, built, image_key);
         }
         p->n_pslots = 0;
         for (auto &cl : p->classes) {
