@@ -171,6 +171,8 @@ def test_sub_ranges_ragged_edges_and_errors(hap):
     assert np.array_equal(out["cost"].cpu().numpy(), costs)
     plan, stats = hap.hap_search_range(hp, 1000, 3001)
     assert plan["index"] == best["index"] and plan["T_iter"] == best["T_iter"] and stats["n_evaluated"] == 3001
+    for key in ("n", "r", "mask", "bottleneck", "T_pipe", "T_sync", "T_opt"):
+        assert plan[key] == best[key], key
     # single candidate, last candidate, empty range
     one = hap.hap_pipeline_dp(hp, o.n_cand - 1, 1)
     torch.cuda.synchronize()

@@ -93,6 +93,9 @@ def test_ragged_ranges_across_configurations(hap):
         plan, stats = hap.hap_search_range(hp, first, count)
         assert plan["T_iter"] == int(sub.min()) and plan["index"] == first + int(np.argmin(sub))
         assert stats["n_evaluated"] == count
+        want = o.eval_index(plan["index"])[0]          # the plan the winning block left, term by term
+        for key in ("n", "r", "mask", "bottleneck", "T_pipe", "T_sync", "T_opt"):
+            assert plan[key] == want[key], (first, count, key)
     hap.hap_problem_destroy(hp)
 
 
