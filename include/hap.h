@@ -289,7 +289,10 @@ hap_status hap_search_range_f64(hap_problem *, uint64_t first, uint64_t count, h
  * S + (M-1) B* (B* its bottleneck, S the configuration's sum over layers of the cheapest type's time) and the
  * refinement runs only for candidates whose bound does not exceed the incumbent; host_stats->n_pruned counts the
  * candidates cut this way, candidates without a feasible partition count as evaluated.  The first such call
- * allocates 8 bytes per candidate of scratch. */
+ * allocates 8 bytes per candidate of scratch.
+ * The plan (partition, levels, terms of Eq. 4) comes from the search itself when every class walks its prefix tree:
+ * each block leaves the plan of its best candidate and the winner's is copied out (the first search of a problem
+ * allocates 112 bytes per block for them); otherwise the winner is evaluated once more alone. */
 hap_status hap_search_range(hap_problem *, uint64_t first, uint64_t count, hap_plan *host_out,
                             hap_search_stats *host_stats, void *stream);
 /* The whole candidate space. */
