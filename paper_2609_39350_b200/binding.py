@@ -171,6 +171,22 @@ def _address_memo(pb) -> dict:
     return _ADDRESSES[key][1]
 
 
+def _field_address(memo: dict, pb, name: str, dtype, keep: list) -> int:
+    """Address of field `name` of the problem as a C-contiguous array of `dtype` (converted if it is not one); the
+    array that owns the memory is appended to `keep`."""
+    a = getattr(pb, name)
+    hit = memo.get(name)
+    if hit is not None and hit[0] is a:
+        keep.append(hit[1])
+        return hit[2]
+    c = a
+    if not (type(c) is np.ndarray and c.dtype == dtype and c.flags.c_contiguous):     # (no copy in the usual case)
+        c = np.ascontiguousarray(np.asarray(c, dtype=dtype))
+    keep.append(c)
+    memo[name] = (a, c, c.ctypes.data)
+    return memo[name][2]
+
+
 def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     """Marshals a plain-data problem (see gen.problems.Problem) into the C descriptors."""
     L = load_library()
@@ -182,17 +198,7 @@ def hap_problem_create(pb, prune: int = 0, flags: int = 0) -> HapProblem:
     memo = _address_memo(pb)
 
     def arr(name, dtype):
-        a = getattr(pb, name)
-        hit = memo.get(name)
-        if hit is not None and hit[0] is a:
-            keep.append(hit[1])
-            return hit[2]
-        c = a
-        if not (type(c) is np.ndarray and c.dtype == dtype and c.flags.c_contiguous):     # (no copy in the usual case)
-            c = np.ascontiguousarray(np.asarray(c, dtype=dtype))
-        keep.append(c)
-        memo[name] = (a, c, c.ctypes.data)
-        return memo[name][2]
+        return _field_address(memo, pb, name, dtype, keep)
 
     mo = _Model()
     for n in ("N", "S", "H", "E", "k", "n_shared", "F_dense", "F_exp", "nq", "nkv", "V", "GB"):

@@ -47,3 +47,34 @@ def test_layouts_match_the_header_sizes():
     from paper_2609_39350_b200 import binding as b
     assert b.PCONF_DTYPE.itemsize == 80 and b.CANDIDATE_DTYPE.itemsize == 96
     assert ctypes.sizeof(b._Plan) == 8 + 8 * 4 + 8 + 3 * 32 + 5 * 8
+
+
+def test_binding_remembers_array_addresses_per_problem_object_only():
+    """The binding keeps the address of a problem's arrays per object and field: a field that is reassigned, a copy of
+    the problem and an array that needs converting each get their own, current address."""
+    import copy
+    import gc
+    import numpy as np
+    from gen import problems
+    from paper_2609_39350_b200 import binding as b
+    pb = problems.tiny()
+    keep = []
+    memo = b._address_memo(pb)
+    assert b._address_memo(pb) is memo
+    a1 = b._field_address(memo, pb, "tdf", np.float64, keep)
+    assert a1 == pb.tdf.ctypes.data and b._field_address(memo, pb, "tdf", np.float64, keep) == a1 and keep[-1] is pb.tdf
+    pb.tdf = pb.tdf.copy()                                           # a new array in the same field
+    a2 = b._field_address(memo, pb, "tdf", np.float64, keep)
+    assert a2 == pb.tdf.ctypes.data and a2 != a1
+    pb.tp_list = [int(x) for x in pb.tp_list]                         # a list: converted, the converted array is kept alive
+    a3 = b._field_address(memo, pb, "tp_list", np.int32, keep)
+    assert a3 == keep[-1].ctypes.data and keep[-1].dtype == np.int32 and keep[-1].tolist() == pb.tp_list
+    assert b._field_address(memo, pb, "tp_list", np.int32, keep) == a3
+    other = copy.deepcopy(pb)                                         # copies start without addresses
+    m2 = b._address_memo(other)
+    assert m2 is not memo and not m2
+    assert b._field_address(m2, other, "tdf", np.float64, keep) == other.tdf.ctypes.data != a2
+    key = id(other)
+    del other, m2
+    gc.collect()
+    assert key not in b._ADDRESSES
