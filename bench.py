@@ -145,6 +145,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--timed-only", action="store_true",
                     help="run the warm-up and the timed steps and stop (for profiler captures): prints a reduced line")
+    ap.add_argument("--search-only", action="store_true",
+                    help="run warm-up + steps calls of hap_search_best (no pruning) on one GPU and stop (for profiler "
+                         "captures of the search form of the kernels): prints a reduced line")
     ap.add_argument("--delta-q", type=int, default=None, help="override the load-balance window (1/1024; <0 = off)")
     ap.add_argument("--backend", default="nccl", choices=["nccl", "gloo"],
                     help="torch.distributed backend of the (cost, index) exchange when launched with several ranks")
@@ -182,6 +185,21 @@ def main():
     pconfs = hap.hap_get_pconfs(hp)
     first, count = shard_ranges(pconfs, len(pb.rc_masks), pb.N, world)[rank]
     stream = torch.cuda.current_stream()
+
+    if args.search_only:
+        ms = []
+        for it in range(warmup + args.steps):
+            flush_s = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if it == 0 else flush_s
+            flush_s.fill_(1)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            plan, stats = hap.hap_search_best(hp)
+            ms.append(1e3 * (time.perf_counter() - t0))
+        print(json.dumps(dict(metric="search_ms", unit="ms", value=statistics.median(ms[warmup:]), n_gpus=1, steps=args.steps, warmup=warmup,
+                              config=dict(workload=args.workload), best=dict(cost=plan["T_iter"], index=plan["index"]),
+                              dp_phase_ms=stats["ms_dp"], note="hap_search_best only (--search-only)")))
+        hap.hap_problem_destroy(hp)
+        return
 
     out = {"cost": torch.empty(max(count, 1), dtype=torch.int64, device="cuda"),
            "bottleneck": torch.empty(max(count, 1), dtype=torch.int64, device="cuda")}
